@@ -1,0 +1,205 @@
+/*
+ * ago.h -- C ABI of the B200 fused-subgraph executor.
+ *
+ * A subgraph is an ordered list of operators with shapes (Section II: a
+ * computational graph whose nodes are operators and whose edges are tensors;
+ * Section III-A: "three operators: 2-d convolution, bias addition, and ReLU").
+ * Operator i consumes the output of operator i-1; operator 0 consumes
+ * subgraph input 0. Operators are either COMPLEX (they reduce: convolution,
+ * matrix multiplication) or SIMPLE (element-wise or row-wise: bias, ReLU, add,
+ * ...), the split of Section I.
+ *
+ * Three execution modes:
+ *   FUSED              one kernel for the whole subgraph; intermediates stay in
+ *                      shared memory / tensor memory (intensive operator
+ *                      fusion, Section III-B).
+ *   PER_MINI_SUBGRAPH  one kernel per complex operator with its trailing simple
+ *                      operators applied in the epilogue (conventional fusion,
+ *                      Section III-A, Fig. "Conventional fusion within a
+ *                      mini-subgraph"); intermediates round-trip device memory.
+ *   PER_OP             one kernel per operator (Section III-A, Fig. "Loop nest
+ *                      of a mini-subgraph without fusion").
+ *
+ * All pointers passed to ago_subgraph_run are DEVICE pointers owned by the
+ * caller; the arrays of pointers themselves are host arrays. The library
+ * allocates no device memory except one 4-byte status word per handle (at the
+ * first run). No call throws or aborts; failures are status codes plus a
+ * thread-local message (ago_last_error). There is no CPU fallback: without a
+ * CUDA device every run returns AGO_ERR_CUDA.
+ *
+ * Layouts (row-major, innermost last, 0-based):
+ *   activations        NHWC
+ *   CONV2D weight      OHWI  [O][R][S][I]; depthwise (groups == C): [R][S][C]
+ *   GEMM weight        [K][N]
+ *   attention Q,K,V,O  [B][S][heads*head_dim], head h at columns h*D..h*D+D-1
+ *   bias vectors       float32 [last dimension]
+ * bf16 tensors are raw 16-bit patterns. Every base pointer must be 16-byte
+ * aligned (AGO_ERR_ALIGNMENT otherwise).
+ */
+#ifndef AGO_H_
+#define AGO_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct ago_subgraph_s* ago_subgraph_t; /* opaque; owned by the library */
+
+typedef enum {
+  AGO_OK = 0,
+  AGO_ERR_INVALID_ARG = 1, /* NULL pointer, bad enum value, bad struct_size          */
+  AGO_ERR_UNSUPPORTED = 2, /* valid chain, but no kernel for it in the asked mode     */
+  AGO_ERR_SHAPE = 3,       /* operator shapes inconsistent                            */
+  AGO_ERR_ALIGNMENT = 4,   /* device pointer not 16-byte aligned                      */
+  AGO_ERR_WORKSPACE = 5,   /* workspace missing or too small                          */
+  AGO_ERR_CUDA = 6,        /* CUDA runtime / driver error (message has the string)    */
+  AGO_ERR_TIMEOUT = 7      /* a bounded device-side wait expired (see ago_subgraph_status) */
+} ago_status_t;
+
+typedef enum { AGO_BF16 = 0, AGO_FP32 = 1 } ago_dtype_t; /* FP32 I/O: depthwise-only subgraphs */
+
+typedef enum {
+  AGO_MODE_FUSED = 0,
+  AGO_MODE_PER_MINI_SUBGRAPH = 1,
+  AGO_MODE_PER_OP = 2
+} ago_mode_t;
+
+typedef enum {
+  /* complex operators (Section I: they contain a reduction) */
+  AGO_OP_CONV2D = 0,      /* p: O, R, S, stride, pad, groups (1, or C for depthwise with O == C) */
+  AGO_OP_GEMM = 1,        /* p: N            out[..., n] = sum_k in[..., k] * w[k][n]          */
+  AGO_OP_BATCHED_QKT = 2, /* p: input index of K, heads, head_dim   [B,S,E] -> [B,heads,S,S]   */
+  AGO_OP_BATCHED_PV = 3,  /* p: input index of V, heads, head_dim   [B,heads,S,S] -> [B,S,E]   */
+  /* simple operators */
+  AGO_OP_BIAS_ADD = 4,    /* + float32 vector over the last dimension (consumes one weight)   */
+  AGO_OP_RELU = 5,        /* max(x, 0)                                                        */
+  AGO_OP_RELU6 = 6,       /* min(max(x, 0), 6)                                                */
+  AGO_OP_GELU_TANH = 7,   /* 0.5 x (1 + tanh(sqrt(2/pi) (x + 0.044715 x^3)))                  */
+  AGO_OP_SCALE = 8,       /* x * f                                                            */
+  AGO_OP_SOFTMAX_ROWS = 9,/* softmax over the last dimension                                  */
+  AGO_OP_ADD_INPUT = 10   /* p: input index; + that subgraph input, element-wise (residual)   */
+} ago_op_kind_t;
+
+typedef struct {
+  int32_t kind;  /* ago_op_kind_t */
+  int32_t p[8];  /* per-kind integer parameters, in the order listed above; rest 0 */
+  float f;       /* AGO_OP_SCALE factor */
+} ago_op_t;
+
+#define AGO_MAX_INPUTS 4
+#define AGO_MAX_RANK 4
+#define AGO_MAX_OPS 32
+
+typedef struct {
+  uint32_t struct_size;                          /* sizeof(ago_subgraph_desc_t), ABI check */
+  int32_t mode;                                  /* ago_mode_t */
+  int32_t num_inputs;                            /* 1..AGO_MAX_INPUTS */
+  int32_t input_rank[AGO_MAX_INPUTS];            /* 2..4 */
+  int64_t input_shape[AGO_MAX_INPUTS][AGO_MAX_RANK];
+  int32_t input_dtype[AGO_MAX_INPUTS];           /* ago_dtype_t; all inputs share one dtype */
+  int32_t num_ops;                               /* 1..AGO_MAX_OPS */
+  const ago_op_t* ops;                           /* copied by create; caller keeps ownership */
+  int32_t output_dtype;                          /* ago_dtype_t; must equal the input dtype */
+} ago_subgraph_desc_t;
+
+/* What ago_subgraph_query can report (all as int64). */
+typedef enum {
+  AGO_Q_NUM_WEIGHTS = 0,       /* entries expected in weights[]                                   */
+  AGO_Q_WEIGHT_BYTES = 1,      /* + index i in the high half: see AGO_Q_INDEXED                    */
+  AGO_Q_OUTPUT_RANK = 2,
+  AGO_Q_OUTPUT_DIM = 3,        /* indexed                                                          */
+  AGO_Q_OUTPUT_BYTES = 4,
+  AGO_Q_FLOPS_TENSOR = 5,      /* 2 * MACs of the dense contractions, as the operators define them */
+  AGO_Q_FLOPS_CUDA = 6,        /* 2 * MACs of depthwise convolutions                               */
+  AGO_Q_SFU_OPS = 7,           /* exp / tanh evaluations                                           */
+  AGO_Q_IO_BYTES = 8,          /* inputs + weights + output; no intermediates                      */
+  AGO_Q_NUM_LINKS = 9,         /* adjacent complex -> complex pairs                                */
+  AGO_Q_LINK_CATEGORY = 10,    /* indexed; ago_link_category_t                                     */
+  AGO_Q_NUM_LAUNCHES = 11,     /* kernels launched by one ago_subgraph_run in this handle's mode   */
+  AGO_Q_FUSED_KERNEL = 12,     /* ago_fused_kernel_t chosen by the planner (0 when not fused)      */
+  AGO_Q_INTERMEDIATE_BYTES = 13,/* bytes written + read for intermediates in PER_MINI_SUBGRAPH mode */
+  AGO_Q_TILE_ROWS = 14,        /* fused kernel: downstream tile extent along the tiled dimension   */
+  AGO_Q_SMEM_BYTES = 15        /* fused kernel: dynamic shared memory per CTA                      */
+} ago_query_t;
+#define AGO_Q_INDEXED(what, i) ((int32_t)(what) | ((int32_t)(i) << 16))
+
+/* Fusion category of a complex -> complex link (Section III-B, "Removing the
+ * Re-computation" and Fig. "Inter-operator data dependency in intensive fusion"). */
+typedef enum {
+  AGO_LINK_DOWNSTREAM_DEPTHWISE = 1, /* downstream tile H2 W2 o2: spatial dims untiled, channels tiled   */
+  AGO_LINK_DOWNSTREAM_POINTWISE = 2, /* downstream tile h2 w2 O2: spatial/rows tiled, all output channels;
+                                        matrix multiplication counts as pointwise                       */
+  AGO_LINK_GENERAL = 3               /* reuse on O2, H2, W2: fusion needs halo recomputation             */
+} ago_link_category_t;
+
+typedef enum {
+  AGO_KERNEL_NONE = 0,
+  AGO_KERNEL_DEPTHWISE = 1,   /* a depthwise-only mini-subgraph                    */
+  AGO_KERNEL_MBV2_BLOCK = 2,  /* 1x1 conv -> depthwise 3x3 -> 1x1 conv [+ residual] */
+  AGO_KERNEL_FFN = 3,         /* GEMM -> GELU -> GEMM                               */
+  AGO_KERNEL_CONV3X3_PAIR = 4,/* conv3x3 -> conv3x3 [+ residual, ReLU]              */
+  AGO_KERNEL_ATTENTION = 5    /* QK^T -> scale -> softmax -> .V                     */
+} ago_fused_kernel_t;
+
+/* Validate the operator list, infer shapes, classify every complex -> complex
+ * link into the categories of Section III-B and pick the kernels for the asked
+ * mode. Host only; no device work. Returns NULL on failure (ago_last_error
+ * tells why). The desc and its ops array are copied. */
+ago_subgraph_t ago_subgraph_create(const ago_subgraph_desc_t* desc);
+
+/* Enqueue the subgraph on `cuda_stream` (a cudaStream_t; NULL = the legacy
+ * default stream) and return without synchronising.
+ *   inputs[num_inputs]  device pointers, in desc order (attention: Q, K, V)
+ *   weights[num_weights] device pointers, in order of appearance in the op
+ *                        list: each CONV2D / GEMM weight and each BIAS_ADD vector
+ *   outputs[1]          device pointer to the result
+ * FUSED mode launches one kernel (Section III-B, Fig. "Intensive fusion program
+ * of two convolutions": the upstream tile is produced inside the downstream
+ * operator's outer tile loops); the unfused modes launch one kernel per
+ * operator / per mini-subgraph and need a workspace (ago_subgraph_set_workspace).
+ * Errors: AGO_ERR_INVALID_ARG (NULL), AGO_ERR_ALIGNMENT, AGO_ERR_WORKSPACE,
+ * AGO_ERR_CUDA (launch failure). */
+ago_status_t ago_subgraph_run(ago_subgraph_t h, const void* const* inputs,
+                              const void* const* weights, void* const* outputs,
+                              void* cuda_stream);
+
+/* Same as ago_subgraph_run, but inputs and the output live in HOST memory
+ * (pinned memory makes the copies asynchronous). Per call: copy each host input
+ * to the caller's device staging buffer dev_inputs[i], run, copy dev_outputs[0]
+ * to host_outputs[0]; all on `cuda_stream`, no synchronisation. Weights stay
+ * device pointers. The staging buffers are caller-owned device memory of the
+ * tensors' sizes. */
+ago_status_t ago_subgraph_run_host(ago_subgraph_t h, const void* const* host_inputs,
+                                   const void* const* weights, void* const* host_outputs,
+                                   void* const* dev_inputs, void* const* dev_outputs,
+                                   void* cuda_stream);
+
+void ago_subgraph_destroy(ago_subgraph_t h); /* NULL is a no-op */
+
+/* Thread-local status and message of the last failing call on this thread. */
+ago_status_t ago_last_error(const char** msg);
+
+/* Device workspace for intermediates (unfused modes; 0 for fused kernels that
+ * need none). The caller allocates at least ago_subgraph_workspace_bytes(h)
+ * bytes, 256-byte aligned, and keeps them alive while the handle is used. */
+size_t ago_subgraph_workspace_bytes(ago_subgraph_t h);
+ago_status_t ago_subgraph_set_workspace(ago_subgraph_t h, void* dev_ptr, size_t bytes);
+
+/* Plan and work counters; `what` is an ago_query_t, optionally AGO_Q_INDEXED. */
+ago_status_t ago_subgraph_query(ago_subgraph_t h, int32_t what, int64_t* out);
+
+/* Synchronises the device and reads the handle's status word: AGO_OK, or
+ * AGO_ERR_TIMEOUT when a kernel gave up a bounded wait (its output is then
+ * undefined). The word is cleared by the call. */
+ago_status_t ago_subgraph_status(ago_subgraph_t h);
+
+/* Library version, "major.minor". */
+const char* ago_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* AGO_H_ */

@@ -1,0 +1,351 @@
+// C-ABI entry points: handle lifetime, argument checks and the dispatch of one
+// run onto the kernels chosen by the planner.
+#include <cuda_runtime.h>
+
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <string>
+
+#include "fused.h"
+#include "kernels.h"
+#include "plan.h"
+
+using namespace ago;
+
+struct ago_subgraph_s {
+  Plan plan;
+  void* workspace = nullptr;
+  size_t workspace_bytes = 0;
+  unsigned int* status_word = nullptr;  // device; allocated at the first run
+  int status_device = -1;
+  FusedState fused;                     // per-kernel host state (tensor maps, launch geometry)
+};
+
+namespace {
+
+thread_local ago_status_t g_status = AGO_OK;
+thread_local std::string g_msg;
+
+ago_status_t fail(ago_status_t s, const std::string& m) {
+  g_status = s;
+  g_msg = m;
+  return s;
+}
+
+ago_status_t cuda_fail(cudaError_t e, const char* what) {
+  return fail(AGO_ERR_CUDA, std::string(what) + ": " + cudaGetErrorString(e));
+}
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+size_t align256(size_t b) { return (b + 255) & ~size_t(255); }
+
+size_t needed_workspace(const Plan& p) {
+  if (p.mode == AGO_MODE_FUSED) return fused_workspace_bytes(p);
+  if (p.stages.size() <= 1) return 0;
+  return 2 * align256((size_t)p.max_intermediate_bytes);
+}
+
+// Translate ops [first, last] (all element-wise) into an epilogue program.
+void make_epilogue(const Plan& p, int first, int last, const void* const* inputs, const void* const* weights,
+                   EpiProgram* e) {
+  e->n = 0;
+  for (int i = first; i <= last; ++i) {
+    const OpInfo& o = p.ops[i];
+    int k = e->n++;
+    e->ptr[k] = nullptr;
+    e->f[k] = 0.0f;
+    switch (o.op.kind) {
+      case AGO_OP_BIAS_ADD: e->code[k] = EPI_BIAS; e->ptr[k] = weights[o.weight]; break;
+      case AGO_OP_RELU: e->code[k] = EPI_RELU; break;
+      case AGO_OP_RELU6: e->code[k] = EPI_RELU6; break;
+      case AGO_OP_GELU_TANH: e->code[k] = EPI_GELU; break;
+      case AGO_OP_SCALE: e->code[k] = EPI_SCALE; e->f[k] = o.op.f; break;
+      case AGO_OP_ADD_INPUT: e->code[k] = EPI_ADD; e->ptr[k] = inputs[o.op.p[0]]; break;
+      default: --e->n; break;
+    }
+  }
+}
+
+cudaError_t launch_complex(const Plan& p, const OpInfo& o, const void* src, void* dst, const void* const* inputs,
+                           const void* const* weights, const EpiProgram& epi, bool tuned_depthwise,
+                           cudaStream_t stream) {
+  const int32_t* q = o.op.p;
+  if (o.op.kind == AGO_OP_CONV2D && o.depthwise()) {
+    DepthwiseArgs a{};
+    a.in = src; a.w = weights[o.weight]; a.out = dst;
+    a.N = (int)o.in.d[0]; a.H = (int)o.in.d[1]; a.W = (int)o.in.d[2]; a.C = (int)o.in.d[3];
+    a.R = q[1]; a.S = q[2]; a.stride = q[3]; a.pad = q[4];
+    a.Ho = (int)o.out.d[1]; a.Wo = (int)o.out.d[2];
+    a.dtype = p.dtype;
+    a.epi = epi;
+    return tuned_depthwise ? launch_depthwise_fused(a, stream) : launch_depthwise_generic(a, stream);
+  }
+  GemmArgs g{};
+  g.A = src; g.C = dst; g.epi = epi;
+  g.batches = 1; g.heads = 1;
+  switch (o.op.kind) {
+    case AGO_OP_CONV2D: {
+      g.B = weights[o.weight];
+      g.H = (int)o.in.d[1]; g.W = (int)o.in.d[2]; g.Cin = (int)o.in.d[3];
+      g.R = q[1]; g.S = q[2]; g.stride = q[3]; g.pad = q[4];
+      g.Ho = (int)o.out.d[1]; g.Wo = (int)o.out.d[2];
+      g.M = (int)(o.out.d[0] * o.out.d[1] * o.out.d[2]);
+      g.N = q[0];
+      g.K = g.R * g.S * g.Cin;
+      g.a_im2col = 1; g.lda = 0;
+      g.b_kmajor = 1; g.ldb = g.K;
+      g.ldc = g.N;
+      break;
+    }
+    case AGO_OP_GEMM: {
+      g.B = weights[o.weight];
+      g.K = (int)o.in.last(); g.N = q[0];
+      g.M = (int)(o.in.numel() / g.K);
+      g.a_im2col = 0; g.lda = g.K;
+      g.b_kmajor = 0; g.ldb = g.N;
+      g.ldc = g.N;
+      break;
+    }
+    case AGO_OP_BATCHED_QKT: {
+      const int64_t B = o.in.d[0], S = o.in.d[1], E = o.in.d[2];
+      const int heads = q[1], hd = q[2];
+      g.B = inputs[q[0]];
+      g.M = (int)S; g.N = (int)S; g.K = hd;
+      g.a_im2col = 0; g.lda = E;
+      g.b_kmajor = 1; g.ldb = E;
+      g.ldc = S;
+      g.batches = (int)(B * heads); g.heads = heads;
+      g.a_sb = S * E; g.a_sh = hd; g.b_sb = S * E; g.b_sh = hd;
+      g.c_sb = (int64_t)heads * S * S; g.c_sh = S * S;
+      break;
+    }
+    case AGO_OP_BATCHED_PV: {
+      const int64_t B = o.in.d[0], S = o.in.d[2];
+      const int heads = q[1], hd = q[2];
+      const int64_t E = (int64_t)heads * hd;
+      g.B = inputs[q[0]];
+      g.M = (int)S; g.N = hd; g.K = (int)S;
+      g.a_im2col = 0; g.lda = S;
+      g.b_kmajor = 0; g.ldb = E;
+      g.ldc = E;
+      g.batches = (int)(B * heads); g.heads = heads;
+      g.a_sb = (int64_t)heads * S * S; g.a_sh = S * S; g.b_sb = S * E; g.b_sh = hd;
+      g.c_sb = S * E; g.c_sh = hd;
+      break;
+    }
+    default:
+      return cudaErrorInvalidValue;
+  }
+  return launch_gemm_generic(g, stream);
+}
+
+// One launch per stage; intermediates ping-pong between the two halves of `ws`.
+ago_status_t run_unfused(ago_subgraph_s* h, const void* const* inputs, const void* const* weights, void* out,
+                         void* ws, size_t ws_bytes, cudaStream_t stream) {
+  const Plan& p = h->plan;
+  const size_t need = p.stages.size() <= 1 ? 0 : 2 * align256((size_t)p.max_intermediate_bytes);
+  if (need > 0 && (ws == nullptr || ws_bytes < need))
+    return fail(AGO_ERR_WORKSPACE, "workspace missing or smaller than ago_subgraph_workspace_bytes()");
+  char* buf[2] = {static_cast<char*>(ws), static_cast<char*>(ws) + need / 2};
+  const void* src = inputs[0];
+  int flip = 0;
+  for (size_t si = 0; si < p.stages.size(); ++si) {
+    const Stage& s = p.stages[si];
+    void* dst = (si + 1 == p.stages.size()) ? out : static_cast<void*>(buf[flip]);
+    cudaError_t e;
+    if (s.softmax) {
+      const Shape& sh = p.ops[s.first].in;
+      e = launch_softmax_rows(src, dst, sh.numel() / sh.last(), (int)sh.last(), p.dtype, stream);
+    } else if (s.complex_index >= 0) {
+      EpiProgram epi;
+      make_epilogue(p, s.first + 1, s.last, inputs, weights, &epi);
+      e = launch_complex(p, p.ops[s.first], src, dst, inputs, weights, epi, false, stream);
+    } else {
+      EpiProgram epi;
+      make_epilogue(p, s.first, s.last, inputs, weights, &epi);
+      const Shape& sh = p.ops[s.first].in;
+      e = launch_elementwise(src, dst, sh.numel(), (int)sh.last(), p.dtype, epi, stream);
+    }
+    if (e != cudaSuccess) return cuda_fail(e, "kernel launch");
+    src = dst;
+    flip ^= 1;
+  }
+  return AGO_OK;
+}
+
+ago_status_t ensure_status_word(ago_subgraph_s* h) {
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return cuda_fail(e, "cudaGetDevice");
+  if (h->status_word && h->status_device == dev) return AGO_OK;
+  if (h->status_word) { cudaFree(h->status_word); h->status_word = nullptr; }
+  e = cudaMalloc(&h->status_word, sizeof(unsigned int));
+  if (e != cudaSuccess) return cuda_fail(e, "cudaMalloc(status word)");
+  e = cudaMemset(h->status_word, 0, sizeof(unsigned int));
+  if (e != cudaSuccess) return cuda_fail(e, "cudaMemset(status word)");
+  h->status_device = dev;
+  return AGO_OK;
+}
+
+ago_status_t check_run_args(ago_subgraph_s* h, const void* const* inputs, const void* const* weights,
+                            void* const* outputs) {
+  if (!h) return fail(AGO_ERR_INVALID_ARG, "handle is NULL");
+  if (!inputs || !outputs) return fail(AGO_ERR_INVALID_ARG, "inputs / outputs array is NULL");
+  const Plan& p = h->plan;
+  if (!p.weight_bytes.empty() && !weights) return fail(AGO_ERR_INVALID_ARG, "weights array is NULL");
+  for (int i = 0; i < p.num_inputs; ++i) {
+    if (!inputs[i]) return fail(AGO_ERR_INVALID_ARG, "inputs[" + std::to_string(i) + "] is NULL");
+    if (!aligned16(inputs[i])) return fail(AGO_ERR_ALIGNMENT, "inputs[" + std::to_string(i) + "] is not 16-byte aligned");
+  }
+  for (size_t i = 0; i < p.weight_bytes.size(); ++i) {
+    if (!weights[i]) return fail(AGO_ERR_INVALID_ARG, "weights[" + std::to_string(i) + "] is NULL");
+    if (!aligned16(weights[i])) return fail(AGO_ERR_ALIGNMENT, "weights[" + std::to_string(i) + "] is not 16-byte aligned");
+  }
+  if (!outputs[0]) return fail(AGO_ERR_INVALID_ARG, "outputs[0] is NULL");
+  if (!aligned16(outputs[0])) return fail(AGO_ERR_ALIGNMENT, "outputs[0] is not 16-byte aligned");
+  return AGO_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* ago_version(void) { return "0.1"; }
+
+ago_status_t ago_last_error(const char** msg) {
+  if (msg) *msg = g_msg.c_str();
+  return g_status;
+}
+
+ago_subgraph_t ago_subgraph_create(const ago_subgraph_desc_t* desc) {
+  ago_subgraph_s* h = new (std::nothrow) ago_subgraph_s();
+  if (!h) { fail(AGO_ERR_INVALID_ARG, "out of host memory"); return nullptr; }
+  std::string err;
+  ago_status_t s = build_plan(desc, &h->plan, &err);
+  if (s == AGO_OK && h->plan.mode == AGO_MODE_FUSED) s = fused_plan(&h->plan, &h->fused, &err);
+  if (s != AGO_OK) {
+    fail(s, err);
+    delete h;
+    return nullptr;
+  }
+  g_status = AGO_OK;
+  g_msg.clear();
+  return h;
+}
+
+void ago_subgraph_destroy(ago_subgraph_t h) {
+  if (!h) return;
+  if (h->status_word) cudaFree(h->status_word);
+  delete h;
+}
+
+size_t ago_subgraph_workspace_bytes(ago_subgraph_t h) { return h ? needed_workspace(h->plan) : 0; }
+
+ago_status_t ago_subgraph_set_workspace(ago_subgraph_t h, void* dev_ptr, size_t bytes) {
+  if (!h) return fail(AGO_ERR_INVALID_ARG, "handle is NULL");
+  if (dev_ptr && (reinterpret_cast<uintptr_t>(dev_ptr) & 255u)) return fail(AGO_ERR_ALIGNMENT, "workspace is not 256-byte aligned");
+  if (bytes < needed_workspace(h->plan)) return fail(AGO_ERR_WORKSPACE, "workspace smaller than ago_subgraph_workspace_bytes()");
+  h->workspace = dev_ptr;
+  h->workspace_bytes = bytes;
+  return AGO_OK;
+}
+
+ago_status_t ago_subgraph_run(ago_subgraph_t h, const void* const* inputs, const void* const* weights,
+                              void* const* outputs, void* cuda_stream) {
+  ago_status_t s = check_run_args(h, inputs, weights, outputs);
+  if (s != AGO_OK) return s;
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  s = ensure_status_word(h);
+  if (s != AGO_OK) return s;
+  const Plan& p = h->plan;
+  if (p.mode != AGO_MODE_FUSED) return run_unfused(h, inputs, weights, outputs[0], h->workspace, h->workspace_bytes, stream);
+  if (p.fused_kernel == AGO_KERNEL_DEPTHWISE) {
+    EpiProgram epi;
+    make_epilogue(p, 1, (int)p.ops.size() - 1, inputs, weights, &epi);
+    if (epi.n != (int)p.ops.size() - 1 || epi.n > kMaxEpi) return fail(AGO_ERR_UNSUPPORTED, "too many simple operators");
+    cudaError_t e = launch_complex(p, p.ops[0], inputs[0], outputs[0], inputs, weights, epi, true, stream);
+    if (e != cudaSuccess) return cuda_fail(e, "depthwise kernel launch");
+    return AGO_OK;
+  }
+  std::string err;
+  if (needed_workspace(p) > 0 && (h->workspace == nullptr || h->workspace_bytes < needed_workspace(p)))
+    return fail(AGO_ERR_WORKSPACE, "workspace missing or smaller than ago_subgraph_workspace_bytes()");
+  s = fused_run(p, &h->fused, inputs, weights, outputs[0], h->workspace, h->status_word, stream, &err);
+  if (s != AGO_OK) return fail(s, err);
+  return AGO_OK;
+}
+
+ago_status_t ago_subgraph_run_host(ago_subgraph_t h, const void* const* host_inputs, const void* const* weights,
+                                   void* const* host_outputs, void* const* dev_inputs, void* const* dev_outputs,
+                                   void* cuda_stream) {
+  if (!h) return fail(AGO_ERR_INVALID_ARG, "handle is NULL");
+  if (!host_inputs || !host_outputs || !dev_inputs || !dev_outputs || !host_outputs[0])
+    return fail(AGO_ERR_INVALID_ARG, "NULL array");
+  const Plan& p = h->plan;
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  for (int i = 0; i < p.num_inputs; ++i) {
+    if (!host_inputs[i] || !dev_inputs[i]) return fail(AGO_ERR_INVALID_ARG, "NULL input buffer");
+    cudaError_t e = cudaMemcpyAsync(dev_inputs[i], host_inputs[i], (size_t)p.inputs[i].numel() * elem_bytes(p.dtype),
+                                    cudaMemcpyHostToDevice, stream);
+    if (e != cudaSuccess) return cuda_fail(e, "host-to-device copy");
+  }
+  ago_status_t s = ago_subgraph_run(h, const_cast<const void* const*>(dev_inputs), weights, dev_outputs, cuda_stream);
+  if (s != AGO_OK) return s;
+  cudaError_t e = cudaMemcpyAsync(host_outputs[0], dev_outputs[0], (size_t)p.output.numel() * elem_bytes(p.dtype),
+                                  cudaMemcpyDeviceToHost, stream);
+  if (e != cudaSuccess) return cuda_fail(e, "device-to-host copy");
+  return AGO_OK;
+}
+
+ago_status_t ago_subgraph_query(ago_subgraph_t h, int32_t what, int64_t* out) {
+  if (!h || !out) return fail(AGO_ERR_INVALID_ARG, "NULL argument");
+  const Plan& p = h->plan;
+  const int idx = (what >> 16) & 0xffff;
+  switch (what & 0xffff) {
+    case AGO_Q_NUM_WEIGHTS: *out = (int64_t)p.weight_bytes.size(); break;
+    case AGO_Q_WEIGHT_BYTES:
+      if (idx >= (int)p.weight_bytes.size()) return fail(AGO_ERR_INVALID_ARG, "weight index out of range");
+      *out = p.weight_bytes[idx]; break;
+    case AGO_Q_OUTPUT_RANK: *out = p.output.rank; break;
+    case AGO_Q_OUTPUT_DIM:
+      if (idx >= p.output.rank) return fail(AGO_ERR_INVALID_ARG, "dimension index out of range");
+      *out = p.output.d[idx]; break;
+    case AGO_Q_OUTPUT_BYTES: *out = p.output.numel() * elem_bytes(p.dtype); break;
+    case AGO_Q_FLOPS_TENSOR: *out = p.flops_tensor; break;
+    case AGO_Q_FLOPS_CUDA: *out = p.flops_cuda; break;
+    case AGO_Q_SFU_OPS: *out = p.sfu_ops; break;
+    case AGO_Q_IO_BYTES: *out = p.io_bytes; break;
+    case AGO_Q_NUM_LINKS: *out = (int64_t)p.link_category.size(); break;
+    case AGO_Q_LINK_CATEGORY:
+      if (idx >= (int)p.link_category.size()) return fail(AGO_ERR_INVALID_ARG, "link index out of range");
+      *out = p.link_category[idx]; break;
+    case AGO_Q_NUM_LAUNCHES: *out = p.num_launches; break;
+    case AGO_Q_FUSED_KERNEL: *out = p.fused_kernel; break;
+    case AGO_Q_INTERMEDIATE_BYTES: *out = p.intermediate_bytes; break;
+    case AGO_Q_TILE_ROWS: *out = p.tile_rows; break;
+    case AGO_Q_SMEM_BYTES: *out = p.smem_bytes; break;
+    default: return fail(AGO_ERR_INVALID_ARG, "unknown query");
+  }
+  return AGO_OK;
+}
+
+ago_status_t ago_subgraph_status(ago_subgraph_t h) {
+  if (!h) return fail(AGO_ERR_INVALID_ARG, "handle is NULL");
+  cudaError_t e = cudaDeviceSynchronize();
+  if (e != cudaSuccess) return cuda_fail(e, "cudaDeviceSynchronize");
+  if (!h->status_word) return AGO_OK;
+  unsigned int w = 0;
+  e = cudaMemcpy(&w, h->status_word, sizeof(w), cudaMemcpyDeviceToHost);
+  if (e != cudaSuccess) return cuda_fail(e, "cudaMemcpy(status word)");
+  if (w != 0) {
+    cudaMemset(h->status_word, 0, sizeof(w));
+    char buf[96];
+    std::snprintf(buf, sizeof(buf), "a bounded device-side wait expired (code 0x%x)", w);
+    return fail(AGO_ERR_TIMEOUT, buf);
+  }
+  return AGO_OK;
+}
+
+}  // extern "C"

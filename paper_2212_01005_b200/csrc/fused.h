@@ -1,0 +1,31 @@
+// Host side of the fused kernels: per-handle state, plan-time tile choice and
+// the run-time dispatch onto the kernel of the matched family.
+#pragma once
+#include <cuda_runtime.h>
+
+#include <string>
+
+#include "plan.h"
+
+namespace ago {
+
+struct FusedState {
+  int tile_rows = 0;       // downstream tile extent along the tiled dimension
+  int grid = 0;            // CTAs
+  int smem_bytes = 0;      // dynamic shared memory per CTA
+  bool attr_set = false;   // cudaFuncSetAttribute done for this process/device
+};
+
+// Chooses tiles and shared-memory budget for plan->fused_kernel; fills
+// plan->tile_rows / smem_bytes. Host only.
+ago_status_t fused_plan(Plan* plan, FusedState* st, std::string* err);
+
+// Scratch the fused kernel needs in device memory (0 for most families).
+size_t fused_workspace_bytes(const Plan& plan);
+
+// Enqueue the fused kernel.
+ago_status_t fused_run(const Plan& plan, FusedState* st, const void* const* inputs, const void* const* weights,
+                       void* output, void* workspace, unsigned int* status_word, cudaStream_t stream,
+                       std::string* err);
+
+}  // namespace ago

@@ -1,0 +1,50 @@
+// Launch functions of the device kernels. Every function enqueues on `stream`
+// and returns the cudaError_t of the launch; none synchronises.
+#pragma once
+#include <cuda_runtime.h>
+
+#include <cstdint>
+
+#include "plan.h"
+
+namespace ago {
+
+// ---- generic kernels of the unfused modes (CUDA cores) ----------------------
+
+// C[m][n] = sum_k A(m,k) * B(n,k), fp32 accumulate, bf16 in/out, epilogue program.
+struct GemmArgs {
+  const void* A; const void* B; void* C;
+  int M, N, K;
+  // A: row-major [M][K] with leading dimension lda, or an implicit im2col view of an NHWC tensor
+  int a_im2col; int64_t lda;
+  int H, W, Cin, R, S, stride, pad, Ho, Wo;
+  // B: K-major ([N][K], ldb) or N-major ([K][N], ldb)
+  int b_kmajor; int64_t ldb;
+  int64_t ldc;
+  // batch = blockIdx.z = b * heads + h
+  int batches, heads;
+  int64_t a_sb, a_sh, b_sb, b_sh, c_sb, c_sh;
+  EpiProgram epi;
+};
+cudaError_t launch_gemm_generic(const GemmArgs& a, cudaStream_t stream);
+
+struct DepthwiseArgs {
+  const void* in; const void* w; void* out;
+  int N, H, W, C, R, S, stride, pad, Ho, Wo;
+  int dtype;  // AGO_BF16 | AGO_FP32 (activations and weights)
+  EpiProgram epi;
+};
+cudaError_t launch_depthwise_generic(const DepthwiseArgs& a, cudaStream_t stream);
+
+// y = program(x) element-wise over a [rows][C] view.
+cudaError_t launch_elementwise(const void* x, void* y, int64_t numel, int C, int dtype, const EpiProgram& epi,
+                               cudaStream_t stream);
+// Row softmax over the last dimension, fp32 math.
+cudaError_t launch_softmax_rows(const void* x, void* y, int64_t rows, int cols, int dtype, cudaStream_t stream);
+
+// ---- fused kernels -------------------------------------------------------------
+
+// Depthwise-only mini-subgraph tuned kernel (vectorised over channels).
+cudaError_t launch_depthwise_fused(const DepthwiseArgs& a, cudaStream_t stream);
+
+}  // namespace ago

@@ -1,0 +1,215 @@
+// Generic CUDA-core kernels of the unfused modes: one launch per operator
+// (Section III-A, "Loop nest of a mini-subgraph without fusion") or per
+// mini-subgraph with the simple operators applied in the epilogue (Section
+// III-A, "Conventional fusion within a mini-subgraph"). They accept any valid
+// shape; intermediates between launches live in device memory.
+#include <cuda_bf16.h>
+
+#include "kernels.h"
+
+namespace ago {
+
+namespace {
+
+__device__ __forceinline__ float gelu_tanh_f(float v) {
+  const float c = 0.7978845608028654f;
+  return 0.5f * v * (1.0f + tanhf(c * (v + 0.044715f * v * v * v)));
+}
+
+template <typename T> __device__ __forceinline__ float ld(const void* p, int64_t i);
+template <> __device__ __forceinline__ float ld<__nv_bfloat16>(const void* p, int64_t i) {
+  return __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(p)[i]);
+}
+template <> __device__ __forceinline__ float ld<float>(const void* p, int64_t i) {
+  return reinterpret_cast<const float*>(p)[i];
+}
+template <typename T> __device__ __forceinline__ void st(void* p, int64_t i, float v);
+template <> __device__ __forceinline__ void st<__nv_bfloat16>(void* p, int64_t i, float v) {
+  reinterpret_cast<__nv_bfloat16*>(p)[i] = __float2bfloat16_rn(v);
+}
+template <> __device__ __forceinline__ void st<float>(void* p, int64_t i, float v) {
+  reinterpret_cast<float*>(p)[i] = v;
+}
+
+// The simple operators, applied in program order to one element. `c` is the
+// index along the last dimension, `idx` the element's linear index.
+template <typename T>
+__device__ __forceinline__ float run_epilogue(const EpiProgram& e, float v, int c, int64_t idx) {
+  for (int i = 0; i < e.n; ++i) {
+    switch (e.code[i]) {
+      case EPI_BIAS: v += reinterpret_cast<const float*>(e.ptr[i])[c]; break;
+      case EPI_RELU: v = fmaxf(v, 0.0f); break;
+      case EPI_RELU6: v = fminf(fmaxf(v, 0.0f), 6.0f); break;
+      case EPI_GELU: v = gelu_tanh_f(v); break;
+      case EPI_SCALE: v *= e.f[i]; break;
+      case EPI_ADD: v += ld<T>(e.ptr[i], idx); break;
+    }
+  }
+  return v;
+}
+
+constexpr int TM = 64, TN = 64, TK = 16;
+
+__global__ void __launch_bounds__(256) gemm_generic_kernel(const GemmArgs a) {
+  __shared__ float As[TK][TM + 4];
+  __shared__ float Bs[TK][TN + 4];
+  const int batch = blockIdx.z;
+  const int bb = batch / a.heads, hh = batch % a.heads;
+  const __nv_bfloat16* A = reinterpret_cast<const __nv_bfloat16*>(a.A) + bb * a.a_sb + hh * a.a_sh;
+  const __nv_bfloat16* B = reinterpret_cast<const __nv_bfloat16*>(a.B) + bb * a.b_sb + hh * a.b_sh;
+  const int64_t c_off = bb * a.c_sb + hh * a.c_sh;
+  const int m0 = blockIdx.x * TM, n0 = blockIdx.y * TN;
+  const int tid = threadIdx.x;
+  const int tx = tid % 16, ty = tid / 16;
+  float acc[4][4] = {};
+
+  for (int k0 = 0; k0 < a.K; k0 += TK) {
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      const int idx = tid + e * 256;
+      const int row = idx / TK, kk = idx % TK;
+      const int m = m0 + row, k = k0 + kk;
+      float v = 0.0f;
+      if (m < a.M && k < a.K) {
+        if (!a.a_im2col) {
+          v = __bfloat162float(A[(int64_t)m * a.lda + k]);
+        } else {
+          const int ci = k % a.Cin;
+          const int rs = k / a.Cin;
+          const int s = rs % a.S, r = rs / a.S;
+          const int wo = m % a.Wo;
+          const int t = m / a.Wo;
+          const int ho = t % a.Ho, img = t / a.Ho;
+          const int h = ho * a.stride + r - a.pad, w = wo * a.stride + s - a.pad;
+          if (h >= 0 && h < a.H && w >= 0 && w < a.W)
+            v = __bfloat162float(A[(((int64_t)img * a.H + h) * a.W + w) * a.Cin + ci]);
+        }
+      }
+      As[kk][row] = v;
+    }
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      const int idx = tid + e * 256;
+      int nn, kk;
+      if (a.b_kmajor) { nn = idx / TK; kk = idx % TK; } else { kk = idx / TN; nn = idx % TN; }
+      const int n = n0 + nn, k = k0 + kk;
+      float v = 0.0f;
+      if (n < a.N && k < a.K)
+        v = __bfloat162float(a.b_kmajor ? B[(int64_t)n * a.ldb + k] : B[(int64_t)k * a.ldb + n]);
+      Bs[kk][nn] = v;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int kk = 0; kk < TK; ++kk) {
+      float av[4], bv[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) av[i] = As[kk][ty * 4 + i];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) bv[j] = Bs[kk][tx * 4 + j];
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(av[i], bv[j], acc[i][j]);
+    }
+    __syncthreads();
+  }
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const int m = m0 + ty * 4 + i;
+    if (m >= a.M) continue;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const int n = n0 + tx * 4 + j;
+      if (n >= a.N) continue;
+      const int64_t idx = c_off + (int64_t)m * a.ldc + n;
+      float v = run_epilogue<__nv_bfloat16>(a.epi, acc[i][j], n, idx);
+      reinterpret_cast<__nv_bfloat16*>(a.C)[idx] = __float2bfloat16_rn(v);
+    }
+  }
+}
+
+template <typename T>
+__global__ void __launch_bounds__(256) depthwise_generic_kernel(const DepthwiseArgs a, int64_t total) {
+  const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= total) return;
+  const int c = (int)(idx % a.C);
+  int64_t t = idx / a.C;
+  const int wo = (int)(t % a.Wo); t /= a.Wo;
+  const int ho = (int)(t % a.Ho);
+  const int64_t n = t / a.Ho;
+  float acc = 0.0f;
+  for (int r = 0; r < a.R; ++r) {
+    const int h = ho * a.stride + r - a.pad;
+    if (h < 0 || h >= a.H) continue;
+    for (int s = 0; s < a.S; ++s) {
+      const int w = wo * a.stride + s - a.pad;
+      if (w < 0 || w >= a.W) continue;
+      acc = fmaf(ld<T>(a.in, ((n * a.H + h) * a.W + w) * a.C + c), ld<T>(a.w, (r * a.S + s) * a.C + c), acc);
+    }
+  }
+  st<T>(a.out, idx, run_epilogue<T>(a.epi, acc, c, idx));
+}
+
+template <typename T>
+__global__ void __launch_bounds__(256) elementwise_kernel(const void* x, void* y, int64_t numel, int C,
+                                                          const EpiProgram epi) {
+  const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= numel) return;
+  st<T>(y, idx, run_epilogue<T>(epi, ld<T>(x, idx), (int)(idx % C), idx));
+}
+
+// One warp per row: p_j = exp(s_j - max) / sum.
+template <typename T>
+__global__ void __launch_bounds__(256) softmax_rows_kernel(const void* x, void* y, int64_t rows, int cols) {
+  const int64_t row = (int64_t)blockIdx.x * (blockDim.x / 32) + threadIdx.x / 32;
+  if (row >= rows) return;
+  const int lane = threadIdx.x % 32;
+  const int64_t base = row * cols;
+  float m = -INFINITY;
+  for (int j = lane; j < cols; j += 32) m = fmaxf(m, ld<T>(x, base + j));
+  for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+  float sum = 0.0f;
+  for (int j = lane; j < cols; j += 32) sum += expf(ld<T>(x, base + j) - m);
+  for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+  const float inv = 1.0f / sum;
+  for (int j = lane; j < cols; j += 32) st<T>(y, base + j, expf(ld<T>(x, base + j) - m) * inv);
+}
+
+}  // namespace
+
+cudaError_t launch_gemm_generic(const GemmArgs& a, cudaStream_t stream) {
+  dim3 grid((a.M + TM - 1) / TM, (a.N + TN - 1) / TN, a.batches);
+  gemm_generic_kernel<<<grid, 256, 0, stream>>>(a);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_depthwise_generic(const DepthwiseArgs& a, cudaStream_t stream) {
+  const int64_t total = (int64_t)a.N * a.Ho * a.Wo * a.C;
+  const unsigned blocks = (unsigned)((total + 255) / 256);
+  if (a.dtype == AGO_FP32)
+    depthwise_generic_kernel<float><<<blocks, 256, 0, stream>>>(a, total);
+  else
+    depthwise_generic_kernel<__nv_bfloat16><<<blocks, 256, 0, stream>>>(a, total);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_elementwise(const void* x, void* y, int64_t numel, int C, int dtype, const EpiProgram& epi,
+                               cudaStream_t stream) {
+  const unsigned blocks = (unsigned)((numel + 255) / 256);
+  if (dtype == AGO_FP32)
+    elementwise_kernel<float><<<blocks, 256, 0, stream>>>(x, y, numel, C, epi);
+  else
+    elementwise_kernel<__nv_bfloat16><<<blocks, 256, 0, stream>>>(x, y, numel, C, epi);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_softmax_rows(const void* x, void* y, int64_t rows, int cols, int dtype, cudaStream_t stream) {
+  const unsigned blocks = (unsigned)((rows + 7) / 8);
+  if (dtype == AGO_FP32)
+    softmax_rows_kernel<float><<<blocks, 256, 0, stream>>>(x, y, rows, cols);
+  else
+    softmax_rows_kernel<__nv_bfloat16><<<blocks, 256, 0, stream>>>(x, y, rows, cols);
+  return cudaGetLastError();
+}
+
+}  // namespace ago

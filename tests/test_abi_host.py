@@ -1,0 +1,138 @@
+"""Host-side checks that need no GPU: the library loads, exports every symbol
+the header declares, validates descriptors, classifies links and counts work."""
+import ctypes
+import os
+import re
+
+import numpy as np
+import pytest
+
+from paper_2212_01005_b200 import binding as B
+from paper_2212_01005_b200 import workloads as WL
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def test_library_exports_every_declared_symbol():
+    lib = B.load()
+    hdr = open(os.path.join(ROOT, "include", "ago.h")).read()
+    hdr = re.sub(r"/\*.*?\*/", "", hdr, flags=re.S)
+    declared = set(re.findall(r"\b(ago_[a-z_]+)\s*\(", hdr))
+    assert declared, "no declarations found"
+    assert declared == set(B.EXPORTS)
+    for name in declared:
+        assert hasattr(lib, name), name
+    assert B.ago_version() == "0.1"
+
+
+def test_desc_struct_matches_header_layout():
+    # int32 fields, then [4][4] int64, ...; the library checks struct_size itself
+    d, _ = B.make_desc([("relu", {})], [(8, 8)], "per_op")
+    h = B.ago_subgraph_create(d)
+    assert h, B.ago_last_error()
+    B.ago_subgraph_destroy(h)
+    d.struct_size = 12
+    assert not B.ago_subgraph_create(d)
+    st, msg = B.ago_last_error()
+    assert st == B.AGO_ERR_INVALID_ARG and "struct_size" in msg
+
+
+@pytest.mark.parametrize("name", WL.ALL)
+def test_plan_counters_match_workload_arithmetic(name):
+    wl = WL.get(name)
+    sg = B.Subgraph(wl.ops, wl.input_shapes, mode="per_mini_subgraph")
+    assert sg.output_shape == tuple(wl.output_shape)
+    assert sg.num_weights == len(wl.weight_shapes)
+    fl = WL.flops(wl)
+    assert sg.query(B.AGO_Q_FLOPS_TENSOR) == int(fl["tensor"])
+    assert sg.query(B.AGO_Q_FLOPS_CUDA) == int(fl["cuda"])
+    assert sg.query(B.AGO_Q_SFU_OPS) == int(fl["sfu"])
+    assert sg.query(B.AGO_Q_IO_BYTES) == WL.io_bytes(wl)
+    for i, (shp, kind) in enumerate(zip(wl.weight_shapes, wl.weight_kinds)):
+        assert sg.query(B.AGO_Q_WEIGHT_BYTES, i) == int(np.prod(shp)) * (4 if kind == "bias" else 2)
+    sg.close()
+
+
+def test_link_categories_follow_the_downstream_operator():
+    # Section III-B: downstream depthwise / downstream pointwise (or matmul) / anything else
+    cases = {
+        "mbv2_56": [B.AGO_LINK_DOWNSTREAM_DEPTHWISE, B.AGO_LINK_DOWNSTREAM_POINTWISE],
+        "ffn_512": [B.AGO_LINK_DOWNSTREAM_POINTWISE],
+        "resnet_56": [B.AGO_LINK_GENERAL],
+        "attn_384": [B.AGO_LINK_DOWNSTREAM_POINTWISE],
+    }
+    for name, want in cases.items():
+        wl = WL.get(name)
+        sg = B.Subgraph(wl.ops, wl.input_shapes, mode="per_op")
+        n = sg.query(B.AGO_Q_NUM_LINKS)
+        assert [sg.query(B.AGO_Q_LINK_CATEGORY, i) for i in range(n)] == want
+        sg.close()
+
+
+def test_launch_counts_per_mode():
+    wl = WL.get("mbv2_14")
+    per_op = B.Subgraph(wl.ops, wl.input_shapes, mode="per_op")
+    mini = B.Subgraph(wl.ops, wl.input_shapes, mode="per_mini_subgraph")
+    assert per_op.query(B.AGO_Q_NUM_LAUNCHES) == len(wl.ops) == 9
+    assert mini.query(B.AGO_Q_NUM_LAUNCHES) == 3
+    assert per_op.workspace_bytes >= 2 * 196 * 192 * 2
+    wl = WL.get("attn_384", batch=1)
+    mini = B.Subgraph(wl.ops, wl.input_shapes, mode="per_mini_subgraph")
+    assert mini.query(B.AGO_Q_NUM_LAUNCHES) == 3          # QK^T+scale | softmax | PV
+    # intermediates of the attention chain: scores and probabilities, written and read once each
+    assert mini.query(B.AGO_Q_INTERMEDIATE_BYTES) == 2 * 2 * 12 * 384 * 384 * 2
+
+
+def _expect_fail(ops, shapes, status, mode="per_op", dtype=B.AGO_BF16, needle=""):
+    with pytest.raises(B.AgoError) as e:
+        B.Subgraph(ops, shapes, mode=mode, dtype=dtype)
+    assert e.value.status == status, str(e.value)
+    assert needle in str(e.value)
+
+
+def test_create_rejects_bad_descriptors():
+    conv = lambda **k: ("conv2d", dict(dict(O=8, R=3, S=3, stride=1, pad=1, groups=1), **k))
+    _expect_fail([conv()], [(4, 8)], B.AGO_ERR_SHAPE, needle="NHWC")
+    _expect_fail([conv(O=12)], [(1, 4, 4, 8)], B.AGO_ERR_SHAPE, needle="multiple")
+    _expect_fail([conv(groups=4)], [(1, 4, 4, 8)], B.AGO_ERR_SHAPE, needle="groups")
+    _expect_fail([conv(R=7, pad=0)], [(1, 4, 4, 8)], B.AGO_ERR_SHAPE, needle="empty")
+    _expect_fail([("gemm", dict(N=0))], [(4, 8)], B.AGO_ERR_SHAPE)
+    _expect_fail([("add_input", dict(input=3))], [(4, 8)], B.AGO_ERR_SHAPE)
+    _expect_fail([("qkt", dict(input=1, heads=3, head_dim=8))], [(1, 8, 16), (1, 8, 16)], B.AGO_ERR_SHAPE)
+    _expect_fail([("relu", {})], [(4, 7)], B.AGO_ERR_SHAPE, needle="16-byte")
+    _expect_fail([("gemm", dict(N=8))], [(4, 8)], B.AGO_ERR_UNSUPPORTED, dtype=B.AGO_FP32)
+    # a chain that is valid but matches no fused family
+    _expect_fail([("gemm", dict(N=8)), ("relu", {})], [(4, 8)], B.AGO_ERR_UNSUPPORTED, mode="fused", needle="family")
+    d, _ = B.make_desc([("relu", {})], [(8, 8)], "per_op")
+    d.ops[0].kind = 99
+    assert not B.ago_subgraph_create(d) and B.ago_last_error()[0] == B.AGO_ERR_INVALID_ARG
+    d, _ = B.make_desc([("relu", {})], [(8, 8)], "per_op")
+    d.mode = 7
+    assert not B.ago_subgraph_create(d) and B.ago_last_error()[0] == B.AGO_ERR_INVALID_ARG
+
+
+def test_null_and_misaligned_arguments_are_rejected_before_any_cuda_call():
+    wl = WL.get("mbv2_14")
+    sg = B.Subgraph(wl.ops, wl.input_shapes, mode="per_op")
+    lib = B.load()
+    assert lib.ago_subgraph_run(None, None, None, None, None) == B.AGO_ERR_INVALID_ARG
+    assert lib.ago_subgraph_run(sg._h, None, None, None, None) == B.AGO_ERR_INVALID_ARG
+    good = [0x1000] * 8
+    assert B.ago_subgraph_run(sg._h, [0], good, good) == B.AGO_ERR_INVALID_ARG
+    assert B.ago_subgraph_run(sg._h, [0x1004], good, good) == B.AGO_ERR_ALIGNMENT
+    assert B.ago_subgraph_run(sg._h, good, [0x1000, 0x1008] + good, good) == B.AGO_ERR_ALIGNMENT
+    assert B.ago_subgraph_set_workspace(sg._h, 0x1010, 1 << 30) == B.AGO_ERR_ALIGNMENT
+    assert B.ago_subgraph_set_workspace(sg._h, 0x1000, 16) == B.AGO_ERR_WORKSPACE
+    assert B.ago_subgraph_workspace_bytes(None) == 0
+    B.ago_subgraph_destroy(None)
+    sg.close()
+
+
+def test_bf16_helpers_round_to_nearest_even():
+    x = np.array([1.0, 1.00390625, 1.001953125, 1.005859375, -2.5, 3.0e38], dtype=np.float32)
+    r = WL.bf16_round(x)
+    # 1 + 2^-8 is a tie between 1 and 1 + 2^-7 -> even (1.0); 1 + 3*2^-9 rounds up to 1 + 2^-7
+    assert r[0] == 1.0 and r[1] == 1.0 and r[2] == 1.0 and r[3] == np.float32(1.0078125) and r[4] == -2.5
+    import torch
+    t = torch.from_numpy(x).to(torch.bfloat16).float().numpy()
+    assert np.array_equal(r, t)

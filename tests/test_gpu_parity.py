@@ -1,0 +1,85 @@
+"""Parity of the CUDA path (through the C-ABI) against the fp64 CPU oracle on
+the same seeded inputs. Tolerance (bf16 in, fp32 accumulate):
+max|gpu - ref| <= 1e-2 * max|ref| + 1e-3 over the whole output tensor; the
+fp32-I/O depthwise check uses 1e-5 * max|ref|."""
+import numpy as np
+import pytest
+
+from oracle import oracle as O
+from paper_2212_01005_b200 import workloads as WL
+from helpers import assert_close, run_gpu
+
+pytestmark = pytest.mark.gpu
+
+UNFUSED = ["per_op", "per_mini_subgraph"]
+
+
+def small_workloads():
+    """Small instances of every chain family: several tiles plus ragged tails."""
+    return {
+        "mbv2_14": WL.get("mbv2_14"),
+        "mbv2_s1_odd": WL.mbv2_block("mbv2_s1_odd", [21], 3, 13, 24, 144, 24, 1, True),
+        "mbv2_s2": WL.mbv2_block("mbv2_s2", [22], 2, 14, 32, 192, 64, 2, False),
+        "mbv2_s2_odd": WL.mbv2_block("mbv2_s2_odd", [23], 2, 9, 16, 96, 32, 2, False),
+        "ffn_small": WL.ffn("ffn_small", [24], 200, 128, 512, 1),
+        "ffn_ragged": WL.ffn("ffn_ragged", [25], 77, 96, 264, 1),
+        "resnet_small": WL.resnet_block("resnet_small", [26], 2, 12, 64),
+        "resnet_odd": WL.resnet_block("resnet_odd", [27], 1, 9, 32),
+        "attn_small": WL.attention("attn_small", [28], 2, 128, 2, 64),
+        "attn_ragged": WL.attention("attn_ragged", [29], 1, 200, 3, 64),
+    }
+
+
+_ref_cache = {}
+
+
+def reference(name, wl, data):
+    if name not in _ref_cache:
+        _ref_cache[name] = O.run_chain(wl.ops, data["inputs"], data["weights"])
+    return _ref_cache[name]
+
+
+@pytest.mark.parametrize("mode", UNFUSED)
+@pytest.mark.parametrize("name", list(small_workloads().keys()))
+def test_unfused_modes_match_oracle(ago, name, mode):
+    wl = small_workloads()[name]
+    data = WL.generate(wl)
+    ref = reference(name, wl, data)
+    gpu = run_gpu(ago, wl, data, mode)
+    assert_close(gpu, ref, what=f"{name}/{mode}")
+
+
+def test_depthwise_fp32_io_matches_oracle_to_1e5(ago):
+    # the 14x14x192 depthwise stage of the N=1 block, fp32 in / fp32 out, fused and per-op
+    wl = WL.Workload("dw14", [0, 99], [(1, 14, 14, 192)],
+                     [("conv2d", dict(O=192, R=3, S=3, stride=1, pad=1, groups=192)), ("bias_add", {}), ("relu6", {})],
+                     samples=1, input_dist=["uniform"])
+    rng = np.random.default_rng([0, 99])
+    data = {"inputs": [rng.uniform(0, 6, size=(1, 14, 14, 192)).astype(np.float32)],
+            "weights": [(rng.standard_normal((3, 3, 192)) * np.sqrt(2 / 9)).astype(np.float32),
+                        rng.uniform(-0.1, 0.1, 192).astype(np.float32)]}
+    ref = O.run_chain(wl.ops, data["inputs"], data["weights"])
+    for mode in ("fused", "per_op", "per_mini_subgraph"):
+        gpu = run_gpu(ago, wl, data, mode, fp32=True)
+        err = np.max(np.abs(gpu - ref))
+        assert err <= 1e-5 * np.max(np.abs(ref)), (mode, err)
+
+
+@pytest.mark.parametrize("stride", [1, 2])
+def test_depthwise_bf16_fused_mini_subgraph(ago, stride):
+    wl = WL.Workload("dwb", [31, stride], [(2, 11, 13, 48)],
+                     [("conv2d", dict(O=48, R=3, S=3, stride=stride, pad=1, groups=48)), ("bias_add", {}), ("relu6", {})],
+                     samples=2, input_dist=["uniform"])
+    data = WL.generate(wl)
+    ref = O.run_chain(wl.ops, data["inputs"], data["weights"])
+    assert_close(run_gpu(ago, wl, data, "fused"), ref, what="dw fused")
+
+
+def test_padding_of_the_intermediate_with_large_bias(ago):
+    # the halo of the depthwise / second conv input is zero, not act(bias)
+    wl = WL.mbv2_block("pad", [33], 1, 6, 8, 16, 8, 1, True)
+    data = WL.generate(wl)
+    data["weights"][1] = np.full(16, 3.0, dtype=np.float32)      # expand bias: ReLU6(b1) = 3 in the halo if mishandled
+    ref = O.run_chain(wl.ops, data["inputs"], data["weights"])
+    for mode in UNFUSED:
+        assert_close(run_gpu(ago, wl, data, mode), ref, what=f"pad/{mode}")
