@@ -88,7 +88,7 @@ class ClockSampler(threading.Thread):
     def __init__(self, index):
         super().__init__(daemon=True)
         self.index, self.samples, self.reasons, self.max_mhz = index, [], set(), None
-        self._stop = threading.Event()
+        self._halt = threading.Event()
         self.ok = False
         try:
             import pynvml
@@ -110,7 +110,7 @@ class ClockSampler(threading.Thread):
             getattr(nv, "nvmlClocksEventReasonSwThermalSlowdown", 0x20): "sw_thermal_slowdown",
             getattr(nv, "nvmlClocksEventReasonSwPowerCap", 0x4): "sw_power_cap",
         }
-        while not self._stop.is_set():
+        while not self._halt.is_set():
             try:
                 self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
                 try:
@@ -125,7 +125,7 @@ class ClockSampler(threading.Thread):
             time.sleep(0.002)
 
     def finish(self):
-        self._stop.set()
+        self._halt.set()
         if self.is_alive():
             self.join(timeout=2)
         if not self.ok or not self.samples:
@@ -135,8 +135,9 @@ class ClockSampler(threading.Thread):
 
 
 def cpu_baseline(wl, name, budget_s=12.0):
-    """The oracle as it stands, timed on this host's cores on a bounded sample
-    (a few independent samples of the same workload)."""
+    """The oracle as it stands, timed on this host's cores on a bounded sample:
+    whole launches' worth of samples (or fewer when one launch takes longer than
+    the budget), repeated until about `budget_s` seconds of CPU work are done."""
     from oracle import oracle
     per = WL.get(name, batch=1)
     d = WL.generate(per)
@@ -144,16 +145,17 @@ def cpu_baseline(wl, name, budget_s=12.0):
     oracle.run_chain(per.ops, d["inputs"], d["weights"])
     t1 = time.perf_counter() - t0
     n = max(1, min(wl.samples, int(budget_s / max(t1, 1e-4))))
-    if n > 1 and t1 < budget_s / 2:
-        big = WL.get(name, batch=n)
-        d = WL.generate(big)
-        t0 = time.perf_counter()
+    big = WL.get(name, batch=n)
+    d = WL.generate(big)
+    calls, t0 = 0, time.perf_counter()
+    while True:
         oracle.run_chain(big.ops, d["inputs"], d["weights"])
+        calls += 1
         t = time.perf_counter() - t0
-    else:
-        n, t = 1, t1
-    return {"value": n / t, "unit": "samples/s", "cores": oracle.threads(), "kind": "oracle",
-            "sample": f"{n} of {wl.samples} samples of {name} per launch, one oracle.run_chain call, {t:.2f} s wall"}
+        if t >= budget_s or calls >= 10000:
+            break
+    return {"value": n * calls / t, "unit": "samples/s", "cores": oracle.threads(), "kind": "oracle",
+            "sample": f"{calls} oracle.run_chain call(s) on {n} of the {wl.samples} samples of one {name} launch, {t:.2f} s wall"}
 
 
 def run_reference(args):

@@ -41,10 +41,22 @@ bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) ==
 
 size_t align256(size_t b) { return (b + 255) & ~size_t(255); }
 
+// Storage of tensors passed between launches: fp32 in PER_OP mode (every
+// operator materialises its full-precision result, as the unfused loop nest of
+// Section III-A does), the I/O dtype in PER_MINI_SUBGRAPH mode.
+int intermediate_dtype(const Plan& p) { return p.mode == AGO_MODE_PER_OP ? AGO_FP32 : p.dtype; }
+
+size_t unfused_workspace(const Plan& p) {
+  if (p.stages.size() <= 1) return 0;
+  const size_t elems = (size_t)(p.max_intermediate_bytes / elem_bytes(p.dtype));
+  bool softmax = false;
+  for (const Stage& s : p.stages) softmax = softmax || s.softmax;
+  return 2 * align256(elems * (size_t)(softmax ? 4 : elem_bytes(intermediate_dtype(p))));
+}
+
 size_t needed_workspace(const Plan& p) {
   if (p.mode == AGO_MODE_FUSED) return fused_workspace_bytes(p);
-  if (p.stages.size() <= 1) return 0;
-  return 2 * align256((size_t)p.max_intermediate_bytes);
+  return unfused_workspace(p);
 }
 
 // Translate ops [first, last] (all element-wise) into an epilogue program.
@@ -68,9 +80,9 @@ void make_epilogue(const Plan& p, int first, int last, const void* const* inputs
   }
 }
 
-cudaError_t launch_complex(const Plan& p, const OpInfo& o, const void* src, void* dst, const void* const* inputs,
-                           const void* const* weights, const EpiProgram& epi, bool tuned_depthwise,
-                           cudaStream_t stream) {
+cudaError_t launch_complex(const Plan& p, const OpInfo& o, const void* src, int src_dtype, void* dst, int dst_dtype,
+                           const void* const* inputs, const void* const* weights, const EpiProgram& epi,
+                           bool tuned_depthwise, cudaStream_t stream) {
   const int32_t* q = o.op.p;
   if (o.op.kind == AGO_OP_CONV2D && o.depthwise()) {
     DepthwiseArgs a{};
@@ -78,12 +90,13 @@ cudaError_t launch_complex(const Plan& p, const OpInfo& o, const void* src, void
     a.N = (int)o.in.d[0]; a.H = (int)o.in.d[1]; a.W = (int)o.in.d[2]; a.C = (int)o.in.d[3];
     a.R = q[1]; a.S = q[2]; a.stride = q[3]; a.pad = q[4];
     a.Ho = (int)o.out.d[1]; a.Wo = (int)o.out.d[2];
-    a.dtype = p.dtype;
+    a.dtype = p.dtype; a.in_dtype = src_dtype; a.out_dtype = dst_dtype;
     a.epi = epi;
     return tuned_depthwise ? launch_depthwise_fused(a, stream) : launch_depthwise_generic(a, stream);
   }
   GemmArgs g{};
   g.A = src; g.C = dst; g.epi = epi;
+  g.a_dtype = src_dtype; g.c_dtype = dst_dtype;
   g.batches = 1; g.heads = 1;
   switch (o.op.kind) {
     case AGO_OP_CONV2D: {
@@ -145,31 +158,39 @@ cudaError_t launch_complex(const Plan& p, const OpInfo& o, const void* src, void
 ago_status_t run_unfused(ago_subgraph_s* h, const void* const* inputs, const void* const* weights, void* out,
                          void* ws, size_t ws_bytes, cudaStream_t stream) {
   const Plan& p = h->plan;
-  const size_t need = p.stages.size() <= 1 ? 0 : 2 * align256((size_t)p.max_intermediate_bytes);
+  const size_t need = unfused_workspace(p);
+  const int mid = intermediate_dtype(p);
   if (need > 0 && (ws == nullptr || ws_bytes < need))
     return fail(AGO_ERR_WORKSPACE, "workspace missing or smaller than ago_subgraph_workspace_bytes()");
   char* buf[2] = {static_cast<char*>(ws), static_cast<char*>(ws) + need / 2};
   const void* src = inputs[0];
+  int src_dtype = p.dtype;
   int flip = 0;
   for (size_t si = 0; si < p.stages.size(); ++si) {
     const Stage& s = p.stages[si];
-    void* dst = (si + 1 == p.stages.size()) ? out : static_cast<void*>(buf[flip]);
+    const bool last = si + 1 == p.stages.size();
+    void* dst = last ? out : static_cast<void*>(buf[flip]);
+    // The tensor a row softmax reads stays fp32 in every mode: scores rounded to
+    // bf16 before the exponential alone exceed the parity tolerance.
+    const bool feeds_softmax = !last && p.stages[si + 1].softmax;
+    const int dst_dtype = last ? p.dtype : (feeds_softmax ? AGO_FP32 : mid);
     cudaError_t e;
     if (s.softmax) {
       const Shape& sh = p.ops[s.first].in;
-      e = launch_softmax_rows(src, dst, sh.numel() / sh.last(), (int)sh.last(), p.dtype, stream);
+      e = launch_softmax_rows(src, dst, sh.numel() / sh.last(), (int)sh.last(), src_dtype, dst_dtype, stream);
     } else if (s.complex_index >= 0) {
       EpiProgram epi;
       make_epilogue(p, s.first + 1, s.last, inputs, weights, &epi);
-      e = launch_complex(p, p.ops[s.first], src, dst, inputs, weights, epi, false, stream);
+      e = launch_complex(p, p.ops[s.first], src, src_dtype, dst, dst_dtype, inputs, weights, epi, false, stream);
     } else {
       EpiProgram epi;
       make_epilogue(p, s.first, s.last, inputs, weights, &epi);
       const Shape& sh = p.ops[s.first].in;
-      e = launch_elementwise(src, dst, sh.numel(), (int)sh.last(), p.dtype, epi, stream);
+      e = launch_elementwise(src, dst, sh.numel(), (int)sh.last(), p.dtype, src_dtype, dst_dtype, epi, stream);
     }
     if (e != cudaSuccess) return cuda_fail(e, "kernel launch");
     src = dst;
+    src_dtype = dst_dtype;
     flip ^= 1;
   }
   return AGO_OK;
@@ -265,7 +286,7 @@ ago_status_t ago_subgraph_run(ago_subgraph_t h, const void* const* inputs, const
     EpiProgram epi;
     make_epilogue(p, 1, (int)p.ops.size() - 1, inputs, weights, &epi);
     if (epi.n != (int)p.ops.size() - 1 || epi.n > kMaxEpi) return fail(AGO_ERR_UNSUPPORTED, "too many simple operators");
-    cudaError_t e = launch_complex(p, p.ops[0], inputs[0], outputs[0], inputs, weights, epi, true, stream);
+    cudaError_t e = launch_complex(p, p.ops[0], inputs[0], p.dtype, outputs[0], p.dtype, inputs, weights, epi, true, stream);
     if (e != cudaSuccess) return cuda_fail(e, "depthwise kernel launch");
     return AGO_OK;
   }

@@ -24,6 +24,7 @@ struct GemmArgs {
   // batch = blockIdx.z = b * heads + h
   int batches, heads;
   int64_t a_sb, a_sh, b_sb, b_sh, c_sb, c_sh;
+  int a_dtype, c_dtype;  // AGO_BF16 | AGO_FP32 storage of A and C (B and EPI_ADD operands are bf16)
   EpiProgram epi;
 };
 cudaError_t launch_gemm_generic(const GemmArgs& a, cudaStream_t stream);
@@ -31,16 +32,20 @@ cudaError_t launch_gemm_generic(const GemmArgs& a, cudaStream_t stream);
 struct DepthwiseArgs {
   const void* in; const void* w; void* out;
   int N, H, W, C, R, S, stride, pad, Ho, Wo;
-  int dtype;  // AGO_BF16 | AGO_FP32 (activations and weights)
+  int dtype;      // AGO_BF16 | AGO_FP32: the subgraph's I/O dtype = dtype of weights and EPI_ADD operands
+  int in_dtype;   // storage of `in`  (an fp32 intermediate in per-op mode, else == dtype)
+  int out_dtype;  // storage of `out`
   EpiProgram epi;
 };
 cudaError_t launch_depthwise_generic(const DepthwiseArgs& a, cudaStream_t stream);
 
 // y = program(x) element-wise over a [rows][C] view.
-cudaError_t launch_elementwise(const void* x, void* y, int64_t numel, int C, int dtype, const EpiProgram& epi,
-                               cudaStream_t stream);
+// `dtype` is the subgraph's I/O dtype (EPI_ADD operands); x and y may be fp32 intermediates.
+cudaError_t launch_elementwise(const void* x, void* y, int64_t numel, int C, int dtype, int x_dtype, int y_dtype,
+                               const EpiProgram& epi, cudaStream_t stream);
 // Row softmax over the last dimension, fp32 math.
-cudaError_t launch_softmax_rows(const void* x, void* y, int64_t rows, int cols, int dtype, cudaStream_t stream);
+cudaError_t launch_softmax_rows(const void* x, void* y, int64_t rows, int cols, int x_dtype, int y_dtype,
+                                cudaStream_t stream);
 
 // ---- fused kernels -------------------------------------------------------------
 

@@ -16,25 +16,19 @@ __device__ __forceinline__ float gelu_tanh_f(float v) {
   return 0.5f * v * (1.0f + tanhf(c * (v + 0.044715f * v * v * v)));
 }
 
-template <typename T> __device__ __forceinline__ float ld(const void* p, int64_t i);
-template <> __device__ __forceinline__ float ld<__nv_bfloat16>(const void* p, int64_t i) {
-  return __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(p)[i]);
+// Storage type is a run-time flag (AGO_BF16 | AGO_FP32), uniform over the grid.
+__device__ __forceinline__ float ld(const void* p, int64_t i, int dtype) {
+  return dtype == AGO_FP32 ? reinterpret_cast<const float*>(p)[i]
+                           : __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(p)[i]);
 }
-template <> __device__ __forceinline__ float ld<float>(const void* p, int64_t i) {
-  return reinterpret_cast<const float*>(p)[i];
-}
-template <typename T> __device__ __forceinline__ void st(void* p, int64_t i, float v);
-template <> __device__ __forceinline__ void st<__nv_bfloat16>(void* p, int64_t i, float v) {
-  reinterpret_cast<__nv_bfloat16*>(p)[i] = __float2bfloat16_rn(v);
-}
-template <> __device__ __forceinline__ void st<float>(void* p, int64_t i, float v) {
-  reinterpret_cast<float*>(p)[i] = v;
+__device__ __forceinline__ void st(void* p, int64_t i, float v, int dtype) {
+  if (dtype == AGO_FP32) reinterpret_cast<float*>(p)[i] = v;
+  else reinterpret_cast<__nv_bfloat16*>(p)[i] = __float2bfloat16_rn(v);
 }
 
 // The simple operators, applied in program order to one element. `c` is the
 // index along the last dimension, `idx` the element's linear index.
-template <typename T>
-__device__ __forceinline__ float run_epilogue(const EpiProgram& e, float v, int c, int64_t idx) {
+__device__ __forceinline__ float run_epilogue(const EpiProgram& e, float v, int c, int64_t idx, int add_dtype) {
   for (int i = 0; i < e.n; ++i) {
     switch (e.code[i]) {
       case EPI_BIAS: v += reinterpret_cast<const float*>(e.ptr[i])[c]; break;
@@ -42,7 +36,7 @@ __device__ __forceinline__ float run_epilogue(const EpiProgram& e, float v, int 
       case EPI_RELU6: v = fminf(fmaxf(v, 0.0f), 6.0f); break;
       case EPI_GELU: v = gelu_tanh_f(v); break;
       case EPI_SCALE: v *= e.f[i]; break;
-      case EPI_ADD: v += ld<T>(e.ptr[i], idx); break;
+      case EPI_ADD: v += ld(e.ptr[i], idx, add_dtype); break;
     }
   }
   return v;
@@ -55,7 +49,7 @@ __global__ void __launch_bounds__(256) gemm_generic_kernel(const GemmArgs a) {
   __shared__ float Bs[TK][TN + 4];
   const int batch = blockIdx.z;
   const int bb = batch / a.heads, hh = batch % a.heads;
-  const __nv_bfloat16* A = reinterpret_cast<const __nv_bfloat16*>(a.A) + bb * a.a_sb + hh * a.a_sh;
+  const int64_t a_off = bb * a.a_sb + hh * a.a_sh;
   const __nv_bfloat16* B = reinterpret_cast<const __nv_bfloat16*>(a.B) + bb * a.b_sb + hh * a.b_sh;
   const int64_t c_off = bb * a.c_sb + hh * a.c_sh;
   const int m0 = blockIdx.x * TM, n0 = blockIdx.y * TN;
@@ -72,7 +66,7 @@ __global__ void __launch_bounds__(256) gemm_generic_kernel(const GemmArgs a) {
       float v = 0.0f;
       if (m < a.M && k < a.K) {
         if (!a.a_im2col) {
-          v = __bfloat162float(A[(int64_t)m * a.lda + k]);
+          v = ld(a.A, a_off + (int64_t)m * a.lda + k, a.a_dtype);
         } else {
           const int ci = k % a.Cin;
           const int rs = k / a.Cin;
@@ -82,9 +76,11 @@ __global__ void __launch_bounds__(256) gemm_generic_kernel(const GemmArgs a) {
           const int ho = t % a.Ho, img = t / a.Ho;
           const int h = ho * a.stride + r - a.pad, w = wo * a.stride + s - a.pad;
           if (h >= 0 && h < a.H && w >= 0 && w < a.W)
-            v = __bfloat162float(A[(((int64_t)img * a.H + h) * a.W + w) * a.Cin + ci]);
+            v = ld(a.A, a_off + (((int64_t)img * a.H + h) * a.W + w) * a.Cin + ci, a.a_dtype);
         }
       }
+      // operands of a contraction are bf16 values: an fp32 intermediate is rounded as it is loaded
+      if (a.a_dtype == AGO_FP32) v = __bfloat162float(__float2bfloat16_rn(v));
       As[kk][row] = v;
     }
 #pragma unroll
@@ -122,13 +118,11 @@ __global__ void __launch_bounds__(256) gemm_generic_kernel(const GemmArgs a) {
       const int n = n0 + tx * 4 + j;
       if (n >= a.N) continue;
       const int64_t idx = c_off + (int64_t)m * a.ldc + n;
-      float v = run_epilogue<__nv_bfloat16>(a.epi, acc[i][j], n, idx);
-      reinterpret_cast<__nv_bfloat16*>(a.C)[idx] = __float2bfloat16_rn(v);
+      st(a.C, idx, run_epilogue(a.epi, acc[i][j], n, idx, AGO_BF16), a.c_dtype);
     }
   }
 }
 
-template <typename T>
 __global__ void __launch_bounds__(256) depthwise_generic_kernel(const DepthwiseArgs a, int64_t total) {
   const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (idx >= total) return;
@@ -144,35 +138,38 @@ __global__ void __launch_bounds__(256) depthwise_generic_kernel(const DepthwiseA
     for (int s = 0; s < a.S; ++s) {
       const int w = wo * a.stride + s - a.pad;
       if (w < 0 || w >= a.W) continue;
-      acc = fmaf(ld<T>(a.in, ((n * a.H + h) * a.W + w) * a.C + c), ld<T>(a.w, (r * a.S + s) * a.C + c), acc);
+      {
+        float x = ld(a.in, ((n * a.H + h) * a.W + w) * a.C + c, a.in_dtype);
+        if (a.in_dtype != a.dtype) x = __bfloat162float(__float2bfloat16_rn(x));
+        acc = fmaf(x, ld(a.w, (r * a.S + s) * a.C + c, a.dtype), acc);
+      }
     }
   }
-  st<T>(a.out, idx, run_epilogue<T>(a.epi, acc, c, idx));
+  st(a.out, idx, run_epilogue(a.epi, acc, c, idx, a.dtype), a.out_dtype);
 }
 
-template <typename T>
-__global__ void __launch_bounds__(256) elementwise_kernel(const void* x, void* y, int64_t numel, int C,
-                                                          const EpiProgram epi) {
+__global__ void __launch_bounds__(256) elementwise_kernel(const void* x, void* y, int64_t numel, int C, int dtype,
+                                                          int x_dtype, int y_dtype, const EpiProgram epi) {
   const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (idx >= numel) return;
-  st<T>(y, idx, run_epilogue<T>(epi, ld<T>(x, idx), (int)(idx % C), idx));
+  st(y, idx, run_epilogue(epi, ld(x, idx, x_dtype), (int)(idx % C), idx, dtype), y_dtype);
 }
 
 // One warp per row: p_j = exp(s_j - max) / sum.
-template <typename T>
-__global__ void __launch_bounds__(256) softmax_rows_kernel(const void* x, void* y, int64_t rows, int cols) {
+__global__ void __launch_bounds__(256) softmax_rows_kernel(const void* x, void* y, int64_t rows, int cols,
+                                                           int x_dtype, int y_dtype) {
   const int64_t row = (int64_t)blockIdx.x * (blockDim.x / 32) + threadIdx.x / 32;
   if (row >= rows) return;
   const int lane = threadIdx.x % 32;
   const int64_t base = row * cols;
   float m = -INFINITY;
-  for (int j = lane; j < cols; j += 32) m = fmaxf(m, ld<T>(x, base + j));
+  for (int j = lane; j < cols; j += 32) m = fmaxf(m, ld(x, base + j, x_dtype));
   for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
   float sum = 0.0f;
-  for (int j = lane; j < cols; j += 32) sum += expf(ld<T>(x, base + j) - m);
+  for (int j = lane; j < cols; j += 32) sum += expf(ld(x, base + j, x_dtype) - m);
   for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
   const float inv = 1.0f / sum;
-  for (int j = lane; j < cols; j += 32) st<T>(y, base + j, expf(ld<T>(x, base + j) - m) * inv);
+  for (int j = lane; j < cols; j += 32) st(y, base + j, expf(ld(x, base + j, x_dtype) - m) * inv, y_dtype);
 }
 
 }  // namespace
@@ -186,29 +183,21 @@ cudaError_t launch_gemm_generic(const GemmArgs& a, cudaStream_t stream) {
 cudaError_t launch_depthwise_generic(const DepthwiseArgs& a, cudaStream_t stream) {
   const int64_t total = (int64_t)a.N * a.Ho * a.Wo * a.C;
   const unsigned blocks = (unsigned)((total + 255) / 256);
-  if (a.dtype == AGO_FP32)
-    depthwise_generic_kernel<float><<<blocks, 256, 0, stream>>>(a, total);
-  else
-    depthwise_generic_kernel<__nv_bfloat16><<<blocks, 256, 0, stream>>>(a, total);
+  depthwise_generic_kernel<<<blocks, 256, 0, stream>>>(a, total);
   return cudaGetLastError();
 }
 
-cudaError_t launch_elementwise(const void* x, void* y, int64_t numel, int C, int dtype, const EpiProgram& epi,
-                               cudaStream_t stream) {
+cudaError_t launch_elementwise(const void* x, void* y, int64_t numel, int C, int dtype, int x_dtype, int y_dtype,
+                               const EpiProgram& epi, cudaStream_t stream) {
   const unsigned blocks = (unsigned)((numel + 255) / 256);
-  if (dtype == AGO_FP32)
-    elementwise_kernel<float><<<blocks, 256, 0, stream>>>(x, y, numel, C, epi);
-  else
-    elementwise_kernel<__nv_bfloat16><<<blocks, 256, 0, stream>>>(x, y, numel, C, epi);
+  elementwise_kernel<<<blocks, 256, 0, stream>>>(x, y, numel, C, dtype, x_dtype, y_dtype, epi);
   return cudaGetLastError();
 }
 
-cudaError_t launch_softmax_rows(const void* x, void* y, int64_t rows, int cols, int dtype, cudaStream_t stream) {
+cudaError_t launch_softmax_rows(const void* x, void* y, int64_t rows, int cols, int x_dtype, int y_dtype,
+                                cudaStream_t stream) {
   const unsigned blocks = (unsigned)((rows + 7) / 8);
-  if (dtype == AGO_FP32)
-    softmax_rows_kernel<float><<<blocks, 256, 0, stream>>>(x, y, rows, cols);
-  else
-    softmax_rows_kernel<__nv_bfloat16><<<blocks, 256, 0, stream>>>(x, y, rows, cols);
+  softmax_rows_kernel<<<blocks, 256, 0, stream>>>(x, y, rows, cols, x_dtype, y_dtype);
   return cudaGetLastError();
 }
 
