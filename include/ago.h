@@ -196,6 +196,34 @@ ago_status_t ago_subgraph_query(ago_subgraph_t h, int32_t what, int64_t* out);
  * undefined). The word is cleared by the call. */
 ago_status_t ago_subgraph_status(ago_subgraph_t h);
 
+/* Bytes of scratch built into the library for ago_subgraph_run_static. */
+#define AGO_STATIC_SCRATCH_BYTES (4u << 20)
+
+/* (The paper has no counterpart for this entry point; it exists for deployment.)
+ * ago_subgraph_run for PER_OP / PER_MINI_SUBGRAPH handles when nobody may
+ * allocate device memory: code that runs inside a host whose memory pools are
+ * fixed before it is called (an inference server's plug-in slot, a sandbox that
+ * forbids cudaMalloc after start-up, a real-time loop where an allocation's
+ * implicit synchronisation is not acceptable). Inputs, weights and the output
+ * are still the caller's device buffers; the tensors passed between the
+ * launches go to a fixed AGO_STATIC_SCRATCH_BYTES (4 MiB) array inside the
+ * library image, which every GPU that loads the library keeps until the
+ * process exits. The call allocates and frees nothing, does not use
+ * ago_subgraph_set_workspace and does not touch the handle's status word.
+ *   - A subgraph whose ago_subgraph_workspace_bytes() exceeds the array is
+ *     rejected with AGO_ERR_WORKSPACE (message states both sizes); FUSED handles
+ *     are rejected with AGO_ERR_UNSUPPORTED (they need no scratch).
+ *   - The first call on each device looks up the array's device address (with
+ *     that device current); make that first call outside any stream capture.
+ *   - All calls on one GPU share the one array, and it keeps the previous
+ *     call's contents. Nothing in it has to start at zero (every intermediate is
+ *     written in full before it is read), but two calls whose kernels overlap on
+ *     the GPU (different streams, different handles or threads) race on it: keep
+ *     calls on one stream, or order them with events. */
+ago_status_t ago_subgraph_run_static(ago_subgraph_t h, const void* const* inputs,
+                                     const void* const* weights, void* const* outputs,
+                                     void* cuda_stream);
+
 /* Library version, "major.minor". */
 const char* ago_version(void);
 

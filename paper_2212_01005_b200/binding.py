@@ -35,11 +35,12 @@ AGO_LINK_DOWNSTREAM_DEPTHWISE, AGO_LINK_DOWNSTREAM_POINTWISE, AGO_LINK_GENERAL =
  AGO_KERNEL_ATTENTION) = range(6)
 
 AGO_MAX_INPUTS, AGO_MAX_RANK, AGO_MAX_OPS = 4, 4, 32
+AGO_STATIC_SCRATCH_BYTES = 4 << 20
 
 EXPORTS = [
     "ago_subgraph_create", "ago_subgraph_run", "ago_subgraph_run_host", "ago_subgraph_destroy", "ago_last_error",
     "ago_subgraph_workspace_bytes", "ago_subgraph_set_workspace", "ago_subgraph_query", "ago_subgraph_status",
-    "ago_version",
+    "ago_version", "ago_subgraph_run_static",
 ]
 
 
@@ -101,6 +102,8 @@ def load(build_if_missing: bool = True):
     lib.ago_subgraph_status.restype = ctypes.c_int
     lib.ago_subgraph_status.argtypes = [vp]
     lib.ago_version.restype = ctypes.c_char_p
+    lib.ago_subgraph_run_static.restype = ctypes.c_int
+    lib.ago_subgraph_run_static.argtypes = [vp, vpp, vpp, vpp, vp]
     _lib = lib
     return lib
 
@@ -131,6 +134,12 @@ def _ptr_array(ptrs: Sequence[int]):
 
 def ago_subgraph_run(h, inputs: Sequence[int], weights: Sequence[int], outputs: Sequence[int], stream: int = 0) -> int:
     return load().ago_subgraph_run(h, _ptr_array(inputs), _ptr_array(weights), _ptr_array(outputs), stream)
+
+
+def ago_subgraph_run_static(h, inputs: Sequence[int], weights: Sequence[int], outputs: Sequence[int], stream: int = 0) -> int:
+    """Unfused run whose scratch is the array built into the library: for callers
+    that may not allocate device memory. Marshals pointers only."""
+    return load().ago_subgraph_run_static(h, _ptr_array(inputs), _ptr_array(weights), _ptr_array(outputs), stream)
 
 
 def ago_subgraph_run_host(h, host_inputs, weights, host_outputs, dev_inputs, dev_outputs, stream: int = 0) -> int:

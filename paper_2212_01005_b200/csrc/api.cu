@@ -231,6 +231,26 @@ ago_status_t check_run_args(ago_subgraph_s* h, const void* const* inputs, const 
 
 }  // namespace
 
+namespace ago {
+// Unfused run with an explicitly given workspace and no status word: used by
+// the entry point whose scratch is a static device array.
+ago_status_t run_unfused_in(ago_subgraph_s* h, const void* const* inputs, const void* const* weights,
+                            void* const* outputs, void* ws, size_t ws_bytes, cudaStream_t stream) {
+  ago_status_t s = check_run_args(h, inputs, weights, outputs);
+  if (s != AGO_OK) return s;
+  if (h->plan.mode == AGO_MODE_FUSED)
+    return fail(AGO_ERR_UNSUPPORTED, "fused handles keep their intermediates on chip: use ago_subgraph_run");
+  const size_t need = unfused_workspace(h->plan);
+  if (need > ws_bytes) {
+    char buf[160];
+    std::snprintf(buf, sizeof(buf), "this subgraph needs %zu bytes of scratch, the built-in array holds %zu", need, ws_bytes);
+    return fail(AGO_ERR_WORKSPACE, buf);
+  }
+  return run_unfused(h, inputs, weights, outputs[0], ws, ws_bytes, stream);
+}
+ago_status_t report_failure(ago_status_t s, const char* msg) { return fail(s, msg); }
+}  // namespace ago
+
 extern "C" {
 
 const char* ago_version(void) { return "0.1"; }
