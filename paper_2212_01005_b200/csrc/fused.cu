@@ -3,10 +3,23 @@
 
 namespace ago {
 
+cudaError_t ensure_max_dynamic_smem(const void* func, int* done_flags) {
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+  if (done_flags[dev]) return cudaSuccess;
+  e = cudaFuncSetAttribute(func, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+  if (e == cudaSuccess) done_flags[dev] = 1;
+  return e;
+}
+
 ago_status_t fused_plan(Plan* plan, FusedState* st, std::string* err) {
   switch (plan->fused_kernel) {
     case AGO_KERNEL_DEPTHWISE:
       return AGO_OK;
+    case AGO_KERNEL_MBV2_BLOCK:
+      return mbv2_plan(plan, st, err);
     default:
       *err = "fused mode: no kernel is built for this family yet";
       return AGO_ERR_UNSUPPORTED;
@@ -15,10 +28,16 @@ ago_status_t fused_plan(Plan* plan, FusedState* st, std::string* err) {
 
 size_t fused_workspace_bytes(const Plan&) { return 0; }
 
-ago_status_t fused_run(const Plan& plan, FusedState*, const void* const*, const void* const*, void*, void*,
-                       unsigned int*, cudaStream_t, std::string* err) {
-  *err = "fused mode: no kernel is built for this family yet";
-  return AGO_ERR_UNSUPPORTED;
+ago_status_t fused_run(const Plan& plan, FusedState* st, const void* const* inputs, const void* const* weights,
+                       void* output, void* workspace, unsigned int* status_word, cudaStream_t stream,
+                       std::string* err) {
+  switch (plan.fused_kernel) {
+    case AGO_KERNEL_MBV2_BLOCK:
+      return mbv2_run(plan, st, inputs, weights, output, status_word, stream, err);
+    default:
+      *err = "fused mode: no kernel is built for this family yet";
+      return AGO_ERR_UNSUPPORTED;
+  }
 }
 
 }  // namespace ago

@@ -13,8 +13,18 @@ struct FusedState {
   int tile_rows = 0;       // downstream tile extent along the tiled dimension
   int grid = 0;            // CTAs
   int smem_bytes = 0;      // dynamic shared memory per CTA
-  bool attr_set = false;   // cudaFuncSetAttribute done for this process/device
+  void* impl = nullptr;                  // kernel-family host state (parameters, tensor-map cache)
+  void (*impl_free)(void*) = nullptr;
+  ~FusedState() { if (impl && impl_free) impl_free(impl); }
 };
+
+// Opt-in to the full 227 KB of dynamic shared memory for `func`, once per device.
+cudaError_t ensure_max_dynamic_smem(const void* func, int* done_flags);
+
+// Kernel families (each in its own file).
+ago_status_t mbv2_plan(Plan* plan, FusedState* st, std::string* err);
+ago_status_t mbv2_run(const Plan& plan, FusedState* st, const void* const* inputs, const void* const* weights,
+                      void* output, unsigned int* status_word, cudaStream_t stream, std::string* err);
 
 // Chooses tiles and shared-memory budget for plan->fused_kernel; fills
 // plan->tile_rows / smem_bytes. Host only.

@@ -83,3 +83,63 @@ def test_padding_of_the_intermediate_with_large_bias(ago):
     ref = O.run_chain(wl.ops, data["inputs"], data["weights"])
     for mode in UNFUSED:
         assert_close(run_gpu(ago, wl, data, mode), ref, what=f"pad/{mode}")
+
+
+# ---- fused kernels -------------------------------------------------------------------
+
+FUSED_SMALL = ["mbv2_14", "mbv2_s1_odd", "mbv2_s2", "mbv2_s2_odd"]
+
+
+@pytest.mark.parametrize("name", FUSED_SMALL)
+def test_fused_matches_oracle(ago, name):
+    wl = small_workloads()[name]
+    data = WL.generate(wl)
+    ref = reference(name, wl, data)
+    gpu = run_gpu(ago, wl, data, "fused")
+    assert_close(gpu, ref, what=f"{name}/fused")
+
+
+@pytest.mark.parametrize("name", FUSED_SMALL)
+def test_fused_agrees_with_unfused_chain(ago, name):
+    # fusion is a loop transformation: same result as the library's own unfused chain, up to bf16 rounding
+    wl = small_workloads()[name]
+    data = WL.generate(wl)
+    fused = run_gpu(ago, wl, data, "fused")
+    mini = run_gpu(ago, wl, data, "per_mini_subgraph")
+    scale = float(np.max(np.abs(mini)))
+    assert float(np.max(np.abs(fused - mini))) <= 2e-2 * scale + 1e-3
+
+
+def test_fused_mbv2_pads_the_intermediate_not_the_input(ago):
+    wl = WL.mbv2_block("pad", [33], 1, 6, 8, 16, 8, 1, True)
+    data = WL.generate(wl)
+    data["weights"][1] = np.full(16, 3.0, dtype=np.float32)
+    ref = O.run_chain(wl.ops, data["inputs"], data["weights"])
+    assert_close(run_gpu(ago, wl, data, "fused"), ref, what="pad/fused")
+
+
+@pytest.mark.parametrize("shape", [
+    dict(N=2, H=7, c_in=16, c_exp=32, c_out=16, stride=1, residual=True),     # 32-byte input rows (Cin 16)
+    dict(N=1, H=20, c_in=64, c_exp=64, c_out=40, stride=1, residual=False),   # 128-byte input rows, Cout not a multiple of 16
+    dict(N=3, H=5, c_in=8, c_exp=16, c_out=8, stride=2, residual=False),      # one chunk, tiny image, odd size
+    dict(N=1, H=30, c_in=40, c_exp=240, c_out=80, stride=2, residual=False),  # Cin padded 40 -> 64
+])
+def test_fused_mbv2_shape_sweep(ago, shape):
+    wl = WL.mbv2_block("sweep", [41, shape["H"], shape["c_in"]], shape["N"], shape["H"], shape["c_in"], shape["c_exp"],
+                       shape["c_out"], shape["stride"], shape["residual"])
+    data = WL.generate(wl)
+    ref = O.run_chain(wl.ops, data["inputs"], data["weights"])
+    assert_close(run_gpu(ago, wl, data, "fused"), ref, what=f"sweep {shape}")
+
+
+@pytest.mark.parametrize("name", ["mbv2_56", "mbv2_28s2"])
+def test_fused_full_size_on_sampled_images(ago, name):
+    # the benchmark's launch configuration; the oracle checks whole images picked from the batch
+    # (images are independent samples, so each is a complete sub-problem)
+    wl = WL.get(name)
+    data = WL.generate(wl)
+    gpu = run_gpu(ago, wl, data, "fused")
+    for img in (0, 17, wl.samples - 1):
+        one = WL.get(name, batch=1)
+        ref = O.run_chain(one.ops, [data["inputs"][0][img:img + 1]], data["weights"])
+        assert_close(gpu[img:img + 1], ref, what=f"{name} image {img}")
