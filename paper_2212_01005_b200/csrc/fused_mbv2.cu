@@ -24,6 +24,7 @@
 #include <cuda.h>
 #include <cuda_bf16.h>
 
+#include <cstdlib>
 #include <unordered_map>
 
 #include "fused.h"
@@ -36,7 +37,10 @@ namespace {
 
 using namespace tc;
 
-constexpr int kThreads = 256;
+constexpr int kComputeWarps = 28;                  // expand epilogue, depthwise, project epilogue
+constexpr int kComputeThreads = kComputeWarps * 32;
+constexpr int kIssuers = 4;                        // one MMA-issuing warp per SM sub-partition
+constexpr int kThreads = kComputeThreads + 32 * kIssuers;
 constexpr int kChunk = 16;      // expanded channels per chunk = one MMA K step of the project GEMM
 constexpr int kChunkRowBytes = 32;
 
@@ -55,11 +59,80 @@ struct Mbv2Params {
   int Kp, row_bytes, swizzle;   // input / W1 tiles: padded K, bytes per row, tc::SwizzleMode
   int Coutp, NC;
   int tmem_cols, ecol0, pcol0;
+  int e_plane, d_plane;         // byte distance between the two 8-channel planes of an E / D chunk
   // shared-memory byte offsets (from the 1024-aligned base)
   int off_x, off_w1, off_e, off_d, off_w3, off_wd, off_b1, off_bd, off_b3, off_bar;
 };
 
-__device__ __forceinline__ float relu6f(float v) { return fminf(fmaxf(v, 0.0f), 6.0f); }
+__device__ __forceinline__ uint32_t relu6_pack(float a, float b) {
+  __nv_bfloat162 h = __floats2bfloat162_rn(a, b);
+  h = __hmin2(__hmax2(h, __floats2bfloat162_rn(0.0f, 0.0f)), __floats2bfloat162_rn(6.0f, 6.0f));
+  return *reinterpret_cast<const uint32_t*>(&h);
+}
+__device__ __forceinline__ float2 bf16x2_to_f2(uint32_t w) { return make_float2(bf16_lo(w), bf16_hi(w)); }
+#ifdef AGO_SCALAR_FMA
+__device__ __forceinline__ float2 fma2(float2 a, float2 b, float2 c) { return make_float2(fmaf(a.x, b.x, c.x), fmaf(a.y, b.y, c.y)); }
+#else
+__device__ __forceinline__ float2 fma2(float2 a, float2 b, float2 c) { return __ffma2_rn(a, b, c); }
+#endif
+
+// Depthwise 3x3 over the resident E chunk for one (channel pair, output column)
+// and output rows [r0, r1): E and D chunks are two planes of [pixel][8 channels]
+// (16 bytes per pixel), which is also the un-swizzled K-major operand layout.
+__device__ __forceinline__ uint32_t lds32(uint32_t saddr) {
+  uint32_t v;
+  asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(saddr));
+  return v;
+}
+__device__ __forceinline__ void sts32(uint32_t saddr, uint32_t v) {
+  asm volatile("st.shared.u32 [%0], %1;" ::"r"(saddr), "r"(v) : "memory");
+}
+
+// Depthwise 3x3 over the resident E chunk for one (channel pair, output column)
+// and output rows [r0, r1): E and D chunks are two planes of [pixel][8 channels]
+// (16 bytes per pixel), which is also the un-swizzled K-major operand layout.
+// e_col / d_col are 32-bit shared-memory addresses.
+template <int STRIDE>
+__device__ __forceinline__ void depthwise_column(uint32_t e_col, uint32_t d_col, int r0, int r1, int IW, int Wo,
+                                                 const float2 (&w)[9], float2 bias) {
+  const uint32_t e_pitch = (uint32_t)IW * 16u, d_pitch = (uint32_t)Wo * 16u;
+  if (STRIDE == 1) {
+    // walk down the input rows once; each row feeds the three output rows it overlaps
+    float2 a0 = bias, a1 = bias, a2 = bias;   // output rows i, i-1, i-2
+    uint32_t src = e_col + (uint32_t)r0 * e_pitch;
+    uint32_t dst = d_col + (uint32_t)r0 * d_pitch;
+    // the first two input rows complete no output
+#pragma unroll
+    for (int pre = 0; pre < 2; ++pre) {
+      const float2 x0 = bf16x2_to_f2(lds32(src)), x1 = bf16x2_to_f2(lds32(src + 16)), x2 = bf16x2_to_f2(lds32(src + 32));
+      src += e_pitch;
+      a0 = fma2(x0, w[0], a0); a0 = fma2(x1, w[1], a0); a0 = fma2(x2, w[2], a0);
+      a1 = fma2(x0, w[3], a1); a1 = fma2(x1, w[4], a1); a1 = fma2(x2, w[5], a1);
+      a2 = a1; a1 = a0; a0 = bias;
+    }
+    for (int i = r0; i < r1; ++i) {   // input row i + 2 completes output row i
+      const float2 x0 = bf16x2_to_f2(lds32(src)), x1 = bf16x2_to_f2(lds32(src + 16)), x2 = bf16x2_to_f2(lds32(src + 32));
+      src += e_pitch;
+      a2 = fma2(x0, w[6], a2); a2 = fma2(x1, w[7], a2); a2 = fma2(x2, w[8], a2);
+      sts32(dst, relu6_pack(a2.x, a2.y));
+      dst += d_pitch;
+      a1 = fma2(x0, w[3], a1); a1 = fma2(x1, w[4], a1); a1 = fma2(x2, w[5], a1);
+      a0 = fma2(x0, w[0], a0); a0 = fma2(x1, w[1], a0); a0 = fma2(x2, w[2], a0);
+      a2 = a1; a1 = a0; a0 = bias;
+    }
+  } else {
+    for (int r = r0; r < r1; ++r) {
+      float2 a = bias;
+      const uint32_t src = e_col + (uint32_t)(r * STRIDE) * e_pitch;
+#pragma unroll
+      for (int kr = 0; kr < 3; ++kr)
+#pragma unroll
+        for (int ks = 0; ks < 3; ++ks)
+          a = fma2(bf16x2_to_f2(lds32(src + (uint32_t)kr * e_pitch + (uint32_t)ks * 16u)), w[kr * 3 + ks], a);
+      sts32(d_col + (uint32_t)r * d_pitch, relu6_pack(a.x, a.y));
+    }
+  }
+}
 
 __global__ void __launch_bounds__(kThreads, 1)
 mbv2_fused_kernel(const __grid_constant__ CUtensorMap tmap_x, const Mbv2Params p) {
@@ -75,227 +148,267 @@ mbv2_fused_kernel(const __grid_constant__ CUtensorMap tmap_x, const Mbv2Params p
   float* sBd = reinterpret_cast<float*>(smem + p.off_bd);
   float* sB3 = reinterpret_cast<float*>(smem + p.off_b3);
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + p.off_bar);
-  uint64_t* bar_x = bars + 0;
-  uint64_t* bar_e = bars + 1;  // [2]
-  uint64_t* bar_d = bars + 3;  // [2]
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 5);
-  volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(bars + 6);
+  uint64_t* bar_x = bars + 0;       // input strip landed (TMA)
+  uint64_t* bar_w = bars + 1;       // weights staged by the compute warps
+  uint64_t* bar_e = bars + 2;       // [2] expand accumulators of buffer b complete (MMA commit)
+  uint64_t* bar_d = bars + 4;       // [2] project MMA has consumed D[b] (MMA commit)
+  uint64_t* bar_tfree = bars + 6;   // [2] expand buffer b drained and E chunk written (compute -> issuer)
+  uint64_t* bar_dready = bars + 8;  // [2] D[b] written (compute -> issuer)
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 10);
+  volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(bars + 11);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+#ifdef AGO_TIMELINE
+  long long* ts = reinterpret_cast<long long*>(p.out) + (tid == 0 ? 0 : 512); int tsi = 0;
+  const bool tsw = blockIdx.x == 0 && (tid == 0 || tid == kComputeThreads);
+#define TS() do { if (tsw) ts[tsi++] = clock64(); } while (0)
+#else
+#define TS() do {} while (0)
+#endif
+  TS();
   const int n = blockIdx.x / p.strips, strip = blockIdx.x % p.strips;
   const int ho0 = strip * p.R;
   const int rows_valid = min(p.R, p.Ho - ho0);
   const int gh0 = ho0 * p.stride - 1;   // image row of tile row 0
-  const int d_bytes = p.M2 * 128 * kChunkRowBytes;
+  const int d_bytes = 2 * p.d_plane;
 
-  if (tid == 0) {
+  if (tid == kComputeThreads) {
+    // first issuer lane: barriers, then the input strip's TMA right away
     *abort_flag = 0u;
     mbar_init(bar_x, 1);
-    mbar_init(bar_e + 0, 1);
-    mbar_init(bar_e + 1, 1);
-    mbar_init(bar_d + 0, 1);
-    mbar_init(bar_d + 1, 1);
+    mbar_init(bar_w, 1);
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(bar_e + i, kIssuers);
+      mbar_init(bar_d + i, kIssuers);
+      mbar_init(bar_tfree + i, 1);
+      mbar_init(bar_dready + i, 1);
+    }
     fence_mbar_init();
     fence_proxy_async_smem();
     tma_prefetch_desc(&tmap_x);
+    mbar_arrive_expect_tx(bar_x, (uint32_t)(p.P_in * p.row_bytes));
+    tma_load_4d(sX, &tmap_x, bar_x, 0, -1, gh0, n);
   }
   if (warp == 0) {
     tmem_alloc(tmem_slot, (uint32_t)p.tmem_cols);
     tmem_relinquish();
   }
-  __syncthreads();
-  if (tid == 0) {
-    mbar_arrive_expect_tx(bar_x, (uint32_t)(p.P_in * p.row_bytes));
-    tma_load_4d(sX, &tmap_x, bar_x, 0, -1, gh0, n);
-  }
-
-  // ---- stage weights and biases (generic proxy), in the operand layouts the MMAs read ----
-  {
-    const int chunks_per_row = p.row_bytes >> 4;
-    for (int i = tid; i < p.Cexp * chunks_per_row; i += kThreads) {
-      const int row = i / chunks_per_row, ch = i % chunks_per_row;
-      uint4 v = make_uint4(0, 0, 0, 0);
-      if (ch * 8 < p.Cin) v = __ldg(reinterpret_cast<const uint4*>(p.w1 + (size_t)row * p.Cin + ch * 8));
-      *reinterpret_cast<uint4*>(sW1 + swz_offset(row, ch, p.row_bytes)) = v;
-    }
-    for (int i = tid; i < p.NC * p.Coutp * 2; i += kThreads) {
-      const int half = i & 1, row = (i >> 1) % p.Coutp, c = (i >> 1) / p.Coutp;
-      uint4 v = make_uint4(0, 0, 0, 0);
-      if (row < p.Cout) v = __ldg(reinterpret_cast<const uint4*>(p.w3 + (size_t)row * p.Cexp + c * kChunk + half * 8));
-      *reinterpret_cast<uint4*>(sW3 + c * p.Coutp * kChunkRowBytes + swz_offset(row, half, kChunkRowBytes)) = v;
-    }
-    for (int i = tid; i < 9 * p.Cexp; i += kThreads) sWd[i] = __bfloat162float(p.wd[i]);
-    for (int i = tid; i < p.Cexp; i += kThreads) { sB1[i] = p.b1[i]; sBd[i] = p.bd[i]; }
-    for (int i = tid; i < p.Coutp; i += kThreads) sB3[i] = i < p.Cout ? p.b3[i] : 0.0f;
-  }
-  fence_proxy_async_smem();
   tcgen05_fence_before_sync();
   __syncthreads();
   tcgen05_fence_after_sync();
   const uint32_t tmem_base = *tmem_slot;
-  const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
 
-  // Which of this thread's expand-tile rows are real in-image pixels (bit k: tile (warp>>2) + 2k).
-  uint32_t inimg_mask = 0;
-  for (int t = warp >> 2, k = 0; t < p.M1; t += 2, ++k) {
-    const int pix = t * 128 + (warp & 3) * 32 + lane;
-    const int ih = pix / p.IW, iw = pix % p.IW;
-    const int gh = gh0 + ih;
-    if (pix < p.P_in && gh >= 0 && gh < p.H && iw >= 1 && iw <= p.W) inimg_mask |= 1u << k;
-  }
+  if (warp >= kComputeWarps) {
+    // ================= MMA issue warps: issuer i owns M tiles i, i+4, ... (one lane each) =================
+    const int iw = warp - kComputeWarps;
+    if (lane == 0) {
+      const uint32_t idesc_e = make_idesc_bf16(128, kChunk);
+      const uint32_t idesc_p = make_idesc_bf16(128, (uint32_t)p.Coutp);
+      const uint32_t sbo_x = 8u * (uint32_t)p.row_bytes;
+      const uint64_t xdesc0 = make_smem_desc(smem_u32(sX), 0, sbo_x, p.swizzle);
+      const uint64_t w1desc0 = make_smem_desc(smem_u32(sW1), 0, sbo_x, p.swizzle);
+      // D: un-swizzled K-major; the two 8-channel planes are the two K core-matrix columns
+      const uint64_t ddesc0 = make_smem_desc(smem_u32(sD), (uint32_t)p.d_plane, 128, SW_NONE);
+      const uint64_t w3desc0 = make_smem_desc(smem_u32(sW3), 0, 256, SW_32B);
+      const int ksteps = p.Kp / 16;
+      const uint32_t a_tile_step = (uint32_t)(128 * p.row_bytes) >> 4;
 
-  mbar_wait(bar_x, 0, abort_flag, p.status, 0x101);
+      auto issue_expand = [&](int c) {
+        const int b = c & 1;
+        const uint64_t bdesc = w1desc0 + (uint64_t)((c * kChunk * p.row_bytes) >> 4);
+        for (int t = iw; t < p.M1; t += kIssuers) {
+          const uint64_t adesc = xdesc0 + (uint64_t)t * a_tile_step;
+          const uint32_t d_tmem = tmem_base + p.ecol0 + (b * p.M1 + t) * kChunk;
+          umma_bf16(d_tmem, adesc, bdesc, idesc_e, 0);
+          for (int ks = 1; ks < ksteps; ++ks) umma_bf16(d_tmem, adesc + 2u * ks, bdesc + 2u * ks, idesc_e, 1);
+        }
+        umma_commit(bar_e + b);
+      };
 
-  const uint32_t idesc_e = make_idesc_bf16(128, kChunk);
-  const uint32_t idesc_p = make_idesc_bf16(128, (uint32_t)p.Coutp);
-  const uint32_t sbo_x = 8u * (uint32_t)p.row_bytes;
-  const uint32_t x_addr = smem_u32(sX), w1_addr = smem_u32(sW1), d_addr = smem_u32(sD), w3_addr = smem_u32(sW3);
-
-  auto issue_expand = [&](int c) {
-    const int b = c & 1;
-    for (int t = 0; t < p.M1; ++t) {
-      for (int ks = 0; ks < p.Kp / 16; ++ks) {
-        const uint64_t ad = make_smem_desc(x_addr + t * 128 * p.row_bytes + ks * 32, 0, sbo_x, p.swizzle);
-        const uint64_t bd = make_smem_desc(w1_addr + c * kChunk * p.row_bytes + ks * 32, 0, sbo_x, p.swizzle);
-        umma_bf16(tmem_base + p.ecol0 + (b * p.M1 + t) * kChunk, ad, bd, idesc_e, ks > 0);
-      }
-    }
-    umma_commit(bar_e + b);
-  };
-
-  if (tid == 0) issue_expand(0);
-
-  for (int c = 0; c < p.NC; ++c) {
-    const int b = c & 1;
-    if (tid == 0 && c + 1 < p.NC) {
+      TS();
+      mbar_wait(bar_w, 0, abort_flag, p.status, 0x100);
+      TS();
+      mbar_wait(bar_x, 0, abort_flag, p.status, 0x101);
+      TS();
       tcgen05_fence_after_sync();
-      issue_expand(c + 1);
-    }
-    mbar_wait(bar_e + b, (c >> 1) & 1, abort_flag, p.status, 0x102);
-    tcgen05_fence_after_sync();
-
-    // ---- P3: expand epilogue -> E chunk [pixel][16 ch] bf16, 32-byte rows, swizzled ----
-    for (int t = warp >> 2, k = 0; t < p.M1; t += 2, ++k) {
-      uint32_t acc[16];
-      tmem_ld_x16(tmem_base + lane_base + p.ecol0 + (b * p.M1 + t) * kChunk, acc);
-      tmem_ld_wait();
-      const int pix = t * 128 + (warp & 3) * 32 + lane;
-      if (pix < p.P_in) {
-        uint32_t w[8];
-        if ((inimg_mask >> k) & 1u) {
-          const float4* bb = reinterpret_cast<const float4*>(sB1 + c * kChunk);
-#pragma unroll
-          for (int j = 0; j < 4; ++j) {
-            const float4 bv = bb[j];
-            w[2 * j] = pack_bf16x2(relu6f(__uint_as_float(acc[4 * j]) + bv.x), relu6f(__uint_as_float(acc[4 * j + 1]) + bv.y));
-            w[2 * j + 1] = pack_bf16x2(relu6f(__uint_as_float(acc[4 * j + 2]) + bv.z), relu6f(__uint_as_float(acc[4 * j + 3]) + bv.w));
-          }
-        } else {
-#pragma unroll
-          for (int j = 0; j < 8; ++j) w[j] = 0u;
+      issue_expand(0);
+      if (p.NC > 1) issue_expand(1);
+      TS();
+      for (int c = 0; c < p.NC; ++c) {
+        const int b = c & 1;
+        const uint32_t ph = (uint32_t)(c >> 1) & 1u;
+        if (c + 2 < p.NC) {
+          mbar_wait(bar_tfree + b, ph, abort_flag, p.status, 0x105);
+          TS();
+          tcgen05_fence_after_sync();
+          issue_expand(c + 2);
+          TS();
         }
-        const uint32_t flip = (pix >> 2) & 1u;
-        uint8_t* row = sE + pix * kChunkRowBytes;
-        *reinterpret_cast<uint4*>(row + ((0u ^ flip) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
-        *reinterpret_cast<uint4*>(row + ((1u ^ flip) << 4)) = make_uint4(w[4], w[5], w[6], w[7]);
+        mbar_wait(bar_dready + b, ph, abort_flag, p.status, 0x106);
+        TS();
+        tcgen05_fence_after_sync();
+        const uint64_t bdesc = w3desc0 + (uint64_t)((c * p.Coutp * kChunkRowBytes) >> 4);
+        for (int t = iw; t < p.M2; t += kIssuers)
+          umma_bf16(tmem_base + p.pcol0 + t * p.Coutp, ddesc0 + (uint64_t)((b * d_bytes + t * 128 * 16) >> 4), bdesc,
+                    idesc_p, c > 0);
+        umma_commit(bar_d + b);
+        TS();
       }
     }
-    tcgen05_fence_before_sync();
-    __syncthreads();
-
-    // D[b] was read by the project MMA of chunk c-2
-    if (c >= 2) mbar_wait(bar_d + b, ((c - 2) >> 1) & 1, abort_flag, p.status, 0x103);
-
-    // ---- P4: depthwise 3x3 + bias + ReLU6 on CUDA cores: E chunk -> D[b] (A operand of the project GEMM) ----
+    __syncwarp();
+  } else {
+    // ================================== compute warps ==================================
+    const int ctid = tid;   // compute warps are warps 0 .. kComputeWarps-1
+    // ---- stage weights and biases (generic proxy), in the operand layouts the MMAs read ----
     {
-      uint8_t* dD = sD + b * d_bytes;
-      const int cg = tid & 1;                      // which 8 of the chunk's 16 channels
-      const int cbase = c * kChunk + cg * 8;
-      float wgt[9][8];
-#pragma unroll
-      for (int tap = 0; tap < 9; ++tap) {
-        const float4 a = *reinterpret_cast<const float4*>(sWd + tap * p.Cexp + cbase);
-        const float4 bq = *reinterpret_cast<const float4*>(sWd + tap * p.Cexp + cbase + 4);
-        wgt[tap][0] = a.x; wgt[tap][1] = a.y; wgt[tap][2] = a.z; wgt[tap][3] = a.w;
-        wgt[tap][4] = bq.x; wgt[tap][5] = bq.y; wgt[tap][6] = bq.z; wgt[tap][7] = bq.w;
+      const int chunks_per_row = p.row_bytes >> 4;
+      for (int i = ctid; i < p.Cexp * chunks_per_row; i += kComputeThreads) {
+        const int row = i / chunks_per_row, ch = i % chunks_per_row;
+        uint4 v = make_uint4(0, 0, 0, 0);
+        if (ch * 8 < p.Cin) v = __ldg(reinterpret_cast<const uint4*>(p.w1 + (size_t)row * p.Cin + ch * 8));
+        *reinterpret_cast<uint4*>(sW1 + swz_offset(row, ch, p.row_bytes)) = v;
       }
-      float bias[8];
-      {
-        const float4 a = *reinterpret_cast<const float4*>(sBd + cbase);
-        const float4 bq = *reinterpret_cast<const float4*>(sBd + cbase + 4);
-        bias[0] = a.x; bias[1] = a.y; bias[2] = a.z; bias[3] = a.w;
-        bias[4] = bq.x; bias[5] = bq.y; bias[6] = bq.z; bias[7] = bq.w;
+      for (int i = ctid; i < p.NC * p.Coutp * 2; i += kComputeThreads) {
+        const int half = i & 1, row = (i >> 1) % p.Coutp, c = (i >> 1) / p.Coutp;
+        uint4 v = make_uint4(0, 0, 0, 0);
+        if (row < p.Cout) v = __ldg(reinterpret_cast<const uint4*>(p.w3 + (size_t)row * p.Cexp + c * kChunk + half * 8));
+        *reinterpret_cast<uint4*>(sW3 + c * p.Coutp * kChunkRowBytes + swz_offset(row, half, kChunkRowBytes)) = v;
       }
-      const int nitems = 2 * p.Wo * rows_valid;
-      for (int item = tid; item < nitems; item += kThreads) {
-        const int rest = item >> 1;
-        const int wo = rest % p.Wo, r = rest / p.Wo;
-        float acc[8];
-#pragma unroll
-        for (int j = 0; j < 8; ++j) acc[j] = bias[j];
-#pragma unroll
-        for (int kr = 0; kr < 3; ++kr) {
-#pragma unroll
-          for (int ks = 0; ks < 3; ++ks) {
-            const int pe = (r * p.stride + kr) * p.IW + wo * p.stride + ks;
-            const uint4 v = *reinterpret_cast<const uint4*>(sE + pe * kChunkRowBytes + ((cg ^ ((pe >> 2) & 1)) << 4));
-            const float* wv = wgt[kr * 3 + ks];
-            acc[0] = fmaf(bf16_lo(v.x), wv[0], acc[0]); acc[1] = fmaf(bf16_hi(v.x), wv[1], acc[1]);
-            acc[2] = fmaf(bf16_lo(v.y), wv[2], acc[2]); acc[3] = fmaf(bf16_hi(v.y), wv[3], acc[3]);
-            acc[4] = fmaf(bf16_lo(v.z), wv[4], acc[4]); acc[5] = fmaf(bf16_hi(v.z), wv[5], acc[5]);
-            acc[6] = fmaf(bf16_lo(v.w), wv[6], acc[6]); acc[7] = fmaf(bf16_hi(v.w), wv[7], acc[7]);
-          }
-        }
-        const int po = r * p.Wo + wo;
-        const uint4 o = make_uint4(pack_bf16x2(relu6f(acc[0]), relu6f(acc[1])), pack_bf16x2(relu6f(acc[2]), relu6f(acc[3])),
-                                   pack_bf16x2(relu6f(acc[4]), relu6f(acc[5])), pack_bf16x2(relu6f(acc[6]), relu6f(acc[7])));
-        *reinterpret_cast<uint4*>(dD + po * kChunkRowBytes + ((cg ^ ((po >> 2) & 1)) << 4)) = o;
-      }
+      for (int i = ctid; i < 9 * p.Cexp; i += kComputeThreads) sWd[i] = __bfloat162float(p.wd[i]);
+      for (int i = ctid; i < p.Cexp; i += kComputeThreads) { sB1[i] = p.b1[i]; sBd[i] = p.bd[i]; }
+      for (int i = ctid; i < p.Coutp; i += kComputeThreads) sB3[i] = i < p.Cout ? p.b3[i] : 0.0f;
     }
     fence_proxy_async_smem();
-    __syncthreads();
+    named_barrier_sync(1, kComputeThreads);
+    if (ctid == 0) mbar_arrive(bar_w);
+    TS();
 
-    // ---- P5: project GEMM accumulates this chunk ----
-    if (tid == 0) {
-      tcgen05_fence_after_sync();
-      for (int t = 0; t < p.M2; ++t) {
-        const uint64_t ad = make_smem_desc(d_addr + b * d_bytes + t * 128 * kChunkRowBytes, 0, 256, SW_32B);
-        const uint64_t bd = make_smem_desc(w3_addr + c * p.Coutp * kChunkRowBytes, 0, 256, SW_32B);
-        umma_bf16(tmem_base + p.pcol0 + t * p.Coutp, ad, bd, idesc_p, c > 0);
+    const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
+    // Depthwise work split: thread = (channel pair, slot); a slot walks one output column of one row group.
+    constexpr int kSlots = kComputeThreads / 8;
+    const int cp = ctid & 7, slot = ctid >> 3;
+    const int groups = max(1, min(rows_valid, kSlots / max(1, min(p.Wo, kSlots))));
+    const int rows_per_group = (rows_valid + groups - 1) / groups;
+    const int dw_items = p.Wo * groups;
+    const int cp_off = (cp & 3) * 4;   // byte offset inside a 16-byte pixel entry
+    // first depthwise item of this slot (most shapes have at most one per slot)
+    const int item0_g = slot / p.Wo, item0_wo = slot - item0_g * p.Wo;
+    // expand-epilogue rows of this thread: tile (warp>>2) + 7k; bit k of the masks: row exists / is an in-image pixel
+    uint32_t e_exist = 0, e_inimg = 0;
+    for (int t = warp >> 2, k = 0; t < p.M1; t += kComputeWarps / 4, ++k) {
+      const int pix = t * 128 + (warp & 3) * 32 + lane;
+      const int ih = pix / p.IW, iw = pix - ih * p.IW;
+      const int gh = gh0 + ih;
+      if (pix < p.P_in) {
+        e_exist |= 1u << k;
+        if (gh >= 0 && gh < p.H && iw >= 1 && iw <= p.W) e_inimg |= 1u << k;
       }
-      umma_commit(bar_d + b);
     }
-  }
 
-  // ---- P6: project epilogue: + b3 (+ residual), bf16, 16-byte stores ----
-  {
-    const int last = p.NC - 1;
-    mbar_wait(bar_d + (last & 1), (last >> 1) & 1, abort_flag, p.status, 0x104);
-    tcgen05_fence_after_sync();
-    const int valid_pix = rows_valid * p.Wo;
-    const size_t gpix0 = ((size_t)n * p.Ho + ho0) * p.Wo;
-    for (int t = warp >> 2; t < p.M2; t += 2) {
-      const int po = t * 128 + (warp & 3) * 32 + lane;
-      for (int j0 = 0; j0 < p.Coutp; j0 += 16) {
+    for (int c = 0; c < p.NC; ++c) {
+      const int b = c & 1;
+      TS();
+      mbar_wait(bar_e + b, (uint32_t)(c >> 1) & 1u, abort_flag, p.status, 0x102);
+      tcgen05_fence_after_sync();
+      TS();
+
+      // ---- P3: expand epilogue -> E chunk: + b1, ReLU6, zero outside the image, bf16 ----
+      for (int t = warp >> 2, k = 0; t < p.M1; t += kComputeWarps / 4, ++k) {
         uint32_t acc[16];
-        tmem_ld_x16(tmem_base + lane_base + p.pcol0 + t * p.Coutp + j0, acc);
+        tmem_ld_x16(tmem_base + lane_base + p.ecol0 + (b * p.M1 + t) * kChunk, acc);
         tmem_ld_wait();
-        if (po < valid_pix) {
+        const int pix = t * 128 + (warp & 3) * 32 + lane;
+        if ((e_exist >> k) & 1u) {
+          uint32_t w[8];
+          if ((e_inimg >> k) & 1u) {
+            const float4* bb = reinterpret_cast<const float4*>(sB1 + c * kChunk);
 #pragma unroll
-          for (int h = 0; h < 2; ++h) {
-            const int j = j0 + h * 8;
-            if (j < p.Cout) {
-              float v[8];
+            for (int j = 0; j < 4; ++j) {
+              const float4 bv = bb[j];
+              w[2 * j] = relu6_pack(__uint_as_float(acc[4 * j]) + bv.x, __uint_as_float(acc[4 * j + 1]) + bv.y);
+              w[2 * j + 1] = relu6_pack(__uint_as_float(acc[4 * j + 2]) + bv.z, __uint_as_float(acc[4 * j + 3]) + bv.w);
+            }
+          } else {
 #pragma unroll
-              for (int q = 0; q < 8; ++q) v[q] = __uint_as_float(acc[h * 8 + q]) + sB3[j + q];
-              const size_t off = (gpix0 + po) * p.Cout + j;
-              if (p.residual) {
-                const uint4 xr = __ldg(reinterpret_cast<const uint4*>(p.x + off));
-                v[0] += bf16_lo(xr.x); v[1] += bf16_hi(xr.x); v[2] += bf16_lo(xr.y); v[3] += bf16_hi(xr.y);
-                v[4] += bf16_lo(xr.z); v[5] += bf16_hi(xr.z); v[6] += bf16_lo(xr.w); v[7] += bf16_hi(xr.w);
+            for (int j = 0; j < 8; ++j) w[j] = 0u;
+          }
+          *reinterpret_cast<uint4*>(sE + pix * 16) = make_uint4(w[0], w[1], w[2], w[3]);
+          *reinterpret_cast<uint4*>(sE + p.e_plane + pix * 16) = make_uint4(w[4], w[5], w[6], w[7]);
+        }
+      }
+      tcgen05_fence_before_sync();
+      named_barrier_sync(1, kComputeThreads);
+      if (ctid == 0) mbar_arrive(bar_tfree + b);
+      TS();
+
+      // D[b] was read by the project MMA of chunk c-2
+      if (c >= 2) mbar_wait(bar_d + b, (uint32_t)((c - 2) >> 1) & 1u, abort_flag, p.status, 0x103);
+      TS();
+
+      // ---- P4: depthwise 3x3 + bias + ReLU6 on CUDA cores: E chunk -> D[b] (A operand of the project GEMM) ----
+      {
+        const int ch = c * kChunk + cp * 2;
+        float2 wgt[9];
+#pragma unroll
+        for (int tap = 0; tap < 9; ++tap) wgt[tap] = *reinterpret_cast<const float2*>(sWd + tap * p.Cexp + ch);
+        const float2 bias = *reinterpret_cast<const float2*>(sBd + ch);
+        const uint32_t e_plane = smem_u32(sE) + (uint32_t)((cp >> 2) * p.e_plane + cp_off);
+        const uint32_t d_plane = smem_u32(sD) + (uint32_t)(b * d_bytes + (cp >> 2) * p.d_plane + cp_off);
+#ifdef AGO_DW_NOITEMS
+        for (int item = slot; item < 0; item += kSlots) {
+#else
+        for (int item = slot; item < dw_items; item += kSlots) {
+#endif
+          int g = item0_g, wo = item0_wo;
+          if (item != slot) { g = item / p.Wo; wo = item - g * p.Wo; }
+          const int r0 = g * rows_per_group, r1 = min(rows_valid, r0 + rows_per_group);
+          if (p.stride == 1)
+            depthwise_column<1>(e_plane + wo * 16, d_plane + wo * 16, r0, r1, p.IW, p.Wo, wgt, bias);
+          else
+            depthwise_column<2>(e_plane + wo * 32, d_plane + wo * 16, r0, r1, p.IW, p.Wo, wgt, bias);
+        }
+      }
+#ifndef AGO_DW_NOFENCE
+      fence_proxy_async_smem();
+#endif
+      named_barrier_sync(1, kComputeThreads);
+      if (ctid == 0) mbar_arrive(bar_dready + b);
+      TS();
+    }
+
+    // ---- P6: project epilogue: + b3 (+ residual), bf16, 16-byte stores ----
+    {
+      const int last = p.NC - 1;
+      mbar_wait(bar_d + (last & 1), (uint32_t)(last >> 1) & 1u, abort_flag, p.status, 0x104);
+      tcgen05_fence_after_sync();
+      const int valid_pix = rows_valid * p.Wo;
+      const size_t gpix0 = ((size_t)n * p.Ho + ho0) * p.Wo;
+#ifdef AGO_TIMELINE
+      if (blockIdx.x != 0)
+#endif
+      for (int t = warp >> 2; t < p.M2; t += kComputeWarps / 4) {
+        const int po = t * 128 + (warp & 3) * 32 + lane;
+        for (int j0 = 0; j0 < p.Coutp; j0 += 16) {
+          uint32_t acc[16];
+          tmem_ld_x16(tmem_base + lane_base + p.pcol0 + t * p.Coutp + j0, acc);
+          tmem_ld_wait();
+          if (po < valid_pix) {
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+              const int j = j0 + h * 8;
+              if (j < p.Cout) {
+                float v[8];
+#pragma unroll
+                for (int q = 0; q < 8; ++q) v[q] = __uint_as_float(acc[h * 8 + q]) + sB3[j + q];
+                const size_t off = (gpix0 + po) * p.Cout + j;
+                if (p.residual) {
+                  const uint4 xr = __ldg(reinterpret_cast<const uint4*>(p.x + off));
+                  v[0] += bf16_lo(xr.x); v[1] += bf16_hi(xr.x); v[2] += bf16_lo(xr.y); v[3] += bf16_hi(xr.y);
+                  v[4] += bf16_lo(xr.z); v[5] += bf16_hi(xr.z); v[6] += bf16_lo(xr.w); v[7] += bf16_hi(xr.w);
+                }
+                *reinterpret_cast<uint4*>(p.out + off) =
+                    make_uint4(pack_bf16x2(v[0], v[1]), pack_bf16x2(v[2], v[3]), pack_bf16x2(v[4], v[5]), pack_bf16x2(v[6], v[7]));
               }
-              *reinterpret_cast<uint4*>(p.out + off) =
-                  make_uint4(pack_bf16x2(v[0], v[1]), pack_bf16x2(v[2], v[3]), pack_bf16x2(v[4], v[5]), pack_bf16x2(v[6], v[7]));
             }
           }
         }
@@ -334,14 +447,18 @@ bool layout(Mbv2Params& q, int R, int* smem_bytes) {
   auto take = [&](int bytes) { int o = off; off = round_up(off + bytes, 1024); return o; };
   q.off_x = take(q.M1 * 128 * q.row_bytes);
   q.off_w1 = take(q.Cexp * q.row_bytes);
-  q.off_e = take(q.P_in * kChunkRowBytes);
-  q.off_d = take(2 * q.M2 * 128 * kChunkRowBytes);
+  // two 8-channel planes per chunk, offset by 64 mod 128 bytes so that a warp's
+  // 2 x 64-byte accesses (4 pixels x 4 channel pairs per plane) never share a bank
+  q.e_plane = round_up(q.P_in * 16, 128) + 64;
+  q.d_plane = q.M2 * 128 * 16 + 64;
+  q.off_e = take(2 * q.e_plane);
+  q.off_d = take(2 * 2 * q.d_plane);
   q.off_w3 = take(q.NC * q.Coutp * kChunkRowBytes);
   q.off_wd = take(9 * q.Cexp * 4);
   q.off_b1 = take(q.Cexp * 4);
   q.off_bd = take(q.Cexp * 4);
   q.off_b3 = take(q.Coutp * 4);
-  q.off_bar = take(64);
+  q.off_bar = take(128);
   *smem_bytes = off + 1024;  // slack for the 1024-byte alignment of the base
   return *smem_bytes <= 227 * 1024;
 }
