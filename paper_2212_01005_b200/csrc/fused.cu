@@ -20,6 +20,8 @@ ago_status_t fused_plan(Plan* plan, FusedState* st, std::string* err) {
       return AGO_OK;
     case AGO_KERNEL_MBV2_BLOCK:
       return mbv2_plan(plan, st, err);
+    case AGO_KERNEL_ATTENTION:
+      return attention_plan(plan, st, err);
     default:
       *err = "fused mode: no kernel is built for this family yet";
       return AGO_ERR_UNSUPPORTED;
@@ -34,6 +36,8 @@ ago_status_t fused_run(const Plan& plan, FusedState* st, const void* const* inpu
   switch (plan.fused_kernel) {
     case AGO_KERNEL_MBV2_BLOCK:
       return mbv2_run(plan, st, inputs, weights, output, status_word, stream, err);
+    case AGO_KERNEL_ATTENTION:
+      return attention_run(plan, st, inputs, weights, output, status_word, stream, err);
     default:
       *err = "fused mode: no kernel is built for this family yet";
       return AGO_ERR_UNSUPPORTED;

@@ -23,6 +23,9 @@ cudaError_t ensure_max_dynamic_smem(const void* func, int* done_flags);
 
 // Kernel families (each in its own file).
 ago_status_t mbv2_plan(Plan* plan, FusedState* st, std::string* err);
+ago_status_t attention_plan(Plan* plan, FusedState* st, std::string* err);
+ago_status_t attention_run(const Plan& plan, FusedState* st, const void* const* inputs, const void* const* weights,
+                           void* output, unsigned int* status_word, cudaStream_t stream, std::string* err);
 ago_status_t mbv2_run(const Plan& plan, FusedState* st, const void* const* inputs, const void* const* weights,
                       void* output, unsigned int* status_word, cudaStream_t stream, std::string* err);
 

@@ -87,7 +87,7 @@ def test_padding_of_the_intermediate_with_large_bias(ago):
 
 # ---- fused kernels -------------------------------------------------------------------
 
-FUSED_SMALL = ["mbv2_14", "mbv2_s1_odd", "mbv2_s2", "mbv2_s2_odd"]
+FUSED_SMALL = ["mbv2_14", "mbv2_s1_odd", "mbv2_s2", "mbv2_s2_odd", "attn_small", "attn_ragged"]
 
 
 @pytest.mark.parametrize("name", FUSED_SMALL)
@@ -143,3 +143,27 @@ def test_fused_full_size_on_sampled_images(ago, name):
         one = WL.get(name, batch=1)
         ref = O.run_chain(one.ops, [data["inputs"][0][img:img + 1]], data["weights"])
         assert_close(gpu[img:img + 1], ref, what=f"{name} image {img}")
+
+
+def test_fused_attention_full_size_on_sampled_batches(ago):
+    wl = WL.get("attn_384")
+    data = WL.generate(wl)
+    gpu = run_gpu(ago, wl, data, "fused")
+    for bi in (0, 13, wl.samples - 1):
+        one = WL.get("attn_384", batch=1)
+        ref = O.run_chain(one.ops, [a[bi:bi + 1] for a in data["inputs"]], data["weights"])
+        assert_close(gpu[bi:bi + 1], ref, what=f"attn_384 batch {bi}")
+
+
+def test_fused_attention_dominant_key_and_uniform_rows(ago):
+    # one key dominates every query of head 0; head 1 has equal scores (uniform average of V)
+    wl = WL.attention("attn_probe", [51], 1, 144, 2, 64)
+    data = WL.generate(wl)
+    q, k, v = (a.copy() for a in data["inputs"])
+    q[:] = 0; k[:] = 0
+    q[0, :, 0] = 1.0; k[0, 77, 0] = 640.0         # head 0: score 640 / 8 = 80 at key 77, 0 elsewhere
+    data["inputs"] = [q, k, v]
+    gpu = run_gpu(ago, wl, data, "fused")
+    ref = O.run_chain(wl.ops, data["inputs"], data["weights"])
+    assert_close(gpu, ref, what="attn probe")
+    np.testing.assert_allclose(gpu[0, :, :64], np.broadcast_to(v[0, 77, :64].astype(np.float64), (144, 64)), atol=2e-2)
