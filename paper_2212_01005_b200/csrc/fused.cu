@@ -22,13 +22,17 @@ ago_status_t fused_plan(Plan* plan, FusedState* st, std::string* err) {
       return mbv2_plan(plan, st, err);
     case AGO_KERNEL_ATTENTION:
       return attention_plan(plan, st, err);
+    case AGO_KERNEL_FFN:
+      return ffn_plan(plan, st, err);
     default:
       *err = "fused mode: no kernel is built for this family yet";
       return AGO_ERR_UNSUPPORTED;
   }
 }
 
-size_t fused_workspace_bytes(const Plan&) { return 0; }
+size_t fused_workspace_bytes(const Plan& plan) {
+  return plan.fused_kernel == AGO_KERNEL_FFN ? ffn_workspace_bytes(plan) : 0;
+}
 
 ago_status_t fused_run(const Plan& plan, FusedState* st, const void* const* inputs, const void* const* weights,
                        void* output, void* workspace, unsigned int* status_word, cudaStream_t stream,
@@ -38,6 +42,8 @@ ago_status_t fused_run(const Plan& plan, FusedState* st, const void* const* inpu
       return mbv2_run(plan, st, inputs, weights, output, status_word, stream, err);
     case AGO_KERNEL_ATTENTION:
       return attention_run(plan, st, inputs, weights, output, status_word, stream, err);
+    case AGO_KERNEL_FFN:
+      return ffn_run(plan, st, inputs, weights, output, workspace, status_word, stream, err);
     default:
       *err = "fused mode: no kernel is built for this family yet";
       return AGO_ERR_UNSUPPORTED;

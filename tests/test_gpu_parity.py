@@ -23,6 +23,7 @@ def small_workloads():
         "mbv2_s2_odd": WL.mbv2_block("mbv2_s2_odd", [23], 2, 9, 16, 96, 32, 2, False),
         "ffn_small": WL.ffn("ffn_small", [24], 200, 128, 512, 1),
         "ffn_ragged": WL.ffn("ffn_ragged", [25], 77, 96, 264, 1),
+        "ffn_rows_ragged": WL.ffn("ffn_rows_ragged", [30], 333, 256, 384, 1),
         "resnet_small": WL.resnet_block("resnet_small", [26], 2, 12, 64),
         "resnet_odd": WL.resnet_block("resnet_odd", [27], 1, 9, 32),
         "attn_small": WL.attention("attn_small", [28], 2, 128, 2, 64),
@@ -87,7 +88,7 @@ def test_padding_of_the_intermediate_with_large_bias(ago):
 
 # ---- fused kernels -------------------------------------------------------------------
 
-FUSED_SMALL = ["mbv2_14", "mbv2_s1_odd", "mbv2_s2", "mbv2_s2_odd", "attn_small", "attn_ragged"]
+FUSED_SMALL = ["mbv2_14", "mbv2_s1_odd", "mbv2_s2", "mbv2_s2_odd", "attn_small", "attn_ragged", "ffn_small", "ffn_rows_ragged"]
 
 
 @pytest.mark.parametrize("name", FUSED_SMALL)
@@ -167,3 +168,31 @@ def test_fused_attention_dominant_key_and_uniform_rows(ago):
     ref = O.run_chain(wl.ops, data["inputs"], data["weights"])
     assert_close(gpu, ref, what="attn probe")
     np.testing.assert_allclose(gpu[0, :, :64], np.broadcast_to(v[0, 77, :64].astype(np.float64), (144, 64)), atol=2e-2)
+
+
+def test_fused_ffn_512_full(ago):
+    wl = WL.get("ffn_512")
+    data = WL.generate(wl)
+    ref = O.run_chain(wl.ops, data["inputs"], data["weights"])
+    gpu = run_gpu(ago, wl, data, "fused")
+    assert_close(gpu, ref, what="ffn_512 fused")
+    # the accumulation buffer must be left clean: a second and third run give the same bits
+    import torch
+    from helpers import to_device
+    sg = ago.Subgraph(wl.ops, wl.input_shapes, mode="fused")
+    ins, ws = to_device(wl, data)
+    a = sg.run(ins, ws).clone(); b = sg.run(ins, ws).clone(); c = sg.run(ins, ws).clone()
+    torch.cuda.synchronize()
+    for t in (a, b, c):
+        assert_close(t.float().cpu().numpy().astype(np.float64), ref, what="ffn_512 repeated run")
+    sg.close()
+
+
+def test_fused_ffn_12288_on_sampled_rows(ago):
+    wl = WL.get("ffn_12288")
+    data = WL.generate(wl)
+    gpu = run_gpu(ago, wl, data, "fused")
+    x = data["inputs"][0]
+    for r0 in (0, 6100, 12288 - 64):          # rows are independent samples of the chain
+        ref = O.run_chain(wl.ops, [x[r0:r0 + 64]], data["weights"])
+        assert_close(gpu[r0:r0 + 64], ref, what=f"ffn_12288 rows {r0}..")
