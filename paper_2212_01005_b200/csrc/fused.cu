@@ -24,6 +24,8 @@ ago_status_t fused_plan(Plan* plan, FusedState* st, std::string* err) {
       return attention_plan(plan, st, err);
     case AGO_KERNEL_FFN:
       return ffn_plan(plan, st, err);
+    case AGO_KERNEL_CONV3X3_PAIR:
+      return conv3x3_plan(plan, st, err);
     default:
       *err = "fused mode: no kernel is built for this family yet";
       return AGO_ERR_UNSUPPORTED;
@@ -44,6 +46,8 @@ ago_status_t fused_run(const Plan& plan, FusedState* st, const void* const* inpu
       return attention_run(plan, st, inputs, weights, output, status_word, stream, err);
     case AGO_KERNEL_FFN:
       return ffn_run(plan, st, inputs, weights, output, workspace, status_word, stream, err);
+    case AGO_KERNEL_CONV3X3_PAIR:
+      return conv3x3_run(plan, st, inputs, weights, output, status_word, stream, err);
     default:
       *err = "fused mode: no kernel is built for this family yet";
       return AGO_ERR_UNSUPPORTED;

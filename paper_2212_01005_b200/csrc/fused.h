@@ -30,6 +30,9 @@ ago_status_t ffn_plan(Plan* plan, FusedState* st, std::string* err);
 size_t ffn_workspace_bytes(const Plan& plan);
 ago_status_t ffn_run(const Plan& plan, FusedState* st, const void* const* inputs, const void* const* weights,
                      void* output, void* workspace, unsigned int* status_word, cudaStream_t stream, std::string* err);
+ago_status_t conv3x3_plan(Plan* plan, FusedState* st, std::string* err);
+ago_status_t conv3x3_run(const Plan& plan, FusedState* st, const void* const* inputs, const void* const* weights,
+                         void* output, unsigned int* status_word, cudaStream_t stream, std::string* err);
 ago_status_t mbv2_run(const Plan& plan, FusedState* st, const void* const* inputs, const void* const* weights,
                       void* output, unsigned int* status_word, cudaStream_t stream, std::string* err);
 

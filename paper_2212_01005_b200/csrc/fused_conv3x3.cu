@@ -1,0 +1,325 @@
+// Fused residual block: conv3x3 + bias + ReLU -> conv3x3 + bias -> + input -> ReLU,
+// one kernel; the first convolution's output never leaves the SM.
+//
+// This link is the "general" category of Section III-B: the downstream 3x3
+// convolution reuses its input along O2, H2 and W2, so any spatial tile of it
+// needs a halo of the upstream output and fusion recomputes that halo. A CTA
+// owns a strip of R output rows of one image (full width, all channels): it
+// computes R + 2 rows of the first convolution (2 of them recomputed by the
+// neighbouring strips) from R + 4 input rows.
+//
+// Both convolutions are implicit GEMMs on tcgen05: the activation tile sits in
+// shared memory as [channel block of 8][pixel][16 bytes] -- the un-swizzled
+// K-major operand layout -- with pixels linearised over the PADDED width, so the
+// operand of filter tap (dr, dc) is the same matrix at a start address shifted
+// by (dr * Wp + dc - 1) pixels. Weights stream through a TMA ring, one
+// [O x I] tap at a time.
+//
+//   P1  TMA (5-d map): input strip with halo -> channel-block planes, zero outside the image
+//   P2  tcgen05.mma: 9 taps x (I / 16) K-steps per 128-pixel tile            (TMEM)
+//   P3  TMEM -> registers: + b1, ReLU, zero outside the image (the second
+//       convolution pads the post-activation tensor), bf16 -> planes in shared memory
+//   P5  tcgen05.mma: second convolution over the resident planes             (TMEM)
+//   P6  TMEM -> registers: + b2 + x, ReLU, bf16, 16-byte stores
+#include <cuda.h>
+#include <cuda_bf16.h>
+
+#include <unordered_map>
+
+#include "fused.h"
+#include "tc_common.cuh"
+#include "tmap.h"
+
+namespace ago {
+
+namespace {
+
+using namespace tc;
+
+constexpr int kEpiThreads = 128;
+constexpr int kThreads = kEpiThreads + 64;   // + TMA warp + MMA warp
+constexpr int kWStages = 6;
+
+struct ConvParams {
+  const __nv_bfloat16* x;
+  const float* b1;
+  const float* b2;
+  __nv_bfloat16* out;
+  unsigned int* status;
+  int N, H, W, C;          // C = input = middle = output channels
+  int R, strips, IH, Wp, P1, M1, P2, M2;
+  int planes;              // C / 8
+  int w_row_bytes, w_swizzle, w_stage_bytes;
+  int x_plane, y_plane;    // bytes between channel-block planes of the input / intermediate tile
+  int off_x, off_y, off_w, off_bar;
+};
+
+__global__ void __launch_bounds__(kThreads, 1)
+conv3x3_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w1,
+                    const __grid_constant__ CUtensorMap tmap_w2, const ConvParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  uint8_t* sX = smem + p.off_x;   // first pixel of plane 0 (one pixel of slack lies before it)
+  uint8_t* sY = smem + p.off_y;
+  uint8_t* sW = smem + p.off_w;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + p.off_bar);
+  uint64_t* bar_x = bars;                      // input strip landed
+  uint64_t* bar_full = bars + 1;               // [kWStages] weight tap landed
+  uint64_t* bar_empty = bars + 1 + kWStages;   // [kWStages] weight tap consumed
+  uint64_t* bar_acc1 = bars + 1 + 2 * kWStages;   // first convolution complete
+  uint64_t* bar_y = bar_acc1 + 1;                 // intermediate planes written
+  uint64_t* bar_acc2 = bar_acc1 + 2;              // second convolution complete
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bar_acc1 + 3);
+  volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(bar_acc1 + 4);
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int n = blockIdx.x / p.strips, strip = blockIdx.x % p.strips;
+  const int h0 = strip * p.R;
+  const int rows_valid = min(p.R, p.H - h0);
+  const int ksteps = p.C / 16;
+
+  if (tid == kEpiThreads) {
+    *abort_flag = 0u;
+    mbar_init(bar_x, 1);
+    for (int i = 0; i < kWStages; ++i) { mbar_init(bar_full + i, 1); mbar_init(bar_empty + i, 1); }
+    mbar_init(bar_acc1, 1); mbar_init(bar_y, 1); mbar_init(bar_acc2, 1);
+    fence_mbar_init();
+    fence_proxy_async_smem();
+  }
+  if (warp == 0) {
+    tmem_alloc(tmem_slot, 512);
+    tmem_relinquish();
+  }
+  tcgen05_fence_before_sync();
+  __syncthreads();
+  tcgen05_fence_after_sync();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == kEpiThreads / 32) {
+    // ================================ TMA producer ================================
+    if (lane == 0) {
+      tma_prefetch_desc(&tmap_x); tma_prefetch_desc(&tmap_w1); tma_prefetch_desc(&tmap_w2);
+      mbar_arrive_expect_tx(bar_x, (uint32_t)(p.planes * p.x_plane));
+      tma_load_5d(sX, &tmap_x, bar_x, 0, -1, h0 - 2, n, 0);
+      for (int i = 0; i < 18; ++i) {            // 9 taps of the first, then 9 taps of the second convolution
+        const int s = i % kWStages;
+        if (i >= kWStages) mbar_wait(bar_empty + s, (uint32_t)((i / kWStages) - 1) & 1u, abort_flag, p.status, 0x401);
+        mbar_arrive_expect_tx(bar_full + s, (uint32_t)(p.C * p.w_row_bytes));
+        tma_load_3d(sW + s * p.w_stage_bytes, i < 9 ? &tmap_w1 : &tmap_w2, bar_full + s, 0, i % 9, 0);
+      }
+    }
+    __syncwarp();
+  } else if (warp == kEpiThreads / 32 + 1) {
+    // ================================ MMA issuer ================================
+    if (lane == 0) {
+      const uint32_t idesc = make_idesc_bf16(128, (uint32_t)p.C);
+      mbar_wait(bar_x, 0, abort_flag, p.status, 0x402);
+      for (int conv = 0; conv < 2; ++conv) {
+        const int tiles = conv == 0 ? p.M1 : p.M2;
+        const uint32_t plane = (uint32_t)(conv == 0 ? p.x_plane : p.y_plane);
+        const uint32_t abase = smem_u32(conv == 0 ? sX : sY);
+        if (conv == 1) mbar_wait(bar_y, 0, abort_flag, p.status, 0x403);
+        tcgen05_fence_after_sync();
+        for (int tap = 0; tap < 9; ++tap) {
+          const int i = conv * 9 + tap, s = i % kWStages;
+          mbar_wait(bar_full + s, (uint32_t)(i / kWStages) & 1u, abort_flag, p.status, 0x404);
+          tcgen05_fence_after_sync();
+          const int shift = (tap / 3) * p.Wp + (tap % 3) - 1;     // pixels
+          const uint64_t bdesc = make_smem_desc(smem_u32(sW + s * p.w_stage_bytes), 0, 8u * p.w_row_bytes, p.w_swizzle);
+          for (int mt = 0; mt < tiles; ++mt) {
+            // A: planes [channel block][pixel][16 B]; K step = two planes (LBO), 8-pixel groups are 128 B apart (SBO)
+            const uint64_t adesc = make_smem_desc(abase + (uint32_t)((mt * 128 + shift) * 16), plane, 128, SW_NONE);
+            for (int ks = 0; ks < ksteps; ++ks)
+              umma_bf16(tmem_base + mt * p.C, adesc + (uint64_t)((2u * ks * plane) >> 4), bdesc + 2u * ks, idesc,
+                        (tap | ks) != 0);
+          }
+          umma_commit(bar_empty + s);
+        }
+        umma_commit(conv == 0 ? bar_acc1 : bar_acc2);
+      }
+    }
+    __syncwarp();
+  } else {
+    // ================================ epilogue warps (thread = pixel row of a tile) ================================
+    const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
+    const int row = warp * 32 + lane;
+
+    // P3: intermediate = ReLU(acc + b1) inside the image, 0 outside -> planes
+    mbar_wait(bar_acc1, 0, abort_flag, p.status, 0x405);
+    tcgen05_fence_after_sync();
+    for (int mt = 0; mt < p.M1; ++mt) {
+      const int m = mt * 128 + row;
+      const int a = m / p.Wp, b = m - a * p.Wp;
+      const int gh = h0 - 1 + a;
+      const bool inside = m < p.P1 && gh >= 0 && gh < p.H && b >= 1 && b <= p.W;
+      for (int c0 = 0; c0 < p.C; c0 += 16) {
+        uint32_t v[16];
+        tmem_ld_x16(tmem_base + lane_base + mt * p.C + c0, v);
+        tmem_ld_wait();
+        uint32_t w[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          const float y0 = fmaxf(__uint_as_float(v[2 * j]) + __ldg(p.b1 + c0 + 2 * j), 0.0f);
+          const float y1 = fmaxf(__uint_as_float(v[2 * j + 1]) + __ldg(p.b1 + c0 + 2 * j + 1), 0.0f);
+          w[j] = inside ? pack_bf16x2(y0, y1) : 0u;
+        }
+        if (m < p.P1 + p.Wp) {   // a little past the tile so that shifted reads of valid rows never see stale data
+          *reinterpret_cast<uint4*>(sY + (size_t)(c0 / 8) * p.y_plane + m * 16) = make_uint4(w[0], w[1], w[2], w[3]);
+          *reinterpret_cast<uint4*>(sY + (size_t)(c0 / 8 + 1) * p.y_plane + m * 16) = make_uint4(w[4], w[5], w[6], w[7]);
+        }
+      }
+    }
+    fence_proxy_async_smem();
+    tcgen05_fence_before_sync();
+    named_barrier_sync(1, kEpiThreads);
+    if (tid == 0) mbar_arrive(bar_y);
+
+    // P6: out = ReLU(acc + b2 + x)
+    mbar_wait(bar_acc2, 0, abort_flag, p.status, 0x406);
+    tcgen05_fence_after_sync();
+    for (int mt = 0; mt < p.M2; ++mt) {
+      const int m = mt * 128 + row;
+      const int r = m / p.Wp, cc = m - r * p.Wp;
+      const bool valid = r < rows_valid && cc >= 1 && cc <= p.W;
+      const size_t pix = ((size_t)n * p.H + h0 + r) * p.W + (cc - 1);
+      for (int c0 = 0; c0 < p.C; c0 += 16) {
+        uint32_t v[16];
+        tmem_ld_x16(tmem_base + lane_base + mt * p.C + c0, v);
+        tmem_ld_wait();
+        if (valid) {
+          const uint4 x0 = __ldg(reinterpret_cast<const uint4*>(p.x + pix * p.C + c0));
+          const uint4 x1 = __ldg(reinterpret_cast<const uint4*>(p.x + pix * p.C + c0 + 8));
+          const uint32_t xs[8] = {x0.x, x0.y, x0.z, x0.w, x1.x, x1.y, x1.z, x1.w};
+          uint32_t w[8];
+#pragma unroll
+          for (int j = 0; j < 8; ++j) {
+            const float y0 = fmaxf(__uint_as_float(v[2 * j]) + __ldg(p.b2 + c0 + 2 * j) + bf16_lo(xs[j]), 0.0f);
+            const float y1 = fmaxf(__uint_as_float(v[2 * j + 1]) + __ldg(p.b2 + c0 + 2 * j + 1) + bf16_hi(xs[j]), 0.0f);
+            w[j] = pack_bf16x2(y0, y1);
+          }
+          *reinterpret_cast<uint4*>(p.out + pix * p.C + c0) = make_uint4(w[0], w[1], w[2], w[3]);
+          *reinterpret_cast<uint4*>(p.out + pix * p.C + c0 + 8) = make_uint4(w[4], w[5], w[6], w[7]);
+        }
+      }
+    }
+  }
+  tcgen05_fence_before_sync();
+  __syncthreads();
+  if (warp == 0) tmem_dealloc(tmem_base, 512);
+}
+
+struct ConvHost {
+  ConvParams prm;
+  int smem_bytes = 0;
+  struct Key { const void* p; int which; bool operator==(const Key& o) const { return p == o.p && which == o.which; } };
+  struct KeyHash { size_t operator()(const Key& k) const { return std::hash<const void*>()(k.p) ^ (size_t)k.which * 0x9e3779b97f4a7c15ull; } };
+  std::unordered_map<Key, CUtensorMap, KeyHash> maps;
+};
+
+int round_up_i(int v, int m) { return (v + m - 1) / m * m; }
+
+bool conv_layout(ConvParams& q, int R, int* smem_bytes) {
+  q.R = R;
+  q.strips = (q.H + R - 1) / R;
+  q.IH = R + 4;
+  q.Wp = q.W + 2;
+  q.P1 = (R + 2) * q.Wp; q.M1 = (q.P1 + 127) / 128;
+  q.P2 = R * q.Wp; q.M2 = (q.P2 + 127) / 128;
+  if (q.IH > 256 || q.Wp > 256 || q.M1 * q.C > 512) return false;
+  q.x_plane = q.IH * q.Wp * 16;
+  // the intermediate planes must hold every pixel a shifted operand row can touch
+  const int y_pixels = std::max(q.P1 + q.Wp, q.M2 * 128 + 2 * q.Wp + 2) + 8;
+  q.y_plane = y_pixels * 16;
+  int off = 1024;   // slack before the input planes: tap (0,0) of pixel 0 starts one pixel early
+  q.off_x = off;
+  const int x_reach = std::max(q.planes * q.x_plane, (q.planes - 1) * q.x_plane + (q.M1 * 128 + 2 * q.Wp + 2) * 16);
+  off = round_up_i(off + x_reach, 1024) + 1024;
+  q.off_y = off;
+  off = round_up_i(off + q.planes * q.y_plane, 1024);
+  q.off_w = off;
+  off += kWStages * q.w_stage_bytes;
+  q.off_bar = off;
+  off += 256;
+  *smem_bytes = off + 1024;
+  return *smem_bytes <= 227 * 1024;
+}
+
+}  // namespace
+
+ago_status_t conv3x3_plan(Plan* plan, FusedState* st, std::string* err) {
+  const OpInfo& c1 = plan->ops[0];
+  auto* host = new ConvHost();
+  ConvParams& q = host->prm;
+  q = ConvParams{};
+  q.N = (int)c1.in.d[0]; q.H = (int)c1.in.d[1]; q.W = (int)c1.in.d[2]; q.C = (int)c1.in.d[3];
+  auto bad = [&](const char* m) { *err = std::string("fused conv3x3 pair: ") + m; delete host; return AGO_ERR_UNSUPPORTED; };
+  if (c1.op.p[0] != q.C || plan->ops[3].op.p[0] != q.C) return bad("input, middle and output channel counts must be equal");
+  if (q.C != 16 && q.C != 32 && q.C != 64) return bad("channel count must be 16, 32 or 64");
+  q.planes = q.C / 8;
+  q.w_row_bytes = q.C * 2;
+  q.w_swizzle = q.C == 16 ? tc::SW_32B : (q.C == 32 ? tc::SW_64B : tc::SW_128B);
+  q.w_stage_bytes = round_up_i(q.C * q.w_row_bytes, 1024);
+  int best_R = 0, best_smem = 0; double best_cost = 0;
+  for (int R = 1; R <= q.H; ++R) {
+    ConvParams t = q; int smem = 0;
+    if (!conv_layout(t, R, &smem)) continue;
+    const long ctas = (long)q.N * t.strips;
+    const long waves = (ctas + 147) / 148;
+    const double cost = (double)waves * (t.M1 + t.M2 + 1.0);
+    if (best_R == 0 || cost < best_cost) { best_R = R; best_cost = cost; best_smem = smem; }
+  }
+  if (best_R == 0) return bad("no row-strip tiling fits shared memory / tensor memory");
+  conv_layout(q, best_R, &best_smem);
+  host->smem_bytes = best_smem;
+  st->impl = host;
+  st->impl_free = [](void* p) { delete static_cast<ConvHost*>(p); };
+  st->tile_rows = best_R; st->grid = q.N * q.strips; st->smem_bytes = best_smem;
+  plan->tile_rows = best_R; plan->smem_bytes = best_smem;
+  return AGO_OK;
+}
+
+ago_status_t conv3x3_run(const Plan& plan, FusedState* st, const void* const* inputs, const void* const* weights,
+                         void* output, unsigned int* status_word, cudaStream_t stream, std::string* err) {
+  ConvHost* host = static_cast<ConvHost*>(st->impl);
+  ConvParams q = host->prm;
+  q.x = static_cast<const __nv_bfloat16*>(inputs[0]);
+  q.b1 = static_cast<const float*>(weights[1]);
+  q.b2 = static_cast<const float*>(weights[3]);
+  q.out = static_cast<__nv_bfloat16*>(output);
+  q.status = status_word;
+  auto get_map = [&](const void* base, int which, CUtensorMap* out) -> bool {
+    ConvHost::Key key{base, which};
+    auto it = host->maps.find(key);
+    if (it == host->maps.end()) {
+      CUtensorMap m;
+      if (which == 0) {
+        const uint64_t dims[5] = {8, (uint64_t)q.W, (uint64_t)q.H, (uint64_t)q.N, (uint64_t)q.planes};
+        const uint64_t strides[4] = {(uint64_t)q.C * 2, (uint64_t)q.W * q.C * 2, (uint64_t)q.H * q.W * q.C * 2, 16};
+        const uint32_t box[5] = {8, (uint32_t)q.Wp, (uint32_t)q.IH, 1, (uint32_t)q.planes};
+        if (!encode_tmap_bf16(&m, base, 5, dims, strides, box, 0, err)) return false;
+      } else {
+        const uint64_t dims[3] = {(uint64_t)q.C, 9, (uint64_t)q.C};
+        const uint64_t strides[2] = {(uint64_t)q.C * 2, (uint64_t)9 * q.C * 2};
+        const uint32_t box[3] = {(uint32_t)q.C, 1, (uint32_t)q.C};
+        if (!encode_tmap_bf16(&m, base, 3, dims, strides, box, q.w_row_bytes, err)) return false;
+      }
+      if (host->maps.size() > 4096) host->maps.clear();
+      it = host->maps.emplace(key, m).first;
+    }
+    *out = it->second;
+    return true;
+  };
+  CUtensorMap mx, mw1, mw2;
+  if (!get_map(inputs[0], 0, &mx) || !get_map(weights[0], 1, &mw1) || !get_map(weights[2], 2, &mw2)) return AGO_ERR_CUDA;
+  {
+    static int smem_opt_in[64] = {};
+    cudaError_t e = ensure_max_dynamic_smem(reinterpret_cast<const void*>(conv3x3_pair_kernel), smem_opt_in);
+    if (e != cudaSuccess) { *err = std::string("cudaFuncSetAttribute: ") + cudaGetErrorString(e); return AGO_ERR_CUDA; }
+  }
+  conv3x3_pair_kernel<<<q.N * q.strips, kThreads, host->smem_bytes, stream>>>(mx, mw1, mw2, q);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) { *err = std::string("fused conv3x3 pair launch: ") + cudaGetErrorString(e); return AGO_ERR_CUDA; }
+  return AGO_OK;
+}
+
+}  // namespace ago

@@ -26,6 +26,7 @@ def small_workloads():
         "ffn_rows_ragged": WL.ffn("ffn_rows_ragged", [30], 333, 256, 384, 1),
         "resnet_small": WL.resnet_block("resnet_small", [26], 2, 12, 64),
         "resnet_odd": WL.resnet_block("resnet_odd", [27], 1, 9, 32),
+        "resnet_16ch": WL.resnet_block("resnet_16ch", [32], 2, 20, 16),
         "attn_small": WL.attention("attn_small", [28], 2, 128, 2, 64),
         "attn_ragged": WL.attention("attn_ragged", [29], 1, 200, 3, 64),
     }
@@ -88,7 +89,7 @@ def test_padding_of_the_intermediate_with_large_bias(ago):
 
 # ---- fused kernels -------------------------------------------------------------------
 
-FUSED_SMALL = ["mbv2_14", "mbv2_s1_odd", "mbv2_s2", "mbv2_s2_odd", "attn_small", "attn_ragged", "ffn_small", "ffn_rows_ragged"]
+FUSED_SMALL = ["mbv2_14", "mbv2_s1_odd", "mbv2_s2", "mbv2_s2_odd", "attn_small", "attn_ragged", "ffn_small", "ffn_rows_ragged", "resnet_small", "resnet_odd", "resnet_16ch"]
 
 
 @pytest.mark.parametrize("name", FUSED_SMALL)
@@ -196,3 +197,22 @@ def test_fused_ffn_12288_on_sampled_rows(ago):
     for r0 in (0, 6100, 12288 - 64):          # rows are independent samples of the chain
         ref = O.run_chain(wl.ops, [x[r0:r0 + 64]], data["weights"])
         assert_close(gpu[r0:r0 + 64], ref, what=f"ffn_12288 rows {r0}..")
+
+
+def test_fused_conv3x3_pads_the_intermediate_not_the_input(ago):
+    # with a large positive first bias, ReLU(b1) in the halo of the intermediate would leak into the border
+    wl = WL.resnet_block("respad", [61], 1, 10, 16)
+    data = WL.generate(wl)
+    data["weights"][1] = np.full(16, 2.0, dtype=np.float32)
+    ref = O.run_chain(wl.ops, data["inputs"], data["weights"])
+    assert_close(run_gpu(ago, wl, data, "fused"), ref, what="resnet pad/fused")
+
+
+def test_fused_resnet_full_size_on_sampled_images(ago):
+    wl = WL.get("resnet_56")
+    data = WL.generate(wl)
+    gpu = run_gpu(ago, wl, data, "fused")
+    for img in (0, 11, wl.samples - 1):
+        one = WL.get("resnet_56", batch=1)
+        ref = O.run_chain(one.ops, [data["inputs"][0][img:img + 1]], data["weights"])
+        assert_close(gpu[img:img + 1], ref, what=f"resnet_56 image {img}")
