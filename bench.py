@@ -205,6 +205,7 @@ def main():
     ap.add_argument("--sets", type=int, default=0, help="rotating buffer sets per step (0 = enough to exceed 4x L2)")
     ap.add_argument("--skip-cpu-baseline", action="store_true")
     ap.add_argument("--skip-unfused", action="store_true")
+    ap.add_argument("--headline-only", action="store_true", help="skip the summary of the other configurations")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
 
@@ -228,44 +229,9 @@ def main():
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=dev)
 
-    wl = WL.get(args.workload)
     peaks = load_peaks()
-    io = WL.io_bytes(wl)
     l2 = torch.cuda.get_device_properties(dev).L2_cache_size
-
-    def make_handle(mode):
-        sg = B.Subgraph(wl.ops, wl.input_shapes, mode=mode)
-        sg.ensure_workspace(dev)
-        return sg
-
-    sg = make_handle(args.mode)
-    per_set = io + sg.workspace_bytes
-    nsets = args.sets or max(2, int(np.ceil(4.0 * l2 / per_set)))
-
-    # Resident buffer sets: set r holds its own inputs, weights and output (seeded, one draw per set).
-    sets = []
-    for r in range(nsets):
-        d = WL.generate(wl, list(wl.seed_seq) + [1000 + r + 10000 * rank])
-        ins = [torch.from_numpy(a).to(dev, torch.bfloat16) for a in d["inputs"]]
-        ws = [torch.from_numpy(a).to(dev, torch.float32 if k == "bias" else torch.bfloat16)
-              for a, k in zip(d["weights"], wl.weight_kinds)]
-        sets.append((ins, ws, sg.empty_output(dev)))
     stream = torch.cuda.Stream(dev)
-
-    def one_pass(handle):
-        for ins, ws, out in sets:
-            handle.run(ins, ws, out=out, stream=stream.cuda_stream)
-
-    def build_step(handle):
-        with torch.cuda.stream(stream):
-            one_pass(handle)                    # first run: status word, attributes, tensor maps
-        stream.synchronize()
-        if args.no_graph:
-            return lambda: one_pass(handle)
-        g = torch.cuda.CUDAGraph()
-        with torch.cuda.graph(g, stream=stream):
-            one_pass(handle)
-        return g.replay
 
     def timed(step_fn, steps, warmup, sampler=None):
         with torch.cuda.stream(stream):
@@ -293,49 +259,113 @@ def main():
             ms = float(t.item())
         return ms / steps
 
-    sampler = ClockSampler(local)
-    step = build_step(sg)
-    ms_step = timed(step, args.steps, args.warmup, sampler)
-    clocks = sampler.finish()
-    assert sg.status() == B.AGO_OK, B.ago_last_error()
-    launches_per_pass = sg.query(B.AGO_Q_NUM_LAUNCHES)
-    sec_per_launch = ms_step * 1e-3 / nsets
-    value = wl.samples * nsets * world / (ms_step * 1e-3)
+    def measure(name, mode, steps, warmup, with_e2e, unfused_modes, sampler=None):
+        """Time one workload: fused (or `mode`) step, optional end-to-end and unfused modes, same buffers."""
+        wl = WL.get(name)
+        io = WL.io_bytes(wl)
 
-    # ---- end to end: pinned host buffers, H2D + run + D2H inside the timed region ------------------
-    h_in = [[t.cpu().pin_memory() for t in ins] for ins, _, _ in sets[:2]]
-    h_out = [torch.empty(wl.output_shape, dtype=torch.bfloat16).pin_memory() for _ in range(2)]
-    e2e_sets = min(nsets, 8)
+        def make_handle(m):
+            h = B.Subgraph(wl.ops, wl.input_shapes, mode=m)
+            h.ensure_workspace(dev)
+            return h
 
-    def e2e_pass():
-        for r in range(e2e_sets):
-            ins, ws, out = sets[r]
-            sg.run_host(h_in[r % 2], ws, h_out[r % 2], ins, out, stream=stream.cuda_stream)
+        sg = make_handle(mode)
+        per_set = io + sg.workspace_bytes
+        nsets = args.sets or max(2, int(np.ceil(4.0 * l2 / per_set)))
+        # Resident buffer sets: set r holds its own inputs, weights and output (seeded, one draw per set).
+        sets = []
+        for r in range(nsets):
+            d = WL.generate(wl, list(wl.seed_seq) + [1000 + r + 10000 * rank])
+            ins = [torch.from_numpy(a).to(dev, torch.bfloat16) for a in d["inputs"]]
+            ws = [torch.from_numpy(a).to(dev, torch.float32 if k == "bias" else torch.bfloat16)
+                  for a, k in zip(d["weights"], wl.weight_kinds)]
+            sets.append((ins, ws, sg.empty_output(dev)))
 
-    ms_e2e = timed(e2e_pass, max(3, min(args.steps, 10)), 3)
-    in_bytes = sum(2 * int(np.prod(s)) for s in wl.input_shapes)
-    out_bytes = 2 * int(np.prod(wl.output_shape))
-    e2e = {"value": wl.samples * e2e_sets * world / (ms_e2e * 1e-3), "unit": "samples/s",
-           "h2d_bytes_per_step": in_bytes * e2e_sets, "d2h_bytes_per_step": out_bytes * e2e_sets,
-           "launches_per_step": e2e_sets}
+        def one_pass(handle):
+            for ins, ws, out in sets:
+                handle.run(ins, ws, out=out, stream=stream.cuda_stream)
 
-    # ---- the unfused modes of the same library, same buffers (context for the fusion speedup) ----
-    unfused = {}
-    if not args.skip_unfused and args.mode == "fused":
-        for mode in ("per_mini_subgraph", "per_op"):
+        def build_step(handle):
+            with torch.cuda.stream(stream):
+                one_pass(handle)                    # first run: status word, attributes, tensor maps
+            stream.synchronize()
+            if args.no_graph:
+                return lambda: one_pass(handle)
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=stream):
+                one_pass(handle)
+            return g.replay
+
+        step = build_step(sg)
+        ms_step = timed(step, steps, warmup, sampler)
+        clocks = sampler.finish() if sampler is not None else None
+        assert sg.status() == B.AGO_OK, B.ago_last_error()
+        res = {"wl": wl, "nsets": nsets, "per_set": per_set, "ms_step": ms_step, "clocks": clocks,
+               "launches_per_pass": sg.query(B.AGO_Q_NUM_LAUNCHES),
+               "sec_per_launch": ms_step * 1e-3 / nsets,
+               "value": wl.samples * nsets * world / (ms_step * 1e-3),
+               "tile_rows": sg.query(B.AGO_Q_TILE_ROWS), "smem_bytes": sg.query(B.AGO_Q_SMEM_BYTES)}
+
+        if with_e2e:
+            # end to end: pinned host buffers, H2D + run + D2H inside the timed region
+            h_in = [[t.cpu().pin_memory() for t in ins] for ins, _, _ in sets[:2]]
+            h_out = [torch.empty(wl.output_shape, dtype=torch.bfloat16).pin_memory() for _ in range(2)]
+            e2e_sets = min(nsets, 8)
+
+            def e2e_pass():
+                for r in range(e2e_sets):
+                    ins, ws, out = sets[r]
+                    sg.run_host(h_in[r % 2], ws, h_out[r % 2], ins, out, stream=stream.cuda_stream)
+
+            ms_e2e = timed(e2e_pass, max(3, min(steps, 10)), 3)
+            in_bytes = sum(2 * int(np.prod(sh)) for sh in wl.input_shapes)
+            out_bytes = 2 * int(np.prod(wl.output_shape))
+            res["e2e"] = {"value": wl.samples * e2e_sets * world / (ms_e2e * 1e-3), "unit": "samples/s",
+                          "h2d_bytes_per_step": in_bytes * e2e_sets, "d2h_bytes_per_step": out_bytes * e2e_sets,
+                          "launches_per_step": e2e_sets}
+
+        # the unfused modes of the same library, same buffers (context for the fusion speedup)
+        unfused = {}
+        for m in unfused_modes:
             try:
-                h2 = make_handle(mode)
+                h2 = make_handle(m)
                 st2 = build_step(h2)
-                ms2 = timed(st2, max(3, args.steps // 5), 3)
-                unfused[mode] = {"value": wl.samples * nsets * world / (ms2 * 1e-3), "unit": "samples/s",
-                                 "us_per_launch_set": ms2 * 1e3 / nsets, "kernels_per_pass": h2.query(B.AGO_Q_NUM_LAUNCHES)}
+                ms2 = timed(st2, max(3, steps // 5), 3)
+                unfused[m] = {"value": wl.samples * nsets * world / (ms2 * 1e-3), "unit": "samples/s",
+                              "us_per_launch_set": ms2 * 1e3 / nsets, "kernels_per_pass": h2.query(B.AGO_Q_NUM_LAUNCHES)}
                 h2.close()
             except B.AgoError as e:
-                unfused[mode] = {"error": str(e)}
-        if "value" in unfused.get("per_mini_subgraph", {}):
-            unfused["speedup_vs_per_mini_subgraph"] = round(value / unfused["per_mini_subgraph"]["value"], 3)
-        if "value" in unfused.get("per_op", {}):
-            unfused["speedup_vs_per_op"] = round(value / unfused["per_op"]["value"], 3)
+                unfused[m] = {"error": str(e)}
+        for m in unfused_modes:
+            if "value" in unfused.get(m, {}):
+                unfused["speedup_vs_" + m] = round(res["value"] / unfused[m]["value"], 3)
+        res["unfused"] = unfused
+        sg.close()
+        del sets
+        torch.cuda.empty_cache()
+        return res
+
+    sampler = ClockSampler(local)
+    head_unfused = [] if (args.skip_unfused or args.mode != "fused") else ["per_mini_subgraph", "per_op"]
+    head = measure(args.workload, args.mode, args.steps, args.warmup, True, head_unfused, sampler)
+    wl, nsets, per_set, ms_step = head["wl"], head["nsets"], head["per_set"], head["ms_step"]
+    clocks, launches_per_pass, sec_per_launch, value = head["clocks"], head["launches_per_pass"], head["sec_per_launch"], head["value"]
+    e2e, unfused = head["e2e"], head["unfused"]
+
+    # the other benchmark configurations, fused, against their own rooflines and per-mini-subgraph chains
+    others = {}
+    if not args.headline_only and world == 1 and args.mode == "fused":
+        for name in WL.ALL:
+            if name == args.workload:
+                continue
+            r = measure(name, "fused", max(3, min(args.steps, 10)), 3, False,
+                        [] if args.skip_unfused else ["per_mini_subgraph"])
+            rf = roofline(r["wl"], peaks, r["sec_per_launch"], NCU_TRAFFIC_BYTES.get((name, "fused")))
+            others[name] = {"value": r["value"], "unit": "samples/s", "us_per_launch": round(r["sec_per_launch"] * 1e6, 3),
+                            "roofline_bound": rf["bound"], "roofline_us": rf["roofline_us"],
+                            "roofline_frac": rf["frac_of_whole_roofline"],
+                            "speedup_vs_per_mini_subgraph": r["unfused"].get("speedup_vs_per_mini_subgraph"),
+                            "tile_rows": r["tile_rows"]}
 
     if rank != 0:
         if dist is not None:
@@ -356,6 +386,7 @@ def main():
         "roofline": roofline(wl, peaks, sec_per_launch, NCU_TRAFFIC_BYTES.get((args.workload, args.mode))),
         "e2e": e2e, "gpu_launches": args.steps * nsets * launches_per_pass, "clocks": clocks,
         "unfused": unfused,
+        "other_workloads": others,
     }
     if not args.skip_cpu_baseline:
         line["cpu_baseline"] = cpu_baseline(wl, args.workload)
