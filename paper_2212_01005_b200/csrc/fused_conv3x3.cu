@@ -36,9 +36,10 @@ namespace {
 
 using namespace tc;
 
-constexpr int kEpiThreads = 128;
+constexpr int kEpiWarps = 8;                 // two per TMEM lane quarter: each takes half of the channels
+constexpr int kEpiThreads = kEpiWarps * 32;
 constexpr int kThreads = kEpiThreads + 64;   // + TMA warp + MMA warp
-constexpr int kWStages = 6;
+constexpr int kMaxWStages = 4;     // ring stages; each holds one filter row = 3 taps
 
 struct ConvParams {
   const __nv_bfloat16* x;
@@ -48,10 +49,12 @@ struct ConvParams {
   unsigned int* status;
   int N, H, W, C;          // C = input = middle = output channels
   int R, strips, IH, Wp, P1, M1, P2, M2;
+  int a1, a2;              // tiles [0,a1) of conv1 / [0,a2) of conv2 form the first pipeline group
   int planes;              // C / 8
   int w_row_bytes, w_swizzle, w_stage_bytes;
+  int wstages;             // ring stages in use (2..kMaxWStages)
   int x_plane, y_plane;    // bytes between channel-block planes of the input / intermediate tile
-  int off_x, off_y, off_w, off_bar;
+  int off_x, off_y, off_w, off_bias, off_bar;
 };
 
 __global__ void __launch_bounds__(kThreads, 1)
@@ -60,19 +63,28 @@ conv3x3_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t* sX = smem + p.off_x;   // first pixel of plane 0 (one pixel of slack lies before it)
-  uint8_t* sY = smem + p.off_y;
+  uint8_t* sY = smem + p.off_y;   // the intermediate planes reuse the input planes' memory, two pixels lower
   uint8_t* sW = smem + p.off_w;
+  float* sBias = reinterpret_cast<float*>(smem + p.off_bias);   // b1[C], b2[C]
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + p.off_bar);
   uint64_t* bar_x = bars;                      // input strip landed
-  uint64_t* bar_full = bars + 1;               // [kWStages] weight tap landed
-  uint64_t* bar_empty = bars + 1 + kWStages;   // [kWStages] weight tap consumed
-  uint64_t* bar_acc1 = bars + 1 + 2 * kWStages;   // first convolution complete
-  uint64_t* bar_y = bar_acc1 + 1;                 // intermediate planes written
-  uint64_t* bar_acc2 = bar_acc1 + 2;              // second convolution complete
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bar_acc1 + 3);
-  volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(bar_acc1 + 4);
+  uint64_t* bar_full = bars + 1;                  // [kMaxWStages] filter row landed
+  uint64_t* bar_empty = bars + 1 + kMaxWStages;   // [kMaxWStages] filter row consumed
+  uint64_t* bar_acc1 = bars + 1 + 2 * kMaxWStages;   // [2] first convolution, tile group g complete
+  uint64_t* bar_y = bar_acc1 + 2;                 // [2] intermediate planes of group g written
+  uint64_t* bar_acc2 = bar_acc1 + 4;              // [2] second convolution, tile group g complete
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bar_acc1 + 6);
+  volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(bar_acc1 + 7);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+#ifdef AGO_TIMELINE
+  long long* ts = reinterpret_cast<long long*>(p.out) + (tid == 0 ? 0 : (tid == kEpiThreads ? 64 : 128)); int tsi = 0;
+  const bool tsw = blockIdx.x == 0 && (tid == 0 || tid == kEpiThreads || tid == kEpiThreads + 32);
+#define TS() do { if (tsw) ts[tsi++] = clock64(); } while (0)
+#else
+#define TS() do {} while (0)
+#endif
+  TS();
   const int n = blockIdx.x / p.strips, strip = blockIdx.x % p.strips;
   const int h0 = strip * p.R;
   const int rows_valid = min(p.R, p.H - h0);
@@ -81,124 +93,186 @@ conv3x3_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
   if (tid == kEpiThreads) {
     *abort_flag = 0u;
     mbar_init(bar_x, 1);
-    for (int i = 0; i < kWStages; ++i) { mbar_init(bar_full + i, 1); mbar_init(bar_empty + i, 1); }
-    mbar_init(bar_acc1, 1); mbar_init(bar_y, 1); mbar_init(bar_acc2, 1);
+    for (int i = 0; i < kMaxWStages; ++i) { mbar_init(bar_full + i, 1); mbar_init(bar_empty + i, 1); }
+    for (int i = 0; i < 6; ++i) mbar_init(bar_acc1 + i, 1);
     fence_mbar_init();
     fence_proxy_async_smem();
+    tma_prefetch_desc(&tmap_x);
+    mbar_arrive_expect_tx(bar_x, (uint32_t)(p.planes * p.IH * p.Wp * 16));
+    for (int k = 0; k < p.planes; ++k) tma_load_5d(sX + (size_t)k * p.x_plane, &tmap_x, bar_x, 0, -1, h0 - 2, n, k);
   }
   if (warp == 0) {
     tmem_alloc(tmem_slot, 512);
     tmem_relinquish();
   }
+  if (tid < 2 * p.C) sBias[tid] = tid < p.C ? p.b1[tid] : p.b2[tid - p.C];
   tcgen05_fence_before_sync();
   __syncthreads();
   tcgen05_fence_after_sync();
   const uint32_t tmem_base = *tmem_slot;
 
-  if (warp == kEpiThreads / 32) {
-    // ================================ TMA producer ================================
+  // The four MMA passes: (convolution, tile group) = (1,A) (1,B) (2,A) (2,B); each streams the 9 taps.
+  const int pass_lo[4] = {0, p.a1, 0, p.a2};
+  const int pass_hi[4] = {p.a1, p.M1, p.a2, p.M2};
+
+  if (warp == kEpiWarps) {
+    // ================================ TMA producer: weight taps ================================
     if (lane == 0) {
-      tma_prefetch_desc(&tmap_x); tma_prefetch_desc(&tmap_w1); tma_prefetch_desc(&tmap_w2);
-      mbar_arrive_expect_tx(bar_x, (uint32_t)(p.planes * p.x_plane));
-      tma_load_5d(sX, &tmap_x, bar_x, 0, -1, h0 - 2, n, 0);
-      for (int i = 0; i < 18; ++i) {            // 9 taps of the first, then 9 taps of the second convolution
-        const int s = i % kWStages;
-        if (i >= kWStages) mbar_wait(bar_empty + s, (uint32_t)((i / kWStages) - 1) & 1u, abort_flag, p.status, 0x401);
-        mbar_arrive_expect_tx(bar_full + s, (uint32_t)(p.C * p.w_row_bytes));
-        tma_load_3d(sW + s * p.w_stage_bytes, i < 9 ? &tmap_w1 : &tmap_w2, bar_full + s, 0, i % 9, 0);
+      tma_prefetch_desc(&tmap_w1); tma_prefetch_desc(&tmap_w2);
+      int i = 0;
+      for (int ps = 0; ps < 4; ++ps) {
+        if (pass_lo[ps] >= pass_hi[ps]) continue;      // empty group: the MMA warp skips it too
+        for (int frow = 0; frow < 3; ++frow, ++i) {
+          const int s = i % p.wstages;
+          if (i >= p.wstages) mbar_wait(bar_empty + s, (uint32_t)((i / p.wstages) - 1) & 1u, abort_flag, p.status, 0x401);
+          mbar_arrive_expect_tx(bar_full + s, (uint32_t)(3 * p.C * p.w_row_bytes));
+          for (int t3 = 0; t3 < 3; ++t3)
+            tma_load_3d(sW + (s * 3 + t3) * p.w_stage_bytes, ps < 2 ? &tmap_w1 : &tmap_w2, bar_full + s, 0, frow * 3 + t3, 0);
+        }
       }
     }
     __syncwarp();
-  } else if (warp == kEpiThreads / 32 + 1) {
+  } else if (warp == kEpiWarps + 1) {
     // ================================ MMA issuer ================================
     if (lane == 0) {
       const uint32_t idesc = make_idesc_bf16(128, (uint32_t)p.C);
+      const uint64_t wdesc0 = make_smem_desc(smem_u32(sW), 0, 8u * p.w_row_bytes, p.w_swizzle);
+      TS();
       mbar_wait(bar_x, 0, abort_flag, p.status, 0x402);
-      for (int conv = 0; conv < 2; ++conv) {
-        const int tiles = conv == 0 ? p.M1 : p.M2;
+      TS();
+      int i = 0;
+      for (int ps = 0; ps < 4; ++ps) {
+        const int conv = ps >> 1, grp = ps & 1;
+        uint64_t* done = (conv == 0 ? bar_acc1 : bar_acc2) + grp;
+        if (conv == 1) mbar_wait(bar_y + grp, 0, abort_flag, p.status, 0x403);   // the planes this group reads are written
+        TS();
+        if (pass_lo[ps] >= pass_hi[ps]) { umma_commit(done); continue; }
         const uint32_t plane = (uint32_t)(conv == 0 ? p.x_plane : p.y_plane);
-        const uint32_t abase = smem_u32(conv == 0 ? sX : sY);
-        if (conv == 1) mbar_wait(bar_y, 0, abort_flag, p.status, 0x403);
+        // A: planes [channel block][pixel][16 B]; K step = two planes (LBO), 8-pixel groups are 128 B apart (SBO).
+        // Descriptor arithmetic is hoisted: one add per tile, constant strides per K step.
+        const uint64_t adesc0 = make_smem_desc(smem_u32(conv == 0 ? sX : sY), plane, 128, SW_NONE);
+        const uint32_t a_kstep = (2u * plane) >> 4;
+        const int lo = pass_lo[ps], hi = pass_hi[ps];
         tcgen05_fence_after_sync();
         for (int tap = 0; tap < 9; ++tap) {
-          const int i = conv * 9 + tap, s = i % kWStages;
-          mbar_wait(bar_full + s, (uint32_t)(i / kWStages) & 1u, abort_flag, p.status, 0x404);
-          tcgen05_fence_after_sync();
-          const int shift = (tap / 3) * p.Wp + (tap % 3) - 1;     // pixels
-          const uint64_t bdesc = make_smem_desc(smem_u32(sW + s * p.w_stage_bytes), 0, 8u * p.w_row_bytes, p.w_swizzle);
-          for (int mt = 0; mt < tiles; ++mt) {
-            // A: planes [channel block][pixel][16 B]; K step = two planes (LBO), 8-pixel groups are 128 B apart (SBO)
-            const uint64_t adesc = make_smem_desc(abase + (uint32_t)((mt * 128 + shift) * 16), plane, 128, SW_NONE);
-            for (int ks = 0; ks < ksteps; ++ks)
-              umma_bf16(tmem_base + mt * p.C, adesc + (uint64_t)((2u * ks * plane) >> 4), bdesc + 2u * ks, idesc,
-                        (tap | ks) != 0);
+          const int s = i % p.wstages;
+          if (tap % 3 == 0) {
+            mbar_wait(bar_full + s, (uint32_t)(i / p.wstages) & 1u, abort_flag, p.status, 0x404);
+            tcgen05_fence_after_sync();
           }
-          umma_commit(bar_empty + s);
+          const int shift = (tap / 3) * p.Wp + (tap % 3) - 1;     // pixels = 16-byte units
+          const uint64_t bdesc = wdesc0 + (uint64_t)((uint32_t)((s * 3 + tap % 3) * p.w_stage_bytes) >> 4);
+          // all per-MMA arithmetic is 32-bit adds on the descriptors' low words
+          const uint32_t a_hi = (uint32_t)(adesc0 >> 32), b_hi = (uint32_t)(bdesc >> 32), b_lo = (uint32_t)bdesc;
+          uint32_t a_lo = (uint32_t)adesc0 + (uint32_t)(lo * 128 + shift);
+          uint32_t d_tmem = tmem_base + lo * p.C;
+          const uint32_t acc0 = tap != 0;
+          if (ksteps == 4) {
+            for (int mt = lo; mt < hi; ++mt, a_lo += 128, d_tmem += p.C) {
+              umma_bf16_lohi(d_tmem, a_lo, a_hi, b_lo, b_hi, idesc, acc0);
+              umma_bf16_lohi(d_tmem, a_lo + a_kstep, a_hi, b_lo + 2, b_hi, idesc, 1);
+              umma_bf16_lohi(d_tmem, a_lo + 2 * a_kstep, a_hi, b_lo + 4, b_hi, idesc, 1);
+              umma_bf16_lohi(d_tmem, a_lo + 3 * a_kstep, a_hi, b_lo + 6, b_hi, idesc, 1);
+            }
+          } else {
+            for (int mt = lo; mt < hi; ++mt, a_lo += 128, d_tmem += p.C)
+              for (int ks = 0; ks < ksteps; ++ks)
+                umma_bf16_lohi(d_tmem, a_lo + ks * a_kstep, a_hi, b_lo + 2 * ks, b_hi, idesc, ks ? 1u : acc0);
+          }
+          if (tap % 3 == 2) { umma_commit(bar_empty + s); ++i; }
         }
-        umma_commit(conv == 0 ? bar_acc1 : bar_acc2);
+        umma_commit(done);
+        TS();
       }
     }
     __syncwarp();
   } else {
-    // ================================ epilogue warps (thread = pixel row of a tile) ================================
-    const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
-    const int row = warp * 32 + lane;
+    // ================ epilogue warps: thread = (pixel row of a tile, half of the channels) ================
+    const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
+    const int row = (warp & 3) * 32 + lane;
+    const int ncol = max(16, p.C / 2);
+    const int col0 = (warp >> 2) * ncol;
+    const bool has_cols = col0 < p.C;
 
-    // P3: intermediate = ReLU(acc + b1) inside the image, 0 outside -> planes
-    mbar_wait(bar_acc1, 0, abort_flag, p.status, 0x405);
-    tcgen05_fence_after_sync();
-    for (int mt = 0; mt < p.M1; ++mt) {
-      const int m = mt * 128 + row;
-      const int a = m / p.Wp, b = m - a * p.Wp;
-      const int gh = h0 - 1 + a;
-      const bool inside = m < p.P1 && gh >= 0 && gh < p.H && b >= 1 && b <= p.W;
-      for (int c0 = 0; c0 < p.C; c0 += 16) {
-        uint32_t v[16];
-        tmem_ld_x16(tmem_base + lane_base + mt * p.C + c0, v);
-        tmem_ld_wait();
-        uint32_t w[8];
-#pragma unroll
-        for (int j = 0; j < 8; ++j) {
-          const float y0 = fmaxf(__uint_as_float(v[2 * j]) + __ldg(p.b1 + c0 + 2 * j), 0.0f);
-          const float y1 = fmaxf(__uint_as_float(v[2 * j + 1]) + __ldg(p.b1 + c0 + 2 * j + 1), 0.0f);
-          w[j] = inside ? pack_bf16x2(y0, y1) : 0u;
-        }
-        if (m < p.P1 + p.Wp) {   // a little past the tile so that shifted reads of valid rows never see stale data
-          *reinterpret_cast<uint4*>(sY + (size_t)(c0 / 8) * p.y_plane + m * 16) = make_uint4(w[0], w[1], w[2], w[3]);
-          *reinterpret_cast<uint4*>(sY + (size_t)(c0 / 8 + 1) * p.y_plane + m * 16) = make_uint4(w[4], w[5], w[6], w[7]);
-        }
-      }
-    }
-    fence_proxy_async_smem();
-    tcgen05_fence_before_sync();
-    named_barrier_sync(1, kEpiThreads);
-    if (tid == 0) mbar_arrive(bar_y);
-
-    // P6: out = ReLU(acc + b2 + x)
-    mbar_wait(bar_acc2, 0, abort_flag, p.status, 0x406);
-    tcgen05_fence_after_sync();
-    for (int mt = 0; mt < p.M2; ++mt) {
-      const int m = mt * 128 + row;
-      const int r = m / p.Wp, cc = m - r * p.Wp;
-      const bool valid = r < rows_valid && cc >= 1 && cc <= p.W;
-      const size_t pix = ((size_t)n * p.H + h0 + r) * p.W + (cc - 1);
-      for (int c0 = 0; c0 < p.C; c0 += 16) {
-        uint32_t v[16];
-        tmem_ld_x16(tmem_base + lane_base + mt * p.C + c0, v);
-        tmem_ld_wait();
-        if (valid) {
-          const uint4 x0 = __ldg(reinterpret_cast<const uint4*>(p.x + pix * p.C + c0));
-          const uint4 x1 = __ldg(reinterpret_cast<const uint4*>(p.x + pix * p.C + c0 + 8));
-          const uint32_t xs[8] = {x0.x, x0.y, x0.z, x0.w, x1.x, x1.y, x1.z, x1.w};
+    // P3: intermediate = ReLU(acc + b1) inside the image, 0 outside -> planes; group A, then group B
+    for (int grp = 0; grp < 2; ++grp) {
+      TS();
+      mbar_wait(bar_acc1 + grp, 0, abort_flag, p.status, 0x405);
+      tcgen05_fence_after_sync();
+      TS();
+      for (int mt = pass_lo[grp]; mt < pass_hi[grp] && has_cols; ++mt) {
+        const int m = mt * 128 + row;
+        const int a = m / p.Wp, b = m - a * p.Wp;
+        const int gh = h0 - 1 + a;
+        const bool inside = m < p.P1 && gh >= 0 && gh < p.H && b >= 1 && b <= p.W;
+        for (int c0 = col0; c0 < col0 + ncol; c0 += 16) {
+          uint32_t v[16];
+          tmem_ld_x16(tmem_base + lane_base + mt * p.C + c0, v);
+          tmem_ld_wait();
           uint32_t w[8];
 #pragma unroll
           for (int j = 0; j < 8; ++j) {
-            const float y0 = fmaxf(__uint_as_float(v[2 * j]) + __ldg(p.b2 + c0 + 2 * j) + bf16_lo(xs[j]), 0.0f);
-            const float y1 = fmaxf(__uint_as_float(v[2 * j + 1]) + __ldg(p.b2 + c0 + 2 * j + 1) + bf16_hi(xs[j]), 0.0f);
-            w[j] = pack_bf16x2(y0, y1);
+            const float y0 = fmaxf(__uint_as_float(v[2 * j]) + sBias[c0 + 2 * j], 0.0f);
+            const float y1 = fmaxf(__uint_as_float(v[2 * j + 1]) + sBias[c0 + 2 * j + 1], 0.0f);
+            w[j] = inside ? pack_bf16x2(y0, y1) : 0u;
           }
-          *reinterpret_cast<uint4*>(p.out + pix * p.C + c0) = make_uint4(w[0], w[1], w[2], w[3]);
-          *reinterpret_cast<uint4*>(p.out + pix * p.C + c0 + 8) = make_uint4(w[4], w[5], w[6], w[7]);
+          if (m < p.P1 + p.Wp) {   // a little past the tile so that shifted reads of valid rows never see stale data
+            *reinterpret_cast<uint4*>(sY + (size_t)(c0 / 8) * p.y_plane + m * 16) = make_uint4(w[0], w[1], w[2], w[3]);
+            *reinterpret_cast<uint4*>(sY + (size_t)(c0 / 8 + 1) * p.y_plane + m * 16) = make_uint4(w[4], w[5], w[6], w[7]);
+          }
+        }
+      }
+      fence_proxy_async_smem();
+      tcgen05_fence_before_sync();
+      named_barrier_sync(1, kEpiThreads);
+      if (tid == 0) mbar_arrive(bar_y + grp);
+      TS();
+    }
+
+    // P6: out = ReLU(acc + b2 + x); the residual is fetched before waiting for the accumulators
+    const float* sB2 = sBias + p.C;
+    for (int grp = 0; grp < 2; ++grp) {
+      for (int mt = pass_lo[2 + grp]; mt < pass_hi[2 + grp] || mt == pass_lo[2 + grp]; ++mt) {
+        const bool tile_ok = mt < pass_hi[2 + grp];
+        const int m = mt * 128 + row;
+        const int r = m / p.Wp, cc = m - r * p.Wp;
+        const bool valid = tile_ok && has_cols && r < rows_valid && cc >= 1 && cc <= p.W;
+        const size_t pix = ((size_t)n * p.H + h0 + r) * p.W + (cc - 1);
+        uint4 xr[4];
+        if (valid) {
+#pragma unroll
+          for (int j = 0; j < 4; ++j)
+            if (j * 8 < ncol) xr[j] = __ldg(reinterpret_cast<const uint4*>(p.x + pix * p.C + col0 + j * 8));
+        }
+        if (mt == pass_lo[2 + grp]) {
+          TS();
+          mbar_wait(bar_acc2 + grp, 0, abort_flag, p.status, 0x406);
+          tcgen05_fence_after_sync();
+          TS();
+        }
+        if (!tile_ok) break;
+        if (has_cols) {
+          for (int c0 = col0, jj = 0; c0 < col0 + ncol; c0 += 16, jj += 2) {
+            uint32_t v[16];
+            tmem_ld_x16(tmem_base + lane_base + mt * p.C + c0, v);
+            tmem_ld_wait();
+#ifdef AGO_TIMELINE
+            if (valid && blockIdx.x != 0) {
+#else
+            if (valid) {
+#endif
+              const uint32_t xs[8] = {xr[jj].x, xr[jj].y, xr[jj].z, xr[jj].w, xr[jj + 1].x, xr[jj + 1].y, xr[jj + 1].z, xr[jj + 1].w};
+              uint32_t w[8];
+#pragma unroll
+              for (int j = 0; j < 8; ++j) {
+                const float y0 = fmaxf(__uint_as_float(v[2 * j]) + sB2[c0 + 2 * j] + bf16_lo(xs[j]), 0.0f);
+                const float y1 = fmaxf(__uint_as_float(v[2 * j + 1]) + sB2[c0 + 2 * j + 1] + bf16_hi(xs[j]), 0.0f);
+                w[j] = pack_bf16x2(y0, y1);
+              }
+              *reinterpret_cast<uint4*>(p.out + pix * p.C + c0) = make_uint4(w[0], w[1], w[2], w[3]);
+              *reinterpret_cast<uint4*>(p.out + pix * p.C + c0 + 8) = make_uint4(w[4], w[5], w[6], w[7]);
+            }
+          }
         }
       }
     }
@@ -226,20 +300,35 @@ bool conv_layout(ConvParams& q, int R, int* smem_bytes) {
   q.P1 = (R + 2) * q.Wp; q.M1 = (q.P1 + 127) / 128;
   q.P2 = R * q.Wp; q.M2 = (q.P2 + 127) / 128;
   if (q.IH > 256 || q.Wp > 256 || q.M1 * q.C > 512) return false;
-  q.x_plane = q.IH * q.Wp * 16;
-  // the intermediate planes must hold every pixel a shifted operand row can touch
-  const int y_pixels = std::max(q.P1 + q.Wp, q.M2 * 128 + 2 * q.Wp + 2) + 8;
-  q.y_plane = y_pixels * 16;
-  int off = 1024;   // slack before the input planes: tap (0,0) of pixel 0 starts one pixel early
+  // at least two pixels of slack after each plane (the aliased intermediate planes start two pixels
+  // early); every plane starts on a 128-byte boundary, which the TMA destination requires
+  q.x_plane = round_up_i(q.IH * q.Wp * 16 + 32, 128);
+  // The intermediate planes alias the input planes, shifted down by two pixels: while the second tile
+  // group of the first convolution still reads input pixels >= a1*128 - 1, the first group's epilogue
+  // writes intermediate pixels < a1*128, i.e. input slots < a1*128 - 2.
+  q.y_plane = q.x_plane;
+  int off = 1024;   // slack before the planes: shifted operand rows start up to three pixels early
   q.off_x = off;
-  const int x_reach = std::max(q.planes * q.x_plane, (q.planes - 1) * q.x_plane + (q.M1 * 128 + 2 * q.Wp + 2) * 16);
-  off = round_up_i(off + x_reach, 1024) + 1024;
-  q.off_y = off;
-  off = round_up_i(off + q.planes * q.y_plane, 1024);
+  q.off_y = off - 32;
+  const int reach_px = std::max(q.M1 * 128 + 2 * q.Wp + 2, q.P1 + q.Wp + 2);
+  const int x_reach = std::max(q.planes * q.x_plane, (q.planes - 1) * q.x_plane + reach_px * 16);
+  off = round_up_i(off + x_reach, 1024);
   q.off_w = off;
-  off += kWStages * q.w_stage_bytes;
+  q.wstages = kMaxWStages;
+  while (q.wstages > 2 && off + q.wstages * 3 * q.w_stage_bytes + 2048 + 1024 > 227 * 1024) --q.wstages;
+  off += q.wstages * 3 * q.w_stage_bytes;
+  q.off_bias = off;
+  off += 1024;
   q.off_bar = off;
   off += 256;
+  // pipeline groups: the second convolution's first group may only read intermediate rows the first
+  // group of the first convolution produces
+  q.a1 = (q.M1 * 3 + 4) / 5;
+  if (q.a1 < 1) q.a1 = 1;
+  q.a2 = (q.a1 * 128 - 2 * q.Wp - 1) / 128;
+  if (q.a2 < 0) q.a2 = 0;
+  if (q.a2 > q.M2) q.a2 = q.M2;
+  if (q.a1 >= q.M1) { q.a1 = q.M1; }
   *smem_bytes = off + 1024;
   return *smem_bytes <= 227 * 1024;
 }
@@ -295,7 +384,7 @@ ago_status_t conv3x3_run(const Plan& plan, FusedState* st, const void* const* in
       if (which == 0) {
         const uint64_t dims[5] = {8, (uint64_t)q.W, (uint64_t)q.H, (uint64_t)q.N, (uint64_t)q.planes};
         const uint64_t strides[4] = {(uint64_t)q.C * 2, (uint64_t)q.W * q.C * 2, (uint64_t)q.H * q.W * q.C * 2, 16};
-        const uint32_t box[5] = {8, (uint32_t)q.Wp, (uint32_t)q.IH, 1, (uint32_t)q.planes};
+        const uint32_t box[5] = {8, (uint32_t)q.Wp, (uint32_t)q.IH, 1, 1};   // one channel block per load
         if (!encode_tmap_bf16(&m, base, 5, dims, strides, box, 0, err)) return false;
       } else {
         const uint64_t dims[3] = {(uint64_t)q.C, 9, (uint64_t)q.C};
