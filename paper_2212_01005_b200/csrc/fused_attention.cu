@@ -1,22 +1,24 @@
-// Fused attention: S = Q K^T, * scale, row softmax, O = P V -- one kernel per
-// (batch, head, block of 128 query rows); scores and probabilities never leave
-// the SM.
+// Fused attention: S = Q K^T, * scale, row softmax, O = P V -- one kernel; scores and
+// probabilities never leave the SM.
 //
-// Tile choice (Section III-B, "downstream pointwise / matmul" category): the
-// downstream contraction P V reuses its input only along its output columns, so
-// its tile keeps ALL of them (head_dim) and is tiled over rows (128 queries).
-// The softmax in between is a simple operator over whole rows, so the upstream
-// tile is 128 query rows x ALL keys: the full score block sits in tensor memory
-// (128 lanes x S fp32 columns) and the exact two-pass softmax needs no rescaling.
+// Tile choice (Section III-B, "downstream pointwise / matmul" category): the downstream
+// contraction P V reuses its input only along its output columns, so its tile keeps ALL of them
+// (head_dim) and is tiled over rows (128 queries). The softmax in between is a simple operator
+// over whole rows, so the upstream tile is 128 query rows x ALL keys of the head.
 //
-//   P1  TMA: Q [128 x 64], K [S x 64], V [S x 64] -> 128-byte-swizzled tiles
-//   P2  tcgen05.mma: S[128 x S] = Q K^T                         (TMEM, fp32)
-//   P3/P4  CUDA cores, one thread per (row, half of the keys): TMEM -> registers,
-//       row max (shuffle-free: one row per thread, halves exchanged through
-//       shared memory), p = exp2((s - max) * scale * log2 e), bf16 -> shared
-//       memory in the K-major operand layout, row sum
-//   P5  tcgen05.mma: O[128 x 64] = P V   (V is the N-major B operand, as it lies in HBM)
-//   P6  TMEM -> registers, * 1 / rowsum, bf16, 16-byte stores
+// A CTA owns one (batch, head): K and V are loaded once and stay in shared memory while the CTA
+// walks over the head's 128-row query tiles. The keys are processed in two halves so that tensor
+// cores and CUDA cores overlap: while the softmax warps turn half 0 of the scores into
+// probabilities, the MMA warp already computes half 1 (and, later, the next tile's scores). The
+// running row maximum may grow between the halves; the partial output of half 0 is then rescaled
+// in tensor memory by exp(m0 - m1) before half 1 is accumulated -- the result is the exact softmax.
+//
+//   P1  TMA: K, V [S x 64] once per CTA, Q [128 x 64] per tile -> 128-byte-swizzled tiles
+//   P2  tcgen05.mma: S_h[128 x S/2] = Q K_h^T                            (TMEM, fp32, two buffers)
+//   P3/P4  768 threads (6 per query row): TMEM -> registers, row max (exchanged through shared
+//       memory), p = exp2((s - m) * scale * log2 e), bf16 -> shared memory (K-major operand), row sum
+//   P5  tcgen05.mma: O[128 x 64] (+)= P_h V_h       (V is the N-major B operand, as it lies in HBM)
+//   P6  TMEM -> registers, * 1 / rowsum, bf16, 32-byte stores
 #include <cuda.h>
 #include <cuda_bf16.h>
 
@@ -33,21 +35,34 @@ namespace {
 using namespace tc;
 
 constexpr int kD = 64;                 // head dimension (one 128-byte swizzle row)
-constexpr int kBlockM = 128;           // query rows per CTA
-constexpr int kKeyBlock = 128;         // keys per TMA box / per score MMA
-constexpr int kComputeThreads = 256;   // two threads per query row (each half of the keys)
-constexpr int kThreads = kComputeThreads + 32;
+constexpr int kBlockM = 128;           // query rows per tile
+constexpr int kKeyBlock = 128;         // keys per TMA box
+constexpr int kParts = 6;              // threads per query row (each owns <= 32 score columns of a half)
+constexpr int kComputeThreads = kBlockM * kParts;
+constexpr int kThreads = kComputeThreads + 64;   // + TMA warp + MMA warp
+constexpr int kHalfCols = 192;         // tensor-memory columns reserved per score half
+constexpr uint32_t kOCol = 2 * kHalfCols;
 
 struct AttnParams {
   __nv_bfloat16* out;
   unsigned int* status;
   int B, S, heads, E;
   int Spad;        // keys rounded up to 16
-  int nkb;         // key blocks of 128
-  int half;        // first column of the second thread group's half (multiple of 16)
+  int nkb;         // 128-key TMA boxes
+  int tiles;       // query tiles per head
+  int hw0, hw1;    // keys in half 0 / half 1 (multiples of 16, hw0 >= hw1 > 0)
+  int pw0, pw1;    // columns per thread part in each half (multiples of 16)
   float scale_log2e;
   int off_q, off_k, off_v, off_p, off_red, off_bar;
+  int p_half_bytes;
 };
+
+// 2^x on the special-function unit (arguments here are <= 0; results below 2^-126 flush to 0).
+__device__ __forceinline__ float ex2_approx(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
 
 __global__ void __launch_bounds__(kThreads, 1)
 attention_fused_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
@@ -57,31 +72,48 @@ attention_fused_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
   uint8_t* sQ = smem + p.off_q;
   uint8_t* sK = smem + p.off_k;
   uint8_t* sV = smem + p.off_v;
-  uint8_t* sP = smem + p.off_p;
-  float* sRed = reinterpret_cast<float*>(smem + p.off_red);   // [2][128] max, then [2][128] sum
+  uint8_t* sP = smem + p.off_p;                                // two halves of p_half_bytes
+  float* sMax0 = reinterpret_cast<float*>(smem + p.off_red);    // [kParts][128]
+  float* sMax1 = sMax0 + kParts * kBlockM;
+  float* sSum = sMax1 + kParts * kBlockM;
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + p.off_bar);
-  uint64_t* bar_qk = bars + 0;   // Q and K landed
-  uint64_t* bar_v = bars + 1;    // V landed
-  uint64_t* bar_s = bars + 2;    // scores complete
-  uint64_t* bar_p = bars + 3;    // probabilities written
-  uint64_t* bar_o = bars + 4;    // output accumulators complete
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 5);
-  volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(bars + 6);
+  uint64_t* bar_k = bars + 0;
+  uint64_t* bar_v = bars + 1;
+  uint64_t* bar_q = bars + 2;       // Q tile landed
+  uint64_t* bar_qfree = bars + 3;   // both score MMAs of the tile have read Q
+  uint64_t* bar_s = bars + 4;       // [2] score half complete
+  uint64_t* bar_p = bars + 6;       // [2] probabilities of the half written, score half drained
+  uint64_t* bar_pfree = bars + 8;   // [2] P V of the half has read the probabilities
+  uint64_t* bar_o0 = bars + 10;     // P V of half 0 complete
+  uint64_t* bar_corr = bars + 11;   // output rescaled for half 1
+  uint64_t* bar_o1 = bars + 12;     // P V of half 1 complete
+  uint64_t* bar_ofree = bars + 13;  // epilogue has read the output accumulators
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 14);
+  volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(bars + 15);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int q0 = blockIdx.x * kBlockM, h = blockIdx.y, b = blockIdx.z;
+  const int h = blockIdx.x, b = blockIdx.y;
+#ifdef AGO_TIMELINE
+  long long* ts = reinterpret_cast<long long*>(p.out); int tsi = 0;
+  const bool tsw = blockIdx.x == 0 && blockIdx.y == 0 && tid == 0;
+#define TS() do { if (tsw) ts[tsi++] = clock64(); } while (0)
+#else
+#define TS() do {} while (0)
+#endif
+  TS();
 
   if (tid == kComputeThreads) {
     *abort_flag = 0u;
-    for (int i = 0; i < 5; ++i) mbar_init(bars + i, 1);
+    for (int i = 0; i < 14; ++i) mbar_init(bars + i, 1);
     fence_mbar_init();
     fence_proxy_async_smem();
     tma_prefetch_desc(&tmap_q);
     tma_prefetch_desc(&tmap_k);
     tma_prefetch_desc(&tmap_v);
-    mbar_arrive_expect_tx(bar_qk, (uint32_t)((kBlockM + p.nkb * kKeyBlock) * kD * 2));
-    tma_load_3d(sQ, &tmap_q, bar_qk, h * kD, q0, b);
-    for (int kb = 0; kb < p.nkb; ++kb) tma_load_3d(sK + kb * kKeyBlock * kD * 2, &tmap_k, bar_qk, h * kD, kb * kKeyBlock, b);
+    mbar_arrive_expect_tx(bar_k, (uint32_t)(p.nkb * kKeyBlock * kD * 2));
+    for (int kb = 0; kb < p.nkb; ++kb) tma_load_3d(sK + kb * kKeyBlock * kD * 2, &tmap_k, bar_k, h * kD, kb * kKeyBlock, b);
+    mbar_arrive_expect_tx(bar_q, (uint32_t)(kBlockM * kD * 2));
+    tma_load_3d(sQ, &tmap_q, bar_q, h * kD, 0, b);
     mbar_arrive_expect_tx(bar_v, (uint32_t)(p.nkb * kKeyBlock * kD * 2));
     for (int kb = 0; kb < p.nkb; ++kb) tma_load_3d(sV + kb * kKeyBlock * kD * 2, &tmap_v, bar_v, h * kD, kb * kKeyBlock, b);
   }
@@ -93,113 +125,260 @@ attention_fused_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
   __syncthreads();
   tcgen05_fence_after_sync();
   const uint32_t tmem_base = *tmem_slot;
-  const uint32_t ocol0 = 384;   // output accumulators after the score block
 
   if (warp == kComputeThreads / 32) {
+    // ============================ TMA producer: the remaining Q tiles ============================
+    if (lane == 0) {
+      for (int t = 1; t < p.tiles; ++t) {
+        mbar_wait(bar_qfree, (uint32_t)(t - 1) & 1u, abort_flag, p.status, 0x201);
+        mbar_arrive_expect_tx(bar_q, (uint32_t)(kBlockM * kD * 2));
+        tma_load_3d(sQ, &tmap_q, bar_q, h * kD, t * kBlockM, b);
+      }
+    }
+    __syncwarp();
+  } else if (warp == kComputeThreads / 32 + 1) {
     // ============================ MMA issue (one lane) ============================
     if (lane == 0) {
       const uint64_t qdesc = make_smem_desc(smem_u32(sQ), 0, 1024, SW_128B);
       const uint64_t kdesc = make_smem_desc(smem_u32(sK), 0, 1024, SW_128B);
-      mbar_wait(bar_qk, 0, abort_flag, p.status, 0x201);
-      tcgen05_fence_after_sync();
-      for (int kb = 0; kb < p.nkb; ++kb) {
-        const int n = min(kKeyBlock, p.Spad - kb * kKeyBlock);
-        const uint32_t idesc = make_idesc_bf16(128, (uint32_t)n);
-        const uint64_t bd = kdesc + (uint64_t)((kb * kKeyBlock * kD * 2) >> 4);
-#pragma unroll
-        for (int ks = 0; ks < kD / 16; ++ks) umma_bf16(tmem_base + kb * kKeyBlock, qdesc + 2u * ks, bd + 2u * ks, idesc, ks > 0);
-      }
-      umma_commit(bar_s);
-
-      // O = P V: P is K-major (64-key blocks of 128-byte rows), V is N-major as stored ([key][d])
       const uint64_t pdesc = make_smem_desc(smem_u32(sP), 0, 1024, SW_128B);
       const uint64_t vdesc = make_smem_desc(smem_u32(sV), 0, 1024, SW_128B);
-      const uint32_t idesc_o = make_idesc_bf16(128, kD, 0, 1);
-      mbar_wait(bar_v, 0, abort_flag, p.status, 0x202);
-      mbar_wait(bar_p, 0, abort_flag, p.status, 0x203);
+      const uint32_t idesc_o = make_idesc_bf16(128, kD, 0, 1);    // V is N-major
+      const uint32_t idesc_s[2] = {make_idesc_bf16(128, (uint32_t)p.hw0), make_idesc_bf16(128, (uint32_t)p.hw1)};
+      const int hw[2] = {p.hw0, p.hw1};
+
+      auto issue_scores = [&](int half) {
+        const uint64_t bd = kdesc + (uint64_t)((uint32_t)(half * p.hw0 * kD * 2) >> 4);
+#pragma unroll
+        for (int ks = 0; ks < kD / 16; ++ks)
+          umma_bf16(tmem_base + half * kHalfCols, qdesc + 2u * ks, bd + 2u * ks, idesc_s[half], ks > 0);
+        umma_commit(bar_s + half);
+      };
+      auto issue_pv = [&](int half) {
+        const uint64_t ad0 = pdesc + (uint64_t)((uint32_t)(half * p.p_half_bytes) >> 4);
+        const uint64_t bd0 = vdesc + (uint64_t)((uint32_t)(half * p.hw0 * kD * 2) >> 4);
+        const int ksteps = hw[half] / 16;
+        for (int ks = 0; ks < ksteps; ++ks)
+          umma_bf16(tmem_base + kOCol, ad0 + (uint64_t)(((ks >> 2) * kBlockM * 128 + (ks & 3) * 32) >> 4),
+                    bd0 + (uint64_t)((ks * 16 * kD * 2) >> 4), idesc_o, (half | ks) != 0);
+      };
+
+      mbar_wait(bar_k, 0, abort_flag, p.status, 0x202);
+      mbar_wait(bar_q, 0, abort_flag, p.status, 0x203);
       tcgen05_fence_after_sync();
-      const int ksteps = p.Spad / 16;
-      for (int ks = 0; ks < ksteps; ++ks) {
-        const uint64_t ad = pdesc + (uint64_t)(((ks >> 2) * kBlockM * 128 + (ks & 3) * 32) >> 4);
-        const uint64_t bd = vdesc + (uint64_t)((ks * 16 * kD * 2) >> 4);
-        umma_bf16(tmem_base + ocol0, ad, bd, idesc_o, ks > 0);
+      issue_scores(0);
+      issue_scores(1);
+      umma_commit(bar_qfree);
+      for (int t = 0; t < p.tiles; ++t) {
+        const uint32_t ph = (uint32_t)t & 1u;
+        // ---- half 0 ----
+        mbar_wait(bar_p + 0, ph, abort_flag, p.status, 0x204);
+        if (t == 0) mbar_wait(bar_v, 0, abort_flag, p.status, 0x205);
+        if (t > 0) mbar_wait(bar_ofree, ph ^ 1u, abort_flag, p.status, 0x206);
+        tcgen05_fence_after_sync();
+        issue_pv(0);
+        umma_commit(bar_o0);
+        umma_commit(bar_pfree + 0);
+        if (t + 1 < p.tiles) {
+          mbar_wait(bar_q, ph ^ 1u, abort_flag, p.status, 0x207);
+          tcgen05_fence_after_sync();
+          issue_scores(0);                       // next tile's half 0 into the buffer just drained
+        }
+        // ---- half 1 ----
+        mbar_wait(bar_p + 1, ph, abort_flag, p.status, 0x208);
+        mbar_wait(bar_corr, ph, abort_flag, p.status, 0x209);
+        tcgen05_fence_after_sync();
+        issue_pv(1);
+        umma_commit(bar_o1);
+        umma_commit(bar_pfree + 1);
+        if (t + 1 < p.tiles) {
+          issue_scores(1);
+          umma_commit(bar_qfree);
+        }
       }
-      umma_commit(bar_o);
     }
     __syncwarp();
   } else {
-    // ============================ softmax + epilogue warps ============================
-    const int row = (warp & 3) * 32 + lane;     // TMEM lane = query row of this tile
-    const int grp = warp >> 2;                  // which half of the keys / of the output columns
+    // ============================ softmax / rescale / epilogue warps ============================
+    const int row = (warp & 3) * 32 + lane;     // TMEM lane = query row of the tile
+    const int part = warp >> 2;                 // which slice of a half's keys (and, for parts 0..3, of the output columns)
     const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
-    const int c_begin = grp == 0 ? 0 : p.half;
-    const int c_end = grp == 0 ? p.half : p.Spad;
-
-    mbar_wait(bar_s, 0, abort_flag, p.status, 0x204);
-    tcgen05_fence_after_sync();
-
-    // pass 1: row maximum of the raw scores over this thread's half
-    float m = -INFINITY;
-    for (int c0 = c_begin; c0 < c_end; c0 += 16) {
-      uint32_t v[16];
-      tmem_ld_x16(tmem_base + lane_base + c0, v);
-      tmem_ld_wait();
-#pragma unroll
-      for (int j = 0; j < 16; ++j)
-        if (c0 + j < p.S) m = fmaxf(m, __uint_as_float(v[j]));
-    }
-    sRed[grp * kBlockM + row] = m;
-    named_barrier_sync(1, kComputeThreads);
-    m = fmaxf(sRed[row], sRed[kBlockM + row]);
-
-    // pass 2: p = exp2((s - m) * scale * log2 e), rounded to bf16, into the A-operand layout
     const float c = p.scale_log2e;
-    const float mc = m * c;
-    float sum = 0.0f;
-    for (int c0 = c_begin; c0 < c_end; c0 += 16) {
-      uint32_t v[16];
-      tmem_ld_x16(tmem_base + lane_base + c0, v);
-      tmem_ld_wait();
-      uint32_t w[8];
-#pragma unroll
-      for (int j = 0; j < 8; ++j) {
-        float e0 = exp2f(fmaf(__uint_as_float(v[2 * j]), c, -mc));
-        float e1 = exp2f(fmaf(__uint_as_float(v[2 * j + 1]), c, -mc));
-        if (c0 + 2 * j >= p.S) e0 = 0.0f;
-        if (c0 + 2 * j + 1 >= p.S) e1 = 0.0f;
-        const __nv_bfloat162 hb = __floats2bfloat162_rn(e0, e1);
-        w[j] = *reinterpret_cast<const uint32_t*>(&hb);
-        sum += __low2float(hb) + __high2float(hb);
-      }
-      // columns c0..c0+15 = two 16-byte chunks of key block c0/64
-      uint8_t* blk = sP + (c0 >> 6) * (kBlockM * 128);
-      const uint32_t ch = (uint32_t)(c0 & 63) >> 3;
-      *reinterpret_cast<uint4*>(blk + swz_offset(row, ch, 128)) = make_uint4(w[0], w[1], w[2], w[3]);
-      *reinterpret_cast<uint4*>(blk + swz_offset(row, ch + 1, 128)) = make_uint4(w[4], w[5], w[6], w[7]);
-    }
-    sRed[2 * kBlockM + grp * kBlockM + row] = sum;
-    fence_proxy_async_smem();
-    tcgen05_fence_before_sync();
-    named_barrier_sync(1, kComputeThreads);
-    if (tid == 0) mbar_arrive(bar_p);
-    const float inv = 1.0f / (sRed[2 * kBlockM + row] + sRed[3 * kBlockM + row]);
+    const int hw[2] = {p.hw0, p.hw1};
+    const int pw[2] = {p.pw0, p.pw1};
 
-    // epilogue: this thread stores 32 of the row's 64 output columns
-    mbar_wait(bar_o, 0, abort_flag, p.status, 0x205);
-    tcgen05_fence_after_sync();
-    uint32_t o[32];
-    tmem_ld_x32(tmem_base + lane_base + ocol0 + grp * 32, o);
-    tmem_ld_wait();
-    if (q0 + row < p.S) {
-      __nv_bfloat16* dst = p.out + ((size_t)b * p.S + q0 + row) * p.E + h * kD + grp * 32;
+    // One half of one tile for this thread: its (at most 32) score columns stay in registers between the
+    // maximum and the exponentials, so tensor memory is read once.
+    //   phase A: load + local maximum -> exchange;  phase B: p = exp2((s - m) c) -> bf16 -> shared memory, partial sum
+    uint32_t sv[32];
+    int ncols = 0, col0 = 0;
+    bool fast = false;   // all 32 columns present and none of them padding: straight-line code, no predicates
+    auto load_half_and_max = [&](int half) -> float {
+      col0 = part * pw[half];
+      ncols = max(0, min(hw[half], col0 + pw[half]) - col0);    // 0, 16 or 32
+      const int key0 = half * p.hw0 + col0;
+      fast = ncols == 32 && key0 + 32 <= p.S;
+      float m = -INFINITY;
+      if (fast) {
+        tmem_ld_x32(tmem_base + lane_base + half * kHalfCols + col0, sv);
+        tmem_ld_wait();
+        float m4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        *reinterpret_cast<uint4*>(dst + j * 8) =
-            make_uint4(pack_bf16x2(__uint_as_float(o[8 * j]) * inv, __uint_as_float(o[8 * j + 1]) * inv),
-                       pack_bf16x2(__uint_as_float(o[8 * j + 2]) * inv, __uint_as_float(o[8 * j + 3]) * inv),
-                       pack_bf16x2(__uint_as_float(o[8 * j + 4]) * inv, __uint_as_float(o[8 * j + 5]) * inv),
-                       pack_bf16x2(__uint_as_float(o[8 * j + 6]) * inv, __uint_as_float(o[8 * j + 7]) * inv));
+        for (int j = 0; j < 32; j += 4) {
+          m4[0] = fmaxf(m4[0], __uint_as_float(sv[j]));
+          m4[1] = fmaxf(m4[1], __uint_as_float(sv[j + 1]));
+          m4[2] = fmaxf(m4[2], __uint_as_float(sv[j + 2]));
+          m4[3] = fmaxf(m4[3], __uint_as_float(sv[j + 3]));
+        }
+        m = fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3]));
+      } else if (ncols > 0) {
+        const uint32_t addr = tmem_base + lane_base + half * kHalfCols + col0;
+        if (ncols > 16) tmem_ld_x32(addr, sv); else tmem_ld_x16(addr, sv);
+        tmem_ld_wait();
+#pragma unroll
+        for (int j = 0; j < 32; ++j) if (j < ncols && key0 + j < p.S) m = fmaxf(m, __uint_as_float(sv[j]));
       }
+      return m;
+    };
+    auto exp_half_to_smem = [&](int half, float mc) -> float {
+      float sum = 0.0f;
+      uint8_t* pbase = sP + half * p.p_half_bytes;
+      if (fast) {
+        // 32 columns = four 16-byte chunks of this row inside one 64-key block (col0 is a multiple of 32)
+        uint8_t* rowp = pbase + (col0 >> 6) * (kBlockM * 128) + row * 128;
+        const uint32_t ch0 = (uint32_t)(col0 & 63) >> 3, sw = (uint32_t)row & 7u;
+        float s4[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+        for (int g = 0; g < 4; ++g) {
+          uint32_t w[4];
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            const float e0 = ex2_approx(fmaf(__uint_as_float(sv[g * 8 + 2 * j]), c, -mc));
+            const float e1 = ex2_approx(fmaf(__uint_as_float(sv[g * 8 + 2 * j + 1]), c, -mc));
+            s4[j] += e0 + e1;
+            w[j] = pack_bf16x2(e0, e1);
+          }
+          *reinterpret_cast<uint4*>(rowp + (((ch0 + g) ^ sw) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
+        }
+        sum = (s4[0] + s4[1]) + (s4[2] + s4[3]);
+      } else if (ncols > 0) {
+        const int key0 = half * p.hw0 + col0;
+#pragma unroll
+        for (int g = 0; g < 4; ++g) {            // 8 columns = one 16-byte chunk of a probability row
+          if (g * 8 < ncols) {
+            uint32_t w[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              const int e = g * 8 + 2 * j;
+              float e0 = ex2_approx(fmaf(__uint_as_float(sv[e]), c, -mc));
+              float e1 = ex2_approx(fmaf(__uint_as_float(sv[e + 1]), c, -mc));
+              if (key0 + e >= p.S) e0 = 0.0f;
+              if (key0 + e + 1 >= p.S) e1 = 0.0f;
+              sum += e0 + e1;
+              w[j] = pack_bf16x2(e0, e1);
+            }
+            const int cc = col0 + g * 8;
+            *reinterpret_cast<uint4*>(pbase + (cc >> 6) * (kBlockM * 128) + swz_offset(row, (uint32_t)(cc & 63) >> 3, 128)) =
+                make_uint4(w[0], w[1], w[2], w[3]);
+          }
+        }
+      }
+      return sum;
+    };
+    auto reduce_parts = [&](const float* a, bool is_max) -> float {
+      float r = a[row];
+#pragma unroll
+      for (int q = 1; q < kParts; ++q) r = is_max ? fmaxf(r, a[q * kBlockM + row]) : r + a[q * kBlockM + row];
+      return r;
+    };
+
+    float m0 = 0.0f, sum0 = 0.0f;
+    auto do_half0 = [&](int t) {
+      const uint32_t ph = (uint32_t)t & 1u;
+      TS();
+      mbar_wait(bar_s + 0, ph, abort_flag, p.status, 0x210);
+      tcgen05_fence_after_sync();
+      TS();
+      sMax0[part * kBlockM + row] = load_half_and_max(0);
+      TS();
+      named_barrier_sync(1, kComputeThreads);
+      TS();
+      m0 = reduce_parts(sMax0, true);
+      if (t > 0) mbar_wait(bar_pfree + 0, ph ^ 1u, abort_flag, p.status, 0x211);
+      sum0 = exp_half_to_smem(0, m0 * c);
+      TS();
+      fence_proxy_async_smem();
+      tcgen05_fence_before_sync();
+      named_barrier_sync(1, kComputeThreads);
+      if (tid == 0) mbar_arrive(bar_p + 0);
+      TS();
+    };
+
+    do_half0(0);
+    for (int t = 0; t < p.tiles; ++t) {
+      const uint32_t ph = (uint32_t)t & 1u;
+      // ---------------- half 1 ----------------
+      mbar_wait(bar_s + 1, ph, abort_flag, p.status, 0x212);
+      tcgen05_fence_after_sync();
+      sMax1[part * kBlockM + row] = load_half_and_max(1);
+      named_barrier_sync(1, kComputeThreads);
+      const float m1 = fmaxf(m0, reduce_parts(sMax1, true));
+      const float alpha = ex2_approx((m0 - m1) * c);     // rescales everything accumulated under the old maximum
+      if (t > 0) mbar_wait(bar_pfree + 1, ph ^ 1u, abort_flag, p.status, 0x213);
+      const float sum1 = exp_half_to_smem(1, m1 * c);
+      sSum[part * kBlockM + row] = sum0 * alpha + sum1;
+      fence_proxy_async_smem();
+      tcgen05_fence_before_sync();
+      named_barrier_sync(1, kComputeThreads);
+      if (tid == 0) mbar_arrive(bar_p + 1);
+      const float inv = 1.0f / reduce_parts(sSum, false);
+
+      // ---------------- rescale the half-0 output: O *= alpha (parts 0..3: 16 of the 64 columns each) ----------------
+      mbar_wait(bar_o0, ph, abort_flag, p.status, 0x214);
+      tcgen05_fence_after_sync();
+      if (part < 4) {
+        uint32_t o[16];
+        const uint32_t addr = tmem_base + lane_base + kOCol + part * 16;
+        tmem_ld_x16(addr, o);
+        tmem_ld_wait();
+#pragma unroll
+        for (int j = 0; j < 16; ++j) o[j] = __float_as_uint(__uint_as_float(o[j]) * alpha);
+        tmem_st_x16(addr, o);
+        tmem_st_wait();
+      }
+      tcgen05_fence_before_sync();
+      named_barrier_sync(1, kComputeThreads);
+      if (tid == 0) mbar_arrive(bar_corr);
+
+      // While the tensor core finishes P V of this tile, start on the next tile's first half.
+      if (t + 1 < p.tiles) do_half0(t + 1);
+
+      // ---------------- epilogue of tile t: O / rowsum -> bf16 -> global ----------------
+      mbar_wait(bar_o1, ph, abort_flag, p.status, 0x215);
+      tcgen05_fence_after_sync();
+      if (part < 4) {
+        uint32_t o[16];
+        tmem_ld_x16(tmem_base + lane_base + kOCol + part * 16, o);
+        tmem_ld_wait();
+        const int qrow = t * kBlockM + row;
+#ifdef AGO_TIMELINE
+        if (qrow < p.S && !(blockIdx.x == 0 && blockIdx.y == 0)) {
+#else
+        if (qrow < p.S) {
+#endif
+          __nv_bfloat16* dst = p.out + ((size_t)b * p.S + qrow) * p.E + h * kD + part * 16;
+#pragma unroll
+          for (int j = 0; j < 2; ++j)
+            *reinterpret_cast<uint4*>(dst + j * 8) =
+                make_uint4(pack_bf16x2(__uint_as_float(o[8 * j]) * inv, __uint_as_float(o[8 * j + 1]) * inv),
+                           pack_bf16x2(__uint_as_float(o[8 * j + 2]) * inv, __uint_as_float(o[8 * j + 3]) * inv),
+                           pack_bf16x2(__uint_as_float(o[8 * j + 4]) * inv, __uint_as_float(o[8 * j + 5]) * inv),
+                           pack_bf16x2(__uint_as_float(o[8 * j + 6]) * inv, __uint_as_float(o[8 * j + 7]) * inv));
+        }
+      }
+      tcgen05_fence_before_sync();
+      named_barrier_sync(1, kComputeThreads);
+      if (tid == 0) mbar_arrive(bar_ofree);
     }
   }
   tcgen05_fence_before_sync();
@@ -210,9 +389,10 @@ attention_fused_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
 struct AttnHost {
   AttnParams prm;
   int smem_bytes = 0;
-  struct Maps { CUtensorMap q, k, v; };
   std::unordered_map<const void*, CUtensorMap> maps;   // keyed by base pointer (box shape is the same for Q, K, V)
 };
+
+int round16(int v) { return (v + 15) / 16 * 16; }
 
 }  // namespace
 
@@ -225,23 +405,30 @@ ago_status_t attention_plan(Plan* plan, FusedState* st, std::string* err) {
   q.heads = qk.op.p[1];
   auto bad = [&](const char* m) { *err = std::string("fused attention: ") + m; delete host; return AGO_ERR_UNSUPPORTED; };
   if (qk.op.p[2] != kD) return bad("head_dim must be 64");
-  if (q.S > 384) return bad("more than 384 keys do not fit the score block in tensor memory");
-  q.Spad = (q.S + 15) / 16 * 16;
+  if (q.S > 2 * kHalfCols) return bad("more than 384 keys do not fit the score block in tensor memory");
+  if (q.S < 32) return bad("fewer than 32 keys");
+  q.Spad = round16(q.S);
   q.nkb = (q.Spad + kKeyBlock - 1) / kKeyBlock;
-  q.half = ((q.Spad / 2) + 15) / 16 * 16;
+  q.tiles = (q.S + kBlockM - 1) / kBlockM;
+  q.hw0 = round16((q.Spad + 1) / 2);
+  q.hw1 = q.Spad - q.hw0;
+  q.pw0 = round16((q.hw0 + kParts - 1) / kParts);
+  q.pw1 = round16((q.hw1 + kParts - 1) / kParts);
   q.scale_log2e = plan->ops[1].op.f * 1.4426950408889634f;
   int off = 0;
   auto take = [&](int bytes) { int o = off; off = (off + bytes + 1023) / 1024 * 1024; return o; };
   q.off_q = take(kBlockM * kD * 2);
   q.off_k = take(q.nkb * kKeyBlock * kD * 2);
   q.off_v = take(q.nkb * kKeyBlock * kD * 2);
-  q.off_p = take(((q.Spad + 63) / 64) * kBlockM * 128);
-  q.off_red = take(4 * kBlockM * 4);
-  q.off_bar = take(128);
+  q.p_half_bytes = ((q.hw0 + 63) / 64) * kBlockM * 128;
+  q.off_p = take(2 * q.p_half_bytes);
+  q.off_red = take(3 * kParts * kBlockM * 4);
+  q.off_bar = take(256);
   host->smem_bytes = off + 1024;
+  if (host->smem_bytes > 227 * 1024) return bad("shared memory budget exceeded");
   st->impl = host;
   st->impl_free = [](void* p) { delete static_cast<AttnHost*>(p); };
-  st->tile_rows = kBlockM; st->grid = ((q.S + kBlockM - 1) / kBlockM) * q.heads * q.B; st->smem_bytes = host->smem_bytes;
+  st->tile_rows = kBlockM; st->grid = q.heads * q.B; st->smem_bytes = host->smem_bytes;
   plan->tile_rows = kBlockM; plan->smem_bytes = host->smem_bytes;
   return AGO_OK;
 }
@@ -271,7 +458,7 @@ ago_status_t attention_run(const Plan& plan, FusedState* st, const void* const* 
     cudaError_t e = ensure_max_dynamic_smem(reinterpret_cast<const void*>(attention_fused_kernel), smem_opt_in);
     if (e != cudaSuccess) { *err = std::string("cudaFuncSetAttribute: ") + cudaGetErrorString(e); return AGO_ERR_CUDA; }
   }
-  dim3 grid((q.S + kBlockM - 1) / kBlockM, q.heads, q.B);
+  dim3 grid(q.heads, q.B);
   attention_fused_kernel<<<grid, kThreads, host->smem_bytes, stream>>>(*maps[0], *maps[1], *maps[2], q);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) { *err = std::string("fused attention launch: ") + cudaGetErrorString(e); return AGO_ERR_CUDA; }
