@@ -93,14 +93,6 @@ attention_fused_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int h = blockIdx.x, b = blockIdx.y;
-#ifdef AGO_TIMELINE
-  long long* ts = reinterpret_cast<long long*>(p.out); int tsi = 0;
-  const bool tsw = blockIdx.x == 0 && blockIdx.y == 0 && tid == 0;
-#define TS() do { if (tsw) ts[tsi++] = clock64(); } while (0)
-#else
-#define TS() do {} while (0)
-#endif
-  TS();
 
   if (tid == kComputeThreads) {
     *abort_flag = 0u;
@@ -295,23 +287,17 @@ attention_fused_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
     float m0 = 0.0f, sum0 = 0.0f;
     auto do_half0 = [&](int t) {
       const uint32_t ph = (uint32_t)t & 1u;
-      TS();
       mbar_wait(bar_s + 0, ph, abort_flag, p.status, 0x210);
       tcgen05_fence_after_sync();
-      TS();
       sMax0[part * kBlockM + row] = load_half_and_max(0);
-      TS();
       named_barrier_sync(1, kComputeThreads);
-      TS();
       m0 = reduce_parts(sMax0, true);
       if (t > 0) mbar_wait(bar_pfree + 0, ph ^ 1u, abort_flag, p.status, 0x211);
       sum0 = exp_half_to_smem(0, m0 * c);
-      TS();
       fence_proxy_async_smem();
       tcgen05_fence_before_sync();
       named_barrier_sync(1, kComputeThreads);
       if (tid == 0) mbar_arrive(bar_p + 0);
-      TS();
     };
 
     do_half0(0);
@@ -361,11 +347,7 @@ attention_fused_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
         tmem_ld_x16(tmem_base + lane_base + kOCol + part * 16, o);
         tmem_ld_wait();
         const int qrow = t * kBlockM + row;
-#ifdef AGO_TIMELINE
-        if (qrow < p.S && !(blockIdx.x == 0 && blockIdx.y == 0)) {
-#else
         if (qrow < p.S) {
-#endif
           __nv_bfloat16* dst = p.out + ((size_t)b * p.S + qrow) * p.E + h * kD + part * 16;
 #pragma unroll
           for (int j = 0; j < 2; ++j)

@@ -77,14 +77,6 @@ conv3x3_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
   volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(bar_acc1 + 7);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-#ifdef AGO_TIMELINE
-  long long* ts = reinterpret_cast<long long*>(p.out) + (tid == 0 ? 0 : (tid == kEpiThreads ? 64 : 128)); int tsi = 0;
-  const bool tsw = blockIdx.x == 0 && (tid == 0 || tid == kEpiThreads || tid == kEpiThreads + 32);
-#define TS() do { if (tsw) ts[tsi++] = clock64(); } while (0)
-#else
-#define TS() do {} while (0)
-#endif
-  TS();
   const int n = blockIdx.x / p.strips, strip = blockIdx.x % p.strips;
   const int h0 = strip * p.R;
   const int rows_valid = min(p.R, p.H - h0);
@@ -137,15 +129,12 @@ conv3x3_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
     if (lane == 0) {
       const uint32_t idesc = make_idesc_bf16(128, (uint32_t)p.C);
       const uint64_t wdesc0 = make_smem_desc(smem_u32(sW), 0, 8u * p.w_row_bytes, p.w_swizzle);
-      TS();
       mbar_wait(bar_x, 0, abort_flag, p.status, 0x402);
-      TS();
       int i = 0;
       for (int ps = 0; ps < 4; ++ps) {
         const int conv = ps >> 1, grp = ps & 1;
         uint64_t* done = (conv == 0 ? bar_acc1 : bar_acc2) + grp;
         if (conv == 1) mbar_wait(bar_y + grp, 0, abort_flag, p.status, 0x403);   // the planes this group reads are written
-        TS();
         if (pass_lo[ps] >= pass_hi[ps]) { umma_commit(done); continue; }
         const uint32_t plane = (uint32_t)(conv == 0 ? p.x_plane : p.y_plane);
         // A: planes [channel block][pixel][16 B]; K step = two planes (LBO), 8-pixel groups are 128 B apart (SBO).
@@ -182,7 +171,6 @@ conv3x3_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
           if (tap % 3 == 2) { umma_commit(bar_empty + s); ++i; }
         }
         umma_commit(done);
-        TS();
       }
     }
     __syncwarp();
@@ -196,10 +184,8 @@ conv3x3_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
 
     // P3: intermediate = ReLU(acc + b1) inside the image, 0 outside -> planes; group A, then group B
     for (int grp = 0; grp < 2; ++grp) {
-      TS();
       mbar_wait(bar_acc1 + grp, 0, abort_flag, p.status, 0x405);
       tcgen05_fence_after_sync();
-      TS();
       for (int mt = pass_lo[grp]; mt < pass_hi[grp] && has_cols; ++mt) {
         const int m = mt * 128 + row;
         const int a = m / p.Wp, b = m - a * p.Wp;
@@ -226,7 +212,6 @@ conv3x3_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
       tcgen05_fence_before_sync();
       named_barrier_sync(1, kEpiThreads);
       if (tid == 0) mbar_arrive(bar_y + grp);
-      TS();
     }
 
     // P6: out = ReLU(acc + b2 + x); the residual is fetched before waiting for the accumulators
@@ -245,10 +230,8 @@ conv3x3_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
             if (j * 8 < ncol) xr[j] = __ldg(reinterpret_cast<const uint4*>(p.x + pix * p.C + col0 + j * 8));
         }
         if (mt == pass_lo[2 + grp]) {
-          TS();
           mbar_wait(bar_acc2 + grp, 0, abort_flag, p.status, 0x406);
           tcgen05_fence_after_sync();
-          TS();
         }
         if (!tile_ok) break;
         if (has_cols) {
@@ -256,11 +239,7 @@ conv3x3_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
             uint32_t v[16];
             tmem_ld_x16(tmem_base + lane_base + mt * p.C + c0, v);
             tmem_ld_wait();
-#ifdef AGO_TIMELINE
-            if (valid && blockIdx.x != 0) {
-#else
             if (valid) {
-#endif
               const uint32_t xs[8] = {xr[jj].x, xr[jj].y, xr[jj].z, xr[jj].w, xr[jj + 1].x, xr[jj + 1].y, xr[jj + 1].z, xr[jj + 1].w};
               uint32_t w[8];
 #pragma unroll

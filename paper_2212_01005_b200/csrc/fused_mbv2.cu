@@ -70,15 +70,8 @@ __device__ __forceinline__ uint32_t relu6_pack(float a, float b) {
   return *reinterpret_cast<const uint32_t*>(&h);
 }
 __device__ __forceinline__ float2 bf16x2_to_f2(uint32_t w) { return make_float2(bf16_lo(w), bf16_hi(w)); }
-#ifdef AGO_SCALAR_FMA
-__device__ __forceinline__ float2 fma2(float2 a, float2 b, float2 c) { return make_float2(fmaf(a.x, b.x, c.x), fmaf(a.y, b.y, c.y)); }
-#else
 __device__ __forceinline__ float2 fma2(float2 a, float2 b, float2 c) { return __ffma2_rn(a, b, c); }
-#endif
 
-// Depthwise 3x3 over the resident E chunk for one (channel pair, output column)
-// and output rows [r0, r1): E and D chunks are two planes of [pixel][8 channels]
-// (16 bytes per pixel), which is also the un-swizzled K-major operand layout.
 __device__ __forceinline__ uint32_t lds32(uint32_t saddr) {
   uint32_t v;
   asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(saddr));
@@ -158,14 +151,6 @@ mbv2_fused_kernel(const __grid_constant__ CUtensorMap tmap_x, const Mbv2Params p
   volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(bars + 11);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-#ifdef AGO_TIMELINE
-  long long* ts = reinterpret_cast<long long*>(p.out) + (tid == 0 ? 0 : 512); int tsi = 0;
-  const bool tsw = blockIdx.x == 0 && (tid == 0 || tid == kComputeThreads);
-#define TS() do { if (tsw) ts[tsi++] = clock64(); } while (0)
-#else
-#define TS() do {} while (0)
-#endif
-  TS();
   const int n = blockIdx.x / p.strips, strip = blockIdx.x % p.strips;
   const int ho0 = strip * p.R;
   const int rows_valid = min(p.R, p.Ho - ho0);
@@ -224,35 +209,26 @@ mbv2_fused_kernel(const __grid_constant__ CUtensorMap tmap_x, const Mbv2Params p
         }
         umma_commit(bar_e + b);
       };
-
-      TS();
       mbar_wait(bar_w, 0, abort_flag, p.status, 0x100);
-      TS();
       mbar_wait(bar_x, 0, abort_flag, p.status, 0x101);
-      TS();
       tcgen05_fence_after_sync();
       issue_expand(0);
       if (p.NC > 1) issue_expand(1);
-      TS();
       for (int c = 0; c < p.NC; ++c) {
         const int b = c & 1;
         const uint32_t ph = (uint32_t)(c >> 1) & 1u;
         if (c + 2 < p.NC) {
           mbar_wait(bar_tfree + b, ph, abort_flag, p.status, 0x105);
-          TS();
           tcgen05_fence_after_sync();
           issue_expand(c + 2);
-          TS();
         }
         mbar_wait(bar_dready + b, ph, abort_flag, p.status, 0x106);
-        TS();
         tcgen05_fence_after_sync();
         const uint64_t bdesc = w3desc0 + (uint64_t)((c * p.Coutp * kChunkRowBytes) >> 4);
         for (int t = iw; t < p.M2; t += kIssuers)
           umma_bf16(tmem_base + p.pcol0 + t * p.Coutp, ddesc0 + (uint64_t)((b * d_bytes + t * 128 * 16) >> 4), bdesc,
                     idesc_p, c > 0);
         umma_commit(bar_d + b);
-        TS();
       }
     }
     __syncwarp();
@@ -281,7 +257,6 @@ mbv2_fused_kernel(const __grid_constant__ CUtensorMap tmap_x, const Mbv2Params p
     fence_proxy_async_smem();
     named_barrier_sync(1, kComputeThreads);
     if (ctid == 0) mbar_arrive(bar_w);
-    TS();
 
     const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
     // Depthwise work split: thread = (channel pair, slot); a slot walks one output column of one row group.
@@ -307,10 +282,8 @@ mbv2_fused_kernel(const __grid_constant__ CUtensorMap tmap_x, const Mbv2Params p
 
     for (int c = 0; c < p.NC; ++c) {
       const int b = c & 1;
-      TS();
       mbar_wait(bar_e + b, (uint32_t)(c >> 1) & 1u, abort_flag, p.status, 0x102);
       tcgen05_fence_after_sync();
-      TS();
 
       // ---- P3: expand epilogue -> E chunk: + b1, ReLU6, zero outside the image, bf16 ----
       for (int t = warp >> 2, k = 0; t < p.M1; t += kComputeWarps / 4, ++k) {
@@ -339,11 +312,9 @@ mbv2_fused_kernel(const __grid_constant__ CUtensorMap tmap_x, const Mbv2Params p
       tcgen05_fence_before_sync();
       named_barrier_sync(1, kComputeThreads);
       if (ctid == 0) mbar_arrive(bar_tfree + b);
-      TS();
 
       // D[b] was read by the project MMA of chunk c-2
       if (c >= 2) mbar_wait(bar_d + b, (uint32_t)((c - 2) >> 1) & 1u, abort_flag, p.status, 0x103);
-      TS();
 
       // ---- P4: depthwise 3x3 + bias + ReLU6 on CUDA cores: E chunk -> D[b] (A operand of the project GEMM) ----
       {
@@ -354,11 +325,7 @@ mbv2_fused_kernel(const __grid_constant__ CUtensorMap tmap_x, const Mbv2Params p
         const float2 bias = *reinterpret_cast<const float2*>(sBd + ch);
         const uint32_t e_plane = smem_u32(sE) + (uint32_t)((cp >> 2) * p.e_plane + cp_off);
         const uint32_t d_plane = smem_u32(sD) + (uint32_t)(b * d_bytes + (cp >> 2) * p.d_plane + cp_off);
-#ifdef AGO_DW_NOITEMS
-        for (int item = slot; item < 0; item += kSlots) {
-#else
         for (int item = slot; item < dw_items; item += kSlots) {
-#endif
           int g = item0_g, wo = item0_wo;
           if (item != slot) { g = item / p.Wo; wo = item - g * p.Wo; }
           const int r0 = g * rows_per_group, r1 = min(rows_valid, r0 + rows_per_group);
@@ -368,12 +335,9 @@ mbv2_fused_kernel(const __grid_constant__ CUtensorMap tmap_x, const Mbv2Params p
             depthwise_column<2>(e_plane + wo * 32, d_plane + wo * 16, r0, r1, p.IW, p.Wo, wgt, bias);
         }
       }
-#ifndef AGO_DW_NOFENCE
       fence_proxy_async_smem();
-#endif
       named_barrier_sync(1, kComputeThreads);
       if (ctid == 0) mbar_arrive(bar_dready + b);
-      TS();
     }
 
     // ---- P6: project epilogue: + b3 (+ residual), bf16, 16-byte stores ----
@@ -383,9 +347,6 @@ mbv2_fused_kernel(const __grid_constant__ CUtensorMap tmap_x, const Mbv2Params p
       tcgen05_fence_after_sync();
       const int valid_pix = rows_valid * p.Wo;
       const size_t gpix0 = ((size_t)n * p.Ho + ho0) * p.Wo;
-#ifdef AGO_TIMELINE
-      if (blockIdx.x != 0)
-#endif
       for (int t = warp >> 2; t < p.M2; t += kComputeWarps / 4) {
         const int po = t * 128 + (warp & 3) * 32 + lane;
         for (int j0 = 0; j0 < p.Coutp; j0 += 16) {
