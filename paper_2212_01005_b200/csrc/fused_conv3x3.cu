@@ -9,17 +9,19 @@
 // neighbouring strips) from R + 4 input rows.
 //
 // Both convolutions are implicit GEMMs on tcgen05: the activation tile sits in
-// shared memory as [channel block of 8][pixel][16 bytes] -- the un-swizzled
-// K-major operand layout -- with pixels linearised over the PADDED width, so the
-// operand of filter tap (dr, dc) is the same matrix at a start address shifted
-// by (dr * Wp + dc - 1) pixels. Weights stream through a TMA ring, one
-// [O x I] tap at a time.
+// shared memory as [pixel][channels] rows in the swizzled K-major operand layout
+// (exactly what one TMA box load produces), with pixels linearised over the
+// PADDED width, so the operand of filter tap (dr, dc) is the same matrix at a
+// start address shifted by (dr * Wp + dc - 1) rows. The swizzle is a function of
+// the absolute shared-memory address, so such row-shifted start addresses are
+// valid operands (verified on the device against a known matrix). Weights stream
+// through a TMA ring, one filter row (3 taps) per stage.
 //
-//   P1  TMA (5-d map): input strip with halo -> channel-block planes, zero outside the image
+//   P1  TMA: input strip with halo -> swizzled [pixel][channel] rows, zero outside the image
 //   P2  tcgen05.mma: 9 taps x (I / 16) K-steps per 128-pixel tile            (TMEM)
 //   P3  TMEM -> registers: + b1, ReLU, zero outside the image (the second
-//       convolution pads the post-activation tensor), bf16 -> planes in shared memory
-//   P5  tcgen05.mma: second convolution over the resident planes             (TMEM)
+//       convolution pads the post-activation tensor), bf16 -> swizzled rows in shared memory
+//   P5  tcgen05.mma: second convolution over the resident rows               (TMEM)
 //   P6  TMEM -> registers: + b2 + x, ReLU, bf16, 16-byte stores
 #include <cuda.h>
 #include <cuda_bf16.h>
@@ -50,10 +52,8 @@ struct ConvParams {
   int N, H, W, C;          // C = input = middle = output channels
   int R, strips, IH, Wp, P1, M1, P2, M2;
   int a1, a2;              // tiles [0,a1) of conv1 / [0,a2) of conv2 form the first pipeline group
-  int planes;              // C / 8
   int w_row_bytes, w_swizzle, w_stage_bytes;
   int wstages;             // ring stages in use (2..kMaxWStages)
-  int x_plane, y_plane;    // bytes between channel-block planes of the input / intermediate tile
   int off_x, off_y, off_w, off_bias, off_bar;
 };
 
@@ -62,8 +62,8 @@ conv3x3_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
                     const __grid_constant__ CUtensorMap tmap_w2, const ConvParams p) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  uint8_t* sX = smem + p.off_x;   // first pixel of plane 0 (one pixel of slack lies before it)
-  uint8_t* sY = smem + p.off_y;   // the intermediate planes reuse the input planes' memory, two pixels lower
+  uint8_t* sX = smem + p.off_x;   // first pixel row (1024-aligned; slack lies before it)
+  uint8_t* sY = smem + p.off_y;   // the intermediate rows reuse the input rows' memory, two pixels lower
   uint8_t* sW = smem + p.off_w;
   float* sBias = reinterpret_cast<float*>(smem + p.off_bias);   // b1[C], b2[C]
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + p.off_bar);
@@ -71,7 +71,7 @@ conv3x3_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
   uint64_t* bar_full = bars + 1;                  // [kMaxWStages] filter row landed
   uint64_t* bar_empty = bars + 1 + kMaxWStages;   // [kMaxWStages] filter row consumed
   uint64_t* bar_acc1 = bars + 1 + 2 * kMaxWStages;   // [2] first convolution, tile group g complete
-  uint64_t* bar_y = bar_acc1 + 2;                 // [2] intermediate planes of group g written
+  uint64_t* bar_y = bar_acc1 + 2;                 // [2] intermediate rows of group g written
   uint64_t* bar_acc2 = bar_acc1 + 4;              // [2] second convolution, tile group g complete
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bar_acc1 + 6);
   volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(bar_acc1 + 7);
@@ -90,8 +90,8 @@ conv3x3_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
     fence_mbar_init();
     fence_proxy_async_smem();
     tma_prefetch_desc(&tmap_x);
-    mbar_arrive_expect_tx(bar_x, (uint32_t)(p.planes * p.IH * p.Wp * 16));
-    for (int k = 0; k < p.planes; ++k) tma_load_5d(sX + (size_t)k * p.x_plane, &tmap_x, bar_x, 0, -1, h0 - 2, n, k);
+    mbar_arrive_expect_tx(bar_x, (uint32_t)(p.IH * p.Wp * p.w_row_bytes));
+    tma_load_4d(sX, &tmap_x, bar_x, 0, -1, h0 - 2, n);
   }
   if (warp == 0) {
     tmem_alloc(tmem_slot, 512);
@@ -134,13 +134,13 @@ conv3x3_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
       for (int ps = 0; ps < 4; ++ps) {
         const int conv = ps >> 1, grp = ps & 1;
         uint64_t* done = (conv == 0 ? bar_acc1 : bar_acc2) + grp;
-        if (conv == 1) mbar_wait(bar_y + grp, 0, abort_flag, p.status, 0x403);   // the planes this group reads are written
+        if (conv == 1) mbar_wait(bar_y + grp, 0, abort_flag, p.status, 0x403);   // the intermediate rows this group reads are written
         if (pass_lo[ps] >= pass_hi[ps]) { umma_commit(done); continue; }
-        const uint32_t plane = (uint32_t)(conv == 0 ? p.x_plane : p.y_plane);
-        // A: planes [channel block][pixel][16 B]; K step = two planes (LBO), 8-pixel groups are 128 B apart (SBO).
+        // A: swizzled [pixel][channel] rows; K step = 32 bytes inside a row, 8-row groups are 8 rows apart (SBO).
         // Descriptor arithmetic is hoisted: one add per tile, constant strides per K step.
-        const uint64_t adesc0 = make_smem_desc(smem_u32(conv == 0 ? sX : sY), plane, 128, SW_NONE);
-        const uint32_t a_kstep = (2u * plane) >> 4;
+        const uint32_t rowu = (uint32_t)p.w_row_bytes >> 4;   // one pixel row in 16-byte units
+        const uint64_t adesc0 = make_smem_desc(smem_u32(conv == 0 ? sX : sY), 0, 8u * p.w_row_bytes, p.w_swizzle);
+        const uint32_t a_kstep = 2u;
         const int lo = pass_lo[ps], hi = pass_hi[ps];
         tcgen05_fence_after_sync();
         for (int tap = 0; tap < 9; ++tap) {
@@ -153,18 +153,18 @@ conv3x3_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
           const uint64_t bdesc = wdesc0 + (uint64_t)((uint32_t)((s * 3 + tap % 3) * p.w_stage_bytes) >> 4);
           // all per-MMA arithmetic is 32-bit adds on the descriptors' low words
           const uint32_t a_hi = (uint32_t)(adesc0 >> 32), b_hi = (uint32_t)(bdesc >> 32), b_lo = (uint32_t)bdesc;
-          uint32_t a_lo = (uint32_t)adesc0 + (uint32_t)(lo * 128 + shift);
+          uint32_t a_lo = (uint32_t)adesc0 + (uint32_t)(lo * 128 + shift) * rowu;
           uint32_t d_tmem = tmem_base + lo * p.C;
           const uint32_t acc0 = tap != 0;
           if (ksteps == 4) {
-            for (int mt = lo; mt < hi; ++mt, a_lo += 128, d_tmem += p.C) {
+            for (int mt = lo; mt < hi; ++mt, a_lo += 128 * rowu, d_tmem += p.C) {
               umma_bf16_lohi(d_tmem, a_lo, a_hi, b_lo, b_hi, idesc, acc0);
               umma_bf16_lohi(d_tmem, a_lo + a_kstep, a_hi, b_lo + 2, b_hi, idesc, 1);
               umma_bf16_lohi(d_tmem, a_lo + 2 * a_kstep, a_hi, b_lo + 4, b_hi, idesc, 1);
               umma_bf16_lohi(d_tmem, a_lo + 3 * a_kstep, a_hi, b_lo + 6, b_hi, idesc, 1);
             }
           } else {
-            for (int mt = lo; mt < hi; ++mt, a_lo += 128, d_tmem += p.C)
+            for (int mt = lo; mt < hi; ++mt, a_lo += 128 * rowu, d_tmem += p.C)
               for (int ks = 0; ks < ksteps; ++ks)
                 umma_bf16_lohi(d_tmem, a_lo + ks * a_kstep, a_hi, b_lo + 2 * ks, b_hi, idesc, ks ? 1u : acc0);
           }
@@ -182,7 +182,9 @@ conv3x3_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
     const int col0 = (warp >> 2) * ncol;
     const bool has_cols = col0 < p.C;
 
-    // P3: intermediate = ReLU(acc + b1) inside the image, 0 outside -> planes; group A, then group B
+    // P3: intermediate = ReLU(acc + b1) inside the image, 0 outside -> swizzled rows; group A, then group B
+    const uint32_t y_addr = smem_u32(sY);
+    const uint32_t swz_mask = ((uint32_t)p.w_row_bytes >> 4) - 1u;
     for (int grp = 0; grp < 2; ++grp) {
       mbar_wait(bar_acc1 + grp, 0, abort_flag, p.status, 0x405);
       tcgen05_fence_after_sync();
@@ -203,8 +205,13 @@ conv3x3_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
             w[j] = inside ? pack_bf16x2(y0, y1) : 0u;
           }
           if (m < p.P1 + p.Wp) {   // a little past the tile so that shifted reads of valid rows never see stale data
-            *reinterpret_cast<uint4*>(sY + (size_t)(c0 / 8) * p.y_plane + m * 16) = make_uint4(w[0], w[1], w[2], w[3]);
-            *reinterpret_cast<uint4*>(sY + (size_t)(c0 / 8 + 1) * p.y_plane + m * 16) = make_uint4(w[4], w[5], w[6], w[7]);
+            // 16-byte chunk index XOR address bits [7, ..): the swizzle the MMA and TMA apply to absolute addresses
+            uint32_t a0 = y_addr + (uint32_t)m * p.w_row_bytes + (uint32_t)c0 * 2u;
+            uint32_t a1 = a0 + 16u;
+            a0 ^= ((a0 >> 7) & swz_mask) << 4;
+            a1 ^= ((a1 >> 7) & swz_mask) << 4;
+            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(a0), "r"(w[0]), "r"(w[1]), "r"(w[2]), "r"(w[3]) : "memory");
+            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(a1), "r"(w[4]), "r"(w[5]), "r"(w[6]), "r"(w[7]) : "memory");
           }
         }
       }
@@ -279,18 +286,14 @@ bool conv_layout(ConvParams& q, int R, int* smem_bytes) {
   q.P1 = (R + 2) * q.Wp; q.M1 = (q.P1 + 127) / 128;
   q.P2 = R * q.Wp; q.M2 = (q.P2 + 127) / 128;
   if (q.IH > 256 || q.Wp > 256 || q.M1 * q.C > 512) return false;
-  // at least two pixels of slack after each plane (the aliased intermediate planes start two pixels
-  // early); every plane starts on a 128-byte boundary, which the TMA destination requires
-  q.x_plane = round_up_i(q.IH * q.Wp * 16 + 32, 128);
-  // The intermediate planes alias the input planes, shifted down by two pixels: while the second tile
+  // The intermediate rows alias the input rows, shifted down by two pixels: while the second tile
   // group of the first convolution still reads input pixels >= a1*128 - 1, the first group's epilogue
   // writes intermediate pixels < a1*128, i.e. input slots < a1*128 - 2.
-  q.y_plane = q.x_plane;
-  int off = 1024;   // slack before the planes: shifted operand rows start up to three pixels early
+  int off = 1024;   // slack before the rows: shifted operand rows start up to three pixels early
   q.off_x = off;
-  q.off_y = off - 32;
-  const int reach_px = std::max(q.M1 * 128 + 2 * q.Wp + 2, q.P1 + q.Wp + 2);
-  const int x_reach = std::max(q.planes * q.x_plane, (q.planes - 1) * q.x_plane + reach_px * 16);
+  q.off_y = off - 2 * q.w_row_bytes;
+  const int reach_px = std::max(std::max(q.M1 * 128 + 2 * q.Wp + 2, q.P1 + q.Wp + 2), q.IH * q.Wp);
+  const int x_reach = reach_px * q.w_row_bytes;
   off = round_up_i(off + x_reach, 1024);
   q.off_w = off;
   q.wstages = kMaxWStages;
@@ -323,7 +326,6 @@ ago_status_t conv3x3_plan(Plan* plan, FusedState* st, std::string* err) {
   auto bad = [&](const char* m) { *err = std::string("fused conv3x3 pair: ") + m; delete host; return AGO_ERR_UNSUPPORTED; };
   if (c1.op.p[0] != q.C || plan->ops[3].op.p[0] != q.C) return bad("input, middle and output channel counts must be equal");
   if (q.C != 16 && q.C != 32 && q.C != 64) return bad("channel count must be 16, 32 or 64");
-  q.planes = q.C / 8;
   q.w_row_bytes = q.C * 2;
   q.w_swizzle = q.C == 16 ? tc::SW_32B : (q.C == 32 ? tc::SW_64B : tc::SW_128B);
   q.w_stage_bytes = round_up_i(q.C * q.w_row_bytes, 1024);
@@ -361,10 +363,10 @@ ago_status_t conv3x3_run(const Plan& plan, FusedState* st, const void* const* in
     if (it == host->maps.end()) {
       CUtensorMap m;
       if (which == 0) {
-        const uint64_t dims[5] = {8, (uint64_t)q.W, (uint64_t)q.H, (uint64_t)q.N, (uint64_t)q.planes};
-        const uint64_t strides[4] = {(uint64_t)q.C * 2, (uint64_t)q.W * q.C * 2, (uint64_t)q.H * q.W * q.C * 2, 16};
-        const uint32_t box[5] = {8, (uint32_t)q.Wp, (uint32_t)q.IH, 1, 1};   // one channel block per load
-        if (!encode_tmap_bf16(&m, base, 5, dims, strides, box, 0, err)) return false;
+        const uint64_t dims[4] = {(uint64_t)q.C, (uint64_t)q.W, (uint64_t)q.H, (uint64_t)q.N};
+        const uint64_t strides[3] = {(uint64_t)q.C * 2, (uint64_t)q.W * q.C * 2, (uint64_t)q.H * q.W * q.C * 2};
+        const uint32_t box[4] = {(uint32_t)q.C, (uint32_t)q.Wp, (uint32_t)q.IH, 1};
+        if (!encode_tmap_bf16(&m, base, 4, dims, strides, box, q.w_row_bytes, err)) return false;
       } else {
         const uint64_t dims[3] = {(uint64_t)q.C, 9, (uint64_t)q.C};
         const uint64_t strides[2] = {(uint64_t)q.C * 2, (uint64_t)9 * q.C * 2};
