@@ -10,14 +10,20 @@
 // expand convolution on the strip's one-row halo.
 //
 // Per CTA (one image, R output rows, full width):
-//   P1  TMA loads the NHWC input strip with halo (out-of-image -> 0, channels
-//       padded to the MMA K granularity by the box) into a swizzled K-major tile.
+//   P1  the compute warps copy the NHWC input strip (with its row halo; rows
+//       outside the image -> 0, channels padded to the MMA K granularity), W1
+//       and W3 into swizzled K-major tiles with coalesced 16-byte loads -- all
+//       loads of a thread are issued before its first store, so the prologue
+//       is one round trip to device memory. (A pixel is Cin * 2 bytes there,
+//       e.g. 48: one TMA box row per pixel was several times slower.)
 //   for each 16-channel chunk c of the expanded tensor:
 //     P2  tcgen05.mma: expand[pixels x 16] = X[pixels x Cin] * W1[c]^T   (TMEM, fp32)
 //     P3  TMEM -> registers: + b1, ReLU6, zero outside the image (the depthwise
-//         conv pads the post-activation tensor), bf16 -> shared memory
-//     P4  CUDA cores: depthwise 3x3 + bd + ReLU6 over the resident chunk, result
-//         written as the K-major A operand of the project GEMM
+//         conv pads the post-activation tensor), bf16 -> shared memory; the
+//         padding columns of the E chunk are written once
+//     P4  CUDA cores: depthwise 3x3 + bd + ReLU6 over the resident chunk with
+//         mixed-precision FMAs (bf16 activations and weights as stored, fp32
+//         accumulate), result written as the K-major A operand of the project GEMM
 //     P5  tcgen05.mma: out[pixels x Cout] += DW[pixels x 16] * W3[:, c]^T  (TMEM)
 //   P6  TMEM -> registers: + b3 (+ x), bf16, 16-byte stores.
 // The expand MMA of chunk c+1 is issued before the CUDA-core work of chunk c.
@@ -25,11 +31,9 @@
 #include <cuda_bf16.h>
 
 #include <cstdlib>
-#include <unordered_map>
 
 #include "fused.h"
 #include "tc_common.cuh"
-#include "tmap.h"
 
 namespace ago {
 
@@ -55,7 +59,7 @@ struct Mbv2Params {
   __nv_bfloat16* out;
   unsigned int* status;
   int N, H, W, Cin, Cexp, Cout, stride, Ho, Wo, residual;
-  int R, strips, IH, IW, P_in, M1, M2;
+  int R, strips, IH, IW, P_x, P_in, M1, M2;   // P_x = IH * W pixels in the input tile, P_in = IH * IW in an E chunk
   int Kp, row_bytes, swizzle;   // input / W1 tiles: padded K, bytes per row, tc::SwizzleMode
   int Coutp, NC;
   int tmem_cols, ecol0, pcol0;
@@ -64,71 +68,92 @@ struct Mbv2Params {
   int off_x, off_w1, off_e, off_d, off_w3, off_wd, off_b1, off_bd, off_b3, off_bar;
 };
 
-__device__ __forceinline__ uint32_t relu6_pack(float a, float b) {
-  __nv_bfloat162 h = __floats2bfloat162_rn(a, b);
-  h = __hmin2(__hmax2(h, __floats2bfloat162_rn(0.0f, 0.0f)), __floats2bfloat162_rn(6.0f, 6.0f));
-  return *reinterpret_cast<const uint32_t*>(&h);
+// bf16x2(min(max(lo, 0), 6), min(max(hi, 0), 6)): the conversion clamps at 0, one packed min caps at 6.
+__device__ __forceinline__ uint32_t relu6_pack(float lo, float hi) {
+  uint32_t r;
+  asm("{\n\t.reg .b32 t, six;\n\tmov.b32 six, 0x40C040C0;\n\tcvt.rn.relu.bf16x2.f32 t, %2, %1;\n\tmin.bf16x2 %0, t, six;\n\t}"
+      : "=r"(r) : "f"(lo), "f"(hi));
+  return r;
 }
-__device__ __forceinline__ float2 bf16x2_to_f2(uint32_t w) { return make_float2(bf16_lo(w), bf16_hi(w)); }
-__device__ __forceinline__ float2 fma2(float2 a, float2 b, float2 c) { return __ffma2_rn(a, b, c); }
 
+// Shared-memory word loads / stores with an immediate byte offset.
+template <int OFF>
 __device__ __forceinline__ uint32_t lds32(uint32_t saddr) {
   uint32_t v;
-  asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(saddr));
+  asm volatile("ld.shared.u32 %0, [%1+%2];" : "=r"(v) : "r"(saddr), "n"(OFF));
   return v;
 }
 __device__ __forceinline__ void sts32(uint32_t saddr, uint32_t v) {
   asm volatile("st.shared.u32 [%0], %1;" ::"r"(saddr), "r"(v) : "memory");
 }
 
+// acc += x * w for a packed pair of bf16 channels: the mixed-precision FMA takes the bf16 operands
+// as they are (exact product, fp32 accumulate) -- no unpacking of the activations or the weights.
+__device__ __forceinline__ void fma_pair(float2& acc, uint32_t x, uint32_t w) {
+  asm("{\n\t.reg .b16 xl, xh, wl, wh;\n\t"
+      "mov.b32 {xl, xh}, %2;\n\tmov.b32 {wl, wh}, %3;\n\t"
+      "fma.rn.f32.bf16 %0, xl, wl, %0;\n\tfma.rn.f32.bf16 %1, xh, wh, %1;\n\t}"
+      : "+f"(acc.x), "+f"(acc.y) : "r"(x), "r"(w));
+}
+
+struct Row3 { uint32_t v0, v1, v2; };   // three horizontally adjacent pixels of one channel pair
+template <int PIX_STEP>
+__device__ __forceinline__ Row3 load_row3(uint32_t a) {
+  Row3 r;
+  r.v0 = lds32<0>(a); r.v1 = lds32<PIX_STEP>(a); r.v2 = lds32<2 * PIX_STEP>(a);
+  return r;
+}
+__device__ __forceinline__ uint32_t depthwise_point(const Row3& a, const Row3& b, const Row3& c, const uint32_t (&w)[9],
+                                                    float2 bias) {
+  float2 acc = bias;
+  fma_pair(acc, a.v0, w[0]); fma_pair(acc, a.v1, w[1]); fma_pair(acc, a.v2, w[2]);
+  fma_pair(acc, b.v0, w[3]); fma_pair(acc, b.v1, w[4]); fma_pair(acc, b.v2, w[5]);
+  fma_pair(acc, c.v0, w[6]); fma_pair(acc, c.v1, w[7]); fma_pair(acc, c.v2, w[8]);
+  return relu6_pack(acc.x, acc.y);
+}
+
 // Depthwise 3x3 over the resident E chunk for one (channel pair, output column)
-// and output rows [r0, r1): E and D chunks are two planes of [pixel][8 channels]
+// and output rows [r0, r1), r1 > r0: E and D chunks are two planes of [pixel][8 channels]
 // (16 bytes per pixel), which is also the un-swizzled K-major operand layout.
-// e_col / d_col are 32-bit shared-memory addresses.
+// e_col / d_col are 32-bit shared-memory addresses. The input rows stay packed in
+// registers; the row window rotates by renaming (the loop body is unrolled over it).
 template <int STRIDE>
 __device__ __forceinline__ void depthwise_column(uint32_t e_col, uint32_t d_col, int r0, int r1, int IW, int Wo,
-                                                 const float2 (&w)[9], float2 bias) {
+                                                 const uint32_t (&w)[9], float2 bias) {
   const uint32_t e_pitch = (uint32_t)IW * 16u, d_pitch = (uint32_t)Wo * 16u;
+  uint32_t src = e_col + (uint32_t)(r0 * STRIDE) * e_pitch;
+  uint32_t dst = d_col + (uint32_t)r0 * d_pitch;
+  int n = r1 - r0;
   if (STRIDE == 1) {
-    // walk down the input rows once; each row feeds the three output rows it overlaps
-    float2 a0 = bias, a1 = bias, a2 = bias;   // output rows i, i-1, i-2
-    uint32_t src = e_col + (uint32_t)r0 * e_pitch;
-    uint32_t dst = d_col + (uint32_t)r0 * d_pitch;
-    // the first two input rows complete no output
-#pragma unroll
-    for (int pre = 0; pre < 2; ++pre) {
-      const float2 x0 = bf16x2_to_f2(lds32(src)), x1 = bf16x2_to_f2(lds32(src + 16)), x2 = bf16x2_to_f2(lds32(src + 32));
-      src += e_pitch;
-      a0 = fma2(x0, w[0], a0); a0 = fma2(x1, w[1], a0); a0 = fma2(x2, w[2], a0);
-      a1 = fma2(x0, w[3], a1); a1 = fma2(x1, w[4], a1); a1 = fma2(x2, w[5], a1);
-      a2 = a1; a1 = a0; a0 = bias;
-    }
-    for (int i = r0; i < r1; ++i) {   // input row i + 2 completes output row i
-      const float2 x0 = bf16x2_to_f2(lds32(src)), x1 = bf16x2_to_f2(lds32(src + 16)), x2 = bf16x2_to_f2(lds32(src + 32));
-      src += e_pitch;
-      a2 = fma2(x0, w[6], a2); a2 = fma2(x1, w[7], a2); a2 = fma2(x2, w[8], a2);
-      sts32(dst, relu6_pack(a2.x, a2.y));
-      dst += d_pitch;
-      a1 = fma2(x0, w[3], a1); a1 = fma2(x1, w[4], a1); a1 = fma2(x2, w[5], a1);
-      a0 = fma2(x0, w[0], a0); a0 = fma2(x1, w[1], a0); a0 = fma2(x2, w[2], a0);
-      a2 = a1; a1 = a0; a0 = bias;
+    Row3 a = load_row3<16>(src), b = load_row3<16>(src + e_pitch), c;
+    src += 2 * e_pitch;
+    while (true) {
+      c = load_row3<16>(src); src += e_pitch;
+      sts32(dst, depthwise_point(a, b, c, w, bias)); dst += d_pitch;
+      if (--n == 0) break;
+      a = load_row3<16>(src); src += e_pitch;
+      sts32(dst, depthwise_point(b, c, a, w, bias)); dst += d_pitch;
+      if (--n == 0) break;
+      b = load_row3<16>(src); src += e_pitch;
+      sts32(dst, depthwise_point(c, a, b, w, bias)); dst += d_pitch;
+      if (--n == 0) break;
     }
   } else {
-    for (int r = r0; r < r1; ++r) {
-      float2 a = bias;
-      const uint32_t src = e_col + (uint32_t)(r * STRIDE) * e_pitch;
-#pragma unroll
-      for (int kr = 0; kr < 3; ++kr)
-#pragma unroll
-        for (int ks = 0; ks < 3; ++ks)
-          a = fma2(bf16x2_to_f2(lds32(src + (uint32_t)kr * e_pitch + (uint32_t)ks * 16u)), w[kr * 3 + ks], a);
-      sts32(d_col + (uint32_t)r * d_pitch, relu6_pack(a.x, a.y));
+    Row3 a = load_row3<16>(src), b, c;
+    src += e_pitch;
+    while (true) {
+      b = load_row3<16>(src); c = load_row3<16>(src + e_pitch); src += 2 * e_pitch;
+      sts32(dst, depthwise_point(a, b, c, w, bias)); dst += d_pitch;
+      if (--n == 0) break;
+      b = load_row3<16>(src); a = load_row3<16>(src + e_pitch); src += 2 * e_pitch;
+      sts32(dst, depthwise_point(c, b, a, w, bias)); dst += d_pitch;
+      if (--n == 0) break;
     }
   }
 }
 
 __global__ void __launch_bounds__(kThreads, 1)
-mbv2_fused_kernel(const __grid_constant__ CUtensorMap tmap_x, const Mbv2Params p) {
+mbv2_fused_kernel(const Mbv2Params p) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t* sX = smem + p.off_x;
@@ -136,13 +161,11 @@ mbv2_fused_kernel(const __grid_constant__ CUtensorMap tmap_x, const Mbv2Params p
   uint8_t* sE = smem + p.off_e;
   uint8_t* sD = smem + p.off_d;
   uint8_t* sW3 = smem + p.off_w3;
-  float* sWd = reinterpret_cast<float*>(smem + p.off_wd);
+  const uint8_t* sWd = smem + p.off_wd;                   // [9][Cexp] bf16, as in device memory
   float* sB1 = reinterpret_cast<float*>(smem + p.off_b1);
   float* sBd = reinterpret_cast<float*>(smem + p.off_bd);
   float* sB3 = reinterpret_cast<float*>(smem + p.off_b3);
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + p.off_bar);
-  uint64_t* bar_x = bars + 0;       // input strip landed (TMA)
-  uint64_t* bar_w = bars + 1;       // weights staged by the compute warps
   uint64_t* bar_e = bars + 2;       // [2] expand accumulators of buffer b complete (MMA commit)
   uint64_t* bar_d = bars + 4;       // [2] project MMA has consumed D[b] (MMA commit)
   uint64_t* bar_tfree = bars + 6;   // [2] expand buffer b drained and E chunk written (compute -> issuer)
@@ -158,10 +181,7 @@ mbv2_fused_kernel(const __grid_constant__ CUtensorMap tmap_x, const Mbv2Params p
   const int d_bytes = 2 * p.d_plane;
 
   if (tid == kComputeThreads) {
-    // first issuer lane: barriers, then the input strip's TMA right away
     *abort_flag = 0u;
-    mbar_init(bar_x, 1);
-    mbar_init(bar_w, 1);
     for (int i = 0; i < 2; ++i) {
       mbar_init(bar_e + i, kIssuers);
       mbar_init(bar_d + i, kIssuers);
@@ -170,13 +190,82 @@ mbv2_fused_kernel(const __grid_constant__ CUtensorMap tmap_x, const Mbv2Params p
     }
     fence_mbar_init();
     fence_proxy_async_smem();
-    tma_prefetch_desc(&tmap_x);
-    mbar_arrive_expect_tx(bar_x, (uint32_t)(p.P_in * p.row_bytes));
-    tma_load_4d(sX, &tmap_x, bar_x, 0, -1, gh0, n);
   }
-  if (warp == 0) {
-    tmem_alloc(tmem_slot, (uint32_t)p.tmem_cols);
-    tmem_relinquish();
+  if (warp < kComputeWarps) {
+    // ---- P1: stage the input strip, the weights and the biases. Every 16-byte chunk is one slot; a thread first
+    // issues the loads of all its slots, then stores them, so that the whole prologue costs one round trip to
+    // device memory. (Pixels are Cin * 2 bytes apart there: coalesced plain loads of the contiguous strip serve
+    // that better than one TMA box row per pixel.) X and W1 rows go to their swizzled K-major tiles, zero beyond
+    // Cin; W3 to one [Coutp x 16 channels] slice per chunk; depthwise weights and biases are copied as they are.
+    constexpr int kBatch = 8;
+    const int cs = p.Kp == 16 ? 1 : (p.Kp == 32 ? 2 : 3);   // log2(16-byte chunks per tile row)
+    const int nX = p.P_x << cs, nW1 = p.Cexp << cs, nW3 = p.NC * p.Coutp * 2;
+    const int nWd = 9 * p.Cexp / 8, nB = p.Cexp / 4, nB3 = p.Cout / 4;
+    const int total = nX + nW1 + nW3 + nWd + 2 * nB + nB3;
+    // tile pixel `pix` is image pixel gh0 * W + pix of image n (strips are full-width rows): in the image for pix in [pix_lo, pix_hi)
+    const int pix_lo = max(0, -gh0 * p.W), pix_hi = min(p.P_x, (p.H - gh0) * p.W);
+    const uint8_t* x0 = reinterpret_cast<const uint8_t*>(p.x) + ((size_t)n * p.H + gh0) * p.W * p.Cin * 2;   // not dereferenced outside the image
+    const uint32_t cmask = (1u << cs) - 1u, cin_chunks = (uint32_t)p.Cin >> 3, cin_bytes = (uint32_t)p.Cin * 2u;
+    const uint32_t swz_mask = ((uint32_t)p.row_bytes >> 4) - 1u;
+    uint4 val[kBatch];
+    uint32_t dst[kBatch];
+    auto issue = [&](int base) {
+#pragma unroll
+      for (int k = 0; k < kBatch; ++k) {
+        uint32_t i = (uint32_t)(base + k * kComputeThreads);
+        const uint8_t* src = nullptr;
+        dst[k] = 0xffffffffu;
+        val[k] = make_uint4(0, 0, 0, 0);
+        if (i < (uint32_t)(nX + nW1)) {
+          // X and W1: row-major [row][Cin] -> swizzled rows of Kp channels; chunk i of the tile lies at byte 16 i,
+          // its 16-byte column XORed with the row's swizzle phase (address bits 7..)
+          const bool is_x = i < (uint32_t)nX;
+          if (!is_x) i -= nX;
+          const uint32_t row = i >> cs, ch = i & cmask;
+          const bool ok = ch < cin_chunks && (!is_x || ((int)row >= pix_lo && (int)row < pix_hi));
+          if (ok) src = (is_x ? x0 : reinterpret_cast<const uint8_t*>(p.w1)) + row * cin_bytes + ch * 16u;
+          dst[k] = (is_x ? p.off_x : p.off_w1) + ((i << 4) ^ (((i >> 3) & swz_mask) << 4));
+        } else if ((i -= nX + nW1) < (uint32_t)nW3) {
+          const uint32_t half = i & 1u, c = (i >> 1) / (uint32_t)p.Coutp, row = (i >> 1) - c * p.Coutp;
+          if (row < (uint32_t)p.Cout) src = reinterpret_cast<const uint8_t*>(p.w3) + (row * p.Cexp + c * kChunk + half * 8u) * 2u;
+          dst[k] = p.off_w3 + c * p.Coutp * kChunkRowBytes + swz_offset(row, half, kChunkRowBytes);
+        } else if ((i -= nW3) < (uint32_t)nWd) {
+          src = reinterpret_cast<const uint8_t*>(p.wd) + i * 16u;
+          dst[k] = p.off_wd + i * 16u;
+        } else if ((i -= nWd) < (uint32_t)nB) {
+          src = reinterpret_cast<const uint8_t*>(p.b1) + i * 16u;
+          dst[k] = p.off_b1 + i * 16u;
+        } else if ((i -= nB) < (uint32_t)nB) {
+          src = reinterpret_cast<const uint8_t*>(p.bd) + i * 16u;
+          dst[k] = p.off_bd + i * 16u;
+        } else if ((i -= nB) < (uint32_t)nB3) {
+          src = reinterpret_cast<const uint8_t*>(p.b3) + i * 16u;
+          dst[k] = p.off_b3 + i * 16u;
+        }
+        if (src) val[k] = __ldg(reinterpret_cast<const uint4*>(src));
+      }
+    };
+    auto commit = [&]() {
+#pragma unroll
+      for (int k = 0; k < kBatch; ++k)
+        if (dst[k] != 0xffffffffu) *reinterpret_cast<uint4*>(smem + dst[k]) = val[k];
+    };
+    issue(tid);
+    if (warp == 0) {
+      tmem_alloc(tmem_slot, (uint32_t)p.tmem_cols);
+      tmem_relinquish();
+    }
+    commit();
+    for (int base = tid + kBatch * kComputeThreads; base < total; base += kBatch * kComputeThreads) {
+      issue(base);
+      commit();
+    }
+    // the zero padding columns of the E chunk (written once: every chunk reuses them)
+    for (int i = tid; i < p.IH * 4; i += kComputeThreads) {
+      const int ih = i >> 2, side = (i >> 1) & 1, plane = i & 1;
+      *reinterpret_cast<uint4*>(sE + plane * p.e_plane + (ih * p.IW + side * (p.IW - 1)) * 16) = make_uint4(0, 0, 0, 0);
+    }
+    fence_proxy_async_smem();
   }
   tcgen05_fence_before_sync();
   __syncthreads();
@@ -209,8 +298,6 @@ mbv2_fused_kernel(const __grid_constant__ CUtensorMap tmap_x, const Mbv2Params p
         }
         umma_commit(bar_e + b);
       };
-      mbar_wait(bar_w, 0, abort_flag, p.status, 0x100);
-      mbar_wait(bar_x, 0, abort_flag, p.status, 0x101);
       tcgen05_fence_after_sync();
       issue_expand(0);
       if (p.NC > 1) issue_expand(1);
@@ -235,29 +322,6 @@ mbv2_fused_kernel(const __grid_constant__ CUtensorMap tmap_x, const Mbv2Params p
   } else {
     // ================================== compute warps ==================================
     const int ctid = tid;   // compute warps are warps 0 .. kComputeWarps-1
-    // ---- stage weights and biases (generic proxy), in the operand layouts the MMAs read ----
-    {
-      const int chunks_per_row = p.row_bytes >> 4;
-      for (int i = ctid; i < p.Cexp * chunks_per_row; i += kComputeThreads) {
-        const int row = i / chunks_per_row, ch = i % chunks_per_row;
-        uint4 v = make_uint4(0, 0, 0, 0);
-        if (ch * 8 < p.Cin) v = __ldg(reinterpret_cast<const uint4*>(p.w1 + (size_t)row * p.Cin + ch * 8));
-        *reinterpret_cast<uint4*>(sW1 + swz_offset(row, ch, p.row_bytes)) = v;
-      }
-      for (int i = ctid; i < p.NC * p.Coutp * 2; i += kComputeThreads) {
-        const int half = i & 1, row = (i >> 1) % p.Coutp, c = (i >> 1) / p.Coutp;
-        uint4 v = make_uint4(0, 0, 0, 0);
-        if (row < p.Cout) v = __ldg(reinterpret_cast<const uint4*>(p.w3 + (size_t)row * p.Cexp + c * kChunk + half * 8));
-        *reinterpret_cast<uint4*>(sW3 + c * p.Coutp * kChunkRowBytes + swz_offset(row, half, kChunkRowBytes)) = v;
-      }
-      for (int i = ctid; i < 9 * p.Cexp; i += kComputeThreads) sWd[i] = __bfloat162float(p.wd[i]);
-      for (int i = ctid; i < p.Cexp; i += kComputeThreads) { sB1[i] = p.b1[i]; sBd[i] = p.bd[i]; }
-      for (int i = ctid; i < p.Coutp; i += kComputeThreads) sB3[i] = i < p.Cout ? p.b3[i] : 0.0f;
-    }
-    fence_proxy_async_smem();
-    named_barrier_sync(1, kComputeThreads);
-    if (ctid == 0) mbar_arrive(bar_w);
-
     const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
     // Depthwise work split: thread = (channel pair, slot); a slot walks one output column of one row group.
     constexpr int kSlots = kComputeThreads / 8;
@@ -268,15 +332,20 @@ mbv2_fused_kernel(const __grid_constant__ CUtensorMap tmap_x, const Mbv2Params p
     const int cp_off = (cp & 3) * 4;   // byte offset inside a 16-byte pixel entry
     // first depthwise item of this slot (most shapes have at most one per slot)
     const int item0_g = slot / p.Wo, item0_wo = slot - item0_g * p.Wo;
-    // expand-epilogue rows of this thread: tile (warp>>2) + 7k; bit k of the masks: row exists / is an in-image pixel
-    uint32_t e_exist = 0, e_inimg = 0;
-    for (int t = warp >> 2, k = 0; t < p.M1; t += kComputeWarps / 4, ++k) {
+    // expand-epilogue rows of this thread: tile (warp>>2) + 7k, k < 2. e_off[k]: byte offset of the pixel in an E
+    // plane (the tile has no padding columns, the E chunk does), -1: no such pixel; bit k of e_inimg: the row lies
+    // inside the image (the rest is the zero padding of the intermediate tensor)
+    int e_off[2] = {-1, -1};
+    uint32_t e_inimg = 0;
+#pragma unroll
+    for (int k = 0; k < 2; ++k) {
+      const int t = (warp >> 2) + k * (kComputeWarps / 4);
       const int pix = t * 128 + (warp & 3) * 32 + lane;
-      const int ih = pix / p.IW, iw = pix - ih * p.IW;
+      const int ih = pix / p.W, iw = pix - ih * p.W;
       const int gh = gh0 + ih;
-      if (pix < p.P_in) {
-        e_exist |= 1u << k;
-        if (gh >= 0 && gh < p.H && iw >= 1 && iw <= p.W) e_inimg |= 1u << k;
+      if (t < p.M1 && pix < p.P_x) {
+        e_off[k] = (ih * p.IW + iw + 1) * 16;
+        if (gh >= 0 && gh < p.H) e_inimg |= 1u << k;
       }
     }
 
@@ -286,12 +355,14 @@ mbv2_fused_kernel(const __grid_constant__ CUtensorMap tmap_x, const Mbv2Params p
       tcgen05_fence_after_sync();
 
       // ---- P3: expand epilogue -> E chunk: + b1, ReLU6, zero outside the image, bf16 ----
-      for (int t = warp >> 2, k = 0; t < p.M1; t += kComputeWarps / 4, ++k) {
+#pragma unroll
+      for (int k = 0; k < 2; ++k) {
+        const int t = (warp >> 2) + k * (kComputeWarps / 4);
+        if (t >= p.M1) break;
         uint32_t acc[16];
         tmem_ld_x16(tmem_base + lane_base + p.ecol0 + (b * p.M1 + t) * kChunk, acc);
         tmem_ld_wait();
-        const int pix = t * 128 + (warp & 3) * 32 + lane;
-        if ((e_exist >> k) & 1u) {
+        if (e_off[k] >= 0) {
           uint32_t w[8];
           if ((e_inimg >> k) & 1u) {
             const float4* bb = reinterpret_cast<const float4*>(sB1 + c * kChunk);
@@ -305,8 +376,8 @@ mbv2_fused_kernel(const __grid_constant__ CUtensorMap tmap_x, const Mbv2Params p
 #pragma unroll
             for (int j = 0; j < 8; ++j) w[j] = 0u;
           }
-          *reinterpret_cast<uint4*>(sE + pix * 16) = make_uint4(w[0], w[1], w[2], w[3]);
-          *reinterpret_cast<uint4*>(sE + p.e_plane + pix * 16) = make_uint4(w[4], w[5], w[6], w[7]);
+          *reinterpret_cast<uint4*>(sE + e_off[k]) = make_uint4(w[0], w[1], w[2], w[3]);
+          *reinterpret_cast<uint4*>(sE + p.e_plane + e_off[k]) = make_uint4(w[4], w[5], w[6], w[7]);
         }
       }
       tcgen05_fence_before_sync();
@@ -319,9 +390,9 @@ mbv2_fused_kernel(const __grid_constant__ CUtensorMap tmap_x, const Mbv2Params p
       // ---- P4: depthwise 3x3 + bias + ReLU6 on CUDA cores: E chunk -> D[b] (A operand of the project GEMM) ----
       {
         const int ch = c * kChunk + cp * 2;
-        float2 wgt[9];
+        uint32_t wgt[9];   // packed bf16 pairs
 #pragma unroll
-        for (int tap = 0; tap < 9; ++tap) wgt[tap] = *reinterpret_cast<const float2*>(sWd + tap * p.Cexp + ch);
+        for (int tap = 0; tap < 9; ++tap) wgt[tap] = *reinterpret_cast<const uint32_t*>(sWd + (tap * p.Cexp + ch) * 2);
         const float2 bias = *reinterpret_cast<const float2*>(sBd + ch);
         const uint32_t e_plane = smem_u32(sE) + (uint32_t)((cp >> 2) * p.e_plane + cp_off);
         const uint32_t d_plane = smem_u32(sD) + (uint32_t)(b * d_bytes + (cp >> 2) * p.d_plane + cp_off);
@@ -329,6 +400,7 @@ mbv2_fused_kernel(const __grid_constant__ CUtensorMap tmap_x, const Mbv2Params p
           int g = item0_g, wo = item0_wo;
           if (item != slot) { g = item / p.Wo; wo = item - g * p.Wo; }
           const int r0 = g * rows_per_group, r1 = min(rows_valid, r0 + rows_per_group);
+          if (r0 >= r1) continue;
           if (p.stride == 1)
             depthwise_column<1>(e_plane + wo * 16, d_plane + wo * 16, r0, r1, p.IW, p.Wo, wgt, bias);
           else
@@ -386,7 +458,6 @@ int round_up(int v, int m) { return (v + m - 1) / m * m; }
 struct Mbv2Host {
   Mbv2Params prm;
   int smem_bytes = 0;
-  std::unordered_map<const void*, CUtensorMap> maps;
 };
 
 bool layout(Mbv2Params& q, int R, int* smem_bytes) {
@@ -395,7 +466,8 @@ bool layout(Mbv2Params& q, int R, int* smem_bytes) {
   q.IH = (R - 1) * q.stride + 3;
   q.IW = q.W + 2;
   q.P_in = q.IH * q.IW;
-  q.M1 = (q.P_in + 127) / 128;
+  q.P_x = q.IH * q.W;
+  q.M1 = (q.P_x + 127) / 128;
   q.M2 = (R * q.Wo + 127) / 128;
   if (q.IH > 256 || q.IW > 256 || q.M1 > 8) return false;
   const int cols = 2 * q.M1 * kChunk + q.M2 * q.Coutp;
@@ -415,7 +487,7 @@ bool layout(Mbv2Params& q, int R, int* smem_bytes) {
   q.off_e = take(2 * q.e_plane);
   q.off_d = take(2 * 2 * q.d_plane);
   q.off_w3 = take(q.NC * q.Coutp * kChunkRowBytes);
-  q.off_wd = take(9 * q.Cexp * 4);
+  q.off_wd = take(9 * q.Cexp * 2);
   q.off_b1 = take(q.Cexp * 4);
   q.off_bd = take(q.Cexp * 4);
   q.off_b3 = take(q.Coutp * 4);
@@ -478,22 +550,12 @@ ago_status_t mbv2_run(const Plan& plan, FusedState* st, const void* const* input
   q.w3 = static_cast<const __nv_bfloat16*>(weights[4]); q.b3 = static_cast<const float*>(weights[5]);
   q.out = static_cast<__nv_bfloat16*>(output);
   q.status = status_word;
-  auto it = host->maps.find(inputs[0]);
-  if (it == host->maps.end()) {
-    CUtensorMap m;
-    const uint64_t dims[4] = {(uint64_t)q.Cin, (uint64_t)q.W, (uint64_t)q.H, (uint64_t)q.N};
-    const uint64_t strides[3] = {(uint64_t)q.Cin * 2, (uint64_t)q.W * q.Cin * 2, (uint64_t)q.H * q.W * q.Cin * 2};
-    const uint32_t box[4] = {(uint32_t)q.Kp, (uint32_t)q.IW, (uint32_t)q.IH, 1};
-    if (!encode_tmap_bf16(&m, inputs[0], 4, dims, strides, box, q.row_bytes, err)) return AGO_ERR_CUDA;
-    if (host->maps.size() > 4096) host->maps.clear();
-    it = host->maps.emplace(inputs[0], m).first;
-  }
   {
     static int smem_opt_in[64] = {};
     cudaError_t e = ensure_max_dynamic_smem(reinterpret_cast<const void*>(mbv2_fused_kernel), smem_opt_in);
     if (e != cudaSuccess) { *err = std::string("cudaFuncSetAttribute: ") + cudaGetErrorString(e); return AGO_ERR_CUDA; }
   }
-  mbv2_fused_kernel<<<q.N * q.strips, kThreads, host->smem_bytes, stream>>>(it->second, q);
+  mbv2_fused_kernel<<<q.N * q.strips, kThreads, host->smem_bytes, stream>>>(q);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) { *err = std::string("fused inverted-residual launch: ") + cudaGetErrorString(e); return AGO_ERR_CUDA; }
   return AGO_OK;
