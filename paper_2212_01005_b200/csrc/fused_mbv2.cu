@@ -83,8 +83,9 @@ __device__ __forceinline__ uint32_t lds32(uint32_t saddr) {
   asm volatile("ld.shared.u32 %0, [%1+%2];" : "=r"(v) : "r"(saddr), "n"(OFF));
   return v;
 }
+template <int OFF = 0>
 __device__ __forceinline__ void sts32(uint32_t saddr, uint32_t v) {
-  asm volatile("st.shared.u32 [%0], %1;" ::"r"(saddr), "r"(v) : "memory");
+  asm volatile("st.shared.u32 [%0+%1], %2;" ::"r"(saddr), "n"(OFF), "r"(v) : "memory");
 }
 
 // acc += x * w for a packed pair of bf16 channels: the mixed-precision FMA takes the bf16 operands
@@ -112,44 +113,61 @@ __device__ __forceinline__ uint32_t depthwise_point(const Row3& a, const Row3& b
   return relu6_pack(acc.x, acc.y);
 }
 
-// Depthwise 3x3 over the resident E chunk for one (channel pair, output column)
-// and output rows [r0, r1), r1 > r0: E and D chunks are two planes of [pixel][8 channels]
-// (16 bytes per pixel), which is also the un-swizzled K-major operand layout.
-// e_col / d_col are 32-bit shared-memory addresses. The input rows stay packed in
-// registers; the row window rotates by renaming (the loop body is unrolled over it).
-template <int STRIDE>
-__device__ __forceinline__ void depthwise_column(uint32_t e_col, uint32_t d_col, int r0, int r1, int IW, int Wo,
-                                                 const uint32_t (&w)[9], float2 bias) {
+// E and D chunks are two planes of [pixel][8 channels] (16 bytes per pixel), which is also the
+// un-swizzled K-major operand layout; all addresses below are 32-bit shared-memory addresses.
+//
+// Stride-2 depthwise 3x3 for one (channel pair, output column) and output rows [r0, r1), r1 > r0:
+// consecutive output rows share one input row, which stays packed in registers (the loop body is
+// unrolled over the two roles of that row).
+__device__ __forceinline__ void depthwise_column_s2(uint32_t e_col, uint32_t d_col, int r0, int r1, int IW, int Wo,
+                                                    const uint32_t (&w)[9], float2 bias) {
   const uint32_t e_pitch = (uint32_t)IW * 16u, d_pitch = (uint32_t)Wo * 16u;
-  uint32_t src = e_col + (uint32_t)(r0 * STRIDE) * e_pitch;
+  uint32_t src = e_col + (uint32_t)(r0 * 2) * e_pitch;
   uint32_t dst = d_col + (uint32_t)r0 * d_pitch;
   int n = r1 - r0;
-  if (STRIDE == 1) {
-    Row3 a = load_row3<16>(src), b = load_row3<16>(src + e_pitch), c;
-    src += 2 * e_pitch;
-    while (true) {
-      c = load_row3<16>(src); src += e_pitch;
-      sts32(dst, depthwise_point(a, b, c, w, bias)); dst += d_pitch;
-      if (--n == 0) break;
-      a = load_row3<16>(src); src += e_pitch;
-      sts32(dst, depthwise_point(b, c, a, w, bias)); dst += d_pitch;
-      if (--n == 0) break;
-      b = load_row3<16>(src); src += e_pitch;
-      sts32(dst, depthwise_point(c, a, b, w, bias)); dst += d_pitch;
-      if (--n == 0) break;
-    }
-  } else {
-    Row3 a = load_row3<16>(src), b, c;
-    src += e_pitch;
-    while (true) {
-      b = load_row3<16>(src); c = load_row3<16>(src + e_pitch); src += 2 * e_pitch;
-      sts32(dst, depthwise_point(a, b, c, w, bias)); dst += d_pitch;
-      if (--n == 0) break;
-      b = load_row3<16>(src); a = load_row3<16>(src + e_pitch); src += 2 * e_pitch;
-      sts32(dst, depthwise_point(c, b, a, w, bias)); dst += d_pitch;
-      if (--n == 0) break;
-    }
+  Row3 a = load_row3<16>(src), b, c;
+  src += e_pitch;
+  while (true) {
+    b = load_row3<16>(src); c = load_row3<16>(src + e_pitch); src += 2 * e_pitch;
+    sts32(dst, depthwise_point(a, b, c, w, bias)); dst += d_pitch;
+    if (--n == 0) break;
+    b = load_row3<16>(src); a = load_row3<16>(src + e_pitch); src += 2 * e_pitch;
+    sts32(dst, depthwise_point(c, b, a, w, bias)); dst += d_pitch;
+    if (--n == 0) break;
   }
+}
+
+// Stride-1 depthwise 3x3 for one (channel pair, output row, segment of 7 output columns), fully
+// unrolled: three input columns (3 rows each) stay packed in registers and rotate by renaming, all
+// shared-memory offsets are immediates. e_row: address of the segment's first input pixel in the
+// row above the output row; d_row: address of its first output pixel; ncol <= 7 columns are stored
+// (the loads of a ragged segment run past the row end, inside shared memory; those results are dropped).
+constexpr int kSegCols = 7;
+__device__ __forceinline__ void depthwise_segment(uint32_t e_row, uint32_t d_row, uint32_t e_pitch, int ncol,
+                                                  const uint32_t (&w)[9], float2 bias) {
+  const uint32_t e0 = e_row, e1 = e_row + e_pitch, e2 = e1 + e_pitch;
+  uint32_t c0[3], c1[3], c2[3];
+  c0[0] = lds32<0>(e0); c0[1] = lds32<0>(e1); c0[2] = lds32<0>(e2);
+  c1[0] = lds32<16>(e0); c1[1] = lds32<16>(e1); c1[2] = lds32<16>(e2);
+#define AGO_DW_STEP(J, A, B, C)                                                                       \
+  {                                                                                                   \
+    C[0] = lds32<(J + 2) * 16>(e0); C[1] = lds32<(J + 2) * 16>(e1); C[2] = lds32<(J + 2) * 16>(e2);   \
+    float2 acc = bias;                                                                                \
+    fma_pair(acc, A[0], w[0]); fma_pair(acc, B[0], w[1]); fma_pair(acc, C[0], w[2]);                  \
+    fma_pair(acc, A[1], w[3]); fma_pair(acc, B[1], w[4]); fma_pair(acc, C[1], w[5]);                  \
+    fma_pair(acc, A[2], w[6]); fma_pair(acc, B[2], w[7]); fma_pair(acc, C[2], w[8]);                  \
+    if (FULL || J < ncol) sts32<J * 16>(d_row, relu6_pack(acc.x, acc.y));                             \
+  }
+  if (ncol == kSegCols) {
+    constexpr bool FULL = true;
+    AGO_DW_STEP(0, c0, c1, c2) AGO_DW_STEP(1, c1, c2, c0) AGO_DW_STEP(2, c2, c0, c1) AGO_DW_STEP(3, c0, c1, c2)
+    AGO_DW_STEP(4, c1, c2, c0) AGO_DW_STEP(5, c2, c0, c1) AGO_DW_STEP(6, c0, c1, c2)
+  } else {
+    constexpr bool FULL = false;
+    AGO_DW_STEP(0, c0, c1, c2) AGO_DW_STEP(1, c1, c2, c0) AGO_DW_STEP(2, c2, c0, c1) AGO_DW_STEP(3, c0, c1, c2)
+    AGO_DW_STEP(4, c1, c2, c0) AGO_DW_STEP(5, c2, c0, c1)
+  }
+#undef AGO_DW_STEP
 }
 
 __global__ void __launch_bounds__(kThreads, 1)
@@ -260,9 +278,9 @@ mbv2_fused_kernel(const Mbv2Params p) {
       issue(base);
       commit();
     }
-    // the zero padding columns of the E chunk (written once: every chunk reuses them)
-    for (int i = tid; i < p.IH * 4; i += kComputeThreads) {
-      const int ih = i >> 2, side = (i >> 1) & 1, plane = i & 1;
+    // the zero padding columns of the two E chunk buffers (written once: every chunk reuses them)
+    for (int i = tid; i < p.IH * 8; i += kComputeThreads) {
+      const int ih = i >> 3, side = (i >> 2) & 1, plane = i & 3;   // 2 buffers x 2 planes
       *reinterpret_cast<uint4*>(sE + plane * p.e_plane + (ih * p.IW + side * (p.IW - 1)) * 16) = make_uint4(0, 0, 0, 0);
     }
     fence_proxy_async_smem();
@@ -323,15 +341,20 @@ mbv2_fused_kernel(const Mbv2Params p) {
     // ================================== compute warps ==================================
     const int ctid = tid;   // compute warps are warps 0 .. kComputeWarps-1
     const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
-    // Depthwise work split: thread = (channel pair, slot); a slot walks one output column of one row group.
+    // Depthwise work split: thread = (channel pair, slot). Stride 1: an item is a segment of 7 output columns of one
+    // output row (56 columns x 14 rows x 8 pairs = one item per thread). Stride 2: an item is one output column of one
+    // row group.
     constexpr int kSlots = kComputeThreads / 8;
     const int cp = ctid & 7, slot = ctid >> 3;
+    const int cp_off = (cp & 3) * 4;   // byte offset inside a 16-byte pixel entry
+    const uint32_t e_pitch = (uint32_t)p.IW * 16u, d_pitch = (uint32_t)p.Wo * 16u;
+    const int nseg = (p.Wo + kSegCols - 1) / kSegCols;
     const int groups = max(1, min(rows_valid, kSlots / max(1, min(p.Wo, kSlots))));
     const int rows_per_group = (rows_valid + groups - 1) / groups;
-    const int dw_items = p.Wo * groups;
-    const int cp_off = (cp & 3) * 4;   // byte offset inside a 16-byte pixel entry
-    // first depthwise item of this slot (most shapes have at most one per slot)
-    const int item0_g = slot / p.Wo, item0_wo = slot - item0_g * p.Wo;
+    const int per_row = p.stride == 1 ? nseg : p.Wo;                       // items per output row / per row group
+    const int dw_items = per_row * (p.stride == 1 ? rows_valid : groups);
+    const int item0_r = slot / per_row, item0_c = slot - item0_r * per_row;   // first item (most shapes have at most one)
+    const int e_bytes = 2 * p.e_plane;
     // expand-epilogue rows of this thread: tile (warp>>2) + 7k, k < 2. e_off[k]: byte offset of the pixel in an E
     // plane (the tile has no padding columns, the E chunk does), -1: no such pixel; bit k of e_inimg: the row lies
     // inside the image (the rest is the zero padding of the intermediate tensor)
@@ -349,12 +372,12 @@ mbv2_fused_kernel(const Mbv2Params p) {
       }
     }
 
-    for (int c = 0; c < p.NC; ++c) {
+    // ---- P3: expand epilogue of chunk c -> E[c & 1]: + b1, ReLU6, zero outside the image, bf16 ----
+    auto expand_epilogue = [&](int c) {
       const int b = c & 1;
       mbar_wait(bar_e + b, (uint32_t)(c >> 1) & 1u, abort_flag, p.status, 0x102);
       tcgen05_fence_after_sync();
-
-      // ---- P3: expand epilogue -> E chunk: + b1, ReLU6, zero outside the image, bf16 ----
+      uint8_t* e_buf = sE + b * e_bytes;
 #pragma unroll
       for (int k = 0; k < 2; ++k) {
         const int t = (warp >> 2) + k * (kComputeWarps / 4);
@@ -376,14 +399,22 @@ mbv2_fused_kernel(const Mbv2Params p) {
 #pragma unroll
             for (int j = 0; j < 8; ++j) w[j] = 0u;
           }
-          *reinterpret_cast<uint4*>(sE + e_off[k]) = make_uint4(w[0], w[1], w[2], w[3]);
-          *reinterpret_cast<uint4*>(sE + p.e_plane + e_off[k]) = make_uint4(w[4], w[5], w[6], w[7]);
+          *reinterpret_cast<uint4*>(e_buf + e_off[k]) = make_uint4(w[0], w[1], w[2], w[3]);
+          *reinterpret_cast<uint4*>(e_buf + p.e_plane + e_off[k]) = make_uint4(w[4], w[5], w[6], w[7]);
         }
       }
       tcgen05_fence_before_sync();
-      named_barrier_sync(1, kComputeThreads);
-      if (ctid == 0) mbar_arrive(bar_tfree + b);
+    };
 
+    expand_epilogue(0);
+    named_barrier_sync(1, kComputeThreads);
+    if (ctid == 0) mbar_arrive(bar_tfree + 0);
+
+    // One barrier per chunk: a warp runs the depthwise stage of chunk c (E[c & 1] -> D[c & 1]) and then the expand
+    // epilogue of chunk c + 1 (-> E[(c + 1) & 1]); the warps drift apart in between, so the tensor-memory load latency
+    // of one hides behind the arithmetic of the others.
+    for (int c = 0; c < p.NC; ++c) {
+      const int b = c & 1;
       // D[b] was read by the project MMA of chunk c-2
       if (c >= 2) mbar_wait(bar_d + b, (uint32_t)((c - 2) >> 1) & 1u, abort_flag, p.status, 0x103);
 
@@ -394,22 +425,28 @@ mbv2_fused_kernel(const Mbv2Params p) {
 #pragma unroll
         for (int tap = 0; tap < 9; ++tap) wgt[tap] = *reinterpret_cast<const uint32_t*>(sWd + (tap * p.Cexp + ch) * 2);
         const float2 bias = *reinterpret_cast<const float2*>(sBd + ch);
-        const uint32_t e_plane = smem_u32(sE) + (uint32_t)((cp >> 2) * p.e_plane + cp_off);
+        const uint32_t e_plane = smem_u32(sE) + (uint32_t)(b * e_bytes + (cp >> 2) * p.e_plane + cp_off);
         const uint32_t d_plane = smem_u32(sD) + (uint32_t)(b * d_bytes + (cp >> 2) * p.d_plane + cp_off);
         for (int item = slot; item < dw_items; item += kSlots) {
-          int g = item0_g, wo = item0_wo;
-          if (item != slot) { g = item / p.Wo; wo = item - g * p.Wo; }
-          const int r0 = g * rows_per_group, r1 = min(rows_valid, r0 + rows_per_group);
-          if (r0 >= r1) continue;
-          if (p.stride == 1)
-            depthwise_column<1>(e_plane + wo * 16, d_plane + wo * 16, r0, r1, p.IW, p.Wo, wgt, bias);
-          else
-            depthwise_column<2>(e_plane + wo * 32, d_plane + wo * 16, r0, r1, p.IW, p.Wo, wgt, bias);
+          int r = item0_r, col = item0_c;
+          if (item != slot) { r = item / per_row; col = item - r * per_row; }
+          if (p.stride == 1) {
+            const int wo = col * kSegCols;
+            depthwise_segment(e_plane + (uint32_t)r * e_pitch + wo * 16, d_plane + (uint32_t)r * d_pitch + wo * 16, e_pitch,
+                              min(kSegCols, p.Wo - wo), wgt, bias);
+          } else {
+            const int r0 = r * rows_per_group, r1 = min(rows_valid, r0 + rows_per_group);
+            if (r0 < r1) depthwise_column_s2(e_plane + col * 32, d_plane + col * 16, r0, r1, p.IW, p.Wo, wgt, bias);
+          }
         }
       }
+      if (c + 1 < p.NC) expand_epilogue(c + 1);
       fence_proxy_async_smem();
       named_barrier_sync(1, kComputeThreads);
-      if (ctid == 0) mbar_arrive(bar_dready + b);
+      if (ctid == 0) {
+        mbar_arrive(bar_dready + b);
+        if (c + 1 < p.NC) mbar_arrive(bar_tfree + ((c + 1) & 1));
+      }
     }
 
     // ---- P6: project epilogue: + b3 (+ residual), bf16, 16-byte stores ----
@@ -484,7 +521,7 @@ bool layout(Mbv2Params& q, int R, int* smem_bytes) {
   // 2 x 64-byte accesses (4 pixels x 4 channel pairs per plane) never share a bank
   q.e_plane = round_up(q.P_in * 16, 128) + 64;
   q.d_plane = q.M2 * 128 * 16 + 64;
-  q.off_e = take(2 * q.e_plane);
+  q.off_e = take(2 * 2 * q.e_plane);   // two chunk buffers
   q.off_d = take(2 * 2 * q.d_plane);
   q.off_w3 = take(q.NC * q.Coutp * kChunkRowBytes);
   q.off_wd = take(9 * q.Cexp * 2);
