@@ -62,6 +62,7 @@ struct Mbv2Params {
   int R, strips, IH, IW, P_x, P_in, M1, M2;   // P_x = IH * W pixels in the input tile, P_in = IH * IW in an E chunk
   int Kp, row_bytes, swizzle;   // input / W1 tiles: padded K, bytes per row, tc::SwizzleMode
   int Coutp, NC;
+  uint32_t coutp_recip;         // 2^32 / Coutp + 1: x / Coutp == __umulhi(x, coutp_recip) for the small x used here
   int tmem_cols, ecol0, pcol0;
   int e_plane, d_plane;         // byte distance between the two 8-channel planes of an E / D chunk
   // shared-memory byte offsets (from the 1024-aligned base)
@@ -215,68 +216,82 @@ mbv2_fused_kernel(const Mbv2Params p) {
     // device memory. (Pixels are Cin * 2 bytes apart there: coalesced plain loads of the contiguous strip serve
     // that better than one TMA box row per pixel.) X and W1 rows go to their swizzled K-major tiles, zero beyond
     // Cin; W3 to one [Coutp x 16 channels] slice per chunk; depthwise weights and biases are copied as they are.
-    constexpr int kBatch = 8;
+    constexpr int kBX = 4, kBW = 2;   // slots per thread in the first (batched) pass: input strip / everything else
     const int cs = p.Kp == 16 ? 1 : (p.Kp == 32 ? 2 : 3);   // log2(16-byte chunks per tile row)
-    const int nX = p.P_x << cs, nW1 = p.Cexp << cs, nW3 = p.NC * p.Coutp * 2;
-    const int nWd = 9 * p.Cexp / 8, nB = p.Cexp / 4, nB3 = p.Cout / 4;
-    const int total = nX + nW1 + nW3 + nWd + 2 * nB + nB3;
+    const uint32_t nX = (uint32_t)p.P_x << cs, nW1 = (uint32_t)p.Cexp << cs, nW3 = (uint32_t)(p.NC * p.Coutp * 2);
+    const uint32_t nWd = 9u * p.Cexp / 8u, nB = (uint32_t)p.Cexp / 4u, nB3 = (uint32_t)p.Cout / 4u;
+    const uint32_t nW = nW1 + nW3 + nWd + 2u * nB + nB3;
     // tile pixel `pix` is image pixel gh0 * W + pix of image n (strips are full-width rows): in the image for pix in [pix_lo, pix_hi)
     const int pix_lo = max(0, -gh0 * p.W), pix_hi = min(p.P_x, (p.H - gh0) * p.W);
     const uint8_t* x0 = reinterpret_cast<const uint8_t*>(p.x) + ((size_t)n * p.H + gh0) * p.W * p.Cin * 2;   // not dereferenced outside the image
     const uint32_t cmask = (1u << cs) - 1u, cin_chunks = (uint32_t)p.Cin >> 3, cin_bytes = (uint32_t)p.Cin * 2u;
     const uint32_t swz_mask = ((uint32_t)p.row_bytes >> 4) - 1u;
-    uint4 val[kBatch];
-    uint32_t dst[kBatch];
-    auto issue = [&](int base) {
-#pragma unroll
-      for (int k = 0; k < kBatch; ++k) {
-        uint32_t i = (uint32_t)(base + k * kComputeThreads);
-        const uint8_t* src = nullptr;
-        dst[k] = 0xffffffffu;
-        val[k] = make_uint4(0, 0, 0, 0);
-        if (i < (uint32_t)(nX + nW1)) {
-          // X and W1: row-major [row][Cin] -> swizzled rows of Kp channels; chunk i of the tile lies at byte 16 i,
-          // its 16-byte column XORed with the row's swizzle phase (address bits 7..)
-          const bool is_x = i < (uint32_t)nX;
-          if (!is_x) i -= nX;
-          const uint32_t row = i >> cs, ch = i & cmask;
-          const bool ok = ch < cin_chunks && (!is_x || ((int)row >= pix_lo && (int)row < pix_hi));
-          if (ok) src = (is_x ? x0 : reinterpret_cast<const uint8_t*>(p.w1)) + row * cin_bytes + ch * 16u;
-          dst[k] = (is_x ? p.off_x : p.off_w1) + ((i << 4) ^ (((i >> 3) & swz_mask) << 4));
-        } else if ((i -= nX + nW1) < (uint32_t)nW3) {
-          const uint32_t half = i & 1u, c = (i >> 1) / (uint32_t)p.Coutp, row = (i >> 1) - c * p.Coutp;
-          if (row < (uint32_t)p.Cout) src = reinterpret_cast<const uint8_t*>(p.w3) + (row * p.Cexp + c * kChunk + half * 8u) * 2u;
-          dst[k] = p.off_w3 + c * p.Coutp * kChunkRowBytes + swz_offset(row, half, kChunkRowBytes);
-        } else if ((i -= nW3) < (uint32_t)nWd) {
-          src = reinterpret_cast<const uint8_t*>(p.wd) + i * 16u;
-          dst[k] = p.off_wd + i * 16u;
-        } else if ((i -= nWd) < (uint32_t)nB) {
-          src = reinterpret_cast<const uint8_t*>(p.b1) + i * 16u;
-          dst[k] = p.off_b1 + i * 16u;
-        } else if ((i -= nB) < (uint32_t)nB) {
-          src = reinterpret_cast<const uint8_t*>(p.bd) + i * 16u;
-          dst[k] = p.off_bd + i * 16u;
-        } else if ((i -= nB) < (uint32_t)nB3) {
-          src = reinterpret_cast<const uint8_t*>(p.b3) + i * 16u;
-          dst[k] = p.off_b3 + i * 16u;
-        }
-        if (src) val[k] = __ldg(reinterpret_cast<const uint4*>(src));
+    // X and W1: row-major [row][Cin] -> swizzled rows of Kp channels; chunk i of a tile lies at byte 16 i, its 16-byte
+    // column XORed with the row's swizzle phase (address bits 7..). Returns the shared-memory offset; src = null: zeros.
+    auto x_slot = [&](uint32_t i, const uint8_t*& src) -> uint32_t {
+      const uint32_t row = i >> cs, ch = i & cmask;
+      src = (ch < cin_chunks && (int)row >= pix_lo && (int)row < pix_hi) ? x0 + row * cin_bytes + ch * 16u : nullptr;
+      return p.off_x + ((i << 4) ^ (((i >> 3) & swz_mask) << 4));
+    };
+    auto w_slot = [&](uint32_t i, const uint8_t*& src) -> uint32_t {
+      if (i < nW1) {
+        const uint32_t row = i >> cs, ch = i & cmask;
+        src = ch < cin_chunks ? reinterpret_cast<const uint8_t*>(p.w1) + row * cin_bytes + ch * 16u : nullptr;
+        return p.off_w1 + ((i << 4) ^ (((i >> 3) & swz_mask) << 4));
       }
+      if ((i -= nW1) < nW3) {
+        const uint32_t half = i & 1u, c = __umulhi(i >> 1, p.coutp_recip), row = (i >> 1) - c * p.Coutp;
+        src = row < (uint32_t)p.Cout ? reinterpret_cast<const uint8_t*>(p.w3) + (row * p.Cexp + c * kChunk + half * 8u) * 2u : nullptr;
+        return p.off_w3 + c * p.Coutp * kChunkRowBytes + swz_offset(row, half, kChunkRowBytes);
+      }
+      if ((i -= nW3) < nWd) { src = reinterpret_cast<const uint8_t*>(p.wd) + i * 16u; return p.off_wd + i * 16u; }
+      if ((i -= nWd) < nB) { src = reinterpret_cast<const uint8_t*>(p.b1) + i * 16u; return p.off_b1 + i * 16u; }
+      if ((i -= nB) < nB) { src = reinterpret_cast<const uint8_t*>(p.bd) + i * 16u; return p.off_bd + i * 16u; }
+      i -= nB;
+      src = reinterpret_cast<const uint8_t*>(p.b3) + i * 16u;
+      return p.off_b3 + i * 16u;
     };
-    auto commit = [&]() {
+    auto load_or_zero = [](const uint8_t* src) {
+      return src ? __ldg(reinterpret_cast<const uint4*>(src)) : make_uint4(0, 0, 0, 0);
+    };
+    uint4 vx[kBX], vw[kBW];
+    uint32_t dx[kBX], dw[kBW];
 #pragma unroll
-      for (int k = 0; k < kBatch; ++k)
-        if (dst[k] != 0xffffffffu) *reinterpret_cast<uint4*>(smem + dst[k]) = val[k];
-    };
-    issue(tid);
+    for (int k = 0; k < kBX; ++k) {
+      const uint32_t i = (uint32_t)(tid + k * kComputeThreads);
+      const uint8_t* src = nullptr;
+      dx[k] = 0xffffffffu;
+      if (i < nX) dx[k] = x_slot(i, src);
+      vx[k] = load_or_zero(src);
+    }
+#pragma unroll
+    for (int k = 0; k < kBW; ++k) {
+      const uint32_t i = (uint32_t)(tid + k * kComputeThreads);
+      const uint8_t* src = nullptr;
+      dw[k] = 0xffffffffu;
+      if (i < nW) dw[k] = w_slot(i, src);
+      vw[k] = load_or_zero(src);
+    }
     if (warp == 0) {
       tmem_alloc(tmem_slot, (uint32_t)p.tmem_cols);
       tmem_relinquish();
     }
-    commit();
-    for (int base = tid + kBatch * kComputeThreads; base < total; base += kBatch * kComputeThreads) {
-      issue(base);
-      commit();
+#pragma unroll
+    for (int k = 0; k < kBX; ++k)
+      if (dx[k] != 0xffffffffu) *reinterpret_cast<uint4*>(smem + dx[k]) = vx[k];
+#pragma unroll
+    for (int k = 0; k < kBW; ++k)
+      if (dw[k] != 0xffffffffu) *reinterpret_cast<uint4*>(smem + dw[k]) = vw[k];
+    // shapes with more slots than the batched pass covers
+    for (uint32_t i = (uint32_t)(tid + kBX * kComputeThreads); i < nX; i += kComputeThreads) {
+      const uint8_t* src;
+      const uint32_t d = x_slot(i, src);
+      *reinterpret_cast<uint4*>(smem + d) = load_or_zero(src);
+    }
+    for (uint32_t i = (uint32_t)(tid + kBW * kComputeThreads); i < nW; i += kComputeThreads) {
+      const uint8_t* src;
+      const uint32_t d = w_slot(i, src);
+      *reinterpret_cast<uint4*>(smem + d) = load_or_zero(src);
     }
     // the zero padding columns of the two E chunk buffers (written once: every chunk reuses them)
     for (int i = tid; i < p.IH * 8; i += kComputeThreads) {
@@ -472,7 +487,8 @@ mbv2_fused_kernel(const Mbv2Params p) {
                 for (int q = 0; q < 8; ++q) v[q] = __uint_as_float(acc[h * 8 + q]) + sB3[j + q];
                 const size_t off = (gpix0 + po) * p.Cout + j;
                 if (p.residual) {
-                  const uint4 xr = __ldg(reinterpret_cast<const uint4*>(p.x + off));
+                  // stride 1, Cin == Cout: output pixel po is pixel po + W of the input tile (one halo row above)
+                  const uint4 xr = *reinterpret_cast<const uint4*>(sX + swz_offset(po + p.W, j >> 3, p.row_bytes));
                   v[0] += bf16_lo(xr.x); v[1] += bf16_hi(xr.x); v[2] += bf16_lo(xr.y); v[3] += bf16_hi(xr.y);
                   v[4] += bf16_lo(xr.z); v[5] += bf16_hi(xr.z); v[6] += bf16_lo(xr.w); v[7] += bf16_hi(xr.w);
                 }
@@ -556,6 +572,7 @@ ago_status_t mbv2_plan(Plan* plan, FusedState* st, std::string* err) {
   q.swizzle = q.Kp == 16 ? tc::SW_32B : (q.Kp == 32 ? tc::SW_64B : tc::SW_128B);
   q.Coutp = round_up(q.Cout, 16);
   q.NC = q.Cexp / kChunk;
+  q.coutp_recip = (uint32_t)((1ull << 32) / (uint64_t)q.Coutp + 1ull);
   // Rows per CTA: fewest waves over the SMs, then least halo + tail work.
   int best_R = 0; double best_cost = 0; int best_smem = 0;
   const int sms = 148;
