@@ -43,7 +43,11 @@ using namespace tc;
 
 constexpr int kComputeWarps = 28;                  // expand epilogue, depthwise, project epilogue
 constexpr int kComputeThreads = kComputeWarps * 32;
-constexpr int kIssuers = 4;                        // one MMA-issuing warp per SM sub-partition
+constexpr int kGroupWarps = kComputeWarps / 2;     // two groups of compute warps on alternating chunks
+constexpr int kGroupThreads = kGroupWarps * 32;
+constexpr int kTilesPerWarp = 3;                   // expand-epilogue tiles per warp: at most 8 tiles over >= 3 warps of a lane quarter
+constexpr int kIssuers = 4;                        // MMA-issuing warps (one per SM sub-partition)
+constexpr int kIssuersPerRole = kIssuers / 2;      // two for the expand GEMMs, two for the project GEMMs
 constexpr int kThreads = kComputeThreads + 32 * kIssuers;
 constexpr int kChunk = 16;      // expanded channels per chunk = one MMA K step of the project GEMM
 constexpr int kChunkRowBytes = 32;
@@ -189,8 +193,10 @@ mbv2_fused_kernel(const Mbv2Params p) {
   uint64_t* bar_d = bars + 4;       // [2] project MMA has consumed D[b] (MMA commit)
   uint64_t* bar_tfree = bars + 6;   // [2] expand buffer b drained and E chunk written (compute -> issuer)
   uint64_t* bar_dready = bars + 8;  // [2] D[b] written (compute -> issuer)
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 10);
-  volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(bars + 11);
+  uint64_t* bar_done = bars + 10;   // every project MMA complete (the groups do not follow each other's bar_d phases)
+  uint64_t* bar_stagger = bars + 11;   // group 0 has finished its first expand epilogue: group 1 starts (half a period behind)
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 12);
+  volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(bars + 13);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int n = blockIdx.x / p.strips, strip = blockIdx.x % p.strips;
@@ -202,11 +208,13 @@ mbv2_fused_kernel(const Mbv2Params p) {
   if (tid == kComputeThreads) {
     *abort_flag = 0u;
     for (int i = 0; i < 2; ++i) {
-      mbar_init(bar_e + i, kIssuers);
-      mbar_init(bar_d + i, kIssuers);
+      mbar_init(bar_e + i, kIssuersPerRole);
+      mbar_init(bar_d + i, kIssuersPerRole);
       mbar_init(bar_tfree + i, 1);
       mbar_init(bar_dready + i, 1);
     }
+    mbar_init(bar_done, kIssuersPerRole);
+    mbar_init(bar_stagger, 1);
     fence_mbar_init();
     fence_proxy_async_smem();
   }
@@ -306,101 +314,116 @@ mbv2_fused_kernel(const Mbv2Params p) {
   const uint32_t tmem_base = *tmem_slot;
 
   if (warp >= kComputeWarps) {
-    // ================= MMA issue warps: issuer i owns M tiles i, i+4, ... (one lane each) =================
-    const int iw = warp - kComputeWarps;
+    // ================= MMA issue warps (one lane each): two issue the expand GEMMs, two the project GEMMs, =================
+    // each pair splitting the M tiles between them. Separate roles keep an issuer from sitting in the wait for one
+    // event while the other kind is due: the project of chunk c has to be through before the depthwise stage of
+    // chunk c + 2 may overwrite its operand.
+    const int role = (warp - kComputeWarps) >> 1;     // 0: expand, 1: project
+    const int iw = (warp - kComputeWarps) & 1;
     if (lane == 0) {
-      const uint32_t idesc_e = make_idesc_bf16(128, kChunk);
-      const uint32_t idesc_p = make_idesc_bf16(128, (uint32_t)p.Coutp);
-      const uint32_t sbo_x = 8u * (uint32_t)p.row_bytes;
-      const uint64_t xdesc0 = make_smem_desc(smem_u32(sX), 0, sbo_x, p.swizzle);
-      const uint64_t w1desc0 = make_smem_desc(smem_u32(sW1), 0, sbo_x, p.swizzle);
-      // D: un-swizzled K-major; the two 8-channel planes are the two K core-matrix columns
-      const uint64_t ddesc0 = make_smem_desc(smem_u32(sD), (uint32_t)p.d_plane, 128, SW_NONE);
-      const uint64_t w3desc0 = make_smem_desc(smem_u32(sW3), 0, 256, SW_32B);
-      const int ksteps = p.Kp / 16;
-      const uint32_t a_tile_step = (uint32_t)(128 * p.row_bytes) >> 4;
-
-      auto issue_expand = [&](int c) {
-        const int b = c & 1;
-        const uint64_t bdesc = w1desc0 + (uint64_t)((c * kChunk * p.row_bytes) >> 4);
-        for (int t = iw; t < p.M1; t += kIssuers) {
-          const uint64_t adesc = xdesc0 + (uint64_t)t * a_tile_step;
-          const uint32_t d_tmem = tmem_base + p.ecol0 + (b * p.M1 + t) * kChunk;
-          umma_bf16(d_tmem, adesc, bdesc, idesc_e, 0);
-          for (int ks = 1; ks < ksteps; ++ks) umma_bf16(d_tmem, adesc + 2u * ks, bdesc + 2u * ks, idesc_e, 1);
-        }
-        umma_commit(bar_e + b);
-      };
       tcgen05_fence_after_sync();
-      issue_expand(0);
-      if (p.NC > 1) issue_expand(1);
-      for (int c = 0; c < p.NC; ++c) {
-        const int b = c & 1;
-        const uint32_t ph = (uint32_t)(c >> 1) & 1u;
-        if (c + 2 < p.NC) {
-          mbar_wait(bar_tfree + b, ph, abort_flag, p.status, 0x105);
-          tcgen05_fence_after_sync();
-          issue_expand(c + 2);
+      if (role == 0) {
+        const uint32_t idesc_e = make_idesc_bf16(128, kChunk);
+        const uint32_t sbo_x = 8u * (uint32_t)p.row_bytes;
+        const uint64_t xdesc0 = make_smem_desc(smem_u32(sX), 0, sbo_x, p.swizzle);
+        const uint64_t w1desc0 = make_smem_desc(smem_u32(sW1), 0, sbo_x, p.swizzle);
+        const int ksteps = p.Kp / 16;
+        const uint32_t a_tile_step = (uint32_t)(128 * p.row_bytes) >> 4;
+        for (int c = 0; c < p.NC; ++c) {
+          const int b = c & 1;
+          if (c >= 2) {   // expand buffer b drained by the expand epilogue of chunk c - 2
+            mbar_wait(bar_tfree + b, (uint32_t)((c - 2) >> 1) & 1u, abort_flag, p.status, 0x105);
+            tcgen05_fence_after_sync();
+          }
+          const uint64_t bdesc = w1desc0 + (uint64_t)((c * kChunk * p.row_bytes) >> 4);
+          for (int t = iw; t < p.M1; t += kIssuersPerRole) {
+            const uint64_t adesc = xdesc0 + (uint64_t)t * a_tile_step;
+            const uint32_t d_tmem = tmem_base + p.ecol0 + (b * p.M1 + t) * kChunk;
+            umma_bf16(d_tmem, adesc, bdesc, idesc_e, 0);
+            for (int ks = 1; ks < ksteps; ++ks) umma_bf16(d_tmem, adesc + 2u * ks, bdesc + 2u * ks, idesc_e, 1);
+          }
+          umma_commit(bar_e + b);
         }
-        mbar_wait(bar_dready + b, ph, abort_flag, p.status, 0x106);
-        tcgen05_fence_after_sync();
-        const uint64_t bdesc = w3desc0 + (uint64_t)((c * p.Coutp * kChunkRowBytes) >> 4);
-        for (int t = iw; t < p.M2; t += kIssuers)
-          umma_bf16(tmem_base + p.pcol0 + t * p.Coutp, ddesc0 + (uint64_t)((b * d_bytes + t * 128 * 16) >> 4), bdesc,
-                    idesc_p, c > 0);
-        umma_commit(bar_d + b);
+      } else {
+        const uint32_t idesc_p = make_idesc_bf16(128, (uint32_t)p.Coutp);
+        // D: un-swizzled K-major; the two 8-channel planes are the two K core-matrix columns
+        const uint64_t ddesc0 = make_smem_desc(smem_u32(sD), (uint32_t)p.d_plane, 128, SW_NONE);
+        const uint64_t w3desc0 = make_smem_desc(smem_u32(sW3), 0, 256, SW_32B);
+        for (int c = 0; c < p.NC; ++c) {
+          const int b = c & 1;
+          mbar_wait(bar_dready + b, (uint32_t)(c >> 1) & 1u, abort_flag, p.status, 0x106);
+          tcgen05_fence_after_sync();
+          const uint64_t bdesc = w3desc0 + (uint64_t)((c * p.Coutp * kChunkRowBytes) >> 4);
+          for (int t = iw; t < p.M2; t += kIssuersPerRole)
+            umma_bf16(tmem_base + p.pcol0 + t * p.Coutp, ddesc0 + (uint64_t)((b * d_bytes + t * 128 * 16) >> 4), bdesc,
+                      idesc_p, c > 0);
+          umma_commit(bar_d + b);
+        }
+        umma_commit(bar_done);
       }
     }
     __syncwarp();
   } else {
     // ================================== compute warps ==================================
-    const int ctid = tid;   // compute warps are warps 0 .. kComputeWarps-1
+    // The compute warps form two groups of 14; group g owns the chunks c = g, g + 2, ... (expand buffer, E buffer and
+    // D buffer g). A group alternates expand epilogue and depthwise stage with a group-wide barrier after each; the
+    // two groups are out of phase, so one group's barrier and tensor-memory latencies hide behind the other's arithmetic.
+    const int g = warp / kGroupWarps;
+    const int gwarp0 = g * kGroupWarps;           // first warp of the group
+    const int gt = tid - gwarp0 * 32;             // thread index in the group
+    const uint32_t gbar = 1u + (uint32_t)g;       // named barrier of the group
     const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
     // Depthwise work split: thread = (channel pair, slot). Stride 1: an item is a segment of 7 output columns of one
-    // output row (56 columns x 14 rows x 8 pairs = one item per thread). Stride 2: an item is one output column of one
-    // row group.
-    constexpr int kSlots = kComputeThreads / 8;
-    const int cp = ctid & 7, slot = ctid >> 3;
+    // output row. Stride 2: an item is one output column of one row group.
+    constexpr int kSlots = kGroupThreads / 8;
+    const int cp = gt & 7, slot = gt >> 3;
     const int cp_off = (cp & 3) * 4;   // byte offset inside a 16-byte pixel entry
     const uint32_t e_pitch = (uint32_t)p.IW * 16u, d_pitch = (uint32_t)p.Wo * 16u;
     const int nseg = (p.Wo + kSegCols - 1) / kSegCols;
-    const int groups = max(1, min(rows_valid, kSlots / max(1, min(p.Wo, kSlots))));
+    const int groups = max(1, min(rows_valid, kSlots / max(1, min(p.Wo, kSlots))));   // stride 2: row groups
     const int rows_per_group = (rows_valid + groups - 1) / groups;
     const int per_row = p.stride == 1 ? nseg : p.Wo;                       // items per output row / per row group
     const int dw_items = per_row * (p.stride == 1 ? rows_valid : groups);
-    const int item0_r = slot / per_row, item0_c = slot - item0_r * per_row;   // first item (most shapes have at most one)
+    const int item0_r = slot / per_row, item0_c = slot - item0_r * per_row;   // the thread's first item
+    const int step_r = kSlots / per_row, step_c = kSlots - step_r * per_row;  // item += kSlots in (row, column) form
     const int e_bytes = 2 * p.e_plane;
-    // expand-epilogue rows of this thread: tile (warp>>2) + 7k, k < 2. e_off[k]: byte offset of the pixel in an E
-    // plane (the tile has no padding columns, the E chunk does), -1: no such pixel; bit k of e_inimg: the row lies
-    // inside the image (the rest is the zero padding of the intermediate tensor)
-    int e_off[2] = {-1, -1};
+    // Expand-epilogue tiles of this warp: the group's warps of one tensor-memory lane quarter (warp & 3) share the M1
+    // tiles round-robin, at most kTilesPerWarp each. e_pix[k]: pixel index in an E plane (the tile has no padding
+    // columns, the E chunk does), -1: no such pixel; bit k of e_inimg: the row lies inside the image (the rest is the
+    // zero padding of the intermediate tensor).
+    const int q_first = (((warp & 3) - gwarp0) & 3);                // group-relative index of the quarter's first warp
+    const int q_mates = (kGroupWarps - q_first + 3) >> 2;           // warps of this quarter in the group (3 or 4)
+    const int q_rank = (warp - gwarp0 - q_first) >> 2;              // this warp's rank among them
+    int e_pix[kTilesPerWarp];
     uint32_t e_inimg = 0;
 #pragma unroll
-    for (int k = 0; k < 2; ++k) {
-      const int t = (warp >> 2) + k * (kComputeWarps / 4);
+    for (int k = 0; k < kTilesPerWarp; ++k) {
+      const int t = q_rank + k * q_mates;
       const int pix = t * 128 + (warp & 3) * 32 + lane;
       const int ih = pix / p.W, iw = pix - ih * p.W;
       const int gh = gh0 + ih;
+      e_pix[k] = -1;
       if (t < p.M1 && pix < p.P_x) {
-        e_off[k] = (ih * p.IW + iw + 1) * 16;
+        e_pix[k] = ih * p.IW + iw + 1;
         if (gh >= 0 && gh < p.H) e_inimg |= 1u << k;
       }
     }
 
-    // ---- P3: expand epilogue of chunk c -> E[c & 1]: + b1, ReLU6, zero outside the image, bf16 ----
-    auto expand_epilogue = [&](int c) {
-      const int b = c & 1;
-      mbar_wait(bar_e + b, (uint32_t)(c >> 1) & 1u, abort_flag, p.status, 0x102);
+    // Keep the groups out of phase: group 1 starts once group 0 is through its first expand epilogue.
+    if (g == 1) mbar_wait(bar_stagger, 0, abort_flag, p.status, 0x107);
+    for (int c = g, it = 0; c < p.NC; c += 2, ++it) {
+      // ---- P3: expand epilogue of chunk c -> E[g]: + b1, ReLU6, zero outside the image, bf16 ----
+      mbar_wait(bar_e + g, (uint32_t)it & 1u, abort_flag, p.status, 0x102);
       tcgen05_fence_after_sync();
-      uint8_t* e_buf = sE + b * e_bytes;
+      uint8_t* e_buf = sE + g * e_bytes;
 #pragma unroll
-      for (int k = 0; k < 2; ++k) {
-        const int t = (warp >> 2) + k * (kComputeWarps / 4);
+      for (int k = 0; k < kTilesPerWarp; ++k) {
+        const int t = q_rank + k * q_mates;
         if (t >= p.M1) break;
         uint32_t acc[16];
-        tmem_ld_x16(tmem_base + lane_base + p.ecol0 + (b * p.M1 + t) * kChunk, acc);
+        tmem_ld_x16(tmem_base + lane_base + p.ecol0 + (g * p.M1 + t) * kChunk, acc);
         tmem_ld_wait();
-        if (e_off[k] >= 0) {
+        if (e_pix[k] >= 0) {
           uint32_t w[8];
           if ((e_inimg >> k) & 1u) {
             const float4* bb = reinterpret_cast<const float4*>(sB1 + c * kChunk);
@@ -414,37 +437,31 @@ mbv2_fused_kernel(const Mbv2Params p) {
 #pragma unroll
             for (int j = 0; j < 8; ++j) w[j] = 0u;
           }
-          *reinterpret_cast<uint4*>(e_buf + e_off[k]) = make_uint4(w[0], w[1], w[2], w[3]);
-          *reinterpret_cast<uint4*>(e_buf + p.e_plane + e_off[k]) = make_uint4(w[4], w[5], w[6], w[7]);
+          *reinterpret_cast<uint4*>(e_buf + e_pix[k] * 16) = make_uint4(w[0], w[1], w[2], w[3]);
+          *reinterpret_cast<uint4*>(e_buf + p.e_plane + e_pix[k] * 16) = make_uint4(w[4], w[5], w[6], w[7]);
         }
       }
       tcgen05_fence_before_sync();
-    };
+      named_barrier_sync(gbar, kGroupThreads);
+      if (gt == 0) {
+        mbar_arrive(bar_tfree + g);
+        if (c == 0) mbar_arrive(bar_stagger);
+      }
 
-    expand_epilogue(0);
-    named_barrier_sync(1, kComputeThreads);
-    if (ctid == 0) mbar_arrive(bar_tfree + 0);
+      // D[g] was read by the project MMA of chunk c-2
+      if (it >= 1) mbar_wait(bar_d + g, (uint32_t)(it - 1) & 1u, abort_flag, p.status, 0x103);
 
-    // One barrier per chunk: a warp runs the depthwise stage of chunk c (E[c & 1] -> D[c & 1]) and then the expand
-    // epilogue of chunk c + 1 (-> E[(c + 1) & 1]); the warps drift apart in between, so the tensor-memory load latency
-    // of one hides behind the arithmetic of the others.
-    for (int c = 0; c < p.NC; ++c) {
-      const int b = c & 1;
-      // D[b] was read by the project MMA of chunk c-2
-      if (c >= 2) mbar_wait(bar_d + b, (uint32_t)((c - 2) >> 1) & 1u, abort_flag, p.status, 0x103);
-
-      // ---- P4: depthwise 3x3 + bias + ReLU6 on CUDA cores: E chunk -> D[b] (A operand of the project GEMM) ----
+      // ---- P4: depthwise 3x3 + bias + ReLU6 on CUDA cores: E[g] -> D[g] (A operand of the project GEMM) ----
       {
         const int ch = c * kChunk + cp * 2;
         uint32_t wgt[9];   // packed bf16 pairs
 #pragma unroll
         for (int tap = 0; tap < 9; ++tap) wgt[tap] = *reinterpret_cast<const uint32_t*>(sWd + (tap * p.Cexp + ch) * 2);
         const float2 bias = *reinterpret_cast<const float2*>(sBd + ch);
-        const uint32_t e_plane = smem_u32(sE) + (uint32_t)(b * e_bytes + (cp >> 2) * p.e_plane + cp_off);
-        const uint32_t d_plane = smem_u32(sD) + (uint32_t)(b * d_bytes + (cp >> 2) * p.d_plane + cp_off);
+        const uint32_t e_plane = smem_u32(sE) + (uint32_t)(g * e_bytes + (cp >> 2) * p.e_plane + cp_off);
+        const uint32_t d_plane = smem_u32(sD) + (uint32_t)(g * d_bytes + (cp >> 2) * p.d_plane + cp_off);
+        int r = item0_r, col = item0_c;
         for (int item = slot; item < dw_items; item += kSlots) {
-          int r = item0_r, col = item0_c;
-          if (item != slot) { r = item / per_row; col = item - r * per_row; }
           if (p.stride == 1) {
             const int wo = col * kSegCols;
             depthwise_segment(e_plane + (uint32_t)r * e_pitch + wo * 16, d_plane + (uint32_t)r * d_pitch + wo * 16, e_pitch,
@@ -453,21 +470,18 @@ mbv2_fused_kernel(const Mbv2Params p) {
             const int r0 = r * rows_per_group, r1 = min(rows_valid, r0 + rows_per_group);
             if (r0 < r1) depthwise_column_s2(e_plane + col * 32, d_plane + col * 16, r0, r1, p.IW, p.Wo, wgt, bias);
           }
+          r += step_r; col += step_c;
+          if (col >= per_row) { col -= per_row; ++r; }
         }
       }
-      if (c + 1 < p.NC) expand_epilogue(c + 1);
       fence_proxy_async_smem();
-      named_barrier_sync(1, kComputeThreads);
-      if (ctid == 0) {
-        mbar_arrive(bar_dready + b);
-        if (c + 1 < p.NC) mbar_arrive(bar_tfree + ((c + 1) & 1));
-      }
+      named_barrier_sync(gbar, kGroupThreads);
+      if (gt == 0) mbar_arrive(bar_dready + g);
     }
 
     // ---- P6: project epilogue: + b3 (+ residual), bf16, 16-byte stores ----
     {
-      const int last = p.NC - 1;
-      mbar_wait(bar_d + (last & 1), (uint32_t)(last >> 1) & 1u, abort_flag, p.status, 0x104);
+      mbar_wait(bar_done, 0, abort_flag, p.status, 0x104);
       tcgen05_fence_after_sync();
       const int valid_pix = rows_valid * p.Wo;
       const size_t gpix0 = ((size_t)n * p.Ho + ho0) * p.Wo;
