@@ -142,35 +142,44 @@ __device__ __forceinline__ void depthwise_column_s2(uint32_t e_col, uint32_t d_c
   }
 }
 
-// Stride-1 depthwise 3x3 for one (channel pair, output row, segment of 7 output columns), fully
-// unrolled: three input columns (3 rows each) stay packed in registers and rotate by renaming, all
-// shared-memory offsets are immediates. e_row: address of the segment's first input pixel in the
-// row above the output row; d_row: address of its first output pixel; ncol <= 7 columns are stored
-// (the loads of a ragged segment run past the row end, inside shared memory; those results are dropped).
+// Stride-1 depthwise 3x3 for one channel pair and a block of 2 output rows x 7 output columns, fully
+// unrolled: three input columns (4 rows each) stay packed in registers and rotate by renaming, all
+// shared-memory offsets are immediates; each loaded pixel feeds up to six outputs. e_row: address of
+// the block's first input pixel in the row above the first output row; d_row: address of its first
+// output pixel; ncol <= 7 columns and nrows <= 2 rows are stored (the loads of a ragged block run
+// past the valid pixels, inside shared memory; those results are dropped).
 constexpr int kSegCols = 7;
-__device__ __forceinline__ void depthwise_segment(uint32_t e_row, uint32_t d_row, uint32_t e_pitch, int ncol,
-                                                  const uint32_t (&w)[9], float2 bias) {
-  const uint32_t e0 = e_row, e1 = e_row + e_pitch, e2 = e1 + e_pitch;
-  uint32_t c0[3], c1[3], c2[3];
-  c0[0] = lds32<0>(e0); c0[1] = lds32<0>(e1); c0[2] = lds32<0>(e2);
-  c1[0] = lds32<16>(e0); c1[1] = lds32<16>(e1); c1[2] = lds32<16>(e2);
+__device__ __forceinline__ void depthwise_block(uint32_t e_row, uint32_t d_row, uint32_t e_pitch, uint32_t d_pitch, int ncol,
+                                                int nrows, const uint32_t (&w)[9], float2 bias) {
+  const uint32_t e0 = e_row, e1 = e0 + e_pitch, e2 = e1 + e_pitch, e3 = e2 + e_pitch;
+  const uint32_t d0 = d_row, d1 = d_row + d_pitch;
+  uint32_t c0[4], c1[4], c2[4];
+  c0[0] = lds32<0>(e0); c0[1] = lds32<0>(e1); c0[2] = lds32<0>(e2); c0[3] = lds32<0>(e3);
+  c1[0] = lds32<16>(e0); c1[1] = lds32<16>(e1); c1[2] = lds32<16>(e2); c1[3] = lds32<16>(e3);
 #define AGO_DW_STEP(J, A, B, C)                                                                       \
   {                                                                                                   \
-    C[0] = lds32<(J + 2) * 16>(e0); C[1] = lds32<(J + 2) * 16>(e1); C[2] = lds32<(J + 2) * 16>(e2);   \
-    float2 acc = bias;                                                                                \
-    fma_pair(acc, A[0], w[0]); fma_pair(acc, B[0], w[1]); fma_pair(acc, C[0], w[2]);                  \
-    fma_pair(acc, A[1], w[3]); fma_pair(acc, B[1], w[4]); fma_pair(acc, C[1], w[5]);                  \
-    fma_pair(acc, A[2], w[6]); fma_pair(acc, B[2], w[7]); fma_pair(acc, C[2], w[8]);                  \
-    if (FULL || J < ncol) sts32<J * 16>(d_row, relu6_pack(acc.x, acc.y));                             \
+    C[0] = lds32<(J + 2) * 16>(e0); C[1] = lds32<(J + 2) * 16>(e1);                                   \
+    C[2] = lds32<(J + 2) * 16>(e2); C[3] = lds32<(J + 2) * 16>(e3);                                   \
+    float2 acc0 = bias, acc1 = bias;                                                                  \
+    fma_pair(acc0, A[0], w[0]); fma_pair(acc0, B[0], w[1]); fma_pair(acc0, C[0], w[2]);               \
+    fma_pair(acc0, A[1], w[3]); fma_pair(acc0, B[1], w[4]); fma_pair(acc0, C[1], w[5]);               \
+    fma_pair(acc1, A[1], w[0]); fma_pair(acc1, B[1], w[1]); fma_pair(acc1, C[1], w[2]);               \
+    fma_pair(acc0, A[2], w[6]); fma_pair(acc0, B[2], w[7]); fma_pair(acc0, C[2], w[8]);               \
+    fma_pair(acc1, A[2], w[3]); fma_pair(acc1, B[2], w[4]); fma_pair(acc1, C[2], w[5]);               \
+    fma_pair(acc1, A[3], w[6]); fma_pair(acc1, B[3], w[7]); fma_pair(acc1, C[3], w[8]);               \
+    if (FULL || J < ncol) {                                                                           \
+      sts32<J * 16>(d0, relu6_pack(acc0.x, acc0.y));                                                  \
+      if (FULL || nrows > 1) sts32<J * 16>(d1, relu6_pack(acc1.x, acc1.y));                           \
+    }                                                                                                 \
   }
-  if (ncol == kSegCols) {
+  if (ncol == kSegCols && nrows == 2) {
     constexpr bool FULL = true;
     AGO_DW_STEP(0, c0, c1, c2) AGO_DW_STEP(1, c1, c2, c0) AGO_DW_STEP(2, c2, c0, c1) AGO_DW_STEP(3, c0, c1, c2)
     AGO_DW_STEP(4, c1, c2, c0) AGO_DW_STEP(5, c2, c0, c1) AGO_DW_STEP(6, c0, c1, c2)
   } else {
     constexpr bool FULL = false;
     AGO_DW_STEP(0, c0, c1, c2) AGO_DW_STEP(1, c1, c2, c0) AGO_DW_STEP(2, c2, c0, c1) AGO_DW_STEP(3, c0, c1, c2)
-    AGO_DW_STEP(4, c1, c2, c0) AGO_DW_STEP(5, c2, c0, c1)
+    AGO_DW_STEP(4, c1, c2, c0) AGO_DW_STEP(5, c2, c0, c1) AGO_DW_STEP(6, c0, c1, c2)
   }
 #undef AGO_DW_STEP
 }
@@ -322,25 +331,31 @@ mbv2_fused_kernel(const Mbv2Params p) {
     const int iw = (warp - kComputeWarps) & 1;
     if (lane == 0) {
       tcgen05_fence_after_sync();
+      // Descriptors as (low, high) words: start address and LBO live in the low word, so the loops advance an
+      // operand with one 32-bit add (shared-memory addresses >> 4 stay below the 14-bit field limit).
       if (role == 0) {
         const uint32_t idesc_e = make_idesc_bf16(128, kChunk);
         const uint32_t sbo_x = 8u * (uint32_t)p.row_bytes;
         const uint64_t xdesc0 = make_smem_desc(smem_u32(sX), 0, sbo_x, p.swizzle);
         const uint64_t w1desc0 = make_smem_desc(smem_u32(sW1), 0, sbo_x, p.swizzle);
+        const uint32_t x_hi = (uint32_t)(xdesc0 >> 32), w1_hi = (uint32_t)(w1desc0 >> 32);
         const int ksteps = p.Kp / 16;
-        const uint32_t a_tile_step = (uint32_t)(128 * p.row_bytes) >> 4;
-        for (int c = 0; c < p.NC; ++c) {
+        const uint32_t a_step = ((uint32_t)(kIssuersPerRole * 128 * p.row_bytes) >> 4) - 2u * (uint32_t)ksteps;
+        const uint32_t a_lo0 = (uint32_t)xdesc0 + ((uint32_t)(iw * 128 * p.row_bytes) >> 4);
+        const uint32_t b_step = (uint32_t)(kChunk * p.row_bytes) >> 4;
+        uint32_t b_lo = (uint32_t)w1desc0;
+        for (int c = 0; c < p.NC; ++c, b_lo += b_step) {
           const int b = c & 1;
           if (c >= 2) {   // expand buffer b drained by the expand epilogue of chunk c - 2
             mbar_wait(bar_tfree + b, (uint32_t)((c - 2) >> 1) & 1u, abort_flag, p.status, 0x105);
             tcgen05_fence_after_sync();
           }
-          const uint64_t bdesc = w1desc0 + (uint64_t)((c * kChunk * p.row_bytes) >> 4);
-          for (int t = iw; t < p.M1; t += kIssuersPerRole) {
-            const uint64_t adesc = xdesc0 + (uint64_t)t * a_tile_step;
-            const uint32_t d_tmem = tmem_base + p.ecol0 + (b * p.M1 + t) * kChunk;
-            umma_bf16(d_tmem, adesc, bdesc, idesc_e, 0);
-            for (int ks = 1; ks < ksteps; ++ks) umma_bf16(d_tmem, adesc + 2u * ks, bdesc + 2u * ks, idesc_e, 1);
+          uint32_t a_lo = a_lo0;
+          uint32_t d_tmem = tmem_base + p.ecol0 + (b * p.M1 + iw) * kChunk;
+          for (int t = iw; t < p.M1; t += kIssuersPerRole, a_lo += a_step, d_tmem += kIssuersPerRole * kChunk) {
+            umma_bf16_lohi(d_tmem, a_lo, x_hi, b_lo, w1_hi, idesc_e, 0);
+            a_lo += 2u;
+            for (int ks = 1; ks < ksteps; ++ks, a_lo += 2u) umma_bf16_lohi(d_tmem, a_lo, x_hi, b_lo + 2u * ks, w1_hi, idesc_e, 1);
           }
           umma_commit(bar_e + b);
         }
@@ -349,14 +364,20 @@ mbv2_fused_kernel(const Mbv2Params p) {
         // D: un-swizzled K-major; the two 8-channel planes are the two K core-matrix columns
         const uint64_t ddesc0 = make_smem_desc(smem_u32(sD), (uint32_t)p.d_plane, 128, SW_NONE);
         const uint64_t w3desc0 = make_smem_desc(smem_u32(sW3), 0, 256, SW_32B);
-        for (int c = 0; c < p.NC; ++c) {
+        const uint32_t d_hi = (uint32_t)(ddesc0 >> 32), w3_hi = (uint32_t)(w3desc0 >> 32);
+        const uint32_t a_step = (uint32_t)(kIssuersPerRole * 128 * 16) >> 4;
+        const uint32_t b_step = (uint32_t)(p.Coutp * kChunkRowBytes) >> 4;
+        const uint32_t a_lo0[2] = {(uint32_t)ddesc0 + ((uint32_t)(iw * 128 * 16) >> 4),
+                                   (uint32_t)ddesc0 + ((uint32_t)(d_bytes + iw * 128 * 16) >> 4)};
+        const uint32_t d_tmem0 = tmem_base + p.pcol0 + iw * p.Coutp;
+        uint32_t b_lo = (uint32_t)w3desc0;
+        for (int c = 0; c < p.NC; ++c, b_lo += b_step) {
           const int b = c & 1;
           mbar_wait(bar_dready + b, (uint32_t)(c >> 1) & 1u, abort_flag, p.status, 0x106);
           tcgen05_fence_after_sync();
-          const uint64_t bdesc = w3desc0 + (uint64_t)((c * p.Coutp * kChunkRowBytes) >> 4);
-          for (int t = iw; t < p.M2; t += kIssuersPerRole)
-            umma_bf16(tmem_base + p.pcol0 + t * p.Coutp, ddesc0 + (uint64_t)((b * d_bytes + t * 128 * 16) >> 4), bdesc,
-                      idesc_p, c > 0);
+          uint32_t a_lo = a_lo0[b], d_tmem = d_tmem0;
+          for (int t = iw; t < p.M2; t += kIssuersPerRole, a_lo += a_step, d_tmem += kIssuersPerRole * p.Coutp)
+            umma_bf16_lohi(d_tmem, a_lo, d_hi, b_lo, w3_hi, idesc_p, c > 0);
           umma_commit(bar_d + b);
         }
         umma_commit(bar_done);
@@ -373,8 +394,9 @@ mbv2_fused_kernel(const Mbv2Params p) {
     const int gt = tid - gwarp0 * 32;             // thread index in the group
     const uint32_t gbar = 1u + (uint32_t)g;       // named barrier of the group
     const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
-    // Depthwise work split: thread = (channel pair, slot). Stride 1: an item is a segment of 7 output columns of one
-    // output row. Stride 2: an item is one output column of one row group.
+    // Depthwise work split: thread = (channel pair, slot). Stride 1: an item is a block of 2 output rows x 7 output
+    // columns (56 columns x 14 rows x 8 pairs = one item per thread of a group). Stride 2: an item is one output column
+    // of one row group.
     constexpr int kSlots = kGroupThreads / 8;
     const int cp = gt & 7, slot = gt >> 3;
     const int cp_off = (cp & 3) * 4;   // byte offset inside a 16-byte pixel entry
@@ -383,7 +405,7 @@ mbv2_fused_kernel(const Mbv2Params p) {
     const int groups = max(1, min(rows_valid, kSlots / max(1, min(p.Wo, kSlots))));   // stride 2: row groups
     const int rows_per_group = (rows_valid + groups - 1) / groups;
     const int per_row = p.stride == 1 ? nseg : p.Wo;                       // items per output row / per row group
-    const int dw_items = per_row * (p.stride == 1 ? rows_valid : groups);
+    const int dw_items = per_row * (p.stride == 1 ? (rows_valid + 1) / 2 : groups);   // stride 1: blocks of two rows
     const int item0_r = slot / per_row, item0_c = slot - item0_r * per_row;   // the thread's first item
     const int step_r = kSlots / per_row, step_c = kSlots - step_r * per_row;  // item += kSlots in (row, column) form
     const int e_bytes = 2 * p.e_plane;
@@ -464,8 +486,8 @@ mbv2_fused_kernel(const Mbv2Params p) {
         for (int item = slot; item < dw_items; item += kSlots) {
           if (p.stride == 1) {
             const int wo = col * kSegCols;
-            depthwise_segment(e_plane + (uint32_t)r * e_pitch + wo * 16, d_plane + (uint32_t)r * d_pitch + wo * 16, e_pitch,
-                              min(kSegCols, p.Wo - wo), wgt, bias);
+            depthwise_block(e_plane + (uint32_t)(2 * r) * e_pitch + wo * 16, d_plane + (uint32_t)(2 * r) * d_pitch + wo * 16, e_pitch,
+                            d_pitch, min(kSegCols, p.Wo - wo), min(2, rows_valid - 2 * r), wgt, bias);
           } else {
             const int r0 = r * rows_per_group, r1 = min(rows_valid, r0 + rows_per_group);
             if (r0 < r1) depthwise_column_s2(e_plane + col * 32, d_plane + col * 16, r0, r1, p.IW, p.Wo, wgt, bias);
