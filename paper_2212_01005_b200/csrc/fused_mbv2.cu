@@ -331,8 +331,10 @@ mbv2_fused_kernel(const Mbv2Params p) {
     const int iw = (warp - kComputeWarps) & 1;
     if (lane == 0) {
       tcgen05_fence_after_sync();
-      // Descriptors as (low, high) words: start address and LBO live in the low word, so the loops advance an
-      // operand with one 32-bit add (shared-memory addresses >> 4 stay below the 14-bit field limit).
+      // Descriptors as (low, high) words: start address and LBO live in the low word (shared-memory addresses >> 4
+      // stay below the 14-bit field limit), and every per-tile term is precomputed: an issuer shares its scheduler
+      // with seven busy compute warps and gets few issue slots, so the loops spend about four instructions per MMA.
+      constexpr int kMaxTiles = 4;   // M tiles per issuer (at most 8 tiles over two issuers)
       if (role == 0) {
         const uint32_t idesc_e = make_idesc_bf16(128, kChunk);
         const uint32_t sbo_x = 8u * (uint32_t)p.row_bytes;
@@ -340,9 +342,15 @@ mbv2_fused_kernel(const Mbv2Params p) {
         const uint64_t w1desc0 = make_smem_desc(smem_u32(sW1), 0, sbo_x, p.swizzle);
         const uint32_t x_hi = (uint32_t)(xdesc0 >> 32), w1_hi = (uint32_t)(w1desc0 >> 32);
         const int ksteps = p.Kp / 16;
-        const uint32_t a_step = ((uint32_t)(kIssuersPerRole * 128 * p.row_bytes) >> 4) - 2u * (uint32_t)ksteps;
-        const uint32_t a_lo0 = (uint32_t)xdesc0 + ((uint32_t)(iw * 128 * p.row_bytes) >> 4);
-        const uint32_t b_step = (uint32_t)(kChunk * p.row_bytes) >> 4;
+        const int my_tiles = (p.M1 - iw + kIssuersPerRole - 1) / kIssuersPerRole;
+        uint32_t a_lo[kMaxTiles], d_off[kMaxTiles];
+#pragma unroll
+        for (int k = 0; k < kMaxTiles; ++k) {
+          const int t = iw + k * kIssuersPerRole;
+          a_lo[k] = (uint32_t)xdesc0 + ((uint32_t)(t * 128 * p.row_bytes) >> 4);
+          d_off[k] = tmem_base + p.ecol0 + t * kChunk;
+        }
+        const uint32_t b_step = (uint32_t)(kChunk * p.row_bytes) >> 4, buf_cols = (uint32_t)(p.M1 * kChunk);
         uint32_t b_lo = (uint32_t)w1desc0;
         for (int c = 0; c < p.NC; ++c, b_lo += b_step) {
           const int b = c & 1;
@@ -350,12 +358,14 @@ mbv2_fused_kernel(const Mbv2Params p) {
             mbar_wait(bar_tfree + b, (uint32_t)((c - 2) >> 1) & 1u, abort_flag, p.status, 0x105);
             tcgen05_fence_after_sync();
           }
-          uint32_t a_lo = a_lo0;
-          uint32_t d_tmem = tmem_base + p.ecol0 + (b * p.M1 + iw) * kChunk;
-          for (int t = iw; t < p.M1; t += kIssuersPerRole, a_lo += a_step, d_tmem += kIssuersPerRole * kChunk) {
-            umma_bf16_lohi(d_tmem, a_lo, x_hi, b_lo, w1_hi, idesc_e, 0);
-            a_lo += 2u;
-            for (int ks = 1; ks < ksteps; ++ks, a_lo += 2u) umma_bf16_lohi(d_tmem, a_lo, x_hi, b_lo + 2u * ks, w1_hi, idesc_e, 1);
+          const uint32_t dcol = b ? buf_cols : 0u;
+#pragma unroll
+          for (int k = 0; k < kMaxTiles; ++k) {
+            if (k < my_tiles) {
+#pragma unroll
+              for (int ks = 0; ks < 4; ++ks)
+                if (ks < ksteps) umma_bf16_lohi(d_off[k] + dcol, a_lo[k] + 2u * ks, x_hi, b_lo + 2u * ks, w1_hi, idesc_e, ks > 0);
+            }
           }
           umma_commit(bar_e + b);
         }
@@ -365,19 +375,25 @@ mbv2_fused_kernel(const Mbv2Params p) {
         const uint64_t ddesc0 = make_smem_desc(smem_u32(sD), (uint32_t)p.d_plane, 128, SW_NONE);
         const uint64_t w3desc0 = make_smem_desc(smem_u32(sW3), 0, 256, SW_32B);
         const uint32_t d_hi = (uint32_t)(ddesc0 >> 32), w3_hi = (uint32_t)(w3desc0 >> 32);
-        const uint32_t a_step = (uint32_t)(kIssuersPerRole * 128 * 16) >> 4;
-        const uint32_t b_step = (uint32_t)(p.Coutp * kChunkRowBytes) >> 4;
-        const uint32_t a_lo0[2] = {(uint32_t)ddesc0 + ((uint32_t)(iw * 128 * 16) >> 4),
-                                   (uint32_t)ddesc0 + ((uint32_t)(d_bytes + iw * 128 * 16) >> 4)};
-        const uint32_t d_tmem0 = tmem_base + p.pcol0 + iw * p.Coutp;
+        const int my_tiles = (p.M2 - iw + kIssuersPerRole - 1) / kIssuersPerRole;
+        uint32_t a_lo[kMaxTiles], d_tm[kMaxTiles];
+#pragma unroll
+        for (int k = 0; k < kMaxTiles; ++k) {
+          const int t = iw + k * kIssuersPerRole;
+          a_lo[k] = (uint32_t)ddesc0 + ((uint32_t)(t * 128 * 16) >> 4);
+          d_tm[k] = tmem_base + p.pcol0 + t * p.Coutp;
+        }
+        const uint32_t b_step = (uint32_t)(p.Coutp * kChunkRowBytes) >> 4, buf_step = (uint32_t)d_bytes >> 4;
         uint32_t b_lo = (uint32_t)w3desc0;
         for (int c = 0; c < p.NC; ++c, b_lo += b_step) {
           const int b = c & 1;
           mbar_wait(bar_dready + b, (uint32_t)(c >> 1) & 1u, abort_flag, p.status, 0x106);
           tcgen05_fence_after_sync();
-          uint32_t a_lo = a_lo0[b], d_tmem = d_tmem0;
-          for (int t = iw; t < p.M2; t += kIssuersPerRole, a_lo += a_step, d_tmem += kIssuersPerRole * p.Coutp)
-            umma_bf16_lohi(d_tmem, a_lo, d_hi, b_lo, w3_hi, idesc_p, c > 0);
+          const uint32_t aoff = b ? buf_step : 0u;
+          const uint32_t acc = c > 0;
+#pragma unroll
+          for (int k = 0; k < kMaxTiles; ++k)
+            if (k < my_tiles) umma_bf16_lohi(d_tm[k], a_lo[k] + aoff, d_hi, b_lo, w3_hi, idesc_p, acc);
           umma_commit(bar_d + b);
         }
         umma_commit(bar_done);
