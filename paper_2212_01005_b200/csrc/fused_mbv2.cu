@@ -41,14 +41,12 @@ namespace {
 
 using namespace tc;
 
-constexpr int kComputeWarps = 28;                  // expand epilogue, depthwise, project epilogue
-constexpr int kComputeThreads = kComputeWarps * 32;
-constexpr int kGroupWarps = kComputeWarps / 2;     // two groups of compute warps on alternating chunks
+constexpr int kWarps = 32;                         // every warp computes; MMAs are issued inline by some of them
+constexpr int kThreads = kWarps * 32;
+constexpr int kGroupWarps = kWarps / 2;            // two groups of warps on alternating chunks
 constexpr int kGroupThreads = kGroupWarps * 32;
-constexpr int kTilesPerWarp = 3;                   // expand-epilogue tiles per warp: at most 8 tiles over >= 3 warps of a lane quarter
-constexpr int kIssuers = 4;                        // MMA-issuing warps (one per SM sub-partition)
-constexpr int kIssuersPerRole = kIssuers / 2;      // two for the expand GEMMs, two for the project GEMMs
-constexpr int kThreads = kComputeThreads + 32 * kIssuers;
+constexpr int kTilesPerWarp = 2;                   // expand-epilogue tiles per warp: at most 8 tiles over the 4 warps of a lane quarter
+constexpr int kExpandIssuers = 2;                  // the last two warps of a group issue its expand GEMMs
 constexpr int kChunk = 16;      // expanded channels per chunk = one MMA K step of the project GEMM
 constexpr int kChunkRowBytes = 32;
 
@@ -200,8 +198,7 @@ mbv2_fused_kernel(const Mbv2Params p) {
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + p.off_bar);
   uint64_t* bar_e = bars + 2;       // [2] expand accumulators of buffer b complete (MMA commit)
   uint64_t* bar_d = bars + 4;       // [2] project MMA has consumed D[b] (MMA commit)
-  uint64_t* bar_tfree = bars + 6;   // [2] expand buffer b drained and E chunk written (compute -> issuer)
-  uint64_t* bar_dready = bars + 8;  // [2] D[b] written (compute -> issuer)
+  uint64_t* bar_first = bars + 6;   // project GEMM of chunk 0 complete (it overwrites the output accumulators: group 1 issues after it)
   uint64_t* bar_done = bars + 10;   // every project MMA complete (the groups do not follow each other's bar_d phases)
   uint64_t* bar_stagger = bars + 11;   // group 0 has finished its first expand epilogue: group 1 starts (half a period behind)
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 12);
@@ -214,20 +211,19 @@ mbv2_fused_kernel(const Mbv2Params p) {
   const int gh0 = ho0 * p.stride - 1;   // image row of tile row 0
   const int d_bytes = 2 * p.d_plane;
 
-  if (tid == kComputeThreads) {
+  if (tid == kThreads - 1) {
     *abort_flag = 0u;
     for (int i = 0; i < 2; ++i) {
-      mbar_init(bar_e + i, kIssuersPerRole);
-      mbar_init(bar_d + i, kIssuersPerRole);
-      mbar_init(bar_tfree + i, 1);
-      mbar_init(bar_dready + i, 1);
+      mbar_init(bar_e + i, kExpandIssuers);
+      mbar_init(bar_d + i, (uint32_t)p.M2);
     }
-    mbar_init(bar_done, kIssuersPerRole);
+    mbar_init(bar_first, (uint32_t)p.M2);
+    mbar_init(bar_done, (uint32_t)(p.M2 * min(p.NC, 2)));
     mbar_init(bar_stagger, 1);
     fence_mbar_init();
     fence_proxy_async_smem();
   }
-  if (warp < kComputeWarps) {
+  {
     // ---- P1: stage the input strip, the weights and the biases. Every 16-byte chunk is one slot; a thread first
     // issues the loads of all its slots, then stores them, so that the whole prologue costs one round trip to
     // device memory. (Pixels are Cin * 2 bytes apart there: coalesced plain loads of the contiguous strip serve
@@ -275,7 +271,7 @@ mbv2_fused_kernel(const Mbv2Params p) {
     uint32_t dx[kBX], dw[kBW];
 #pragma unroll
     for (int k = 0; k < kBX; ++k) {
-      const uint32_t i = (uint32_t)(tid + k * kComputeThreads);
+      const uint32_t i = (uint32_t)(tid + k * kThreads);
       const uint8_t* src = nullptr;
       dx[k] = 0xffffffffu;
       if (i < nX) dx[k] = x_slot(i, src);
@@ -283,7 +279,7 @@ mbv2_fused_kernel(const Mbv2Params p) {
     }
 #pragma unroll
     for (int k = 0; k < kBW; ++k) {
-      const uint32_t i = (uint32_t)(tid + k * kComputeThreads);
+      const uint32_t i = (uint32_t)(tid + k * kThreads);
       const uint8_t* src = nullptr;
       dw[k] = 0xffffffffu;
       if (i < nW) dw[k] = w_slot(i, src);
@@ -300,18 +296,18 @@ mbv2_fused_kernel(const Mbv2Params p) {
     for (int k = 0; k < kBW; ++k)
       if (dw[k] != 0xffffffffu) *reinterpret_cast<uint4*>(smem + dw[k]) = vw[k];
     // shapes with more slots than the batched pass covers
-    for (uint32_t i = (uint32_t)(tid + kBX * kComputeThreads); i < nX; i += kComputeThreads) {
+    for (uint32_t i = (uint32_t)(tid + kBX * kThreads); i < nX; i += kThreads) {
       const uint8_t* src;
       const uint32_t d = x_slot(i, src);
       *reinterpret_cast<uint4*>(smem + d) = load_or_zero(src);
     }
-    for (uint32_t i = (uint32_t)(tid + kBW * kComputeThreads); i < nW; i += kComputeThreads) {
+    for (uint32_t i = (uint32_t)(tid + kBW * kThreads); i < nW; i += kThreads) {
       const uint8_t* src;
       const uint32_t d = w_slot(i, src);
       *reinterpret_cast<uint4*>(smem + d) = load_or_zero(src);
     }
     // the zero padding columns of the two E chunk buffers (written once: every chunk reuses them)
-    for (int i = tid; i < p.IH * 8; i += kComputeThreads) {
+    for (int i = tid; i < p.IH * 8; i += kThreads) {
       const int ih = i >> 3, side = (i >> 2) & 1, plane = i & 3;   // 2 buffers x 2 planes
       *reinterpret_cast<uint4*>(sE + plane * p.e_plane + (ih * p.IW + side * (p.IW - 1)) * 16) = make_uint4(0, 0, 0, 0);
     }
@@ -322,94 +318,22 @@ mbv2_fused_kernel(const Mbv2Params p) {
   tcgen05_fence_after_sync();
   const uint32_t tmem_base = *tmem_slot;
 
-  if (warp >= kComputeWarps) {
-    // ================= MMA issue warps (one lane each): two issue the expand GEMMs, two the project GEMMs, =================
-    // each pair splitting the M tiles between them. Separate roles keep an issuer from sitting in the wait for one
-    // event while the other kind is due: the project of chunk c has to be through before the depthwise stage of
-    // chunk c + 2 may overwrite its operand.
-    const int role = (warp - kComputeWarps) >> 1;     // 0: expand, 1: project
-    const int iw = (warp - kComputeWarps) & 1;
-    if (lane == 0) {
-      tcgen05_fence_after_sync();
-      // Descriptors as (low, high) words: start address and LBO live in the low word (shared-memory addresses >> 4
-      // stay below the 14-bit field limit), and every per-tile term is precomputed: an issuer shares its scheduler
-      // with seven busy compute warps and gets few issue slots, so the loops spend about four instructions per MMA.
-      constexpr int kMaxTiles = 4;   // M tiles per issuer (at most 8 tiles over two issuers)
-      if (role == 0) {
-        const uint32_t idesc_e = make_idesc_bf16(128, kChunk);
-        const uint32_t sbo_x = 8u * (uint32_t)p.row_bytes;
-        const uint64_t xdesc0 = make_smem_desc(smem_u32(sX), 0, sbo_x, p.swizzle);
-        const uint64_t w1desc0 = make_smem_desc(smem_u32(sW1), 0, sbo_x, p.swizzle);
-        const uint32_t x_hi = (uint32_t)(xdesc0 >> 32), w1_hi = (uint32_t)(w1desc0 >> 32);
-        const int ksteps = p.Kp / 16;
-        const int my_tiles = (p.M1 - iw + kIssuersPerRole - 1) / kIssuersPerRole;
-        uint32_t a_lo[kMaxTiles], d_off[kMaxTiles];
-#pragma unroll
-        for (int k = 0; k < kMaxTiles; ++k) {
-          const int t = iw + k * kIssuersPerRole;
-          a_lo[k] = (uint32_t)xdesc0 + ((uint32_t)(t * 128 * p.row_bytes) >> 4);
-          d_off[k] = tmem_base + p.ecol0 + t * kChunk;
-        }
-        const uint32_t b_step = (uint32_t)(kChunk * p.row_bytes) >> 4, buf_cols = (uint32_t)(p.M1 * kChunk);
-        uint32_t b_lo = (uint32_t)w1desc0;
-        for (int c = 0; c < p.NC; ++c, b_lo += b_step) {
-          const int b = c & 1;
-          if (c >= 2) {   // expand buffer b drained by the expand epilogue of chunk c - 2
-            mbar_wait(bar_tfree + b, (uint32_t)((c - 2) >> 1) & 1u, abort_flag, p.status, 0x105);
-            tcgen05_fence_after_sync();
-          }
-          const uint32_t dcol = b ? buf_cols : 0u;
-#pragma unroll
-          for (int k = 0; k < kMaxTiles; ++k) {
-            if (k < my_tiles) {
-#pragma unroll
-              for (int ks = 0; ks < 4; ++ks)
-                if (ks < ksteps) umma_bf16_lohi(d_off[k] + dcol, a_lo[k] + 2u * ks, x_hi, b_lo + 2u * ks, w1_hi, idesc_e, ks > 0);
-            }
-          }
-          umma_commit(bar_e + b);
-        }
-      } else {
-        const uint32_t idesc_p = make_idesc_bf16(128, (uint32_t)p.Coutp);
-        // D: un-swizzled K-major; the two 8-channel planes are the two K core-matrix columns
-        const uint64_t ddesc0 = make_smem_desc(smem_u32(sD), (uint32_t)p.d_plane, 128, SW_NONE);
-        const uint64_t w3desc0 = make_smem_desc(smem_u32(sW3), 0, 256, SW_32B);
-        const uint32_t d_hi = (uint32_t)(ddesc0 >> 32), w3_hi = (uint32_t)(w3desc0 >> 32);
-        const int my_tiles = (p.M2 - iw + kIssuersPerRole - 1) / kIssuersPerRole;
-        uint32_t a_lo[kMaxTiles], d_tm[kMaxTiles];
-#pragma unroll
-        for (int k = 0; k < kMaxTiles; ++k) {
-          const int t = iw + k * kIssuersPerRole;
-          a_lo[k] = (uint32_t)ddesc0 + ((uint32_t)(t * 128 * 16) >> 4);
-          d_tm[k] = tmem_base + p.pcol0 + t * p.Coutp;
-        }
-        const uint32_t b_step = (uint32_t)(p.Coutp * kChunkRowBytes) >> 4, buf_step = (uint32_t)d_bytes >> 4;
-        uint32_t b_lo = (uint32_t)w3desc0;
-        for (int c = 0; c < p.NC; ++c, b_lo += b_step) {
-          const int b = c & 1;
-          mbar_wait(bar_dready + b, (uint32_t)(c >> 1) & 1u, abort_flag, p.status, 0x106);
-          tcgen05_fence_after_sync();
-          const uint32_t aoff = b ? buf_step : 0u;
-          const uint32_t acc = c > 0;
-#pragma unroll
-          for (int k = 0; k < kMaxTiles; ++k)
-            if (k < my_tiles) umma_bf16_lohi(d_tm[k], a_lo[k] + aoff, d_hi, b_lo, w3_hi, idesc_p, acc);
-          umma_commit(bar_d + b);
-        }
-        umma_commit(bar_done);
-      }
-    }
-    __syncwarp();
-  } else {
-    // ================================== compute warps ==================================
-    // The compute warps form two groups of 14; group g owns the chunks c = g, g + 2, ... (expand buffer, E buffer and
-    // D buffer g). A group alternates expand epilogue and depthwise stage with a group-wide barrier after each; the
-    // two groups are out of phase, so one group's barrier and tensor-memory latencies hide behind the other's arithmetic.
+  {
+    // The warps form two groups of 16; group g owns the chunks c = g, g + 2, ... (expand buffer, E buffer and D
+    // buffer g). A group alternates expand epilogue and depthwise stage with a group-wide barrier after each; the two
+    // groups are out of phase, so one group's barrier and tensor-memory latencies hide behind the other's arithmetic.
+    // MMAs are issued inline, right after the barrier that makes their operands ready: the expand GEMM of chunk c + 2
+    // by the group's last two warps (at 56 x 56 they have no depthwise item), the project GEMM of chunk c by M2 warps,
+    // one tile each -- a parked issuer warp would share its scheduler with busy warps and issue an MMA every few
+    // hundred cycles, and the project GEMM is urgent: it must be through before the depthwise stage of chunk c + 2
+    // may overwrite its operand.
     const int g = warp / kGroupWarps;
     const int gwarp0 = g * kGroupWarps;           // first warp of the group
     const int gt = tid - gwarp0 * 32;             // thread index in the group
     const uint32_t gbar = 1u + (uint32_t)g;       // named barrier of the group
     const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
+    const int gw = warp - gwarp0;                 // warp index in the group
+    const int xi = gw - (kGroupWarps - kExpandIssuers);   // >= 0: this warp issues expand tiles xi, xi + 2, ...
     // Depthwise work split: thread = (channel pair, slot). Stride 1: an item is a block of 2 output rows x 7 output
     // columns (56 columns x 14 rows x 8 pairs = one item per thread of a group). Stride 2: an item is one output column
     // of one row group.
@@ -447,6 +371,40 @@ mbv2_fused_kernel(const Mbv2Params p) {
       }
     }
 
+    // Descriptors as (low, high) words: start address and LBO live in the low word, so an operand advances with one
+    // 32-bit add (shared-memory addresses >> 4 stay below the 14-bit field limit).
+    const uint32_t sbo_x = 8u * (uint32_t)p.row_bytes;
+    const uint64_t xdesc0 = make_smem_desc(smem_u32(sX), 0, sbo_x, p.swizzle);
+    const uint64_t w1desc0 = make_smem_desc(smem_u32(sW1), 0, sbo_x, p.swizzle);
+    // D: un-swizzled K-major; the two 8-channel planes are the two K core-matrix columns
+    const uint64_t ddesc0 = make_smem_desc(smem_u32(sD), (uint32_t)p.d_plane, 128, SW_NONE);
+    const uint64_t w3desc0 = make_smem_desc(smem_u32(sW3), 0, 256, SW_32B);
+    auto issue_expand = [&](int c) {   // one lane of an expand-issuing warp: tiles xi, xi + 2, ... of chunk c -> buffer g
+      const uint32_t idesc_e = make_idesc_bf16(128, kChunk);
+      const uint32_t x_hi = (uint32_t)(xdesc0 >> 32), w1_hi = (uint32_t)(w1desc0 >> 32);
+      const uint32_t b_lo = (uint32_t)w1desc0 + ((uint32_t)(c * kChunk * p.row_bytes) >> 4);
+      const uint32_t a_step = (uint32_t)(kExpandIssuers * 128 * p.row_bytes) >> 4;
+      uint32_t a_lo = (uint32_t)xdesc0 + ((uint32_t)(xi * 128 * p.row_bytes) >> 4);
+      uint32_t d_tmem = tmem_base + p.ecol0 + (g * p.M1 + xi) * kChunk;
+      const int ksteps = p.Kp / 16;
+      for (int t = xi; t < p.M1; t += kExpandIssuers, a_lo += a_step, d_tmem += kExpandIssuers * kChunk) {
+#pragma unroll
+        for (int ks = 0; ks < 4; ++ks)
+          if (ks < ksteps) umma_bf16_lohi(d_tmem, a_lo + 2u * ks, x_hi, b_lo + 2u * ks, w1_hi, idesc_e, ks > 0);
+      }
+      umma_commit(bar_e + g);
+    };
+    auto issue_project = [&](int c) {   // one lane of warp gw < M2: tile gw of chunk c
+      const uint32_t idesc_p = make_idesc_bf16(128, (uint32_t)p.Coutp);
+      const uint32_t a_lo = (uint32_t)ddesc0 + ((uint32_t)(g * d_bytes + gw * 128 * 16) >> 4);
+      const uint32_t b_lo = (uint32_t)w3desc0 + ((uint32_t)(c * p.Coutp * kChunkRowBytes) >> 4);
+      umma_bf16_lohi(tmem_base + p.pcol0 + gw * p.Coutp, a_lo, (uint32_t)(ddesc0 >> 32), b_lo, (uint32_t)(w3desc0 >> 32), idesc_p,
+                     c > 0);
+      umma_commit(bar_d + g);
+      if (c == 0) umma_commit(bar_first);
+    };
+    if (xi >= 0 && lane == 0 && g < p.NC) issue_expand(g);
+    __syncwarp();
     // Keep the groups out of phase: group 1 starts once group 0 is through its first expand epilogue.
     if (g == 1) mbar_wait(bar_stagger, 0, abort_flag, p.status, 0x107);
     for (int c = g, it = 0; c < p.NC; c += 2, ++it) {
@@ -481,9 +439,13 @@ mbv2_fused_kernel(const Mbv2Params p) {
       }
       tcgen05_fence_before_sync();
       named_barrier_sync(gbar, kGroupThreads);
-      if (gt == 0) {
-        mbar_arrive(bar_tfree + g);
-        if (c == 0) mbar_arrive(bar_stagger);
+      if (gt == 0 && c == 0) mbar_arrive(bar_stagger);
+      if (xi >= 0 && c + 2 < p.NC) {   // expand buffer g is drained: the expand GEMM of the group's next chunk
+        if (lane == 0) {
+          tcgen05_fence_after_sync();
+          issue_expand(c + 2);
+        }
+        __syncwarp();
       }
 
       // D[g] was read by the project MMA of chunk c-2
@@ -514,7 +476,16 @@ mbv2_fused_kernel(const Mbv2Params p) {
       }
       fence_proxy_async_smem();
       named_barrier_sync(gbar, kGroupThreads);
-      if (gt == 0) mbar_arrive(bar_dready + g);
+      if (gw < p.M2) {   // D[g] is complete: the project GEMM of chunk c, one tile per warp
+        if (lane == 0) {
+          // chunk 0 overwrites the accumulators: everything else is issued after it
+          if (c == 1) mbar_wait(bar_first, 0, abort_flag, p.status, 0x106);
+          tcgen05_fence_after_sync();
+          issue_project(c);
+          if (c + 2 >= p.NC) umma_commit(bar_done);
+        }
+        __syncwarp();
+      }
     }
 
     // ---- P6: project epilogue: + b3 (+ residual), bf16, 16-byte stores ----
@@ -523,7 +494,7 @@ mbv2_fused_kernel(const Mbv2Params p) {
       tcgen05_fence_after_sync();
       const int valid_pix = rows_valid * p.Wo;
       const size_t gpix0 = ((size_t)n * p.Ho + ho0) * p.Wo;
-      for (int t = warp >> 2; t < p.M2; t += kComputeWarps / 4) {
+      for (int t = warp >> 2; t < p.M2; t += kWarps / 4) {
         const int po = t * 128 + (warp & 3) * 32 + lane;
         for (int j0 = 0; j0 < p.Coutp; j0 += 16) {
           uint32_t acc[16];
