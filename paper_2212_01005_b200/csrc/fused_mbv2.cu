@@ -200,7 +200,6 @@ mbv2_fused_kernel(const Mbv2Params p) {
   uint64_t* bar_d = bars + 4;       // [2] project MMA has consumed D[b] (MMA commit)
   uint64_t* bar_first = bars + 6;   // project GEMM of chunk 0 complete (it overwrites the output accumulators: group 1 issues after it)
   uint64_t* bar_done = bars + 10;   // every project MMA complete (the groups do not follow each other's bar_d phases)
-  uint64_t* bar_stagger = bars + 11;   // group 0 has finished its first expand epilogue: group 1 starts (half a period behind)
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 12);
   volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(bars + 13);
 
@@ -219,7 +218,6 @@ mbv2_fused_kernel(const Mbv2Params p) {
     }
     mbar_init(bar_first, (uint32_t)p.M2);
     mbar_init(bar_done, (uint32_t)(p.M2 * min(p.NC, 2)));
-    mbar_init(bar_stagger, 1);
     fence_mbar_init();
     fence_proxy_async_smem();
   }
@@ -379,37 +377,47 @@ mbv2_fused_kernel(const Mbv2Params p) {
     // D: un-swizzled K-major; the two 8-channel planes are the two K core-matrix columns
     const uint64_t ddesc0 = make_smem_desc(smem_u32(sD), (uint32_t)p.d_plane, 128, SW_NONE);
     const uint64_t w3desc0 = make_smem_desc(smem_u32(sW3), 0, 256, SW_32B);
-    auto issue_expand = [&](int c) {   // one lane of an expand-issuing warp: tiles xi, xi + 2, ... of chunk c -> buffer g
-      const uint32_t idesc_e = make_idesc_bf16(128, kChunk);
-      const uint32_t x_hi = (uint32_t)(xdesc0 >> 32), w1_hi = (uint32_t)(w1desc0 >> 32);
-      const uint32_t b_lo = (uint32_t)w1desc0 + ((uint32_t)(c * kChunk * p.row_bytes) >> 4);
-      const uint32_t a_step = (uint32_t)(kExpandIssuers * 128 * p.row_bytes) >> 4;
-      uint32_t a_lo = (uint32_t)xdesc0 + ((uint32_t)(xi * 128 * p.row_bytes) >> 4);
-      uint32_t d_tmem = tmem_base + p.ecol0 + (g * p.M1 + xi) * kChunk;
-      const int ksteps = p.Kp / 16;
-      for (int t = xi; t < p.M1; t += kExpandIssuers, a_lo += a_step, d_tmem += kExpandIssuers * kChunk) {
+    // Expand issue state of the group's last two warps: tiles xi, xi + 2, ... of the group's chunks -> buffer g.
+    const uint32_t idesc_e = make_idesc_bf16(128, kChunk);
+    const uint32_t x_hi = (uint32_t)(xdesc0 >> 32), w1_hi = (uint32_t)(w1desc0 >> 32);
+    const uint32_t exp_a_step = (uint32_t)(kExpandIssuers * 128 * p.row_bytes) >> 4;
+    const uint32_t exp_a_lo0 = (uint32_t)xdesc0 + ((uint32_t)(max(xi, 0) * 128 * p.row_bytes) >> 4);
+    const uint32_t exp_d_tmem0 = tmem_base + p.ecol0 + (g * p.M1 + max(xi, 0)) * kChunk;
+    const uint32_t exp_b_step = (uint32_t)(2 * kChunk * p.row_bytes) >> 4;   // the group's next chunk is c + 2
+    uint32_t exp_b_lo = (uint32_t)w1desc0 + ((uint32_t)(g * kChunk * p.row_bytes) >> 4);
+    const int ksteps = p.Kp / 16;
+    auto issue_expand = [&]() {   // one lane; advances to the group's next chunk
+      uint32_t a_lo = exp_a_lo0, d_tmem = exp_d_tmem0;
+      for (int t = xi; t < p.M1; t += kExpandIssuers, a_lo += exp_a_step, d_tmem += kExpandIssuers * kChunk) {
 #pragma unroll
         for (int ks = 0; ks < 4; ++ks)
-          if (ks < ksteps) umma_bf16_lohi(d_tmem, a_lo + 2u * ks, x_hi, b_lo + 2u * ks, w1_hi, idesc_e, ks > 0);
+          if (ks < ksteps) umma_bf16_lohi(d_tmem, a_lo + 2u * ks, x_hi, exp_b_lo + 2u * ks, w1_hi, idesc_e, ks > 0);
       }
       umma_commit(bar_e + g);
+      exp_b_lo += exp_b_step;
     };
-    auto issue_project = [&](int c) {   // one lane of warp gw < M2: tile gw of chunk c
-      const uint32_t idesc_p = make_idesc_bf16(128, (uint32_t)p.Coutp);
-      const uint32_t a_lo = (uint32_t)ddesc0 + ((uint32_t)(g * d_bytes + gw * 128 * 16) >> 4);
-      const uint32_t b_lo = (uint32_t)w3desc0 + ((uint32_t)(c * p.Coutp * kChunkRowBytes) >> 4);
-      umma_bf16_lohi(tmem_base + p.pcol0 + gw * p.Coutp, a_lo, (uint32_t)(ddesc0 >> 32), b_lo, (uint32_t)(w3desc0 >> 32), idesc_p,
-                     c > 0);
-      umma_commit(bar_d + g);
-      if (c == 0) umma_commit(bar_first);
-    };
-    if (xi >= 0 && lane == 0 && g < p.NC) issue_expand(g);
+    // Project issue state of warp gw < M2 (tile gw), kept in three registers: a warp that runs a serial instruction
+    // chain next to warps with dense arithmetic gets an issue slot only every few tens of cycles, so the path from
+    // the barrier to the MMA is one add, the MMA and the commit.
+    constexpr uint32_t kDescVersion = 1u << 14;   // high descriptor word: SBO >> 4, version 1 at bit 46, layout at bits 61..63
+    constexpr uint32_t d_hi = (128u >> 4) | kDescVersion | ((uint32_t)SW_NONE << 29);
+    constexpr uint32_t w3_hi = (256u >> 4) | kDescVersion | ((uint32_t)SW_32B << 29);
+    const uint32_t idesc_p = make_idesc_bf16(128, (uint32_t)p.Coutp);
+    const uint32_t proj_a_lo = (uint32_t)ddesc0 + ((uint32_t)(g * d_bytes + gw * 128 * 16) >> 4);
+    const uint32_t proj_d_tmem = tmem_base + p.pcol0 + gw * p.Coutp;
+    const uint32_t proj_b_step = (uint32_t)(2 * p.Coutp * kChunkRowBytes) >> 4;     // the group's next chunk is c + 2
+    uint32_t proj_b_lo = (uint32_t)w3desc0 + ((uint32_t)(g * p.Coutp * kChunkRowBytes) >> 4);
+    if (xi >= 0 && lane == 0 && g < p.NC) issue_expand();
     __syncwarp();
-    // Keep the groups out of phase: group 1 starts once group 0 is through its first expand epilogue.
-    if (g == 1) mbar_wait(bar_stagger, 0, abort_flag, p.status, 0x107);
+    // Waits on MMA completion are taken by ONE warp of the group, just before it arrives at the group barrier that
+    // the others are parked at: a polling warp spends issue slots, sixteen of them a large share of the SM's.
+    const bool waiter = gw == kGroupWarps - 1;
+    if (g < p.NC) {
+      if (waiter) mbar_wait(bar_e + g, 0, abort_flag, p.status, 0x102);   // the group's first expand GEMM
+      named_barrier_sync(gbar, kGroupThreads);
+    }
     for (int c = g, it = 0; c < p.NC; c += 2, ++it) {
       // ---- P3: expand epilogue of chunk c -> E[g]: + b1, ReLU6, zero outside the image, bf16 ----
-      mbar_wait(bar_e + g, (uint32_t)it & 1u, abort_flag, p.status, 0x102);
       tcgen05_fence_after_sync();
       uint8_t* e_buf = sE + g * e_bytes;
 #pragma unroll
@@ -438,18 +446,16 @@ mbv2_fused_kernel(const Mbv2Params p) {
         }
       }
       tcgen05_fence_before_sync();
+      // D[g] was read by the project GEMM of chunk c - 2
+      if (waiter && it >= 1) mbar_wait(bar_d + g, (uint32_t)(it - 1) & 1u, abort_flag, p.status, 0x103);
       named_barrier_sync(gbar, kGroupThreads);
-      if (gt == 0 && c == 0) mbar_arrive(bar_stagger);
       if (xi >= 0 && c + 2 < p.NC) {   // expand buffer g is drained: the expand GEMM of the group's next chunk
         if (lane == 0) {
           tcgen05_fence_after_sync();
-          issue_expand(c + 2);
+          issue_expand();
         }
         __syncwarp();
       }
-
-      // D[g] was read by the project MMA of chunk c-2
-      if (it >= 1) mbar_wait(bar_d + g, (uint32_t)(it - 1) & 1u, abort_flag, p.status, 0x103);
 
       // ---- P4: depthwise 3x3 + bias + ReLU6 on CUDA cores: E[g] -> D[g] (A operand of the project GEMM) ----
       {
@@ -475,22 +481,28 @@ mbv2_fused_kernel(const Mbv2Params p) {
         }
       }
       fence_proxy_async_smem();
+      // the expand GEMM of the group's next chunk (issued after the previous barrier) is complete
+      if (waiter && c + 2 < p.NC) mbar_wait(bar_e + g, (uint32_t)(it + 1) & 1u, abort_flag, p.status, 0x102);
       named_barrier_sync(gbar, kGroupThreads);
       if (gw < p.M2) {   // D[g] is complete: the project GEMM of chunk c, one tile per warp
         if (lane == 0) {
           // chunk 0 overwrites the accumulators: everything else is issued after it
           if (c == 1) mbar_wait(bar_first, 0, abort_flag, p.status, 0x106);
           tcgen05_fence_after_sync();
-          issue_project(c);
+          umma_bf16_lohi(proj_d_tmem, proj_a_lo, d_hi, proj_b_lo, w3_hi, idesc_p, c > 0);
+          umma_commit(bar_d + g);
+          if (c == 0) umma_commit(bar_first);
           if (c + 2 >= p.NC) umma_commit(bar_done);
         }
         __syncwarp();
       }
+      proj_b_lo += proj_b_step;
     }
 
     // ---- P6: project epilogue: + b3 (+ residual), bf16, 16-byte stores ----
     {
-      mbar_wait(bar_done, 0, abort_flag, p.status, 0x104);
+      if (warp == kWarps - 1) mbar_wait(bar_done, 0, abort_flag, p.status, 0x104);
+      __syncthreads();
       tcgen05_fence_after_sync();
       const int valid_pix = rows_valid * p.Wo;
       const size_t gpix0 = ((size_t)n * p.Ho + ho0) * p.Wo;
