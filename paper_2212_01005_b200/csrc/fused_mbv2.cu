@@ -221,7 +221,6 @@ mbv2_fused_kernel(const Mbv2Params p) {
     fence_mbar_init();
     fence_proxy_async_smem();
   }
-  {
     // ---- P1: stage the input strip, the weights and the biases. Every 16-byte chunk is one slot; a thread first
     // issues the loads of all its slots, then stores them, so that the whole prologue costs one round trip to
     // device memory. (Pixels are Cin * 2 bytes apart there: coalesced plain loads of the contiguous strip serve
@@ -283,48 +282,7 @@ mbv2_fused_kernel(const Mbv2Params p) {
       if (i < nW) dw[k] = w_slot(i, src);
       vw[k] = load_or_zero(src);
     }
-    if (warp == 0) {
-      tmem_alloc(tmem_slot, (uint32_t)p.tmem_cols);
-      tmem_relinquish();
-    }
-#pragma unroll
-    for (int k = 0; k < kBX; ++k)
-      if (dx[k] != 0xffffffffu) *reinterpret_cast<uint4*>(smem + dx[k]) = vx[k];
-#pragma unroll
-    for (int k = 0; k < kBW; ++k)
-      if (dw[k] != 0xffffffffu) *reinterpret_cast<uint4*>(smem + dw[k]) = vw[k];
-    // shapes with more slots than the batched pass covers
-    for (uint32_t i = (uint32_t)(tid + kBX * kThreads); i < nX; i += kThreads) {
-      const uint8_t* src;
-      const uint32_t d = x_slot(i, src);
-      *reinterpret_cast<uint4*>(smem + d) = load_or_zero(src);
-    }
-    for (uint32_t i = (uint32_t)(tid + kBW * kThreads); i < nW; i += kThreads) {
-      const uint8_t* src;
-      const uint32_t d = w_slot(i, src);
-      *reinterpret_cast<uint4*>(smem + d) = load_or_zero(src);
-    }
-    // the zero padding columns of the two E chunk buffers (written once: every chunk reuses them)
-    for (int i = tid; i < p.IH * 8; i += kThreads) {
-      const int ih = i >> 3, side = (i >> 2) & 1, plane = i & 3;   // 2 buffers x 2 planes
-      *reinterpret_cast<uint4*>(sE + plane * p.e_plane + (ih * p.IW + side * (p.IW - 1)) * 16) = make_uint4(0, 0, 0, 0);
-    }
-    fence_proxy_async_smem();
-  }
-  tcgen05_fence_before_sync();
-  __syncthreads();
-  tcgen05_fence_after_sync();
-  const uint32_t tmem_base = *tmem_slot;
-
-  {
-    // The warps form two groups of 16; group g owns the chunks c = g, g + 2, ... (expand buffer, E buffer and D
-    // buffer g). A group alternates expand epilogue and depthwise stage with a group-wide barrier after each; the two
-    // groups are out of phase, so one group's barrier and tensor-memory latencies hide behind the other's arithmetic.
-    // MMAs are issued inline, right after the barrier that makes their operands ready: the expand GEMM of chunk c + 2
-    // by the group's last two warps (at 56 x 56 they have no depthwise item), the project GEMM of chunk c by M2 warps,
-    // one tile each -- a parked issuer warp would share its scheduler with busy warps and issue an MMA every few
-    // hundred cycles, and the project GEMM is urgent: it must be through before the depthwise stage of chunk c + 2
-    // may overwrite its operand.
+    // ---- per-thread work mapping, computed while the loads are in flight ----
     const int g = warp / kGroupWarps;
     const int gwarp0 = g * kGroupWarps;           // first warp of the group
     const int gt = tid - gwarp0 * 32;             // thread index in the group
@@ -369,6 +327,46 @@ mbv2_fused_kernel(const Mbv2Params p) {
       }
     }
 
+    if (warp == 0) {
+      tmem_alloc(tmem_slot, (uint32_t)p.tmem_cols);
+      tmem_relinquish();
+    }
+#pragma unroll
+    for (int k = 0; k < kBX; ++k)
+      if (dx[k] != 0xffffffffu) *reinterpret_cast<uint4*>(smem + dx[k]) = vx[k];
+#pragma unroll
+    for (int k = 0; k < kBW; ++k)
+      if (dw[k] != 0xffffffffu) *reinterpret_cast<uint4*>(smem + dw[k]) = vw[k];
+    // shapes with more slots than the batched pass covers
+    for (uint32_t i = (uint32_t)(tid + kBX * kThreads); i < nX; i += kThreads) {
+      const uint8_t* src;
+      const uint32_t d = x_slot(i, src);
+      *reinterpret_cast<uint4*>(smem + d) = load_or_zero(src);
+    }
+    for (uint32_t i = (uint32_t)(tid + kBW * kThreads); i < nW; i += kThreads) {
+      const uint8_t* src;
+      const uint32_t d = w_slot(i, src);
+      *reinterpret_cast<uint4*>(smem + d) = load_or_zero(src);
+    }
+    // the zero padding columns of the two E chunk buffers (written once: every chunk reuses them)
+    for (int i = tid; i < p.IH * 8; i += kThreads) {
+      const int ih = i >> 3, side = (i >> 2) & 1, plane = i & 3;   // 2 buffers x 2 planes
+      *reinterpret_cast<uint4*>(sE + plane * p.e_plane + (ih * p.IW + side * (p.IW - 1)) * 16) = make_uint4(0, 0, 0, 0);
+    }
+    fence_proxy_async_smem();
+  tcgen05_fence_before_sync();
+  __syncthreads();
+  tcgen05_fence_after_sync();
+  const uint32_t tmem_base = *tmem_slot;
+
+    // The warps form two groups of 16; group g owns the chunks c = g, g + 2, ... (expand buffer, E buffer and D
+    // buffer g). A group alternates expand epilogue and depthwise stage with a group-wide barrier after each; the two
+    // groups are out of phase, so one group's barrier and tensor-memory latencies hide behind the other's arithmetic.
+    // MMAs are issued inline, right after the barrier that makes their operands ready: the expand GEMM of chunk c + 2
+    // by the group's last two warps (at 56 x 56 they have no depthwise item), the project GEMM of chunk c by M2 warps,
+    // one tile each -- a parked issuer warp would share its scheduler with busy warps and issue an MMA every few
+    // hundred cycles, and the project GEMM is urgent: it must be through before the depthwise stage of chunk c + 2
+    // may overwrite its operand.
     // Descriptors as (low, high) words: start address and LBO live in the low word, so an operand advances with one
     // 32-bit add (shared-memory addresses >> 4 stay below the 14-bit field limit).
     const uint32_t sbo_x = 8u * (uint32_t)p.row_bytes;
@@ -535,7 +533,6 @@ mbv2_fused_kernel(const Mbv2Params p) {
         }
       }
     }
-  }
   tcgen05_fence_before_sync();
   __syncthreads();
   if (warp == 0) tmem_dealloc(tmem_base, (uint32_t)p.tmem_cols);
