@@ -40,7 +40,8 @@ using namespace tc;
 
 constexpr int kEpiWarps = 8;                 // two per TMEM lane quarter: each takes half of the channels
 constexpr int kEpiThreads = kEpiWarps * 32;
-constexpr int kThreads = kEpiThreads + 64;   // + TMA warp + MMA warp
+constexpr int kMmaWarps = 2;                 // one issuing lane each, alternating M tiles: a single thread issues an MMA every ~70 cycles, the tensor pipe takes one every ~50
+constexpr int kThreads = kEpiThreads + 32 + 32 * kMmaWarps;   // + TMA warp + MMA warps
 constexpr int kMaxWStages = 4;     // ring stages; each holds one filter row = 3 taps
 
 struct ConvParams {
@@ -85,8 +86,8 @@ conv3x3_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
   if (tid == kEpiThreads) {
     *abort_flag = 0u;
     mbar_init(bar_x, 1);
-    for (int i = 0; i < kMaxWStages; ++i) { mbar_init(bar_full + i, 1); mbar_init(bar_empty + i, 1); }
-    for (int i = 0; i < 6; ++i) mbar_init(bar_acc1 + i, 1);
+    for (int i = 0; i < kMaxWStages; ++i) { mbar_init(bar_full + i, 1); mbar_init(bar_empty + i, kMmaWarps); }
+    for (int i = 0; i < 6; ++i) mbar_init(bar_acc1 + i, (i == 2 || i == 3) ? 1 : kMmaWarps);   // bar_y is arrived by one epilogue thread
     fence_mbar_init();
     fence_proxy_async_smem();
     tma_prefetch_desc(&tmap_x);
@@ -124,8 +125,9 @@ conv3x3_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
       }
     }
     __syncwarp();
-  } else if (warp == kEpiWarps + 1) {
-    // ================================ MMA issuer ================================
+  } else if (warp > kEpiWarps) {
+    // ================================ MMA issuers ================================
+    const int iw = warp - kEpiWarps - 1;   // issuer iw takes tiles lo + iw, lo + iw + kMmaWarps, ...
     if (lane == 0) {
       const uint32_t idesc = make_idesc_bf16(128, (uint32_t)p.C);
       const uint64_t wdesc0 = make_smem_desc(smem_u32(sW), 0, 8u * p.w_row_bytes, p.w_swizzle);
@@ -153,18 +155,18 @@ conv3x3_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
           const uint64_t bdesc = wdesc0 + (uint64_t)((uint32_t)((s * 3 + tap % 3) * p.w_stage_bytes) >> 4);
           // all per-MMA arithmetic is 32-bit adds on the descriptors' low words
           const uint32_t a_hi = (uint32_t)(adesc0 >> 32), b_hi = (uint32_t)(bdesc >> 32), b_lo = (uint32_t)bdesc;
-          uint32_t a_lo = (uint32_t)adesc0 + (uint32_t)(lo * 128 + shift) * rowu;
-          uint32_t d_tmem = tmem_base + lo * p.C;
+          uint32_t a_lo = (uint32_t)adesc0 + (uint32_t)((lo + iw) * 128 + shift) * rowu;
+          uint32_t d_tmem = tmem_base + (lo + iw) * p.C;
           const uint32_t acc0 = tap != 0;
           if (ksteps == 4) {
-            for (int mt = lo; mt < hi; ++mt, a_lo += 128 * rowu, d_tmem += p.C) {
+            for (int mt = lo + iw; mt < hi; mt += kMmaWarps, a_lo += kMmaWarps * 128 * rowu, d_tmem += kMmaWarps * p.C) {
               umma_bf16_lohi(d_tmem, a_lo, a_hi, b_lo, b_hi, idesc, acc0);
               umma_bf16_lohi(d_tmem, a_lo + a_kstep, a_hi, b_lo + 2, b_hi, idesc, 1);
               umma_bf16_lohi(d_tmem, a_lo + 2 * a_kstep, a_hi, b_lo + 4, b_hi, idesc, 1);
               umma_bf16_lohi(d_tmem, a_lo + 3 * a_kstep, a_hi, b_lo + 6, b_hi, idesc, 1);
             }
           } else {
-            for (int mt = lo; mt < hi; ++mt, a_lo += 128 * rowu, d_tmem += p.C)
+            for (int mt = lo + iw; mt < hi; mt += kMmaWarps, a_lo += kMmaWarps * 128 * rowu, d_tmem += kMmaWarps * p.C)
               for (int ks = 0; ks < ksteps; ++ks)
                 umma_bf16_lohi(d_tmem, a_lo + ks * a_kstep, a_hi, b_lo + 2 * ks, b_hi, idesc, ks ? 1u : acc0);
           }
