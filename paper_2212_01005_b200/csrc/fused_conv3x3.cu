@@ -40,7 +40,7 @@ using namespace tc;
 
 constexpr int kEpiWarps = 8;                 // two per TMEM lane quarter: each takes half of the channels
 constexpr int kEpiThreads = kEpiWarps * 32;
-constexpr int kMmaWarps = 2;                 // one issuing lane each, alternating M tiles: a single thread issues an MMA every ~70 cycles, the tensor pipe takes one every ~50
+constexpr int kMmaWarps = 4;                 // one issuing lane each, alternating M tiles: a single thread issues an MMA every ~70 cycles, the tensor pipe takes one every ~50
 constexpr int kThreads = kEpiThreads + 32 + 32 * kMmaWarps;   // + TMA warp + MMA warps
 constexpr int kMaxWStages = 4;     // ring stages; each holds one filter row = 3 taps
 
@@ -53,6 +53,7 @@ struct ConvParams {
   int N, H, W, C;          // C = input = middle = output channels
   int R, strips, IH, Wp, P1, M1, P2, M2;
   int a1, a2;              // tiles [0,a1) of conv1 / [0,a2) of conv2 form the first pipeline group
+  int stage_ok;            // the first 16 KB of the input rows are free for output staging whenever an output epilogue runs
   int w_row_bytes, w_swizzle, w_stage_bytes;
   int wstages;             // ring stages in use (2..kMaxWStages)
   int off_x, off_y, off_w, off_bias, off_bar;
@@ -223,8 +224,17 @@ conv3x3_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
       if (tid == 0) mbar_arrive(bar_y + grp);
     }
 
-    // P6: out = ReLU(acc + b2 + x); the residual is fetched before waiting for the accumulators
+    // P6: out = ReLU(acc + b2 + x); the residual is fetched before waiting for the accumulators. A thread owns one
+    // pixel row of a tile, and pixels are C * 2 bytes apart in device memory: stored straight from the registers, a
+    // warp's 16-byte stores would hit 32 different lines each. Instead the warp transposes its [32 pixels x ncol]
+    // block through a private 2 KB staging area (the start of the input rows, no longer read by then), so that
+    // consecutive lanes store consecutive 16-byte chunks of a pixel.
     const float* sB2 = sBias + p.C;
+    const bool stage = p.stage_ok != 0;
+    const uint32_t stg = smem_u32(sX) + (uint32_t)warp * 2048u;
+    const int chl = ncol == 32 ? 2 : 1;                  // log2(16-byte chunks per staged row)
+    const uint32_t rb = (uint32_t)ncol * 2u;             // bytes per staged row
+    const uint32_t swz_w = ((uint32_t)lane >> (3 - chl)) & ((1u << chl) - 1u);   // chunk XOR of this lane's row
     for (int grp = 0; grp < 2; ++grp) {
       for (int mt = pass_lo[2 + grp]; mt < pass_hi[2 + grp] || mt == pass_lo[2 + grp]; ++mt) {
         const bool tile_ok = mt < pass_hi[2 + grp];
@@ -257,9 +267,32 @@ conv3x3_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
                 const float y1 = fmaxf(__uint_as_float(v[2 * j + 1]) + sB2[c0 + 2 * j + 1] + bf16_hi(xs[j]), 0.0f);
                 w[j] = pack_bf16x2(y0, y1);
               }
-              *reinterpret_cast<uint4*>(p.out + pix * p.C + c0) = make_uint4(w[0], w[1], w[2], w[3]);
-              *reinterpret_cast<uint4*>(p.out + pix * p.C + c0 + 8) = make_uint4(w[4], w[5], w[6], w[7]);
+              if (stage) {
+                const uint32_t k0 = (uint32_t)(c0 - col0) >> 3;
+                const uint32_t a0 = stg + (uint32_t)lane * rb + ((k0 ^ swz_w) << 4), a1 = stg + (uint32_t)lane * rb + (((k0 + 1u) ^ swz_w) << 4);
+                asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(a0), "r"(w[0]), "r"(w[1]), "r"(w[2]), "r"(w[3]) : "memory");
+                asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(a1), "r"(w[4]), "r"(w[5]), "r"(w[6]), "r"(w[7]) : "memory");
+              } else {
+                *reinterpret_cast<uint4*>(p.out + pix * p.C + c0) = make_uint4(w[0], w[1], w[2], w[3]);
+                *reinterpret_cast<uint4*>(p.out + pix * p.C + c0 + 8) = make_uint4(w[4], w[5], w[6], w[7]);
+              }
             }
+          }
+          if (stage) {
+            __syncwarp();
+            const uint32_t vmask = __ballot_sync(0xffffffffu, valid);
+            const unsigned long long goff = ((unsigned long long)pix * p.C + col0) * 2ull;   // byte offset of this lane's row
+            for (int it = 0; it < (1 << chl); ++it) {
+              const int pl = it * (32 >> chl) + (lane >> chl);
+              const uint32_t ch = (uint32_t)lane & ((1u << chl) - 1u);
+              const uint32_t lo = __shfl_sync(0xffffffffu, (uint32_t)goff, pl), hi = __shfl_sync(0xffffffffu, (uint32_t)(goff >> 32), pl);
+              const uint32_t sw = ((uint32_t)pl >> (3 - chl)) & ((1u << chl) - 1u);
+              uint4 val;
+              asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(val.x), "=r"(val.y), "=r"(val.z), "=r"(val.w) : "r"(stg + (uint32_t)pl * rb + ((ch ^ sw) << 4)));
+              if ((vmask >> pl) & 1u)
+                *reinterpret_cast<uint4*>(reinterpret_cast<uint8_t*>(p.out) + (((unsigned long long)hi << 32) | lo) + ch * 16u) = val;
+            }
+            __syncwarp();
           }
         }
       }
@@ -313,6 +346,11 @@ bool conv_layout(ConvParams& q, int R, int* smem_bytes) {
   if (q.a2 < 0) q.a2 = 0;
   if (q.a2 > q.M2) q.a2 = q.M2;
   if (q.a1 >= q.M1) { q.a1 = q.M1; }
+  // Output staging uses the first 16 KB of the input rows. While the second group of the second convolution is
+  // still being computed it reads intermediate pixels >= a2 * 128 - Wp - 1, which lie two pixel slots lower.
+  const bool overlap = q.a2 > 0 && q.a2 < q.M2;   // an output epilogue runs next to MMAs that still read the rows
+  const long free_bytes = overlap ? (long)(q.a2 * 128 - q.Wp - 3) * q.w_row_bytes : (long)x_reach;
+  q.stage_ok = free_bytes >= 8 * 2048 ? 1 : 0;
   *smem_bytes = off + 1024;
   return *smem_bytes <= 227 * 1024;
 }
