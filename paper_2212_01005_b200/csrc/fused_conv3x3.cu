@@ -38,7 +38,7 @@ namespace {
 
 using namespace tc;
 
-constexpr int kEpiWarps = 8;                 // two per TMEM lane quarter: each takes half of the channels
+constexpr int kEpiWarps = 16;                // four per TMEM lane quarter: each takes a quarter of the channels (at least 16)
 constexpr int kEpiThreads = kEpiWarps * 32;
 constexpr int kMmaWarps = 4;                 // one issuing lane each, alternating M tiles: a single thread issues an MMA every ~70 cycles, the tensor pipe takes one every ~50
 constexpr int kThreads = kEpiThreads + 32 + 32 * kMmaWarps;   // + TMA warp + MMA warps
@@ -181,7 +181,7 @@ conv3x3_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
     // ================ epilogue warps: thread = (pixel row of a tile, half of the channels) ================
     const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
     const int row = (warp & 3) * 32 + lane;
-    const int ncol = max(16, p.C / 2);
+    const int ncol = max(16, p.C / (kEpiWarps / 4));
     const int col0 = (warp >> 2) * ncol;
     const bool has_cols = col0 < p.C;
 
@@ -350,7 +350,7 @@ bool conv_layout(ConvParams& q, int R, int* smem_bytes) {
   // still being computed it reads intermediate pixels >= a2 * 128 - Wp - 1, which lie two pixel slots lower.
   const bool overlap = q.a2 > 0 && q.a2 < q.M2;   // an output epilogue runs next to MMAs that still read the rows
   const long free_bytes = overlap ? (long)(q.a2 * 128 - q.Wp - 3) * q.w_row_bytes : (long)x_reach;
-  q.stage_ok = free_bytes >= 8 * 2048 ? 1 : 0;
+  q.stage_ok = free_bytes >= kEpiWarps * 2048 ? 1 : 0;
   *smem_bytes = off + 1024;
   return *smem_bytes <= 227 * 1024;
 }
