@@ -224,6 +224,43 @@ ago_status_t ago_subgraph_run_static(ago_subgraph_t h, const void* const* inputs
                                      const void* const* weights, void* const* outputs,
                                      void* cuda_stream);
 
+/* ---- Redundancy of intensive fusion (Section III-B, the GS / TS analysis) -----------------
+ * Two stacked convolutions (stride-1 upstream producing [N, O1, H1, W1]; downstream with an
+ * R2 x C2 window and stride `stride2` producing [N, O2, H2, W2], windows without padding, so
+ * H1 = (H2 - 1) * stride2 + R2 and likewise W1). After tiling the downstream output into tiles
+ * of (o2, h2, w2) and fusing, the upstream tile that each downstream tile needs is computed
+ * inside the downstream tile loops; an upstream element needed by several downstream tiles is
+ * computed once per tile. The call returns how many upstream output elements (and reduction-body
+ * executions, x I1 R1 C1) are computed with and without fusion, i.e. the paper's
+ * |GS2/TS2 x (GS1/TS1 - GS2/TS2)| * |TS1| against |GS1|, with ragged edge tiles counted exactly.
+ * A dense downstream operator (depthwise2 == 0) needs all O1 upstream channels for every tile of
+ * output channels; a depthwise one (depthwise2 != 0, O2 == O1) needs the tile's own channels.
+ * Tile extents are clamped to the tensor extents. Host-only; no device is touched.
+ * Errors: AGO_ERR_INVALID_ARG for NULL pointers, a wrong struct_size or non-positive extents;
+ * AGO_ERR_SHAPE when depthwise2 is set and O2 != O1. */
+typedef struct {
+  uint32_t struct_size;
+  int32_t  depthwise2;            /* downstream operator is depthwise (channel c reads upstream channel c) */
+  int64_t  N;
+  int64_t  O1, I1, R1, C1;        /* upstream: output channels; reduction extents (input channels, window) */
+  int64_t  O2, R2, C2, stride2;   /* downstream: output channels, window, stride */
+  int64_t  H2, W2;                /* downstream output extent */
+  int64_t  o2, h2, w2;            /* downstream tile */
+} ago_redundancy_query_t;
+
+typedef struct {
+  int64_t num_tiles;              /* downstream tiles = |GS2 / TS2| */
+  int64_t upstream_elems_unfused; /* N O1 H1 W1 */
+  int64_t upstream_elems_fused;   /* sum over the downstream tiles of the upstream tile each one needs */
+  int64_t upstream_macs_unfused;  /* x I1 R1 C1 */
+  int64_t upstream_macs_fused;
+  double  factor;                 /* fused / unfused; 1.0 = no recomputation */
+  int32_t category;               /* ago_link_category_t of the pair */
+  int32_t reserved;
+} ago_redundancy_result_t;
+
+ago_status_t ago_fusion_redundancy(const ago_redundancy_query_t* q, ago_redundancy_result_t* out);
+
 /* Library version, "major.minor". */
 const char* ago_version(void);
 

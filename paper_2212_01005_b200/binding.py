@@ -40,8 +40,23 @@ AGO_STATIC_SCRATCH_BYTES = 4 << 20
 EXPORTS = [
     "ago_subgraph_create", "ago_subgraph_run", "ago_subgraph_run_host", "ago_subgraph_destroy", "ago_last_error",
     "ago_subgraph_workspace_bytes", "ago_subgraph_set_workspace", "ago_subgraph_query", "ago_subgraph_status",
-    "ago_version", "ago_subgraph_run_static",
+    "ago_version", "ago_subgraph_run_static", "ago_fusion_redundancy",
 ]
+
+
+class ago_redundancy_query_t(ctypes.Structure):
+    _fields_ = [("struct_size", ctypes.c_uint32), ("depthwise2", ctypes.c_int32), ("N", ctypes.c_int64),
+                ("O1", ctypes.c_int64), ("I1", ctypes.c_int64), ("R1", ctypes.c_int64), ("C1", ctypes.c_int64),
+                ("O2", ctypes.c_int64), ("R2", ctypes.c_int64), ("C2", ctypes.c_int64), ("stride2", ctypes.c_int64),
+                ("H2", ctypes.c_int64), ("W2", ctypes.c_int64),
+                ("o2", ctypes.c_int64), ("h2", ctypes.c_int64), ("w2", ctypes.c_int64)]
+
+
+class ago_redundancy_result_t(ctypes.Structure):
+    _fields_ = [("num_tiles", ctypes.c_int64), ("upstream_elems_unfused", ctypes.c_int64),
+                ("upstream_elems_fused", ctypes.c_int64), ("upstream_macs_unfused", ctypes.c_int64),
+                ("upstream_macs_fused", ctypes.c_int64), ("factor", ctypes.c_double),
+                ("category", ctypes.c_int32), ("reserved", ctypes.c_int32)]
 
 
 class ago_op_t(ctypes.Structure):
@@ -102,6 +117,8 @@ def load(build_if_missing: bool = True):
     lib.ago_subgraph_status.restype = ctypes.c_int
     lib.ago_subgraph_status.argtypes = [vp]
     lib.ago_version.restype = ctypes.c_char_p
+    lib.ago_fusion_redundancy.restype = ctypes.c_int
+    lib.ago_fusion_redundancy.argtypes = [ctypes.POINTER(ago_redundancy_query_t), ctypes.POINTER(ago_redundancy_result_t)]
     lib.ago_subgraph_run_static.restype = ctypes.c_int
     lib.ago_subgraph_run_static.argtypes = [vp, vpp, vpp, vpp, vp]
     _lib = lib
@@ -134,6 +151,26 @@ def _ptr_array(ptrs: Sequence[int]):
 
 def ago_subgraph_run(h, inputs: Sequence[int], weights: Sequence[int], outputs: Sequence[int], stream: int = 0) -> int:
     return load().ago_subgraph_run(h, _ptr_array(inputs), _ptr_array(weights), _ptr_array(outputs), stream)
+
+
+def ago_fusion_redundancy(**kw) -> dict:
+    """Upstream work of two stacked convolutions with and without intensive fusion (Section III-B).
+
+    Keyword arguments are the fields of ago_redundancy_query_t except struct_size (depthwise2 defaults to 0,
+    stride2, N, I1, R1, C1 to 1). Returns the fields of ago_redundancy_result_t as a dict; raises ValueError
+    with the library's message on a non-zero status.
+    """
+    q = ago_redundancy_query_t()
+    q.struct_size = ctypes.sizeof(ago_redundancy_query_t)
+    defaults = dict(depthwise2=0, N=1, I1=1, R1=1, C1=1, stride2=1)
+    defaults.update(kw)
+    for k, v in defaults.items():
+        setattr(q, k, int(v))
+    r = ago_redundancy_result_t()
+    st = load().ago_fusion_redundancy(ctypes.byref(q), ctypes.byref(r))
+    if st != AGO_OK:
+        raise ValueError(f"ago_fusion_redundancy: status {st}: {ago_last_error()[1]}")
+    return {name: getattr(r, name) for name, _ in ago_redundancy_result_t._fields_ if name != "reserved"}
 
 
 def ago_subgraph_run_static(h, inputs: Sequence[int], weights: Sequence[int], outputs: Sequence[int], stream: int = 0) -> int:
