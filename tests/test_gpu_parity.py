@@ -24,6 +24,9 @@ def small_workloads():
         "ffn_small": WL.ffn("ffn_small", [24], 200, 128, 512, 1),
         "ffn_ragged": WL.ffn("ffn_ragged", [25], 77, 96, 264, 1),
         "ffn_rows_ragged": WL.ffn("ffn_rows_ragged", [30], 333, 256, 384, 1),
+        # tall enough that the fused kernel keeps 2 / 3 hidden tiles per CTA (100 row blocks x 6 / 9 hidden tiles)
+        "ffn_g2": WL.ffn("ffn_g2", [31], 12800, 128, 768, 1),
+        "ffn_g3": WL.ffn("ffn_g3", [32], 12800, 128, 1152, 1),
         "resnet_small": WL.resnet_block("resnet_small", [26], 2, 12, 64),
         "resnet_odd": WL.resnet_block("resnet_odd", [27], 1, 9, 32),
         "resnet_16ch": WL.resnet_block("resnet_16ch", [32], 2, 20, 16),
@@ -89,7 +92,7 @@ def test_padding_of_the_intermediate_with_large_bias(ago):
 
 # ---- fused kernels -------------------------------------------------------------------
 
-FUSED_SMALL = ["mbv2_14", "mbv2_s1_odd", "mbv2_s2", "mbv2_s2_odd", "attn_small", "attn_ragged", "ffn_small", "ffn_rows_ragged", "resnet_small", "resnet_odd", "resnet_16ch"]
+FUSED_SMALL = ["mbv2_14", "mbv2_s1_odd", "mbv2_s2", "mbv2_s2_odd", "attn_small", "attn_ragged", "ffn_small", "ffn_rows_ragged", "ffn_g2", "ffn_g3", "resnet_small", "resnet_odd", "resnet_16ch"]
 
 
 @pytest.mark.parametrize("name", FUSED_SMALL)
