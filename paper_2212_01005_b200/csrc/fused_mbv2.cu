@@ -30,6 +30,7 @@
 #include <cuda.h>
 #include <cuda_bf16.h>
 
+#include <algorithm>
 #include <cstdlib>
 
 #include "fused.h"
@@ -64,7 +65,9 @@ struct Mbv2Params {
   int R, strips, IH, IW, P_x, P_in, M1, M2;   // P_x = IH * W pixels in the input tile, P_in = IH * IW in an E chunk
   int Kp, row_bytes, swizzle;   // input / W1 tiles: padded K, bytes per row, tc::SwizzleMode
   int Coutp, NC;
-  uint32_t coutp_recip;         // 2^32 / Coutp + 1: x / Coutp == __umulhi(x, coutp_recip) for the small x used here
+  // 2^32 / d + 1 for the run-time divisors of the index arithmetic: x / d == __umulhi(x, recip) for x, d < 65536
+  uint32_t coutp_recip, w_recip, strips_recip, per_row_recip;
+  int per_row, nseg, step_r, step_c, col_slots;   // depthwise item geometry (see the kernel), fixed per shape
   int tmem_cols, ecol0, pcol0;
   int e_plane, d_plane;         // byte distance between the two 8-channel planes of an E / D chunk
   // shared-memory byte offsets (from the 1024-aligned base)
@@ -204,7 +207,7 @@ mbv2_fused_kernel(const Mbv2Params p) {
   volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(bars + 13);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int n = blockIdx.x / p.strips, strip = blockIdx.x % p.strips;
+  const int n = (int)__umulhi(blockIdx.x, p.strips_recip), strip = (int)blockIdx.x - n * p.strips;
   const int ho0 = strip * p.R;
   const int rows_valid = min(p.R, p.Ho - ho0);
   const int gh0 = ho0 * p.stride - 1;   // image row of tile row 0
@@ -297,13 +300,15 @@ mbv2_fused_kernel(const Mbv2Params p) {
     const int cp = gt & 7, slot = gt >> 3;
     const int cp_off = (cp & 3) * 4;   // byte offset inside a 16-byte pixel entry
     const uint32_t e_pitch = (uint32_t)p.IW * 16u, d_pitch = (uint32_t)p.Wo * 16u;
-    const int nseg = (p.Wo + kSegCols - 1) / kSegCols;
-    const int groups = max(1, min(rows_valid, kSlots / max(1, min(p.Wo, kSlots))));   // stride 2: row groups
-    const int rows_per_group = (rows_valid + groups - 1) / groups;
-    const int per_row = p.stride == 1 ? nseg : p.Wo;                       // items per output row / per row group
+    const int per_row = p.per_row;                                         // items per output row (stride 1: column segments) / per row group
+    int groups = 1, rows_per_group = rows_valid;                           // stride 2: row groups
+    if (p.stride != 1) {
+      groups = max(1, min(rows_valid, p.col_slots));
+      rows_per_group = (rows_valid + groups - 1) / groups;
+    }
     const int dw_items = per_row * (p.stride == 1 ? (rows_valid + 1) / 2 : groups);   // stride 1: blocks of two rows
-    const int item0_r = slot / per_row, item0_c = slot - item0_r * per_row;   // the thread's first item
-    const int step_r = kSlots / per_row, step_c = kSlots - step_r * per_row;  // item += kSlots in (row, column) form
+    const int item0_r = (int)__umulhi((uint32_t)slot, p.per_row_recip), item0_c = slot - item0_r * per_row;   // the thread's first item
+    const int step_r = p.step_r, step_c = p.step_c;                        // item += kSlots in (row, column) form
     const int e_bytes = 2 * p.e_plane;
     // Expand-epilogue tiles of this warp: the group's warps of one tensor-memory lane quarter (warp & 3) share the M1
     // tiles round-robin, at most kTilesPerWarp each. e_pix[k]: pixel index in an E plane (the tile has no padding
@@ -318,7 +323,7 @@ mbv2_fused_kernel(const Mbv2Params p) {
     for (int k = 0; k < kTilesPerWarp; ++k) {
       const int t = q_rank + k * q_mates;
       const int pix = t * 128 + (warp & 3) * 32 + lane;
-      const int ih = pix / p.W, iw = pix - ih * p.W;
+      const int ih = (int)__umulhi((uint32_t)pix, p.w_recip), iw = pix - ih * p.W;
       const int gh = gh0 + ih;
       e_pix[k] = -1;
       if (t < p.M1 && pix < p.P_x) {
@@ -548,6 +553,7 @@ struct Mbv2Host {
 bool layout(Mbv2Params& q, int R, int* smem_bytes) {
   q.R = R;
   q.strips = (q.Ho + R - 1) / R;
+  q.strips_recip = (uint32_t)((1ull << 32) / (uint64_t)q.strips + 1ull);
   q.IH = (R - 1) * q.stride + 3;
   q.IW = q.W + 2;
   q.P_in = q.IH * q.IW;
@@ -604,7 +610,17 @@ ago_status_t mbv2_plan(Plan* plan, FusedState* st, std::string* err) {
   q.swizzle = q.Kp == 16 ? tc::SW_32B : (q.Kp == 32 ? tc::SW_64B : tc::SW_128B);
   q.Coutp = round_up(q.Cout, 16);
   q.NC = q.Cexp / kChunk;
-  q.coutp_recip = (uint32_t)((1ull << 32) / (uint64_t)q.Coutp + 1ull);
+  auto recip = [](int d) { return (uint32_t)((1ull << 32) / (uint64_t)d + 1ull); };
+  q.coutp_recip = recip(q.Coutp);
+  q.w_recip = recip(q.W);
+  {
+    constexpr int kSlots = kGroupThreads / 8;
+    q.nseg = (q.Wo + kSegCols - 1) / kSegCols;
+    q.per_row = q.stride == 1 ? q.nseg : q.Wo;
+    q.per_row_recip = recip(q.per_row);
+    q.step_r = kSlots / q.per_row; q.step_c = kSlots - q.step_r * q.per_row;
+    q.col_slots = kSlots / std::max(1, std::min(q.Wo, kSlots));
+  }
   // Rows per CTA: fewest waves over the SMs, then least halo + tail work.
   int best_R = 0; double best_cost = 0; int best_smem = 0;
   const int sms = 148;
