@@ -340,7 +340,7 @@ bool conv_layout(ConvParams& q, int R, int* smem_bytes) {
   off += 256;
   // pipeline groups: the second convolution's first group may only read intermediate rows the first
   // group of the first convolution produces
-  q.a1 = (q.M1 * 3 + 4) / 5;
+  q.a1 = (q.M1 + 1) / 2;   // even groups: a pass of only three tiles keeps the tensor pipe less busy than one of four or five
   if (q.a1 < 1) q.a1 = 1;
   q.a2 = (q.a1 * 128 - 2 * q.Wp - 1) / 128;
   if (q.a2 < 0) q.a2 = 0;
