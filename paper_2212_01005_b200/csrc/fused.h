@@ -36,6 +36,25 @@ ago_status_t conv3x3_run(const Plan& plan, FusedState* st, const void* const* in
 ago_status_t mbv2_run(const Plan& plan, FusedState* st, const void* const* inputs, const void* const* weights,
                       void* output, unsigned int* status_word, cudaStream_t stream, std::string* err);
 
+// Launch configuration of a fused kernel: programmatic stream serialization allowed, so the grid may be
+// scheduled while the previous grid of the stream drains (the kernels call griddepcontrol.wait before
+// touching device memory). Use with cudaLaunchKernelEx(&cfg.config, kernel, args...).
+struct FusedLaunch {
+  cudaLaunchConfig_t config;
+  cudaLaunchAttribute attr[1];
+  FusedLaunch(dim3 grid, int threads, size_t smem_bytes, cudaStream_t stream) {
+    config = cudaLaunchConfig_t{};
+    config.gridDim = grid;
+    config.blockDim = dim3((unsigned)threads, 1, 1);
+    config.dynamicSmemBytes = smem_bytes;
+    config.stream = stream;
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    config.attrs = attr;
+    config.numAttrs = 1;
+  }
+};
+
 // Chooses tiles and shared-memory budget for plan->fused_kernel; fills
 // plan->tile_rows / smem_bytes. Host only.
 ago_status_t fused_plan(Plan* plan, FusedState* st, std::string* err);

@@ -93,6 +93,8 @@ attention_fused_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int h = blockIdx.x, b = blockIdx.y;
+  grid_dependency_wait();      // the previous grid of the stream has completed; device memory may be touched
+  grid_launch_dependents();
 
   if (tid == kComputeThreads) {
     *abort_flag = 0u;
@@ -441,8 +443,8 @@ ago_status_t attention_run(const Plan& plan, FusedState* st, const void* const* 
     if (e != cudaSuccess) { *err = std::string("cudaFuncSetAttribute: ") + cudaGetErrorString(e); return AGO_ERR_CUDA; }
   }
   dim3 grid(q.heads, q.B);
-  attention_fused_kernel<<<grid, kThreads, host->smem_bytes, stream>>>(*maps[0], *maps[1], *maps[2], q);
-  cudaError_t e = cudaGetLastError();
+  FusedLaunch launch(grid, kThreads, (size_t)host->smem_bytes, stream);
+  cudaError_t e = cudaLaunchKernelEx(&launch.config, attention_fused_kernel, *maps[0], *maps[1], *maps[2], q);
   if (e != cudaSuccess) { *err = std::string("fused attention launch: ") + cudaGetErrorString(e); return AGO_ERR_CUDA; }
   return AGO_OK;
 }

@@ -84,6 +84,8 @@ conv3x3_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
   const int rows_valid = min(p.R, p.H - h0);
   const int ksteps = p.C / 16;
 
+  grid_dependency_wait();      // the previous grid of the stream has completed; device memory may be touched
+  grid_launch_dependents();
   if (tid == kEpiThreads) {
     *abort_flag = 0u;
     mbar_init(bar_x, 1);
@@ -426,8 +428,8 @@ ago_status_t conv3x3_run(const Plan& plan, FusedState* st, const void* const* in
     cudaError_t e = ensure_max_dynamic_smem(reinterpret_cast<const void*>(conv3x3_pair_kernel), smem_opt_in);
     if (e != cudaSuccess) { *err = std::string("cudaFuncSetAttribute: ") + cudaGetErrorString(e); return AGO_ERR_CUDA; }
   }
-  conv3x3_pair_kernel<<<q.N * q.strips, kThreads, host->smem_bytes, stream>>>(mx, mw1, mw2, q);
-  cudaError_t e = cudaGetLastError();
+  FusedLaunch launch(dim3((unsigned)(q.N * q.strips)), kThreads, (size_t)host->smem_bytes, stream);
+  cudaError_t e = cudaLaunchKernelEx(&launch.config, conv3x3_pair_kernel, mx, mw1, mw2, q);
   if (e != cudaSuccess) { *err = std::string("fused conv3x3 pair launch: ") + cudaGetErrorString(e); return AGO_ERR_CUDA; }
   return AGO_OK;
 }

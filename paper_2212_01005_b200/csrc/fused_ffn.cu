@@ -97,6 +97,8 @@ ffn_fused_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
   const int hc = blockIdx.x, rb = blockIdx.y;   // group of G hidden tiles, row block
   const int row0 = rb * kBM;
   const int G = p.G, stages = p.stages;
+  grid_dependency_wait();      // the previous grid of the stream has completed; device memory may be touched
+  grid_launch_dependents();
   // tensor memory: columns [0, 256) two first-GEMM accumulators, [256, 512) two output-slice accumulators
   constexpr uint32_t kOutCol = 256;
 
@@ -384,8 +386,8 @@ ago_status_t ffn_run(const Plan& plan, FusedState* st, const void* const* inputs
     if (e != cudaSuccess) { *err = std::string("cudaFuncSetAttribute: ") + cudaGetErrorString(e); return AGO_ERR_CUDA; }
   }
   dim3 grid(q.hctas, (q.M + kBM - 1) / kBM);
-  ffn_fused_kernel<<<grid, kThreads, host->smem_bytes, stream>>>(mx, mw1, mw2, q);
-  cudaError_t e = cudaGetLastError();
+  FusedLaunch launch(grid, kThreads, (size_t)host->smem_bytes, stream);
+  cudaError_t e = cudaLaunchKernelEx(&launch.config, ffn_fused_kernel, mx, mw1, mw2, q);
   if (e != cudaSuccess) { *err = std::string("fused feed-forward launch: ") + cudaGetErrorString(e); return AGO_ERR_CUDA; }
   return AGO_OK;
 }

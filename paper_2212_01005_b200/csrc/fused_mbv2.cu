@@ -267,25 +267,8 @@ mbv2_fused_kernel(const Mbv2Params p) {
     auto load_or_zero = [](const uint8_t* src) {
       return src ? __ldg(reinterpret_cast<const uint4*>(src)) : make_uint4(0, 0, 0, 0);
     };
-    uint4 vx[kBX], vw[kBW];
-    uint32_t dx[kBX], dw[kBW];
-#pragma unroll
-    for (int k = 0; k < kBX; ++k) {
-      const uint32_t i = (uint32_t)(tid + k * kThreads);
-      const uint8_t* src = nullptr;
-      dx[k] = 0xffffffffu;
-      if (i < nX) dx[k] = x_slot(i, src);
-      vx[k] = load_or_zero(src);
-    }
-#pragma unroll
-    for (int k = 0; k < kBW; ++k) {
-      const uint32_t i = (uint32_t)(tid + k * kThreads);
-      const uint8_t* src = nullptr;
-      dw[k] = 0xffffffffu;
-      if (i < nW) dw[k] = w_slot(i, src);
-      vw[k] = load_or_zero(src);
-    }
-    // ---- per-thread work mapping, computed while the loads are in flight ----
+    // ---- per-thread work mapping: needs no device memory, so it runs before the wait for the previous grid of the
+    // stream (with back-to-back launches it overlaps that grid's tail) ----
     const int g = warp / kGroupWarps;
     const int gwarp0 = g * kGroupWarps;           // first warp of the group
     const int gt = tid - gwarp0 * 32;             // thread index in the group
@@ -332,6 +315,26 @@ mbv2_fused_kernel(const Mbv2Params p) {
       }
     }
 
+    uint4 vx[kBX], vw[kBW];
+    uint32_t dx[kBX], dw[kBW];
+    grid_dependency_wait();      // first access to device memory below
+    grid_launch_dependents();
+#pragma unroll
+    for (int k = 0; k < kBX; ++k) {
+      const uint32_t i = (uint32_t)(tid + k * kThreads);
+      const uint8_t* src = nullptr;
+      dx[k] = 0xffffffffu;
+      if (i < nX) dx[k] = x_slot(i, src);
+      vx[k] = load_or_zero(src);
+    }
+#pragma unroll
+    for (int k = 0; k < kBW; ++k) {
+      const uint32_t i = (uint32_t)(tid + k * kThreads);
+      const uint8_t* src = nullptr;
+      dw[k] = 0xffffffffu;
+      if (i < nW) dw[k] = w_slot(i, src);
+      vw[k] = load_or_zero(src);
+    }
     if (warp == 0) {
       tmem_alloc(tmem_slot, (uint32_t)p.tmem_cols);
       tmem_relinquish();
@@ -657,8 +660,8 @@ ago_status_t mbv2_run(const Plan& plan, FusedState* st, const void* const* input
     cudaError_t e = ensure_max_dynamic_smem(reinterpret_cast<const void*>(mbv2_fused_kernel), smem_opt_in);
     if (e != cudaSuccess) { *err = std::string("cudaFuncSetAttribute: ") + cudaGetErrorString(e); return AGO_ERR_CUDA; }
   }
-  mbv2_fused_kernel<<<q.N * q.strips, kThreads, host->smem_bytes, stream>>>(q);
-  cudaError_t e = cudaGetLastError();
+  FusedLaunch launch(dim3((unsigned)(q.N * q.strips)), kThreads, (size_t)host->smem_bytes, stream);
+  cudaError_t e = cudaLaunchKernelEx(&launch.config, mbv2_fused_kernel, q);
   if (e != cudaSuccess) { *err = std::string("fused inverted-residual launch: ") + cudaGetErrorString(e); return AGO_ERR_CUDA; }
   return AGO_OK;
 }

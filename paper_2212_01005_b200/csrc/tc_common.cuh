@@ -95,6 +95,15 @@ __device__ __forceinline__ void named_barrier_sync(uint32_t id, uint32_t threads
   asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
 }
 
+// ---- programmatic dependent launch -----------------------------------------------------------------
+// The fused kernels are launched with programmatic stream serialization: a grid may be scheduled while the
+// previous grid of the stream is still running, so that its launch latency and its set-up (barriers, tensor
+// memory, index arithmetic) overlap that grid's tail. grid_dependency_wait() returns once the previous grid has
+// completed and its memory is visible -- every thread calls it before its first access to device memory.
+// (Without the launch attribute both are no-ops.)
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 // ---- proxies and fences ---------------------------------------------------------------
 
 // Make generic-proxy shared-memory writes visible to the async proxy (TMA, tcgen05.mma).
