@@ -275,17 +275,31 @@ ffn_fused_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
     named_barrier_sync(1, kEpiThreads);
     if (*last_flag) {
       __threadfence();
-      // the epilogue threads sweep the row block's rows with coalesced 16-byte accesses
+      // the epilogue threads sweep the row block's rows with coalesced 16-byte accesses, eight loads in flight per
+      // thread (one CTA finalises a whole row block: the sweep is latency-bound otherwise)
       const int vec_per_row = p.N2 / 4;
       const int rows_here = min(kBM, p.M - row0);
-      for (int idx = tid; idx < rows_here * vec_per_row; idx += kEpiThreads) {
-        const int r = idx / vec_per_row, c = (idx - r * vec_per_row) * 4;
-        float4* src = reinterpret_cast<float4*>(p.acc + (size_t)(row0 + r) * p.N2 + c);
-        const float4 a = __ldcg(src);
-        const float4 bb = __ldg(reinterpret_cast<const float4*>(p.b2 + c));
-        *src = make_float4(0.f, 0.f, 0.f, 0.f);
-        const uint2 o = make_uint2(pack_bf16x2(a.x + bb.x, a.y + bb.y), pack_bf16x2(a.z + bb.z, a.w + bb.w));
-        *reinterpret_cast<uint2*>(p.out + (size_t)(row0 + r) * p.N2 + c) = o;
+      const int total = rows_here * vec_per_row;
+      float4* acc0 = reinterpret_cast<float4*>(p.acc + (size_t)row0 * p.N2);      // the row block is contiguous
+      uint2* out0 = reinterpret_cast<uint2*>(p.out + (size_t)row0 * p.N2);
+      constexpr int kInFlight = 8;
+      for (int base = tid; base < total; base += kInFlight * kEpiThreads) {
+        float4 a[kInFlight];
+#pragma unroll
+        for (int k = 0; k < kInFlight; ++k) {
+          const int idx = base + k * kEpiThreads;
+          a[k] = idx < total ? __ldcg(acc0 + idx) : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+#pragma unroll
+        for (int k = 0; k < kInFlight; ++k) {
+          const int idx = base + k * kEpiThreads;
+          if (idx < total) {
+            const int c = (idx % vec_per_row) * 4;
+            const float4 bb = __ldg(reinterpret_cast<const float4*>(p.b2 + c));
+            acc0[idx] = make_float4(0.f, 0.f, 0.f, 0.f);
+            out0[idx] = make_uint2(pack_bf16x2(a[k].x + bb.x, a[k].y + bb.y), pack_bf16x2(a[k].z + bb.z, a[k].w + bb.w));
+          }
+        }
       }
       if (tid == 0) p.counters[rb] = 0u;
     }
