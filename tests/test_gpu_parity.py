@@ -128,6 +128,8 @@ def test_fused_mbv2_pads_the_intermediate_not_the_input(ago):
     dict(N=1, H=20, c_in=64, c_exp=64, c_out=40, stride=1, residual=False),   # 128-byte input rows, Cout not a multiple of 16
     dict(N=3, H=5, c_in=8, c_exp=16, c_out=8, stride=2, residual=False),      # one chunk, tiny image, odd size
     dict(N=1, H=30, c_in=40, c_exp=240, c_out=80, stride=2, residual=False),  # Cin padded 40 -> 64
+    dict(N=1, H=32, c_in=64, c_exp=64, c_out=64, stride=1, residual=True),    # large 128-byte-row tile: more input slots than one staging pass
+    dict(N=2, H=24, c_in=64, c_exp=384, c_out=64, stride=1, residual=True),   # many weight slots, 24 chunks
 ])
 def test_fused_mbv2_shape_sweep(ago, shape):
     wl = WL.mbv2_block("sweep", [41, shape["H"], shape["c_in"]], shape["N"], shape["H"], shape["c_in"], shape["c_exp"],
