@@ -261,6 +261,33 @@ typedef struct {
 
 ago_status_t ago_fusion_redundancy(const ago_redundancy_query_t* q, ago_redundancy_result_t* out);
 
+/* ---- Graph partitioning of the frontend (Section IV, Eq. 1 and Algorithm 1) ----------------
+ * Host-only. ago_op_weight is Eq. 1: c * prod over the operator's loops of log(extent) + b
+ * (natural logarithm; the paper prints no values for c and b, they are the caller's).
+ *
+ * ago_graph_cluster runs Algorithm 1 ("Cluster") on a DAG of num_nodes operators with the given
+ * weights and num_edges directed edges (edges[2e] -> edges[2e + 1]): repeatedly the heaviest
+ * candidate (hyper) node v absorbs the lightest node u of its affix set (adjacent to v, exactly
+ * one topological stage above or below, Definitions 2 and 3) while w_v + w_u < threshold, else v
+ * leaves the candidates; stages and edges are updated after every merge. By Theorem 1 the
+ * resulting partition is acyclic. Ties: heavier first, then the smaller smallest-member id;
+ * lighter first, then the smaller smallest-member id.
+ * Output: subgraph_of_node[num_nodes] (subgraphs numbered by their smallest member) and
+ * *num_subgraphs. Errors: AGO_ERR_INVALID_ARG for NULL arguments, a wrong struct_size, an empty
+ * graph, an edge that names no node or a self loop, or a cyclic input graph. */
+typedef struct {
+  uint32_t struct_size;
+  int32_t  num_nodes;
+  const double*  weights;   /* [num_nodes] */
+  int32_t  num_edges;
+  int32_t  reserved;
+  const int32_t* edges;     /* [2 * num_edges] */
+  double   threshold;       /* Td: a merged subgraph's weight stays below it */
+} ago_graph_desc_t;
+
+double       ago_op_weight(const int64_t* loop_extents, int32_t num_loops, double c, double b);
+ago_status_t ago_graph_cluster(const ago_graph_desc_t* g, int32_t* subgraph_of_node, int32_t* num_subgraphs);
+
 /* Library version, "major.minor". */
 const char* ago_version(void);
 

@@ -40,7 +40,7 @@ AGO_STATIC_SCRATCH_BYTES = 4 << 20
 EXPORTS = [
     "ago_subgraph_create", "ago_subgraph_run", "ago_subgraph_run_host", "ago_subgraph_destroy", "ago_last_error",
     "ago_subgraph_workspace_bytes", "ago_subgraph_set_workspace", "ago_subgraph_query", "ago_subgraph_status",
-    "ago_version", "ago_subgraph_run_static", "ago_fusion_redundancy",
+    "ago_version", "ago_subgraph_run_static", "ago_fusion_redundancy", "ago_op_weight", "ago_graph_cluster",
 ]
 
 
@@ -57,6 +57,12 @@ class ago_redundancy_result_t(ctypes.Structure):
                 ("upstream_elems_fused", ctypes.c_int64), ("upstream_macs_unfused", ctypes.c_int64),
                 ("upstream_macs_fused", ctypes.c_int64), ("factor", ctypes.c_double),
                 ("category", ctypes.c_int32), ("reserved", ctypes.c_int32)]
+
+
+class ago_graph_desc_t(ctypes.Structure):
+    _fields_ = [("struct_size", ctypes.c_uint32), ("num_nodes", ctypes.c_int32), ("weights", ctypes.POINTER(ctypes.c_double)),
+                ("num_edges", ctypes.c_int32), ("reserved", ctypes.c_int32), ("edges", ctypes.POINTER(ctypes.c_int32)),
+                ("threshold", ctypes.c_double)]
 
 
 class ago_op_t(ctypes.Structure):
@@ -117,6 +123,10 @@ def load(build_if_missing: bool = True):
     lib.ago_subgraph_status.restype = ctypes.c_int
     lib.ago_subgraph_status.argtypes = [vp]
     lib.ago_version.restype = ctypes.c_char_p
+    lib.ago_op_weight.restype = ctypes.c_double
+    lib.ago_op_weight.argtypes = [ctypes.POINTER(ctypes.c_int64), ctypes.c_int32, ctypes.c_double, ctypes.c_double]
+    lib.ago_graph_cluster.restype = ctypes.c_int
+    lib.ago_graph_cluster.argtypes = [ctypes.POINTER(ago_graph_desc_t), ctypes.POINTER(ctypes.c_int32), ctypes.POINTER(ctypes.c_int32)]
     lib.ago_fusion_redundancy.restype = ctypes.c_int
     lib.ago_fusion_redundancy.argtypes = [ctypes.POINTER(ago_redundancy_query_t), ctypes.POINTER(ago_redundancy_result_t)]
     lib.ago_subgraph_run_static.restype = ctypes.c_int
@@ -151,6 +161,29 @@ def _ptr_array(ptrs: Sequence[int]):
 
 def ago_subgraph_run(h, inputs: Sequence[int], weights: Sequence[int], outputs: Sequence[int], stream: int = 0) -> int:
     return load().ago_subgraph_run(h, _ptr_array(inputs), _ptr_array(weights), _ptr_array(outputs), stream)
+
+
+def ago_op_weight(loop_extents: Sequence[int], c: float = 1.0, b: float = 0.0) -> float:
+    """Eq. 1: c * prod(log(extent)) + b."""
+    arr = (ctypes.c_int64 * max(1, len(loop_extents)))(*[int(x) for x in loop_extents])
+    return float(load().ago_op_weight(arr, len(loop_extents), float(c), float(b)))
+
+
+def ago_graph_cluster(weights: Sequence[float], edges: Sequence[Sequence[int]], threshold: float):
+    """Algorithm 1 on a DAG: returns the subgraph index of every node (numbered by smallest member)."""
+    n = len(weights)
+    w = (ctypes.c_double * max(1, n))(*[float(x) for x in weights])
+    flat = [int(x) for e in edges for x in e]
+    ed = (ctypes.c_int32 * max(1, len(flat)))(*flat)
+    g = ago_graph_desc_t()
+    g.struct_size = ctypes.sizeof(ago_graph_desc_t)
+    g.num_nodes, g.weights, g.num_edges, g.edges, g.threshold = n, w, len(edges), ed, float(threshold)
+    out = (ctypes.c_int32 * max(1, n))()
+    cnt = ctypes.c_int32(0)
+    st = load().ago_graph_cluster(ctypes.byref(g), out, ctypes.byref(cnt))
+    if st != AGO_OK:
+        raise ValueError(f"ago_graph_cluster: status {st}: {ago_last_error()[1]}")
+    return list(out[:n]), int(cnt.value)
 
 
 def ago_fusion_redundancy(**kw) -> dict:
