@@ -92,7 +92,9 @@ cudaError_t launch_complex(const Plan& p, const OpInfo& o, const void* src, int 
     a.Ho = (int)o.out.d[1]; a.Wo = (int)o.out.d[2];
     a.dtype = p.dtype; a.in_dtype = src_dtype; a.out_dtype = dst_dtype;
     a.epi = epi;
-    return tuned_depthwise ? launch_depthwise_fused(a, stream) : launch_depthwise_generic(a, stream);
+    // the vectorised kernel serves every stage whose input and output are stored in the I/O dtype
+    const bool vec_ok = src_dtype == p.dtype && dst_dtype == p.dtype && a.C % (p.dtype == AGO_FP32 ? 4 : 8) == 0;
+    return (tuned_depthwise || vec_ok) ? launch_depthwise_fused(a, stream) : launch_depthwise_generic(a, stream);
   }
   GemmArgs g{};
   g.A = src; g.C = dst; g.epi = epi;
@@ -151,6 +153,7 @@ cudaError_t launch_complex(const Plan& p, const OpInfo& o, const void* src, int 
     default:
       return cudaErrorInvalidValue;
   }
+  if (p.dtype == AGO_BF16 && gemm_tc_supported(g)) return launch_gemm_tc(g, p.dtype, stream);
   return launch_gemm_generic(g, stream);
 }
 
