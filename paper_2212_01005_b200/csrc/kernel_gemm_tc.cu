@@ -11,6 +11,7 @@
 #include <cuda.h>
 #include <cuda_bf16.h>
 
+#include <algorithm>
 #include <mutex>
 #include <unordered_map>
 
@@ -25,7 +26,7 @@ namespace {
 using namespace tc;
 
 constexpr int kBM = 128, kBN = 128, kBK = 64;
-constexpr int kStages = 4;
+constexpr int kMaxStages = 4;   // ring stages in use = min(4, K blocks): short reductions leave room for several CTAs per SM
 constexpr int kStageBytes = 32 * 1024;
 constexpr int kEpiThreads = 128;
 constexpr int kThreads = kEpiThreads + 64;   // + TMA warp + MMA warp
@@ -36,7 +37,8 @@ struct GemmTcParams {
   int64_t ldc;
   int b_kmajor;
   int c_dtype, add_dtype;
-  int kblocks;
+  int kblocks, stages;
+  int bar_off;             // shared-memory offset of the barriers: after the ring and after the epilogue's staging tile
   // the simple operators in canonical order: + bias, activation 1, * scale, + tensor, activation 2
   const float* bias;       // or null
   const void* add;         // or null; same shape and leading dimension as C
@@ -55,15 +57,16 @@ __device__ __forceinline__ float gelu_tanh_f(float v) {
   return 0.5f * v * (1.0f + tanhf(c * (v + 0.044715f * v * v * v)));
 }
 
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __launch_bounds__(kThreads)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b, const GemmTcParams p) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t* sRing = smem;
-  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + kStages * kStageBytes);
+  const int kStages = p.stages;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + p.bar_off);
   uint64_t* bar_full = bars;
-  uint64_t* bar_empty = bars + kStages;
-  uint64_t* bar_acc = bars + 2 * kStages;
+  uint64_t* bar_empty = bars + kMaxStages;
+  uint64_t* bar_acc = bars + 2 * kMaxStages;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bar_acc + 1);
   volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(bar_acc + 2);
 
@@ -272,13 +275,19 @@ cudaError_t launch_gemm_tc(const GemmArgs& a, int add_dtype, cudaStream_t stream
   p.c_dtype = a.c_dtype; p.add_dtype = add_dtype;
   p.kblocks = (a.K + kBK - 1) / kBK;
   canonical_epilogue(a.epi, &p);
-  const int smem = kStages * kStageBytes + 256 + 1024;
+  p.stages = std::min(kMaxStages, p.kblocks);
+  // the epilogue stages the output tile (128 rows x (columns x element size + 16) bytes) over the idle ring
+  const int tile_cols = std::min(kBN, (a.N + 15) & ~15);
+  const int staging = kBM * (tile_cols * (a.c_dtype == AGO_FP32 ? 4 : 2) + 16);
+  p.bar_off = (std::max(p.stages * kStageBytes, staging) + 1023) & ~1023;
+  const int smem = p.bar_off + 256 + 1024;
+  const int smem_max = kMaxStages * kStageBytes + 256 + 1024;
   static std::once_flag once[64];
   int dev = 0;
   cudaError_t e = cudaGetDevice(&dev);
   if (e != cudaSuccess) return e;
   if (dev >= 0 && dev < 64)
-    std::call_once(once[dev], [&] { cudaFuncSetAttribute(gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem); });
+    std::call_once(once[dev], [&] { cudaFuncSetAttribute(gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_max); });
   dim3 grid((a.M + kBM - 1) / kBM, (a.N + kBN - 1) / kBN);
   gemm_tc_kernel<<<grid, kThreads, smem, stream>>>(ma, mb, p);
   return cudaGetLastError();
