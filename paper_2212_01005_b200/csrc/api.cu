@@ -102,6 +102,17 @@ cudaError_t launch_complex(const Plan& p, const OpInfo& o, const void* src, int 
   g.batches = 1; g.heads = 1;
   switch (o.op.kind) {
     case AGO_OP_CONV2D: {
+      // 3x3 convolutions of equal width with a (bias)(relu) or (bias)(add)(relu) epilogue: tensor-core stage kernel
+      if (p.dtype == AGO_BF16 && src_dtype == AGO_BF16 && dst_dtype == AGO_BF16 &&
+          conv3x3_tc_supported((int)o.in.d[1], (int)o.in.d[2], (int)o.in.d[3], q[0], q[1], q[2], q[3], q[4])) {
+        const float* bias = nullptr; const void* res = nullptr; int relu = 0, k = 0;
+        if (k < epi.n && epi.code[k] == EPI_BIAS) bias = static_cast<const float*>(epi.ptr[k++]);
+        if (k < epi.n && epi.code[k] == EPI_ADD) res = epi.ptr[k++];
+        if (k < epi.n && epi.code[k] == EPI_RELU) { relu = 1; ++k; }
+        if (k == epi.n)
+          return launch_conv3x3_tc(src, weights[o.weight], bias, res, dst, (int)o.in.d[0], (int)o.in.d[1], (int)o.in.d[2],
+                                   (int)o.in.d[3], relu, stream);
+      }
       g.B = weights[o.weight];
       g.H = (int)o.in.d[1]; g.W = (int)o.in.d[2]; g.Cin = (int)o.in.d[3];
       g.R = q[1]; g.S = q[2]; g.stride = q[3]; g.pad = q[4];

@@ -26,6 +26,8 @@
 #include <cuda.h>
 #include <cuda_bf16.h>
 
+#include <algorithm>
+#include <mutex>
 #include <unordered_map>
 
 #include "fused.h"
@@ -54,11 +56,17 @@ struct ConvParams {
   int R, strips, IH, Wp, P1, M1, P2, M2;
   int a1, a2;              // tiles [0,a1) of conv1 / [0,a2) of conv2 form the first pipeline group
   int stage_ok;            // the first 16 KB of the input rows are free for output staging whenever an output epilogue runs
+  // single-convolution variant (a stage of the unfused mode): out = [relu](conv(x) + b2 [+ res])
+  const __nv_bfloat16* res; // residual tensor (the pair kernel adds its own input)
+  int residual, relu;
   int w_row_bytes, w_swizzle, w_stage_bytes;
   int wstages;             // ring stages in use (2..kMaxWStages)
   int off_x, off_y, off_w, off_bias, off_bar;
 };
 
+// SINGLE = false: the fused pair. SINGLE = true: one convolution with its simple operators (second-convolution
+// passes only, reading the input rows directly), the tensor-core stage kernel of the unfused mode.
+template <bool SINGLE>
 __global__ void __launch_bounds__(kThreads, 1)
 conv3x3_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w1,
                     const __grid_constant__ CUtensorMap tmap_w2, const ConvParams p) {
@@ -95,21 +103,21 @@ conv3x3_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
     fence_proxy_async_smem();
     tma_prefetch_desc(&tmap_x);
     mbar_arrive_expect_tx(bar_x, (uint32_t)(p.IH * p.Wp * p.w_row_bytes));
-    tma_load_4d(sX, &tmap_x, bar_x, 0, -1, h0 - 2, n);
+    tma_load_4d(sX, &tmap_x, bar_x, 0, -1, SINGLE ? h0 - 1 : h0 - 2, n);
   }
   if (warp == 0) {
     tmem_alloc(tmem_slot, 512);
     tmem_relinquish();
   }
-  if (tid < 2 * p.C) sBias[tid] = tid < p.C ? p.b1[tid] : p.b2[tid - p.C];
+  if (tid < 2 * p.C) sBias[tid] = SINGLE ? (tid >= p.C && p.b2 ? p.b2[tid - p.C] : 0.0f) : (tid < p.C ? p.b1[tid] : p.b2[tid - p.C]);
   tcgen05_fence_before_sync();
   __syncthreads();
   tcgen05_fence_after_sync();
   const uint32_t tmem_base = *tmem_slot;
 
   // The four MMA passes: (convolution, tile group) = (1,A) (1,B) (2,A) (2,B); each streams the 9 taps.
-  const int pass_lo[4] = {0, p.a1, 0, p.a2};
-  const int pass_hi[4] = {p.a1, p.M1, p.a2, p.M2};
+  const int pass_lo[4] = {0, SINGLE ? 0 : p.a1, 0, p.a2};
+  const int pass_hi[4] = {SINGLE ? 0 : p.a1, SINGLE ? 0 : p.M1, p.a2, p.M2};
 
   if (warp == kEpiWarps) {
     // ================================ TMA producer: weight taps ================================
@@ -139,7 +147,7 @@ conv3x3_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
       for (int ps = 0; ps < 4; ++ps) {
         const int conv = ps >> 1, grp = ps & 1;
         uint64_t* done = (conv == 0 ? bar_acc1 : bar_acc2) + grp;
-        if (conv == 1) mbar_wait(bar_y + grp, 0, abort_flag, p.status, 0x403);   // the intermediate rows this group reads are written
+        if (conv == 1 && !SINGLE) mbar_wait(bar_y + grp, 0, abort_flag, p.status, 0x403);   // the intermediate rows this group reads are written
         if (pass_lo[ps] >= pass_hi[ps]) { umma_commit(done); continue; }
         // A: swizzled [pixel][channel] rows; K step = 32 bytes inside a row, 8-row groups are 8 rows apart (SBO).
         // Descriptor arithmetic is hoisted: one add per tile, constant strides per K step.
@@ -190,7 +198,7 @@ conv3x3_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
     // P3: intermediate = ReLU(acc + b1) inside the image, 0 outside -> swizzled rows; group A, then group B
     const uint32_t y_addr = smem_u32(sY);
     const uint32_t swz_mask = ((uint32_t)p.w_row_bytes >> 4) - 1u;
-    for (int grp = 0; grp < 2; ++grp) {
+    for (int grp = 0; grp < (SINGLE ? 0 : 2); ++grp) {
       mbar_wait(bar_acc1 + grp, 0, abort_flag, p.status, 0x405);
       tcgen05_fence_after_sync();
       for (int mt = pass_lo[grp]; mt < pass_hi[grp] && has_cols; ++mt) {
@@ -244,11 +252,16 @@ conv3x3_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
         const int r = m / p.Wp, cc = m - r * p.Wp;
         const bool valid = tile_ok && has_cols && r < rows_valid && cc >= 1 && cc <= p.W;
         const size_t pix = ((size_t)n * p.H + h0 + r) * p.W + (cc - 1);
+        const bool do_res = SINGLE ? p.residual != 0 : true, do_relu = SINGLE ? p.relu != 0 : true;
         uint4 xr[4];
-        if (valid) {
+        if (SINGLE) {
+#pragma unroll
+          for (int j = 0; j < 4; ++j) xr[j] = make_uint4(0u, 0u, 0u, 0u);
+        }
+        if (valid && do_res) {
 #pragma unroll
           for (int j = 0; j < 4; ++j)
-            if (j * 8 < ncol) xr[j] = __ldg(reinterpret_cast<const uint4*>(p.x + pix * p.C + col0 + j * 8));
+            if (j * 8 < ncol) xr[j] = __ldg(reinterpret_cast<const uint4*>((SINGLE ? p.res : p.x) + pix * p.C + col0 + j * 8));
         }
         if (mt == pass_lo[2 + grp]) {
           mbar_wait(bar_acc2 + grp, 0, abort_flag, p.status, 0x406);
@@ -265,8 +278,9 @@ conv3x3_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
               uint32_t w[8];
 #pragma unroll
               for (int j = 0; j < 8; ++j) {
-                const float y0 = fmaxf(__uint_as_float(v[2 * j]) + sB2[c0 + 2 * j] + bf16_lo(xs[j]), 0.0f);
-                const float y1 = fmaxf(__uint_as_float(v[2 * j + 1]) + sB2[c0 + 2 * j + 1] + bf16_hi(xs[j]), 0.0f);
+                float y0 = __uint_as_float(v[2 * j]) + sB2[c0 + 2 * j] + bf16_lo(xs[j]);      // xs is zero without a residual
+                float y1 = __uint_as_float(v[2 * j + 1]) + sB2[c0 + 2 * j + 1] + bf16_hi(xs[j]);
+                if (do_relu) { y0 = fmaxf(y0, 0.0f); y1 = fmaxf(y1, 0.0f); }
                 w[j] = pack_bf16x2(y0, y1);
               }
               if (stage) {
@@ -399,6 +413,7 @@ ago_status_t conv3x3_run(const Plan& plan, FusedState* st, const void* const* in
   q.b2 = static_cast<const float*>(weights[3]);
   q.out = static_cast<__nv_bfloat16*>(output);
   q.status = status_word;
+  q.res = q.x; q.residual = 1; q.relu = 1;
   auto get_map = [&](const void* base, int which, CUtensorMap* out) -> bool {
     ConvHost::Key key{base, which};
     auto it = host->maps.find(key);
@@ -425,13 +440,123 @@ ago_status_t conv3x3_run(const Plan& plan, FusedState* st, const void* const* in
   if (!get_map(inputs[0], 0, &mx) || !get_map(weights[0], 1, &mw1) || !get_map(weights[2], 2, &mw2)) return AGO_ERR_CUDA;
   {
     static int smem_opt_in[64] = {};
-    cudaError_t e = ensure_max_dynamic_smem(reinterpret_cast<const void*>(conv3x3_pair_kernel), smem_opt_in);
+    cudaError_t e = ensure_max_dynamic_smem(reinterpret_cast<const void*>(conv3x3_pair_kernel<false>), smem_opt_in);
     if (e != cudaSuccess) { *err = std::string("cudaFuncSetAttribute: ") + cudaGetErrorString(e); return AGO_ERR_CUDA; }
   }
   FusedLaunch launch(dim3((unsigned)(q.N * q.strips)), kThreads, (size_t)host->smem_bytes, stream);
-  cudaError_t e = cudaLaunchKernelEx(&launch.config, conv3x3_pair_kernel, mx, mw1, mw2, q);
+  cudaError_t e = cudaLaunchKernelEx(&launch.config, conv3x3_pair_kernel<false>, mx, mw1, mw2, q);
   if (e != cudaSuccess) { *err = std::string("fused conv3x3 pair launch: ") + cudaGetErrorString(e); return AGO_ERR_CUDA; }
   return AGO_OK;
+}
+
+// ---- one convolution on the same kernel: the tensor-core stage of the unfused modes ------------------
+
+namespace {
+
+bool conv_layout_single(ConvParams& q, int R, int* smem_bytes) {
+  q.R = R;
+  q.strips = (q.H + R - 1) / R;
+  q.IH = R + 2;
+  q.Wp = q.W + 2;
+  q.P1 = 0; q.M1 = 0;
+  q.P2 = R * q.Wp; q.M2 = (q.P2 + 127) / 128;
+  if (q.IH > 256 || q.Wp > 256 || q.M2 * q.C > 512) return false;
+  int off = 1024;
+  q.off_x = off;
+  q.off_y = off;            // the convolution reads the input rows themselves
+  const int reach_px = std::max(q.M2 * 128 + 2 * q.Wp + 2, q.IH * q.Wp);
+  const int x_reach = reach_px * q.w_row_bytes;
+  off = round_up_i(off + x_reach, 1024);
+  q.off_w = off;
+  q.wstages = kMaxWStages;
+  while (q.wstages > 2 && off + q.wstages * 3 * q.w_stage_bytes + 2048 + 1024 > 227 * 1024) --q.wstages;
+  off += q.wstages * 3 * q.w_stage_bytes;
+  q.off_bias = off;
+  off += 1024;
+  q.off_bar = off;
+  off += 256;
+  q.a1 = 0;
+  q.a2 = (q.M2 + 1) / 2;
+  const bool overlap = q.a2 > 0 && q.a2 < q.M2;
+  const long free_bytes = overlap ? (long)(q.a2 * 128 - q.Wp - 1) * q.w_row_bytes : (long)x_reach;
+  q.stage_ok = free_bytes >= kEpiWarps * 2048 ? 1 : 0;
+  *smem_bytes = off + 1024;
+  return *smem_bytes <= 227 * 1024;
+}
+
+struct SingleKey {
+  const void *x, *w; int N, H, W, C;
+  bool operator==(const SingleKey& o) const { return x == o.x && w == o.w && N == o.N && H == o.H && W == o.W && C == o.C; }
+};
+struct SingleKeyHash {
+  size_t operator()(const SingleKey& k) const {
+    return std::hash<const void*>()(k.x) ^ (std::hash<const void*>()(k.w) * 31u) ^ ((size_t)k.N << 40) ^ ((size_t)k.H << 24) ^ ((size_t)k.W << 8) ^ (size_t)k.C;
+  }
+};
+struct SingleEntry { ConvParams prm; int smem_bytes; CUtensorMap mx, mw; };
+std::mutex g_single_mutex;
+std::unordered_map<SingleKey, SingleEntry, SingleKeyHash> g_single;
+
+}  // namespace
+
+bool conv3x3_tc_supported(int H, int W, int Cin, int Cout, int R, int S, int stride, int pad) {
+  if (R != 3 || S != 3 || stride != 1 || pad != 1 || Cin != Cout) return false;
+  if (Cin != 16 && Cin != 32 && Cin != 64) return false;
+  return H >= 1 && W + 2 <= 256;
+}
+
+cudaError_t launch_conv3x3_tc(const void* x, const void* w, const float* bias, const void* res, void* out, int N, int H,
+                              int W, int C, int relu, cudaStream_t stream) {
+  SingleEntry entry;
+  {
+    std::lock_guard<std::mutex> lock(g_single_mutex);
+    const SingleKey key{x, w, N, H, W, C};
+    auto it = g_single.find(key);
+    if (it == g_single.end()) {
+      SingleEntry e{};
+      ConvParams& q = e.prm;
+      q.N = N; q.H = H; q.W = W; q.C = C;
+      q.w_row_bytes = C * 2;
+      q.w_swizzle = C == 16 ? tc::SW_32B : (C == 32 ? tc::SW_64B : tc::SW_128B);
+      q.w_stage_bytes = round_up_i(C * q.w_row_bytes, 1024);
+      int best_R = 0, best_smem = 0; double best_cost = 0;
+      for (int R = 1; R <= H; ++R) {
+        ConvParams t = q; int smem = 0;
+        if (!conv_layout_single(t, R, &smem)) continue;
+        const long waves = ((long)N * t.strips + 147) / 148;
+        const double cost = (double)waves * (t.M2 + 1.0);
+        if (best_R == 0 || cost < best_cost) { best_R = R; best_cost = cost; best_smem = smem; }
+      }
+      if (best_R == 0) return cudaErrorInvalidConfiguration;
+      conv_layout_single(q, best_R, &best_smem);
+      e.smem_bytes = best_smem;
+      std::string err;
+      const uint64_t xd[4] = {(uint64_t)C, (uint64_t)W, (uint64_t)H, (uint64_t)N};
+      const uint64_t xs[3] = {(uint64_t)C * 2, (uint64_t)W * C * 2, (uint64_t)H * W * C * 2};
+      const uint32_t xb[4] = {(uint32_t)C, (uint32_t)q.Wp, (uint32_t)q.IH, 1};
+      if (!encode_tmap_bf16(&e.mx, x, 4, xd, xs, xb, q.w_row_bytes, &err)) return cudaErrorInvalidValue;
+      const uint64_t wd[3] = {(uint64_t)C, 9, (uint64_t)C};
+      const uint64_t ws[2] = {(uint64_t)C * 2, (uint64_t)9 * C * 2};
+      const uint32_t wb[3] = {(uint32_t)C, 1, (uint32_t)C};
+      if (!encode_tmap_bf16(&e.mw, w, 3, wd, ws, wb, q.w_row_bytes, &err)) return cudaErrorInvalidValue;
+      if (g_single.size() > 4096) g_single.clear();
+      it = g_single.emplace(key, e).first;
+    }
+    entry = it->second;
+  }
+  ConvParams q = entry.prm;
+  q.x = static_cast<const __nv_bfloat16*>(x);
+  q.b1 = nullptr; q.b2 = bias;
+  q.res = static_cast<const __nv_bfloat16*>(res); q.residual = res != nullptr; q.relu = relu;
+  q.out = static_cast<__nv_bfloat16*>(out);
+  q.status = nullptr;
+  {
+    static int smem_opt_in[64] = {};
+    cudaError_t e = ensure_max_dynamic_smem(reinterpret_cast<const void*>(conv3x3_pair_kernel<true>), smem_opt_in);
+    if (e != cudaSuccess) return e;
+  }
+  conv3x3_pair_kernel<true><<<q.N * q.strips, kThreads, entry.smem_bytes, stream>>>(entry.mx, entry.mw, entry.mw, q);
+  return cudaGetLastError();
 }
 
 }  // namespace ago

@@ -52,6 +52,12 @@ cudaError_t launch_elementwise(const void* x, void* y, int64_t numel, int C, int
 cudaError_t launch_softmax_rows(const void* x, void* y, int64_t rows, int cols, int x_dtype, int y_dtype,
                                 cudaStream_t stream);
 
+// 3x3 stride-1 pad-1 convolution with equal channel counts (16, 32 or 64) on tensor cores: the fused pair's kernel
+// restricted to one convolution. out = [relu](conv(x, w) + bias [+ res]); bf16 NHWC / OHWI, bias and res may be null.
+bool conv3x3_tc_supported(int H, int W, int Cin, int Cout, int R, int S, int stride, int pad);
+cudaError_t launch_conv3x3_tc(const void* x, const void* w, const float* bias, const void* res, void* out, int N, int H,
+                              int W, int C, int relu, cudaStream_t stream);
+
 // ---- fused kernels -------------------------------------------------------------
 
 // Depthwise-only mini-subgraph tuned kernel (vectorised over channels).

@@ -80,6 +80,27 @@ def test_depthwise_bf16_fused_mini_subgraph(ago, stride):
     assert_close(run_gpu(ago, wl, data, "fused"), ref, what="dw fused")
 
 
+@pytest.mark.parametrize("tail", ["bias_relu", "bias", "none", "relu", "bias_add_relu"])
+@pytest.mark.parametrize("shape", [(2, 23, 17, 16), (1, 40, 56, 64), (3, 9, 30, 32)])
+def test_single_conv3x3_stage_epilogues(ago, shape, tail):
+    # one 3x3 convolution of equal width with each simple-operator tail the tensor-core stage kernel accepts,
+    # on images of several strips with ragged last strips and non-square extents
+    ch = shape[3]
+    ops = [("conv2d", dict(O=ch, R=3, S=3, stride=1, pad=1, groups=1))]
+    for t in tail.split("_"):
+        if t == "bias":
+            ops.append(("bias_add", {}))
+        elif t == "add":
+            ops.append(("add_input", dict(input=0)))
+        elif t == "relu":
+            ops.append(("relu", {}))
+    wl = WL.Workload("conv1", [71, ch, len(ops)], [shape], ops, samples=shape[0])
+    data = WL.generate(wl)
+    ref = O.run_chain(wl.ops, data["inputs"], data["weights"])
+    for mode in UNFUSED:
+        assert_close(run_gpu(ago, wl, data, mode), ref, what=f"conv1 {shape} {tail}/{mode}")
+
+
 def test_padding_of_the_intermediate_with_large_bias(ago):
     # the halo of the depthwise / second conv input is zero, not act(bias)
     wl = WL.mbv2_block("pad", [33], 1, 6, 8, 16, 8, 1, True)
