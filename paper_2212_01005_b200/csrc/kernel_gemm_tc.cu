@@ -1,8 +1,8 @@
 // Tensor-core GEMM of the unfused modes: C[M][N] = epilogue(A[M][K] * B), one launch per complex
 // operator with its simple operators applied in the epilogue (Section III-A, "Conventional fusion
 // within a mini-subgraph"). It serves the 1x1 convolutions (B = [N][K], K-major) and the GEMM
-// operator (B = [K][N], N-major) whenever the operands are bf16; everything else stays on the
-// generic CUDA-core kernel. The point of this kernel is an honest baseline for the fused kernels:
+// operator (B = [K][N], N-major) and the batched per-head products of attention whenever the operands
+// are bf16; everything else stays on the generic CUDA-core kernel. The point of this kernel is an honest baseline for the fused kernels:
 // the intermediate tensors still travel through device memory, but the contraction itself runs on
 // tcgen05 like theirs.
 //
@@ -38,6 +38,8 @@ struct GemmTcParams {
   int b_kmajor;
   int c_dtype, add_dtype;
   int kblocks, stages;
+  int heads;               // blockIdx.z = batch * heads + head
+  int64_t c_sb, c_sh;      // element offsets of a batch / head in C (and in the EPI_ADD operand)
   int bar_off;             // shared-memory offset of the barriers: after the ring and after the epilogue's staging tile
   // the simple operators in canonical order: + bias, activation 1, * scale, + tensor, activation 2
   const float* bias;       // or null
@@ -72,6 +74,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int row0 = blockIdx.x * kBM, n0 = blockIdx.y * kBN;
+  const int zb = blockIdx.z / p.heads, zh = blockIdx.z - zb * p.heads;
   const int ncols = min(kBN, (p.N - n0 + 15) & ~15);   // MMA N of this tile (multiple of 16)
 
   if (tid == kEpiThreads) {
@@ -100,12 +103,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
         if (i >= kStages) mbar_wait(bar_empty + s, (uint32_t)((i / kStages) - 1) & 1u, abort_flag, nullptr, 0x501);
         uint8_t* st = sRing + s * kStageBytes;
         mbar_arrive_expect_tx(bar_full + s, kStageBytes);
-        tma_load_2d(st, &tmap_a, bar_full + s, i * kBK, row0);                  // A [128 rows x 64 k]
+        tma_load_4d(st, &tmap_a, bar_full + s, i * kBK, row0, zh, zb);          // A [128 rows x 64 k]
         if (p.b_kmajor) {
-          tma_load_2d(st + 16384, &tmap_b, bar_full + s, i * kBK, n0);          // B [128 n x 64 k]
+          tma_load_4d(st + 16384, &tmap_b, bar_full + s, i * kBK, n0, zh, zb);  // B [128 n x 64 k]
         } else {
-          tma_load_2d(st + 16384, &tmap_b, bar_full + s, n0, i * kBK);          // B [64 k x 64 n], twice
-          tma_load_2d(st + 16384 + 8192, &tmap_b, bar_full + s, n0 + 64, i * kBK);
+          tma_load_4d(st + 16384, &tmap_b, bar_full + s, n0, i * kBK, zh, zb);  // B [64 k x 64 n], twice
+          tma_load_4d(st + 16384 + 8192, &tmap_b, bar_full + s, n0 + 64, i * kBK, zh, zb);
         }
       }
     }
@@ -162,7 +165,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
 #pragma unroll
       for (int j = 0; j < 16; ++j) y[j] = (gelu1 ? gelu_tanh_f(y[j]) : activate(y[j], p.act1)) * p.scale;
       if (p.add && row0 + r < p.M) {
-        const int64_t idx = (int64_t)(row0 + r) * p.ldc + col;
+        const int64_t idx = zb * p.c_sb + zh * p.c_sh + (int64_t)(row0 + r) * p.ldc + col;
 #pragma unroll
         for (int h = 0; h < 2; ++h) {
           if (h * 8 < nv) {
@@ -194,7 +197,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
     // consecutive threads store consecutive 16-byte chunks of a row
     const int chunks = ncv * esz / 16;
     const int rows_here = min(kBM, p.M - row0);
-    uint8_t* cbase = reinterpret_cast<uint8_t*>(p.C) + ((int64_t)row0 * p.ldc + n0) * esz;
+    uint8_t* cbase = reinterpret_cast<uint8_t*>(p.C) + (zb * p.c_sb + zh * p.c_sh + (int64_t)row0 * p.ldc + n0) * esz;
     for (int i = tid; i < rows_here * chunks; i += kEpiThreads) {
       const int rr = i / chunks, ch = i - rr * chunks;
       *reinterpret_cast<uint4*>(cbase + (int64_t)rr * p.ldc * esz + ch * 16) = *reinterpret_cast<const uint4*>(stage + rr * pitch + ch * 16);
@@ -206,29 +209,33 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
 }
 
 struct MapKey {
-  const void* p; int d0, d1, b0, b1;
-  bool operator==(const MapKey& o) const { return p == o.p && d0 == o.d0 && d1 == o.d1 && b0 == o.b0 && b1 == o.b1; }
+  const void* p; int d0, d1, d2, d3, b0, b1; int64_t ld, sh, sb;
+  bool operator==(const MapKey& o) const {
+    return p == o.p && d0 == o.d0 && d1 == o.d1 && d2 == o.d2 && d3 == o.d3 && b0 == o.b0 && b1 == o.b1 && ld == o.ld && sh == o.sh && sb == o.sb;
+  }
 };
 struct MapKeyHash {
   size_t operator()(const MapKey& k) const {
-    return std::hash<const void*>()(k.p) ^ ((size_t)k.d0 * 1000003u) ^ ((size_t)k.d1 * 10007u) ^ ((size_t)k.b0 << 7) ^ (size_t)k.b1;
+    return std::hash<const void*>()(k.p) ^ ((size_t)k.d0 * 1000003u) ^ ((size_t)k.d1 * 10007u) ^ ((size_t)k.d2 * 131u) ^ ((size_t)k.d3 * 31u) ^
+           ((size_t)k.b0 << 7) ^ (size_t)k.b1 ^ ((size_t)k.ld << 20) ^ ((size_t)k.sh << 3) ^ ((size_t)k.sb << 11);
   }
 };
 std::mutex g_map_mutex;
 std::unordered_map<MapKey, CUtensorMap, MapKeyHash> g_maps;
 
-// 2-d bf16 tensor [d1 rows][d0 columns] contiguous, box [b1][b0], 128-byte swizzle
-bool get_map(const void* base, int d0, int d1, int b0, int b1, CUtensorMap* out) {
+// bf16 matrices [d1 rows][d0 columns] with leading dimension ld, d2 heads sh elements apart in each of d3 batches
+// sb elements apart; box [b1][b0] of one matrix, 128-byte swizzle
+bool get_map(const void* base, int d0, int d1, int d2, int d3, int64_t ld, int64_t sh, int64_t sb, int b0, int b1, CUtensorMap* out) {
   std::lock_guard<std::mutex> lock(g_map_mutex);
-  const MapKey key{base, d0, d1, b0, b1};
+  const MapKey key{base, d0, d1, d2, d3, b0, b1, ld, sh, sb};
   auto it = g_maps.find(key);
   if (it == g_maps.end()) {
     CUtensorMap m;
-    const uint64_t dims[2] = {(uint64_t)d0, (uint64_t)d1};
-    const uint64_t strides[1] = {(uint64_t)d0 * 2};
-    const uint32_t box[2] = {(uint32_t)b0, (uint32_t)b1};
+    const uint64_t dims[4] = {(uint64_t)d0, (uint64_t)d1, (uint64_t)d2, (uint64_t)d3};
+    const uint64_t strides[3] = {(uint64_t)ld * 2, (uint64_t)sh * 2, (uint64_t)sb * 2};
+    const uint32_t box[4] = {(uint32_t)b0, (uint32_t)b1, 1, 1};
     std::string err;
-    if (!encode_tmap_bf16(&m, base, 2, dims, strides, box, 128, &err)) return false;
+    if (!encode_tmap_bf16(&m, base, 4, dims, strides, box, 128, &err)) return false;
     if (g_maps.size() > 4096) g_maps.clear();
     it = g_maps.emplace(key, m).first;
   }
@@ -258,22 +265,34 @@ static bool canonical_epilogue(const EpiProgram& e, GemmTcParams* p) {
 bool gemm_tc_supported(const GemmArgs& a) {
   GemmTcParams probe{};
   if (!canonical_epilogue(a.epi, &probe)) return false;
-  if (a.a_dtype != AGO_BF16 || a.batches != 1) return false;
+  if (a.a_dtype != AGO_BF16) return false;
   if (a.a_im2col && !(a.R == 1 && a.S == 1 && a.stride == 1 && a.pad == 0)) return false;
-  if (!a.a_im2col && a.lda != a.K) return false;
-  if (a.K % 8 != 0 || a.N % 8 != 0 || a.ldc != a.N) return false;
-  if (a.b_kmajor ? a.ldb != a.K : a.ldb != a.N) return false;
+  if (a.K % 8 != 0 || a.N % 8 != 0) return false;
+  // 16-byte rows, heads and batches for TMA and for the vector stores
+  const int heads = std::max(a.heads, 1);
+  if (!a.a_im2col && a.lda % 8 != 0) return false;
+  if (a.ldb % 8 != 0 || a.ldc % 8 != 0) return false;
+  if (a.batches > 1 && (a.a_sb % 8 || a.a_sh % 8 || a.b_sb % 8 || a.b_sh % 8 || a.c_sb % 8 || a.c_sh % 8)) return false;
+  if (a.batches > 65535 || a.batches % heads != 0) return false;
   return true;
 }
 
 cudaError_t launch_gemm_tc(const GemmArgs& a, int add_dtype, cudaStream_t stream) {
   CUtensorMap ma, mb;
-  if (!get_map(a.A, a.K, a.M, kBK, kBM, &ma)) return cudaErrorInvalidValue;
-  if (a.b_kmajor ? !get_map(a.B, a.K, a.N, kBK, kBN, &mb) : !get_map(a.B, a.N, a.K, 64, kBK, &mb)) return cudaErrorInvalidValue;
+  const int heads = a.batches > 1 ? std::max(a.heads, 1) : 1, nb = std::max(a.batches, 1) / heads;
+  const int64_t lda = a.a_im2col ? a.K : a.lda;
+  // unbatched operands: the outer two dimensions have extent 1, their strides only need to be legal
+  const int64_t a_sh = a.batches > 1 ? a.a_sh : lda * a.M, a_sb = a.batches > 1 ? a.a_sb : lda * a.M;
+  const int64_t b_rows = a.b_kmajor ? a.N : a.K;
+  const int64_t b_sh = a.batches > 1 ? a.b_sh : a.ldb * b_rows, b_sb = a.batches > 1 ? a.b_sb : a.ldb * b_rows;
+  if (!get_map(a.A, a.K, a.M, heads, nb, lda, a_sh, a_sb, kBK, kBM, &ma)) return cudaErrorInvalidValue;
+  if (a.b_kmajor ? !get_map(a.B, a.K, a.N, heads, nb, a.ldb, b_sh, b_sb, kBK, kBN, &mb)
+                 : !get_map(a.B, a.N, a.K, heads, nb, a.ldb, b_sh, b_sb, 64, kBK, &mb)) return cudaErrorInvalidValue;
   GemmTcParams p{};
   p.C = a.C; p.M = a.M; p.N = a.N; p.K = a.K; p.ldc = a.ldc; p.b_kmajor = a.b_kmajor;
   p.c_dtype = a.c_dtype; p.add_dtype = add_dtype;
   p.kblocks = (a.K + kBK - 1) / kBK;
+  p.heads = heads; p.c_sb = a.batches > 1 ? a.c_sb : 0; p.c_sh = a.batches > 1 ? a.c_sh : 0;
   canonical_epilogue(a.epi, &p);
   p.stages = std::min(kMaxStages, p.kblocks);
   // the epilogue stages the output tile (128 rows x (columns x element size + 16) bytes) over the idle ring
@@ -288,7 +307,7 @@ cudaError_t launch_gemm_tc(const GemmArgs& a, int add_dtype, cudaStream_t stream
   if (e != cudaSuccess) return e;
   if (dev >= 0 && dev < 64)
     std::call_once(once[dev], [&] { cudaFuncSetAttribute(gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_max); });
-  dim3 grid((a.M + kBM - 1) / kBM, (a.N + kBN - 1) / kBN);
+  dim3 grid((a.M + kBM - 1) / kBM, (a.N + kBN - 1) / kBN, heads * nb);
   gemm_tc_kernel<<<grid, kThreads, smem, stream>>>(ma, mb, p);
   return cudaGetLastError();
 }

@@ -29,8 +29,8 @@ struct GemmArgs {
 };
 cudaError_t launch_gemm_generic(const GemmArgs& a, cudaStream_t stream);
 
-// The same contraction on tcgen05 for the shapes it serves (bf16 A, plain [M][K] view, K and N multiples of 8,
-// no batching); `add_dtype` is the storage type of EPI_ADD operands (the subgraph's I/O dtype).
+// The same contraction on tcgen05 for the shapes it serves (bf16 A, plain [M][K] view, K, N, leading dimensions and
+// batch / head strides multiples of 8); `add_dtype` is the storage type of EPI_ADD operands (the subgraph's I/O dtype).
 bool gemm_tc_supported(const GemmArgs& a);
 cudaError_t launch_gemm_tc(const GemmArgs& a, int add_dtype, cudaStream_t stream);
 
