@@ -141,7 +141,12 @@ typedef enum {
   AGO_KERNEL_MBV2_BLOCK = 2,  /* 1x1 conv -> depthwise 3x3 -> 1x1 conv [+ residual] */
   AGO_KERNEL_FFN = 3,         /* GEMM -> GELU -> GEMM                               */
   AGO_KERNEL_CONV3X3_PAIR = 4,/* conv3x3 -> conv3x3 [+ residual, ReLU]              */
-  AGO_KERNEL_ATTENTION = 5    /* QK^T -> scale -> softmax -> .V                     */
+  AGO_KERNEL_ATTENTION = 5,   /* QK^T -> scale -> softmax -> .V                     */
+  /* the two-complex-operator pairs of the fusion-strategy micro-benchmark (Section VI-B) */
+  AGO_KERNEL_PW_DW = 6,       /* 1x1 conv -> depthwise 3x3                           */
+  AGO_KERNEL_DW_PW = 7,       /* depthwise 3x3 -> 1x1 conv                           */
+  AGO_KERNEL_DW_DW = 8,       /* depthwise 3x3 -> depthwise 3x3                      */
+  AGO_KERNEL_PW_PW = 9        /* 1x1 conv -> 1x1 conv                                */
 } ago_fused_kernel_t;
 
 /* Validate the operator list, infer shapes, classify every complex -> complex

@@ -32,7 +32,7 @@ MODES = {"fused": AGO_MODE_FUSED, "per_mini_subgraph": AGO_MODE_PER_MINI_SUBGRAP
 
 AGO_LINK_DOWNSTREAM_DEPTHWISE, AGO_LINK_DOWNSTREAM_POINTWISE, AGO_LINK_GENERAL = 1, 2, 3
 (AGO_KERNEL_NONE, AGO_KERNEL_DEPTHWISE, AGO_KERNEL_MBV2_BLOCK, AGO_KERNEL_FFN, AGO_KERNEL_CONV3X3_PAIR,
- AGO_KERNEL_ATTENTION) = range(6)
+ AGO_KERNEL_ATTENTION, AGO_KERNEL_PW_DW, AGO_KERNEL_DW_PW, AGO_KERNEL_DW_DW, AGO_KERNEL_PW_PW) = range(10)
 
 AGO_MAX_INPUTS, AGO_MAX_RANK, AGO_MAX_OPS = 4, 4, 32
 AGO_STATIC_SCRATCH_BYTES = 4 << 20

@@ -19,6 +19,8 @@ ago_status_t fused_plan(Plan* plan, FusedState* st, std::string* err) {
     case AGO_KERNEL_DEPTHWISE:
       return AGO_OK;
     case AGO_KERNEL_MBV2_BLOCK:
+    case AGO_KERNEL_PW_DW:
+    case AGO_KERNEL_DW_PW:
       return mbv2_plan(plan, st, err);
     case AGO_KERNEL_ATTENTION:
       return attention_plan(plan, st, err);
@@ -41,6 +43,8 @@ ago_status_t fused_run(const Plan& plan, FusedState* st, const void* const* inpu
                        std::string* err) {
   switch (plan.fused_kernel) {
     case AGO_KERNEL_MBV2_BLOCK:
+    case AGO_KERNEL_PW_DW:
+    case AGO_KERNEL_DW_PW:
       return mbv2_run(plan, st, inputs, weights, output, status_word, stream, err);
     case AGO_KERNEL_ATTENTION:
       return attention_run(plan, st, inputs, weights, output, status_word, stream, err);

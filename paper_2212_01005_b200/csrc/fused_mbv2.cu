@@ -185,6 +185,10 @@ __device__ __forceinline__ void depthwise_block(uint32_t e_row, uint32_t d_row, 
 #undef AGO_DW_STEP
 }
 
+// EXPAND / PROJECT select the pairs of the block: <true, true> the whole block, <true, false> pointwise -> depthwise
+// (the depthwise result of every chunk goes to device memory), <false, true> depthwise -> pointwise (every chunk of
+// the input is copied into the E buffers instead of being computed).
+template <bool EXPAND, bool PROJECT>
 __global__ void __launch_bounds__(kThreads, 1)
 mbv2_fused_kernel(const Mbv2Params p) {
   extern __shared__ uint8_t smem_raw[];
@@ -231,9 +235,10 @@ mbv2_fused_kernel(const Mbv2Params p) {
     // Cin; W3 to one [Coutp x 16 channels] slice per chunk; depthwise weights and biases are copied as they are.
     constexpr int kBX = 4, kBW = 2;   // slots per thread in the first (batched) pass: input strip / everything else
     const int cs = p.Kp == 16 ? 1 : (p.Kp == 32 ? 2 : 3);   // log2(16-byte chunks per tile row)
-    const uint32_t nX = (uint32_t)p.P_x << cs, nW1 = (uint32_t)p.Cexp << cs, nW3 = (uint32_t)(p.NC * p.Coutp * 2);
-    const uint32_t nWd = 9u * p.Cexp / 8u, nB = (uint32_t)p.Cexp / 4u, nB3 = (uint32_t)p.Cout / 4u;
-    const uint32_t nW = nW1 + nW3 + nWd + 2u * nB + nB3;
+    const uint32_t nX = EXPAND ? (uint32_t)p.P_x << cs : 0u, nW1 = EXPAND ? (uint32_t)p.Cexp << cs : 0u;
+    const uint32_t nW3 = PROJECT ? (uint32_t)(p.NC * p.Coutp * 2) : 0u;
+    const uint32_t nWd = 9u * p.Cexp / 8u, nB = (uint32_t)p.Cexp / 4u, nB1 = EXPAND ? nB : 0u, nB3 = PROJECT ? (uint32_t)p.Cout / 4u : 0u;
+    const uint32_t nW = nW1 + nW3 + nWd + nB1 + nB + nB3;
     // tile pixel `pix` is image pixel gh0 * W + pix of image n (strips are full-width rows): in the image for pix in [pix_lo, pix_hi)
     const int pix_lo = max(0, -gh0 * p.W), pix_hi = min(p.P_x, (p.H - gh0) * p.W);
     const uint8_t* x0 = reinterpret_cast<const uint8_t*>(p.x) + ((size_t)n * p.H + gh0) * p.W * p.Cin * 2;   // not dereferenced outside the image
@@ -258,8 +263,8 @@ mbv2_fused_kernel(const Mbv2Params p) {
         return p.off_w3 + c * p.Coutp * kChunkRowBytes + swz_offset(row, half, kChunkRowBytes);
       }
       if ((i -= nW3) < nWd) { src = reinterpret_cast<const uint8_t*>(p.wd) + i * 16u; return p.off_wd + i * 16u; }
-      if ((i -= nWd) < nB) { src = reinterpret_cast<const uint8_t*>(p.b1) + i * 16u; return p.off_b1 + i * 16u; }
-      if ((i -= nB) < nB) { src = reinterpret_cast<const uint8_t*>(p.bd) + i * 16u; return p.off_bd + i * 16u; }
+      if ((i -= nWd) < nB1) { src = reinterpret_cast<const uint8_t*>(p.b1) + i * 16u; return p.off_b1 + i * 16u; }
+      if ((i -= nB1) < nB) { src = reinterpret_cast<const uint8_t*>(p.bd) + i * 16u; return p.off_bd + i * 16u; }
       i -= nB;
       src = reinterpret_cast<const uint8_t*>(p.b3) + i * 16u;
       return p.off_b3 + i * 16u;
@@ -357,8 +362,9 @@ mbv2_fused_kernel(const Mbv2Params p) {
       *reinterpret_cast<uint4*>(smem + d) = load_or_zero(src);
     }
     // the zero padding columns of the two E chunk buffers (written once: every chunk reuses them)
-    for (int i = tid; i < p.IH * 8; i += kThreads) {
-      const int ih = i >> 3, side = (i >> 2) & 1, plane = i & 3;   // 2 buffers x 2 planes
+    constexpr int kEShift = EXPAND ? 2 : 3;   // 2 E buffers x 2 planes, or 4 x 2 when the chunks are copied in (two per group)
+    for (int i = tid; i < p.IH << (kEShift + 1); i += kThreads) {
+      const int ih = i >> (kEShift + 1), side = (i >> kEShift) & 1, plane = i & ((1 << kEShift) - 1);
       *reinterpret_cast<uint4*>(sE + plane * p.e_plane + (ih * p.IW + side * (p.IW - 1)) * 16) = make_uint4(0, 0, 0, 0);
     }
     fence_proxy_async_smem();
@@ -413,17 +419,53 @@ mbv2_fused_kernel(const Mbv2Params p) {
     const uint32_t proj_d_tmem = tmem_base + p.pcol0 + gw * p.Coutp;
     const uint32_t proj_b_step = (uint32_t)(2 * p.Coutp * kChunkRowBytes) >> 4;     // the group's next chunk is c + 2
     uint32_t proj_b_lo = (uint32_t)w3desc0 + ((uint32_t)(g * p.Coutp * kChunkRowBytes) >> 4);
-    if (xi >= 0 && lane == 0 && g < p.NC) issue_expand();
+    if (EXPAND && xi >= 0 && lane == 0 && g < p.NC) issue_expand();
     __syncwarp();
     // Waits on MMA completion are taken by ONE warp of the group, just before it arrives at the group barrier that
     // the others are parked at: a polling warp spends issue slots, sixteen of them a large share of the SM's.
     const bool waiter = gw == kGroupWarps - 1;
-    if (g < p.NC) {
+    if (EXPAND && g < p.NC) {
       if (waiter) mbar_wait(bar_e + g, 0, abort_flag, p.status, 0x102);   // the group's first expand GEMM
       named_barrier_sync(gbar, kGroupThreads);
     }
+    // Without the expand GEMM a chunk is 16 channels of the input strip, copied asynchronously into one of the
+    // group's two E buffers two chunks ahead: 16-byte pieces (pixel, 8-channel plane), rows outside the image
+    // zero-filled. The piece geometry is the same for every chunk.
+    constexpr int kPieces = 4;                      // P_x * 2 pieces <= 8 tiles * 128 * 2 over the group's threads
+    uint32_t ld_src[kPieces], ld_dst[kPieces], ld_ok = 0u, ld_in = 0u;
+    const uint8_t* xin = reinterpret_cast<const uint8_t*>(p.x) + ((int64_t)n * p.H + gh0) * p.W * p.Cexp * 2;   // row gh0 may lie outside
+    if (!EXPAND) {
+#pragma unroll
+      for (int k = 0; k < kPieces; ++k) {
+        const int i = gt + k * kGroupThreads;
+        ld_src[k] = 0u; ld_dst[k] = 0u;
+        if (i < p.P_x * 2) {
+          const int pix = i >> 1, plane = i & 1;
+          const int ih = (int)__umulhi((uint32_t)pix, p.w_recip), iw = pix - ih * p.W;
+          ld_ok |= 1u << k;
+          ld_dst[k] = (uint32_t)(plane * p.e_plane + (ih * p.IW + iw + 1) * 16);
+          if (gh0 + ih >= 0 && gh0 + ih < p.H) { ld_in |= 1u << k; ld_src[k] = (uint32_t)(pix * p.Cexp * 2 + plane * 16); }
+        }
+      }
+    }
+    auto load_chunk = [&](int c, int b) {   // chunk c -> E buffer (g, b); always one commit group
+      if (c < p.NC) {
+        const uint32_t e0 = smem_u32(sE) + (uint32_t)((g * 2 + b) * e_bytes);
+#pragma unroll
+        for (int k = 0; k < kPieces; ++k) {
+          if ((ld_ok >> k) & 1u) {
+            const bool in = (ld_in >> k) & 1u;
+            cp_async_16(e0 + ld_dst[k], in ? xin + ld_src[k] + c * kChunkRowBytes : reinterpret_cast<const uint8_t*>(p.x), in ? 16u : 0u);
+          }
+        }
+      }
+      cp_async_commit();
+    };
+    if (!EXPAND) { load_chunk(g, 0); load_chunk(g + 2, 1); }
     for (int c = g, it = 0; c < p.NC; c += 2, ++it) {
       // ---- P3: expand epilogue of chunk c -> E[g]: + b1, ReLU6, zero outside the image, bf16 ----
+      if (!EXPAND) cp_async_wait_but_one();   // this thread's pieces of chunk c have landed
+      if (EXPAND) {
       tcgen05_fence_after_sync();
       uint8_t* e_buf = sE + g * e_bytes;
 #pragma unroll
@@ -452,10 +494,11 @@ mbv2_fused_kernel(const Mbv2Params p) {
         }
       }
       tcgen05_fence_before_sync();
+      }
       // D[g] was read by the project GEMM of chunk c - 2
-      if (waiter && it >= 1) mbar_wait(bar_d + g, (uint32_t)(it - 1) & 1u, abort_flag, p.status, 0x103);
+      if (PROJECT && waiter && it >= 1) mbar_wait(bar_d + g, (uint32_t)(it - 1) & 1u, abort_flag, p.status, 0x103);
       named_barrier_sync(gbar, kGroupThreads);
-      if (xi >= 0 && c + 2 < p.NC) {   // expand buffer g is drained: the expand GEMM of the group's next chunk
+      if (EXPAND && xi >= 0 && c + 2 < p.NC) {   // expand buffer g is drained: the expand GEMM of the group's next chunk
         if (lane == 0) {
           tcgen05_fence_after_sync();
           issue_expand();
@@ -470,7 +513,7 @@ mbv2_fused_kernel(const Mbv2Params p) {
 #pragma unroll
         for (int tap = 0; tap < 9; ++tap) wgt[tap] = *reinterpret_cast<const uint32_t*>(sWd + (tap * p.Cexp + ch) * 2);
         const float2 bias = *reinterpret_cast<const float2*>(sBd + ch);
-        const uint32_t e_plane = smem_u32(sE) + (uint32_t)(g * e_bytes + (cp >> 2) * p.e_plane + cp_off);
+        const uint32_t e_plane = smem_u32(sE) + (uint32_t)((EXPAND ? g : g * 2 + (it & 1)) * e_bytes + (cp >> 2) * p.e_plane + cp_off);
         const uint32_t d_plane = smem_u32(sD) + (uint32_t)(g * d_bytes + (cp >> 2) * p.d_plane + cp_off);
         int r = item0_r, col = item0_c;
         for (int item = slot; item < dw_items; item += kSlots) {
@@ -488,9 +531,20 @@ mbv2_fused_kernel(const Mbv2Params p) {
       }
       fence_proxy_async_smem();
       // the expand GEMM of the group's next chunk (issued after the previous barrier) is complete
-      if (waiter && c + 2 < p.NC) mbar_wait(bar_e + g, (uint32_t)(it + 1) & 1u, abort_flag, p.status, 0x102);
+      if (EXPAND && waiter && c + 2 < p.NC) mbar_wait(bar_e + g, (uint32_t)(it + 1) & 1u, abort_flag, p.status, 0x102);
       named_barrier_sync(gbar, kGroupThreads);
-      if (gw < p.M2) {   // D[g] is complete: the project GEMM of chunk c, one tile per warp
+      if (!EXPAND) load_chunk(c + 4, it & 1);   // the E buffer of chunk c is free
+      if (!PROJECT) {
+        // the depthwise result of the chunk is the output: 16-byte pieces (pixel, plane) of D[g] to device memory
+        const int pieces = rows_valid * p.Wo * 2;
+        __nv_bfloat16* o0 = p.out + ((size_t)n * p.Ho + ho0) * p.Wo * p.Cexp + c * kChunk;
+        for (int i = gt; i < pieces; i += kGroupThreads) {
+          const int pix = i >> 1, plane = i & 1;
+          *reinterpret_cast<uint4*>(o0 + (size_t)pix * p.Cexp + plane * 8) =
+              *reinterpret_cast<const uint4*>(sD + g * d_bytes + plane * p.d_plane + pix * 16);
+        }
+      }
+      if (PROJECT && gw < p.M2) {   // D[g] is complete: the project GEMM of chunk c, one tile per warp
         if (lane == 0) {
           // chunk 0 overwrites the accumulators: everything else is issued after it
           if (c == 1) mbar_wait(bar_first, 0, abort_flag, p.status, 0x106);
@@ -506,7 +560,7 @@ mbv2_fused_kernel(const Mbv2Params p) {
     }
 
     // ---- P6: project epilogue: + b3 (+ residual), bf16, 16-byte stores ----
-    {
+    if (PROJECT) {
       if (warp == kWarps - 1) mbar_wait(bar_done, 0, abort_flag, p.status, 0x104);
       __syncthreads();
       tcgen05_fence_after_sync();
@@ -527,7 +581,7 @@ mbv2_fused_kernel(const Mbv2Params p) {
 #pragma unroll
                 for (int q = 0; q < 8; ++q) v[q] = __uint_as_float(acc[h * 8 + q]) + sB3[j + q];
                 const size_t off = (gpix0 + po) * p.Cout + j;
-                if (p.residual) {
+                if (EXPAND && p.residual) {
                   // stride 1, Cin == Cout: output pixel po is pixel po + W of the input tile (one halo row above)
                   const uint4 xr = *reinterpret_cast<const uint4*>(sX + swz_offset(po + p.W, j >> 3, p.row_bytes));
                   v[0] += bf16_lo(xr.x); v[1] += bf16_hi(xr.x); v[2] += bf16_lo(xr.y); v[3] += bf16_hi(xr.y);
@@ -551,9 +605,10 @@ int round_up(int v, int m) { return (v + m - 1) / m * m; }
 struct Mbv2Host {
   Mbv2Params prm;
   int smem_bytes = 0;
+  bool expand = true, project = true;
 };
 
-bool layout(Mbv2Params& q, int R, int* smem_bytes) {
+bool layout(Mbv2Params& q, int R, bool expand, bool project, int* smem_bytes) {
   q.R = R;
   q.strips = (q.Ho + R - 1) / R;
   q.strips_recip = (uint32_t)((1ull << 32) / (uint64_t)q.strips + 1ull);
@@ -564,27 +619,27 @@ bool layout(Mbv2Params& q, int R, int* smem_bytes) {
   q.M1 = (q.P_x + 127) / 128;
   q.M2 = (R * q.Wo + 127) / 128;
   if (q.IH > 256 || q.IW > 256 || q.M1 > 8) return false;
-  const int cols = 2 * q.M1 * kChunk + q.M2 * q.Coutp;
+  const int cols = (expand ? 2 * q.M1 * kChunk : 0) + (project ? q.M2 * q.Coutp : 0);
   if (cols > 512) return false;
   q.tmem_cols = 32;
   while (q.tmem_cols < cols) q.tmem_cols *= 2;
   q.ecol0 = 0;
-  q.pcol0 = 2 * q.M1 * kChunk;
+  q.pcol0 = expand ? 2 * q.M1 * kChunk : 0;
   int off = 0;
   auto take = [&](int bytes) { int o = off; off = round_up(off + bytes, 1024); return o; };
-  q.off_x = take(q.M1 * 128 * q.row_bytes);
-  q.off_w1 = take(q.Cexp * q.row_bytes);
+  q.off_x = take(expand ? q.M1 * 128 * q.row_bytes : 0);
+  q.off_w1 = take(expand ? q.Cexp * q.row_bytes : 0);
   // two 8-channel planes per chunk, offset by 64 mod 128 bytes so that a warp's
   // 2 x 64-byte accesses (4 pixels x 4 channel pairs per plane) never share a bank
   q.e_plane = round_up(q.P_in * 16, 128) + 64;
   q.d_plane = q.M2 * 128 * 16 + 64;
-  q.off_e = take(2 * 2 * q.e_plane);   // two chunk buffers
+  q.off_e = take((expand ? 2 : 4) * 2 * q.e_plane);   // one chunk buffer per group, two when the chunks are copied in
   q.off_d = take(2 * 2 * q.d_plane);
-  q.off_w3 = take(q.NC * q.Coutp * kChunkRowBytes);
+  q.off_w3 = take(project ? q.NC * q.Coutp * kChunkRowBytes : 0);
   q.off_wd = take(9 * q.Cexp * 2);
-  q.off_b1 = take(q.Cexp * 4);
+  q.off_b1 = take(expand ? q.Cexp * 4 : 0);
   q.off_bd = take(q.Cexp * 4);
-  q.off_b3 = take(q.Coutp * 4);
+  q.off_b3 = take(project ? q.Coutp * 4 : 0);
   q.off_bar = take(128);
   *smem_bytes = off + 1024;  // slack for the 1024-byte alignment of the base
   return *smem_bytes <= 227 * 1024;
@@ -593,16 +648,22 @@ bool layout(Mbv2Params& q, int R, int* smem_bytes) {
 }  // namespace
 
 ago_status_t mbv2_plan(Plan* plan, FusedState* st, std::string* err) {
-  const OpInfo& e = plan->ops[0];
-  const OpInfo& d = plan->ops[3];
-  const OpInfo& pr = plan->ops[6];
+  // operator indices of the three convolutions in the chain (-1: the pair has none)
+  const bool expand = plan->fused_kernel != AGO_KERNEL_DW_PW, project = plan->fused_kernel != AGO_KERNEL_PW_DW;
+  const int i_dw = expand ? 3 : 0, i_pr = expand ? 6 : 3;
+  const OpInfo& first = plan->ops[0];
+  const OpInfo& d = plan->ops[i_dw];
   auto* host = new Mbv2Host();
+  host->expand = expand; host->project = project;
   Mbv2Params& q = host->prm;
   q = Mbv2Params{};
-  q.N = (int)e.in.d[0]; q.H = (int)e.in.d[1]; q.W = (int)e.in.d[2]; q.Cin = (int)e.in.d[3];
-  q.Cexp = e.op.p[0]; q.Cout = pr.op.p[0]; q.stride = d.op.p[3];
+  q.N = (int)first.in.d[0]; q.H = (int)first.in.d[1]; q.W = (int)first.in.d[2];
+  q.Cexp = (int)d.in.d[3];
+  q.Cin = expand ? (int)first.in.d[3] : 16;
+  q.Cout = project ? plan->ops[i_pr].op.p[0] : 16;
+  q.stride = d.op.p[3];
   q.Ho = (int)d.out.d[1]; q.Wo = (int)d.out.d[2];
-  q.residual = plan->ops.size() == 9 ? 1 : 0;
+  q.residual = plan->fused_kernel == AGO_KERNEL_MBV2_BLOCK && plan->ops.size() == 9 ? 1 : 0;
   auto bad = [&](const char* m) { *err = std::string("fused inverted-residual block: ") + m; delete host; return AGO_ERR_UNSUPPORTED; };
   if (q.Cin > 64) return bad("more than 64 input channels is not supported yet");
   if (q.Cexp % kChunk != 0) return bad("expanded channels must be a multiple of 16");
@@ -629,14 +690,14 @@ ago_status_t mbv2_plan(Plan* plan, FusedState* st, std::string* err) {
   const int sms = 148;
   for (int R = 1; R <= q.Ho; ++R) {
     Mbv2Params t = q; int smem = 0;
-    if (!layout(t, R, &smem)) continue;
+    if (!layout(t, R, expand, project, &smem)) continue;
     const long ctas = (long)q.N * t.strips;
     const long waves = (ctas + sms - 1) / sms;
     const double cost = (double)waves * (t.M1 * 128.0 + 3.0 * t.M2 * 128.0 + 200.0);
     if (best_R == 0 || cost < best_cost) { best_R = R; best_cost = cost; best_smem = smem; }
   }
   if (best_R == 0) return bad("no row-strip tiling fits shared memory / tensor memory");
-  layout(q, best_R, &best_smem);
+  layout(q, best_R, expand, project, &best_smem);
   host->smem_bytes = best_smem;
   st->impl = host;
   st->impl_free = [](void* p) { delete static_cast<Mbv2Host*>(p); };
@@ -645,25 +706,35 @@ ago_status_t mbv2_plan(Plan* plan, FusedState* st, std::string* err) {
   return AGO_OK;
 }
 
+namespace {
+
+template <bool EXPAND, bool PROJECT>
+ago_status_t launch_variant(const Mbv2Params& q, int smem_bytes, cudaStream_t stream, std::string* err) {
+  static int smem_opt_in[64] = {};
+  cudaError_t e = ensure_max_dynamic_smem(reinterpret_cast<const void*>(mbv2_fused_kernel<EXPAND, PROJECT>), smem_opt_in);
+  if (e != cudaSuccess) { *err = std::string("cudaFuncSetAttribute: ") + cudaGetErrorString(e); return AGO_ERR_CUDA; }
+  FusedLaunch launch(dim3((unsigned)(q.N * q.strips)), kThreads, (size_t)smem_bytes, stream);
+  e = cudaLaunchKernelEx(&launch.config, mbv2_fused_kernel<EXPAND, PROJECT>, q);
+  if (e != cudaSuccess) { *err = std::string("fused inverted-residual launch: ") + cudaGetErrorString(e); return AGO_ERR_CUDA; }
+  return AGO_OK;
+}
+
+}  // namespace
+
 ago_status_t mbv2_run(const Plan& plan, FusedState* st, const void* const* inputs, const void* const* weights,
                       void* output, unsigned int* status_word, cudaStream_t stream, std::string* err) {
   Mbv2Host* host = static_cast<Mbv2Host*>(st->impl);
   Mbv2Params q = host->prm;
   q.x = static_cast<const __nv_bfloat16*>(inputs[0]);
-  q.w1 = static_cast<const __nv_bfloat16*>(weights[0]); q.b1 = static_cast<const float*>(weights[1]);
-  q.wd = static_cast<const __nv_bfloat16*>(weights[2]); q.bd = static_cast<const float*>(weights[3]);
-  q.w3 = static_cast<const __nv_bfloat16*>(weights[4]); q.b3 = static_cast<const float*>(weights[5]);
+  int w = 0;   // weights in chain order: (w1, b1) (wd, bd) (w3, b3), without the pair's missing convolution
+  if (host->expand) { q.w1 = static_cast<const __nv_bfloat16*>(weights[w]); q.b1 = static_cast<const float*>(weights[w + 1]); w += 2; }
+  q.wd = static_cast<const __nv_bfloat16*>(weights[w]); q.bd = static_cast<const float*>(weights[w + 1]); w += 2;
+  if (host->project) { q.w3 = static_cast<const __nv_bfloat16*>(weights[w]); q.b3 = static_cast<const float*>(weights[w + 1]); }
   q.out = static_cast<__nv_bfloat16*>(output);
   q.status = status_word;
-  {
-    static int smem_opt_in[64] = {};
-    cudaError_t e = ensure_max_dynamic_smem(reinterpret_cast<const void*>(mbv2_fused_kernel), smem_opt_in);
-    if (e != cudaSuccess) { *err = std::string("cudaFuncSetAttribute: ") + cudaGetErrorString(e); return AGO_ERR_CUDA; }
-  }
-  FusedLaunch launch(dim3((unsigned)(q.N * q.strips)), kThreads, (size_t)host->smem_bytes, stream);
-  cudaError_t e = cudaLaunchKernelEx(&launch.config, mbv2_fused_kernel, q);
-  if (e != cudaSuccess) { *err = std::string("fused inverted-residual launch: ") + cudaGetErrorString(e); return AGO_ERR_CUDA; }
-  return AGO_OK;
+  if (!host->expand) return launch_variant<false, true>(q, host->smem_bytes, stream, err);
+  if (!host->project) return launch_variant<true, false>(q, host->smem_bytes, stream, err);
+  return launch_variant<true, true>(q, host->smem_bytes, stream, err);
 }
 
 }  // namespace ago

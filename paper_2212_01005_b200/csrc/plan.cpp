@@ -75,6 +75,22 @@ int match_fused_family(const Plan& p) {
       if (ok) return AGO_KERNEL_MBV2_BLOCK;
     }
   }
+  // the two-complex-operator pairs of the micro-benchmark (Section VI-B), each convolution with bias (+ ReLU6)
+  {
+    auto dw3x3 = [](const OpInfo& o) {
+      return o.depthwise() && o.op.p[1] == 3 && o.op.p[2] == 3 && o.op.p[4] == 1 && (o.op.p[3] == 1 || o.op.p[3] == 2);
+    };
+    if (kinds_are(ops, {AGO_OP_CONV2D, AGO_OP_BIAS_ADD, AGO_OP_RELU6, AGO_OP_CONV2D, AGO_OP_BIAS_ADD, AGO_OP_RELU6})) {
+      if (ops[0].pointwise() && dw3x3(ops[3])) return AGO_KERNEL_PW_DW;
+      if (dw3x3(ops[0]) && dw3x3(ops[3]) && ops[0].op.p[3] == 1 && ops[3].op.p[3] == 1) return AGO_KERNEL_DW_DW;
+    }
+    if (kinds_are(ops, {AGO_OP_CONV2D, AGO_OP_BIAS_ADD, AGO_OP_RELU6, AGO_OP_CONV2D, AGO_OP_BIAS_ADD}) && dw3x3(ops[0]) &&
+        ops[3].pointwise())
+      return AGO_KERNEL_DW_PW;
+    if (kinds_are(ops, {AGO_OP_CONV2D, AGO_OP_BIAS_ADD, AGO_OP_CONV2D, AGO_OP_BIAS_ADD, AGO_OP_RELU6}) && ops[0].pointwise() &&
+        ops[2].pointwise())
+      return AGO_KERNEL_PW_PW;
+  }
   if (kinds_are(ops, {AGO_OP_GEMM, AGO_OP_BIAS_ADD, AGO_OP_GELU_TANH, AGO_OP_GEMM, AGO_OP_BIAS_ADD}))
     return AGO_KERNEL_FFN;
   if (kinds_are(ops, {AGO_OP_CONV2D, AGO_OP_BIAS_ADD, AGO_OP_RELU, AGO_OP_CONV2D, AGO_OP_BIAS_ADD,
@@ -259,8 +275,8 @@ ago_status_t build_plan(const ago_subgraph_desc_t* desc, Plan* plan, std::string
   if (p.mode == AGO_MODE_FUSED) {
     p.fused_kernel = match_fused_family(p);
     if (p.fused_kernel == AGO_KERNEL_NONE) {
-      *err = "fused mode: the operator chain matches no fused kernel family (depthwise-only; 1x1 -> depthwise 3x3 -> 1x1; "
-             "GEMM -> GELU -> GEMM; conv3x3 -> conv3x3 + input -> ReLU; QK^T -> scale -> softmax -> PV)";
+      *err = "fused mode: the operator chain matches no fused kernel family (depthwise-only; 1x1 -> depthwise 3x3 -> 1x1 "
+             "and its pairs; GEMM -> GELU -> GEMM; conv3x3 -> conv3x3 + input -> ReLU; QK^T -> scale -> softmax -> PV)";
       return AGO_ERR_UNSUPPORTED;
     }
     p.num_launches = 1;

@@ -117,6 +117,15 @@ __device__ __forceinline__ void tcgen05_fence_after_sync() {
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
 }
 
+// ---- per-thread asynchronous copies (global -> shared, 16 bytes, zero-filled beyond src_bytes) ----------
+
+__device__ __forceinline__ void cp_async_16(uint32_t dst_saddr, const void* src, uint32_t src_bytes) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst_saddr), "l"(src), "r"(src_bytes) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+// all of this thread's commit groups but the most recent one are complete
+__device__ __forceinline__ void cp_async_wait_but_one() { asm volatile("cp.async.wait_group 1;" ::: "memory"); }
+
 // ---- TMA (cp.async.bulk.tensor), no multicast ----------------------------------------------
 
 __device__ __forceinline__ void tma_prefetch_desc(const void* tmap) {

@@ -153,6 +153,33 @@ def attention(name, seed_seq, B, S, heads, head_dim) -> Workload:
                     input_dist=["normal"] * 3)
 
 
+# The two-complex-operator pairs of the fusion-strategy micro-benchmark (Section VI-B): pointwise and depthwise
+# convolutions with their bias / ReLU6 as they follow each other in MobileNetV2-like blocks.
+_PW = lambda o: ("conv2d", dict(O=o, R=1, S=1, stride=1, pad=0, groups=1))
+_DW = lambda c, stride: ("conv2d", dict(O=c, R=3, S=3, stride=stride, pad=1, groups=c))
+
+
+def pw_dw(name, seed_seq, N, H, c_in, c_exp, stride) -> Workload:
+    ops = [_PW(c_exp), ("bias_add", {}), ("relu6", {}), _DW(c_exp, stride), ("bias_add", {}), ("relu6", {})]
+    return Workload(name, seed_seq, [(N, H, H, c_in)], ops, samples=N, input_dist=["uniform"])
+
+
+def dw_pw(name, seed_seq, N, H, c_exp, c_out, stride) -> Workload:
+    ops = [_DW(c_exp, stride), ("bias_add", {}), ("relu6", {}), _PW(c_out), ("bias_add", {})]
+    return Workload(name, seed_seq, [(N, H, H, c_exp)], ops, samples=N, input_dist=["relu_normal"])
+
+
+def dw_dw(name, seed_seq, N, H, c) -> Workload:
+    ops = [_DW(c, 1), ("bias_add", {}), ("relu6", {}), _DW(c, 1), ("bias_add", {}), ("relu6", {})]
+    return Workload(name, seed_seq, [(N, H, H, c)], ops, samples=N, input_dist=["relu_normal"])
+
+
+def pw_pw(name, seed_seq, N, H, c_in, c_mid, c_out) -> Workload:
+    # the linear bottleneck of one block followed by the expansion of the next
+    ops = [_PW(c_mid), ("bias_add", {}), _PW(c_out), ("bias_add", {}), ("relu6", {})]
+    return Workload(name, seed_seq, [(N, H, H, c_in)], ops, samples=N, input_dist=["relu_normal"])
+
+
 def get(name: str, batch: int | None = None) -> Workload:
     """The benchmark configurations. ``batch`` overrides the number of
     independent samples (images, sequences) while keeping per-sample shapes."""
@@ -171,10 +198,20 @@ def get(name: str, batch: int | None = None) -> Workload:
     if name == "ffn_12288":      # config 4b
         b = batch or 32
         return ffn(name, [4, 1], 384 * b, 768, 3072, samples=b)
+    # pairs of the 56 x 56 block (24 -> 144 -> 24), batch 32
+    if name == "pw_dw_56":
+        return pw_dw(name, [5, 0], batch or 32, 56, 24, 144, 1)
+    if name == "dw_pw_56":
+        return dw_pw(name, [5, 1], batch or 32, 56, 144, 24, 1)
+    if name == "dw_dw_56":
+        return dw_dw(name, [5, 2], batch or 32, 56, 144)
+    if name == "pw_pw_56":
+        return pw_pw(name, [5, 3], batch or 32, 56, 144, 24, 144)
     raise KeyError(name)
 
 
-ALL = ["mbv2_14", "ffn_512", "mbv2_56", "mbv2_28s2", "resnet_56", "attn_384", "ffn_12288"]
+PAIRS = ["pw_dw_56", "dw_pw_56"]
+ALL = ["mbv2_14", "ffn_512", "mbv2_56", "mbv2_28s2", "resnet_56", "attn_384", "ffn_12288"] + PAIRS
 
 
 # ---- seeded tensors ---------------------------------------------------------------

@@ -136,6 +136,43 @@ def test_fused_agrees_with_unfused_chain(ago, name):
     assert float(np.max(np.abs(fused - mini))) <= 2e-2 * scale + 1e-3
 
 
+PAIR_SMALL = {
+    "pw_dw_s1": lambda: WL.pw_dw("pw_dw_s1", [81], 2, 14, 32, 192, 1),
+    "pw_dw_s1_odd": lambda: WL.pw_dw("pw_dw_s1_odd", [82], 3, 13, 24, 144, 1),
+    "pw_dw_s2": lambda: WL.pw_dw("pw_dw_s2", [83], 2, 14, 32, 192, 2),
+    "pw_dw_s2_odd": lambda: WL.pw_dw("pw_dw_s2_odd", [84], 2, 9, 16, 96, 2),
+    "pw_dw_tall": lambda: WL.pw_dw("pw_dw_tall", [85], 1, 40, 24, 48, 1),
+    "dw_pw_s1": lambda: WL.dw_pw("dw_pw_s1", [86], 2, 14, 192, 32, 1),
+    "dw_pw_s1_odd": lambda: WL.dw_pw("dw_pw_s1_odd", [87], 3, 13, 144, 24, 1),
+    "dw_pw_s2": lambda: WL.dw_pw("dw_pw_s2", [88], 2, 14, 192, 64, 2),
+    "dw_pw_s2_odd": lambda: WL.dw_pw("dw_pw_s2_odd", [89], 2, 9, 96, 32, 2),
+    "dw_pw_tall": lambda: WL.dw_pw("dw_pw_tall", [90], 1, 40, 48, 24, 1),
+    "dw_pw_one_chunk": lambda: WL.dw_pw("dw_pw_one_chunk", [91], 1, 11, 16, 8, 1),
+}
+
+
+@pytest.mark.parametrize("name", list(PAIR_SMALL.keys()))
+def test_fused_pairs_match_oracle(ago, name):
+    # the two-complex-operator pairs: stride 1 and 2, ragged strips, one to twelve channel chunks
+    wl = PAIR_SMALL[name]()
+    data = WL.generate(wl)
+    ref = O.run_chain(wl.ops, data["inputs"], data["weights"])
+    assert_close(run_gpu(ago, wl, data, "fused"), ref, what=f"{name}/fused")
+    for mode in UNFUSED:
+        assert_close(run_gpu(ago, wl, data, mode), ref, what=f"{name}/{mode}")
+
+
+@pytest.mark.parametrize("name", ["pw_dw_56", "dw_pw_56"])
+def test_fused_pairs_full_size_on_sampled_images(ago, name):
+    wl = WL.get(name)
+    data = WL.generate(wl)
+    gpu = run_gpu(ago, wl, data, "fused")
+    for img in (0, 17, wl.samples - 1):
+        one = WL.get(name, batch=1)
+        ref = O.run_chain(one.ops, [data["inputs"][0][img:img + 1]], data["weights"])
+        assert_close(gpu[img:img + 1], ref, what=f"{name} image {img}")
+
+
 def test_fused_mbv2_pads_the_intermediate_not_the_input(ago):
     wl = WL.mbv2_block("pad", [33], 1, 6, 8, 16, 8, 1, True)
     data = WL.generate(wl)
