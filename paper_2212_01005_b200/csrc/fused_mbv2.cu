@@ -33,6 +33,7 @@
 #include <algorithm>
 #include <cstdlib>
 
+#include "dw_common.cuh"
 #include "fused.h"
 #include "tc_common.cuh"
 
@@ -41,6 +42,7 @@ namespace ago {
 namespace {
 
 using namespace tc;
+using namespace dw;
 
 constexpr int kWarps = 32;                         // every warp computes; MMAs are issued inline by some of them
 constexpr int kThreads = kWarps * 32;
@@ -74,117 +76,6 @@ struct Mbv2Params {
   int off_x, off_w1, off_e, off_d, off_w3, off_wd, off_b1, off_bd, off_b3, off_bar;
 };
 
-// bf16x2(min(max(lo, 0), 6), min(max(hi, 0), 6)): the conversion clamps at 0, one packed min caps at 6.
-__device__ __forceinline__ uint32_t relu6_pack(float lo, float hi) {
-  uint32_t r;
-  asm("{\n\t.reg .b32 t, six;\n\tmov.b32 six, 0x40C040C0;\n\tcvt.rn.relu.bf16x2.f32 t, %2, %1;\n\tmin.bf16x2 %0, t, six;\n\t}"
-      : "=r"(r) : "f"(lo), "f"(hi));
-  return r;
-}
-
-// Shared-memory word loads / stores with an immediate byte offset.
-template <int OFF>
-__device__ __forceinline__ uint32_t lds32(uint32_t saddr) {
-  uint32_t v;
-  asm volatile("ld.shared.u32 %0, [%1+%2];" : "=r"(v) : "r"(saddr), "n"(OFF));
-  return v;
-}
-template <int OFF = 0>
-__device__ __forceinline__ void sts32(uint32_t saddr, uint32_t v) {
-  asm volatile("st.shared.u32 [%0+%1], %2;" ::"r"(saddr), "n"(OFF), "r"(v) : "memory");
-}
-
-// acc += x * w for a packed pair of bf16 channels: the mixed-precision FMA takes the bf16 operands
-// as they are (exact product, fp32 accumulate) -- no unpacking of the activations or the weights.
-__device__ __forceinline__ void fma_pair(float2& acc, uint32_t x, uint32_t w) {
-  asm("{\n\t.reg .b16 xl, xh, wl, wh;\n\t"
-      "mov.b32 {xl, xh}, %2;\n\tmov.b32 {wl, wh}, %3;\n\t"
-      "fma.rn.f32.bf16 %0, xl, wl, %0;\n\tfma.rn.f32.bf16 %1, xh, wh, %1;\n\t}"
-      : "+f"(acc.x), "+f"(acc.y) : "r"(x), "r"(w));
-}
-
-struct Row3 { uint32_t v0, v1, v2; };   // three horizontally adjacent pixels of one channel pair
-template <int PIX_STEP>
-__device__ __forceinline__ Row3 load_row3(uint32_t a) {
-  Row3 r;
-  r.v0 = lds32<0>(a); r.v1 = lds32<PIX_STEP>(a); r.v2 = lds32<2 * PIX_STEP>(a);
-  return r;
-}
-__device__ __forceinline__ uint32_t depthwise_point(const Row3& a, const Row3& b, const Row3& c, const uint32_t (&w)[9],
-                                                    float2 bias) {
-  float2 acc = bias;
-  fma_pair(acc, a.v0, w[0]); fma_pair(acc, a.v1, w[1]); fma_pair(acc, a.v2, w[2]);
-  fma_pair(acc, b.v0, w[3]); fma_pair(acc, b.v1, w[4]); fma_pair(acc, b.v2, w[5]);
-  fma_pair(acc, c.v0, w[6]); fma_pair(acc, c.v1, w[7]); fma_pair(acc, c.v2, w[8]);
-  return relu6_pack(acc.x, acc.y);
-}
-
-// E and D chunks are two planes of [pixel][8 channels] (16 bytes per pixel), which is also the
-// un-swizzled K-major operand layout; all addresses below are 32-bit shared-memory addresses.
-//
-// Stride-2 depthwise 3x3 for one (channel pair, output column) and output rows [r0, r1), r1 > r0:
-// consecutive output rows share one input row, which stays packed in registers (the loop body is
-// unrolled over the two roles of that row).
-__device__ __forceinline__ void depthwise_column_s2(uint32_t e_col, uint32_t d_col, int r0, int r1, int IW, int Wo,
-                                                    const uint32_t (&w)[9], float2 bias) {
-  const uint32_t e_pitch = (uint32_t)IW * 16u, d_pitch = (uint32_t)Wo * 16u;
-  uint32_t src = e_col + (uint32_t)(r0 * 2) * e_pitch;
-  uint32_t dst = d_col + (uint32_t)r0 * d_pitch;
-  int n = r1 - r0;
-  Row3 a = load_row3<16>(src), b, c;
-  src += e_pitch;
-  while (true) {
-    b = load_row3<16>(src); c = load_row3<16>(src + e_pitch); src += 2 * e_pitch;
-    sts32(dst, depthwise_point(a, b, c, w, bias)); dst += d_pitch;
-    if (--n == 0) break;
-    b = load_row3<16>(src); a = load_row3<16>(src + e_pitch); src += 2 * e_pitch;
-    sts32(dst, depthwise_point(c, b, a, w, bias)); dst += d_pitch;
-    if (--n == 0) break;
-  }
-}
-
-// Stride-1 depthwise 3x3 for one channel pair and a block of 2 output rows x 7 output columns, fully
-// unrolled: three input columns (4 rows each) stay packed in registers and rotate by renaming, all
-// shared-memory offsets are immediates; each loaded pixel feeds up to six outputs. e_row: address of
-// the block's first input pixel in the row above the first output row; d_row: address of its first
-// output pixel; ncol <= 7 columns and nrows <= 2 rows are stored (the loads of a ragged block run
-// past the valid pixels, inside shared memory; those results are dropped).
-constexpr int kSegCols = 7;
-__device__ __forceinline__ void depthwise_block(uint32_t e_row, uint32_t d_row, uint32_t e_pitch, uint32_t d_pitch, int ncol,
-                                                int nrows, const uint32_t (&w)[9], float2 bias) {
-  const uint32_t e0 = e_row, e1 = e0 + e_pitch, e2 = e1 + e_pitch, e3 = e2 + e_pitch;
-  const uint32_t d0 = d_row, d1 = d_row + d_pitch;
-  uint32_t c0[4], c1[4], c2[4];
-  c0[0] = lds32<0>(e0); c0[1] = lds32<0>(e1); c0[2] = lds32<0>(e2); c0[3] = lds32<0>(e3);
-  c1[0] = lds32<16>(e0); c1[1] = lds32<16>(e1); c1[2] = lds32<16>(e2); c1[3] = lds32<16>(e3);
-#define AGO_DW_STEP(J, A, B, C)                                                                       \
-  {                                                                                                   \
-    C[0] = lds32<(J + 2) * 16>(e0); C[1] = lds32<(J + 2) * 16>(e1);                                   \
-    C[2] = lds32<(J + 2) * 16>(e2); C[3] = lds32<(J + 2) * 16>(e3);                                   \
-    float2 acc0 = bias, acc1 = bias;                                                                  \
-    fma_pair(acc0, A[0], w[0]); fma_pair(acc0, B[0], w[1]); fma_pair(acc0, C[0], w[2]);               \
-    fma_pair(acc0, A[1], w[3]); fma_pair(acc0, B[1], w[4]); fma_pair(acc0, C[1], w[5]);               \
-    fma_pair(acc1, A[1], w[0]); fma_pair(acc1, B[1], w[1]); fma_pair(acc1, C[1], w[2]);               \
-    fma_pair(acc0, A[2], w[6]); fma_pair(acc0, B[2], w[7]); fma_pair(acc0, C[2], w[8]);               \
-    fma_pair(acc1, A[2], w[3]); fma_pair(acc1, B[2], w[4]); fma_pair(acc1, C[2], w[5]);               \
-    fma_pair(acc1, A[3], w[6]); fma_pair(acc1, B[3], w[7]); fma_pair(acc1, C[3], w[8]);               \
-    if (FULL || J < ncol) {                                                                           \
-      sts32<J * 16>(d0, relu6_pack(acc0.x, acc0.y));                                                  \
-      if (FULL || nrows > 1) sts32<J * 16>(d1, relu6_pack(acc1.x, acc1.y));                           \
-    }                                                                                                 \
-  }
-  if (ncol == kSegCols && nrows == 2) {
-    constexpr bool FULL = true;
-    AGO_DW_STEP(0, c0, c1, c2) AGO_DW_STEP(1, c1, c2, c0) AGO_DW_STEP(2, c2, c0, c1) AGO_DW_STEP(3, c0, c1, c2)
-    AGO_DW_STEP(4, c1, c2, c0) AGO_DW_STEP(5, c2, c0, c1) AGO_DW_STEP(6, c0, c1, c2)
-  } else {
-    constexpr bool FULL = false;
-    AGO_DW_STEP(0, c0, c1, c2) AGO_DW_STEP(1, c1, c2, c0) AGO_DW_STEP(2, c2, c0, c1) AGO_DW_STEP(3, c0, c1, c2)
-    AGO_DW_STEP(4, c1, c2, c0) AGO_DW_STEP(5, c2, c0, c1) AGO_DW_STEP(6, c0, c1, c2)
-  }
-#undef AGO_DW_STEP
-}
-
 // EXPAND / PROJECT select the pairs of the block: <true, true> the whole block, <true, false> pointwise -> depthwise
 // (the depthwise result of every chunk goes to device memory), <false, true> depthwise -> pointwise (every chunk of
 // the input is copied into the E buffers instead of being computed).
@@ -211,7 +102,7 @@ mbv2_fused_kernel(const Mbv2Params p) {
   volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(bars + 13);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int n = (int)__umulhi(blockIdx.x, p.strips_recip), strip = (int)blockIdx.x - n * p.strips;
+  const int n = (int)fast_div(blockIdx.x, (uint32_t)p.strips, p.strips_recip), strip = (int)blockIdx.x - n * p.strips;
   const int ho0 = strip * p.R;
   const int rows_valid = min(p.R, p.Ho - ho0);
   const int gh0 = ho0 * p.stride - 1;   // image row of tile row 0
@@ -295,7 +186,7 @@ mbv2_fused_kernel(const Mbv2Params p) {
       rows_per_group = (rows_valid + groups - 1) / groups;
     }
     const int dw_items = per_row * (p.stride == 1 ? (rows_valid + 1) / 2 : groups);   // stride 1: blocks of two rows
-    const int item0_r = (int)__umulhi((uint32_t)slot, p.per_row_recip), item0_c = slot - item0_r * per_row;   // the thread's first item
+    const int item0_r = (int)fast_div((uint32_t)slot, (uint32_t)per_row, p.per_row_recip), item0_c = slot - item0_r * per_row;   // the thread's first item
     const int step_r = p.step_r, step_c = p.step_c;                        // item += kSlots in (row, column) form
     const int e_bytes = 2 * p.e_plane;
     // Expand-epilogue tiles of this warp: the group's warps of one tensor-memory lane quarter (warp & 3) share the M1
@@ -311,7 +202,7 @@ mbv2_fused_kernel(const Mbv2Params p) {
     for (int k = 0; k < kTilesPerWarp; ++k) {
       const int t = q_rank + k * q_mates;
       const int pix = t * 128 + (warp & 3) * 32 + lane;
-      const int ih = (int)__umulhi((uint32_t)pix, p.w_recip), iw = pix - ih * p.W;
+      const int ih = (int)fast_div((uint32_t)pix, (uint32_t)p.W, p.w_recip), iw = pix - ih * p.W;
       const int gh = gh0 + ih;
       e_pix[k] = -1;
       if (t < p.M1 && pix < p.P_x) {
@@ -441,7 +332,7 @@ mbv2_fused_kernel(const Mbv2Params p) {
         ld_src[k] = 0u; ld_dst[k] = 0u;
         if (i < p.P_x * 2) {
           const int pix = i >> 1, plane = i & 1;
-          const int ih = (int)__umulhi((uint32_t)pix, p.w_recip), iw = pix - ih * p.W;
+          const int ih = (int)fast_div((uint32_t)pix, (uint32_t)p.W, p.w_recip), iw = pix - ih * p.W;
           ld_ok |= 1u << k;
           ld_dst[k] = (uint32_t)(plane * p.e_plane + (ih * p.IW + iw + 1) * 16);
           if (gh0 + ih >= 0 && gh0 + ih < p.H) { ld_in |= 1u << k; ld_src[k] = (uint32_t)(pix * p.Cexp * 2 + plane * 16); }
@@ -611,7 +502,7 @@ struct Mbv2Host {
 bool layout(Mbv2Params& q, int R, bool expand, bool project, int* smem_bytes) {
   q.R = R;
   q.strips = (q.Ho + R - 1) / R;
-  q.strips_recip = (uint32_t)((1ull << 32) / (uint64_t)q.strips + 1ull);
+  q.strips_recip = fast_div_recip(q.strips);
   q.IH = (R - 1) * q.stride + 3;
   q.IW = q.W + 2;
   q.P_in = q.IH * q.IW;
@@ -674,7 +565,7 @@ ago_status_t mbv2_plan(Plan* plan, FusedState* st, std::string* err) {
   q.swizzle = q.Kp == 16 ? tc::SW_32B : (q.Kp == 32 ? tc::SW_64B : tc::SW_128B);
   q.Coutp = round_up(q.Cout, 16);
   q.NC = q.Cexp / kChunk;
-  auto recip = [](int d) { return (uint32_t)((1ull << 32) / (uint64_t)d + 1ull); };
+  auto recip = [](int d) { return tc::fast_div_recip(d); };
   q.coutp_recip = recip(q.Coutp);
   q.w_recip = recip(q.W);
   {
@@ -698,6 +589,7 @@ ago_status_t mbv2_plan(Plan* plan, FusedState* st, std::string* err) {
   }
   if (best_R == 0) return bad("no row-strip tiling fits shared memory / tensor memory");
   layout(q, best_R, expand, project, &best_smem);
+  if ((long)q.N * q.strips > 65535) return bad("more than 65535 row strips in the batch");
   host->smem_bytes = best_smem;
   st->impl = host;
   st->impl_free = [](void* p) { delete static_cast<Mbv2Host*>(p); };

@@ -117,6 +117,11 @@ __device__ __forceinline__ void tcgen05_fence_after_sync() {
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
 }
 
+// x / d for x, d < 65536 with recip = 2^32 / d + 1 computed on the host (fast_div_recip); d == 1 has no 32-bit
+// reciprocal and is passed through.
+__device__ __forceinline__ uint32_t fast_div(uint32_t x, uint32_t d, uint32_t recip) { return d == 1u ? x : __umulhi(x, recip); }
+inline uint32_t fast_div_recip(int d) { return (uint32_t)((1ull << 32) / (uint64_t)d + 1ull); }
+
 // ---- per-thread asynchronous copies (global -> shared, 16 bytes, zero-filled beyond src_bytes) ----------
 
 __device__ __forceinline__ void cp_async_16(uint32_t dst_saddr, const void* src, uint32_t src_bytes) {
@@ -124,6 +129,7 @@ __device__ __forceinline__ void cp_async_16(uint32_t dst_saddr, const void* src,
 }
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 // all of this thread's commit groups but the most recent one are complete
+__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
 __device__ __forceinline__ void cp_async_wait_but_one() { asm volatile("cp.async.wait_group 1;" ::: "memory"); }
 
 // ---- TMA (cp.async.bulk.tensor), no multicast ----------------------------------------------

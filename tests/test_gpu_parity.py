@@ -148,6 +148,10 @@ PAIR_SMALL = {
     "dw_pw_s2_odd": lambda: WL.dw_pw("dw_pw_s2_odd", [89], 2, 9, 96, 32, 2),
     "dw_pw_tall": lambda: WL.dw_pw("dw_pw_tall", [90], 1, 40, 48, 24, 1),
     "dw_pw_one_chunk": lambda: WL.dw_pw("dw_pw_one_chunk", [91], 1, 11, 16, 8, 1),
+    "dw_dw_14": lambda: WL.dw_dw("dw_dw_14", [92], 2, 14, 192),
+    "dw_dw_odd": lambda: WL.dw_dw("dw_dw_odd", [93], 3, 13, 48),
+    "dw_dw_tall": lambda: WL.dw_dw("dw_dw_tall", [94], 1, 45, 32),
+    "dw_dw_tiny": lambda: WL.dw_dw("dw_dw_tiny", [95], 1, 3, 16),
 }
 
 
@@ -162,7 +166,7 @@ def test_fused_pairs_match_oracle(ago, name):
         assert_close(run_gpu(ago, wl, data, mode), ref, what=f"{name}/{mode}")
 
 
-@pytest.mark.parametrize("name", ["pw_dw_56", "dw_pw_56"])
+@pytest.mark.parametrize("name", ["pw_dw_56", "dw_pw_56", "dw_dw_56"])
 def test_fused_pairs_full_size_on_sampled_images(ago, name):
     wl = WL.get(name)
     data = WL.generate(wl)
@@ -188,6 +192,9 @@ def test_fused_mbv2_pads_the_intermediate_not_the_input(ago):
     dict(N=1, H=30, c_in=40, c_exp=240, c_out=80, stride=2, residual=False),  # Cin padded 40 -> 64
     dict(N=1, H=32, c_in=64, c_exp=64, c_out=64, stride=1, residual=True),    # large 128-byte-row tile: more input slots than one staging pass
     dict(N=2, H=24, c_in=64, c_exp=384, c_out=64, stride=1, residual=True),   # many weight slots, 24 chunks
+    dict(N=2, H=6, c_in=8, c_exp=16, c_out=8, stride=1, residual=True),       # one column segment per row
+    dict(N=4, H=3, c_in=16, c_exp=32, c_out=24, stride=1, residual=False),    # images of one strip
+    dict(N=2, H=2, c_in=16, c_exp=16, c_out=16, stride=2, residual=False),    # one output pixel per image
 ])
 def test_fused_mbv2_shape_sweep(ago, shape):
     wl = WL.mbv2_block("sweep", [41, shape["H"], shape["c_in"]], shape["N"], shape["H"], shape["c_in"], shape["c_exp"],
