@@ -24,6 +24,8 @@ ago_status_t fused_plan(Plan* plan, FusedState* st, std::string* err) {
       return mbv2_plan(plan, st, err);
     case AGO_KERNEL_DW_DW:
       return dwdw_plan(plan, st, err);
+    case AGO_KERNEL_PW_PW:
+      return pwpw_plan(plan, st, err);
     case AGO_KERNEL_ATTENTION:
       return attention_plan(plan, st, err);
     case AGO_KERNEL_FFN:
@@ -50,6 +52,8 @@ ago_status_t fused_run(const Plan& plan, FusedState* st, const void* const* inpu
       return mbv2_run(plan, st, inputs, weights, output, status_word, stream, err);
     case AGO_KERNEL_DW_DW:
       return dwdw_run(plan, st, inputs, weights, output, status_word, stream, err);
+    case AGO_KERNEL_PW_PW:
+      return pwpw_run(plan, st, inputs, weights, output, status_word, stream, err);
     case AGO_KERNEL_ATTENTION:
       return attention_run(plan, st, inputs, weights, output, status_word, stream, err);
     case AGO_KERNEL_FFN:

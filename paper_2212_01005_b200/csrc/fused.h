@@ -33,6 +33,9 @@ ago_status_t ffn_run(const Plan& plan, FusedState* st, const void* const* inputs
 ago_status_t conv3x3_plan(Plan* plan, FusedState* st, std::string* err);
 ago_status_t conv3x3_run(const Plan& plan, FusedState* st, const void* const* inputs, const void* const* weights,
                          void* output, unsigned int* status_word, cudaStream_t stream, std::string* err);
+ago_status_t pwpw_plan(Plan* plan, FusedState* st, std::string* err);
+ago_status_t pwpw_run(const Plan& plan, FusedState* st, const void* const* inputs, const void* const* weights,
+                      void* output, unsigned int* status_word, cudaStream_t stream, std::string* err);
 ago_status_t dwdw_plan(Plan* plan, FusedState* st, std::string* err);
 ago_status_t dwdw_run(const Plan& plan, FusedState* st, const void* const* inputs, const void* const* weights,
                       void* output, unsigned int* status_word, cudaStream_t stream, std::string* err);

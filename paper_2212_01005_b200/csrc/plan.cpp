@@ -87,9 +87,14 @@ int match_fused_family(const Plan& p) {
     if (kinds_are(ops, {AGO_OP_CONV2D, AGO_OP_BIAS_ADD, AGO_OP_RELU6, AGO_OP_CONV2D, AGO_OP_BIAS_ADD}) && dw3x3(ops[0]) &&
         ops[3].pointwise())
       return AGO_KERNEL_DW_PW;
-    if (kinds_are(ops, {AGO_OP_CONV2D, AGO_OP_BIAS_ADD, AGO_OP_CONV2D, AGO_OP_BIAS_ADD, AGO_OP_RELU6}) && ops[0].pointwise() &&
-        ops[2].pointwise())
-      return AGO_KERNEL_PW_PW;
+    // conv, bias, [ReLU6], conv, bias, [ReLU6] with two pointwise convolutions
+    if (ops.size() >= 4 && ops.size() <= 6 && ops[0].pointwise() && ops[1].op.kind == AGO_OP_BIAS_ADD) {
+      size_t i = 2;
+      if (ops[i].op.kind == AGO_OP_RELU6) ++i;
+      if (i + 1 < ops.size() && ops[i].pointwise() && ops[i + 1].op.kind == AGO_OP_BIAS_ADD &&
+          (i + 2 == ops.size() || (i + 3 == ops.size() && ops[i + 2].op.kind == AGO_OP_RELU6)))
+        return AGO_KERNEL_PW_PW;
+    }
   }
   if (kinds_are(ops, {AGO_OP_GEMM, AGO_OP_BIAS_ADD, AGO_OP_GELU_TANH, AGO_OP_GEMM, AGO_OP_BIAS_ADD}))
     return AGO_KERNEL_FFN;

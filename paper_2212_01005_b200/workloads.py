@@ -174,9 +174,10 @@ def dw_dw(name, seed_seq, N, H, c) -> Workload:
     return Workload(name, seed_seq, [(N, H, H, c)], ops, samples=N, input_dist=["relu_normal"])
 
 
-def pw_pw(name, seed_seq, N, H, c_in, c_mid, c_out) -> Workload:
-    # the linear bottleneck of one block followed by the expansion of the next
-    ops = [_PW(c_mid), ("bias_add", {}), _PW(c_out), ("bias_add", {}), ("relu6", {})]
+def pw_pw(name, seed_seq, N, H, c_in, c_mid, c_out, act1=False, act2=True) -> Workload:
+    # default: the linear bottleneck of one block followed by the expansion of the next
+    ops = [_PW(c_mid), ("bias_add", {})] + ([("relu6", {})] if act1 else []) + [_PW(c_out), ("bias_add", {})] + \
+          ([("relu6", {})] if act2 else [])
     return Workload(name, seed_seq, [(N, H, H, c_in)], ops, samples=N, input_dist=["relu_normal"])
 
 
@@ -210,7 +211,7 @@ def get(name: str, batch: int | None = None) -> Workload:
     raise KeyError(name)
 
 
-PAIRS = ["pw_dw_56", "dw_pw_56", "dw_dw_56"]
+PAIRS = ["pw_dw_56", "dw_pw_56", "dw_dw_56", "pw_pw_56"]
 ALL = ["mbv2_14", "ffn_512", "mbv2_56", "mbv2_28s2", "resnet_56", "attn_384", "ffn_12288"] + PAIRS
 
 

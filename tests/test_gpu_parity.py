@@ -152,6 +152,11 @@ PAIR_SMALL = {
     "dw_dw_odd": lambda: WL.dw_dw("dw_dw_odd", [93], 3, 13, 48),
     "dw_dw_tall": lambda: WL.dw_dw("dw_dw_tall", [94], 1, 45, 32),
     "dw_dw_tiny": lambda: WL.dw_dw("dw_dw_tiny", [95], 1, 3, 16),
+    "pw_pw_14": lambda: WL.pw_pw("pw_pw_14", [96], 2, 14, 192, 32, 192),
+    "pw_pw_ragged": lambda: WL.pw_pw("pw_pw_ragged", [97], 3, 13, 144, 24, 144),          # 507 rows, channel counts 8 mod 16
+    "pw_pw_act_first": lambda: WL.pw_pw("pw_pw_act_first", [98], 1, 20, 64, 128, 40, act1=True, act2=False),
+    "pw_pw_act_both": lambda: WL.pw_pw("pw_pw_act_both", [99], 1, 9, 8, 8, 8, act1=True, act2=True),
+    "pw_pw_linear": lambda: WL.pw_pw("pw_pw_linear", [100], 2, 16, 160, 128, 256, act1=False, act2=False),
 }
 
 
@@ -166,7 +171,7 @@ def test_fused_pairs_match_oracle(ago, name):
         assert_close(run_gpu(ago, wl, data, mode), ref, what=f"{name}/{mode}")
 
 
-@pytest.mark.parametrize("name", ["pw_dw_56", "dw_pw_56", "dw_dw_56"])
+@pytest.mark.parametrize("name", ["pw_dw_56", "dw_pw_56", "dw_dw_56", "pw_pw_56"])
 def test_fused_pairs_full_size_on_sampled_images(ago, name):
     wl = WL.get(name)
     data = WL.generate(wl)
