@@ -7,7 +7,7 @@
 // tile it needs is the same rows with all middle channels -- nothing is recomputed. CTAs are persistent (two per SM,
 // out of phase: one copies while the other computes) and walk over tiles of 128 pixel rows. Per tile:
 //   P1  TMA: the X tile as K-major blocks of 64 channels (128-byte swizzle); rows past the tensor and channels past
-//       C0 read as zero. Both weight matrices are fetched once per CTA the same way.
+//       C0 read as zero. Both weight matrices are fetched once per CTA into the same layout with plain loads.
 //   P2  tcgen05.mma: mid[128 x C1] = X[128 x C0] * W1^T                         (TMEM, fp32)
 //   P3  TMEM -> registers: + b1 [ReLU6], bf16 -> shared memory as the swizzled A operand of the second product
 //   P4  tcgen05.mma: out[128 x C2] = mid[128 x C1] * W2^T                       (TMEM, same columns)
@@ -35,6 +35,8 @@ constexpr int kBM = 128, kBK = 64;
 constexpr int kXBlock = kBM * kBK * 2;   // one K block of the X / mid tile: 16 KB
 
 struct PwPwParams {
+  const __nv_bfloat16* w1;   // [C1][C0]
+  const __nv_bfloat16* w2;   // [C2][C1]
   const float* b1;
   const float* b2;
   __nv_bfloat16* out;        // [M][C2]
@@ -44,8 +46,9 @@ struct PwPwParams {
   int nkb0, nkb1;            // 64-channel K blocks of the first / second product
   int act1, act2;            // ReLU6 after the first / second convolution
   uint32_t k2_recip;         // reciprocal of the 16-byte pieces per output row (C2 / 8)
+  uint32_t c0_recip, c1_recip;   // ... per padded weight row (C0p / 8, C1p / 8)
   int pitch;                 // row pitch of the staging tile
-  int x_tx, w_tx;            // bytes one X tile / both weight matrices bring in (TMA transaction counts)
+  int x_tx;                  // bytes one X tile brings in (TMA transaction count)
   int tmem_cols;
   int off_x, off_a, off_w1, off_w2, off_b, off_bar;
 };
@@ -53,8 +56,7 @@ struct PwPwParams {
 __device__ __forceinline__ float relu6f(float v) { return fminf(fmaxf(v, 0.0f), 6.0f); }
 
 __global__ void __launch_bounds__(kThreads)
-pwpw_fused_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w1,
-                  const __grid_constant__ CUtensorMap tmap_w2, const PwPwParams p) {
+pwpw_fused_kernel(const __grid_constant__ CUtensorMap tmap_x, const PwPwParams p) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t* sX = smem + p.off_x;
@@ -65,7 +67,6 @@ pwpw_fused_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
   float* sB2 = sB1 + p.C1p;
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + p.off_bar);
   uint64_t* bar_x = bars;        // X tile landed
-  uint64_t* bar_w = bars + 1;    // weights landed (once)
   uint64_t* bar_m1 = bars + 2;   // first product complete
   uint64_t* bar_m2 = bars + 3;   // second product complete
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 4);
@@ -81,8 +82,6 @@ pwpw_fused_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
     fence_mbar_init();
     fence_proxy_async_smem();
     tma_prefetch_desc(&tmap_x);
-    tma_prefetch_desc(&tmap_w1);
-    tma_prefetch_desc(&tmap_w2);
   }
   if (warp == 1) {
     tmem_alloc(tmem_slot, (uint32_t)p.tmem_cols);
@@ -94,14 +93,42 @@ pwpw_fused_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
   };
   grid_dependency_wait();
   grid_launch_dependents();
-  if (tid == 0) {
-    mbar_arrive_expect_tx(bar_w, (uint32_t)p.w_tx);
-    for (int kb = 0; kb < p.nkb0; ++kb) tma_load_2d(sW1 + kb * p.C1p * 128, &tmap_w1, bar_w, kb * kBK, 0);
-    for (int kb = 0; kb < p.nkb1; ++kb) tma_load_2d(sW2 + kb * p.C2p * 128, &tmap_w2, bar_w, kb * kBK, 0);
-    if ((int)blockIdx.x < ntiles) load_x(blockIdx.x);
+  if (tid == 0 && (int)blockIdx.x < ntiles) load_x(blockIdx.x);
+  // Weights: every CTA of the grid reads the same few kilobytes at the same time, so they are fetched with a few
+  // wide coalesced requests per warp (16 bytes per thread, all loads of a batch in flight before its first store)
+  // instead of one TMA request per matrix row, and written to the swizzled K-major blocks by hand; rows and
+  // reduction channels added by the padding are zero.
+  {
+    constexpr int kBatch = 4;
+    const int c0 = p.C0p >> 3, c1 = p.C1p >> 3;              // 16-byte chunks per padded row
+    const int n1 = p.C1p * c0, nw = n1 + p.C2p * c1;
+    for (int base = tid; base < nw; base += kBatch * kThreads) {
+      uint4 v[kBatch];
+      uint32_t dst[kBatch];
+#pragma unroll
+      for (int k = 0; k < kBatch; ++k) {
+        const int i = base + k * kThreads;
+        v[k] = make_uint4(0, 0, 0, 0);
+        dst[k] = 0xffffffffu;
+        if (i < nw) {
+          const bool first = i < n1;
+          const int j = first ? i : i - n1;
+          const int cpr = first ? c0 : c1;
+          const int row = (int)fast_div((uint32_t)j, (uint32_t)cpr, first ? p.c0_recip : p.c1_recip), ch = j - row * cpr;
+          const int K = first ? p.C0 : p.C1, R = first ? p.C1 : p.C2, Rp = first ? p.C1p : p.C2p;
+          dst[k] = (uint32_t)((first ? p.off_w1 : p.off_w2) + (ch >> 3) * Rp * 128) + swz_offset((uint32_t)row, (uint32_t)(ch & 7), 128);
+          if (row < R && ch * 8 < K)
+            v[k] = __ldg(reinterpret_cast<const uint4*>((first ? p.w1 : p.w2) + (int64_t)row * K + ch * 8));
+        }
+      }
+#pragma unroll
+      for (int k = 0; k < kBatch; ++k)
+        if (dst[k] != 0xffffffffu) *reinterpret_cast<uint4*>(smem + dst[k]) = v[k];
+    }
   }
   for (int i = tid; i < p.C1p + p.C2p; i += kThreads)
     sB1[i] = i < p.C1p ? (i < p.C1 ? __ldg(p.b1 + i) : 0.0f) : (i - p.C1p < p.C2 ? __ldg(p.b2 + i - p.C1p) : 0.0f);
+  fence_proxy_async_smem();
   tcgen05_fence_before_sync();
   __syncthreads();
   tcgen05_fence_after_sync();
@@ -116,7 +143,6 @@ pwpw_fused_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
     const int row0 = tile * kBM, rows = min(kBM, p.M - row0);
     // ---- P2: first product ----
     if (tid == 0) {
-      if (it == 0) mbar_wait(bar_w, 0, abort_flag, p.status, 0x603);
       mbar_wait(bar_x, par, abort_flag, p.status, 0x600);
       tcgen05_fence_after_sync();
       for (int kb = 0; kb < p.nkb0; ++kb) {
@@ -207,9 +233,7 @@ struct PwPwHost {
   PwPwParams prm;
   int smem_bytes = 0;
   int grid = 0;   // persistent CTAs: two per SM
-  struct Key { const void* p; int which; bool operator==(const Key& o) const { return p == o.p && which == o.which; } };
-  struct KeyHash { size_t operator()(const Key& k) const { return std::hash<const void*>()(k.p) ^ (size_t)k.which * 0x9e3779b97f4a7c15ull; } };
-  std::unordered_map<Key, CUtensorMap, KeyHash> maps;
+  std::unordered_map<const void*, CUtensorMap> maps;   // X tensor maps by base address
 };
 
 }  // namespace
@@ -234,9 +258,9 @@ ago_status_t pwpw_plan(Plan* plan, FusedState* st, std::string* err) {
   if (q.C1p > 256 || q.C2p > 256) return bad("more than 256 middle or output channels is not supported");
   q.nkb0 = (q.C0 + kBK - 1) / kBK; q.nkb1 = (q.C1p + kBK - 1) / kBK;
   q.k2_recip = fast_div_recip(q.C2 / 8);
+  q.c0_recip = fast_div_recip(q.C0p / 8); q.c1_recip = fast_div_recip(q.C1p / 8);
   q.pitch = q.C2 * 2 + 16;
   q.x_tx = q.nkb0 * kXBlock;
-  q.w_tx = q.nkb0 * q.C1p * 128 + q.nkb1 * q.C2p * 128;
   q.tmem_cols = 32;
   while (q.tmem_cols < std::max(q.C1p, q.C2p)) q.tmem_cols *= 2;
   int off = 0;
@@ -249,7 +273,8 @@ ago_status_t pwpw_plan(Plan* plan, FusedState* st, std::string* err) {
   q.off_bar = take(64);
   host->smem_bytes = off + 1024;
   if (host->smem_bytes > 227 * 1024) return bad("the operands of one row tile do not fit shared memory");
-  if ((long)kBM * (q.C2 / 8) > 65535) return bad("output rows too wide for the copy index arithmetic");
+  if ((long)kBM * (q.C2 / 8) > 65535 || (long)q.C1p * (q.C0p / 8) > 65535 || (long)q.C2p * (q.C1p / 8) > 65535)
+    return bad("operands too large for the copy index arithmetic");
   host->grid = std::min((q.M + kBM - 1) / kBM, 2 * 148);
   st->impl = host;
   st->impl_free = [](void* p) { delete static_cast<PwPwHost*>(p); };
@@ -263,38 +288,32 @@ ago_status_t pwpw_run(const Plan& plan, FusedState* st, const void* const* input
   (void)plan;
   PwPwHost* host = static_cast<PwPwHost*>(st->impl);
   PwPwParams q = host->prm;
-  q.b1 = static_cast<const float*>(weights[1]);
-  q.b2 = static_cast<const float*>(weights[3]);
+  q.w1 = static_cast<const __nv_bfloat16*>(weights[0]); q.b1 = static_cast<const float*>(weights[1]);
+  q.w2 = static_cast<const __nv_bfloat16*>(weights[2]); q.b2 = static_cast<const float*>(weights[3]);
   q.out = static_cast<__nv_bfloat16*>(output);
   q.status = status_word;
-  // [rows][K] bf16 matrices as K-major tiles of 64 channels: X [M][C0], W1 [C1][C0], W2 [C2][C1]
-  auto get_map = [&](const void* base, int which, CUtensorMap* out) -> bool {
-    PwPwHost::Key key{base, which};
-    auto it = host->maps.find(key);
+  // X [M][C0] as K-major tiles of 128 rows x 64 channels
+  CUtensorMap mx;
+  {
+    auto it = host->maps.find(inputs[0]);
     if (it == host->maps.end()) {
       CUtensorMap m;
-      const int K = which == 2 ? q.C1 : q.C0;
-      const int rows = which == 0 ? q.M : (which == 1 ? q.C1 : q.C2);
-      const int box_rows = which == 0 ? kBM : (which == 1 ? q.C1p : q.C2p);
-      const uint64_t dims[2] = {(uint64_t)K, (uint64_t)rows};
-      const uint64_t strides[1] = {(uint64_t)K * 2};
-      const uint32_t box[2] = {(uint32_t)kBK, (uint32_t)box_rows};
-      if (!encode_tmap_bf16(&m, base, 2, dims, strides, box, 128, err)) return false;
+      const uint64_t dims[2] = {(uint64_t)q.C0, (uint64_t)q.M};
+      const uint64_t strides[1] = {(uint64_t)q.C0 * 2};
+      const uint32_t box[2] = {(uint32_t)kBK, (uint32_t)kBM};
+      if (!encode_tmap_bf16(&m, inputs[0], 2, dims, strides, box, 128, err)) return AGO_ERR_CUDA;
       if (host->maps.size() > 4096) host->maps.clear();
-      it = host->maps.emplace(key, m).first;
+      it = host->maps.emplace(inputs[0], m).first;
     }
-    *out = it->second;
-    return true;
-  };
-  CUtensorMap mx, mw1, mw2;
-  if (!get_map(inputs[0], 0, &mx) || !get_map(weights[0], 1, &mw1) || !get_map(weights[2], 2, &mw2)) return AGO_ERR_CUDA;
+    mx = it->second;
+  }
   {
     static int smem_opt_in[64] = {};
     cudaError_t e = ensure_max_dynamic_smem(reinterpret_cast<const void*>(pwpw_fused_kernel), smem_opt_in);
     if (e != cudaSuccess) { *err = std::string("cudaFuncSetAttribute: ") + cudaGetErrorString(e); return AGO_ERR_CUDA; }
   }
   FusedLaunch launch(dim3((unsigned)host->grid), kThreads, (size_t)host->smem_bytes, stream);
-  cudaError_t e = cudaLaunchKernelEx(&launch.config, pwpw_fused_kernel, mx, mw1, mw2, q);
+  cudaError_t e = cudaLaunchKernelEx(&launch.config, pwpw_fused_kernel, mx, q);
   if (e != cudaSuccess) { *err = std::string("fused pointwise pair launch: ") + cudaGetErrorString(e); return AGO_ERR_CUDA; }
   return AGO_OK;
 }
