@@ -152,7 +152,19 @@ typedef enum {
 /* Validate the operator list, infer shapes, classify every complex -> complex
  * link into the categories of Section III-B and pick the kernels for the asked
  * mode. Host only; no device work. Returns NULL on failure (ago_last_error
- * tells why). The desc and its ops array are copied. */
+ * tells why). The desc and its ops array are copied.
+ * FUSED mode serves the chains that have a kernel (ago_fused_kernel_t; query
+ * AGO_Q_FUSED_KERNEL) and fails with AGO_ERR_UNSUPPORTED on any other chain or
+ * on shapes outside a kernel's limits -- there is no silent fallback:
+ *   CONV1x1 BIAS RELU6 DW3x3 BIAS RELU6 CONV1x1 BIAS [ADD_INPUT 0]   inverted residual
+ *   CONV1x1 BIAS RELU6 DW3x3 BIAS RELU6 / DW3x3 BIAS RELU6 CONV1x1 BIAS /
+ *   DW3x3 BIAS RELU6 DW3x3 BIAS RELU6 (stride 1) /
+ *   CONV1x1 BIAS [RELU6] CONV1x1 BIAS [RELU6]                        the pairs of Section VI-B
+ *   GEMM BIAS GELU GEMM BIAS                                         feed-forward chain
+ *   CONV3x3 BIAS RELU CONV3x3 BIAS ADD_INPUT 0 RELU                  residual 3x3 pair
+ *   QKT SCALE SOFTMAX PV                                             attention
+ *   DW (any window) followed by simple operators only                depthwise mini-subgraph
+ * (DW3x3: depthwise, 3x3 window, pad 1, stride 1 or 2). */
 ago_subgraph_t ago_subgraph_create(const ago_subgraph_desc_t* desc);
 
 /* Enqueue the subgraph on `cuda_stream` (a cudaStream_t; NULL = the legacy
