@@ -80,7 +80,11 @@ typedef enum {
   AGO_OP_GELU_TANH = 7,   /* 0.5 x (1 + tanh(sqrt(2/pi) (x + 0.044715 x^3)))                  */
   AGO_OP_SCALE = 8,       /* x * f                                                            */
   AGO_OP_SOFTMAX_ROWS = 9,/* softmax over the last dimension                                  */
-  AGO_OP_ADD_INPUT = 10   /* p: input index; + that subgraph input, element-wise (residual)   */
+  AGO_OP_ADD_INPUT = 10,  /* p: input index; + that subgraph input, element-wise (residual)   */
+  /* layout operators (the reshape / transpose runs of attention blocks, Section VI-B) */
+  AGO_OP_RESHAPE = 11,    /* p: rank, d0..d3; same elements in row-major order under a new shape
+                             with the same last dimension: a view, never a launch               */
+  AGO_OP_TRANSPOSE = 12   /* p: axis a, axis b (neither the last): swap two leading dimensions  */
 } ago_op_kind_t;
 
 typedef struct {
@@ -146,7 +150,8 @@ typedef enum {
   AGO_KERNEL_PW_DW = 6,       /* 1x1 conv -> depthwise 3x3                           */
   AGO_KERNEL_DW_PW = 7,       /* depthwise 3x3 -> 1x1 conv                           */
   AGO_KERNEL_DW_DW = 8,       /* depthwise 3x3 -> depthwise 3x3                      */
-  AGO_KERNEL_PW_PW = 9        /* 1x1 conv -> 1x1 conv                                */
+  AGO_KERNEL_PW_PW = 9,       /* 1x1 conv -> 1x1 conv                                */
+  AGO_KERNEL_GEMM_PERMUTE_GEMM = 10 /* GEMM -> + input -> row transpose -> GEMM (reshapes in between) */
 } ago_fused_kernel_t;
 
 /* Validate the operator list, infer shapes, classify every complex -> complex
@@ -163,6 +168,8 @@ typedef enum {
  *   GEMM BIAS GELU GEMM BIAS                                         feed-forward chain
  *   CONV3x3 BIAS RELU CONV3x3 BIAS ADD_INPUT 0 RELU                  residual 3x3 pair
  *   QKT SCALE SOFTMAX PV                                             attention
+ *   GEMM RESHAPE ADD_INPUT RESHAPE TRANSPOSE RESHAPE GEMM RESHAPE    projection chain of a
+ *                                   patch-unfolded attention block (rows permuted between the GEMMs)
  *   DW (any window) followed by simple operators only                depthwise mini-subgraph
  * (DW3x3: depthwise, 3x3 window, pad 1, stride 1 or 2). */
 ago_subgraph_t ago_subgraph_create(const ago_subgraph_desc_t* desc);

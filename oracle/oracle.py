@@ -209,6 +209,21 @@ def batched_pv(p, v, heads: int, head_dim: int) -> np.ndarray:
 # ---- a whole subgraph, operator after operator ------------------------------
 
 
+def reshape(x: np.ndarray, shape) -> np.ndarray:
+    """The same elements in row-major order under a new shape (the layout
+    operators between the matrix multiplications of an attention block,
+    Section VI-B): element i of the flattened tensor stays element i."""
+    flat = np.ascontiguousarray(x).ravel()
+    if int(np.prod(shape)) != flat.size:
+        raise ValueError("reshape: element count changes")
+    return flat.reshape(shape)
+
+
+def transpose(x: np.ndarray, a: int, b: int) -> np.ndarray:
+    """Swap axes a and b: out[..., i_a = u, ..., i_b = v, ...] = x[..., v, ..., u, ...]."""
+    return np.ascontiguousarray(np.swapaxes(x, a, b))
+
+
 def run_chain(ops: Sequence, inputs: Sequence, weights: Sequence,
               return_intermediates: bool = False):
     """Apply ``ops`` in order to ``inputs[0]``; every operator materialises its
@@ -251,6 +266,10 @@ def run_chain(ops: Sequence, inputs: Sequence, weights: Sequence,
             x = softmax_rows(x)
         elif kind == "add_input":
             x = add(x, ins[int(prm["input"])])
+        elif kind == "reshape":
+            x = reshape(x, tuple(int(v) for v in prm["shape"]))
+        elif kind == "transpose":
+            x = transpose(x, int(prm["a"]), int(prm["b"]))
         else:
             raise ValueError(f"unknown operator kind {kind!r}")
         if return_intermediates:

@@ -24,7 +24,8 @@ AGO_MODE_FUSED, AGO_MODE_PER_MINI_SUBGRAPH, AGO_MODE_PER_OP = 0, 1, 2
 MODES = {"fused": AGO_MODE_FUSED, "per_mini_subgraph": AGO_MODE_PER_MINI_SUBGRAPH, "per_op": AGO_MODE_PER_OP}
 
 (AGO_OP_CONV2D, AGO_OP_GEMM, AGO_OP_BATCHED_QKT, AGO_OP_BATCHED_PV, AGO_OP_BIAS_ADD, AGO_OP_RELU,
- AGO_OP_RELU6, AGO_OP_GELU_TANH, AGO_OP_SCALE, AGO_OP_SOFTMAX_ROWS, AGO_OP_ADD_INPUT) = range(11)
+ AGO_OP_RELU6, AGO_OP_GELU_TANH, AGO_OP_SCALE, AGO_OP_SOFTMAX_ROWS, AGO_OP_ADD_INPUT, AGO_OP_RESHAPE,
+ AGO_OP_TRANSPOSE) = range(13)
 
 (AGO_Q_NUM_WEIGHTS, AGO_Q_WEIGHT_BYTES, AGO_Q_OUTPUT_RANK, AGO_Q_OUTPUT_DIM, AGO_Q_OUTPUT_BYTES,
  AGO_Q_FLOPS_TENSOR, AGO_Q_FLOPS_CUDA, AGO_Q_SFU_OPS, AGO_Q_IO_BYTES, AGO_Q_NUM_LINKS, AGO_Q_LINK_CATEGORY,
@@ -32,7 +33,8 @@ MODES = {"fused": AGO_MODE_FUSED, "per_mini_subgraph": AGO_MODE_PER_MINI_SUBGRAP
 
 AGO_LINK_DOWNSTREAM_DEPTHWISE, AGO_LINK_DOWNSTREAM_POINTWISE, AGO_LINK_GENERAL = 1, 2, 3
 (AGO_KERNEL_NONE, AGO_KERNEL_DEPTHWISE, AGO_KERNEL_MBV2_BLOCK, AGO_KERNEL_FFN, AGO_KERNEL_CONV3X3_PAIR,
- AGO_KERNEL_ATTENTION, AGO_KERNEL_PW_DW, AGO_KERNEL_DW_PW, AGO_KERNEL_DW_DW, AGO_KERNEL_PW_PW) = range(10)
+ AGO_KERNEL_ATTENTION, AGO_KERNEL_PW_DW, AGO_KERNEL_DW_PW, AGO_KERNEL_DW_DW, AGO_KERNEL_PW_PW,
+ AGO_KERNEL_GEMM_PERMUTE_GEMM) = range(11)
 
 AGO_MAX_INPUTS, AGO_MAX_RANK, AGO_MAX_OPS = 4, 4, 32
 AGO_STATIC_SCRATCH_BYTES = 4 << 20
@@ -246,7 +248,8 @@ def ago_version() -> str:
 
 _KIND = {"conv2d": AGO_OP_CONV2D, "gemm": AGO_OP_GEMM, "qkt": AGO_OP_BATCHED_QKT, "pv": AGO_OP_BATCHED_PV,
          "bias_add": AGO_OP_BIAS_ADD, "relu": AGO_OP_RELU, "relu6": AGO_OP_RELU6, "gelu_tanh": AGO_OP_GELU_TANH,
-         "scale": AGO_OP_SCALE, "softmax_rows": AGO_OP_SOFTMAX_ROWS, "add_input": AGO_OP_ADD_INPUT}
+         "scale": AGO_OP_SCALE, "softmax_rows": AGO_OP_SOFTMAX_ROWS, "add_input": AGO_OP_ADD_INPUT,
+         "reshape": AGO_OP_RESHAPE, "transpose": AGO_OP_TRANSPOSE}
 
 
 def make_desc(ops, input_shapes, mode="fused", dtype=AGO_BF16):
@@ -263,6 +266,10 @@ def make_desc(ops, input_shapes, mode="fused", dtype=AGO_BF16):
             vals = [prm["input"], prm["heads"], prm["head_dim"]]
         elif kind == "add_input":
             vals = [prm["input"]]
+        elif kind == "reshape":
+            vals = [len(prm["shape"])] + list(prm["shape"])
+        elif kind == "transpose":
+            vals = [prm["a"], prm["b"]]
         else:
             vals = []
         for k, v in enumerate(vals):

@@ -192,6 +192,9 @@ ago_status_t run_unfused(ago_subgraph_s* h, const void* const* inputs, const voi
     if (s.softmax) {
       const Shape& sh = p.ops[s.first].in;
       e = launch_softmax_rows(src, dst, sh.numel() / sh.last(), (int)sh.last(), src_dtype, dst_dtype, stream);
+    } else if (s.transpose) {
+      const OpInfo& o = p.ops[s.first];
+      e = launch_transpose(src, dst, o.in.d, o.in.rank, o.op.p[0], o.op.p[1], src_dtype, dst_dtype, stream);
     } else if (s.complex_index >= 0) {
       EpiProgram epi;
       make_epilogue(p, s.first + 1, s.last, inputs, weights, &epi);

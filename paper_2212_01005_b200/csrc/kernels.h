@@ -52,6 +52,10 @@ cudaError_t launch_elementwise(const void* x, void* y, int64_t numel, int C, int
 cudaError_t launch_softmax_rows(const void* x, void* y, int64_t rows, int cols, int x_dtype, int y_dtype,
                                 cudaStream_t stream);
 
+// y = x with axes a and b (both below the last axis) swapped; x has shape dims[rank], rank <= 4.
+cudaError_t launch_transpose(const void* x, void* y, const int64_t* dims, int rank, int a, int b, int x_dtype, int y_dtype,
+                             cudaStream_t stream);
+
 // 3x3 stride-1 pad-1 convolution with equal channel counts (16, 32 or 64) on tensor cores: the fused pair's kernel
 // restricted to one convolution. out = [relu](conv(x, w) + bias [+ res]); bf16 NHWC / OHWI, bias and res may be null.
 bool conv3x3_tc_supported(int H, int W, int Cin, int Cout, int R, int S, int stride, int pad);

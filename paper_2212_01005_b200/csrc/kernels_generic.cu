@@ -172,7 +172,71 @@ __global__ void __launch_bounds__(256) softmax_rows_kernel(const void* x, void* 
   for (int j = lane; j < cols; j += 32) st(y, base + j, expf(ld(x, base + j, x_dtype) - m) * inv, y_dtype);
 }
 
+// Swap of two leading axes: the last axis moves as whole rows. One thread per VEC elements of an output row
+// (VEC = 16 bytes when both tensors share a storage type and the row length allows it, else 1).
+struct TransposeArgs {
+  int64_t od[4];   // output shape padded to rank 4 in front
+  int64_t is[4];   // input stride (elements) of every OUTPUT axis
+};
+template <int VEC, typename T>
+__global__ void __launch_bounds__(256) transpose_vec_kernel(const T* x, T* y, const TransposeArgs a, int64_t total_vec) {
+  const int64_t gid = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (gid >= total_vec) return;
+  const int64_t cv = a.od[3] / VEC;
+  const int64_t c = (gid % cv) * VEC;
+  int64_t t = gid / cv;
+  const int64_t i2 = t % a.od[2]; t /= a.od[2];
+  const int64_t i1 = t % a.od[1];
+  const int64_t i0 = t / a.od[1];
+  const int64_t src = i0 * a.is[0] + i1 * a.is[1] + i2 * a.is[2] + c;
+  if (VEC * sizeof(T) == 16) {
+    *reinterpret_cast<uint4*>(y + gid * VEC) = __ldg(reinterpret_cast<const uint4*>(x + src));
+  } else {
+    y[gid] = x[src];
+  }
+}
+__global__ void __launch_bounds__(256) transpose_any_kernel(const void* x, void* y, const TransposeArgs a, int64_t total,
+                                                            int x_dtype, int y_dtype) {
+  const int64_t gid = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (gid >= total) return;
+  const int64_t c = gid % a.od[3];
+  int64_t t = gid / a.od[3];
+  const int64_t i2 = t % a.od[2]; t /= a.od[2];
+  const int64_t i1 = t % a.od[1];
+  const int64_t i0 = t / a.od[1];
+  st(y, gid, ld(x, i0 * a.is[0] + i1 * a.is[1] + i2 * a.is[2] + c, x_dtype), y_dtype);
+}
+
 }  // namespace
+
+cudaError_t launch_transpose(const void* x, void* y, const int64_t* dims, int rank, int a, int b, int x_dtype, int y_dtype,
+                             cudaStream_t stream) {
+  if (rank < 3 || rank > 4 || a == b || a < 0 || b < 0 || a >= rank - 1 || b >= rank - 1) return cudaErrorInvalidValue;
+  int64_t id[4] = {1, 1, 1, 1}, istr[4];
+  const int pad = 4 - rank;
+  for (int k = 0; k < rank; ++k) id[pad + k] = dims[k];
+  istr[3] = 1;
+  for (int k = 2; k >= 0; --k) istr[k] = istr[k + 1] * id[k + 1];
+  int perm[4] = {0, 1, 2, 3};
+  perm[pad + a] = pad + b; perm[pad + b] = pad + a;
+  TransposeArgs t;
+  for (int k = 0; k < 4; ++k) { t.od[k] = id[perm[k]]; t.is[k] = istr[perm[k]]; }
+  const int64_t total = id[0] * id[1] * id[2] * id[3];
+  const int esz = x_dtype == AGO_FP32 ? 4 : 2;
+  const int vec = 16 / esz;
+  if (x_dtype == y_dtype && id[3] % vec == 0) {
+    const int64_t tv = total / vec;
+    const unsigned blocks = (unsigned)((tv + 255) / 256);
+    if (esz == 4)
+      transpose_vec_kernel<4, float><<<blocks, 256, 0, stream>>>(static_cast<const float*>(x), static_cast<float*>(y), t, tv);
+    else
+      transpose_vec_kernel<8, __nv_bfloat16><<<blocks, 256, 0, stream>>>(static_cast<const __nv_bfloat16*>(x), static_cast<__nv_bfloat16*>(y), t, tv);
+  } else {
+    const unsigned blocks = (unsigned)((total + 255) / 256);
+    transpose_any_kernel<<<blocks, 256, 0, stream>>>(x, y, t, total, x_dtype, y_dtype);
+  }
+  return cudaGetLastError();
+}
 
 cudaError_t launch_gemm_generic(const GemmArgs& a, cudaStream_t stream) {
   dim3 grid((a.M + TM - 1) / TM, (a.N + TN - 1) / TN, a.batches);

@@ -5,6 +5,7 @@
 
 #include <cstdio>
 #include <cstring>
+#include <utility>
 
 namespace ago {
 
@@ -23,7 +24,7 @@ int64_t out_extent(int64_t H, int64_t R, int64_t stride, int64_t pad) {
 
 bool is_simple_elementwise(int kind) {
   return kind == AGO_OP_BIAS_ADD || kind == AGO_OP_RELU || kind == AGO_OP_RELU6 || kind == AGO_OP_GELU_TANH ||
-         kind == AGO_OP_SCALE || kind == AGO_OP_ADD_INPUT;
+         kind == AGO_OP_SCALE || kind == AGO_OP_ADD_INPUT || kind == AGO_OP_RESHAPE;   // a reshape is a view
 }
 
 // Category of the link whose downstream operator is `down` (Section III-B):
@@ -96,6 +97,13 @@ int match_fused_family(const Plan& p) {
         return AGO_KERNEL_PW_PW;
     }
   }
+  // GEMM -> [M, N1] viewed as [G, A, B, N1] -> + input -> swap (A, B) -> [M, N1] -> GEMM: between the two products
+  // the rows are only permuted
+  if (kinds_are(ops, {AGO_OP_GEMM, AGO_OP_RESHAPE, AGO_OP_ADD_INPUT, AGO_OP_RESHAPE, AGO_OP_TRANSPOSE, AGO_OP_RESHAPE,
+                      AGO_OP_GEMM, AGO_OP_RESHAPE}) &&
+      ops[0].in.rank == 2 && ops[3].out.rank == 4 && ops[4].op.p[0] + ops[4].op.p[1] == 3 && ops[5].out.rank == 2 &&
+      ops[2].op.p[0] == 1)
+    return AGO_KERNEL_GEMM_PERMUTE_GEMM;
   if (kinds_are(ops, {AGO_OP_GEMM, AGO_OP_BIAS_ADD, AGO_OP_GELU_TANH, AGO_OP_GEMM, AGO_OP_BIAS_ADD}))
     return AGO_KERNEL_FFN;
   if (kinds_are(ops, {AGO_OP_CONV2D, AGO_OP_BIAS_ADD, AGO_OP_RELU, AGO_OP_CONV2D, AGO_OP_BIAS_ADD,
@@ -197,6 +205,30 @@ ago_status_t build_plan(const ago_subgraph_desc_t* desc, Plan* plan, std::string
         cur.rank = 3; cur.d[0] = B; cur.d[1] = S; cur.d[2] = heads * hd; cur.d[3] = 0;
         break;
       }
+      case AGO_OP_RESHAPE: {
+        const int r = q[0];
+        if (r < 2 || r > AGO_MAX_RANK) { *err = fmt("op %lld (RESHAPE): rank must be 2..4", i); return AGO_ERR_SHAPE; }
+        Shape nsh; nsh.rank = r;
+        for (int k = 0; k < r; ++k) nsh.d[k] = q[1 + k];
+        for (int k = 0; k < r; ++k)
+          if (nsh.d[k] <= 0) { *err = fmt("op %lld (RESHAPE): dimension %lld must be positive", i, k); return AGO_ERR_SHAPE; }
+        if (nsh.numel() != cur.numel() || nsh.last() != cur.last()) {
+          *err = fmt("op %lld (RESHAPE): the new shape must keep the element count and the last dimension", i);
+          return AGO_ERR_SHAPE;
+        }
+        if (i == 0) { *err = "op 0 (RESHAPE): a reshape must follow an operator"; return AGO_ERR_UNSUPPORTED; }
+        cur = nsh;
+        break;
+      }
+      case AGO_OP_TRANSPOSE: {
+        const int a = q[0], b = q[1];
+        if (a < 0 || b < 0 || a == b || a >= cur.rank - 1 || b >= cur.rank - 1) {
+          *err = fmt("op %lld (TRANSPOSE): two different axes below the last one are required", i);
+          return AGO_ERR_SHAPE;
+        }
+        std::swap(cur.d[a], cur.d[b]);
+        break;
+      }
       case AGO_OP_BIAS_ADD:
         oi.weight = nw++;
         p.weight_bytes.push_back(cur.last() * 4);
@@ -236,9 +268,11 @@ ago_status_t build_plan(const ago_subgraph_desc_t* desc, Plan* plan, std::string
   // Launch list of the unfused modes.
   if (p.mode == AGO_MODE_PER_OP) {
     for (int i = 0; i < (int)p.ops.size(); ++i) {
+      if (p.ops[i].op.kind == AGO_OP_RESHAPE && !p.stages.empty()) { p.stages.back().last = i; continue; }   // a view
       Stage s; s.first = s.last = i;
       s.complex_index = p.ops[i].complex_op() ? i : -1;
       s.softmax = p.ops[i].op.kind == AGO_OP_SOFTMAX_ROWS;
+      s.transpose = p.ops[i].op.kind == AGO_OP_TRANSPOSE;
       p.stages.push_back(s);
     }
   } else {
@@ -248,7 +282,13 @@ ago_status_t build_plan(const ago_subgraph_desc_t* desc, Plan* plan, std::string
     int i = 0, n = (int)p.ops.size();
     while (i < n) {
       Stage s; s.first = i;
-      if (p.ops[i].op.kind == AGO_OP_SOFTMAX_ROWS) { s.softmax = true; s.last = i; ++i; p.stages.push_back(s); continue; }
+      if (p.ops[i].op.kind == AGO_OP_SOFTMAX_ROWS || p.ops[i].op.kind == AGO_OP_TRANSPOSE) {
+        s.softmax = p.ops[i].op.kind == AGO_OP_SOFTMAX_ROWS; s.transpose = !s.softmax;
+        s.last = i; ++i;
+        while (i < n && p.ops[i].op.kind == AGO_OP_RESHAPE) s.last = i++;   // views of its result
+        p.stages.push_back(s);
+        continue;
+      }
       if (p.ops[i].complex_op()) s.complex_index = i;
       int j = i + 1, cnt = p.ops[i].complex_op() ? 0 : 1;
       while (j < n && is_simple_elementwise(p.ops[j].op.kind) && cnt < kMaxEpi) { ++j; ++cnt; }
@@ -265,8 +305,13 @@ ago_status_t build_plan(const ago_subgraph_desc_t* desc, Plan* plan, std::string
   {
     int n = (int)p.ops.size();
     for (int i = 0; i + 1 < n; ++i) {
-      bool boundary = p.ops[i + 1].complex_op() || p.ops[i + 1].op.kind == AGO_OP_SOFTMAX_ROWS ||
-                      p.ops[i].op.kind == AGO_OP_SOFTMAX_ROWS;
+      // launch boundaries of that mode; views on either side of a boundary do not move it
+      int nx = i + 1;
+      while (nx < n && p.ops[nx].op.kind == AGO_OP_RESHAPE) ++nx;
+      if (nx >= n || p.ops[i].op.kind == AGO_OP_RESHAPE) continue;
+      const int kn = p.ops[nx].op.kind, ki = p.ops[i].op.kind;
+      bool boundary = p.ops[nx].complex_op() || kn == AGO_OP_SOFTMAX_ROWS || kn == AGO_OP_TRANSPOSE ||
+                      ki == AGO_OP_SOFTMAX_ROWS || ki == AGO_OP_TRANSPOSE;
       if (boundary) p.intermediate_bytes += 2 * p.ops[i].out.numel() * elem_bytes(p.dtype);
     }
   }
@@ -281,7 +326,8 @@ ago_status_t build_plan(const ago_subgraph_desc_t* desc, Plan* plan, std::string
     p.fused_kernel = match_fused_family(p);
     if (p.fused_kernel == AGO_KERNEL_NONE) {
       *err = "fused mode: the operator chain matches no fused kernel family (depthwise-only; 1x1 -> depthwise 3x3 -> 1x1 "
-             "and its pairs; GEMM -> GELU -> GEMM; conv3x3 -> conv3x3 + input -> ReLU; QK^T -> scale -> softmax -> PV)";
+             "and its pairs; GEMM -> GELU -> GEMM; conv3x3 -> conv3x3 + input -> ReLU; QK^T -> scale -> softmax -> PV; "
+             "GEMM -> + input -> row transpose -> GEMM)";
       return AGO_ERR_UNSUPPORTED;
     }
     p.num_launches = 1;

@@ -44,6 +44,7 @@ struct Stage {
   int first = 0, last = 0;
   int complex_index = -1;  // index of the complex op (== first) or -1 for a simple-only stage
   bool softmax = false;    // a SOFTMAX_ROWS launch
+  bool transpose = false;  // a TRANSPOSE launch
 };
 
 // Element-wise operator program executed in a kernel epilogue (conventional

@@ -95,6 +95,10 @@ class Workload:
                 shp = (B, S_, p["heads"] * p["head_dim"])
             elif kind == "bias_add":
                 ws.append((shp[-1],)); kinds.append("bias"); fans.append(1)
+            elif kind == "reshape":
+                shp = tuple(p["shape"])
+            elif kind == "transpose":
+                l = list(shp); l[p["a"]], l[p["b"]] = l[p["b"]], l[p["a"]]; shp = tuple(l)
         self.weight_shapes, self.weight_kinds, self.weight_fan_in = ws, kinds, fans
         self.output_shape = shp
 
@@ -181,6 +185,18 @@ def pw_pw(name, seed_seq, N, H, c_in, c_mid, c_out, act1=False, act2=True) -> Wo
     return Workload(name, seed_seq, [(N, H, H, c_in)], ops, samples=N, input_dist=["relu_normal"])
 
 
+def unfold_chain(name, seed_seq, B, P, N, d, d_out) -> Workload:
+    """Two projections of a patch-unfolded attention block (MobileViT-like: B images, P pixels per patch, N patches,
+    d channels) with the layout operators between them: matrix multiplication, reshape, add, reshape, transpose,
+    reshape, matrix multiplication, reshape (Section VI-B). Rows are (image, pixel, patch) before the transpose and
+    (image, patch, pixel) after it."""
+    M = B * P * N
+    ops = [("gemm", dict(N=d)), ("reshape", dict(shape=(B * P, N, d))), ("add_input", dict(input=1)),
+           ("reshape", dict(shape=(B, P, N, d))), ("transpose", dict(a=1, b=2)), ("reshape", dict(shape=(M, d))),
+           ("gemm", dict(N=d_out)), ("reshape", dict(shape=(B, N, P, d_out)))]
+    return Workload(name, seed_seq, [(M, d), (B * P, N, d)], ops, samples=B, input_dist=["normal", "normal"])
+
+
 def get(name: str, batch: int | None = None) -> Workload:
     """The benchmark configurations. ``batch`` overrides the number of
     independent samples (images, sequences) while keeping per-sample shapes."""
@@ -208,6 +224,8 @@ def get(name: str, batch: int | None = None) -> Workload:
         return dw_dw(name, [5, 2], batch or 32, 56, 144)
     if name == "pw_pw_56":
         return pw_pw(name, [5, 3], batch or 32, 56, 144, 24, 144)
+    if name == "unfold_96":      # d = 96, 2 x 2 patches of a 32 x 32 feature map, expansion to 2 d
+        return unfold_chain(name, [6], batch or 32, 4, 256, 96, 192)
     raise KeyError(name)
 
 
@@ -285,4 +303,8 @@ def flops(wl: Workload) -> Dict[str, float]:
             shp = (B, S_, p["heads"] * p["head_dim"])
         elif kind in ("gelu_tanh", "softmax_rows"):
             sfu += float(np.prod(shp))
+        elif kind == "reshape":
+            shp = tuple(p["shape"])
+        elif kind == "transpose":
+            l = list(shp); l[p["a"]], l[p["b"]] = l[p["b"]], l[p["a"]]; shp = tuple(l)
     return {"tensor": tensor, "cuda": cuda, "sfu": sfu}

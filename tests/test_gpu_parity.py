@@ -136,6 +136,23 @@ def test_fused_agrees_with_unfused_chain(ago, name):
     assert float(np.max(np.abs(fused - mini))) <= 2e-2 * scale + 1e-3
 
 
+UNFOLD_SMALL = {
+    "unfold_small": lambda: WL.unfold_chain("unfold_small", [101], 2, 4, 64, 96, 192),      # 512 rows
+    "unfold_ragged": lambda: WL.unfold_chain("unfold_ragged", [102], 3, 4, 25, 64, 128),    # 300 rows: ragged last tile
+    "unfold_narrow": lambda: WL.unfold_chain("unfold_narrow", [103], 1, 9, 49, 24, 40),     # channel counts 8 mod 16
+    "unfold_wide": lambda: WL.unfold_chain("unfold_wide", [104], 2, 4, 16, 144, 256),
+}
+
+
+@pytest.mark.parametrize("mode", UNFUSED)
+@pytest.mark.parametrize("name", list(UNFOLD_SMALL.keys()))
+def test_unfold_chain_unfused_modes_match_oracle(ago, name, mode):
+    wl = UNFOLD_SMALL[name]()
+    data = WL.generate(wl)
+    ref = O.run_chain(wl.ops, data["inputs"], data["weights"])
+    assert_close(run_gpu(ago, wl, data, mode), ref, what=f"{name}/{mode}")
+
+
 PAIR_SMALL = {
     "pw_dw_s1": lambda: WL.pw_dw("pw_dw_s1", [81], 2, 14, 32, 192, 1),
     "pw_dw_s1_odd": lambda: WL.pw_dw("pw_dw_s1_odd", [82], 3, 13, 24, 144, 1),

@@ -312,6 +312,51 @@ def test_attention_chain_against_torch():
     np.testing.assert_allclose(y, ref.numpy(), rtol=0, atol=1e-13)
 
 
+# ---- layout operators and the chain around them (Section VI-B) ---------------------
+
+
+def test_transpose_matches_hand_written_example_and_is_an_involution():
+    x = np.arange(12, dtype=np.float64).reshape(2, 3, 2)
+    want = np.loadtxt(os.path.join(GOLDEN, "transpose_2x3x2.txt")).reshape(3, 2, 2)
+    got = O.transpose(x, 0, 1)
+    assert got.shape == (3, 2, 2) and np.array_equal(got, want)
+    y = rng.standard_normal((2, 3, 4, 5))
+    assert np.array_equal(O.transpose(O.transpose(y, 1, 2), 1, 2), y)
+    assert O.transpose(y, 1, 2)[1, 3, 2, 4] == y[1, 2, 3, 4]
+    assert O.transpose(y, 0, 2)[3, 1, 0, 2] == y[0, 1, 3, 2]
+
+
+def test_reshape_keeps_row_major_order():
+    x = rng.standard_normal((4, 6, 5))
+    r = O.reshape(x, (2, 2, 6, 5))
+    assert r[1, 0, 3, 2] == x[2, 3, 2] and r[0, 1, 5, 4] == x[1, 5, 4]
+    assert np.array_equal(O.reshape(r, (24, 5)).ravel(), x.ravel())
+    with pytest.raises(ValueError):
+        O.reshape(x, (4, 6, 4))
+
+
+def test_unfold_chain_against_element_by_element_definition():
+    # matmul, reshape, add, reshape, transpose, reshape, matmul, reshape: rows are (image, pixel, patch) before the
+    # transpose and (image, patch, pixel) after it; written out with explicit indices, no reshape or transpose
+    B, P, N, d, d2 = 2, 3, 4, 5, 6
+    M = B * P * N
+    x = rng.standard_normal((M, d)); r = rng.standard_normal((B * P, N, d))
+    w1 = rng.standard_normal((d, d)); w2 = rng.standard_normal((d, d2))
+    ops = [("gemm", dict(N=d)), ("reshape", dict(shape=(B * P, N, d))), ("add_input", dict(input=1)),
+           ("reshape", dict(shape=(B, P, N, d))), ("transpose", dict(a=1, b=2)), ("reshape", dict(shape=(M, d))),
+           ("gemm", dict(N=d2)), ("reshape", dict(shape=(B, N, P, d2)))]
+    got = O.run_chain(ops, [x, r], [w1, w2])
+    assert got.shape == (B, N, P, d2)
+    for b in range(B):
+        for p in range(P):
+            for n in range(N):
+                row = (b * P + p) * N + n
+                mid = [sum(x[row, k] * w1[k, j] for k in range(d)) + r[b * P + p, n, j] for j in range(d)]
+                for o in range(d2):
+                    want = sum(mid[j] * w2[j, o] for j in range(d))
+                    assert abs(got[b, n, p, o] - want) <= 1e-12 * max(1.0, abs(want))
+
+
 def test_run_chain_rejects_unconsumed_weights():
     with pytest.raises(ValueError):
         O.run_chain([("relu", {})], [np.zeros(3)], [np.zeros(3)])
