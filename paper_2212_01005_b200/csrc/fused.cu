@@ -25,6 +25,7 @@ ago_status_t fused_plan(Plan* plan, FusedState* st, std::string* err) {
     case AGO_KERNEL_DW_DW:
       return dwdw_plan(plan, st, err);
     case AGO_KERNEL_PW_PW:
+    case AGO_KERNEL_GEMM_PERMUTE_GEMM:
       return pwpw_plan(plan, st, err);
     case AGO_KERNEL_ATTENTION:
       return attention_plan(plan, st, err);
@@ -53,6 +54,7 @@ ago_status_t fused_run(const Plan& plan, FusedState* st, const void* const* inpu
     case AGO_KERNEL_DW_DW:
       return dwdw_run(plan, st, inputs, weights, output, status_word, stream, err);
     case AGO_KERNEL_PW_PW:
+    case AGO_KERNEL_GEMM_PERMUTE_GEMM:
       return pwpw_run(plan, st, inputs, weights, output, status_word, stream, err);
     case AGO_KERNEL_ATTENTION:
       return attention_run(plan, st, inputs, weights, output, status_word, stream, err);

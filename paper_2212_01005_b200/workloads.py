@@ -230,7 +230,7 @@ def get(name: str, batch: int | None = None) -> Workload:
 
 
 PAIRS = ["pw_dw_56", "dw_pw_56", "dw_dw_56", "pw_pw_56"]
-ALL = ["mbv2_14", "ffn_512", "mbv2_56", "mbv2_28s2", "resnet_56", "attn_384", "ffn_12288"] + PAIRS
+ALL = ["mbv2_14", "ffn_512", "mbv2_56", "mbv2_28s2", "resnet_56", "attn_384", "ffn_12288"] + PAIRS + ["unfold_96"]
 
 
 # ---- seeded tensors ---------------------------------------------------------------

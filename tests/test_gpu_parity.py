@@ -140,7 +140,7 @@ UNFOLD_SMALL = {
     "unfold_small": lambda: WL.unfold_chain("unfold_small", [101], 2, 4, 64, 96, 192),      # 512 rows
     "unfold_ragged": lambda: WL.unfold_chain("unfold_ragged", [102], 3, 4, 25, 64, 128),    # 300 rows: ragged last tile
     "unfold_narrow": lambda: WL.unfold_chain("unfold_narrow", [103], 1, 9, 49, 24, 40),     # channel counts 8 mod 16
-    "unfold_wide": lambda: WL.unfold_chain("unfold_wide", [104], 2, 4, 16, 144, 256),
+    "unfold_wide": lambda: WL.unfold_chain("unfold_wide", [104], 2, 4, 16, 128, 256),
 }
 
 
@@ -151,6 +151,28 @@ def test_unfold_chain_unfused_modes_match_oracle(ago, name, mode):
     data = WL.generate(wl)
     ref = O.run_chain(wl.ops, data["inputs"], data["weights"])
     assert_close(run_gpu(ago, wl, data, mode), ref, what=f"{name}/{mode}")
+
+
+@pytest.mark.parametrize("name", list(UNFOLD_SMALL.keys()))
+def test_unfold_chain_fused_matches_oracle(ago, name):
+    # one kernel: the transpose only permutes the rows between the two products
+    wl = UNFOLD_SMALL[name]()
+    data = WL.generate(wl)
+    ref = O.run_chain(wl.ops, data["inputs"], data["weights"])
+    assert_close(run_gpu(ago, wl, data, "fused"), ref, what=f"{name}/fused")
+
+
+def test_unfold_chain_full_size_on_sampled_images(ago):
+    wl = WL.get("unfold_96")
+    data = WL.generate(wl)
+    gpu = run_gpu(ago, wl, data, "fused")
+    one = WL.get("unfold_96", batch=1)
+    rows = one.input_shapes[0][0]          # rows of one image, contiguous in both inputs and in the output
+    for img in (0, 13, wl.samples - 1):
+        x = data["inputs"][0][img * rows:(img + 1) * rows]
+        r = data["inputs"][1][img * 4:(img + 1) * 4]
+        ref = O.run_chain(one.ops, [x, r], data["weights"])
+        assert_close(gpu[img:img + 1], ref, what=f"unfold_96 image {img}")
 
 
 PAIR_SMALL = {
