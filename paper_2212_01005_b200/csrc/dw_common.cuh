@@ -11,8 +11,8 @@ namespace dw {
 // bf16x2(min(max(lo, 0), 6), min(max(hi, 0), 6)): the conversion clamps at 0, one packed min caps at 6.
 __device__ __forceinline__ uint32_t relu6_pack(float lo, float hi) {
   uint32_t r;
-  asm("{\n\t.reg .b32 t, six;\n\tmov.b32 six, 0x40C040C0;\n\tcvt.rn.relu.bf16x2.f32 t, %2, %1;\n\tmin.bf16x2 %0, t, six;\n\t}"
-      : "=r"(r) : "f"(lo), "f"(hi));
+  asm("{\n\t.reg .b32 t;\n\tcvt.rn.relu.bf16x2.f32 t, %2, %1;\n\tmin.bf16x2 %0, t, %3;\n\t}"
+      : "=r"(r) : "f"(lo), "f"(hi), "r"(0x40C040C0u));   // the packed 6.0 is an operand, so one register serves every call
   return r;
 }
 

@@ -68,13 +68,24 @@ struct Mbv2Params {
   int Kp, row_bytes, swizzle;   // input / W1 tiles: padded K, bytes per row, tc::SwizzleMode
   int Coutp, NC;
   // 2^32 / d + 1 for the run-time divisors of the index arithmetic: x / d == __umulhi(x, recip) for x, d < 65536
-  uint32_t coutp_recip, w_recip, strips_recip, per_row_recip;
+  uint32_t coutp_recip, w_recip, strips_recip, per_row_recip, cexp8_recip;   // cexp8: Cexp / 8 (>= 2)
   int per_row, nseg, step_r, step_c, col_slots;   // depthwise item geometry (see the kernel), fixed per shape
   int tmem_cols, ecol0, pcol0;
   int e_plane, d_plane;         // byte distance between the two 8-channel planes of an E / D chunk
   // shared-memory byte offsets (from the 1024-aligned base)
   int off_x, off_w1, off_e, off_d, off_w3, off_wd, off_b1, off_bd, off_b3, off_bar;
 };
+
+// 16-byte shared-memory accesses by 32-bit shared address (immediate byte offset for the load).
+template <int OFF>
+__device__ __forceinline__ float4 lds128f(uint32_t saddr) {
+  float4 v;
+  asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4+%5];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(saddr), "n"(OFF));
+  return v;
+}
+__device__ __forceinline__ void sts128(uint32_t saddr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+  asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(saddr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
+}
 
 // EXPAND / PROJECT select the pairs of the block: <true, true> the whole block, <true, false> pointwise -> depthwise
 // (the depthwise result of every chunk goes to device memory), <false, true> depthwise -> pointwise (every chunk of
@@ -89,7 +100,7 @@ mbv2_fused_kernel(const Mbv2Params p) {
   uint8_t* sE = smem + p.off_e;
   uint8_t* sD = smem + p.off_d;
   uint8_t* sW3 = smem + p.off_w3;
-  const uint8_t* sWd = smem + p.off_wd;                   // [9][Cexp] bf16, as in device memory
+  const uint8_t* sWd = smem + p.off_wd;                   // [chunk][9 taps][16 channels] bf16
   float* sB1 = reinterpret_cast<float*>(smem + p.off_b1);
   float* sBd = reinterpret_cast<float*>(smem + p.off_bd);
   float* sB3 = reinterpret_cast<float*>(smem + p.off_b3);
@@ -153,7 +164,11 @@ mbv2_fused_kernel(const Mbv2Params p) {
         src = row < (uint32_t)p.Cout ? reinterpret_cast<const uint8_t*>(p.w3) + (row * p.Cexp + c * kChunk + half * 8u) * 2u : nullptr;
         return p.off_w3 + c * p.Coutp * kChunkRowBytes + swz_offset(row, half, kChunkRowBytes);
       }
-      if ((i -= nW3) < nWd) { src = reinterpret_cast<const uint8_t*>(p.wd) + i * 16u; return p.off_wd + i * 16u; }
+      if ((i -= nW3) < nWd) {   // [tap][Cexp] in device memory -> [chunk][tap][16 channels]: a thread's nine taps lie 32 bytes apart
+        const uint32_t tap = __umulhi(i, p.cexp8_recip), c8 = i - tap * ((uint32_t)p.Cexp >> 3);
+        src = reinterpret_cast<const uint8_t*>(p.wd) + i * 16u;
+        return p.off_wd + (c8 >> 1) * (9u * kChunkRowBytes) + tap * kChunkRowBytes + (c8 & 1u) * 16u;
+      }
       if ((i -= nWd) < nB1) { src = reinterpret_cast<const uint8_t*>(p.b1) + i * 16u; return p.off_b1 + i * 16u; }
       if ((i -= nB1) < nB) { src = reinterpret_cast<const uint8_t*>(p.bd) + i * 16u; return p.off_bd + i * 16u; }
       i -= nB;
@@ -196,7 +211,8 @@ mbv2_fused_kernel(const Mbv2Params p) {
     const int q_first = (((warp & 3) - gwarp0) & 3);                // group-relative index of the quarter's first warp
     const int q_mates = (kGroupWarps - q_first + 3) >> 2;           // warps of this quarter in the group (3 or 4)
     const int q_rank = (warp - gwarp0 - q_first) >> 2;              // this warp's rank among them
-    int e_pix[kTilesPerWarp];
+    constexpr uint32_t kNone = 0xffffffffu;
+    uint32_t e_off[kTilesPerWarp];   // shared-memory address of the thread's pixel in plane 0 of the group's E buffer
     uint32_t e_inimg = 0;
 #pragma unroll
     for (int k = 0; k < kTilesPerWarp; ++k) {
@@ -204,9 +220,9 @@ mbv2_fused_kernel(const Mbv2Params p) {
       const int pix = t * 128 + (warp & 3) * 32 + lane;
       const int ih = (int)fast_div((uint32_t)pix, (uint32_t)p.W, p.w_recip), iw = pix - ih * p.W;
       const int gh = gh0 + ih;
-      e_pix[k] = -1;
+      e_off[k] = kNone;
       if (t < p.M1 && pix < p.P_x) {
-        e_pix[k] = ih * p.IW + iw + 1;
+        e_off[k] = smem_u32(sE) + (uint32_t)(g * e_bytes + (ih * p.IW + iw + 1) * 16);
         if (gh >= 0 && gh < p.H) e_inimg |= 1u << k;
       }
     }
@@ -274,6 +290,12 @@ mbv2_fused_kernel(const Mbv2Params p) {
     // may overwrite its operand.
     // Descriptors as (low, high) words: start address and LBO live in the low word, so an operand advances with one
     // 32-bit add (shared-memory addresses >> 4 stay below the 14-bit field limit).
+    uint32_t e_tm[kTilesPerWarp];   // tensor-memory address of this warp's k-th expand tile (buffer g)
+#pragma unroll
+    for (int k = 0; k < kTilesPerWarp; ++k) {
+      const int t = q_rank + k * q_mates;
+      e_tm[k] = t < p.M1 ? tmem_base + lane_base + p.ecol0 + (g * p.M1 + t) * kChunk : kNone;
+    }
     const uint32_t sbo_x = 8u * (uint32_t)p.row_bytes;
     const uint64_t xdesc0 = make_smem_desc(smem_u32(sX), 0, sbo_x, p.swizzle);
     const uint64_t w1desc0 = make_smem_desc(smem_u32(sW1), 0, sbo_x, p.swizzle);
@@ -353,37 +375,56 @@ mbv2_fused_kernel(const Mbv2Params p) {
       cp_async_commit();
     };
     if (!EXPAND) { load_chunk(g, 0); load_chunk(g + 2, 1); }
+    // The thread's first depthwise item (for most shapes its only one) is the same for every chunk: offsets of its
+    // first input / output pixel inside a plane and its extent (stride 1: columns, rows; stride 2: first and last row).
+    const bool has_item = slot < dw_items;
+    uint32_t it_e, it_d; int it_a, it_b;
+    if (p.stride == 1) {
+      const int wo = item0_c * kSegCols;
+      it_e = (uint32_t)(2 * item0_r) * e_pitch + wo * 16; it_d = (uint32_t)(2 * item0_r) * d_pitch + wo * 16;
+      it_a = min(kSegCols, p.Wo - wo); it_b = min(2, rows_valid - 2 * item0_r);
+    } else {
+      it_e = item0_c * 32; it_d = item0_c * 16;
+      it_a = item0_r * rows_per_group; it_b = min(rows_valid, it_a + rows_per_group);
+    }
+    const uint32_t e_plane0 = smem_u32(sE) + (uint32_t)((EXPAND ? g : g * 2) * e_bytes + (cp >> 2) * p.e_plane + cp_off);
+    const uint32_t d_plane = smem_u32(sD) + (uint32_t)(g * d_bytes + (cp >> 2) * p.d_plane + cp_off);
+    // running shared-memory addresses of this thread's depthwise weights / bias and of the chunk's expand bias
+    uint32_t wd_addr = smem_u32(sWd) + (uint32_t)(g * 9 * kChunkRowBytes + cp * 4);
+    uint32_t bd_addr = smem_u32(sBd) + (uint32_t)((g * kChunk + cp * 2) * 4);
+    uint32_t b1_addr = smem_u32(sB1) + (uint32_t)(g * kChunk * 4);
     for (int c = g, it = 0; c < p.NC; c += 2, ++it) {
       // ---- P3: expand epilogue of chunk c -> E[g]: + b1, ReLU6, zero outside the image, bf16 ----
       if (!EXPAND) cp_async_wait_but_one();   // this thread's pieces of chunk c have landed
       if (EXPAND) {
       tcgen05_fence_after_sync();
-      uint8_t* e_buf = sE + g * e_bytes;
 #pragma unroll
       for (int k = 0; k < kTilesPerWarp; ++k) {
-        const int t = q_rank + k * q_mates;
-        if (t >= p.M1) break;
+        if (e_tm[k] == kNone) break;   // warp-uniform
         uint32_t acc[16];
-        tmem_ld_x16(tmem_base + lane_base + p.ecol0 + (g * p.M1 + t) * kChunk, acc);
+        tmem_ld_x16(e_tm[k], acc);
         tmem_ld_wait();
-        if (e_pix[k] >= 0) {
+        if (e_off[k] != kNone) {
           uint32_t w[8];
           if ((e_inimg >> k) & 1u) {
-            const float4* bb = reinterpret_cast<const float4*>(sB1 + c * kChunk);
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-              const float4 bv = bb[j];
-              w[2 * j] = relu6_pack(__uint_as_float(acc[4 * j]) + bv.x, __uint_as_float(acc[4 * j + 1]) + bv.y);
-              w[2 * j + 1] = relu6_pack(__uint_as_float(acc[4 * j + 2]) + bv.z, __uint_as_float(acc[4 * j + 3]) + bv.w);
-            }
+            const float4 b0 = lds128f<0>(b1_addr), b1v = lds128f<16>(b1_addr), b2 = lds128f<32>(b1_addr), b3v = lds128f<48>(b1_addr);
+            w[0] = relu6_pack(__uint_as_float(acc[0]) + b0.x, __uint_as_float(acc[1]) + b0.y);
+            w[1] = relu6_pack(__uint_as_float(acc[2]) + b0.z, __uint_as_float(acc[3]) + b0.w);
+            w[2] = relu6_pack(__uint_as_float(acc[4]) + b1v.x, __uint_as_float(acc[5]) + b1v.y);
+            w[3] = relu6_pack(__uint_as_float(acc[6]) + b1v.z, __uint_as_float(acc[7]) + b1v.w);
+            w[4] = relu6_pack(__uint_as_float(acc[8]) + b2.x, __uint_as_float(acc[9]) + b2.y);
+            w[5] = relu6_pack(__uint_as_float(acc[10]) + b2.z, __uint_as_float(acc[11]) + b2.w);
+            w[6] = relu6_pack(__uint_as_float(acc[12]) + b3v.x, __uint_as_float(acc[13]) + b3v.y);
+            w[7] = relu6_pack(__uint_as_float(acc[14]) + b3v.z, __uint_as_float(acc[15]) + b3v.w);
           } else {
 #pragma unroll
             for (int j = 0; j < 8; ++j) w[j] = 0u;
           }
-          *reinterpret_cast<uint4*>(e_buf + e_pix[k] * 16) = make_uint4(w[0], w[1], w[2], w[3]);
-          *reinterpret_cast<uint4*>(e_buf + p.e_plane + e_pix[k] * 16) = make_uint4(w[4], w[5], w[6], w[7]);
+          sts128(e_off[k], w[0], w[1], w[2], w[3]);
+          sts128(e_off[k] + (uint32_t)p.e_plane, w[4], w[5], w[6], w[7]);
         }
       }
+      b1_addr += 2u * kChunk * 4u;
       tcgen05_fence_before_sync();
       }
       // D[g] was read by the project GEMM of chunk c - 2
@@ -399,25 +440,32 @@ mbv2_fused_kernel(const Mbv2Params p) {
 
       // ---- P4: depthwise 3x3 + bias + ReLU6 on CUDA cores: E[g] -> D[g] (A operand of the project GEMM) ----
       {
-        const int ch = c * kChunk + cp * 2;
         uint32_t wgt[9];   // packed bf16 pairs
-#pragma unroll
-        for (int tap = 0; tap < 9; ++tap) wgt[tap] = *reinterpret_cast<const uint32_t*>(sWd + (tap * p.Cexp + ch) * 2);
-        const float2 bias = *reinterpret_cast<const float2*>(sBd + ch);
-        const uint32_t e_plane = smem_u32(sE) + (uint32_t)((EXPAND ? g : g * 2 + (it & 1)) * e_bytes + (cp >> 2) * p.e_plane + cp_off);
-        const uint32_t d_plane = smem_u32(sD) + (uint32_t)(g * d_bytes + (cp >> 2) * p.d_plane + cp_off);
-        int r = item0_r, col = item0_c;
-        for (int item = slot; item < dw_items; item += kSlots) {
-          if (p.stride == 1) {
-            const int wo = col * kSegCols;
-            depthwise_block(e_plane + (uint32_t)(2 * r) * e_pitch + wo * 16, d_plane + (uint32_t)(2 * r) * d_pitch + wo * 16, e_pitch,
-                            d_pitch, min(kSegCols, p.Wo - wo), min(2, rows_valid - 2 * r), wgt, bias);
-          } else {
-            const int r0 = r * rows_per_group, r1 = min(rows_valid, r0 + rows_per_group);
-            if (r0 < r1) depthwise_column_s2(e_plane + col * 32, d_plane + col * 16, r0, r1, p.IW, p.Wo, wgt, bias);
-          }
-          r += step_r; col += step_c;
+        wgt[0] = lds32<0>(wd_addr); wgt[1] = lds32<32>(wd_addr); wgt[2] = lds32<64>(wd_addr);
+        wgt[3] = lds32<96>(wd_addr); wgt[4] = lds32<128>(wd_addr); wgt[5] = lds32<160>(wd_addr);
+        wgt[6] = lds32<192>(wd_addr); wgt[7] = lds32<224>(wd_addr); wgt[8] = lds32<256>(wd_addr);
+        const float2 bias = make_float2(__uint_as_float(lds32<0>(bd_addr)), __uint_as_float(lds32<4>(bd_addr)));
+        wd_addr += 2u * 9u * kChunkRowBytes; bd_addr += 2u * kChunk * 4u;   // the group's next chunk is c + 2
+        const uint32_t e_plane = e_plane0 + (EXPAND ? 0u : (uint32_t)((it & 1) * e_bytes));
+        if (has_item) {   // the thread's first item: geometry fixed before the chunk loop
+          if (p.stride == 1) depthwise_block(e_plane + it_e, d_plane + it_d, e_pitch, d_pitch, it_a, it_b, wgt, bias);
+          else if (it_a < it_b) depthwise_column_s2(e_plane + it_e, d_plane + it_d, it_a, it_b, p.IW, p.Wo, wgt, bias);
+        }
+        if (dw_items > kSlots) {   // shapes with more items than slots
+          int r = item0_r + step_r, col = item0_c + step_c;
           if (col >= per_row) { col -= per_row; ++r; }
+          for (int item = slot + kSlots; item < dw_items; item += kSlots) {
+            if (p.stride == 1) {
+              const int wo = col * kSegCols;
+              depthwise_block(e_plane + (uint32_t)(2 * r) * e_pitch + wo * 16, d_plane + (uint32_t)(2 * r) * d_pitch + wo * 16, e_pitch,
+                              d_pitch, min(kSegCols, p.Wo - wo), min(2, rows_valid - 2 * r), wgt, bias);
+            } else {
+              const int r0 = r * rows_per_group, r1 = min(rows_valid, r0 + rows_per_group);
+              if (r0 < r1) depthwise_column_s2(e_plane + col * 32, d_plane + col * 16, r0, r1, p.IW, p.Wo, wgt, bias);
+            }
+            r += step_r; col += step_c;
+            if (col >= per_row) { col -= per_row; ++r; }
+          }
         }
       }
       fence_proxy_async_smem();
@@ -568,6 +616,7 @@ ago_status_t mbv2_plan(Plan* plan, FusedState* st, std::string* err) {
   auto recip = [](int d) { return tc::fast_div_recip(d); };
   q.coutp_recip = recip(q.Coutp);
   q.w_recip = recip(q.W);
+  q.cexp8_recip = recip(q.Cexp / 8);
   {
     constexpr int kSlots = kGroupThreads / 8;
     q.nseg = (q.Wo + kSegCols - 1) / kSegCols;
