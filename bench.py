@@ -38,10 +38,15 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu
 # captures summarised under profiles/ (None until a capture exists for that workload and mode).
 NCU_TRAFFIC_BYTES = {
-    ("mbv2_56", "fused"): 4893696 + 0,            # profiles/mbv2_fused_kernel__mbv2_56.txt (output still dirty in L2)
-    ("attn_384", "fused"): 56695296 + 751104,     # profiles/attention_fused_kernel__attn_384.txt
-    ("resnet_56", "fused"): 13328384 + 2048,      # profiles/conv3x3_pair_kernel__resnet_56.txt
-    ("ffn_12288", "fused"): 66140928 + 9042688,   # profiles/ffn_fused_kernel__ffn_12288.txt
+    ("mbv2_56", "fused"): 4904192 + 0,            # profiles/mbv2_fused_kernel__mbv2_56.txt (output still dirty in L2)
+    ("attn_384", "fused"): 56694784 + 719104,     # profiles/attention_fused_kernel__attn_384.txt
+    ("resnet_56", "fused"): 13311744 + 3840,      # profiles/conv3x3_pair_kernel__resnet_56.txt
+    ("ffn_12288", "fused"): 66143488 + 9655552,   # profiles/ffn_fused_kernel__ffn_12288.txt
+    ("pw_dw_56", "fused"): 4894464 + 5120,        # profiles/mbv2_fused_kernel__pw_dw_56.txt
+    ("dw_pw_56", "fused"): 28972032 + 512,        # profiles/mbv2_fused_kernel__dw_pw_56.txt
+    ("dw_dw_56", "fused"): 28978432 + 962560,     # profiles/dwdw_fused_kernel__dw_dw_56.txt
+    ("pw_pw_56", "fused"): 28948736 + 35584,      # profiles/pwpw_fused_kernel__pw_pw_56.txt
+    ("unfold_96", "fused"): 12670976 + 0,         # profiles/pwpw_fused_kernel__unfold_96.txt
 }
 
 
