@@ -83,6 +83,51 @@ def test_launch_counts_per_mode():
     assert mini.query(B.AGO_Q_INTERMEDIATE_BYTES) == 2 * 2 * 12 * 384 * 384 * 2
 
 
+def test_fused_planner_matches_every_chain_family_and_its_limits():
+    # plan-time only: which kernel the fused mode picks, and what it refuses (no silent fallback)
+    want = {"mbv2_56": B.AGO_KERNEL_MBV2_BLOCK, "mbv2_28s2": B.AGO_KERNEL_MBV2_BLOCK, "ffn_512": B.AGO_KERNEL_FFN,
+            "resnet_56": B.AGO_KERNEL_CONV3X3_PAIR, "attn_384": B.AGO_KERNEL_ATTENTION, "pw_dw_56": B.AGO_KERNEL_PW_DW,
+            "dw_pw_56": B.AGO_KERNEL_DW_PW, "dw_dw_56": B.AGO_KERNEL_DW_DW, "pw_pw_56": B.AGO_KERNEL_PW_PW,
+            "unfold_96": B.AGO_KERNEL_GEMM_PERMUTE_GEMM}
+    for name, kernel in want.items():
+        wl = WL.get(name)
+        sg = B.Subgraph(wl.ops, wl.input_shapes, mode="fused")
+        assert sg.query(B.AGO_Q_FUSED_KERNEL) == kernel, name
+        assert sg.query(B.AGO_Q_NUM_LAUNCHES) == 1
+        assert 0 < sg.query(B.AGO_Q_SMEM_BYTES) <= 227 * 1024 and sg.query(B.AGO_Q_TILE_ROWS) >= 1
+        sg.close()
+    # the two depthwise convolutions of the pair kernel are stride 1; a strided pair has no kernel
+    wl = WL.dw_dw("x", [1], 1, 8, 16)
+    ops = list(wl.ops); ops[3] = ("conv2d", dict(O=16, R=3, S=3, stride=2, pad=1, groups=16))
+    _expect_fail(ops, wl.input_shapes, B.AGO_ERR_UNSUPPORTED, mode="fused", needle="family")
+    # pointwise pair: more middle channels than tensor memory holds
+    wl = WL.pw_pw("x", [1], 1, 8, 64, 512, 64)
+    _expect_fail(wl.ops, wl.input_shapes, B.AGO_ERR_UNSUPPORTED, mode="fused", needle="256")
+    # a transpose of other axes than the two middle ones is not a row permutation the chain kernel knows
+    wl = WL.unfold_chain("x", [1], 2, 4, 8, 16, 32)
+    ops = list(wl.ops); ops[4] = ("transpose", dict(a=0, b=1)); ops[5] = ("reshape", dict(shape=(64, 16))); ops[7] = ("reshape", dict(shape=(4, 2, 8, 32)))
+    _expect_fail(ops, wl.input_shapes, B.AGO_ERR_UNSUPPORTED, mode="fused", needle="family")
+
+
+def test_layout_operators_in_the_planner():
+    wl = WL.get("unfold_96", batch=2)
+    per_op = B.Subgraph(wl.ops, wl.input_shapes, mode="per_op")
+    mini = B.Subgraph(wl.ops, wl.input_shapes, mode="per_mini_subgraph")
+    assert per_op.output_shape == (2, 256, 4, 192)
+    assert per_op.query(B.AGO_Q_NUM_LAUNCHES) == 4        # GEMM | add | transpose | GEMM: reshapes are views
+    assert mini.query(B.AGO_Q_NUM_LAUNCHES) == 3          # GEMM + add | transpose | GEMM
+    # intermediates of that mode: the middle tensor before and after the transpose, written and read once each
+    assert mini.query(B.AGO_Q_INTERMEDIATE_BYTES) == 2 * 2 * (2 * 4 * 256 * 96) * 2
+    n = per_op.query(B.AGO_Q_NUM_LINKS)
+    assert [per_op.query(B.AGO_Q_LINK_CATEGORY, i) for i in range(n)] == [B.AGO_LINK_DOWNSTREAM_POINTWISE]
+    rs = lambda *shape: ("reshape", dict(shape=shape))
+    _expect_fail([("relu", {}), rs(4, 16)], [(8, 8)], B.AGO_ERR_SHAPE, needle="last dimension")
+    _expect_fail([("relu", {}), rs(3, 8)], [(8, 8)], B.AGO_ERR_SHAPE, needle="element count")
+    _expect_fail([rs(4, 2, 8)], [(8, 8)], B.AGO_ERR_UNSUPPORTED, needle="follow")
+    _expect_fail([("relu", {}), ("transpose", dict(a=0, b=2))], [(2, 4, 8)], B.AGO_ERR_SHAPE, needle="axes")
+    _expect_fail([("relu", {}), ("transpose", dict(a=1, b=1))], [(2, 4, 8, 8)], B.AGO_ERR_SHAPE, needle="axes")
+
+
 def _expect_fail(ops, shapes, status, mode="per_op", dtype=B.AGO_BF16, needle=""):
     with pytest.raises(B.AgoError) as e:
         B.Subgraph(ops, shapes, mode=mode, dtype=dtype)
