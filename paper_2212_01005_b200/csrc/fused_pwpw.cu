@@ -38,7 +38,8 @@ namespace {
 
 using namespace tc;
 
-constexpr int kThreads = 256;
+constexpr int kThreads = 512;
+constexpr int kColWarps = kThreads / 128;   // warps that share the 16-column groups of one tensor-memory lane quarter
 constexpr int kBM = 128, kBK = 64;
 constexpr int kXBlock = kBM * kBK * 2;   // one K block of the X / mid tile: 16 KB
 
@@ -156,7 +157,7 @@ pwpw_fused_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
   tcgen05_fence_after_sync();
   const uint32_t tmem_base = *tmem_slot;
   const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
-  const int half = warp >> 2;             // warps 0-3 and 4-7 share the 16-column groups of an epilogue alternately
+  const int half = warp >> 2;             // the warps of a lane quarter take the 16-column groups of an epilogue round-robin
   const int r = (warp & 3) * 32 + lane;   // this thread's row of the tile = its tensor-memory lane
   const uint32_t idesc1 = make_idesc_bf16(128, (uint32_t)p.C1p, 0, (uint32_t)p.w_nmajor);
   const uint32_t idesc2 = make_idesc_bf16(128, (uint32_t)p.C2p, 0, (uint32_t)p.w_nmajor);
@@ -190,7 +191,7 @@ pwpw_fused_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
     if (p.has_res) mbar_wait(bar_x, par, abort_flag, p.status, 0x604);   // every reader of the added tensor observes its arrival
     tcgen05_fence_after_sync();
     // ---- P3: + b1 [ReLU6] -> swizzled A operand of the second product ----
-    for (int g = half; g < p.C1p / 16; g += 2) {
+    for (int g = half; g < p.C1p / 16; g += kColWarps) {
       uint32_t v[16];
       tmem_ld_x16(tmem_base + lane_base + g * 16, v);
       tmem_ld_wait();
@@ -234,7 +235,7 @@ pwpw_fused_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
     mbar_wait(bar_m2, par, abort_flag, p.status, 0x602);
     tcgen05_fence_after_sync();
     // ---- P5: + b2 [ReLU6] -> staging tile over the X tile (the first product has read it) -> device memory ----
-    for (int g = half; g < p.C2p / 16; g += 2) {
+    for (int g = half; g < p.C2p / 16; g += kColWarps) {
       uint32_t v[16];
       tmem_ld_x16(tmem_base + lane_base + g * 16, v);
       tmem_ld_wait();
