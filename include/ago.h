@@ -312,6 +312,12 @@ typedef struct {
 double       ago_op_weight(const int64_t* loop_extents, int32_t num_loops, double c, double b);
 ago_status_t ago_graph_cluster(const ago_graph_desc_t* g, int32_t* subgraph_of_node, int32_t* num_subgraphs);
 
+/* Enqueue a kernel of `grid` CTAs x `block` threads that does nothing, launched the way the fused kernels are
+ * (programmatic stream serialization, dynamic shared memory `smem_bytes`): the launch floor against which the
+ * launch-bound configurations are read. No device memory is touched. Errors: AGO_ERR_INVALID_ARG for sizes
+ * outside 1..65535 CTAs / 1..1024 threads / 0..227 KB, AGO_ERR_CUDA for a failed launch. */
+ago_status_t ago_launch_empty(int32_t grid, int32_t block, int32_t smem_bytes, void* cuda_stream);
+
 /* Library version, "major.minor". */
 const char* ago_version(void);
 

@@ -43,6 +43,7 @@ EXPORTS = [
     "ago_subgraph_create", "ago_subgraph_run", "ago_subgraph_run_host", "ago_subgraph_destroy", "ago_last_error",
     "ago_subgraph_workspace_bytes", "ago_subgraph_set_workspace", "ago_subgraph_query", "ago_subgraph_status",
     "ago_version", "ago_subgraph_run_static", "ago_fusion_redundancy", "ago_op_weight", "ago_graph_cluster",
+    "ago_launch_empty",
 ]
 
 
@@ -125,6 +126,8 @@ def load(build_if_missing: bool = True):
     lib.ago_subgraph_status.restype = ctypes.c_int
     lib.ago_subgraph_status.argtypes = [vp]
     lib.ago_version.restype = ctypes.c_char_p
+    lib.ago_launch_empty.restype = ctypes.c_int
+    lib.ago_launch_empty.argtypes = [ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, vp]
     lib.ago_op_weight.restype = ctypes.c_double
     lib.ago_op_weight.argtypes = [ctypes.POINTER(ctypes.c_int64), ctypes.c_int32, ctypes.c_double, ctypes.c_double]
     lib.ago_graph_cluster.restype = ctypes.c_int
@@ -237,6 +240,12 @@ def ago_subgraph_query(h, what: int, index: int = 0) -> int:
 
 def ago_subgraph_status(h) -> int:
     return load().ago_subgraph_status(h)
+
+
+def ago_launch_empty(grid: int, block: int, smem_bytes: int = 0, stream: int = 0) -> None:
+    st = load().ago_launch_empty(int(grid), int(block), int(smem_bytes), ctypes.c_void_p(stream))
+    if st != AGO_OK:
+        raise AgoError(*ago_last_error())
 
 
 def ago_version() -> str:

@@ -268,9 +268,28 @@ ago_status_t run_unfused_in(ago_subgraph_s* h, const void* const* inputs, const 
 ago_status_t report_failure(ago_status_t s, const char* msg) { return fail(s, msg); }
 }  // namespace ago
 
+namespace {
+__global__ void empty_kernel() {
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+}  // namespace
+
 extern "C" {
 
 const char* ago_version(void) { return "0.1"; }
+
+ago_status_t ago_launch_empty(int32_t grid, int32_t block, int32_t smem_bytes, void* cuda_stream) {
+  if (grid < 1 || grid > 65535 || block < 1 || block > 1024 || smem_bytes < 0 || smem_bytes > 227 * 1024)
+    return fail(AGO_ERR_INVALID_ARG, "ago_launch_empty: grid 1..65535, block 1..1024, shared memory 0..227 KB");
+  static int smem_opt_in[64] = {};
+  cudaError_t e = ago::ensure_max_dynamic_smem(reinterpret_cast<const void*>(empty_kernel), smem_opt_in);
+  if (e != cudaSuccess) return cuda_fail(e, "cudaFuncSetAttribute");
+  ago::FusedLaunch launch(dim3((unsigned)grid), block, (size_t)smem_bytes, static_cast<cudaStream_t>(cuda_stream));
+  e = cudaLaunchKernelEx(&launch.config, empty_kernel);
+  if (e != cudaSuccess) return cuda_fail(e, "empty kernel launch");
+  return AGO_OK;
+}
 
 ago_status_t ago_last_error(const char** msg) {
   if (msg) *msg = g_msg.c_str();
