@@ -26,7 +26,8 @@ namespace {
 using namespace tc;
 
 constexpr int kBM = 128, kBN = 128, kBK = 64;
-constexpr int kMaxStages = 4;   // ring stages in use = min(4, K blocks): short reductions leave room for several CTAs per SM
+constexpr int kMaxStages = 4;   // ring stages: 3 when the grid exceeds one CTA per SM (two CTAs then share an SM and one CTA's epilogue
+                                // overlaps the other's products), else 4; never more than the K blocks
 constexpr int kStageBytes = 32 * 1024;
 constexpr int kEpiThreads = 128;
 constexpr int kThreads = kEpiThreads + 64;   // + TMA warp + MMA warp
@@ -294,7 +295,8 @@ cudaError_t launch_gemm_tc(const GemmArgs& a, int add_dtype, cudaStream_t stream
   p.kblocks = (a.K + kBK - 1) / kBK;
   p.heads = heads; p.c_sb = a.batches > 1 ? a.c_sb : 0; p.c_sh = a.batches > 1 ? a.c_sh : 0;
   canonical_epilogue(a.epi, &p);
-  p.stages = std::min(kMaxStages, p.kblocks);
+  const long ctas = (long)((a.M + kBM - 1) / kBM) * ((a.N + kBN - 1) / kBN) * heads * nb;
+  p.stages = std::min(ctas > 148 ? 3 : kMaxStages, p.kblocks);
   // the epilogue stages the output tile (128 rows x (columns x element size + 16) bytes) over the idle ring
   const int tile_cols = std::min(kBN, (a.N + 15) & ~15);
   const int staging = kBM * (tile_cols * (a.c_dtype == AGO_FP32 ? 4 : 2) + 16);
