@@ -29,8 +29,11 @@ ago_status_t fused_plan(Plan* plan, FusedState* st, std::string* err) {
       return pwpw_plan(plan, st, err);
     case AGO_KERNEL_ATTENTION:
       return attention_plan(plan, st, err);
-    case AGO_KERNEL_FFN:
-      return ffn_plan(plan, st, err);
+    case AGO_KERNEL_FFN: {
+      // the cluster kernel where the shape splits over 2..4 CTAs, else the kernel that tiles the reduction
+      const ago_status_t s = ffn_cluster_plan(plan, st, err);
+      return s == AGO_ERR_UNSUPPORTED ? ffn_plan(plan, st, err) : s;
+    }
     case AGO_KERNEL_CONV3X3_PAIR:
       return conv3x3_plan(plan, st, err);
     default:
@@ -40,7 +43,7 @@ ago_status_t fused_plan(Plan* plan, FusedState* st, std::string* err) {
 }
 
 size_t fused_workspace_bytes(const Plan& plan) {
-  return plan.fused_kernel == AGO_KERNEL_FFN ? ffn_workspace_bytes(plan) : 0;
+  return plan.fused_kernel == AGO_KERNEL_FFN && plan.fused_variant == 0 ? ffn_workspace_bytes(plan) : 0;
 }
 
 ago_status_t fused_run(const Plan& plan, FusedState* st, const void* const* inputs, const void* const* weights,
@@ -59,6 +62,7 @@ ago_status_t fused_run(const Plan& plan, FusedState* st, const void* const* inpu
     case AGO_KERNEL_ATTENTION:
       return attention_run(plan, st, inputs, weights, output, status_word, stream, err);
     case AGO_KERNEL_FFN:
+      if (st->variant == 1) return ffn_cluster_run(plan, st, inputs, weights, output, status_word, stream, err);
       return ffn_run(plan, st, inputs, weights, output, workspace, status_word, stream, err);
     case AGO_KERNEL_CONV3X3_PAIR:
       return conv3x3_run(plan, st, inputs, weights, output, status_word, stream, err);

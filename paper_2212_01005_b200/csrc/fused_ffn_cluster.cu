@@ -1,0 +1,389 @@
+// Fused feed-forward chain on a thread-block cluster: Y = GELU(X W1 + b1) W2 + b2, one kernel, the hidden
+// activations H never leave the SMs and nothing is reduced through device memory.
+//
+// Tile choice (Section III-B, "downstream pointwise / matmul"): the second GEMM reuses H only along its output
+// columns, so the downstream tile keeps ALL output columns of a block of 128 rows. Those (768 fp32 columns for
+// BERT-base) do not fit the tensor memory of one SM next to the first GEMM's accumulator -- but they fit the tensor
+// memory of a CLUSTER: CS CTAs (CS = 2..4) work on the same 128 rows, CTA r owns output columns
+// [r N2/CS, (r+1) N2/CS) and computes every CS-th tile of 128 hidden units. A finished H tile (bias, GELU, bf16,
+// 32 KB as a swizzled K-major operand) is copied to the same shared-memory slot of every peer with one bulk
+// shared-to-shared copy per peer (distributed shared memory), so every H tile is computed once and multiplied
+// into all N2 output columns without recomputation and without reductions outside the SM.
+//
+// Per CTA (rank r), T = hidden tiles / CS steps:
+//   ring   TMA producer warp: 32 KB stages -- X [128 x 64] + W1 [64 x 128] for the first GEMM, W2 [64 x N2/CS]
+//          for the second
+//   MMA    one thread: G1(t+1): Hacc[(t+1) & 1] = X W1[:, tile (t+1) CS + r]; then for k = 0..CS-1
+//          G2(k): out += H slot k * W2[tile t CS + k, own columns]; its completion is committed onto CTA k's
+//          "slot consumed" barrier
+//   epi    8 warps: Hacc[t & 1] -> + b1, GELU, bf16 -> own slot r (after every CTA has consumed its previous
+//          content) -> announce locally, bulk-copy to the peers' slot r with completion on their "slot full" barrier
+//   end    out (TMEM) -> + b2 -> bf16 -> device memory
+// Every wait is bounded; a CTA leaves only after a cluster barrier, so no peer copies into an exited CTA.
+#include <cuda.h>
+#include <cuda_bf16.h>
+
+#include <algorithm>
+#include <unordered_map>
+
+#include "fused.h"
+#include "tc_common.cuh"
+#include "tmap.h"
+
+namespace ago {
+
+namespace {
+
+using namespace tc;
+
+constexpr int kBM = 128;        // rows per cluster
+constexpr int kBH = 128;        // hidden units per tile
+constexpr int kBK = 64;         // reduction elements per ring stage
+constexpr int kMaxCS = 4;       // CTAs per cluster
+constexpr int kBlocks = 7;      // 32 KB blocks of shared memory: CS slots for H tiles + ring stages
+constexpr int kMaxStages = 5;
+constexpr int kStageBytes = 32 * 1024;
+constexpr int kEpiWarps = 8;    // two per tensor-memory lane quarter: each takes 64 of a tile's 128 columns
+constexpr int kEpiThreads = kEpiWarps * 32;
+constexpr int kThreads = kEpiThreads + 64;   // + TMA warp + MMA warp
+constexpr uint32_t kOutCol = 256;            // tensor memory: [0, 256) two first-GEMM accumulators, [256, 256 + NC) the output
+
+struct FfnClusterParams {
+  const float* b1;
+  const float* b2;
+  __nv_bfloat16* out;
+  unsigned int* status;
+  int M, K, Hid, N2;
+  int CS, NC;              // CTAs per cluster, output columns per CTA (N2 / CS, a multiple of 64, <= 256)
+  int T;                   // steps = Hid / 128 / CS
+  int kblocks;             // K / 64
+  int stages;              // ring stages = 7 - CS (at most 5)
+};
+
+__device__ __forceinline__ float gelu_tanh_fast(float v) {
+  const float u = 0.7978845608028654f * (v + 0.044715f * v * v * v);
+  float t;
+  asm("tanh.approx.f32 %0, %1;" : "=f"(t) : "f"(u));
+  return 0.5f * v * (1.0f + t);
+}
+
+__global__ void __launch_bounds__(kThreads, 1)
+ffn_cluster_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w1,
+                   const __grid_constant__ CUtensorMap tmap_w2, const FfnClusterParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  // the same offset in every CTA of the cluster: peers address each other's slots and barriers by it
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  const int CS = p.CS, stages = p.stages;
+  uint8_t* sRing = smem;                                   // stages x 32 KB
+  uint8_t* sH = smem + stages * kStageBytes;               // CS slots x (2 x [128 x 64] bf16, 128-byte-swizzled)
+  uint64_t* bars = reinterpret_cast<uint64_t*>(sH + CS * kStageBytes);
+  uint64_t* bar_full = bars;                       // [kMaxStages] ring stage landed
+  uint64_t* bar_empty = bars + kMaxStages;         // [kMaxStages] ring stage consumed
+  uint64_t* bar_hacc = bars + 2 * kMaxStages;      // [2] first GEMM complete in accumulator b
+  uint64_t* bar_hfree = bar_hacc + 2;              // [2] accumulator b drained
+  uint64_t* bar_hfull = bar_hacc + 4;              // [kMaxCS] H tile present in slot k (from CTA k)
+  uint64_t* bar_hdone = bar_hfull + kMaxCS;        // own slot consumed by every CTA of the cluster (count CS)
+  uint64_t* bar_out = bar_hdone + 1;               // second GEMM complete
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bar_out + 1);
+  volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(bar_out + 2);
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int r = (int)cluster_ctarank();
+  const int row0 = blockIdx.y * kBM;
+  const int T = p.T;
+  grid_dependency_wait();      // the previous grid of the stream has completed; device memory may be touched
+  grid_launch_dependents();
+
+  if (tid == kEpiThreads) {
+    *abort_flag = 0u;
+    for (int i = 0; i < kMaxStages; ++i) { mbar_init(bar_full + i, 1); mbar_init(bar_empty + i, 1); }
+    for (int i = 0; i < 2; ++i) { mbar_init(bar_hacc + i, 1); mbar_init(bar_hfree + i, 1); }
+    for (int i = 0; i < kMaxCS; ++i) mbar_init(bar_hfull + i, 1);
+    mbar_init(bar_hdone, (uint32_t)CS);
+    mbar_init(bar_out, 1);
+    fence_mbar_init();
+    fence_proxy_async_smem();
+  }
+  if (warp == 0) {
+    tmem_alloc(tmem_slot, 512);
+    tmem_relinquish();
+  }
+  tcgen05_fence_before_sync();
+  __syncthreads();
+  cluster_sync_all();          // every CTA's barriers exist before a peer signals them
+  tcgen05_fence_after_sync();
+  const uint32_t tmem_base = *tmem_slot;
+  const int n0 = r * p.NC;     // first output column of this CTA
+
+  if (warp == kEpiWarps) {
+    // ================================ TMA producer ================================
+    if (lane == 0) {
+      tma_prefetch_desc(&tmap_x);
+      tma_prefetch_desc(&tmap_w1);
+      tma_prefetch_desc(&tmap_w2);
+      int s = 0, round = 0;
+      auto next_stage = [&]() -> uint8_t* {
+        if (round > 0) mbar_wait(bar_empty + s, (uint32_t)(round - 1) & 1u, abort_flag, p.status, 0x701);
+        mbar_arrive_expect_tx(bar_full + s, kStageBytes);
+        return sRing + s * kStageBytes;
+      };
+      auto advance = [&]() { if (++s == stages) { s = 0; ++round; } };
+      auto load_g1 = [&](int t) {          // first GEMM of this CTA's t-th hidden tile
+        const int hid0 = (t * CS + r) * kBH;
+        for (int kb = 0; kb < p.kblocks; ++kb) {
+          uint8_t* st = next_stage();
+          tma_load_2d(st, &tmap_x, bar_full + s, kb * kBK, row0);                          // X [128 rows x 64 k]
+          tma_load_2d(st + 16384, &tmap_w1, bar_full + s, hid0, kb * kBK);                 // W1 [64 k x 64 n] twice
+          tma_load_2d(st + 16384 + 8192, &tmap_w1, bar_full + s, hid0 + 64, kb * kBK);
+          advance();
+        }
+      };
+      load_g1(0);
+      for (int t = 0; t < T; ++t) {
+        if (t + 1 < T) load_g1(t + 1);
+        for (int k = 0; k < CS; ++k) {      // second GEMM over hidden tile t CS + k: two stages of 64 hidden units
+          const int hid0 = (t * CS + k) * kBH;
+          for (int h = 0; h < 2; ++h) {
+            uint8_t* st = next_stage();
+            for (int nb = 0; nb < 4; ++nb)   // W2 [64 k x 64 n] per block; blocks past NC read as zero and are not multiplied
+              tma_load_2d(st + nb * 8192, &tmap_w2, bar_full + s, nb * 64 < p.NC ? n0 + nb * 64 : p.N2, hid0 + h * 64);
+            advance();
+          }
+        }
+      }
+    }
+    __syncwarp();
+  } else if (warp == kEpiWarps + 1) {
+    // ================================ MMA issuer ================================
+    if (lane == 0) {
+      const uint32_t idesc1 = make_idesc_bf16(128, kBH, 0, 1);              // A K-major, B N-major (weights as they lie in memory)
+      const uint32_t idesc2 = make_idesc_bf16(128, (uint32_t)p.NC, 0, 1);
+      int s = 0, round = 0;
+      auto advance = [&]() { if (++s == stages) { s = 0; ++round; } };
+      auto g1 = [&](int t) {
+        const int b = t & 1;
+        if (t >= 2) {
+          mbar_wait(bar_hfree + b, (uint32_t)((t - 2) >> 1) & 1u, abort_flag, p.status, 0x702);
+          tcgen05_fence_after_sync();
+        }
+        for (int kb = 0; kb < p.kblocks; ++kb) {
+          mbar_wait(bar_full + s, (uint32_t)round & 1u, abort_flag, p.status, 0x703);
+          tcgen05_fence_after_sync();
+          const uint32_t st = smem_u32(sRing + s * kStageBytes);
+          const uint64_t ad = make_smem_desc(st, 0, 1024, SW_128B);
+          const uint64_t bd = make_smem_desc(st + 16384, 8192, 1024, SW_128B);
+#pragma unroll
+          for (int ks = 0; ks < kBK / 16; ++ks)
+            umma_bf16(tmem_base + b * kBH, ad + 2u * ks, bd + (uint64_t)((ks * 2048) >> 4), idesc1, (kb | ks) != 0);
+          umma_commit(bar_empty + s);
+          advance();
+        }
+        umma_commit(bar_hacc + b);
+      };
+      g1(0);
+      for (int t = 0; t < T; ++t) {
+        if (t + 1 < T) g1(t + 1);
+        for (int k = 0; k < CS; ++k) {
+          mbar_wait(bar_hfull + k, (uint32_t)t & 1u, abort_flag, p.status, 0x704);      // H tile t CS + k is in slot k
+          for (int h = 0; h < 2; ++h) {
+            mbar_wait(bar_full + s, (uint32_t)round & 1u, abort_flag, p.status, 0x705);
+            tcgen05_fence_after_sync();
+            const uint64_t hd = make_smem_desc(smem_u32(sH + k * kStageBytes + h * (kBM * 128)), 0, 1024, SW_128B);
+            const uint64_t bd = make_smem_desc(smem_u32(sRing + s * kStageBytes), 8192, 1024, SW_128B);
+#pragma unroll
+            for (int ks = 0; ks < 4; ++ks)
+              umma_bf16(tmem_base + kOutCol, hd + 2u * ks, bd + (uint64_t)((ks * 2048) >> 4), idesc2, (t | k | h | ks) != 0);
+            umma_commit(bar_empty + s);
+            advance();
+          }
+          // slot k of this CTA has been read: tell its producer (CTA k)
+          umma_commit_cluster(cluster_map(smem_u32(bar_hdone), (uint32_t)k));
+        }
+      }
+      umma_commit(bar_out);
+    }
+    __syncwarp();
+  } else {
+    // ================ epilogue warps: thread = (row, half of a tile's 128 columns) ================
+    const int row = (warp & 3) * 32 + lane;
+    const int half = warp >> 2;
+    const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
+    const bool row_ok = row0 + row < p.M;
+    uint8_t* slot = sH + r * kStageBytes;          // this CTA produces into slot r everywhere
+
+    for (int t = 0; t < T; ++t) {
+      const int b = t & 1;
+      mbar_wait(bar_hacc + b, (uint32_t)(t >> 1) & 1u, abort_flag, p.status, 0x706);
+      tcgen05_fence_after_sync();
+      // every CTA has multiplied the previous content of slot r (and the copies that delivered it are complete)
+      if (t >= 1) mbar_wait(bar_hdone, (uint32_t)(t - 1) & 1u, abort_flag, p.status, 0x707);
+      uint8_t* tile = slot + half * (kBM * 128);
+      const float* bb = p.b1 + (size_t)(t * CS + r) * kBH + half * 64;
+#pragma unroll
+      for (int c0 = 0; c0 < 64; c0 += 32) {
+        uint32_t v[32];
+        tmem_ld_x32(tmem_base + lane_base + b * kBH + half * 64 + c0, v);
+        tmem_ld_wait();
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          const float4 b0 = __ldg(reinterpret_cast<const float4*>(bb + c0 + q * 8));
+          const float4 b1v = __ldg(reinterpret_cast<const float4*>(bb + c0 + q * 8 + 4));
+          const float bv[8] = {b0.x, b0.y, b0.z, b0.w, b1v.x, b1v.y, b1v.z, b1v.w};
+          uint32_t w[4];
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            const int e = q * 8 + j * 2;
+            w[j] = pack_bf16x2(gelu_tanh_fast(__uint_as_float(v[e]) + bv[2 * j]),
+                               gelu_tanh_fast(__uint_as_float(v[e + 1]) + bv[2 * j + 1]));
+          }
+          *reinterpret_cast<uint4*>(tile + swz_offset(row, (c0 >> 3) + q, 128)) = make_uint4(w[0], w[1], w[2], w[3]);
+        }
+      }
+      fence_proxy_async_smem();      // the MMA and the bulk copies read the tile through the async proxy
+      tcgen05_fence_before_sync();
+      named_barrier_sync(1, kEpiThreads);
+      if (tid == 0) {
+        mbar_arrive(bar_hfree + b);
+        mbar_arrive(bar_hfull + r);                                   // the local consumer
+        const uint32_t src = smem_u32(slot), bar = smem_u32(bar_hfull + r);
+        for (int q = 1; q < CS; ++q) {                                // the peers, starting with the next rank
+          const uint32_t peer = (uint32_t)((r + q) % CS);
+          const uint32_t rbar = cluster_map(bar, peer);
+          mbar_remote_arrive_expect_tx(rbar, kStageBytes);
+          bulk_copy_to_cluster(cluster_map(src, peer), src, kStageBytes, rbar);
+        }
+      }
+    }
+
+    // ---- output: out (TMEM) -> + b2 -> bf16 -> device memory; thread = (row, half of the CTA's NC columns) ----
+    mbar_wait(bar_out, 0, abort_flag, p.status, 0x708);
+    tcgen05_fence_after_sync();
+    const int hc = p.NC >> 1;                                          // columns per half: 32, 64, 96 or 128
+    __nv_bfloat16* orow = p.out + (size_t)(row0 + row) * p.N2 + n0 + half * hc;
+    const float* b2 = p.b2 + n0 + half * hc;
+    for (int c0 = 0; c0 < hc; c0 += 32) {
+      uint32_t v[32];
+      tmem_ld_x32(tmem_base + lane_base + kOutCol + half * hc + c0, v);
+      tmem_ld_wait();
+      if (row_ok) {
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          const float4 b0 = __ldg(reinterpret_cast<const float4*>(b2 + c0 + q * 8));
+          const float4 b1v = __ldg(reinterpret_cast<const float4*>(b2 + c0 + q * 8 + 4));
+          *reinterpret_cast<uint4*>(orow + c0 + q * 8) =
+              make_uint4(pack_bf16x2(__uint_as_float(v[q * 8]) + b0.x, __uint_as_float(v[q * 8 + 1]) + b0.y),
+                         pack_bf16x2(__uint_as_float(v[q * 8 + 2]) + b0.z, __uint_as_float(v[q * 8 + 3]) + b0.w),
+                         pack_bf16x2(__uint_as_float(v[q * 8 + 4]) + b1v.x, __uint_as_float(v[q * 8 + 5]) + b1v.y),
+                         pack_bf16x2(__uint_as_float(v[q * 8 + 6]) + b1v.z, __uint_as_float(v[q * 8 + 7]) + b1v.w));
+        }
+      }
+    }
+  }
+  tcgen05_fence_before_sync();
+  __syncthreads();
+  cluster_sync_all();          // no CTA leaves while a peer may still copy into it or signal its barriers
+  if (warp == 0) tmem_dealloc(tmem_base, 512);
+}
+
+struct FfnClusterHost {
+  FfnClusterParams prm;
+  int smem_bytes = 0;
+  struct Key { const void* p; int which; bool operator==(const Key& o) const { return p == o.p && which == o.which; } };
+  struct KeyHash { size_t operator()(const Key& k) const { return std::hash<const void*>()(k.p) ^ (size_t)k.which * 0x9e3779b97f4a7c15ull; } };
+  std::unordered_map<Key, CUtensorMap, KeyHash> maps;
+};
+
+void fill_launch(cudaLaunchConfig_t* cfg, cudaLaunchAttribute* attr, const FfnClusterParams& q, int smem_bytes, cudaStream_t stream) {
+  *cfg = cudaLaunchConfig_t{};
+  cfg->gridDim = dim3((unsigned)q.CS, (unsigned)((q.M + kBM - 1) / kBM), 1);
+  cfg->blockDim = dim3(kThreads, 1, 1);
+  cfg->dynamicSmemBytes = (size_t)smem_bytes;
+  cfg->stream = stream;
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = (unsigned)q.CS; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
+  cfg->attrs = attr;
+  cfg->numAttrs = 2;
+}
+
+}  // namespace
+
+// AGO_ERR_UNSUPPORTED (without touching *err) when the shape has no cluster split: the caller falls back to the
+// kernel that tiles the second GEMM's reduction across independent CTAs.
+ago_status_t ffn_cluster_plan(Plan* plan, FusedState* st, std::string* err) {
+  (void)err;
+  FfnClusterParams q{};
+  q.K = (int)plan->inputs[0].last();
+  q.M = (int)(plan->inputs[0].numel() / q.K);
+  q.Hid = plan->ops[0].op.p[0];
+  q.N2 = plan->ops[3].op.p[0];
+  if (q.K % kBK != 0 || q.Hid % kBH != 0) return AGO_ERR_UNSUPPORTED;
+  const int htiles = q.Hid / kBH;
+  q.CS = 0;
+  for (int cs = 2; cs <= kMaxCS; ++cs) {   // the smallest cluster whose column share fits tensor memory
+    if (q.N2 % cs != 0 || htiles % cs != 0) continue;
+    const int nc = q.N2 / cs;
+    if (nc % 64 != 0 || nc > 256) continue;
+    q.CS = cs; q.NC = nc;
+    break;
+  }
+  if (q.CS == 0) return AGO_ERR_UNSUPPORTED;
+  // one cluster per block of 128 rows: worth it only when the clusters fill the SMs; few rows are better served by the
+  // kernel that spreads the hidden tiles of a row block over independent CTAs
+  if ((long)((q.M + kBM - 1) / kBM) * q.CS < 120) return AGO_ERR_UNSUPPORTED;
+  q.T = htiles / q.CS;
+  q.kblocks = q.K / kBK;
+  q.stages = std::min(kMaxStages, kBlocks - q.CS);
+  auto* host = new FfnClusterHost();
+  host->prm = q;
+  host->smem_bytes = (q.stages + q.CS) * kStageBytes + 256 + 1024;
+  st->impl = host;
+  st->impl_free = [](void* p) { delete static_cast<FfnClusterHost*>(p); };
+  st->variant = 1;
+  st->tile_rows = kBM; st->grid = q.CS * ((q.M + kBM - 1) / kBM); st->smem_bytes = host->smem_bytes;
+  plan->tile_rows = kBM; plan->smem_bytes = host->smem_bytes;
+  plan->fused_variant = 1;
+  return AGO_OK;
+}
+
+ago_status_t ffn_cluster_run(const Plan& plan, FusedState* st, const void* const* inputs, const void* const* weights,
+                             void* output, unsigned int* status_word, cudaStream_t stream, std::string* err) {
+  (void)plan;
+  FfnClusterHost* host = static_cast<FfnClusterHost*>(st->impl);
+  FfnClusterParams q = host->prm;
+  q.b1 = static_cast<const float*>(weights[1]);
+  q.b2 = static_cast<const float*>(weights[3]);
+  q.out = static_cast<__nv_bfloat16*>(output);
+  q.status = status_word;
+  auto get_map = [&](const void* base, int which, CUtensorMap* out) -> bool {
+    FfnClusterHost::Key key{base, which};
+    auto it = host->maps.find(key);
+    if (it == host->maps.end()) {
+      CUtensorMap m;
+      uint64_t dims[2]; uint64_t strides[1]; uint32_t box[2];
+      if (which == 0) { dims[0] = q.K; dims[1] = q.M; strides[0] = (uint64_t)q.K * 2; box[0] = kBK; box[1] = kBM; }
+      else if (which == 1) { dims[0] = q.Hid; dims[1] = q.K; strides[0] = (uint64_t)q.Hid * 2; box[0] = 64; box[1] = kBK; }
+      else { dims[0] = q.N2; dims[1] = q.Hid; strides[0] = (uint64_t)q.N2 * 2; box[0] = 64; box[1] = 64; }
+      if (!encode_tmap_bf16(&m, base, 2, dims, strides, box, 128, err)) return false;
+      if (host->maps.size() > 4096) host->maps.clear();
+      it = host->maps.emplace(key, m).first;
+    }
+    *out = it->second;
+    return true;
+  };
+  CUtensorMap mx, mw1, mw2;
+  if (!get_map(inputs[0], 0, &mx) || !get_map(weights[0], 1, &mw1) || !get_map(weights[2], 2, &mw2)) return AGO_ERR_CUDA;
+  {
+    static int smem_opt_in[64] = {};
+    cudaError_t e = ensure_max_dynamic_smem(reinterpret_cast<const void*>(ffn_cluster_kernel), smem_opt_in);
+    if (e != cudaSuccess) { *err = std::string("cudaFuncSetAttribute: ") + cudaGetErrorString(e); return AGO_ERR_CUDA; }
+  }
+  cudaLaunchConfig_t cfg; cudaLaunchAttribute attr[2];
+  fill_launch(&cfg, attr, q, host->smem_bytes, stream);
+  cudaError_t e = cudaLaunchKernelEx(&cfg, ffn_cluster_kernel, mx, mw1, mw2, q);
+  if (e != cudaSuccess) { *err = std::string("fused feed-forward (cluster) launch: ") + cudaGetErrorString(e); return AGO_ERR_CUDA; }
+  return AGO_OK;
+}
+
+}  // namespace ago

@@ -69,6 +69,7 @@ struct Plan {
   std::vector<int> link_category;     // per complex -> complex pair
   Shape output;
   int fused_kernel = AGO_KERNEL_NONE;
+  int fused_variant = 0;              // kernel variant within the family, chosen at plan time
   int64_t flops_tensor = 0, flops_cuda = 0, sfu_ops = 0, io_bytes = 0, intermediate_bytes = 0;
   int64_t max_intermediate_bytes = 0;  // largest tensor passed between launches
   int tile_rows = 0;

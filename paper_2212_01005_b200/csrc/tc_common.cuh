@@ -122,6 +122,38 @@ __device__ __forceinline__ void tcgen05_fence_after_sync() {
 __device__ __forceinline__ uint32_t fast_div(uint32_t x, uint32_t d, uint32_t recip) { return d == 1u ? x : __umulhi(x, recip); }
 inline uint32_t fast_div_recip(int d) { return (uint32_t)((1ull << 32) / (uint64_t)d + 1ull); }
 
+// ---- thread-block clusters: distributed shared memory, remote barriers ---------------------------
+
+// Shared-memory address of `local_saddr` (a shared::cta address of this CTA's layout) in CTA `rank` of the cluster.
+__device__ __forceinline__ uint32_t cluster_map(uint32_t local_saddr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local_saddr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+// Every thread of every CTA of the cluster arrives; returns when all have (release / acquire at cluster scope).
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// One arrival on the mbarrier at cluster address `remote_bar` that also announces `bytes` of pending copy traffic.
+__device__ __forceinline__ void mbar_remote_arrive_expect_tx(uint32_t remote_bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.release.cluster.shared::cluster.b64 _, [%0], %1;" ::"r"(remote_bar), "r"(bytes) : "memory");
+}
+// Bulk copy of `bytes` (a multiple of 16; both addresses 16-byte aligned) from this CTA's shared memory to the
+// cluster address `remote_dst`; completion is counted in bytes on the mbarrier at cluster address `remote_bar`.
+__device__ __forceinline__ void bulk_copy_to_cluster(uint32_t remote_dst, uint32_t local_src, uint32_t bytes, uint32_t remote_bar) {
+  asm volatile("cp.async.bulk.shared::cluster.shared::cta.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+               ::"r"(remote_dst), "r"(local_src), "r"(bytes), "r"(remote_bar) : "memory");
+}
+// tcgen05.commit onto an mbarrier given by its cluster address (this CTA's or a peer's).
+__device__ __forceinline__ void umma_commit_cluster(uint32_t bar_cluster_addr) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar_cluster_addr) : "memory");
+}
+
 // ---- per-thread asynchronous copies (global -> shared, 16 bytes, zero-filled beyond src_bytes) ----------
 
 __device__ __forceinline__ void cp_async_16(uint32_t dst_saddr, const void* src, uint32_t src_bytes) {

@@ -142,8 +142,8 @@ def mbv2_block(name, seed_seq, N, H, c_in, c_exp, c_out, stride, residual) -> Wo
                     samples=N, input_dist=["uniform"])
 
 
-def ffn(name, seed_seq, M, d_model, hidden, samples) -> Workload:
-    return Workload(name, seed_seq, [(M, d_model)], _ffn_ops(hidden, d_model), samples=samples)
+def ffn(name, seed_seq, M, d_model, hidden, samples, d_out=None) -> Workload:
+    return Workload(name, seed_seq, [(M, d_model)], _ffn_ops(hidden, d_out or d_model), samples=samples)
 
 
 def resnet_block(name, seed_seq, N, H, ch) -> Workload:

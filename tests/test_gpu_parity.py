@@ -27,6 +27,11 @@ def small_workloads():
         # tall enough that the fused kernel keeps 2 / 3 hidden tiles per CTA (100 row blocks x 6 / 9 hidden tiles)
         "ffn_g2": WL.ffn("ffn_g2", [31], 12800, 128, 768, 1),
         "ffn_g3": WL.ffn("ffn_g3", [32], 12800, 128, 1152, 1),
+        # enough row blocks for the thread-block-cluster kernel: clusters of 2, 3 and 4 CTAs, one and two steps,
+        # 64 to 256 output columns per CTA, a ragged last row block
+        "ffn_c2": WL.ffn("ffn_c2", [33], 9637, 64, 256, 1, d_out=384),
+        "ffn_c3": WL.ffn("ffn_c3", [34], 6400, 128, 768, 1, d_out=192),
+        "ffn_c4": WL.ffn("ffn_c4", [35], 4864, 64, 512, 1, d_out=1024),
         "resnet_small": WL.resnet_block("resnet_small", [26], 2, 12, 64),
         "resnet_odd": WL.resnet_block("resnet_odd", [27], 1, 9, 32),
         "resnet_16ch": WL.resnet_block("resnet_16ch", [32], 2, 20, 16),
@@ -113,7 +118,8 @@ def test_padding_of_the_intermediate_with_large_bias(ago):
 
 # ---- fused kernels -------------------------------------------------------------------
 
-FUSED_SMALL = ["mbv2_14", "mbv2_s1_odd", "mbv2_s2", "mbv2_s2_odd", "attn_small", "attn_ragged", "ffn_small", "ffn_rows_ragged", "ffn_g2", "ffn_g3", "resnet_small", "resnet_odd", "resnet_16ch"]
+FUSED_SMALL = ["mbv2_14", "mbv2_s1_odd", "mbv2_s2", "mbv2_s2_odd", "attn_small", "attn_ragged", "ffn_small", "ffn_rows_ragged", "ffn_g2", "ffn_g3",
+               "ffn_c2", "ffn_c3", "ffn_c4", "resnet_small", "resnet_odd", "resnet_16ch"]
 
 
 @pytest.mark.parametrize("name", FUSED_SMALL)
