@@ -63,27 +63,33 @@ def load_peaks():
     return p
 
 
-def roofline(wl, peaks, seconds_per_launch, traffic):
+def roofline(wl, peaks, seconds_per_launch, traffic, clocks=None):
     """The roofline that bounds one fused launch: the slowest of HBM (inputs +
     weights + output), tensor cores (dense contractions) and plain ALUs
     (depthwise FMAs). `achieved` / `peak` are in that bound's unit."""
     fl = WL.flops(wl)
     io = WL.io_bytes(wl)
     t_hbm = io / (peaks["hbm_gbs"] * 1e9)
-    t_tensor = fl["tensor"] / (peaks["bf16_tflops"] * 1e12)
+    # tensor peak: the burst measurement, unless the clocks sampled during the timed region show the power cap at
+    # work (median SM clock below 90 % of the maximum): then the sustained measurement is the one that applies
+    capped = bool(clocks) and clocks.get("sm_mhz", 0) and clocks["sm_mhz"] < 0.9 * clocks.get("sm_max_mhz", 0)
+    tensor_peak = (peaks.get("bf16_tflops_sustained") if capped else None) or peaks["bf16_tflops"]
+    t_tensor = fl["tensor"] / (tensor_peak * 1e12)
     t_alu = fl["cuda"] / (FP32_PEAK_TFLOPS * 1e12)
     bound = max((t_hbm, "hbm"), (t_tensor, "tensor"), (t_alu, "alu"))[1]
     if bound == "hbm":
         achieved, peak, unit = io / seconds_per_launch / 1e9, peaks["hbm_gbs"], "GB/s"
     elif bound == "tensor":
-        achieved, peak, unit = fl["tensor"] / seconds_per_launch / 1e12, peaks["bf16_tflops"], "TFLOP/s"
+        achieved, peak, unit = fl["tensor"] / seconds_per_launch / 1e12, tensor_peak, "TFLOP/s"
     else:
         achieved, peak, unit = fl["cuda"] / seconds_per_launch / 1e12, FP32_PEAK_TFLOPS, "TFLOP/s"
     t_roof = max(t_hbm, t_tensor, t_alu)
     return {
         "bound": bound, "achieved": round(achieved, 3), "peak": round(peak, 3), "unit": unit,
         "frac": round(achieved / peak, 4), "traffic": traffic,
-        "peak_source": ("of measured" if peaks["_source"] == "measured" else "of fallback") if bound != "alu"
+        "peak_source": (("of measured" if peaks["_source"] == "measured" else "of fallback") +
+                        (" (sustained bf16 figure: SM clocks were power-capped during the timed region)" if bound == "tensor" and capped else ""))
+        if bound != "alu"
         else "derived: 148 SM x 128 lanes x 2 x 1.965 GHz",
         "roofline_us": round(t_roof * 1e6, 3),
         "t_hbm_us": round(t_hbm * 1e6, 3), "t_tensor_us": round(t_tensor * 1e6, 3), "t_alu_us": round(t_alu * 1e6, 3),
@@ -442,7 +448,7 @@ def main():
             "cuda_graph": not args.no_graph, "parallelism": f"replicas x{world}",
             "us_per_launch": round(sec_per_launch * 1e6, 3),
         },
-        "roofline": roofline(wl, peaks, sec_per_launch, NCU_TRAFFIC_BYTES.get((args.workload, args.mode))),
+        "roofline": roofline(wl, peaks, sec_per_launch, NCU_TRAFFIC_BYTES.get((args.workload, args.mode)), clocks),
         "e2e": e2e, "gpu_launches": args.steps * nsets * launches_per_pass, "clocks": clocks,
         "unfused": unfused,
         "context": head["context"],

@@ -83,14 +83,20 @@ ffn_cluster_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
   uint64_t* bar_hfree = bar_hacc + 2;              // [2] accumulator b drained
   uint64_t* bar_hfull = bar_hacc + 4;              // [kMaxCS] H tile present in slot k (from CTA k)
   uint64_t* bar_hdone = bar_hfull + kMaxCS;        // own slot consumed by every CTA of the cluster (count CS)
-  uint64_t* bar_out = bar_hdone + 1;               // second GEMM complete
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bar_out + 1);
-  volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(bar_out + 2);
+  uint64_t* bar_out = bar_hdone + 1;               // second GEMM of a row block complete
+  uint64_t* bar_outfree = bar_out + 1;             // output accumulators drained: the next row block may overwrite them
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bar_outfree + 1);
+  volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(bar_outfree + 2);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int r = (int)cluster_ctarank();
-  const int row0 = blockIdx.y * kBM;
   const int T = p.T;
+  // A cluster walks over the row blocks blockIdx.y, + gridDim.y, ...: its steps (row block, hidden tile of this CTA)
+  // form one sequence, so the first GEMM of the next row block overlaps the tail of the current one.
+  const int row_blocks = (p.M + kBM - 1) / kBM;
+  const int my_blocks = ((int)blockIdx.y < row_blocks) ? (row_blocks - 1 - (int)blockIdx.y) / (int)gridDim.y + 1 : 0;
+  const int steps = my_blocks * T;
+  auto row0_of = [&](int step) { return ((int)blockIdx.y + (step / T) * (int)gridDim.y) * kBM; };
   grid_dependency_wait();      // the previous grid of the stream has completed; device memory may be touched
   grid_launch_dependents();
 
@@ -101,6 +107,7 @@ ffn_cluster_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
     for (int i = 0; i < kMaxCS; ++i) mbar_init(bar_hfull + i, 1);
     mbar_init(bar_hdone, (uint32_t)CS);
     mbar_init(bar_out, 1);
+    mbar_init(bar_outfree, 1);
     fence_mbar_init();
     fence_proxy_async_smem();
   }
@@ -128,8 +135,8 @@ ffn_cluster_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
         return sRing + s * kStageBytes;
       };
       auto advance = [&]() { if (++s == stages) { s = 0; ++round; } };
-      auto load_g1 = [&](int t) {          // first GEMM of this CTA's t-th hidden tile
-        const int hid0 = (t * CS + r) * kBH;
+      auto load_g1 = [&](int step) {       // first GEMM of this CTA's hidden tile of that step
+        const int hid0 = ((step % T) * CS + r) * kBH, row0 = row0_of(step);
         for (int kb = 0; kb < p.kblocks; ++kb) {
           uint8_t* st = next_stage();
           tma_load_2d(st, &tmap_x, bar_full + s, kb * kBK, row0);                          // X [128 rows x 64 k]
@@ -138,11 +145,11 @@ ffn_cluster_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
           advance();
         }
       };
-      load_g1(0);
-      for (int t = 0; t < T; ++t) {
-        if (t + 1 < T) load_g1(t + 1);
+      if (steps > 0) load_g1(0);
+      for (int step = 0; step < steps; ++step) {
+        if (step + 1 < steps) load_g1(step + 1);
         for (int k = 0; k < CS; ++k) {      // second GEMM over hidden tile t CS + k: two stages of 64 hidden units
-          const int hid0 = (t * CS + k) * kBH;
+          const int hid0 = ((step % T) * CS + k) * kBH;
           for (int h = 0; h < 2; ++h) {
             uint8_t* st = next_stage();
             for (int nb = 0; nb < 4; ++nb)   // W2 [64 k x 64 n] per block; blocks past NC read as zero and are not multiplied
@@ -160,10 +167,10 @@ ffn_cluster_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
       const uint32_t idesc2 = make_idesc_bf16(128, (uint32_t)p.NC, 0, 1);
       int s = 0, round = 0;
       auto advance = [&]() { if (++s == stages) { s = 0; ++round; } };
-      auto g1 = [&](int t) {
-        const int b = t & 1;
-        if (t >= 2) {
-          mbar_wait(bar_hfree + b, (uint32_t)((t - 2) >> 1) & 1u, abort_flag, p.status, 0x702);
+      auto g1 = [&](int step) {
+        const int b = step & 1;
+        if (step >= 2) {
+          mbar_wait(bar_hfree + b, (uint32_t)((step - 2) >> 1) & 1u, abort_flag, p.status, 0x702);
           tcgen05_fence_after_sync();
         }
         for (int kb = 0; kb < p.kblocks; ++kb) {
@@ -180,11 +187,16 @@ ffn_cluster_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
         }
         umma_commit(bar_hacc + b);
       };
-      g1(0);
-      for (int t = 0; t < T; ++t) {
-        if (t + 1 < T) g1(t + 1);
+      if (steps > 0) g1(0);
+      for (int step = 0; step < steps; ++step) {
+        if (step + 1 < steps) g1(step + 1);
+        const int t = step % T, bi = step / T;
+        if (t == 0 && bi >= 1) {   // the output accumulators of the previous row block have been drained
+          mbar_wait(bar_outfree, (uint32_t)(bi - 1) & 1u, abort_flag, p.status, 0x709);
+          tcgen05_fence_after_sync();
+        }
         for (int k = 0; k < CS; ++k) {
-          mbar_wait(bar_hfull + k, (uint32_t)t & 1u, abort_flag, p.status, 0x704);      // H tile t CS + k is in slot k
+          mbar_wait(bar_hfull + k, (uint32_t)step & 1u, abort_flag, p.status, 0x704);   // H tile t CS + k is in slot k
           for (int h = 0; h < 2; ++h) {
             mbar_wait(bar_full + s, (uint32_t)round & 1u, abort_flag, p.status, 0x705);
             tcgen05_fence_after_sync();
@@ -199,8 +211,8 @@ ffn_cluster_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
           // slot k of this CTA has been read: tell its producer (CTA k)
           umma_commit_cluster(cluster_map(smem_u32(bar_hdone), (uint32_t)k));
         }
+        if (t == T - 1) umma_commit(bar_out);
       }
-      umma_commit(bar_out);
     }
     __syncwarp();
   } else {
@@ -208,15 +220,14 @@ ffn_cluster_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
     const int row = (warp & 3) * 32 + lane;
     const int half = warp >> 2;
     const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
-    const bool row_ok = row0 + row < p.M;
     uint8_t* slot = sH + r * kStageBytes;          // this CTA produces into slot r everywhere
 
-    for (int t = 0; t < T; ++t) {
-      const int b = t & 1;
-      mbar_wait(bar_hacc + b, (uint32_t)(t >> 1) & 1u, abort_flag, p.status, 0x706);
+    for (int step = 0; step < steps; ++step) {
+      const int b = step & 1, t = step % T;
+      mbar_wait(bar_hacc + b, (uint32_t)(step >> 1) & 1u, abort_flag, p.status, 0x706);
       tcgen05_fence_after_sync();
       // every CTA has multiplied the previous content of slot r (and the copies that delivered it are complete)
-      if (t >= 1) mbar_wait(bar_hdone, (uint32_t)(t - 1) & 1u, abort_flag, p.status, 0x707);
+      if (step >= 1) mbar_wait(bar_hdone, (uint32_t)(step - 1) & 1u, abort_flag, p.status, 0x707);
       uint8_t* tile = slot + half * (kBM * 128);
       const float* bb = p.b1 + (size_t)(t * CS + r) * kBH + half * 64;
 #pragma unroll
@@ -253,29 +264,35 @@ ffn_cluster_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
           bulk_copy_to_cluster(cluster_map(src, peer), src, kStageBytes, rbar);
         }
       }
-    }
-
-    // ---- output: out (TMEM) -> + b2 -> bf16 -> device memory; thread = (row, half of the CTA's NC columns) ----
-    mbar_wait(bar_out, 0, abort_flag, p.status, 0x708);
-    tcgen05_fence_after_sync();
-    const int hc = p.NC >> 1;                                          // columns per half: 32, 64, 96 or 128
-    __nv_bfloat16* orow = p.out + (size_t)(row0 + row) * p.N2 + n0 + half * hc;
-    const float* b2 = p.b2 + n0 + half * hc;
-    for (int c0 = 0; c0 < hc; c0 += 32) {
-      uint32_t v[32];
-      tmem_ld_x32(tmem_base + lane_base + kOutCol + half * hc + c0, v);
-      tmem_ld_wait();
-      if (row_ok) {
+      if (t == T - 1) {
+        // ---- output of the row block: out (TMEM) -> + b2 -> bf16 -> device memory; thread = (row, half of the CTA's columns) ----
+        const int bi = step / T, row0 = row0_of(step);
+        const bool row_ok = row0 + row < p.M;
+        mbar_wait(bar_out, (uint32_t)bi & 1u, abort_flag, p.status, 0x708);
+        tcgen05_fence_after_sync();
+        const int hc = p.NC >> 1;                                          // columns per half: 32, 64, 96 or 128
+        __nv_bfloat16* orow = p.out + (size_t)(row0 + row) * p.N2 + n0 + half * hc;
+        const float* b2 = p.b2 + n0 + half * hc;
+        for (int c0 = 0; c0 < hc; c0 += 32) {
+          uint32_t v[32];
+          tmem_ld_x32(tmem_base + lane_base + kOutCol + half * hc + c0, v);
+          tmem_ld_wait();
+          if (row_ok) {
 #pragma unroll
-        for (int q = 0; q < 4; ++q) {
-          const float4 b0 = __ldg(reinterpret_cast<const float4*>(b2 + c0 + q * 8));
-          const float4 b1v = __ldg(reinterpret_cast<const float4*>(b2 + c0 + q * 8 + 4));
-          *reinterpret_cast<uint4*>(orow + c0 + q * 8) =
-              make_uint4(pack_bf16x2(__uint_as_float(v[q * 8]) + b0.x, __uint_as_float(v[q * 8 + 1]) + b0.y),
-                         pack_bf16x2(__uint_as_float(v[q * 8 + 2]) + b0.z, __uint_as_float(v[q * 8 + 3]) + b0.w),
-                         pack_bf16x2(__uint_as_float(v[q * 8 + 4]) + b1v.x, __uint_as_float(v[q * 8 + 5]) + b1v.y),
-                         pack_bf16x2(__uint_as_float(v[q * 8 + 6]) + b1v.z, __uint_as_float(v[q * 8 + 7]) + b1v.w));
+            for (int q = 0; q < 4; ++q) {
+              const float4 b0 = __ldg(reinterpret_cast<const float4*>(b2 + c0 + q * 8));
+              const float4 b1v = __ldg(reinterpret_cast<const float4*>(b2 + c0 + q * 8 + 4));
+              *reinterpret_cast<uint4*>(orow + c0 + q * 8) =
+                  make_uint4(pack_bf16x2(__uint_as_float(v[q * 8]) + b0.x, __uint_as_float(v[q * 8 + 1]) + b0.y),
+                             pack_bf16x2(__uint_as_float(v[q * 8 + 2]) + b0.z, __uint_as_float(v[q * 8 + 3]) + b0.w),
+                             pack_bf16x2(__uint_as_float(v[q * 8 + 4]) + b1v.x, __uint_as_float(v[q * 8 + 5]) + b1v.y),
+                             pack_bf16x2(__uint_as_float(v[q * 8 + 6]) + b1v.z, __uint_as_float(v[q * 8 + 7]) + b1v.w));
+            }
+          }
         }
+        tcgen05_fence_before_sync();
+        named_barrier_sync(1, kEpiThreads);
+        if (tid == 0) mbar_arrive(bar_outfree);
       }
     }
   }
@@ -288,14 +305,16 @@ ffn_cluster_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
 struct FfnClusterHost {
   FfnClusterParams prm;
   int smem_bytes = 0;
+  int clusters = 0;   // clusters launched = min(row blocks, clusters the device keeps resident); 0: not asked yet
   struct Key { const void* p; int which; bool operator==(const Key& o) const { return p == o.p && which == o.which; } };
   struct KeyHash { size_t operator()(const Key& k) const { return std::hash<const void*>()(k.p) ^ (size_t)k.which * 0x9e3779b97f4a7c15ull; } };
   std::unordered_map<Key, CUtensorMap, KeyHash> maps;
 };
 
-void fill_launch(cudaLaunchConfig_t* cfg, cudaLaunchAttribute* attr, const FfnClusterParams& q, int smem_bytes, cudaStream_t stream) {
+void fill_launch(cudaLaunchConfig_t* cfg, cudaLaunchAttribute* attr, const FfnClusterParams& q, int clusters, int smem_bytes,
+                 cudaStream_t stream) {
   *cfg = cudaLaunchConfig_t{};
-  cfg->gridDim = dim3((unsigned)q.CS, (unsigned)((q.M + kBM - 1) / kBM), 1);
+  cfg->gridDim = dim3((unsigned)q.CS, (unsigned)clusters, 1);
   cfg->blockDim = dim3(kThreads, 1, 1);
   cfg->dynamicSmemBytes = (size_t)smem_bytes;
   cfg->stream = stream;
@@ -320,13 +339,21 @@ ago_status_t ffn_cluster_plan(Plan* plan, FusedState* st, std::string* err) {
   q.N2 = plan->ops[3].op.p[0];
   if (q.K % kBK != 0 || q.Hid % kBH != 0) return AGO_ERR_UNSUPPORTED;
   const int htiles = q.Hid / kBH;
+  // Cluster size: among the sizes whose column share fits tensor memory, the one with the least estimated time =
+  // rounds of resident clusters x steps per row block x ring stages per step. Resident clusters of 1-CTA-per-SM
+  // kernels on a B200 (148 SMs in GPCs of unequal size), as cudaOccupancyMaxActiveClusters reports them: 74 / 45 / 33
+  // for sizes 2 / 3 / 4; the launch asks the device again and sizes its grid by the answer.
+  const int row_blocks_plan = (q.M + kBM - 1) / kBM;
+  const int resident[kMaxCS + 1] = {0, 0, 74, 45, 33};
   q.CS = 0;
-  for (int cs = 2; cs <= kMaxCS; ++cs) {   // the smallest cluster whose column share fits tensor memory
+  long best = 0;
+  for (int cs = 2; cs <= kMaxCS; ++cs) {
     if (q.N2 % cs != 0 || htiles % cs != 0) continue;
     const int nc = q.N2 / cs;
     if (nc % 64 != 0 || nc > 256) continue;
-    q.CS = cs; q.NC = nc;
-    break;
+    const long rounds = (row_blocks_plan + resident[cs] - 1) / resident[cs];
+    const long cost = rounds * (htiles / cs) * (q.K / kBK + 2 * cs);
+    if (q.CS == 0 || cost < best) { q.CS = cs; q.NC = nc; best = cost; }
   }
   if (q.CS == 0) return AGO_ERR_UNSUPPORTED;
   // one cluster per block of 128 rows: worth it only when the clusters fill the SMs; few rows are better served by the
@@ -380,7 +407,19 @@ ago_status_t ffn_cluster_run(const Plan& plan, FusedState* st, const void* const
     if (e != cudaSuccess) { *err = std::string("cudaFuncSetAttribute: ") + cudaGetErrorString(e); return AGO_ERR_CUDA; }
   }
   cudaLaunchConfig_t cfg; cudaLaunchAttribute attr[2];
-  fill_launch(&cfg, attr, q, host->smem_bytes, stream);
+  const int row_blocks = (q.M + kBM - 1) / kBM;
+  if (host->clusters == 0) {
+    // persistent clusters: as many as the device keeps resident at once (one CTA per SM, CS SMs of one GPC each)
+    fill_launch(&cfg, attr, q, row_blocks, host->smem_bytes, stream);
+    int resident = 0;
+    cudaError_t e = cudaOccupancyMaxActiveClusters(&resident, ffn_cluster_kernel, &cfg);
+    if (e != cudaSuccess || resident < 1) {
+      *err = std::string("fused feed-forward (cluster): no cluster of this size is schedulable: ") + cudaGetErrorString(e);
+      return AGO_ERR_CUDA;
+    }
+    host->clusters = std::min(row_blocks, resident);
+  }
+  fill_launch(&cfg, attr, q, host->clusters, host->smem_bytes, stream);
   cudaError_t e = cudaLaunchKernelEx(&cfg, ffn_cluster_kernel, mx, mw1, mw2, q);
   if (e != cudaSuccess) { *err = std::string("fused feed-forward (cluster) launch: ") + cudaGetErrorString(e); return AGO_ERR_CUDA; }
   return AGO_OK;
