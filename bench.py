@@ -42,7 +42,8 @@ NCU_TRAFFIC_BYTES = {
     ("mbv2_56", "fused"): 4904192 + 0,            # profiles/mbv2_fused_kernel__mbv2_56.txt (output still dirty in L2)
     ("attn_384", "fused"): 56694784 + 719104,     # profiles/attention_fused_kernel__attn_384.txt
     ("resnet_56", "fused"): 13311744 + 3840,      # profiles/conv3x3_pair_kernel__resnet_56.txt
-    ("ffn_12288", "fused"): 66143488 + 9655552,   # profiles/ffn_fused_kernel__ffn_12288.txt
+    ("ffn_12288", "fused"): 28403712 + 1280,      # profiles/ffn_cluster_kernel__ffn_12288.txt (output still dirty in L2)
+    ("ffn_512", "fused"): 11877632 + 0,           # profiles/ffn_fused_kernel__ffn_512.txt
     ("pw_dw_56", "fused"): 4894464 + 5120,        # profiles/mbv2_fused_kernel__pw_dw_56.txt
     ("dw_pw_56", "fused"): 28972032 + 512,        # profiles/mbv2_fused_kernel__dw_pw_56.txt
     ("dw_dw_56", "fused"): 28978432 + 962560,     # profiles/dwdw_fused_kernel__dw_dw_56.txt
