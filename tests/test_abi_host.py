@@ -173,6 +173,13 @@ def test_null_and_misaligned_arguments_are_rejected_before_any_cuda_call():
     sg.close()
 
 
+def test_launch_floor_entry_validates_its_sizes_before_any_cuda_call():
+    lib = B.load()
+    for grid, block, smem in ((0, 128, 0), (70000, 128, 0), (1, 0, 0), (1, 2048, 0), (1, 128, -1), (1, 128, 300 * 1024)):
+        assert lib.ago_launch_empty(grid, block, smem, None) == B.AGO_ERR_INVALID_ARG
+        assert "ago_launch_empty" in B.ago_last_error()[1]
+
+
 def test_bf16_helpers_round_to_nearest_even():
     x = np.array([1.0, 1.00390625, 1.001953125, 1.005859375, -2.5, 3.0e38], dtype=np.float32)
     r = WL.bf16_round(x)
