@@ -44,6 +44,7 @@ struct DwDwParams {
   int N, H, W, C;
   int R, strips, NC, IW;      // output rows per CTA, strips per image, channel chunks, W + 2
   int nseg;                   // 7-column segments per row
+  int step_r, step_c;         // kThreads / 2 pixels as (rows, columns) of the image width
   uint32_t w_recip, nseg_recip;
   int x_plane, m_plane, d_plane;   // byte distance between the two 8-channel planes of each buffer
   int off_x, off_m, off_d;
@@ -70,12 +71,20 @@ dwdw_fused_kernel(const DwDwParams p) {
   {
     const uint8_t* xin = reinterpret_cast<const uint8_t*>(p.x) + ((int64_t)n * p.H + gx0) * p.W * p.C * 2 + c * kChunk * 2;
     const int pieces = XH * p.W * 2;
+    // piece i = (pixel i / 2, plane i % 2); a thread's pieces are kThreads / 2 pixels apart: row and column advance
+    // by fixed steps (one wrap at most), so the division is done once
+    int pix = tid >> 1;
+    const int plane = tid & 1;
+    int ih = (int)fast_div((uint32_t)pix, (uint32_t)p.W, p.w_recip), iw = pix - ih * p.W;
+    const uint8_t* src = xin + (int64_t)pix * p.C * 2 + plane * 16;
+    uint32_t dst = sx + (uint32_t)(plane * p.x_plane + (ih * p.IW + iw + 1) * 16);
+    const int64_t src_step = (int64_t)(kThreads / 2) * p.C * 2;
+    const uint32_t dst_step = (uint32_t)((p.step_r * p.IW + p.step_c) * 16);
     for (int i = tid; i < pieces; i += kThreads) {
-      const int pix = i >> 1, plane = i & 1;
-      const int ih = (int)fast_div((uint32_t)pix, (uint32_t)p.W, p.w_recip), iw = pix - ih * p.W;
       const bool in = gx0 + ih >= 0 && gx0 + ih < p.H;
-      cp_async_16(sx + (uint32_t)(plane * p.x_plane + (ih * p.IW + iw + 1) * 16),
-                  in ? xin + (int64_t)pix * p.C * 2 + plane * 16 : reinterpret_cast<const uint8_t*>(p.x), in ? 16u : 0u);
+      cp_async_16(dst, in ? src : reinterpret_cast<const uint8_t*>(p.x), in ? 16u : 0u);
+      src += src_step; dst += dst_step; ih += p.step_r; iw += p.step_c;
+      if (iw >= p.W) { iw -= p.W; ++ih; dst += 2u * 16u; }   // the next row starts two padding columns later
     }
     cp_async_commit();
   }
@@ -141,11 +150,12 @@ dwdw_fused_kernel(const DwDwParams p) {
   {
     __nv_bfloat16* o0 = p.out + ((size_t)n * p.H + ho0) * p.W * p.C + c * kChunk;
     const int pieces = rows_valid * p.W * 2;
-    for (int i = tid; i < pieces; i += kThreads) {
-      const int pix = i >> 1, plane = i & 1;
-      *reinterpret_cast<uint4*>(o0 + (size_t)pix * p.C + plane * 8) =
-          *reinterpret_cast<const uint4*>(smem + p.off_d + plane * p.d_plane + pix * 16);
-    }
+    const int plane = tid & 1;
+    __nv_bfloat16* dst = o0 + (size_t)(tid >> 1) * p.C + plane * 8;
+    const uint8_t* src = smem + p.off_d + plane * p.d_plane + (tid >> 1) * 16;
+    const size_t dst_step = (size_t)(kThreads / 2) * p.C;
+    for (int i = tid; i < pieces; i += kThreads, dst += dst_step, src += (kThreads / 2) * 16)
+      *reinterpret_cast<uint4*>(dst) = *reinterpret_cast<const uint4*>(src);
   }
 }
 
@@ -188,6 +198,7 @@ ago_status_t dwdw_plan(Plan* plan, FusedState* st, std::string* err) {
   q.IW = q.W + 2;
   q.nseg = (q.W + kSegCols - 1) / kSegCols;
   q.w_recip = fast_div_recip(q.W);
+  q.step_r = (kThreads / 2) / q.W; q.step_c = (kThreads / 2) % q.W;
   q.nseg_recip = fast_div_recip(q.nseg);
   // Rows per CTA: the halo (4 input rows, 2 intermediate rows) is amortised over R rows, while at least two CTAs
   // should share an SM (one computes while the other copies) and the grid should cover the SMs a few times.
