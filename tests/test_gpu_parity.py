@@ -328,6 +328,18 @@ def test_fused_conv3x3_pads_the_intermediate_not_the_input(ago):
     assert_close(run_gpu(ago, wl, data, "fused"), ref, what="resnet pad/fused")
 
 
+@pytest.mark.parametrize("name", ["mbv2_56", "resnet_56", "pw_pw_56"])
+def test_unfused_baseline_full_size_on_sampled_images(ago, name):
+    # the per-mini-subgraph baseline at the size the bench times it (tensor-core stage kernels, their tile choices)
+    wl = WL.get(name)
+    data = WL.generate(wl)
+    gpu = run_gpu(ago, wl, data, "per_mini_subgraph")
+    for img in (0, wl.samples - 1):
+        one = WL.get(name, batch=1)
+        ref = O.run_chain(one.ops, [data["inputs"][0][img:img + 1]], data["weights"])
+        assert_close(gpu[img:img + 1], ref, what=f"{name} per_mini_subgraph image {img}")
+
+
 def test_fused_resnet_full_size_on_sampled_images(ago):
     wl = WL.get("resnet_56")
     data = WL.generate(wl)
