@@ -62,6 +62,7 @@ struct ConvParams {
   int w_row_bytes, w_swizzle, w_stage_bytes;
   int wstages;             // ring stages in use (2..kMaxWStages)
   int off_x, off_y, off_w, off_bias, off_bar;
+  uint32_t wp_recip;        // 2^32 / Wp + 1: pixel index -> (row, column) of the padded strip without a division
 };
 
 // SINGLE = false: the fused pair. SINGLE = true: one convolution with its simple operators (second-convolution
@@ -198,12 +199,21 @@ conv3x3_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
     // P3: intermediate = ReLU(acc + b1) inside the image, 0 outside -> swizzled rows; group A, then group B
     const uint32_t y_addr = smem_u32(sY);
     const uint32_t swz_mask = ((uint32_t)p.w_row_bytes >> 4) - 1u;
+    // a thread's columns are fixed (ncol == 16 for 16, 32 and 64 channels): its biases stay in registers
+    float bias1[16], bias2[16];
+#pragma unroll
+    for (int j = 0; j < 16; j += 4) {
+      const float4 u = has_cols ? *reinterpret_cast<const float4*>(sBias + col0 + j) : make_float4(0.f, 0.f, 0.f, 0.f);
+      const float4 w = has_cols ? *reinterpret_cast<const float4*>(sBias + p.C + col0 + j) : make_float4(0.f, 0.f, 0.f, 0.f);
+      bias1[j] = u.x; bias1[j + 1] = u.y; bias1[j + 2] = u.z; bias1[j + 3] = u.w;
+      bias2[j] = w.x; bias2[j + 1] = w.y; bias2[j + 2] = w.z; bias2[j + 3] = w.w;
+    }
     for (int grp = 0; grp < (SINGLE ? 0 : 2); ++grp) {
       mbar_wait(bar_acc1 + grp, 0, abort_flag, p.status, 0x405);
       tcgen05_fence_after_sync();
       for (int mt = pass_lo[grp]; mt < pass_hi[grp] && has_cols; ++mt) {
         const int m = mt * 128 + row;
-        const int a = m / p.Wp, b = m - a * p.Wp;
+        const int a = (int)fast_div((uint32_t)m, (uint32_t)p.Wp, p.wp_recip), b = m - a * p.Wp;
         const int gh = h0 - 1 + a;
         const bool inside = m < p.P1 && gh >= 0 && gh < p.H && b >= 1 && b <= p.W;
         for (int c0 = col0; c0 < col0 + ncol; c0 += 16) {
@@ -213,8 +223,8 @@ conv3x3_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
           uint32_t w[8];
 #pragma unroll
           for (int j = 0; j < 8; ++j) {
-            const float y0 = fmaxf(__uint_as_float(v[2 * j]) + sBias[c0 + 2 * j], 0.0f);
-            const float y1 = fmaxf(__uint_as_float(v[2 * j + 1]) + sBias[c0 + 2 * j + 1], 0.0f);
+            const float y0 = fmaxf(__uint_as_float(v[2 * j]) + bias1[2 * j], 0.0f);
+            const float y1 = fmaxf(__uint_as_float(v[2 * j + 1]) + bias1[2 * j + 1], 0.0f);
             w[j] = inside ? pack_bf16x2(y0, y1) : 0u;
           }
           if (m < p.P1 + p.Wp) {   // a little past the tile so that shifted reads of valid rows never see stale data
@@ -239,7 +249,6 @@ conv3x3_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
     // warp's 16-byte stores would hit 32 different lines each. Instead the warp transposes its [32 pixels x ncol]
     // block through a private 2 KB staging area (the start of the input rows, no longer read by then), so that
     // consecutive lanes store consecutive 16-byte chunks of a pixel.
-    const float* sB2 = sBias + p.C;
     const bool stage = p.stage_ok != 0;
     const uint32_t stg = smem_u32(sX) + (uint32_t)warp * 2048u;
     const int chl = ncol == 32 ? 2 : 1;                  // log2(16-byte chunks per staged row)
@@ -249,7 +258,7 @@ conv3x3_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
       for (int mt = pass_lo[2 + grp]; mt < pass_hi[2 + grp] || mt == pass_lo[2 + grp]; ++mt) {
         const bool tile_ok = mt < pass_hi[2 + grp];
         const int m = mt * 128 + row;
-        const int r = m / p.Wp, cc = m - r * p.Wp;
+        const int r = (int)fast_div((uint32_t)m, (uint32_t)p.Wp, p.wp_recip), cc = m - r * p.Wp;
         const bool valid = tile_ok && has_cols && r < rows_valid && cc >= 1 && cc <= p.W;
         const size_t pix = ((size_t)n * p.H + h0 + r) * p.W + (cc - 1);
         const bool do_res = SINGLE ? p.residual != 0 : true, do_relu = SINGLE ? p.relu != 0 : true;
@@ -278,8 +287,8 @@ conv3x3_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
               uint32_t w[8];
 #pragma unroll
               for (int j = 0; j < 8; ++j) {
-                float y0 = __uint_as_float(v[2 * j]) + sB2[c0 + 2 * j] + bf16_lo(xs[j]);      // xs is zero without a residual
-                float y1 = __uint_as_float(v[2 * j + 1]) + sB2[c0 + 2 * j + 1] + bf16_hi(xs[j]);
+                float y0 = __uint_as_float(v[2 * j]) + bias2[2 * j] + bf16_lo(xs[j]);      // xs is zero without a residual
+                float y1 = __uint_as_float(v[2 * j + 1]) + bias2[2 * j + 1] + bf16_hi(xs[j]);
                 if (do_relu) { y0 = fmaxf(y0, 0.0f); y1 = fmaxf(y1, 0.0f); }
                 w[j] = pack_bf16x2(y0, y1);
               }
@@ -334,6 +343,7 @@ bool conv_layout(ConvParams& q, int R, int* smem_bytes) {
   q.strips = (q.H + R - 1) / R;
   q.IH = R + 4;
   q.Wp = q.W + 2;
+  q.wp_recip = tc::fast_div_recip(q.Wp);
   q.P1 = (R + 2) * q.Wp; q.M1 = (q.P1 + 127) / 128;
   q.P2 = R * q.Wp; q.M2 = (q.P2 + 127) / 128;
   if (q.IH > 256 || q.Wp > 256 || q.M1 * q.C > 512) return false;
@@ -458,6 +468,7 @@ bool conv_layout_single(ConvParams& q, int R, int* smem_bytes) {
   q.strips = (q.H + R - 1) / R;
   q.IH = R + 2;
   q.Wp = q.W + 2;
+  q.wp_recip = tc::fast_div_recip(q.Wp);
   q.P1 = 0; q.M1 = 0;
   q.P2 = R * q.Wp; q.M2 = (q.P2 + 127) / 128;
   if (q.IH > 256 || q.Wp > 256 || q.M2 * q.C > 512) return false;
