@@ -211,7 +211,8 @@ conv3x3_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
     for (int grp = 0; grp < (SINGLE ? 0 : 2); ++grp) {
       mbar_wait(bar_acc1 + grp, 0, abort_flag, p.status, 0x405);
       tcgen05_fence_after_sync();
-      for (int mt = pass_lo[grp]; mt < pass_hi[grp] && has_cols; ++mt) {
+      const int lo1 = grp ? p.a1 : 0, hi1 = grp ? p.M1 : p.a1;   // the group's tiles of the first convolution
+      for (int mt = lo1; mt < hi1 && has_cols; ++mt) {
         const int m = mt * 128 + row;
         const int a = (int)fast_div((uint32_t)m, (uint32_t)p.Wp, p.wp_recip), b = m - a * p.Wp;
         const int gh = h0 - 1 + a;
@@ -255,8 +256,9 @@ conv3x3_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
     const uint32_t rb = (uint32_t)ncol * 2u;             // bytes per staged row
     const uint32_t swz_w = ((uint32_t)lane >> (3 - chl)) & ((1u << chl) - 1u);   // chunk XOR of this lane's row
     for (int grp = 0; grp < 2; ++grp) {
-      for (int mt = pass_lo[2 + grp]; mt < pass_hi[2 + grp] || mt == pass_lo[2 + grp]; ++mt) {
-        const bool tile_ok = mt < pass_hi[2 + grp];
+      const int lo2 = grp ? p.a2 : 0, hi2 = grp ? p.M2 : p.a2;   // the group's tiles of the second convolution
+      for (int mt = lo2; mt < hi2 || mt == lo2; ++mt) {
+        const bool tile_ok = mt < hi2;
         const int m = mt * 128 + row;
         const int r = (int)fast_div((uint32_t)m, (uint32_t)p.Wp, p.wp_recip), cc = m - r * p.Wp;
         const bool valid = tile_ok && has_cols && r < rows_valid && cc >= 1 && cc <= p.W;
@@ -272,7 +274,7 @@ conv3x3_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
           for (int j = 0; j < 4; ++j)
             if (j * 8 < ncol) xr[j] = __ldg(reinterpret_cast<const uint4*>((SINGLE ? p.res : p.x) + pix * p.C + col0 + j * 8));
         }
-        if (mt == pass_lo[2 + grp]) {
+        if (mt == lo2) {
           mbar_wait(bar_acc2 + grp, 0, abort_flag, p.status, 0x406);
           tcgen05_fence_after_sync();
         }
