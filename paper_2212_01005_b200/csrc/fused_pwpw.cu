@@ -205,10 +205,16 @@ pwpw_fused_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
         add[0] = a0.x; add[1] = a0.y; add[2] = a0.z; add[3] = a0.w; add[4] = a1.x; add[5] = a1.y; add[6] = a1.z; add[7] = a1.w;
       }
       uint32_t w[8];
+      float bv[16];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const float4 t4 = *reinterpret_cast<const float4*>(sB1 + g * 16 + 4 * j);
+        bv[4 * j] = t4.x; bv[4 * j + 1] = t4.y; bv[4 * j + 2] = t4.z; bv[4 * j + 3] = t4.w;
+      }
 #pragma unroll
       for (int j = 0; j < 8; ++j) {
-        float y0 = __uint_as_float(v[2 * j]) + sB1[g * 16 + 2 * j] + bf16_lo(add[j]);
-        float y1 = __uint_as_float(v[2 * j + 1]) + sB1[g * 16 + 2 * j + 1] + bf16_hi(add[j]);
+        float y0 = __uint_as_float(v[2 * j]) + bv[2 * j] + bf16_lo(add[j]);
+        float y1 = __uint_as_float(v[2 * j + 1]) + bv[2 * j + 1] + bf16_hi(add[j]);
         if (p.act1) { y0 = relu6f(y0); y1 = relu6f(y1); }
         w[j] = pack_bf16x2(y0, y1);
       }
@@ -240,9 +246,15 @@ pwpw_fused_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
       tmem_ld_x16(tmem_base + lane_base + g * 16, v);
       tmem_ld_wait();
       uint32_t w[8];
+      float bv[16];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const float4 t4 = *reinterpret_cast<const float4*>(sB2 + g * 16 + 4 * j);
+        bv[4 * j] = t4.x; bv[4 * j + 1] = t4.y; bv[4 * j + 2] = t4.z; bv[4 * j + 3] = t4.w;
+      }
 #pragma unroll
       for (int j = 0; j < 8; ++j) {
-        float y0 = __uint_as_float(v[2 * j]) + sB2[g * 16 + 2 * j], y1 = __uint_as_float(v[2 * j + 1]) + sB2[g * 16 + 2 * j + 1];
+        float y0 = __uint_as_float(v[2 * j]) + bv[2 * j], y1 = __uint_as_float(v[2 * j + 1]) + bv[2 * j + 1];
         if (p.act2) { y0 = relu6f(y0); y1 = relu6f(y1); }
         w[j] = pack_bf16x2(y0, y1);
       }
