@@ -64,6 +64,7 @@ struct Mbv2Params {
   __nv_bfloat16* out;
   unsigned int* status;
   int N, H, W, Cin, Cexp, Cout, stride, Ho, Wo, residual;
+  int fold_b1;                  // the expand bias rides in two spare reduction channels of the expand GEMM (Cin < Kp)
   int R, strips, IH, IW, P_x, P_in, M1, M2;   // P_x = IH * W pixels in the input tile, P_in = IH * IW in an E chunk
   int Kp, row_bytes, swizzle;   // input / W1 tiles: padded K, bytes per row, tc::SwizzleMode
   int Coutp, NC;
@@ -151,12 +152,14 @@ mbv2_fused_kernel(const Mbv2Params p) {
     auto x_slot = [&](uint32_t i, const uint8_t*& src) -> uint32_t {
       const uint32_t row = i >> cs, ch = i & cmask;
       src = (ch < cin_chunks && (int)row >= pix_lo && (int)row < pix_hi) ? x0 + row * cin_bytes + ch * 16u : nullptr;
+      if (p.fold_b1 && ch == cin_chunks) src = reinterpret_cast<const uint8_t*>(uintptr_t(1));   // two channels of 1.0 (tag 1)
       return p.off_x + ((i << 4) ^ (((i >> 3) & swz_mask) << 4));
     };
     auto w_slot = [&](uint32_t i, const uint8_t*& src) -> uint32_t {
       if (i < nW1) {
         const uint32_t row = i >> cs, ch = i & cmask;
         src = ch < cin_chunks ? reinterpret_cast<const uint8_t*>(p.w1) + row * cin_bytes + ch * 16u : nullptr;
+        if (p.fold_b1 && ch == cin_chunks) src = reinterpret_cast<const uint8_t*>(reinterpret_cast<uintptr_t>(p.b1 + row) | 2u);   // the bias (tag 2)
         return p.off_w1 + ((i << 4) ^ (((i >> 3) & swz_mask) << 4));
       }
       if ((i -= nW1) < nW3) {
@@ -175,8 +178,17 @@ mbv2_fused_kernel(const Mbv2Params p) {
       src = reinterpret_cast<const uint8_t*>(p.b3) + i * 16u;
       return p.off_b3 + i * 16u;
     };
+    // A slot's source: a 16-byte aligned address (or null: zeros); tag 1: the two channels of ones that multiply the
+    // folded bias; tag 2: the address of one fp32 bias, split into bf16 high and low parts (their sum carries 16
+    // mantissa bits, and 1.0 * part is exact in the fp32 accumulator).
     auto load_or_zero = [](const uint8_t* src) {
-      return src ? __ldg(reinterpret_cast<const uint4*>(src)) : make_uint4(0, 0, 0, 0);
+      const uintptr_t a = reinterpret_cast<uintptr_t>(src);
+      if ((a & 3u) == 0u) return src ? __ldg(reinterpret_cast<const uint4*>(src)) : make_uint4(0, 0, 0, 0);
+      if ((a & 3u) == 1u) return make_uint4(0x3F803F80u, 0, 0, 0);
+      const float b = __ldg(reinterpret_cast<const float*>(a & ~uintptr_t(3)));
+      const __nv_bfloat16 hi = __float2bfloat16_rn(b);
+      const __nv_bfloat16 lo = __float2bfloat16_rn(b - __bfloat162float(hi));
+      return make_uint4((uint32_t)__bfloat16_as_ushort(hi) | ((uint32_t)__bfloat16_as_ushort(lo) << 16), 0, 0, 0);
     };
     // ---- per-thread work mapping: needs no device memory, so it runs before the wait for the previous grid of the
     // stream (with back-to-back launches it overlaps that grid's tail) ----
@@ -406,7 +418,10 @@ mbv2_fused_kernel(const Mbv2Params p) {
         tmem_ld_wait();
         if (e_off[k] != kNone) {
           uint32_t w[8];
-          if ((e_inimg >> k) & 1u) {
+          if (((e_inimg >> k) & 1u) && p.fold_b1) {   // the bias came out of the expand GEMM
+#pragma unroll
+            for (int j = 0; j < 8; ++j) w[j] = relu6_pack(__uint_as_float(acc[2 * j]), __uint_as_float(acc[2 * j + 1]));
+          } else if ((e_inimg >> k) & 1u) {
             const float4 b0 = lds128f<0>(b1_addr), b1v = lds128f<16>(b1_addr), b2 = lds128f<32>(b1_addr), b3v = lds128f<48>(b1_addr);
             w[0] = relu6_pack(__uint_as_float(acc[0]) + b0.x, __uint_as_float(acc[1]) + b0.y);
             w[1] = relu6_pack(__uint_as_float(acc[2]) + b0.z, __uint_as_float(acc[3]) + b0.w);
@@ -612,6 +627,7 @@ ago_status_t mbv2_plan(Plan* plan, FusedState* st, std::string* err) {
   q.row_bytes = q.Kp * 2;
   q.swizzle = q.Kp == 16 ? tc::SW_32B : (q.Kp == 32 ? tc::SW_64B : tc::SW_128B);
   q.Coutp = round_up(q.Cout, 16);
+  q.fold_b1 = expand && q.Cin % 8 == 0 && q.Cin < q.Kp ? 1 : 0;
   q.NC = q.Cexp / kChunk;
   auto recip = [](int d) { return tc::fast_div_recip(d); };
   q.coutp_recip = recip(q.Coutp);
