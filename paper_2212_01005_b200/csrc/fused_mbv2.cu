@@ -88,10 +88,11 @@ __device__ __forceinline__ void sts128(uint32_t saddr, uint32_t a, uint32_t b, u
   asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(saddr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
 }
 
-// EXPAND / PROJECT select the pairs of the block: <true, true> the whole block, <true, false> pointwise -> depthwise
+// FOLD: the expand bias rides in the expand GEMM (see the prologue). EXPAND / PROJECT select the pairs of the
+// block: <true, true> the whole block, <true, false> pointwise -> depthwise
 // (the depthwise result of every chunk goes to device memory), <false, true> depthwise -> pointwise (every chunk of
 // the input is copied into the E buffers instead of being computed).
-template <bool EXPAND, bool PROJECT>
+template <bool EXPAND, bool PROJECT, bool FOLD>
 __global__ void __launch_bounds__(kThreads, 1)
 mbv2_fused_kernel(const Mbv2Params p) {
   extern __shared__ uint8_t smem_raw[];
@@ -152,14 +153,14 @@ mbv2_fused_kernel(const Mbv2Params p) {
     auto x_slot = [&](uint32_t i, const uint8_t*& src) -> uint32_t {
       const uint32_t row = i >> cs, ch = i & cmask;
       src = (ch < cin_chunks && (int)row >= pix_lo && (int)row < pix_hi) ? x0 + row * cin_bytes + ch * 16u : nullptr;
-      if (p.fold_b1 && ch == cin_chunks) src = reinterpret_cast<const uint8_t*>(uintptr_t(1));   // two channels of 1.0 (tag 1)
+      if (FOLD && ch == cin_chunks) src = reinterpret_cast<const uint8_t*>(uintptr_t(1));   // two channels of 1.0 (tag 1)
       return p.off_x + ((i << 4) ^ (((i >> 3) & swz_mask) << 4));
     };
     auto w_slot = [&](uint32_t i, const uint8_t*& src) -> uint32_t {
       if (i < nW1) {
         const uint32_t row = i >> cs, ch = i & cmask;
         src = ch < cin_chunks ? reinterpret_cast<const uint8_t*>(p.w1) + row * cin_bytes + ch * 16u : nullptr;
-        if (p.fold_b1 && ch == cin_chunks) src = reinterpret_cast<const uint8_t*>(reinterpret_cast<uintptr_t>(p.b1 + row) | 2u);   // the bias (tag 2)
+        if (FOLD && ch == cin_chunks) src = reinterpret_cast<const uint8_t*>(reinterpret_cast<uintptr_t>(p.b1 + row) | 2u);   // the bias (tag 2)
         return p.off_w1 + ((i << 4) ^ (((i >> 3) & swz_mask) << 4));
       }
       if ((i -= nW1) < nW3) {
@@ -183,7 +184,7 @@ mbv2_fused_kernel(const Mbv2Params p) {
     // mantissa bits, and 1.0 * part is exact in the fp32 accumulator).
     auto load_or_zero = [](const uint8_t* src) {
       const uintptr_t a = reinterpret_cast<uintptr_t>(src);
-      if ((a & 3u) == 0u) return src ? __ldg(reinterpret_cast<const uint4*>(src)) : make_uint4(0, 0, 0, 0);
+      if (!FOLD || (a & 3u) == 0u) return src ? __ldg(reinterpret_cast<const uint4*>(src)) : make_uint4(0, 0, 0, 0);
       if ((a & 3u) == 1u) return make_uint4(0x3F803F80u, 0, 0, 0);
       const float b = __ldg(reinterpret_cast<const float*>(a & ~uintptr_t(3)));
       const __nv_bfloat16 hi = __float2bfloat16_rn(b);
@@ -418,7 +419,7 @@ mbv2_fused_kernel(const Mbv2Params p) {
         tmem_ld_wait();
         if (e_off[k] != kNone) {
           uint32_t w[8];
-          if (((e_inimg >> k) & 1u) && p.fold_b1) {   // the bias came out of the expand GEMM
+          if (FOLD && ((e_inimg >> k) & 1u)) {   // the bias came out of the expand GEMM
 #pragma unroll
             for (int j = 0; j < 8; ++j) w[j] = relu6_pack(__uint_as_float(acc[2 * j]), __uint_as_float(acc[2 * j + 1]));
           } else if ((e_inimg >> k) & 1u) {
@@ -665,13 +666,13 @@ ago_status_t mbv2_plan(Plan* plan, FusedState* st, std::string* err) {
 
 namespace {
 
-template <bool EXPAND, bool PROJECT>
+template <bool EXPAND, bool PROJECT, bool FOLD>
 ago_status_t launch_variant(const Mbv2Params& q, int smem_bytes, cudaStream_t stream, std::string* err) {
   static int smem_opt_in[64] = {};
-  cudaError_t e = ensure_max_dynamic_smem(reinterpret_cast<const void*>(mbv2_fused_kernel<EXPAND, PROJECT>), smem_opt_in);
+  cudaError_t e = ensure_max_dynamic_smem(reinterpret_cast<const void*>(mbv2_fused_kernel<EXPAND, PROJECT, FOLD>), smem_opt_in);
   if (e != cudaSuccess) { *err = std::string("cudaFuncSetAttribute: ") + cudaGetErrorString(e); return AGO_ERR_CUDA; }
   FusedLaunch launch(dim3((unsigned)(q.N * q.strips)), kThreads, (size_t)smem_bytes, stream);
-  e = cudaLaunchKernelEx(&launch.config, mbv2_fused_kernel<EXPAND, PROJECT>, q);
+  e = cudaLaunchKernelEx(&launch.config, mbv2_fused_kernel<EXPAND, PROJECT, FOLD>, q);
   if (e != cudaSuccess) { *err = std::string("fused inverted-residual launch: ") + cudaGetErrorString(e); return AGO_ERR_CUDA; }
   return AGO_OK;
 }
@@ -689,9 +690,12 @@ ago_status_t mbv2_run(const Plan& plan, FusedState* st, const void* const* input
   if (host->project) { q.w3 = static_cast<const __nv_bfloat16*>(weights[w]); q.b3 = static_cast<const float*>(weights[w + 1]); }
   q.out = static_cast<__nv_bfloat16*>(output);
   q.status = status_word;
-  if (!host->expand) return launch_variant<false, true>(q, host->smem_bytes, stream, err);
-  if (!host->project) return launch_variant<true, false>(q, host->smem_bytes, stream, err);
-  return launch_variant<true, true>(q, host->smem_bytes, stream, err);
+  if (!host->expand) return launch_variant<false, true, false>(q, host->smem_bytes, stream, err);
+  if (!host->project)
+    return q.fold_b1 ? launch_variant<true, false, true>(q, host->smem_bytes, stream, err)
+                     : launch_variant<true, false, false>(q, host->smem_bytes, stream, err);
+  return q.fold_b1 ? launch_variant<true, true, true>(q, host->smem_bytes, stream, err)
+                   : launch_variant<true, true, false>(q, host->smem_bytes, stream, err);
 }
 
 }  // namespace ago
