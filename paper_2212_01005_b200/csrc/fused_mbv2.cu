@@ -242,8 +242,42 @@ mbv2_fused_kernel(const Mbv2Params p) {
 
     uint4 vx[kBX], vw[kBW];
     uint32_t dx[kBX], dw[kBW];
+    // Without the expand GEMM a chunk is 16 channels of the input strip, copied asynchronously into one of the
+    // group's two E buffers two chunks ahead: 16-byte pieces (pixel, 8-channel plane), rows outside the image
+    // zero-filled. The piece geometry is the same for every chunk.
+    constexpr int kPieces = 4;                      // P_x * 2 pieces <= 8 tiles * 128 * 2 over the group's threads
+    uint32_t ld_src[kPieces], ld_dst[kPieces], ld_ok = 0u, ld_in = 0u;
+    const uint8_t* xin = reinterpret_cast<const uint8_t*>(p.x) + ((int64_t)n * p.H + gh0) * p.W * p.Cexp * 2;   // row gh0 may lie outside
+    if (!EXPAND) {
+#pragma unroll
+      for (int k = 0; k < kPieces; ++k) {
+        const int i = gt + k * kGroupThreads;
+        ld_src[k] = 0u; ld_dst[k] = 0u;
+        if (i < p.P_x * 2) {
+          const int pix = i >> 1, plane = i & 1;
+          const int ih = (int)fast_div((uint32_t)pix, (uint32_t)p.W, p.w_recip), iw = pix - ih * p.W;
+          ld_ok |= 1u << k;
+          ld_dst[k] = (uint32_t)(plane * p.e_plane + (ih * p.IW + iw + 1) * 16);
+          if (gh0 + ih >= 0 && gh0 + ih < p.H) { ld_in |= 1u << k; ld_src[k] = (uint32_t)(pix * p.Cexp * 2 + plane * 16); }
+        }
+      }
+    }
+    auto load_chunk = [&](int c, int b) {   // chunk c -> E buffer (g, b); always one commit group
+      if (c < p.NC) {
+        const uint32_t e0 = smem_u32(sE) + (uint32_t)((g * 2 + b) * e_bytes);
+#pragma unroll
+        for (int k = 0; k < kPieces; ++k) {
+          if ((ld_ok >> k) & 1u) {
+            const bool in = (ld_in >> k) & 1u;
+            cp_async_16(e0 + ld_dst[k], in ? xin + ld_src[k] + c * kChunkRowBytes : reinterpret_cast<const uint8_t*>(p.x), in ? 16u : 0u);
+          }
+        }
+      }
+      cp_async_commit();
+    };
     grid_dependency_wait();      // first access to device memory below
     grid_launch_dependents();
+    if (!EXPAND) { load_chunk(g, 0); load_chunk(g + 2, 1); }   // the first two chunks travel while the weights are staged
 #pragma unroll
     for (int k = 0; k < kBX; ++k) {
       const uint32_t i = (uint32_t)(tid + k * kThreads);
@@ -354,40 +388,6 @@ mbv2_fused_kernel(const Mbv2Params p) {
       if (waiter) mbar_wait(bar_e + g, 0, abort_flag, p.status, 0x102);   // the group's first expand GEMM
       named_barrier_sync(gbar, kGroupThreads);
     }
-    // Without the expand GEMM a chunk is 16 channels of the input strip, copied asynchronously into one of the
-    // group's two E buffers two chunks ahead: 16-byte pieces (pixel, 8-channel plane), rows outside the image
-    // zero-filled. The piece geometry is the same for every chunk.
-    constexpr int kPieces = 4;                      // P_x * 2 pieces <= 8 tiles * 128 * 2 over the group's threads
-    uint32_t ld_src[kPieces], ld_dst[kPieces], ld_ok = 0u, ld_in = 0u;
-    const uint8_t* xin = reinterpret_cast<const uint8_t*>(p.x) + ((int64_t)n * p.H + gh0) * p.W * p.Cexp * 2;   // row gh0 may lie outside
-    if (!EXPAND) {
-#pragma unroll
-      for (int k = 0; k < kPieces; ++k) {
-        const int i = gt + k * kGroupThreads;
-        ld_src[k] = 0u; ld_dst[k] = 0u;
-        if (i < p.P_x * 2) {
-          const int pix = i >> 1, plane = i & 1;
-          const int ih = (int)fast_div((uint32_t)pix, (uint32_t)p.W, p.w_recip), iw = pix - ih * p.W;
-          ld_ok |= 1u << k;
-          ld_dst[k] = (uint32_t)(plane * p.e_plane + (ih * p.IW + iw + 1) * 16);
-          if (gh0 + ih >= 0 && gh0 + ih < p.H) { ld_in |= 1u << k; ld_src[k] = (uint32_t)(pix * p.Cexp * 2 + plane * 16); }
-        }
-      }
-    }
-    auto load_chunk = [&](int c, int b) {   // chunk c -> E buffer (g, b); always one commit group
-      if (c < p.NC) {
-        const uint32_t e0 = smem_u32(sE) + (uint32_t)((g * 2 + b) * e_bytes);
-#pragma unroll
-        for (int k = 0; k < kPieces; ++k) {
-          if ((ld_ok >> k) & 1u) {
-            const bool in = (ld_in >> k) & 1u;
-            cp_async_16(e0 + ld_dst[k], in ? xin + ld_src[k] + c * kChunkRowBytes : reinterpret_cast<const uint8_t*>(p.x), in ? 16u : 0u);
-          }
-        }
-      }
-      cp_async_commit();
-    };
-    if (!EXPAND) { load_chunk(g, 0); load_chunk(g + 2, 1); }
     // The thread's first depthwise item (for most shapes its only one) is the same for every chunk: offsets of its
     // first input / output pixel inside a plane and its extent (stride 1: columns, rows; stride 2: first and last row).
     const bool has_item = slot < dw_items;
