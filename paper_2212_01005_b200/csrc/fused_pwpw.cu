@@ -51,6 +51,7 @@ struct PwPwParams {
   __nv_bfloat16* out;        // [M][C2]
   unsigned int* status;
   int M, C0, C1, C2;
+  int BR;                    // rows per tile (<= 128): chosen so that the tiles split evenly over the resident CTAs
   int C0p, C1p, C2p;         // padded to the MMA granularity (16)
   int nkb0, nkb1;            // 64-channel K blocks of the first / second product
   int act1, act2;            // ReLU6 after the first / second convolution
@@ -88,7 +89,7 @@ pwpw_fused_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int k2 = p.C2 >> 3;
-  const int ntiles = (p.M + kBM - 1) / kBM;
+  const int ntiles = (p.M + p.BR - 1) / p.BR;   // tiles of BR <= 128 rows: the MMAs still span 128 rows, the rest is ignored
 
   if (tid == 0) {
     *abort_flag = 0u;
@@ -104,9 +105,9 @@ pwpw_fused_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
   }
   auto load_x = [&](int tile) {   // one thread
     mbar_arrive_expect_tx(bar_x, (uint32_t)p.x_tx);
-    for (int kb = 0; kb < p.nkb0; ++kb) tma_load_2d(sX + kb * kXBlock, &tmap_x, bar_x, kb * kBK, tile * kBM);
+    for (int kb = 0; kb < p.nkb0; ++kb) tma_load_2d(sX + kb * kXBlock, &tmap_x, bar_x, kb * kBK, tile * p.BR);
     if (p.has_res)   // the second product of the previous tile has read this buffer
-      for (int kb = 0; kb < p.nkb1; ++kb) tma_load_2d(sA + kb * kXBlock, &tmap_r, bar_x, kb * kBK, tile * kBM);
+      for (int kb = 0; kb < p.nkb1; ++kb) tma_load_2d(sA + kb * kXBlock, &tmap_r, bar_x, kb * kBK, tile * p.BR);
   };
   grid_dependency_wait();
   grid_launch_dependents();
@@ -164,7 +165,7 @@ pwpw_fused_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
 
   for (int tile = blockIdx.x, it = 0; tile < ntiles; tile += gridDim.x, ++it) {
     const uint32_t par = (uint32_t)it & 1u;
-    const int row0 = tile * kBM, rows = min(kBM, p.M - row0);
+    const int row0 = tile * p.BR, rows = min(p.BR, p.M - row0);
     if (p.perm_a > 0 && tid < kBM) {   // read after two barriers below
       const int m = row0 + tid, ab = p.perm_a * p.perm_b;
       const int g = m / ab, rem = m - g * ab, i = rem / p.perm_b, j = rem - i * p.perm_b;
@@ -332,7 +333,6 @@ ago_status_t pwpw_plan(Plan* plan, FusedState* st, std::string* err) {
   q.w1_block = w1_rows * 128; q.w2_block = w2_rows * 128;
   const int w1_bytes = (w1_chunks + 7) / 8 * q.w1_block, w2_bytes = (w2_chunks + 7) / 8 * q.w2_block;
   q.pitch = q.C2 * 2 + 16;
-  q.x_tx = (q.nkb0 + (q.has_res ? q.nkb1 : 0)) * kXBlock;
   q.tmem_cols = 32;
   while (q.tmem_cols < std::max(q.C1p, q.C2p)) q.tmem_cols *= 2;
   int off = 0;
@@ -348,11 +348,17 @@ ago_status_t pwpw_plan(Plan* plan, FusedState* st, std::string* err) {
   if (host->smem_bytes > 227 * 1024) return bad("the operands of one row tile do not fit shared memory");
   if ((long)kBM * (q.C2 / 8) > 65535 || (long)w1_rows * w1_chunks > 65535 || (long)w2_rows * w2_chunks > 65535)
     return bad("operands too large for the copy index arithmetic");
-  host->grid = std::min((q.M + kBM - 1) / kBM, 2 * 148);
+  // Rows per tile: with k = rounds of 128-row tiles over the resident CTAs, the smallest tile height that still
+  // needs k rounds -- the same number of rounds, less work in each
+  const int per_sm = host->smem_bytes <= 113 * 1024 ? 2 : 1, slots = per_sm * 148;
+  const long k = ((long)(q.M + kBM - 1) / kBM + slots - 1) / slots;
+  q.BR = (int)std::min<long>(kBM, (q.M + k * slots - 1) / (k * slots));
+  q.x_tx = (q.nkb0 + (q.has_res ? q.nkb1 : 0)) * q.BR * 128;
+  host->grid = std::min((q.M + q.BR - 1) / q.BR, slots);
   st->impl = host;
   st->impl_free = [](void* p) { delete static_cast<PwPwHost*>(p); };
-  st->tile_rows = kBM; st->grid = host->grid; st->smem_bytes = host->smem_bytes;
-  plan->tile_rows = kBM; plan->smem_bytes = host->smem_bytes;
+  st->tile_rows = q.BR; st->grid = host->grid; st->smem_bytes = host->smem_bytes;
+  plan->tile_rows = q.BR; plan->smem_bytes = host->smem_bytes;
   return AGO_OK;
 }
 
@@ -377,7 +383,7 @@ ago_status_t pwpw_run(const Plan& plan, FusedState* st, const void* const* input
       CUtensorMap m;
       const uint64_t dims[2] = {(uint64_t)C, (uint64_t)q.M};
       const uint64_t strides[1] = {(uint64_t)C * 2};
-      const uint32_t box[2] = {(uint32_t)kBK, (uint32_t)kBM};
+      const uint32_t box[2] = {(uint32_t)kBK, (uint32_t)q.BR};
       if (!encode_tmap_bf16(&m, base, 2, dims, strides, box, 128, err)) return false;
       if (cache.size() > 4096) cache.clear();
       it = cache.emplace(base, m).first;
