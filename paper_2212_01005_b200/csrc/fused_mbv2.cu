@@ -379,7 +379,12 @@ mbv2_fused_kernel(const Mbv2Params p) {
     const uint32_t proj_d_tmem = tmem_base + p.pcol0 + gw * p.Coutp;
     const uint32_t proj_b_step = (uint32_t)(2 * p.Coutp * kChunkRowBytes) >> 4;     // the group's next chunk is c + 2
     uint32_t proj_b_lo = (uint32_t)w3desc0 + ((uint32_t)(g * p.Coutp * kChunkRowBytes) >> 4);
-    if (EXPAND && xi >= 0 && lane == 0 && g < p.NC) issue_expand();
+    if (EXPAND && xi >= 0 && lane == 0 && g < p.NC) {
+      // group 1 issues its first expand GEMM once group 0's is through the tensor pipe: group 0 has the longer chain
+      // of chunks, and its first epilogue would otherwise wait for both groups' MMAs
+      if (g == 1) mbar_wait(bar_e, 0, abort_flag, p.status, 0x107);
+      issue_expand();
+    }
     __syncwarp();
     // Waits on MMA completion are taken by ONE warp of the group, just before it arrives at the group barrier that
     // the others are parked at: a polling warp spends issue slots, sixteen of them a large share of the SM's.
