@@ -109,6 +109,20 @@ def test_fused_planner_matches_every_chain_family_and_its_limits():
     _expect_fail(ops, wl.input_shapes, B.AGO_ERR_UNSUPPORTED, mode="fused", needle="family")
 
 
+def test_feed_forward_planner_picks_the_cluster_kernel_where_the_shape_splits():
+    # cluster kernel: no workspace (nothing is reduced through device memory); split-reduction kernel: an fp32 buffer
+    def ws(M, K, hid, out):
+        wl = WL.ffn("x", [1], M, K, hid, 1, d_out=out)
+        sg = B.Subgraph(wl.ops, wl.input_shapes, mode="fused")
+        w = sg.workspace_bytes
+        sg.close()
+        return w
+    assert ws(12288, 768, 3072, 768) == 0          # 96 row blocks, clusters of 3 or 4
+    assert ws(9637, 64, 256, 384) == 0             # clusters of 2, ragged last row block
+    assert ws(512, 768, 3072, 768) >= 512 * 768 * 4    # four row blocks do not fill the SMs with clusters
+    assert ws(12800, 256, 384, 256) >= 12800 * 256 * 4  # three hidden tiles, 256 columns: no cluster size divides both
+
+
 def test_layout_operators_in_the_planner():
     wl = WL.get("unfold_96", batch=2)
     per_op = B.Subgraph(wl.ops, wl.input_shapes, mode="per_op")
