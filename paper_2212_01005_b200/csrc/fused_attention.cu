@@ -6,14 +6,17 @@
 // (head_dim) and is tiled over rows (128 queries). The softmax in between is a simple operator
 // over whole rows, so the upstream tile is 128 query rows x ALL keys of the head.
 //
-// A CTA owns one (batch, head): K and V are loaded once and stay in shared memory while the CTA
-// walks over the head's 128-row query tiles. The keys are processed in two halves so that tensor
+// The (batch, head, 128-row query tile) items are numbered in that order and dealt out in equal
+// consecutive runs to one persistent CTA per SM. K and V of the current (batch, head) stay in shared
+// memory while the CTA walks over its query tiles; when the run crosses into the next head, the new K
+// is fetched as soon as the last score product of the old head has completed and the new V as soon as
+// its last P V has, both behind the softmax of the tiles in flight. The keys are processed in two halves so that tensor
 // cores and CUDA cores overlap: while the softmax warps turn half 0 of the scores into
 // probabilities, the MMA warp already computes half 1 (and, later, the next tile's scores). The
 // running row maximum may grow between the halves; the partial output of half 0 is then rescaled
 // in tensor memory by exp(m0 - m1) before half 1 is accumulated -- the result is the exact softmax.
 //
-//   P1  TMA: K, V [S x 64] once per CTA, Q [128 x 64] per tile -> 128-byte-swizzled tiles
+//   P1  TMA: K, V [S x 64] once per head of the run, Q [128 x 64] per tile -> 128-byte-swizzled tiles
 //   P2  tcgen05.mma: S_h[128 x S/2] = Q K_h^T                            (TMEM, fp32, two buffers)
 //   P3/P4  768 threads (6 per query row): TMEM -> registers, row max (exchanged through shared
 //       memory), p = exp2((s - m) * scale * log2 e), bf16 -> shared memory (K-major operand), row sum
@@ -22,6 +25,7 @@
 #include <cuda.h>
 #include <cuda_bf16.h>
 
+#include <algorithm>
 #include <unordered_map>
 
 #include "fused.h"
@@ -42,6 +46,7 @@ constexpr int kComputeThreads = kBlockM * kParts;
 constexpr int kThreads = kComputeThreads + 64;   // + TMA warp + MMA warp
 constexpr int kHalfCols = 192;         // tensor-memory columns reserved per score half
 constexpr uint32_t kOCol = 2 * kHalfCols;
+constexpr int kSMs = 148;              // B200
 
 struct AttnParams {
   __nv_bfloat16* out;
@@ -50,6 +55,7 @@ struct AttnParams {
   int Spad;        // keys rounded up to 16
   int nkb;         // 128-key TMA boxes
   int tiles;       // query tiles per head
+  int total;       // items = B * heads * tiles
   int hw0, hw1;    // keys in half 0 / half 1 (multiples of 16, hw0 >= hw1 > 0)
   int pw0, pw1;    // columns per thread part in each half (multiples of 16)
   float scale_log2e;
@@ -88,28 +94,33 @@ attention_fused_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
   uint64_t* bar_corr = bars + 11;   // output rescaled for half 1
   uint64_t* bar_o1 = bars + 12;     // P V of half 1 complete
   uint64_t* bar_ofree = bars + 13;  // epilogue has read the output accumulators
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 14);
-  volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(bars + 15);
+  uint64_t* bar_vfree = bars + 14;  // the last P V of a head has read V
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 15);
+  volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(bars + 16);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int h = blockIdx.x, b = blockIdx.y;
+  // This CTA's run of items [g0, g0 + n); item g = ((b * heads + h) * tiles + t).
+  const int g0 = (int)((long long)blockIdx.x * p.total / gridDim.x);
+  const int n = (int)((long long)(blockIdx.x + 1) * p.total / gridDim.x) - g0;
+  const int u0 = g0 / p.tiles, t0 = g0 - u0 * p.tiles;
+  const int b0 = u0 / p.heads, h0 = u0 - b0 * p.heads;
   grid_dependency_wait();      // the previous grid of the stream has completed; device memory may be touched
   grid_launch_dependents();
 
   if (tid == kComputeThreads) {
     *abort_flag = 0u;
-    for (int i = 0; i < 14; ++i) mbar_init(bars + i, 1);
+    for (int i = 0; i < 15; ++i) mbar_init(bars + i, 1);
     fence_mbar_init();
     fence_proxy_async_smem();
     tma_prefetch_desc(&tmap_q);
     tma_prefetch_desc(&tmap_k);
     tma_prefetch_desc(&tmap_v);
     mbar_arrive_expect_tx(bar_k, (uint32_t)(p.nkb * kKeyBlock * kD * 2));
-    for (int kb = 0; kb < p.nkb; ++kb) tma_load_3d(sK + kb * kKeyBlock * kD * 2, &tmap_k, bar_k, h * kD, kb * kKeyBlock, b);
+    for (int kb = 0; kb < p.nkb; ++kb) tma_load_3d(sK + kb * kKeyBlock * kD * 2, &tmap_k, bar_k, h0 * kD, kb * kKeyBlock, b0);
     mbar_arrive_expect_tx(bar_q, (uint32_t)(kBlockM * kD * 2));
-    tma_load_3d(sQ, &tmap_q, bar_q, h * kD, 0, b);
+    tma_load_3d(sQ, &tmap_q, bar_q, h0 * kD, t0 * kBlockM, b0);
     mbar_arrive_expect_tx(bar_v, (uint32_t)(p.nkb * kKeyBlock * kD * 2));
-    for (int kb = 0; kb < p.nkb; ++kb) tma_load_3d(sV + kb * kKeyBlock * kD * 2, &tmap_v, bar_v, h * kD, kb * kKeyBlock, b);
+    for (int kb = 0; kb < p.nkb; ++kb) tma_load_3d(sV + kb * kKeyBlock * kD * 2, &tmap_v, bar_v, h0 * kD, kb * kKeyBlock, b0);
   }
   if (warp == 0) {
     tmem_alloc(tmem_slot, 512);
@@ -121,12 +132,26 @@ attention_fused_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
   const uint32_t tmem_base = *tmem_slot;
 
   if (warp == kComputeThreads / 32) {
-    // ============================ TMA producer: the remaining Q tiles ============================
+    // ============================ TMA producer: the remaining Q tiles, K and V of the following heads ============================
     if (lane == 0) {
-      for (int t = 1; t < p.tiles; ++t) {
-        mbar_wait(bar_qfree, (uint32_t)(t - 1) & 1u, abort_flag, p.status, 0x201);
+      int t = t0, h = h0, b = b0;
+      uint32_t heads_done = 0;
+      for (int i = 1; i < n; ++i) {
+        const bool new_head = ++t == p.tiles;
+        if (new_head) { t = 0; if (++h == p.heads) { h = 0; ++b; } }
+        mbar_wait(bar_qfree, (uint32_t)(i - 1) & 1u, abort_flag, p.status, 0x201);   // every score product of item i - 1 has completed
+        if (new_head) {
+          mbar_arrive_expect_tx(bar_k, (uint32_t)(p.nkb * kKeyBlock * kD * 2));
+          for (int kb = 0; kb < p.nkb; ++kb) tma_load_3d(sK + kb * kKeyBlock * kD * 2, &tmap_k, bar_k, h * kD, kb * kKeyBlock, b);
+        }
         mbar_arrive_expect_tx(bar_q, (uint32_t)(kBlockM * kD * 2));
         tma_load_3d(sQ, &tmap_q, bar_q, h * kD, t * kBlockM, b);
+        if (new_head) {
+          mbar_wait(bar_vfree, heads_done & 1u, abort_flag, p.status, 0x216);
+          ++heads_done;
+          mbar_arrive_expect_tx(bar_v, (uint32_t)(p.nkb * kKeyBlock * kD * 2));
+          for (int kb = 0; kb < p.nkb; ++kb) tma_load_3d(sV + kb * kKeyBlock * kD * 2, &tmap_v, bar_v, h * kD, kb * kKeyBlock, b);
+        }
       }
     }
     __syncwarp();
@@ -163,18 +188,23 @@ attention_fused_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
       issue_scores(0);
       issue_scores(1);
       umma_commit(bar_qfree);
-      for (int t = 0; t < p.tiles; ++t) {
-        const uint32_t ph = (uint32_t)t & 1u;
+      int t = t0;
+      uint32_t head_ph = 0;      // parity of the K / V loads of the current head
+      bool first_of_head = true;
+      for (int i = 0; i < n; ++i) {
+        const uint32_t ph = (uint32_t)i & 1u;
+        const bool last_of_head = t + 1 == p.tiles;   // the next item of the run, if any, belongs to the next head
         // ---- half 0 ----
         mbar_wait(bar_p + 0, ph, abort_flag, p.status, 0x204);
-        if (t == 0) mbar_wait(bar_v, 0, abort_flag, p.status, 0x205);
-        if (t > 0) mbar_wait(bar_ofree, ph ^ 1u, abort_flag, p.status, 0x206);
+        if (first_of_head) mbar_wait(bar_v, head_ph, abort_flag, p.status, 0x205);
+        if (i > 0) mbar_wait(bar_ofree, ph ^ 1u, abort_flag, p.status, 0x206);
         tcgen05_fence_after_sync();
         issue_pv(0);
         umma_commit(bar_o0);
         umma_commit(bar_pfree + 0);
-        if (t + 1 < p.tiles) {
+        if (i + 1 < n) {
           mbar_wait(bar_q, ph ^ 1u, abort_flag, p.status, 0x207);
+          if (last_of_head) mbar_wait(bar_k, head_ph ^ 1u, abort_flag, p.status, 0x202);
           tcgen05_fence_after_sync();
           issue_scores(0);                       // next tile's half 0 into the buffer just drained
         }
@@ -185,10 +215,13 @@ attention_fused_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
         issue_pv(1);
         umma_commit(bar_o1);
         umma_commit(bar_pfree + 1);
-        if (t + 1 < p.tiles) {
+        if (last_of_head) umma_commit(bar_vfree);
+        if (i + 1 < n) {
           issue_scores(1);
           umma_commit(bar_qfree);
         }
+        first_of_head = last_of_head;
+        if (last_of_head) { t = 0; head_ph ^= 1u; } else ++t;
       }
     }
     __syncwarp();
@@ -287,7 +320,7 @@ attention_fused_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
     };
 
     float m0 = 0.0f, sum0 = 0.0f;
-    auto do_half0 = [&](int t) {
+    auto do_half0 = [&](int t) {              // t: position of the item in this CTA's run
       const uint32_t ph = (uint32_t)t & 1u;
       mbar_wait(bar_s + 0, ph, abort_flag, p.status, 0x210);
       tcgen05_fence_after_sync();
@@ -303,7 +336,8 @@ attention_fused_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
     };
 
     do_half0(0);
-    for (int t = 0; t < p.tiles; ++t) {
+    int tq = t0, h = h0, b = b0;                // the item's query tile, head and batch
+    for (int t = 0; t < n; ++t) {
       const uint32_t ph = (uint32_t)t & 1u;
       // ---------------- half 1 ----------------
       mbar_wait(bar_s + 1, ph, abort_flag, p.status, 0x212);
@@ -339,7 +373,7 @@ attention_fused_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
       if (tid == 0) mbar_arrive(bar_corr);
 
       // While the tensor core finishes P V of this tile, start on the next tile's first half.
-      if (t + 1 < p.tiles) do_half0(t + 1);
+      if (t + 1 < n) do_half0(t + 1);
 
       // ---------------- epilogue of tile t: O / rowsum -> bf16 -> global ----------------
       mbar_wait(bar_o1, ph, abort_flag, p.status, 0x215);
@@ -348,7 +382,7 @@ attention_fused_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
         uint32_t o[16];
         tmem_ld_x16(tmem_base + lane_base + kOCol + part * 16, o);
         tmem_ld_wait();
-        const int qrow = t * kBlockM + row;
+        const int qrow = tq * kBlockM + row;
         if (qrow < p.S) {
           __nv_bfloat16* dst = p.out + ((size_t)b * p.S + qrow) * p.E + h * kD + part * 16;
 #pragma unroll
@@ -363,6 +397,7 @@ attention_fused_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
       tcgen05_fence_before_sync();
       named_barrier_sync(1, kComputeThreads);
       if (tid == 0) mbar_arrive(bar_ofree);
+      if (++tq == p.tiles) { tq = 0; if (++h == p.heads) { h = 0; ++b; } }
     }
   }
   tcgen05_fence_before_sync();
@@ -394,6 +429,8 @@ ago_status_t attention_plan(Plan* plan, FusedState* st, std::string* err) {
   q.Spad = round16(q.S);
   q.nkb = (q.Spad + kKeyBlock - 1) / kKeyBlock;
   q.tiles = (q.S + kBlockM - 1) / kBlockM;
+  if ((long long)q.B * q.heads * q.tiles > 0x7fffffffLL) return bad("too many query tiles");
+  q.total = q.B * q.heads * q.tiles;
   q.hw0 = round16((q.Spad + 1) / 2);
   q.hw1 = q.Spad - q.hw0;
   q.pw0 = round16((q.hw0 + kParts - 1) / kParts);
@@ -412,7 +449,7 @@ ago_status_t attention_plan(Plan* plan, FusedState* st, std::string* err) {
   if (host->smem_bytes > 227 * 1024) return bad("shared memory budget exceeded");
   st->impl = host;
   st->impl_free = [](void* p) { delete static_cast<AttnHost*>(p); };
-  st->tile_rows = kBlockM; st->grid = q.heads * q.B; st->smem_bytes = host->smem_bytes;
+  st->tile_rows = kBlockM; st->grid = std::min(q.total, kSMs); st->smem_bytes = host->smem_bytes;
   plan->tile_rows = kBlockM; plan->smem_bytes = host->smem_bytes;
   return AGO_OK;
 }
@@ -442,7 +479,7 @@ ago_status_t attention_run(const Plan& plan, FusedState* st, const void* const* 
     cudaError_t e = ensure_max_dynamic_smem(reinterpret_cast<const void*>(attention_fused_kernel), smem_opt_in);
     if (e != cudaSuccess) { *err = std::string("cudaFuncSetAttribute: ") + cudaGetErrorString(e); return AGO_ERR_CUDA; }
   }
-  dim3 grid(q.heads, q.B);
+  dim3 grid((unsigned)std::min(q.total, kSMs));     // one persistent CTA per SM (the shared memory admits no second one)
   FusedLaunch launch(grid, kThreads, (size_t)host->smem_bytes, stream);
   cudaError_t e = cudaLaunchKernelEx(&launch.config, attention_fused_kernel, *maps[0], *maps[1], *maps[2], q);
   if (e != cudaSuccess) { *err = std::string("fused attention launch: ") + cudaGetErrorString(e); return AGO_ERR_CUDA; }

@@ -37,6 +37,10 @@ def small_workloads():
         "resnet_16ch": WL.resnet_block("resnet_16ch", [32], 2, 20, 16),
         "attn_small": WL.attention("attn_small", [28], 2, 128, 2, 64),
         "attn_ragged": WL.attention("attn_ragged", [29], 1, 200, 3, 64),
+        # more query tiles than SMs: the persistent CTAs' runs of 1-2 and of 3-4 items cross from one head (and batch) into the next
+        # at every position of a run; ragged last tiles
+        "attn_runs2": WL.attention("attn_runs2", [36], 5, 200, 16, 64),
+        "attn_runs4": WL.attention("attn_runs4", [37], 8, 296, 20, 64),
     }
 
 
@@ -118,7 +122,7 @@ def test_padding_of_the_intermediate_with_large_bias(ago):
 
 # ---- fused kernels -------------------------------------------------------------------
 
-FUSED_SMALL = ["mbv2_14", "mbv2_s1_odd", "mbv2_s2", "mbv2_s2_odd", "attn_small", "attn_ragged", "ffn_small", "ffn_rows_ragged", "ffn_g2", "ffn_g3",
+FUSED_SMALL = ["mbv2_14", "mbv2_s1_odd", "mbv2_s2", "mbv2_s2_odd", "attn_small", "attn_ragged", "attn_runs2", "attn_runs4", "ffn_small", "ffn_rows_ragged", "ffn_g2", "ffn_g3",
                "ffn_c2", "ffn_c3", "ffn_c4", "resnet_small", "resnet_odd", "resnet_16ch"]
 
 
