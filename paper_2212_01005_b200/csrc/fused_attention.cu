@@ -21,7 +21,9 @@
 //   P3/P4  768 threads (6 per query row): TMEM -> registers, row max (exchanged through shared
 //       memory), p = exp2((s - m) * scale * log2 e), bf16 -> shared memory (K-major operand), row sum
 //   P5  tcgen05.mma: O[128 x 64] (+)= P_h V_h       (V is the N-major B operand, as it lies in HBM)
-//   P6  TMEM -> registers, * 1 / rowsum, bf16, 32-byte stores
+//   P6  TMEM -> registers, * 1 / rowsum, bf16 -> a swizzled tile in shared memory (the probability buffer of half 1, idle
+//       by then) -> one TMA store per tile (a row of one head is 128 bytes of a 2 E-byte output row: stores from
+//       the row-per-lane accumulator layout would touch 32 lines per instruction)
 #include <cuda.h>
 #include <cuda_bf16.h>
 
@@ -72,7 +74,8 @@ __device__ __forceinline__ float ex2_approx(float x) {
 
 __global__ void __launch_bounds__(kThreads, 1)
 attention_fused_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
-                       const __grid_constant__ CUtensorMap tmap_v, const AttnParams p) {
+                       const __grid_constant__ CUtensorMap tmap_v, const __grid_constant__ CUtensorMap tmap_o,
+                       const AttnParams p) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t* sQ = smem + p.off_q;
@@ -115,6 +118,7 @@ attention_fused_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
     tma_prefetch_desc(&tmap_q);
     tma_prefetch_desc(&tmap_k);
     tma_prefetch_desc(&tmap_v);
+    tma_prefetch_desc(&tmap_o);
     mbar_arrive_expect_tx(bar_k, (uint32_t)(p.nkb * kKeyBlock * kD * 2));
     for (int kb = 0; kb < p.nkb; ++kb) tma_load_3d(sK + kb * kKeyBlock * kD * 2, &tmap_k, bar_k, h0 * kD, kb * kKeyBlock, b0);
     mbar_arrive_expect_tx(bar_q, (uint32_t)(kBlockM * kD * 2));
@@ -343,6 +347,7 @@ attention_fused_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
       mbar_wait(bar_s + 1, ph, abort_flag, p.status, 0x212);
       tcgen05_fence_after_sync();
       sMax1[part * kBlockM + row] = load_half_and_max(1);
+      if (tid == 0) bulk_wait_group_read_all();      // the previous tile's output store has read its staging tile (the half-1 buffer)
       named_barrier_sync(1, kComputeThreads);
       const float m1 = fmaxf(m0, reduce_parts(sMax1, true));
       const float alpha = ex2_approx((m0 - m1) * c);     // rescales everything accumulated under the old maximum
@@ -382,23 +387,26 @@ attention_fused_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
         uint32_t o[16];
         tmem_ld_x16(tmem_base + lane_base + kOCol + part * 16, o);
         tmem_ld_wait();
-        const int qrow = tq * kBlockM + row;
-        if (qrow < p.S) {
-          __nv_bfloat16* dst = p.out + ((size_t)b * p.S + qrow) * p.E + h * kD + part * 16;
+        uint8_t* stage = sP + p.p_half_bytes;      // P V of half 1 has completed: its probabilities are dead
 #pragma unroll
-          for (int j = 0; j < 2; ++j)
-            *reinterpret_cast<uint4*>(dst + j * 8) =
-                make_uint4(pack_bf16x2(__uint_as_float(o[8 * j]) * inv, __uint_as_float(o[8 * j + 1]) * inv),
-                           pack_bf16x2(__uint_as_float(o[8 * j + 2]) * inv, __uint_as_float(o[8 * j + 3]) * inv),
-                           pack_bf16x2(__uint_as_float(o[8 * j + 4]) * inv, __uint_as_float(o[8 * j + 5]) * inv),
-                           pack_bf16x2(__uint_as_float(o[8 * j + 6]) * inv, __uint_as_float(o[8 * j + 7]) * inv));
-        }
+        for (int j = 0; j < 2; ++j)
+          *reinterpret_cast<uint4*>(stage + swz_offset(row, (uint32_t)(part * 2 + j), 128)) =
+              make_uint4(pack_bf16x2(__uint_as_float(o[8 * j]) * inv, __uint_as_float(o[8 * j + 1]) * inv),
+                         pack_bf16x2(__uint_as_float(o[8 * j + 2]) * inv, __uint_as_float(o[8 * j + 3]) * inv),
+                         pack_bf16x2(__uint_as_float(o[8 * j + 4]) * inv, __uint_as_float(o[8 * j + 5]) * inv),
+                         pack_bf16x2(__uint_as_float(o[8 * j + 6]) * inv, __uint_as_float(o[8 * j + 7]) * inv));
       }
+      fence_proxy_async_smem();
       tcgen05_fence_before_sync();
       named_barrier_sync(1, kComputeThreads);
-      if (tid == 0) mbar_arrive(bar_ofree);
+      if (tid == 0) {
+        mbar_arrive(bar_ofree);
+        tma_store_3d(&tmap_o, sP + p.p_half_bytes, h * kD, tq * kBlockM, b);   // rows past S are clipped
+        bulk_commit_group();
+      }
       if (++tq == p.tiles) { tq = 0; if (++h == p.heads) { h = 0; ++b; } }
     }
+    if (tid == 0) bulk_wait_group_all();
   }
   tcgen05_fence_before_sync();
   __syncthreads();
@@ -460,17 +468,22 @@ ago_status_t attention_run(const Plan& plan, FusedState* st, const void* const* 
   AttnParams q = host->prm;
   q.out = static_cast<__nv_bfloat16*>(output);
   q.status = status_word;
-  const CUtensorMap* maps[3];
-  for (int i = 0; i < 3; ++i) {
-    auto it = host->maps.find(inputs[i]);
+  const CUtensorMap* maps[4];
+  for (int i = 0; i < 4; ++i) {
+    const void* base = i < 3 ? inputs[i] : output;
+    auto it = host->maps.find(base);
     if (it == host->maps.end()) {
       CUtensorMap m;
       const uint64_t dims[3] = {(uint64_t)q.E, (uint64_t)q.S, (uint64_t)q.B};
       const uint64_t strides[2] = {(uint64_t)q.E * 2, (uint64_t)q.S * q.E * 2};
       const uint32_t box[3] = {(uint32_t)kD, (uint32_t)kKeyBlock, 1};
-      if (!encode_tmap_bf16(&m, inputs[i], 3, dims, strides, box, 128, err)) return AGO_ERR_CUDA;
-      if (host->maps.size() > 4096) host->maps.clear();
-      it = host->maps.emplace(inputs[i], m).first;
+      if (!encode_tmap_bf16(&m, base, 3, dims, strides, box, 128, err)) return AGO_ERR_CUDA;
+      if (host->maps.size() > 4096) {     // pointers already fetched stay valid: unordered_map keeps its nodes until erased
+        host->maps.clear();
+        i = -1;
+        continue;
+      }
+      it = host->maps.emplace(base, m).first;
     }
     maps[i] = &it->second;
   }
@@ -481,7 +494,7 @@ ago_status_t attention_run(const Plan& plan, FusedState* st, const void* const* 
   }
   dim3 grid((unsigned)std::min(q.total, kSMs));     // one persistent CTA per SM (the shared memory admits no second one)
   FusedLaunch launch(grid, kThreads, (size_t)host->smem_bytes, stream);
-  cudaError_t e = cudaLaunchKernelEx(&launch.config, attention_fused_kernel, *maps[0], *maps[1], *maps[2], q);
+  cudaError_t e = cudaLaunchKernelEx(&launch.config, attention_fused_kernel, *maps[0], *maps[1], *maps[2], *maps[3], q);
   if (e != cudaSuccess) { *err = std::string("fused attention launch: ") + cudaGetErrorString(e); return AGO_ERR_CUDA; }
   return AGO_OK;
 }
