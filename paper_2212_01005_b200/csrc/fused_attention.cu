@@ -10,20 +10,26 @@
 // consecutive runs to one persistent CTA per SM. K and V of the current (batch, head) stay in shared
 // memory while the CTA walks over its query tiles; when the run crosses into the next head, the new K
 // is fetched as soon as the last score product of the old head has completed and the new V as soon as
-// its last P V has, both behind the softmax of the tiles in flight. The keys are processed in two halves so that tensor
-// cores and CUDA cores overlap: while the softmax warps turn half 0 of the scores into
-// probabilities, the MMA warp already computes half 1 (and, later, the next tile's scores). The
-// running row maximum may grow between the halves; the partial output of half 0 is then rescaled
-// in tensor memory by exp(m0 - m1) before half 1 is accumulated -- the result is the exact softmax.
+// its last P V has, both behind the softmax of the tiles in flight.
+//
+// The keys are processed in two halves by two independent groups of 384 threads (3 per query row and half).
+// Each half is a softmax of its own -- its own row maximum, row sum and output accumulator P_h V_h in tensor
+// memory -- and the epilogue joins them: with m = max(m_0, m_1) and f_h = exp(m_h - m),
+// O = (f_0 O_0 + f_1 O_1) / (f_0 sum_0 + f_1 sum_1), the exact softmax over all keys. Nothing but the epilogue
+// orders the groups against each other, so they drift apart: while one group keeps the special-function
+// unit busy with its exponentials, the other waits for scores, reads tensor memory or exchanges maxima,
+// and the tensor core runs ahead on the next tile's scores.
 //
 //   P1  TMA: K, V [S x 64] once per head of the run, Q [128 x 64] per tile -> 128-byte-swizzled tiles
 //   P2  tcgen05.mma: S_h[128 x S/2] = Q K_h^T                            (TMEM, fp32, two buffers)
-//   P3/P4  768 threads (6 per query row): TMEM -> registers, row max (exchanged through shared
-//       memory), p = exp2((s - m) * scale * log2 e), bf16 -> shared memory (K-major operand), row sum
-//   P5  tcgen05.mma: O[128 x 64] (+)= P_h V_h       (V is the N-major B operand, as it lies in HBM)
-//   P6  TMEM -> registers, * 1 / rowsum, bf16 -> a swizzled tile in shared memory (the probability buffer of half 1, idle
-//       by then) -> one TMA store per tile (a row of one head is 128 bytes of a 2 E-byte output row: stores from
-//       the row-per-lane accumulator layout would touch 32 lines per instruction)
+//   P3/P4  per half 384 threads (3 per query row, <= 64 score columns each, read from tensor memory in chunks of 32:
+//       once for the row maximum, exchanged through shared memory, once more for
+//       p = exp2((s - m_h) * scale * log2 e) -> bf16 -> shared memory (K-major operand) and the row sum)
+//   P5  tcgen05.mma: O_h[128 x 64] = P_h V_h        (V is the N-major B operand, as it lies in HBM)
+//   P6  the group of half 1: TMEM -> registers, (f_0 O_0 + f_1 O_1) / sum, bf16 -> a swizzled tile in shared memory (the
+//       probability buffer of half 1, idle by then) -> one TMA store per tile, issued by a thread of its own (a row
+//       of one head is 128 bytes of a 2 E-byte output row: stores from the row-per-lane accumulator layout would
+//       touch 32 lines per instruction)
 #include <cuda.h>
 #include <cuda_bf16.h>
 
@@ -43,11 +49,12 @@ using namespace tc;
 constexpr int kD = 64;                 // head dimension (one 128-byte swizzle row)
 constexpr int kBlockM = 128;           // query rows per tile
 constexpr int kKeyBlock = 128;         // keys per TMA box
-constexpr int kParts = 6;              // threads per query row (each owns <= 32 score columns of a half)
-constexpr int kComputeThreads = kBlockM * kParts;
+constexpr int kSubParts = 3;           // threads per query row and half (each owns <= 64 score columns: two chunks of 32)
+constexpr int kGroupThreads = kBlockM * kSubParts;
+constexpr int kComputeThreads = 2 * kGroupThreads;
 constexpr int kThreads = kComputeThreads + 64;   // + TMA warp + MMA warp
 constexpr int kHalfCols = 192;         // tensor-memory columns reserved per score half
-constexpr uint32_t kOCol = 2 * kHalfCols;
+constexpr uint32_t kOCol = 2 * kHalfCols;   // O_0 at kOCol, O_1 at kOCol + kD
 constexpr int kSMs = 148;              // B200
 
 struct AttnParams {
@@ -59,7 +66,7 @@ struct AttnParams {
   int tiles;       // query tiles per head
   int total;       // items = B * heads * tiles
   int hw0, hw1;    // keys in half 0 / half 1 (multiples of 16, hw0 >= hw1 > 0)
-  int pw0, pw1;    // columns per thread part in each half (multiples of 16)
+  int pw0, pw1;    // columns per thread in each half (multiples of 32, <= 64)
   float scale_log2e;
   int off_q, off_k, off_v, off_p, off_red, off_bar;
   int p_half_bytes;
@@ -82,9 +89,8 @@ attention_fused_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
   uint8_t* sK = smem + p.off_k;
   uint8_t* sV = smem + p.off_v;
   uint8_t* sP = smem + p.off_p;                                // two halves of p_half_bytes
-  float* sMax0 = reinterpret_cast<float*>(smem + p.off_red);    // [kParts][128]
-  float* sMax1 = sMax0 + kParts * kBlockM;
-  float* sSum = sMax1 + kParts * kBlockM;
+  float* sMax = reinterpret_cast<float*>(smem + p.off_red);     // [half][tile parity][kSubParts][128]: partial row maxima
+  float* sSum = sMax + 2 * 2 * kSubParts * kBlockM;             // the same for the partial row sums
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + p.off_bar);
   uint64_t* bar_k = bars + 0;
   uint64_t* bar_v = bars + 1;
@@ -94,12 +100,13 @@ attention_fused_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
   uint64_t* bar_p = bars + 6;       // [2] probabilities of the half written, score half drained
   uint64_t* bar_pfree = bars + 8;   // [2] P V of the half has read the probabilities
   uint64_t* bar_o0 = bars + 10;     // P V of half 0 complete
-  uint64_t* bar_corr = bars + 11;   // output rescaled for half 1
+  uint64_t* bar_stage = bars + 11;  // output tile staged in shared memory
   uint64_t* bar_o1 = bars + 12;     // P V of half 1 complete
   uint64_t* bar_ofree = bars + 13;  // epilogue has read the output accumulators
   uint64_t* bar_vfree = bars + 14;  // the last P V of a head has read V
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 15);
-  volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(bars + 16);
+  uint64_t* bar_stfree = bars + 15; // the output store has read the staged tile
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 16);
+  volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(bars + 17);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   // This CTA's run of items [g0, g0 + n); item g = ((b * heads + h) * tiles + t).
@@ -112,7 +119,7 @@ attention_fused_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
 
   if (tid == kComputeThreads) {
     *abort_flag = 0u;
-    for (int i = 0; i < 15; ++i) mbar_init(bars + i, 1);
+    for (int i = 0; i < 16; ++i) mbar_init(bars + i, 1);
     fence_mbar_init();
     fence_proxy_async_smem();
     tma_prefetch_desc(&tmap_q);
@@ -170,20 +177,26 @@ attention_fused_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
       const uint32_t idesc_s[2] = {make_idesc_bf16(128, (uint32_t)p.hw0), make_idesc_bf16(128, (uint32_t)p.hw1)};
       const int hw[2] = {p.hw0, p.hw1};
 
+      // Descriptors as (low, high) words: the start address lives in the low word, so every operand of the unrolled
+      // issue loops is one 32-bit add away from its base.
+      const uint32_t q_lo = (uint32_t)qdesc, q_hi = (uint32_t)(qdesc >> 32), k_lo = (uint32_t)kdesc, k_hi = (uint32_t)(kdesc >> 32);
+      const uint32_t p_lo = (uint32_t)pdesc, p_hi = (uint32_t)(pdesc >> 32), v_lo = (uint32_t)vdesc, v_hi = (uint32_t)(vdesc >> 32);
       auto issue_scores = [&](int half) {
-        const uint64_t bd = kdesc + (uint64_t)((uint32_t)(half * p.hw0 * kD * 2) >> 4);
+        const uint32_t b0 = k_lo + ((uint32_t)(half * p.hw0 * kD * 2) >> 4);
 #pragma unroll
         for (int ks = 0; ks < kD / 16; ++ks)
-          umma_bf16(tmem_base + half * kHalfCols, qdesc + 2u * ks, bd + 2u * ks, idesc_s[half], ks > 0);
+          umma_bf16_lohi(tmem_base + half * kHalfCols, q_lo + 2u * ks, q_hi, b0 + 2u * ks, k_hi, idesc_s[half], ks > 0);
         umma_commit(bar_s + half);
       };
       auto issue_pv = [&](int half) {
-        const uint64_t ad0 = pdesc + (uint64_t)((uint32_t)(half * p.p_half_bytes) >> 4);
-        const uint64_t bd0 = vdesc + (uint64_t)((uint32_t)(half * p.hw0 * kD * 2) >> 4);
+        const uint32_t a0 = p_lo + ((uint32_t)(half * p.p_half_bytes) >> 4);
+        const uint32_t b0 = v_lo + ((uint32_t)(half * p.hw0 * kD * 2) >> 4);
         const int ksteps = hw[half] / 16;
-        for (int ks = 0; ks < ksteps; ++ks)
-          umma_bf16(tmem_base + kOCol, ad0 + (uint64_t)(((ks >> 2) * kBlockM * 128 + (ks & 3) * 32) >> 4),
-                    bd0 + (uint64_t)((ks * 16 * kD * 2) >> 4), idesc_o, (half | ks) != 0);
+#pragma unroll
+        for (int ks = 0; ks < kHalfCols / 16; ++ks)
+          if (ks < ksteps)
+            umma_bf16_lohi(tmem_base + kOCol + half * kD, a0 + (uint32_t)(((ks >> 2) * kBlockM * 128 + (ks & 3) * 32) >> 4), p_hi,
+                           b0 + (uint32_t)((ks * 16 * kD * 2) >> 4), v_hi, idesc_o, ks != 0);
       };
 
       mbar_wait(bar_k, 0, abort_flag, p.status, 0x202);
@@ -200,23 +213,22 @@ attention_fused_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
         const bool last_of_head = t + 1 == p.tiles;   // the next item of the run, if any, belongs to the next head
         // ---- half 0 ----
         mbar_wait(bar_p + 0, ph, abort_flag, p.status, 0x204);
+        if (i + 1 < n) {
+          mbar_wait(bar_q, ph ^ 1u, abort_flag, p.status, 0x207);
+          if (last_of_head) mbar_wait(bar_k, head_ph ^ 1u, abort_flag, p.status, 0x202);
+          tcgen05_fence_after_sync();
+          issue_scores(0);                       // next tile's half 0 into the buffer just drained: its group is waiting for it
+        }
         if (first_of_head) mbar_wait(bar_v, head_ph, abort_flag, p.status, 0x205);
         if (i > 0) mbar_wait(bar_ofree, ph ^ 1u, abort_flag, p.status, 0x206);
         tcgen05_fence_after_sync();
         issue_pv(0);
         umma_commit(bar_o0);
         umma_commit(bar_pfree + 0);
-        if (i + 1 < n) {
-          mbar_wait(bar_q, ph ^ 1u, abort_flag, p.status, 0x207);
-          if (last_of_head) mbar_wait(bar_k, head_ph ^ 1u, abort_flag, p.status, 0x202);
-          tcgen05_fence_after_sync();
-          issue_scores(0);                       // next tile's half 0 into the buffer just drained
-        }
         // ---- half 1 ----
         mbar_wait(bar_p + 1, ph, abort_flag, p.status, 0x208);
-        mbar_wait(bar_corr, ph, abort_flag, p.status, 0x209);
         tcgen05_fence_after_sync();
-        issue_pv(1);
+        issue_pv(1);                             // first: the epilogue of this tile waits for it
         umma_commit(bar_o1);
         umma_commit(bar_pfree + 1);
         if (last_of_head) umma_commit(bar_vfree);
@@ -230,29 +242,34 @@ attention_fused_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
     }
     __syncwarp();
   } else {
-    // ============================ softmax / rescale / epilogue warps ============================
+    // ============================ softmax / epilogue warps ============================
     const int row = (warp & 3) * 32 + lane;     // TMEM lane = query row of the tile
-    const int part = warp >> 2;                 // which slice of a half's keys (and, for parts 0..3, of the output columns)
+    const int part = warp >> 2;
+    const int grp = part >= kSubParts ? 1 : 0;  // the half of the keys this thread's group owns
+    const int sub = part - grp * kSubParts;     // which slice of the half
     const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
     const float c = p.scale_log2e;
-    const int hw[2] = {p.hw0, p.hw1};
-    const int pw[2] = {p.pw0, p.pw1};
+    const int hw = grp ? p.hw1 : p.hw0;
+    const int pw = grp ? p.pw1 : p.pw0;
+    const int nch = pw >> 5;                    // chunks of 32 columns per thread
+    const int key_base = grp * p.hw0;
+    const uint32_t s_addr = tmem_base + lane_base + grp * kHalfCols;
+    uint8_t* pbase = sP + grp * p.p_half_bytes;
+    const uint32_t bar_id = 1u + (uint32_t)grp;
+    const bool leader = sub == 0 && row == 0;
+    float* gMax = sMax + grp * (2 * kSubParts * kBlockM);
+    float* gSum = sSum + grp * (2 * kSubParts * kBlockM);
 
-    // One half of one tile for this thread: its (at most 32) score columns stay in registers between the
-    // maximum and the exponentials, so tensor memory is read once.
-    //   phase A: load + local maximum -> exchange;  phase B: p = exp2((s - m) c) -> bf16 -> shared memory, partial sum
     uint32_t sv[32];
-    int ncols = 0, col0 = 0;
-    bool fast = false;   // all 32 columns present and none of them padding: straight-line code, no predicates
-    auto load_half_and_max = [&](int half) -> float {
-      col0 = part * pw[half];
-      ncols = max(0, min(hw[half], col0 + pw[half]) - col0);    // 0, 16 or 32
-      const int key0 = half * p.hw0 + col0;
-      fast = ncols == 32 && key0 + 32 <= p.S;
+    // One chunk of (at most) 32 score columns of this thread's row: col0 within the half, ncols in {0, 16, 32};
+    // fast = all 32 present and none of them padding: straight-line code, no predicates.
+    auto load_chunk = [&](int col0, int ncols) {
+      if (ncols > 16) tmem_ld_x32(s_addr + col0, sv); else tmem_ld_x16(s_addr + col0, sv);
+      tmem_ld_wait();
+    };
+    auto chunk_max = [&](int col0, int ncols, bool fast) -> float {
       float m = -INFINITY;
       if (fast) {
-        tmem_ld_x32(tmem_base + lane_base + half * kHalfCols + col0, sv);
-        tmem_ld_wait();
         float m4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
         for (int j = 0; j < 32; j += 4) {
@@ -262,18 +279,15 @@ attention_fused_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
           m4[3] = fmaxf(m4[3], __uint_as_float(sv[j + 3]));
         }
         m = fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3]));
-      } else if (ncols > 0) {
-        const uint32_t addr = tmem_base + lane_base + half * kHalfCols + col0;
-        if (ncols > 16) tmem_ld_x32(addr, sv); else tmem_ld_x16(addr, sv);
-        tmem_ld_wait();
+      } else {
+        const int key0 = key_base + col0;
 #pragma unroll
         for (int j = 0; j < 32; ++j) if (j < ncols && key0 + j < p.S) m = fmaxf(m, __uint_as_float(sv[j]));
       }
       return m;
     };
-    auto exp_half_to_smem = [&](int half, float mc) -> float {
+    auto chunk_exp = [&](int col0, int ncols, bool fast, float mc) -> float {
       float sum = 0.0f;
-      uint8_t* pbase = sP + half * p.p_half_bytes;
       if (fast) {
         // 32 columns = four 16-byte chunks of this row inside one 64-key block (col0 is a multiple of 32)
         uint8_t* rowp = pbase + (col0 >> 6) * (kBlockM * 128) + row * 128;
@@ -292,8 +306,8 @@ attention_fused_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
           *reinterpret_cast<uint4*>(rowp + (((ch0 + g) ^ sw) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
         }
         sum = (s4[0] + s4[1]) + (s4[2] + s4[3]);
-      } else if (ncols > 0) {
-        const int key0 = half * p.hw0 + col0;
+      } else {
+        const int key0 = key_base + col0;
 #pragma unroll
         for (int g = 0; g < 4; ++g) {            // 8 columns = one 16-byte chunk of a probability row
           if (g * 8 < ncols) {
@@ -316,97 +330,96 @@ attention_fused_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
       }
       return sum;
     };
-    auto reduce_parts = [&](const float* a, bool is_max) -> float {
-      float r = a[row];
-#pragma unroll
-      for (int q = 1; q < kParts; ++q) r = is_max ? fmaxf(r, a[q * kBlockM + row]) : r + a[q * kBlockM + row];
-      return r;
+    auto reduce3 = [&](const float* a, bool is_max) -> float {
+      const float x = a[row], y = a[kBlockM + row], z = a[2 * kBlockM + row];
+      return is_max ? fmaxf(x, fmaxf(y, z)) : x + y + z;
     };
 
-    float m0 = 0.0f, sum0 = 0.0f;
-    auto do_half0 = [&](int t) {              // t: position of the item in this CTA's run
-      const uint32_t ph = (uint32_t)t & 1u;
-      mbar_wait(bar_s + 0, ph, abort_flag, p.status, 0x210);
-      tcgen05_fence_after_sync();
-      sMax0[part * kBlockM + row] = load_half_and_max(0);
-      named_barrier_sync(1, kComputeThreads);
-      m0 = reduce_parts(sMax0, true);
-      if (t > 0) mbar_wait(bar_pfree + 0, ph ^ 1u, abort_flag, p.status, 0x211);
-      sum0 = exp_half_to_smem(0, m0 * c);
-      fence_proxy_async_smem();
-      tcgen05_fence_before_sync();
-      named_barrier_sync(1, kComputeThreads);
-      if (tid == 0) mbar_arrive(bar_p + 0);
-    };
-
-    do_half0(0);
     int tq = t0, h = h0, b = b0;                // the item's query tile, head and batch
-    for (int t = 0; t < n; ++t) {
+    for (int t = 0; t < n; ++t) {               // t: position of the item in this CTA's run
       const uint32_t ph = (uint32_t)t & 1u;
-      // ---------------- half 1 ----------------
-      mbar_wait(bar_s + 1, ph, abort_flag, p.status, 0x212);
+      float* myMax = gMax + ph * (kSubParts * kBlockM);
+      float* mySum = gSum + ph * (kSubParts * kBlockM);
+      // ---------------- pass 1: row maximum of this half ----------------
+      mbar_wait(bar_s + grp, ph, abort_flag, p.status, 0x210);
       tcgen05_fence_after_sync();
-      sMax1[part * kBlockM + row] = load_half_and_max(1);
-      if (tid == 0) bulk_wait_group_read_all();      // the previous tile's output store has read its staging tile (the half-1 buffer)
-      named_barrier_sync(1, kComputeThreads);
-      const float m1 = fmaxf(m0, reduce_parts(sMax1, true));
-      const float alpha = ex2_approx((m0 - m1) * c);     // rescales everything accumulated under the old maximum
-      if (t > 0) mbar_wait(bar_pfree + 1, ph ^ 1u, abort_flag, p.status, 0x213);
-      const float sum1 = exp_half_to_smem(1, m1 * c);
-      sSum[part * kBlockM + row] = sum0 * alpha + sum1;
+      float m = -INFINITY;
+      for (int ch = 0; ch < nch; ++ch) {
+        const int col0 = sub * pw + ch * 32;
+        const int ncols = max(0, min(hw, col0 + 32) - col0);
+        if (ncols > 0) {
+          load_chunk(col0, ncols);
+          m = fmaxf(m, chunk_max(col0, ncols, ncols == 32 && key_base + col0 + 32 <= p.S));
+        }
+      }
+      myMax[sub * kBlockM + row] = m;
+      if (leader && t > 0) {
+        mbar_wait(bar_pfree + grp, ph ^ 1u, abort_flag, p.status, 0x211);       // P V of the previous tile has read this half's probabilities
+        if (grp == 1) bulk_wait_group_read_all();       // and this thread's output store has read its staged tile (same buffer)
+      }
+      named_barrier_sync(bar_id, kGroupThreads);
+      const float mh = reduce3(myMax, true);
+      // ---------------- pass 2: probabilities and row sum ----------------
+      float sum = 0.0f;
+      for (int ch = 0; ch < nch; ++ch) {
+        const int col0 = sub * pw + ch * 32;
+        const int ncols = max(0, min(hw, col0 + 32) - col0);
+        if (ncols > 0) {
+          load_chunk(col0, ncols);
+          sum += chunk_exp(col0, ncols, ncols == 32 && key_base + col0 + 32 <= p.S, mh * c);
+        }
+      }
+      mySum[sub * kBlockM + row] = sum;
       fence_proxy_async_smem();
       tcgen05_fence_before_sync();
-      named_barrier_sync(1, kComputeThreads);
-      if (tid == 0) mbar_arrive(bar_p + 1);
-      const float inv = 1.0f / reduce_parts(sSum, false);
+      named_barrier_sync(bar_id, kGroupThreads);
+      if (leader) mbar_arrive(bar_p + grp);      // probabilities written, score half drained
 
-      // ---------------- rescale the half-0 output: O *= alpha (parts 0..3: 16 of the 64 columns each) ----------------
-      mbar_wait(bar_o0, ph, abort_flag, p.status, 0x214);
-      tcgen05_fence_after_sync();
-      if (part < 4) {
-        uint32_t o[16];
-        const uint32_t addr = tmem_base + lane_base + kOCol + part * 16;
-        tmem_ld_x16(addr, o);
-        tmem_ld_wait();
+      if (grp == 1) {
+        // ---------------- epilogue of the tile: join the halves, normalise, stage, store ----------------
+        mbar_wait(bar_o0, ph, abort_flag, p.status, 0x214);
+        mbar_wait(bar_o1, ph, abort_flag, p.status, 0x215);
+        tcgen05_fence_after_sync();
+        if (sub < 2) {                           // 32 of the 64 output columns each
+          // Half 0's maxima and sums of this tile: written before that group's barriers, which precede its arrival on
+          // bar_p[0], the P V product and hence bar_o0.
+          const float m0 = reduce3(sMax + ph * (kSubParts * kBlockM), true);
+          const float s0 = reduce3(sSum + ph * (kSubParts * kBlockM), false);
+          const float s1 = reduce3(mySum, false);
+          const float mm = fmaxf(m0, mh);
+          float f0 = ex2_approx((m0 - mm) * c), f1 = ex2_approx((mh - mm) * c);
+          const float inv = 1.0f / (f0 * s0 + f1 * s1);
+          f0 *= inv; f1 *= inv;
+          uint8_t* stage = pbase;                // P V of half 1 has completed: its probabilities are dead
 #pragma unroll
-        for (int j = 0; j < 16; ++j) o[j] = __float_as_uint(__uint_as_float(o[j]) * alpha);
-        tmem_st_x16(addr, o);
-        tmem_st_wait();
-      }
-      tcgen05_fence_before_sync();
-      named_barrier_sync(1, kComputeThreads);
-      if (tid == 0) mbar_arrive(bar_corr);
-
-      // While the tensor core finishes P V of this tile, start on the next tile's first half.
-      if (t + 1 < n) do_half0(t + 1);
-
-      // ---------------- epilogue of tile t: O / rowsum -> bf16 -> global ----------------
-      mbar_wait(bar_o1, ph, abort_flag, p.status, 0x215);
-      tcgen05_fence_after_sync();
-      if (part < 4) {
-        uint32_t o[16];
-        tmem_ld_x16(tmem_base + lane_base + kOCol + part * 16, o);
-        tmem_ld_wait();
-        uint8_t* stage = sP + p.p_half_bytes;      // P V of half 1 has completed: its probabilities are dead
+          for (int k = 0; k < 2; ++k) {
+            uint32_t oa[16], ob[16];
+            const uint32_t addr = tmem_base + lane_base + kOCol + sub * 32 + k * 16;
+            tmem_ld_x16(addr, oa);
+            tmem_ld_x16(addr + kD, ob);
+            tmem_ld_wait();
+            float o[16];
 #pragma unroll
-        for (int j = 0; j < 2; ++j)
-          *reinterpret_cast<uint4*>(stage + swz_offset(row, (uint32_t)(part * 2 + j), 128)) =
-              make_uint4(pack_bf16x2(__uint_as_float(o[8 * j]) * inv, __uint_as_float(o[8 * j + 1]) * inv),
-                         pack_bf16x2(__uint_as_float(o[8 * j + 2]) * inv, __uint_as_float(o[8 * j + 3]) * inv),
-                         pack_bf16x2(__uint_as_float(o[8 * j + 4]) * inv, __uint_as_float(o[8 * j + 5]) * inv),
-                         pack_bf16x2(__uint_as_float(o[8 * j + 6]) * inv, __uint_as_float(o[8 * j + 7]) * inv));
+            for (int j = 0; j < 16; ++j) o[j] = fmaf(__uint_as_float(oa[j]), f0, __uint_as_float(ob[j]) * f1);
+#pragma unroll
+            for (int j = 0; j < 2; ++j)
+              *reinterpret_cast<uint4*>(stage + swz_offset(row, (uint32_t)(sub * 4 + k * 2 + j), 128)) =
+                  make_uint4(pack_bf16x2(o[8 * j], o[8 * j + 1]), pack_bf16x2(o[8 * j + 2], o[8 * j + 3]),
+                             pack_bf16x2(o[8 * j + 4], o[8 * j + 5]), pack_bf16x2(o[8 * j + 6], o[8 * j + 7]));
+          }
+        }
+        fence_proxy_async_smem();
+        tcgen05_fence_before_sync();
+        named_barrier_sync(bar_id, kGroupThreads);
+        if (leader) {
+          mbar_arrive(bar_ofree);
+          tma_store_3d(&tmap_o, pbase, h * kD, tq * kBlockM, b);   // rows past S are clipped
+          bulk_commit_group();
+        }
+        if (++tq == p.tiles) { tq = 0; if (++h == p.heads) { h = 0; ++b; } }
       }
-      fence_proxy_async_smem();
-      tcgen05_fence_before_sync();
-      named_barrier_sync(1, kComputeThreads);
-      if (tid == 0) {
-        mbar_arrive(bar_ofree);
-        tma_store_3d(&tmap_o, sP + p.p_half_bytes, h * kD, tq * kBlockM, b);   // rows past S are clipped
-        bulk_commit_group();
-      }
-      if (++tq == p.tiles) { tq = 0; if (++h == p.heads) { h = 0; ++b; } }
     }
-    if (tid == 0) bulk_wait_group_all();
+    if (leader && grp == 1) bulk_wait_group_all();
   }
   tcgen05_fence_before_sync();
   __syncthreads();
@@ -441,8 +454,8 @@ ago_status_t attention_plan(Plan* plan, FusedState* st, std::string* err) {
   q.total = q.B * q.heads * q.tiles;
   q.hw0 = round16((q.Spad + 1) / 2);
   q.hw1 = q.Spad - q.hw0;
-  q.pw0 = round16((q.hw0 + kParts - 1) / kParts);
-  q.pw1 = round16((q.hw1 + kParts - 1) / kParts);
+  q.pw0 = ((q.hw0 + kSubParts - 1) / kSubParts + 31) / 32 * 32;
+  q.pw1 = ((q.hw1 + kSubParts - 1) / kSubParts + 31) / 32 * 32;
   q.scale_log2e = plan->ops[1].op.f * 1.4426950408889634f;
   int off = 0;
   auto take = [&](int bytes) { int o = off; off = (off + bytes + 1023) / 1024 * 1024; return o; };
@@ -451,7 +464,7 @@ ago_status_t attention_plan(Plan* plan, FusedState* st, std::string* err) {
   q.off_v = take(q.nkb * kKeyBlock * kD * 2);
   q.p_half_bytes = ((q.hw0 + 63) / 64) * kBlockM * 128;
   q.off_p = take(2 * q.p_half_bytes);
-  q.off_red = take(3 * kParts * kBlockM * 4);
+  q.off_red = take(2 * 2 * 2 * kSubParts * kBlockM * 4);
   q.off_bar = take(256);
   host->smem_bytes = off + 1024;
   if (host->smem_bytes > 227 * 1024) return bad("shared memory budget exceeded");
