@@ -27,9 +27,12 @@
 //       p = exp2((s - m_h) * scale * log2 e) -> bf16 -> shared memory (K-major operand) and the row sum)
 //   P5  tcgen05.mma: O_h[128 x 64] = P_h V_h        (V is the N-major B operand, as it lies in HBM)
 //   P6  the group of half 1: TMEM -> registers, (f_0 O_0 + f_1 O_1) / sum, bf16 -> a swizzled tile in shared memory (the
-//       probability buffer of half 1, idle by then) -> one TMA store per tile, issued by a thread of its own (a row
-//       of one head is 128 bytes of a 2 E-byte output row: stores from the row-per-lane accumulator layout would
-//       touch 32 lines per instruction)
+//       probability buffer of half 1, idle by then) -> one TMA store per tile (a row of one head is 128 bytes of a
+//       2 E-byte output row: stores from the row-per-lane accumulator layout would touch 32 lines per instruction)
+//
+// Issue order of the MMA thread: when half 0's probabilities arrive, the next tile's half-0 scores go first (that
+// group has nothing else to do) and P_0 V second; when half 1's arrive, P_1 V goes first (the epilogue waits for
+// it) and the next half-1 scores second.
 #include <cuda.h>
 #include <cuda_bf16.h>
 
