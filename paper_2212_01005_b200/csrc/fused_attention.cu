@@ -339,6 +339,42 @@ attention_fused_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
     };
 
     int tq = t0, h = h0, b = b0;                // the item's query tile, head and batch
+    // Threads whose 64 columns are all present and real keys read them in four pieces of 16 through two register
+    // buffers: the load of the next piece is in flight while the current one is consumed.
+    const bool piped = pw == 64 && sub * pw + 64 <= hw && key_base + sub * pw + 64 <= p.S;
+    const uint32_t c_addr = s_addr + (uint32_t)(sub * pw);
+    auto max16 = [&](const uint32_t (&v)[16]) -> float {
+      float m4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll
+      for (int j = 0; j < 16; j += 4) {
+        m4[0] = fmaxf(m4[0], __uint_as_float(v[j]));
+        m4[1] = fmaxf(m4[1], __uint_as_float(v[j + 1]));
+        m4[2] = fmaxf(m4[2], __uint_as_float(v[j + 2]));
+        m4[3] = fmaxf(m4[3], __uint_as_float(v[j + 3]));
+      }
+      return fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3]));
+    };
+    // 16 columns (piece q of the thread's 64) -> two 16-byte chunks of the probability row; returns their sum
+    auto exp16 = [&](const uint32_t (&v)[16], int q, float mc) -> float {
+      const int col = sub * 64 + q * 16;
+      uint8_t* rowp = pbase + (col >> 6) * (kBlockM * 128) + row * 128;
+      const uint32_t ch0 = (uint32_t)(col & 63) >> 3, sw = (uint32_t)row & 7u;
+      float s2[2] = {0.f, 0.f};
+#pragma unroll
+      for (int g = 0; g < 2; ++g) {
+        uint32_t w[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          const float e0 = ex2_approx(fmaf(__uint_as_float(v[g * 8 + 2 * j]), c, -mc));
+          const float e1 = ex2_approx(fmaf(__uint_as_float(v[g * 8 + 2 * j + 1]), c, -mc));
+          s2[j & 1] += e0 + e1;
+          w[j] = pack_bf16x2(e0, e1);
+        }
+        *reinterpret_cast<uint4*>(rowp + (((ch0 + g) ^ sw) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
+      }
+      return s2[0] + s2[1];
+    };
+
     for (int t = 0; t < n; ++t) {               // t: position of the item in this CTA's run
       const uint32_t ph = (uint32_t)t & 1u;
       float* myMax = gMax + ph * (kSubParts * kBlockM);
@@ -347,12 +383,29 @@ attention_fused_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
       mbar_wait(bar_s + grp, ph, abort_flag, p.status, 0x210);
       tcgen05_fence_after_sync();
       float m = -INFINITY;
-      for (int ch = 0; ch < nch; ++ch) {
-        const int col0 = sub * pw + ch * 32;
-        const int ncols = max(0, min(hw, col0 + 32) - col0);
-        if (ncols > 0) {
-          load_chunk(col0, ncols);
-          m = fmaxf(m, chunk_max(col0, ncols, ncols == 32 && key_base + col0 + 32 <= p.S));
+      if (piped) {
+        uint32_t (&va)[16] = reinterpret_cast<uint32_t (&)[16]>(sv[0]);
+        uint32_t (&vb)[16] = reinterpret_cast<uint32_t (&)[16]>(sv[16]);
+        tmem_ld_x16(c_addr, va);
+        tmem_ld_wait_on(va);
+        tmem_ld_x16(c_addr + 16, vb);
+        m = max16(va);
+        tmem_ld_wait_on(vb);
+        tmem_ld_x16(c_addr + 32, va);
+        m = fmaxf(m, max16(vb));
+        tmem_ld_wait_on(va);
+        tmem_ld_x16(c_addr + 48, vb);
+        m = fmaxf(m, max16(va));
+        tmem_ld_wait_on(vb);
+        m = fmaxf(m, max16(vb));
+      } else {
+        for (int ch = 0; ch < nch; ++ch) {
+          const int col0 = sub * pw + ch * 32;
+          const int ncols = max(0, min(hw, col0 + 32) - col0);
+          if (ncols > 0) {
+            load_chunk(col0, ncols);
+            m = fmaxf(m, chunk_max(col0, ncols, ncols == 32 && key_base + col0 + 32 <= p.S));
+          }
         }
       }
       myMax[sub * kBlockM + row] = m;
@@ -364,12 +417,30 @@ attention_fused_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
       const float mh = reduce3(myMax, true);
       // ---------------- pass 2: probabilities and row sum ----------------
       float sum = 0.0f;
-      for (int ch = 0; ch < nch; ++ch) {
-        const int col0 = sub * pw + ch * 32;
-        const int ncols = max(0, min(hw, col0 + 32) - col0);
-        if (ncols > 0) {
-          load_chunk(col0, ncols);
-          sum += chunk_exp(col0, ncols, ncols == 32 && key_base + col0 + 32 <= p.S, mh * c);
+      if (piped) {
+        const float mc = mh * c;
+        uint32_t (&va)[16] = reinterpret_cast<uint32_t (&)[16]>(sv[0]);
+        uint32_t (&vb)[16] = reinterpret_cast<uint32_t (&)[16]>(sv[16]);
+        tmem_ld_x16(c_addr, va);
+        tmem_ld_wait_on(va);
+        tmem_ld_x16(c_addr + 16, vb);
+        sum = exp16(va, 0, mc);
+        tmem_ld_wait_on(vb);
+        tmem_ld_x16(c_addr + 32, va);
+        sum += exp16(vb, 1, mc);
+        tmem_ld_wait_on(va);
+        tmem_ld_x16(c_addr + 48, vb);
+        sum += exp16(va, 2, mc);
+        tmem_ld_wait_on(vb);
+        sum += exp16(vb, 3, mc);
+      } else {
+        for (int ch = 0; ch < nch; ++ch) {
+          const int col0 = sub * pw + ch * 32;
+          const int ncols = max(0, min(hw, col0 + 32) - col0);
+          if (ncols > 0) {
+            load_chunk(col0, ncols);
+            sum += chunk_exp(col0, ncols, ncols == 32 && key_base + col0 + 32 <= p.S, mh * c);
+          }
         }
       }
       mySum[sub * kBlockM + row] = sum;
