@@ -338,7 +338,6 @@ attention_fused_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
       return is_max ? fmaxf(x, fmaxf(y, z)) : x + y + z;
     };
 
-    int tq = t0, h = h0, b = b0;                // the item's query tile, head and batch
     // Threads whose 64 columns are all present and real keys read them in four pieces of 16 through two register
     // buffers: the load of the next piece is in flight while the current one is consumed.
     const bool piped = pw == 64 && sub * pw + 64 <= hw && key_base + sub * pw + 64 <= p.S;
@@ -487,10 +486,10 @@ attention_fused_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
         named_barrier_sync(bar_id, kGroupThreads);
         if (leader) {
           mbar_arrive(bar_ofree);
-          tma_store_3d(&tmap_o, pbase, h * kD, tq * kBlockM, b);   // rows past S are clipped
+          const int u = (g0 + t) / p.tiles, tq = g0 + t - u * p.tiles, b = u / p.heads;
+          tma_store_3d(&tmap_o, pbase, (u - b * p.heads) * kD, tq * kBlockM, b);   // rows past S are clipped
           bulk_commit_group();
         }
-        if (++tq == p.tiles) { tq = 0; if (++h == p.heads) { h = 0; ++b; } }
       }
     }
     if (leader && grp == 1) bulk_wait_group_all();
