@@ -39,16 +39,16 @@ NOMINAL_PEAKS = {"hbm_gbs": 8000.0, "bf16_tflops": 2250.0}     # data-sheet figu
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu
 # captures summarised under profiles/ (None until a capture exists for that workload and mode).
 NCU_TRAFFIC_BYTES = {
-    ("mbv2_56", "fused"): 4908288 + 0,            # profiles/mbv2_fused_kernel__mbv2_56.txt (output still dirty in L2)
-    ("attn_384", "fused"): 56695296 + 809984,     # profiles/attention_fused_kernel__attn_384.txt
-    ("resnet_56", "fused"): 13347328 + 2560,      # profiles/conv3x3_pair_kernel__resnet_56.txt
-    ("ffn_12288", "fused"): 28403456 + 0,         # profiles/ffn_cluster_kernel__ffn_12288.txt (output still dirty in L2)
+    ("mbv2_56", "fused"): 4906752 + 0,            # profiles/mbv2_fused_kernel__mbv2_56.txt (output still dirty in L2)
+    ("attn_384", "fused"): 56902400 + 2771456,    # profiles/attention_fused_kernel__attn_384.txt
+    ("resnet_56", "fused"): 13343744 + 3328,      # profiles/conv3x3_pair_kernel__resnet_56.txt
+    ("ffn_12288", "fused"): 28403712 + 0,         # profiles/ffn_cluster_kernel__ffn_12288.txt (output still dirty in L2)
     ("ffn_512", "fused"): 11877632 + 0,           # profiles/ffn_fused_kernel__ffn_512.txt
-    ("pw_dw_56", "fused"): 4894976 + 1024,        # profiles/mbv2_fused_kernel__pw_dw_56.txt
-    ("dw_pw_56", "fused"): 28970496 + 256,        # profiles/mbv2_fused_kernel__dw_pw_56.txt
-    ("dw_dw_56", "fused"): 28977152 + 1248512,    # profiles/dwdw_fused_kernel__dw_dw_56.txt
-    ("pw_pw_56", "fused"): 28948224 + 38400,      # profiles/pwpw_fused_kernel__pw_pw_56.txt
-    ("unfold_96", "fused"): 12670976 + 0,         # profiles/pwpw_fused_kernel__unfold_96.txt
+    ("pw_dw_56", "fused"): 4894464 + 1280,        # profiles/mbv2_fused_kernel__pw_dw_56.txt
+    ("dw_pw_56", "fused"): 28972288 + 256,        # profiles/mbv2_fused_kernel__dw_pw_56.txt
+    ("dw_dw_56", "fused"): 28976640 + 1269504,    # profiles/dwdw_fused_kernel__dw_dw_56.txt
+    ("pw_pw_56", "fused"): 28948992 + 112384,     # profiles/pwpw_fused_kernel__pw_pw_56.txt
+    ("unfold_96", "fused"): 12671232 + 0,         # profiles/pwpw_fused_kernel__unfold_96.txt
 }
 
 
