@@ -295,6 +295,32 @@ def test_fused_attention_dominant_key_and_uniform_rows(ago):
     np.testing.assert_allclose(gpu[0, :, :64], np.broadcast_to(v[0, 77, :64].astype(np.float64), (144, 64)), atol=2e-2)
 
 
+@pytest.mark.parametrize("S", [128, 200, 256, 384])
+def test_fused_attention_each_query_selects_its_keys(ago, S):
+    # Query row r scores 32 on the keys j with j = r + 5 (mod 64) and 0 elsewhere, so its probabilities are (almost) one-hot
+    # per 64-key block; V row k carries k + 1 in the column of its block. The output names, per query and key block, the V
+    # row that met the probability: a product that pairs a 16-key step of P with the wrong rows of V shows up as a wrong
+    # integer. Key counts of one, two and three 128-key loads, with and without a ragged last tile.
+    wl = WL.attention("attn_select", [52], 1, S, 1, 64)
+    q = np.zeros((1, S, 64), np.float32); k = np.zeros_like(q); v = np.zeros_like(q)
+    for r in range(S):
+        q[0, r, (r + 5) % 64] = 16.0
+        k[0, r, r % 64] = 16.0
+        v[0, r, r // 64] = (r % 64) + 1
+    data = {"inputs": [q, k, v], "weights": []}
+    gpu = run_gpu(ago, wl, data, "fused")
+    ref = O.run_chain(wl.ops, data["inputs"], data["weights"])
+    assert_close(gpu, ref, what=f"attn_select S={S}")
+    nb = (S + 63) // 64
+    for blk in range(nb):
+        rows = np.arange(64)
+        want = (rows + 5) % 64
+        present = blk * 64 + want < S                       # the last block of a ragged S lacks some keys
+        hits = np.array([sum(1 for b2 in range(nb) if b2 * 64 + w < S) for w in want])
+        got = gpu[0, :64, blk].astype(np.float64) * hits - 1
+        np.testing.assert_allclose(got[present], want[present], atol=0.26, err_msg=f"S={S} key block {blk}")
+
+
 def test_fused_ffn_512_full(ago):
     wl = WL.get("ffn_512")
     data = WL.generate(wl)

@@ -219,6 +219,18 @@ def test_attention_dominant_score_selects_that_v_row_per_head():
     np.testing.assert_allclose(o[0, :, D:], np.broadcast_to(v[0, 1, D:], (S, D)), atol=1e-12)
 
 
+def test_attention_each_query_selects_its_own_key():
+    # query r points at key (r + 2) mod S only (score 50 after the scale, 0 elsewhere): a permutation of the rows of V --
+    # a transposed score matrix or a softmax over the wrong axis gives the inverse permutation or a blend
+    B, S, Hh, D = 1, 8, 1, 8
+    q = np.zeros((B, S, D)); k = np.zeros((B, S, D)); v = rng.standard_normal((B, S, D))
+    for r in range(S):
+        q[0, r, (r + 2) % S] = 10.0
+        k[0, r, r] = 5.0 * np.sqrt(D)
+    o = _attn(q, k, v, Hh, D)
+    np.testing.assert_allclose(o[0], v[0, (np.arange(S) + 2) % S], atol=1e-12)
+
+
 def test_attention_matches_torch_float64_per_head():
     B, S, Hh, D = 2, 7, 3, 4
     q, k, v = (rng.standard_normal((B, S, Hh * D)) for _ in range(3))
