@@ -167,7 +167,8 @@ typedef enum {
  *   CONV1x1 BIAS [RELU6] CONV1x1 BIAS [RELU6]                        the pairs of Section VI-B
  *   GEMM BIAS GELU GEMM BIAS                                         feed-forward chain
  *   CONV3x3 BIAS RELU CONV3x3 BIAS ADD_INPUT 0 RELU                  residual 3x3 pair
- *   QKT SCALE SOFTMAX PV                                             attention
+ *   QKT SCALE SOFTMAX PV                                             attention (head_dim 64,
+ *                                   32..384 keys, scale > 0)
  *   GEMM RESHAPE ADD_INPUT RESHAPE TRANSPOSE RESHAPE GEMM RESHAPE    projection chain of a
  *                                   patch-unfolded attention block (rows permuted between the GEMMs)
  *   DW (any window) followed by simple operators only                depthwise mini-subgraph

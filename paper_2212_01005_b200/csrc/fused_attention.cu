@@ -520,6 +520,7 @@ ago_status_t attention_plan(Plan* plan, FusedState* st, std::string* err) {
   if (qk.op.p[2] != kD) return bad("head_dim must be 64");
   if (q.S > 2 * kHalfCols) return bad("more than 384 keys do not fit the score block in tensor memory");
   if (q.S < 32) return bad("fewer than 32 keys");
+  if (!(plan->ops[1].op.f > 0.0f)) return bad("the score scale must be positive (the row maximum is taken before scaling)");
   q.Spad = round16(q.S);
   q.nkb = (q.Spad + kKeyBlock - 1) / kKeyBlock;
   q.tiles = (q.S + kBlockM - 1) / kBlockM;

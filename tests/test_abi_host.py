@@ -103,6 +103,11 @@ def test_fused_planner_matches_every_chain_family_and_its_limits():
     # pointwise pair: more middle channels than tensor memory holds
     wl = WL.pw_pw("x", [1], 1, 8, 64, 512, 64)
     _expect_fail(wl.ops, wl.input_shapes, B.AGO_ERR_UNSUPPORTED, mode="fused", needle="256")
+    # the attention kernel takes the row maximum of the raw scores: a non-positive scale is left to the unfused modes
+    wl = WL.attention("x", [1], 1, 64, 1, 64)
+    ops = list(wl.ops); ops[1] = ("scale", dict(f=-0.125))
+    _expect_fail(ops, wl.input_shapes, B.AGO_ERR_UNSUPPORTED, mode="fused", needle="positive")
+    B.Subgraph(ops, wl.input_shapes, mode="per_mini_subgraph").close()
     # a transpose of other axes than the two middle ones is not a row permutation the chain kernel knows
     wl = WL.unfold_chain("x", [1], 2, 4, 8, 16, 32)
     ops = list(wl.ops); ops[4] = ("transpose", dict(a=0, b=1)); ops[5] = ("reshape", dict(shape=(64, 16))); ops[7] = ("reshape", dict(shape=(4, 2, 8, 32)))
