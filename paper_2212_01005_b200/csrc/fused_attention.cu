@@ -450,36 +450,60 @@ attention_fused_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
 
       if (grp == 1) {
         // ---------------- epilogue of the tile: join the halves, normalise, stage, store ----------------
+        // Half 0's product, maxima and sums are long complete (bar_o0 follows that group's barriers and its arrival on
+        // bar_p[0]): the weights and the f_0 O_0 terms are computed while the tensor core still works on P_1 V.
         mbar_wait(bar_o0, ph, abort_flag, p.status, 0x214);
-        mbar_wait(bar_o1, ph, abort_flag, p.status, 0x215);
         tcgen05_fence_after_sync();
+        uint32_t (&oa)[16] = reinterpret_cast<uint32_t (&)[16]>(sv[0]);
+        uint32_t (&ob)[16] = reinterpret_cast<uint32_t (&)[16]>(sv[16]);
+        const uint32_t o_addr = tmem_base + lane_base + kOCol + sub * 32;
+        float f1 = 0.0f;
         if (sub < 2) {                           // 32 of the 64 output columns each
-          // Half 0's maxima and sums of this tile: written before that group's barriers, which precede its arrival on
-          // bar_p[0], the P V product and hence bar_o0.
+          tmem_ld_x16(o_addr, oa);
+          tmem_ld_x16(o_addr + 16, ob);
           const float m0 = reduce3(sMax + ph * (kSubParts * kBlockM), true);
           const float s0 = reduce3(sSum + ph * (kSubParts * kBlockM), false);
           const float s1 = reduce3(mySum, false);
           const float mm = fmaxf(m0, mh);
-          float f0 = ex2_approx((m0 - mm) * c), f1 = ex2_approx((mh - mm) * c);
+          float f0 = ex2_approx((m0 - mm) * c);
+          f1 = ex2_approx((mh - mm) * c);
           const float inv = 1.0f / (f0 * s0 + f1 * s1);
           f0 *= inv; f1 *= inv;
-          uint8_t* stage = pbase;                // P V of half 1 has completed: its probabilities are dead
+          tmem_ld_wait_on(oa);
+          tmem_ld_wait_on(ob);
 #pragma unroll
-          for (int k = 0; k < 2; ++k) {
-            uint32_t oa[16], ob[16];
-            const uint32_t addr = tmem_base + lane_base + kOCol + sub * 32 + k * 16;
-            tmem_ld_x16(addr, oa);
-            tmem_ld_x16(addr + kD, ob);
-            tmem_ld_wait();
-            float o[16];
-#pragma unroll
-            for (int j = 0; j < 16; ++j) o[j] = fmaf(__uint_as_float(oa[j]), f0, __uint_as_float(ob[j]) * f1);
-#pragma unroll
-            for (int j = 0; j < 2; ++j)
-              *reinterpret_cast<uint4*>(stage + swz_offset(row, (uint32_t)(sub * 4 + k * 2 + j), 128)) =
-                  make_uint4(pack_bf16x2(o[8 * j], o[8 * j + 1]), pack_bf16x2(o[8 * j + 2], o[8 * j + 3]),
-                             pack_bf16x2(o[8 * j + 4], o[8 * j + 5]), pack_bf16x2(o[8 * j + 6], o[8 * j + 7]));
+          for (int j = 0; j < 16; ++j) {
+            oa[j] = __float_as_uint(__uint_as_float(oa[j]) * f0);
+            ob[j] = __float_as_uint(__uint_as_float(ob[j]) * f0);
           }
+        }
+        mbar_wait(bar_o1, ph, abort_flag, p.status, 0x215);
+        tcgen05_fence_after_sync();
+        if (sub < 2) {
+          uint8_t* stage = pbase;                // P V of half 1 has completed: its probabilities are dead
+          uint32_t oc[16];
+          tmem_ld_x16(o_addr + kD, oc);
+          tmem_ld_wait_on(oc);
+#pragma unroll
+          for (int j = 0; j < 16; ++j) oa[j] = __float_as_uint(fmaf(__uint_as_float(oc[j]), f1, __uint_as_float(oa[j])));
+          tmem_ld_x16(o_addr + kD + 16, oc);     // in flight while the first 16 columns are packed and staged
+#pragma unroll
+          for (int j = 0; j < 2; ++j)
+            *reinterpret_cast<uint4*>(stage + swz_offset(row, (uint32_t)(sub * 4 + j), 128)) =
+                make_uint4(pack_bf16x2(__uint_as_float(oa[8 * j]), __uint_as_float(oa[8 * j + 1])),
+                           pack_bf16x2(__uint_as_float(oa[8 * j + 2]), __uint_as_float(oa[8 * j + 3])),
+                           pack_bf16x2(__uint_as_float(oa[8 * j + 4]), __uint_as_float(oa[8 * j + 5])),
+                           pack_bf16x2(__uint_as_float(oa[8 * j + 6]), __uint_as_float(oa[8 * j + 7])));
+          tmem_ld_wait_on(oc);
+#pragma unroll
+          for (int j = 0; j < 16; ++j) ob[j] = __float_as_uint(fmaf(__uint_as_float(oc[j]), f1, __uint_as_float(ob[j])));
+#pragma unroll
+          for (int j = 0; j < 2; ++j)
+            *reinterpret_cast<uint4*>(stage + swz_offset(row, (uint32_t)(sub * 4 + 2 + j), 128)) =
+                make_uint4(pack_bf16x2(__uint_as_float(ob[8 * j]), __uint_as_float(ob[8 * j + 1])),
+                           pack_bf16x2(__uint_as_float(ob[8 * j + 2]), __uint_as_float(ob[8 * j + 3])),
+                           pack_bf16x2(__uint_as_float(ob[8 * j + 4]), __uint_as_float(ob[8 * j + 5])),
+                           pack_bf16x2(__uint_as_float(ob[8 * j + 6]), __uint_as_float(ob[8 * j + 7])));
         }
         fence_proxy_async_smem();
         tcgen05_fence_before_sync();
