@@ -321,6 +321,31 @@ def test_fused_attention_each_query_selects_its_keys(ago, S):
         np.testing.assert_allclose(got[present], want[present], atol=0.26, err_msg=f"S={S} key block {blk}")
 
 
+@pytest.mark.parametrize("name", ["resnet_56", "attn_384", "ffn_12288", "pw_dw_56", "dw_dw_56", "pw_pw_56", "unfold_96"])
+def test_fused_kernels_repeat_bit_for_bit(ago, name):
+    # These kernels have no atomics and a fixed accumulation order: back-to-back launches at the bench's sizes, with other
+    # launches of the same kernel still in flight on the GPU, must reproduce the first result exactly. A race between the
+    # asynchronous copies, the tensor core and the CUDA-core stages shows up as a difference in some launch.
+    # (Not in the list: the kernels with a project GEMM fed by two thread groups -- the inverted-residual block and the
+    # depthwise -> pointwise pair -- add the channel chunks in the order the groups finish them, and the split-reduction
+    # feed-forward kernel adds with atomics: their last bit may differ from launch to launch.)
+    import torch
+    wl = WL.get(name)
+    data = WL.generate(wl)
+    sg = ago.Subgraph(wl.ops, wl.input_shapes, mode="fused")
+    from helpers import to_device
+    ins, ws = to_device(wl, data)
+    outs = [torch.empty(wl.output_shape, dtype=torch.bfloat16, device="cuda:0") for _ in range(6)]
+    for o in outs:
+        sg.run(ins, ws, out=o)
+    torch.cuda.synchronize()
+    assert sg.status() == ago.AGO_OK, ago.ago_last_error()
+    first = outs[0].view(torch.int16)
+    for k, o in enumerate(outs[1:], 1):
+        assert torch.equal(first, o.view(torch.int16)), f"{name}: launch {k} differs from launch 0"
+    sg.close()
+
+
 def test_fused_ffn_512_full(ago):
     wl = WL.get("ffn_512")
     data = WL.generate(wl)
