@@ -345,6 +345,18 @@ def main():
                 return g.replay
 
             context["hot_l2_us_per_launch"] = round(timed(graph_of(hot_pass), max(3, steps // 5), 3) * 1e3 / nsets, 3)
+            # the same launches dealt alternately to two streams: independent batches overlap, so the SMs one grid
+            # leaves idle (and its tail) are taken by the next grid -- throughput of concurrent requests, not the
+            # latency of one
+            side = torch.cuda.Stream(dev)
+
+            def two_stream_pass():
+                side.wait_stream(stream)
+                for r, (ins, ws, out) in enumerate(sets):
+                    sg.run(ins, ws, out=out, stream=(stream if r % 2 == 0 else side).cuda_stream)
+                stream.wait_stream(side)
+
+            context["two_streams_us_per_launch"] = round(timed(graph_of(two_stream_pass), max(3, steps // 5), 3) * 1e3 / nsets, 3)
             grid = max(1, int(sg.query(B.AGO_Q_NUM_LAUNCHES)))
             smem = int(sg.query(B.AGO_Q_SMEM_BYTES)) if mode == "fused" else 0
 
