@@ -40,7 +40,7 @@ NOMINAL_PEAKS = {"hbm_gbs": 8000.0, "bf16_tflops": 2250.0}     # data-sheet figu
 # captures summarised under profiles/ (None until a capture exists for that workload and mode).
 NCU_TRAFFIC_BYTES = {
     ("mbv2_56", "fused"): 4906752 + 0,            # profiles/mbv2_fused_kernel__mbv2_56.txt (output still dirty in L2)
-    ("attn_384", "fused"): 56902400 + 2771456,    # profiles/attention_fused_kernel__attn_384.txt
+    ("attn_384", "fused"): 56796672 + 2367232,    # profiles/attention_fused_kernel__attn_384.txt
     ("resnet_56", "fused"): 13343744 + 3328,      # profiles/conv3x3_pair_kernel__resnet_56.txt
     ("ffn_12288", "fused"): 28403712 + 0,         # profiles/ffn_cluster_kernel__ffn_12288.txt (output still dirty in L2)
     ("ffn_512", "fused"): 11877632 + 0,           # profiles/ffn_fused_kernel__ffn_512.txt
