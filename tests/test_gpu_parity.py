@@ -346,6 +346,52 @@ def test_fused_kernels_repeat_bit_for_bit(ago, name):
     sg.close()
 
 
+def test_fused_attention_full_size_constant_values_come_back(ago):
+    # Any-size property, every element of the bench's output checked: when all keys of a (batch, head) carry the same value
+    # vector, the softmax-weighted mean returns that vector whatever the scores are. The kernel divides a sum of bf16-rounded
+    # probabilities times the constant by the fp32 sum of the unrounded ones: within 2^-9 relative.
+    wl = WL.get("attn_384")
+    data = WL.generate(wl)
+    q, k, v = data["inputs"]
+    B_, S, E = v.shape
+    const = ((np.arange(B_)[:, None] * 7 + np.arange(E)[None, :] * 3) % 33 - 16).astype(np.float32) / 8.0   # bf16-exact
+    v = np.broadcast_to(const[:, None, :], (B_, S, E)).copy()
+    data["inputs"] = [q, k, v]
+    gpu = run_gpu(ago, wl, data, "fused")
+    err = np.abs(gpu - const[:, None, :].astype(np.float64))
+    assert err.max() <= 2.0 * 2.0 ** -8, f"max deviation {err.max():.4g} at {np.unravel_index(err.argmax(), err.shape)}"
+
+
+@pytest.mark.parametrize("name", ["mbv2_56", "mbv2_28s2"])
+def test_fused_inverted_residual_full_size_with_zero_expand_weights(ago, name):
+    # Any-size property at the bench's size, every output element checked against a closed form: with zero expand
+    # weights the expanded tensor is relu6(b1) inside the image and 0 in the padding ring the depthwise convolution sees,
+    # so the depthwise output depends on a pixel's position only through the taps that fall inside the image. A strip
+    # halo that is padded, dropped or taken from the wrong row changes the border rows of some strip.
+    wl = WL.get(name)
+    data = WL.generate(wl)
+    w1, b1, wd, bd, w3, b3 = (a.astype(np.float64) for a in data["weights"])
+    data["weights"][0] = np.zeros_like(data["weights"][0])
+    x = data["inputs"][0].astype(np.float64)
+    N, H, W, _ = x.shape
+    stride = wl.ops[3][1]["stride"]
+    Ho, Wo = wl.output_shape[1], wl.output_shape[2]
+    e = np.clip(b1, 0.0, 6.0)                                    # [Cexp]
+    ho, wo = np.arange(Ho) * stride, np.arange(Wo) * stride
+    acc = np.zeros((Ho, Wo, e.size))
+    for r in range(3):
+        for c in range(3):
+            inside = ((ho + r - 1 >= 0) & (ho + r - 1 < H))[:, None] & ((wo + c - 1 >= 0) & (wo + c - 1 < W))[None, :]
+            acc += inside[:, :, None] * (wd[r, c] * e)[None, None, :]
+    d = np.clip(acc + bd, 0.0, 6.0)                              # [Ho, Wo, Cexp], the same for every image
+    out = d @ w3.reshape(w3.shape[0], -1).T + b3                 # [Ho, Wo, Cout]
+    ref = np.broadcast_to(out, (N,) + out.shape).copy()
+    if len(wl.ops) == 9:
+        ref += x
+    gpu = run_gpu(ago, wl, data, "fused")
+    assert_close(gpu, ref, what=f"{name} with zero expand weights")
+
+
 def test_fused_ffn_512_full(ago):
     wl = WL.get("ffn_512")
     data = WL.generate(wl)

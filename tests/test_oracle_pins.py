@@ -291,6 +291,34 @@ def test_mbv2_chain_against_second_path_and_torch():
         np.testing.assert_allclose(y, ref, rtol=0, atol=1e-12)
 
 
+@pytest.mark.parametrize("stride,residual", [(1, True), (2, False)])
+def test_mbv2_chain_with_zero_expand_weights_has_a_closed_form(stride, residual):
+    # With zero expand weights the expanded tensor is relu6(b1) inside the image and 0 in the padding ring of the
+    # depthwise convolution: its output depends on the position only through the taps inside the image. This pins the
+    # order "bias and ReLU6 first, padding afterwards" and the stride / padding geometry of the chain.
+    from paper_2212_01005_b200 import workloads as WL
+    wl = WL.mbv2_block("pin", [77, stride], 2, 9 + stride, 8, 32, 8 if residual else 16, stride, residual)
+    data = WL.generate(wl)
+    w1, b1, wd, bd, w3, b3 = (a.astype(np.float64) for a in data["weights"])
+    data["weights"][0] = np.zeros_like(data["weights"][0])
+    x = data["inputs"][0].astype(np.float64)
+    N, H, W, _ = x.shape
+    Ho, Wo = wl.output_shape[1], wl.output_shape[2]
+    e = np.clip(b1, 0.0, 6.0)
+    ho, wo = np.arange(Ho) * stride, np.arange(Wo) * stride
+    acc = np.zeros((Ho, Wo, e.size))
+    for r in range(3):
+        for c in range(3):
+            inside = ((ho + r - 1 >= 0) & (ho + r - 1 < H))[:, None] & ((wo + c - 1 >= 0) & (wo + c - 1 < W))[None, :]
+            acc += inside[:, :, None] * (wd[r, c] * e)[None, None, :]
+    out = np.clip(acc + bd, 0.0, 6.0) @ w3.reshape(w3.shape[0], -1).T + b3
+    ref = np.broadcast_to(out, (N,) + out.shape).copy()
+    if residual:
+        ref += x
+    got = O.run_chain(wl.ops, data["inputs"], data["weights"])
+    np.testing.assert_allclose(got, ref, atol=1e-12)
+
+
 def test_ffn_chain_against_torch():
     from paper_2212_01005_b200 import workloads as WL
     wl = WL.ffn("t", [9], 10, 16, 40, 1)
