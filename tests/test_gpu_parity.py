@@ -392,6 +392,51 @@ def test_fused_inverted_residual_full_size_with_zero_expand_weights(ago, name):
     assert_close(gpu, ref, what=f"{name} with zero expand weights")
 
 
+def _taps_inside(H, W):
+    """inside[r][c]: [H, W] mask of the output pixels whose tap (r, c) of a 3x3 window, pad 1, stride 1 lies in the image."""
+    h, w = np.arange(H), np.arange(W)
+    return [[((h + r - 1 >= 0) & (h + r - 1 < H))[:, None] & ((w + c - 1 >= 0) & (w + c - 1 < W))[None, :] for c in range(3)]
+            for r in range(3)]
+
+
+@pytest.mark.parametrize("name", ["resnet_56", "dw_dw_56", "ffn_12288", "pw_pw_56"])
+def test_fused_pairs_full_size_with_zero_first_weights(ago, name):
+    # The first complex operator gets zero weights, so its output is act(b1) everywhere inside the image (and 0 in the
+    # padding ring a 3x3 second operator sees). The result then has a closed form by pixel position, the same for every
+    # image or row: every element of the bench-sized output is checked, whichever CTA, strip or cluster wrote it.
+    wl = WL.get(name)
+    data = WL.generate(wl)
+    data["weights"][0] = np.zeros_like(data["weights"][0])
+    x = data["inputs"][0].astype(np.float64)
+    w2, b2 = data["weights"][2].astype(np.float64), data["weights"][3].astype(np.float64)
+    b1 = data["weights"][1].astype(np.float64)
+    if name == "resnet_56":
+        N, H, W, _ = x.shape
+        mid = np.maximum(b1, 0.0)
+        ins = _taps_inside(H, W)
+        out = np.zeros((H, W, w2.shape[0]))
+        for r in range(3):
+            for c in range(3):
+                out += ins[r][c][:, :, None] * (w2[:, r, c, :] @ mid)[None, None, :]
+        ref = np.maximum(out[None] + b2 + x, 0.0)
+    elif name == "dw_dw_56":
+        N, H, W, _ = x.shape
+        mid = np.clip(b1, 0.0, 6.0)
+        ins = _taps_inside(H, W)
+        out = np.zeros((H, W, mid.size))
+        for r in range(3):
+            for c in range(3):
+                out += ins[r][c][:, :, None] * (w2[r, c] * mid)[None, None, :]
+        ref = np.broadcast_to(np.clip(out + b2, 0.0, 6.0), x.shape[:3] + (mid.size,))
+    else:
+        # no window: every row / pixel gives the same vector; the oracle computes it for one row / pixel
+        one = [x[:1]] if name == "ffn_12288" else [x[:1, :1, :1]]
+        row = O.run_chain(wl.ops, one, data["weights"])
+        ref = np.broadcast_to(row.reshape(-1), wl.output_shape)
+    gpu = run_gpu(ago, wl, data, "fused")
+    assert_close(gpu, np.asarray(ref, np.float64), what=f"{name} with zero first weights")
+
+
 def test_fused_ffn_512_full(ago):
     wl = WL.get("ffn_512")
     data = WL.generate(wl)
