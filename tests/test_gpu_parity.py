@@ -399,7 +399,7 @@ def _taps_inside(H, W):
             for r in range(3)]
 
 
-@pytest.mark.parametrize("name", ["resnet_56", "dw_dw_56", "ffn_12288", "pw_pw_56"])
+@pytest.mark.parametrize("name", ["resnet_56", "dw_dw_56", "pw_dw_56", "ffn_12288", "pw_pw_56", "dw_pw_56"])
 def test_fused_pairs_full_size_with_zero_first_weights(ago, name):
     # The first complex operator gets zero weights, so its output is act(b1) everywhere inside the image (and 0 in the
     # padding ring a 3x3 second operator sees). The result then has a closed form by pixel position, the same for every
@@ -419,7 +419,7 @@ def test_fused_pairs_full_size_with_zero_first_weights(ago, name):
             for c in range(3):
                 out += ins[r][c][:, :, None] * (w2[:, r, c, :] @ mid)[None, None, :]
         ref = np.maximum(out[None] + b2 + x, 0.0)
-    elif name == "dw_dw_56":
+    elif name in ("dw_dw_56", "pw_dw_56"):
         N, H, W, _ = x.shape
         mid = np.clip(b1, 0.0, 6.0)
         ins = _taps_inside(H, W)
@@ -428,6 +428,9 @@ def test_fused_pairs_full_size_with_zero_first_weights(ago, name):
             for c in range(3):
                 out += ins[r][c][:, :, None] * (w2[r, c] * mid)[None, None, :]
         ref = np.broadcast_to(np.clip(out + b2, 0.0, 6.0), x.shape[:3] + (mid.size,))
+    elif name == "dw_pw_56":
+        # zero depthwise weights: relu6(b1) at every pixel, padding or not; the pointwise product of that vector
+        ref = np.broadcast_to(w2.reshape(w2.shape[0], -1) @ np.clip(b1, 0.0, 6.0) + b2, wl.output_shape)
     else:
         # no window: every row / pixel gives the same vector; the oracle computes it for one row / pixel
         one = [x[:1]] if name == "ffn_12288" else [x[:1, :1, :1]]
