@@ -3,7 +3,7 @@
  *
  * A subgraph is an ordered list of operators with shapes (Section II: a
  * computational graph whose nodes are operators and whose edges are tensors;
- * Section III-A: "three operators: 2-d convolution, bias addition, and ReLU").
+ * Section III-A, the convolution / bias / ReLU mini-subgraph).
  * Operator i consumes the output of operator i-1; operator 0 consumes
  * subgraph input 0. Operators are either COMPLEX (they reduce: convolution,
  * matrix multiplication) or SIMPLE (element-wise or row-wise: bias, ReLU, add,
@@ -209,7 +209,13 @@ ago_status_t ago_last_error(const char** msg);
 
 /* Device workspace for intermediates (unfused modes; 0 for fused kernels that
  * need none). The caller allocates at least ago_subgraph_workspace_bytes(h)
- * bytes, 256-byte aligned, and keeps them alive while the handle is used. */
+ * bytes, 256-byte aligned, and keeps them alive while the handle is used.
+ * The workspace is EXCLUSIVE to the handle between set_workspace and the last
+ * run that uses it: a fused kernel that reduces through it (the feed-forward
+ * chain at small row counts) zeroes it at the first run after each
+ * set_workspace and relies on finding it as it left it afterwards. A caller
+ * that lent the buffer to anything else, or whose run failed midway, calls
+ * set_workspace again (same pointer is fine) before the next run. */
 size_t ago_subgraph_workspace_bytes(ago_subgraph_t h);
 ago_status_t ago_subgraph_set_workspace(ago_subgraph_t h, void* dev_ptr, size_t bytes);
 
@@ -220,6 +226,27 @@ ago_status_t ago_subgraph_query(ago_subgraph_t h, int32_t what, int64_t* out);
  * AGO_ERR_TIMEOUT when a kernel gave up a bounded wait (its output is then
  * undefined). The word is cleared by the call. */
 ago_status_t ago_subgraph_status(ago_subgraph_t h);
+
+/* Test hook for the failure path (Section II, last paragraph, and Section IV
+ * "Acyclic Partitioning": the run-time failure the paper names is a wait that
+ * never ends, a deadlock between subgraphs that depend on each other; on the
+ * device its counterpart is a wait on a signal that never comes). Every
+ * device-side wait of this library is bounded; this call lets a test make one
+ * run out on a tiny problem without faulting, trapping or hanging the GPU:
+ *   AGO_DEBUG_WAIT_BUDGET_US  value = budget of every bounded wait of this
+ *                             handle's kernels in microseconds (0 = default, 1 s)
+ *   AGO_DEBUG_SKIP_SIGNAL     value = code of a wait site whose producer skips
+ *                             its signal (an mbarrier arrival) in every run
+ *                             until the value is set back to 0. Sites that
+ *                             honour it: 0x104 (fused inverted-residual block:
+ *                             "all project MMAs complete"), 0x503 (tensor-core
+ *                             GEMM of the unfused modes: "accumulator complete")
+ * The waiter gives up after the budget, the kernel runs to its end (output
+ * undefined), frees its tensor memory, and ago_subgraph_status returns
+ * AGO_ERR_TIMEOUT with the site code in the message. Synchronises the device
+ * when the handle has already run. Errors: AGO_ERR_INVALID_ARG. */
+typedef enum { AGO_DEBUG_WAIT_BUDGET_US = 1, AGO_DEBUG_SKIP_SIGNAL = 2 } ago_debug_t;
+ago_status_t ago_subgraph_debug(ago_subgraph_t h, int32_t what, int64_t value);
 
 /* Bytes of scratch built into the library for ago_subgraph_run_static. */
 #define AGO_STATIC_SCRATCH_BYTES (4u << 20)
@@ -234,7 +261,9 @@ ago_status_t ago_subgraph_status(ago_subgraph_t h);
  * launches go to a fixed AGO_STATIC_SCRATCH_BYTES (4 MiB) array inside the
  * library image, which every GPU that loads the library keeps until the
  * process exits. The call allocates and frees nothing, does not use
- * ago_subgraph_set_workspace and does not touch the handle's status word.
+ * ago_subgraph_set_workspace and does not touch the handle's status word, so
+ * a bounded device-side wait that gives up in one of these launches goes
+ * unreported (ago_subgraph_status stays AGO_OK).
  *   - A subgraph whose ago_subgraph_workspace_bytes() exceeds the array is
  *     rejected with AGO_ERR_WORKSPACE (message states both sizes); FUSED handles
  *     are rejected with AGO_ERR_UNSUPPORTED (they need no scratch).

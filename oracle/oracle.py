@@ -1,7 +1,7 @@
 """CPU oracle for the fused-subgraph executor -- TEST INFRASTRUCTURE ONLY.
 
 A subgraph is an ordered list of operators (Section II: nodes are operators,
-edges are tensors; Section III-A: "2-d convolution, bias addition, and ReLU").
+edges are tensors; Section III-A: the convolution / bias / ReLU mini-subgraph).
 ``run_chain`` applies the operators one after the other, each materialising
 its complete output in fp64, which is the unfused program of Section III-A
 (Fig. "Loop nest of a mini-subgraph without fusion"). Fusion and tiling are
@@ -224,16 +224,38 @@ def transpose(x: np.ndarray, a: int, b: int) -> np.ndarray:
     return np.ascontiguousarray(np.swapaxes(x, a, b))
 
 
+def round_to_bf16(x: np.ndarray) -> np.ndarray:
+    """fp64 -> nearest bfloat16 (ties to even) -> fp64. Used only by the
+    diagnostic switch of ``run_chain``."""
+    u = np.ascontiguousarray(x, dtype=np.float32).view(np.uint32).astype(np.uint64)
+    u = (u + 0x7FFF + ((u >> 16) & 1)) & 0xFFFF0000
+    return u.astype(np.uint32).view(np.float32).astype(np.float64).reshape(np.shape(x))
+
+
+_COMPLEX = ("conv2d", "gemm", "qkt", "pv")
+
+
 def run_chain(ops: Sequence, inputs: Sequence, weights: Sequence,
-              return_intermediates: bool = False):
+              return_intermediates: bool = False, round_intermediates_to_bf16: bool = False):
     """Apply ``ops`` in order to ``inputs[0]``; every operator materialises its
-    whole output in fp64 (no intermediate rounding)."""
+    whole output in fp64 (no intermediate rounding).
+
+    ``round_intermediates_to_bf16`` is a DIAGNOSTIC switch, never the pass/fail
+    reference: it rounds the tensor each complex operator after the first reads
+    to bfloat16, which is where a bf16 tensor-core pipeline must round (its
+    operands are bf16). The difference between the two runs is rounding noise;
+    what remains between the CUDA path and the rounded run is not."""
     ins = [_f64(t) for t in inputs]
     ws = [_f64(t) for t in weights]
     wi = 0
     x = ins[0]
     trace = []
+    seen_complex = False
     for kind, prm in ops:
+        if kind in _COMPLEX:
+            if round_intermediates_to_bf16 and seen_complex:
+                x = round_to_bf16(x)
+            seen_complex = True
         if kind == "conv2d":
             w = ws[wi]; wi += 1
             C = x.shape[-1]

@@ -43,7 +43,7 @@ EXPORTS = [
     "ago_subgraph_create", "ago_subgraph_run", "ago_subgraph_run_host", "ago_subgraph_destroy", "ago_last_error",
     "ago_subgraph_workspace_bytes", "ago_subgraph_set_workspace", "ago_subgraph_query", "ago_subgraph_status",
     "ago_version", "ago_subgraph_run_static", "ago_fusion_redundancy", "ago_op_weight", "ago_graph_cluster",
-    "ago_launch_empty",
+    "ago_launch_empty", "ago_subgraph_debug",
 ]
 
 
@@ -134,6 +134,8 @@ def load(build_if_missing: bool = True):
     lib.ago_graph_cluster.argtypes = [ctypes.POINTER(ago_graph_desc_t), ctypes.POINTER(ctypes.c_int32), ctypes.POINTER(ctypes.c_int32)]
     lib.ago_fusion_redundancy.restype = ctypes.c_int
     lib.ago_fusion_redundancy.argtypes = [ctypes.POINTER(ago_redundancy_query_t), ctypes.POINTER(ago_redundancy_result_t)]
+    lib.ago_subgraph_debug.restype = ctypes.c_int
+    lib.ago_subgraph_debug.argtypes = [vp, ctypes.c_int32, ctypes.c_int64]
     lib.ago_subgraph_run_static.restype = ctypes.c_int
     lib.ago_subgraph_run_static.argtypes = [vp, vpp, vpp, vpp, vp]
     _lib = lib
@@ -240,6 +242,14 @@ def ago_subgraph_query(h, what: int, index: int = 0) -> int:
 
 def ago_subgraph_status(h) -> int:
     return load().ago_subgraph_status(h)
+
+
+AGO_DEBUG_WAIT_BUDGET_US, AGO_DEBUG_SKIP_SIGNAL = 1, 2
+
+
+def ago_subgraph_debug(h, what: int, value: int) -> int:
+    """Test hook of the failure path: wait budget in microseconds / wait site whose producer skips its signal."""
+    return load().ago_subgraph_debug(h, int(what), int(value))
 
 
 def ago_launch_empty(grid: int, block: int, smem_bytes: int = 0, stream: int = 0) -> None:

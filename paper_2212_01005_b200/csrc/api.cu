@@ -17,8 +17,10 @@ struct ago_subgraph_s {
   Plan plan;
   void* workspace = nullptr;
   size_t workspace_bytes = 0;
-  unsigned int* status_word = nullptr;  // device; allocated at the first run
+  unsigned int* status_word = nullptr;  // device status block (code, wait budget, test hook, spare); allocated at the first run
   int status_device = -1;
+  unsigned int wait_budget_us = 0;      // 0: the kernels' default
+  unsigned int skip_signal_code = 0;    // test hook, 0: none
   FusedState fused;                     // per-kernel host state (tensor maps, launch geometry)
 };
 
@@ -36,6 +38,8 @@ ago_status_t fail(ago_status_t s, const std::string& m) {
 ago_status_t cuda_fail(cudaError_t e, const char* what) {
   return fail(AGO_ERR_CUDA, std::string(what) + ": " + cudaGetErrorString(e));
 }
+
+constexpr size_t kStatusBlockBytes = 4 * sizeof(unsigned int);   // tc::kStatusWords
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
@@ -82,7 +86,7 @@ void make_epilogue(const Plan& p, int first, int last, const void* const* inputs
 
 cudaError_t launch_complex(const Plan& p, const OpInfo& o, const void* src, int src_dtype, void* dst, int dst_dtype,
                            const void* const* inputs, const void* const* weights, const EpiProgram& epi,
-                           bool tuned_depthwise, cudaStream_t stream) {
+                           bool tuned_depthwise, unsigned int* status, cudaStream_t stream) {
   const int32_t* q = o.op.p;
   if (o.op.kind == AGO_OP_CONV2D && o.depthwise()) {
     DepthwiseArgs a{};
@@ -100,6 +104,7 @@ cudaError_t launch_complex(const Plan& p, const OpInfo& o, const void* src, int 
   g.A = src; g.C = dst; g.epi = epi;
   g.a_dtype = src_dtype; g.c_dtype = dst_dtype;
   g.batches = 1; g.heads = 1;
+  g.status = status;
   switch (o.op.kind) {
     case AGO_OP_CONV2D: {
       // 3x3 convolutions of equal width with a (bias)(relu) or (bias)(add)(relu) epilogue: tensor-core stage kernel
@@ -111,7 +116,7 @@ cudaError_t launch_complex(const Plan& p, const OpInfo& o, const void* src, int 
         if (k < epi.n && epi.code[k] == EPI_RELU) { relu = 1; ++k; }
         if (k == epi.n)
           return launch_conv3x3_tc(src, weights[o.weight], bias, res, dst, (int)o.in.d[0], (int)o.in.d[1], (int)o.in.d[2],
-                                   (int)o.in.d[3], relu, stream);
+                                   (int)o.in.d[3], relu, status, stream);
       }
       g.B = weights[o.weight];
       g.H = (int)o.in.d[1]; g.W = (int)o.in.d[2]; g.Cin = (int)o.in.d[3];
@@ -170,7 +175,7 @@ cudaError_t launch_complex(const Plan& p, const OpInfo& o, const void* src, int 
 
 // One launch per stage; intermediates ping-pong between the two halves of `ws`.
 ago_status_t run_unfused(ago_subgraph_s* h, const void* const* inputs, const void* const* weights, void* out,
-                         void* ws, size_t ws_bytes, cudaStream_t stream) {
+                         void* ws, size_t ws_bytes, unsigned int* status, cudaStream_t stream) {
   const Plan& p = h->plan;
   const size_t need = unfused_workspace(p);
   const int mid = intermediate_dtype(p);
@@ -198,7 +203,7 @@ ago_status_t run_unfused(ago_subgraph_s* h, const void* const* inputs, const voi
     } else if (s.complex_index >= 0) {
       EpiProgram epi;
       make_epilogue(p, s.first + 1, s.last, inputs, weights, &epi);
-      e = launch_complex(p, p.ops[s.first], src, src_dtype, dst, dst_dtype, inputs, weights, epi, false, stream);
+      e = launch_complex(p, p.ops[s.first], src, src_dtype, dst, dst_dtype, inputs, weights, epi, false, status, stream);
     } else {
       EpiProgram epi;
       make_epilogue(p, s.first, s.last, inputs, weights, &epi);
@@ -219,10 +224,11 @@ ago_status_t ensure_status_word(ago_subgraph_s* h) {
   if (e != cudaSuccess) return cuda_fail(e, "cudaGetDevice");
   if (h->status_word && h->status_device == dev) return AGO_OK;
   if (h->status_word) { cudaFree(h->status_word); h->status_word = nullptr; }
-  e = cudaMalloc(&h->status_word, sizeof(unsigned int));
-  if (e != cudaSuccess) return cuda_fail(e, "cudaMalloc(status word)");
-  e = cudaMemset(h->status_word, 0, sizeof(unsigned int));
-  if (e != cudaSuccess) return cuda_fail(e, "cudaMemset(status word)");
+  e = cudaMalloc(&h->status_word, kStatusBlockBytes);
+  if (e != cudaSuccess) return cuda_fail(e, "cudaMalloc(status block)");
+  const unsigned int init[4] = {0u, h->wait_budget_us, h->skip_signal_code, 0u};
+  e = cudaMemcpy(h->status_word, init, sizeof(init), cudaMemcpyHostToDevice);
+  if (e != cudaSuccess) return cuda_fail(e, "cudaMemcpy(status block)");
   h->status_device = dev;
   return AGO_OK;
 }
@@ -263,7 +269,7 @@ ago_status_t run_unfused_in(ago_subgraph_s* h, const void* const* inputs, const 
     std::snprintf(buf, sizeof(buf), "this subgraph needs %zu bytes of scratch, the built-in array holds %zu", need, ws_bytes);
     return fail(AGO_ERR_WORKSPACE, buf);
   }
-  return run_unfused(h, inputs, weights, outputs[0], ws, ws_bytes, stream);
+  return run_unfused(h, inputs, weights, outputs[0], ws, ws_bytes, nullptr, stream);
 }
 ago_status_t report_failure(ago_status_t s, const char* msg) { return fail(s, msg); }
 }  // namespace ago
@@ -326,6 +332,7 @@ ago_status_t ago_subgraph_set_workspace(ago_subgraph_t h, void* dev_ptr, size_t 
   if (bytes < needed_workspace(h->plan)) return fail(AGO_ERR_WORKSPACE, "workspace smaller than ago_subgraph_workspace_bytes()");
   h->workspace = dev_ptr;
   h->workspace_bytes = bytes;
+  ++h->fused.workspace_epoch;   // nothing remembered about the old contents survives an attach
   return AGO_OK;
 }
 
@@ -337,12 +344,12 @@ ago_status_t ago_subgraph_run(ago_subgraph_t h, const void* const* inputs, const
   s = ensure_status_word(h);
   if (s != AGO_OK) return s;
   const Plan& p = h->plan;
-  if (p.mode != AGO_MODE_FUSED) return run_unfused(h, inputs, weights, outputs[0], h->workspace, h->workspace_bytes, stream);
+  if (p.mode != AGO_MODE_FUSED) return run_unfused(h, inputs, weights, outputs[0], h->workspace, h->workspace_bytes, h->status_word, stream);
   if (p.fused_kernel == AGO_KERNEL_DEPTHWISE) {
     EpiProgram epi;
     make_epilogue(p, 1, (int)p.ops.size() - 1, inputs, weights, &epi);
     if (epi.n != (int)p.ops.size() - 1 || epi.n > kMaxEpi) return fail(AGO_ERR_UNSUPPORTED, "too many simple operators");
-    cudaError_t e = launch_complex(p, p.ops[0], inputs[0], p.dtype, outputs[0], p.dtype, inputs, weights, epi, true, stream);
+    cudaError_t e = launch_complex(p, p.ops[0], inputs[0], p.dtype, outputs[0], p.dtype, inputs, weights, epi, true, h->status_word, stream);
     if (e != cudaSuccess) return cuda_fail(e, "depthwise kernel launch");
     return AGO_OK;
   }
@@ -404,6 +411,22 @@ ago_status_t ago_subgraph_query(ago_subgraph_t h, int32_t what, int64_t* out) {
     case AGO_Q_TILE_ROWS: *out = p.tile_rows; break;
     case AGO_Q_SMEM_BYTES: *out = p.smem_bytes; break;
     default: return fail(AGO_ERR_INVALID_ARG, "unknown query");
+  }
+  return AGO_OK;
+}
+
+ago_status_t ago_subgraph_debug(ago_subgraph_t h, int32_t what, int64_t value) {
+  if (!h) return fail(AGO_ERR_INVALID_ARG, "handle is NULL");
+  if (value < 0 || value > 0xffffffffll) return fail(AGO_ERR_INVALID_ARG, "ago_subgraph_debug: value out of range");
+  if (what == AGO_DEBUG_WAIT_BUDGET_US) h->wait_budget_us = (unsigned int)value;
+  else if (what == AGO_DEBUG_SKIP_SIGNAL) h->skip_signal_code = (unsigned int)value;
+  else return fail(AGO_ERR_INVALID_ARG, "ago_subgraph_debug: unknown selector");
+  if (h->status_word) {   // already on a device: update the block once the work in flight is done
+    cudaError_t e = cudaDeviceSynchronize();
+    if (e != cudaSuccess) return cuda_fail(e, "cudaDeviceSynchronize");
+    const unsigned int words[2] = {h->wait_budget_us, h->skip_signal_code};
+    e = cudaMemcpy(h->status_word + 1, words, sizeof(words), cudaMemcpyHostToDevice);
+    if (e != cudaSuccess) return cuda_fail(e, "cudaMemcpy(status block)");
   }
   return AGO_OK;
 }

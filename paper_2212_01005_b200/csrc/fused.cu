@@ -1,17 +1,41 @@
 // Dispatch of the fused kernel families.
 #include "fused.h"
 
+#include <mutex>
+
 namespace ago {
 
 cudaError_t ensure_max_dynamic_smem(const void* func, int* done_flags) {
+  static std::mutex guard;   // the per-kernel flag arrays are shared by every handle and thread
   int dev = 0;
   cudaError_t e = cudaGetDevice(&dev);
   if (e != cudaSuccess) return e;
   if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+  std::lock_guard<std::mutex> lock(guard);
   if (done_flags[dev]) return cudaSuccess;
   e = cudaFuncSetAttribute(func, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
   if (e == cudaSuccess) done_flags[dev] = 1;
   return e;
+}
+
+int device_sm_count() {
+  static std::mutex guard;
+  static int cached[64] = {};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) {
+    cudaGetLastError();   // planning on a host without a device is legal: clear the sticky "no device" error
+    return kDefaultSMs;
+  }
+  std::lock_guard<std::mutex> lock(guard);
+  if (cached[dev] == 0) {
+    int n = 0;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n < 1) {
+      cudaGetLastError();
+      return kDefaultSMs;
+    }
+    cached[dev] = n;
+  }
+  return cached[dev];
 }
 
 ago_status_t fused_plan(Plan* plan, FusedState* st, std::string* err) {

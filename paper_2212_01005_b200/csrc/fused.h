@@ -14,13 +14,20 @@ struct FusedState {
   int grid = 0;            // CTAs
   int smem_bytes = 0;      // dynamic shared memory per CTA
   int variant = 0;         // kernel variant within the family (feed-forward chain: 1 = thread-block cluster)
+  unsigned workspace_epoch = 0;   // bumped by every ago_subgraph_set_workspace: whatever a kernel family remembers about
+                                  // the workspace contents (e.g. "already zeroed") is void after a new attach
   void* impl = nullptr;                  // kernel-family host state (parameters, tensor-map cache)
   void (*impl_free)(void*) = nullptr;
   ~FusedState() { if (impl && impl_free) impl_free(impl); }
 };
 
-// Opt-in to the full 227 KB of dynamic shared memory for `func`, once per device.
+// Opt-in to the full 227 KB of dynamic shared memory for `func`, once per device (thread-safe).
 cudaError_t ensure_max_dynamic_smem(const void* func, int* done_flags);
+
+// SMs of the current device (cudaDevAttrMultiProcessorCount, cached per device). Planning is host-only and may run
+// where no device is present: then the count of the part this library is written for (B200: 148).
+constexpr int kDefaultSMs = 148;
+int device_sm_count();
 
 // Kernel families (each in its own file).
 ago_status_t mbv2_plan(Plan* plan, FusedState* st, std::string* err);

@@ -58,7 +58,6 @@ constexpr int kComputeThreads = 2 * kGroupThreads;
 constexpr int kThreads = kComputeThreads + 64;   // + TMA warp + MMA warp
 constexpr int kHalfCols = 192;         // tensor-memory columns reserved per score half
 constexpr uint32_t kOCol = 2 * kHalfCols;   // O_0 at kOCol, O_1 at kOCol + kD
-constexpr int kSMs = 148;              // B200
 
 struct AttnParams {
   __nv_bfloat16* out;
@@ -568,7 +567,7 @@ ago_status_t attention_plan(Plan* plan, FusedState* st, std::string* err) {
   if (host->smem_bytes > 227 * 1024) return bad("shared memory budget exceeded");
   st->impl = host;
   st->impl_free = [](void* p) { delete static_cast<AttnHost*>(p); };
-  st->tile_rows = kBlockM; st->grid = std::min(q.total, kSMs); st->smem_bytes = host->smem_bytes;
+  st->tile_rows = kBlockM; st->grid = std::min(q.total, device_sm_count()); st->smem_bytes = host->smem_bytes;
   plan->tile_rows = kBlockM; plan->smem_bytes = host->smem_bytes;
   return AGO_OK;
 }
@@ -603,7 +602,7 @@ ago_status_t attention_run(const Plan& plan, FusedState* st, const void* const* 
     cudaError_t e = ensure_max_dynamic_smem(reinterpret_cast<const void*>(attention_fused_kernel), smem_opt_in);
     if (e != cudaSuccess) { *err = std::string("cudaFuncSetAttribute: ") + cudaGetErrorString(e); return AGO_ERR_CUDA; }
   }
-  dim3 grid((unsigned)std::min(q.total, kSMs));     // one persistent CTA per SM (the shared memory admits no second one)
+  dim3 grid((unsigned)std::min(q.total, device_sm_count()));     // one persistent CTA per SM (the shared memory admits no second one)
   FusedLaunch launch(grid, kThreads, (size_t)host->smem_bytes, stream);
   cudaError_t e = cudaLaunchKernelEx(&launch.config, attention_fused_kernel, *maps[0], *maps[1], *maps[2], *maps[3], q);
   if (e != cudaSuccess) { *err = std::string("fused attention launch: ") + cudaGetErrorString(e); return AGO_ERR_CUDA; }

@@ -402,7 +402,7 @@ ago_status_t conv3x3_plan(Plan* plan, FusedState* st, std::string* err) {
     ConvParams t = q; int smem = 0;
     if (!conv_layout(t, R, &smem)) continue;
     const long ctas = (long)q.N * t.strips;
-    const long waves = (ctas + 147) / 148;
+    const long sms = device_sm_count(), waves = (ctas + sms - 1) / sms;
     const double cost = (double)waves * (t.M1 + t.M2 + 1.0);
     if (best_R == 0 || cost < best_cost) { best_R = R; best_cost = cost; best_smem = smem; }
   }
@@ -519,7 +519,7 @@ bool conv3x3_tc_supported(int H, int W, int Cin, int Cout, int R, int S, int str
 }
 
 cudaError_t launch_conv3x3_tc(const void* x, const void* w, const float* bias, const void* res, void* out, int N, int H,
-                              int W, int C, int relu, cudaStream_t stream) {
+                              int W, int C, int relu, unsigned int* status, cudaStream_t stream) {
   SingleEntry entry;
   {
     std::lock_guard<std::mutex> lock(g_single_mutex);
@@ -536,7 +536,7 @@ cudaError_t launch_conv3x3_tc(const void* x, const void* w, const float* bias, c
       for (int R = 1; R <= H; ++R) {
         ConvParams t = q; int smem = 0;
         if (!conv_layout_single(t, R, &smem)) continue;
-        const long waves = ((long)N * t.strips + 147) / 148;
+        const long sms = device_sm_count(), waves = ((long)N * t.strips + sms - 1) / sms;
         const double cost = (double)waves * (t.M2 + 1.0);
         if (best_R == 0 || cost < best_cost) { best_R = R; best_cost = cost; best_smem = smem; }
       }
@@ -562,7 +562,7 @@ cudaError_t launch_conv3x3_tc(const void* x, const void* w, const float* bias, c
   q.b1 = nullptr; q.b2 = bias;
   q.res = static_cast<const __nv_bfloat16*>(res); q.residual = res != nullptr; q.relu = relu;
   q.out = static_cast<__nv_bfloat16*>(out);
-  q.status = nullptr;
+  q.status = status;
   {
     static int smem_opt_in[64] = {};
     cudaError_t e = ensure_max_dynamic_smem(reinterpret_cast<const void*>(conv3x3_pair_kernel<true>), smem_opt_in);

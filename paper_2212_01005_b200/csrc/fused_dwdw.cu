@@ -209,7 +209,7 @@ ago_status_t dwdw_plan(Plan* plan, FusedState* st, std::string* err) {
     if (smem > 110 * 1024) break;
     const long ctas = (long)q.N * t.strips * q.NC;
     const int per_sm = std::min(4, (227 * 1024) / (smem + 1024));
-    const long waves = (ctas + 148L * per_sm - 1) / (148L * per_sm);
+    const long slots = (long)device_sm_count() * per_sm, waves = (ctas + slots - 1) / slots;
     // time of a wave ~ arithmetic of its CTAs on one SM: rows of depthwise 1 + rows of depthwise 2, in slot-sized steps
     const int s1 = (t.nseg * ((R + 3) / 2) + kSlots - 1) / kSlots, s2 = (t.nseg * ((R + 1) / 2) + kSlots - 1) / kSlots;
     const double cost = (double)waves * per_sm * (s1 + s2 + 0.5);

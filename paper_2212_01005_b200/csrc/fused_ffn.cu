@@ -313,7 +313,8 @@ struct FfnHost {
   FfnParams prm;
   int smem_bytes = 0;
   size_t acc_bytes = 0, ws_bytes = 0;
-  const void* clean_ws = nullptr;   // workspace known to be zeroed (kept so by the kernel itself)
+  const void* clean_ws = nullptr;   // workspace known to be zeroed (kept so by the kernel itself) ...
+  unsigned clean_epoch = 0;         // ... as of this attach (FusedState::workspace_epoch)
   struct Key { const void* p; int which; bool operator==(const Key& o) const { return p == o.p && which == o.which; } };
   struct KeyHash { size_t operator()(const Key& k) const { return std::hash<const void*>()(k.p) ^ (size_t)k.which * 0x9e3779b97f4a7c15ull; } };
   std::unordered_map<Key, CUtensorMap, KeyHash> maps;
@@ -347,7 +348,7 @@ ago_status_t ffn_plan(Plan* plan, FusedState* st, std::string* err) {
   const int htiles = q.Hid / kBH, row_blocks = (q.M + kBM - 1) / kBM;
   q.G = 1;
   for (int g = kMaxG; g >= 2; --g)
-    if (htiles % g == 0 && (long)row_blocks * (htiles / g) >= 2 * 148) { q.G = g; break; }
+    if (htiles % g == 0 && (long)row_blocks * (htiles / g) >= 2 * device_sm_count()) { q.G = g; break; }
   q.hctas = htiles / q.G;
   q.stages = std::min(kMaxStages, 7 - q.G);
   host->smem_bytes = (q.stages + q.G) * kStageBytes + 256 + 1024;
@@ -370,11 +371,13 @@ ago_status_t ffn_run(const Plan& plan, FusedState* st, const void* const* inputs
   q.acc = static_cast<float*>(workspace);
   q.counters = reinterpret_cast<unsigned int*>(static_cast<char*>(workspace) + host->acc_bytes);
   q.status = status_word;
-  if (host->clean_ws != workspace) {
-    // a workspace seen for the first time is zeroed once; after that every launch leaves it zeroed
+  if (host->clean_ws != workspace || host->clean_epoch != st->workspace_epoch) {
+    // a workspace is zeroed at the first run after each attach; after that every launch leaves it zeroed (the caller
+    // must not touch it in between: see ago_subgraph_set_workspace)
     cudaError_t e = cudaMemsetAsync(workspace, 0, host->ws_bytes, stream);
     if (e != cudaSuccess) { *err = std::string("cudaMemsetAsync(workspace): ") + cudaGetErrorString(e); return AGO_ERR_CUDA; }
     host->clean_ws = workspace;
+    host->clean_epoch = st->workspace_epoch;
   }
   auto get_map = [&](const void* base, int which, CUtensorMap* out) -> bool {
     FfnHost::Key key{base, which};

@@ -350,7 +350,7 @@ ago_status_t pwpw_plan(Plan* plan, FusedState* st, std::string* err) {
     return bad("operands too large for the copy index arithmetic");
   // Rows per tile: with k = rounds of 128-row tiles over the resident CTAs, the smallest tile height that still
   // needs k rounds -- the same number of rounds, less work in each
-  const int per_sm = host->smem_bytes <= 113 * 1024 ? 2 : 1, slots = per_sm * 148;
+  const int per_sm = host->smem_bytes <= 113 * 1024 ? 2 : 1, slots = per_sm * device_sm_count();
   const long k = ((long)(q.M + kBM - 1) / kBM + slots - 1) / slots;
   q.BR = (int)std::min<long>(kBM, (q.M + k * slots - 1) / (k * slots));
   q.x_tx = (q.nkb0 + (q.has_res ? q.nkb1 : 0)) * q.BR * 128;

@@ -15,6 +15,7 @@
 #include <mutex>
 #include <unordered_map>
 
+#include "fused.h"
 #include "kernels.h"
 #include "tc_common.cuh"
 #include "tmap.h"
@@ -47,6 +48,7 @@ struct GemmTcParams {
   const void* add;         // or null; same shape and leading dimension as C
   int act1, act2;          // EPI_RELU | EPI_RELU6 | EPI_GELU | -1
   float scale;             // 1 when absent
+  unsigned int* status;    // records a bounded wait that gave up (or null)
 };
 
 __device__ __forceinline__ float activate(float x, int act) {
@@ -101,7 +103,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
       tma_prefetch_desc(&tmap_b);
       for (int i = 0; i < p.kblocks; ++i) {
         const int s = i % kStages;
-        if (i >= kStages) mbar_wait(bar_empty + s, (uint32_t)((i / kStages) - 1) & 1u, abort_flag, nullptr, 0x501);
+        if (i >= kStages) mbar_wait(bar_empty + s, (uint32_t)((i / kStages) - 1) & 1u, abort_flag, p.status, 0x501);
         uint8_t* st = sRing + s * kStageBytes;
         mbar_arrive_expect_tx(bar_full + s, kStageBytes);
         tma_load_4d(st, &tmap_a, bar_full + s, i * kBK, row0, zh, zb);          // A [128 rows x 64 k]
@@ -120,7 +122,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
       const uint32_t idesc = make_idesc_bf16(128, (uint32_t)ncols, 0, p.b_kmajor ? 0 : 1);
       for (int i = 0; i < p.kblocks; ++i) {
         const int s = i % kStages;
-        mbar_wait(bar_full + s, (uint32_t)(i / kStages) & 1u, abort_flag, nullptr, 0x502);
+        mbar_wait(bar_full + s, (uint32_t)(i / kStages) & 1u, abort_flag, p.status, 0x502);
         tcgen05_fence_after_sync();
         const uint32_t st = smem_u32(sRing + s * kStageBytes);
         const uint64_t ad = make_smem_desc(st, 0, 1024, SW_128B);
@@ -130,7 +132,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
           umma_bf16(tmem_base, ad + 2u * ks, bd + (p.b_kmajor ? (uint64_t)(2u * ks) : (uint64_t)((ks * 2048) >> 4)), idesc, (i | ks) != 0);
         umma_commit(bar_empty + s);
       }
-      umma_commit(bar_acc);
+      if (!skip_signal_for_test(p.status, 0x503)) umma_commit(bar_acc);
     }
     __syncwarp();
   } else {
@@ -141,7 +143,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
     const int ncv = min(ncols, p.N - n0);                 // valid columns of this tile (a multiple of 8)
     const int pitch = ncols * esz + 16;                   // staged row pitch: 16-byte stores of a quarter-warp hit distinct banks
     uint8_t* stage = sRing;                               // the ring is idle once the accumulator is complete
-    mbar_wait(bar_acc, 0, abort_flag, nullptr, 0x503);
+    mbar_wait(bar_acc, 0, abort_flag, p.status, 0x503);
     tcgen05_fence_after_sync();
     const bool gelu1 = p.act1 == EPI_GELU, gelu2 = p.act2 == EPI_GELU;
     for (int c0 = 0; c0 < ncols; c0 += 16) {
@@ -295,8 +297,9 @@ cudaError_t launch_gemm_tc(const GemmArgs& a, int add_dtype, cudaStream_t stream
   p.kblocks = (a.K + kBK - 1) / kBK;
   p.heads = heads; p.c_sb = a.batches > 1 ? a.c_sb : 0; p.c_sh = a.batches > 1 ? a.c_sh : 0;
   canonical_epilogue(a.epi, &p);
+  p.status = a.status;
   const long ctas = (long)((a.M + kBM - 1) / kBM) * ((a.N + kBN - 1) / kBN) * heads * nb;
-  p.stages = std::min(ctas > 148 ? 3 : kMaxStages, p.kblocks);
+  p.stages = std::min(ctas > device_sm_count() ? 3 : kMaxStages, p.kblocks);
   // the epilogue stages the output tile (128 rows x (columns x element size + 16) bytes) over the idle ring
   const int tile_cols = std::min(kBN, (a.N + 15) & ~15);
   const int staging = kBM * (tile_cols * (a.c_dtype == AGO_FP32 ? 4 : 2) + 16);

@@ -26,6 +26,7 @@ struct GemmArgs {
   int64_t a_sb, a_sh, b_sb, b_sh, c_sb, c_sh;
   int a_dtype, c_dtype;  // AGO_BF16 | AGO_FP32 storage of A and C (B and EPI_ADD operands are bf16)
   EpiProgram epi;
+  unsigned int* status;  // device word that records a bounded wait that gave up (tensor-core kernel), or null
 };
 cudaError_t launch_gemm_generic(const GemmArgs& a, cudaStream_t stream);
 
@@ -60,7 +61,7 @@ cudaError_t launch_transpose(const void* x, void* y, const int64_t* dims, int ra
 // restricted to one convolution. out = [relu](conv(x, w) + bias [+ res]); bf16 NHWC / OHWI, bias and res may be null.
 bool conv3x3_tc_supported(int H, int W, int Cin, int Cout, int R, int S, int stride, int pad);
 cudaError_t launch_conv3x3_tc(const void* x, const void* w, const float* bias, const void* res, void* out, int N, int H,
-                              int W, int C, int relu, cudaStream_t stream);
+                              int W, int C, int relu, unsigned int* status, cudaStream_t stream);
 
 // ---- fused kernels -------------------------------------------------------------
 

@@ -18,6 +18,18 @@ namespace tc {
 
 constexpr unsigned long long kWaitBudgetNs = 1000000000ull;  // 1 s per wait
 
+// The handle's device status block (four 32-bit words; kernels get a pointer to word 0, or null):
+//   [0] code of the first wait site that gave up (0: none)       -- written by kernels, read and cleared by the host
+//   [1] wait budget in microseconds (0: the default above)        -- written by the host only
+//   [2] test hook: the site code whose producer skips ONE signal  -- written by the host only (0: none)
+// Words 1 and 2 exist so that a test can make a bounded wait run out on a tiny problem without faulting, trapping
+// or hanging anything: the skipped signal is an mbarrier arrival, the waiter gives up after the budget, the kernel
+// runs to its end and frees its tensor memory.
+constexpr int kStatusWords = 4;
+__device__ __forceinline__ bool skip_signal_for_test(const unsigned int* status, uint32_t code) {
+  return status != nullptr && __ldg(status + 2) == code;
+}
+
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
   return static_cast<uint32_t>(__cvta_generic_to_shared(p));
 }
@@ -73,11 +85,13 @@ __device__ __forceinline__ bool mbar_try_wait_parked(uint64_t* bar, uint32_t par
 static __device__ __noinline__ bool mbar_wait_slow(uint64_t* bar, uint32_t parity, volatile uint32_t* abort_flag,
                                             unsigned int* status, uint32_t code) {
   const unsigned long long t0 = globaltimer_ns();
+  const unsigned int budget_us = status ? *(volatile const unsigned int*)(status + 1) : 0u;
+  const unsigned long long budget = budget_us ? (unsigned long long)budget_us * 1000ull : kWaitBudgetNs;
   while (true) {
     for (int i = 0; i < 16; ++i)
       if (mbar_try_wait_parked(bar, parity, 20000u)) return true;
     if (*abort_flag) return false;
-    if (globaltimer_ns() - t0 > kWaitBudgetNs) {
+    if (globaltimer_ns() - t0 > budget) {
       *abort_flag = 1u;
       if (status) atomicCAS(status, 0u, code);
       return false;
