@@ -169,6 +169,7 @@ cudaError_t launch_complex(const Plan& p, const OpInfo& o, const void* src, int 
     default:
       return cudaErrorInvalidValue;
   }
+  if (p.dtype == AGO_BF16 && gemm_pair_supported(g)) return launch_gemm_pair(g, stream);
   if (p.dtype == AGO_BF16 && gemm_tc_supported(g)) return launch_gemm_tc(g, p.dtype, stream);
   return launch_gemm_generic(g, stream);
 }

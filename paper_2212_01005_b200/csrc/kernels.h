@@ -34,6 +34,9 @@ cudaError_t launch_gemm_generic(const GemmArgs& a, cudaStream_t stream);
 // batch / head strides multiples of 8); `add_dtype` is the storage type of EPI_ADD operands (the subgraph's I/O dtype).
 bool gemm_tc_supported(const GemmArgs& a);
 cudaError_t launch_gemm_tc(const GemmArgs& a, int add_dtype, cudaStream_t stream);
+// Large unbatched products on paired CTAs (256 x 256 tiles, persistent; epilogues without a tensor operand).
+bool gemm_pair_supported(const GemmArgs& a);
+cudaError_t launch_gemm_pair(const GemmArgs& a, cudaStream_t stream);
 
 struct DepthwiseArgs {
   const void* in; const void* w; void* out;

@@ -104,6 +104,33 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
   return mbar_wait_slow(bar, parity, abort_flag, status, code);
 }
 
+// The same bounded wait for the single-thread roles (TMA producer, MMA issuer) of a pipelined main loop: it polls
+// with the plain try_wait (which itself blocks for a short, implementation-defined time) instead of parking with a
+// long suspend hint, so the role reacts to the completion at once; one polling thread costs few issue slots.
+static __device__ __noinline__ bool mbar_wait_poll_slow(uint64_t* bar, uint32_t parity, volatile uint32_t* abort_flag,
+                                                        unsigned int* status, uint32_t code) {
+  const unsigned long long t0 = globaltimer_ns();
+  const unsigned int budget_us = status ? *(volatile const unsigned int*)(status + 1) : 0u;
+  const unsigned long long budget = budget_us ? (unsigned long long)budget_us * 1000ull : kWaitBudgetNs;
+  while (true) {
+    for (int i = 0; i < 256; ++i)
+      if (mbar_try_wait(bar, parity)) return true;
+    if (*abort_flag) return false;
+    if (globaltimer_ns() - t0 > budget) {
+      *abort_flag = 1u;
+      if (status) atomicCAS(status, 0u, code);
+      return false;
+    }
+  }
+}
+__device__ __forceinline__ bool mbar_wait_poll(uint64_t* bar, uint32_t parity, volatile uint32_t* abort_flag,
+                                               unsigned int* status, uint32_t code) {
+#pragma unroll 1
+  for (int i = 0; i < 64; ++i)
+    if (mbar_try_wait(bar, parity)) return true;
+  return mbar_wait_poll_slow(bar, parity, abort_flag, status, code);
+}
+
 // Barrier among a subset of the CTA's warps (id 1..15; `threads` a multiple of 32).
 __device__ __forceinline__ void named_barrier_sync(uint32_t id, uint32_t threads) {
   asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
@@ -289,6 +316,60 @@ __device__ __forceinline__ void umma_bf16_lohi(uint32_t d_tmem, uint32_t a_lo, u
 // (implies tcgen05.fence::before_thread_sync).
 __device__ __forceinline__ void umma_commit(uint64_t* bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
+               : "memory");
+}
+
+// ---- paired CTAs (cta_group::2): one MMA spans the two CTAs of a cluster of two -------------------------------
+// The CTA with the even cluster rank (the leader) issues every MMA; an M = 256 product takes rows 0..127 of A and of
+// the accumulator from the leader and rows 128..255 from its peer, and each CTA holds one half (N / 2 columns) of B
+// at the same shared-memory offsets. Each CTA fetches its own operands with its own TMA loads (no multicast); the
+// loads of both CTAs complete on the leader's barrier.
+
+// TMA load whose completion is counted on a barrier that may live in the peer CTA (`bar_cluster_addr` is a
+// shared::cluster address, see cluster_map); the data lands in the issuing CTA.
+__device__ __forceinline__ void tma_load_4d_pair(void* dst, const void* tmap, uint32_t bar_cluster_addr, int c0, int c1, int c2, int c3) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
+      ::"r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(tmap)), "r"(bar_cluster_addr), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
+      : "memory");
+}
+__device__ __forceinline__ void tma_load_2d_pair(void* dst, const void* tmap, uint32_t bar_cluster_addr, int c0, int c1) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+      ::"r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(tmap)), "r"(bar_cluster_addr), "r"(c0), "r"(c1)
+      : "memory");
+}
+// Plain arrival on a barrier given by its cluster address (this CTA's or the peer's).
+__device__ __forceinline__ void mbar_remote_arrive(uint32_t bar_cluster_addr) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(bar_cluster_addr) : "memory");
+}
+__device__ __forceinline__ void tmem_alloc_pair(uint32_t* dst_smem, uint32_t ncols) {
+  asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(dst_smem)), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish_pair() {
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc_pair(uint32_t taddr, uint32_t ncols) {
+  asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+// D[tmem of both CTAs] (+)= A * B across the pair; issued by ONE thread of the leader CTA.
+__device__ __forceinline__ void umma_bf16_pair(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// Arrive on the barrier at cluster address `bar_cluster_addr` once all MMAs issued so far by this thread have
+// completed in both CTAs.
+__device__ __forceinline__ void umma_commit_pair(uint32_t bar_cluster_addr) {
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar_cluster_addr) : "memory");
+}
+// TMA store of a 2-D tile (clipped at the tensor's edges); bulk-group completion as tma_store_3d.
+__device__ __forceinline__ void tma_store_2d(const void* tmap, const void* src, int c0, int c1) {
+  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
+               ::"l"(reinterpret_cast<uint64_t>(tmap)), "r"(smem_u32(src)), "r"(c0), "r"(c1)
                : "memory");
 }
 
