@@ -64,7 +64,14 @@ typedef enum { AGO_BF16 = 0, AGO_FP32 = 1 } ago_dtype_t; /* FP32 I/O: depthwise-
 typedef enum {
   AGO_MODE_FUSED = 0,
   AGO_MODE_PER_MINI_SUBGRAPH = 1,
-  AGO_MODE_PER_OP = 2
+  AGO_MODE_PER_OP = 2,
+  /* The planner decides between FUSED and PER_MINI_SUBGRAPH (Section VI-B: for some pointwise -> pointwise
+   * chains the version WITHOUT intensive fusion is the faster one). It fuses unless the chain has no fused
+   * kernel, or the round trip of the intermediates through device memory costs less than about a third of the
+   * tensor-core time of the contractions (then both modes are bound by the contractions, and two plain GEMM
+   * launches stream their operands better than one kernel that keeps the intermediate on chip). The handle then
+   * behaves like a handle of the chosen mode (AGO_Q_MODE tells which; workspace rules of that mode apply). */
+  AGO_MODE_AUTO = 3
 } ago_mode_t;
 
 typedef enum {
@@ -126,7 +133,8 @@ typedef enum {
   AGO_Q_FUSED_KERNEL = 12,     /* ago_fused_kernel_t chosen by the planner (0 when not fused)      */
   AGO_Q_INTERMEDIATE_BYTES = 13,/* bytes written + read for intermediates in PER_MINI_SUBGRAPH mode */
   AGO_Q_TILE_ROWS = 14,        /* fused kernel: downstream tile extent along the tiled dimension   */
-  AGO_Q_SMEM_BYTES = 15        /* fused kernel: dynamic shared memory per CTA                      */
+  AGO_Q_SMEM_BYTES = 15,       /* fused kernel: dynamic shared memory per CTA                      */
+  AGO_Q_MODE = 16              /* the mode the handle runs in (what AGO_MODE_AUTO resolved to)     */
 } ago_query_t;
 #define AGO_Q_INDEXED(what, i) ((int32_t)(what) | ((int32_t)(i) << 16))
 

@@ -20,8 +20,8 @@ AGO_OK = 0
 AGO_ERR_INVALID_ARG, AGO_ERR_UNSUPPORTED, AGO_ERR_SHAPE, AGO_ERR_ALIGNMENT = 1, 2, 3, 4
 AGO_ERR_WORKSPACE, AGO_ERR_CUDA, AGO_ERR_TIMEOUT = 5, 6, 7
 AGO_BF16, AGO_FP32 = 0, 1
-AGO_MODE_FUSED, AGO_MODE_PER_MINI_SUBGRAPH, AGO_MODE_PER_OP = 0, 1, 2
-MODES = {"fused": AGO_MODE_FUSED, "per_mini_subgraph": AGO_MODE_PER_MINI_SUBGRAPH, "per_op": AGO_MODE_PER_OP}
+AGO_MODE_FUSED, AGO_MODE_PER_MINI_SUBGRAPH, AGO_MODE_PER_OP, AGO_MODE_AUTO = 0, 1, 2, 3
+MODES = {"fused": AGO_MODE_FUSED, "per_mini_subgraph": AGO_MODE_PER_MINI_SUBGRAPH, "per_op": AGO_MODE_PER_OP, "auto": AGO_MODE_AUTO}
 
 (AGO_OP_CONV2D, AGO_OP_GEMM, AGO_OP_BATCHED_QKT, AGO_OP_BATCHED_PV, AGO_OP_BIAS_ADD, AGO_OP_RELU,
  AGO_OP_RELU6, AGO_OP_GELU_TANH, AGO_OP_SCALE, AGO_OP_SOFTMAX_ROWS, AGO_OP_ADD_INPUT, AGO_OP_RESHAPE,
@@ -29,7 +29,7 @@ MODES = {"fused": AGO_MODE_FUSED, "per_mini_subgraph": AGO_MODE_PER_MINI_SUBGRAP
 
 (AGO_Q_NUM_WEIGHTS, AGO_Q_WEIGHT_BYTES, AGO_Q_OUTPUT_RANK, AGO_Q_OUTPUT_DIM, AGO_Q_OUTPUT_BYTES,
  AGO_Q_FLOPS_TENSOR, AGO_Q_FLOPS_CUDA, AGO_Q_SFU_OPS, AGO_Q_IO_BYTES, AGO_Q_NUM_LINKS, AGO_Q_LINK_CATEGORY,
- AGO_Q_NUM_LAUNCHES, AGO_Q_FUSED_KERNEL, AGO_Q_INTERMEDIATE_BYTES, AGO_Q_TILE_ROWS, AGO_Q_SMEM_BYTES) = range(16)
+ AGO_Q_NUM_LAUNCHES, AGO_Q_FUSED_KERNEL, AGO_Q_INTERMEDIATE_BYTES, AGO_Q_TILE_ROWS, AGO_Q_SMEM_BYTES, AGO_Q_MODE) = range(17)
 
 AGO_LINK_DOWNSTREAM_DEPTHWISE, AGO_LINK_DOWNSTREAM_POINTWISE, AGO_LINK_GENERAL = 1, 2, 3
 (AGO_KERNEL_NONE, AGO_KERNEL_DEPTHWISE, AGO_KERNEL_MBV2_BLOCK, AGO_KERNEL_FFN, AGO_KERNEL_CONV3X3_PAIR,

@@ -303,7 +303,29 @@ ago_status_t ago_last_error(const char** msg) {
   return g_status;
 }
 
+namespace {
+// AGO_MODE_AUTO: does fusing this (fusable) chain pay? Not when the intermediates' round trip through device memory
+// costs less than about a third of the contractions' tensor-core time: both modes are then bound by the contractions
+// (Section VI-B reports the same for pointwise -> pointwise chains). Data-sheet-class constants; only the ratio matters.
+bool fusion_pays(const Plan& p) {
+  const double t_intermediates = (double)p.intermediate_bytes / 6.5e12;
+  const double t_tensor = (double)p.flops_tensor / 1.6e15;
+  return !(t_tensor > 0.0 && t_intermediates < 0.35 * t_tensor);
+}
+}  // namespace
+
 ago_subgraph_t ago_subgraph_create(const ago_subgraph_desc_t* desc) {
+  if (desc && desc->struct_size == sizeof(ago_subgraph_desc_t) && desc->mode == AGO_MODE_AUTO) {
+    ago_subgraph_desc_t d = *desc;
+    d.mode = AGO_MODE_FUSED;
+    ago_subgraph_t h = ago_subgraph_create(&d);
+    if (h && fusion_pays(h->plan)) return h;
+    const bool invalid = !h && g_status != AGO_ERR_UNSUPPORTED;   // a malformed chain fails in every mode
+    ago_subgraph_destroy(h);
+    if (invalid) return nullptr;
+    d.mode = AGO_MODE_PER_MINI_SUBGRAPH;
+    return ago_subgraph_create(&d);
+  }
   ago_subgraph_s* h = new (std::nothrow) ago_subgraph_s();
   if (!h) { fail(AGO_ERR_INVALID_ARG, "out of host memory"); return nullptr; }
   std::string err;
@@ -411,6 +433,7 @@ ago_status_t ago_subgraph_query(ago_subgraph_t h, int32_t what, int64_t* out) {
     case AGO_Q_INTERMEDIATE_BYTES: *out = p.intermediate_bytes; break;
     case AGO_Q_TILE_ROWS: *out = p.tile_rows; break;
     case AGO_Q_SMEM_BYTES: *out = p.smem_bytes; break;
+    case AGO_Q_MODE: *out = p.mode; break;
     default: return fail(AGO_ERR_INVALID_ARG, "unknown query");
   }
   return AGO_OK;

@@ -207,3 +207,24 @@ def test_bf16_helpers_round_to_nearest_even():
     import torch
     t = torch.from_numpy(x).to(torch.bfloat16).float().numpy()
     assert np.array_equal(r, t)
+
+
+def test_auto_mode_fuses_unless_the_contractions_bound_both_modes():
+    # AGO_MODE_AUTO resolves at create time (host only): chains whose intermediates dominate the traffic are fused;
+    # the feed-forward chain (two large GEMMs, Section VI-B's pointwise -> pointwise observation) and chains without
+    # a fused kernel run per mini-subgraph
+    from paper_2212_01005_b200 import workloads as WL
+    want = {"attn_384": B.AGO_MODE_FUSED, "mbv2_56": B.AGO_MODE_FUSED, "mbv2_28s2": B.AGO_MODE_FUSED, "resnet_56": B.AGO_MODE_FUSED,
+            "pw_pw_56": B.AGO_MODE_FUSED, "dw_dw_56": B.AGO_MODE_FUSED, "unfold_96": B.AGO_MODE_FUSED,
+            "ffn_12288": B.AGO_MODE_PER_MINI_SUBGRAPH, "ffn_512": B.AGO_MODE_PER_MINI_SUBGRAPH}
+    for name, mode in want.items():
+        wl = WL.get(name)
+        sg = B.Subgraph(wl.ops, wl.input_shapes, mode="auto")
+        assert sg.query(B.AGO_Q_MODE) == mode, name
+        assert sg.query(B.AGO_Q_NUM_LAUNCHES) == (1 if mode == B.AGO_MODE_FUSED else B.Subgraph(wl.ops, wl.input_shapes, mode="per_mini_subgraph").query(B.AGO_Q_NUM_LAUNCHES))
+        sg.close()
+    lone = B.Subgraph([("gemm", {"N": 64}), ("relu", {})], [(256, 64)], mode="auto")     # no fused family: not an error in AUTO
+    assert lone.query(B.AGO_Q_MODE) == B.AGO_MODE_PER_MINI_SUBGRAPH
+    lone.close()
+    with pytest.raises(B.AgoError):
+        B.Subgraph([("gemm", {"N": 0})], [(256, 64)], mode="auto")                        # malformed in every mode

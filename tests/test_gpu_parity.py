@@ -32,6 +32,11 @@ def small_workloads():
         "ffn_c2": WL.ffn("ffn_c2", [33], 9637, 64, 256, 1, d_out=384),
         "ffn_c3": WL.ffn("ffn_c3", [34], 6400, 128, 768, 1, d_out=192),
         "ffn_c4": WL.ffn("ffn_c4", [35], 4864, 64, 512, 1, d_out=1024),
+        # the paired-cluster kernel (two CTA pairs on 256 rows): 128 / 256 / 384 output columns per pair, one to three steps
+        # per row block, one and two row blocks per cluster, ragged last block
+        "ffn_p1": WL.ffn("ffn_p1", [38], 8349, 64, 512, 1, d_out=256),
+        "ffn_p2": WL.ffn("ffn_p2", [39], 7680, 128, 256, 1, d_out=512),
+        "ffn_p3": WL.ffn("ffn_p3", [40], 12000, 192, 768, 1, d_out=768),
         "resnet_small": WL.resnet_block("resnet_small", [26], 2, 12, 64),
         "resnet_odd": WL.resnet_block("resnet_odd", [27], 1, 9, 32),
         "resnet_16ch": WL.resnet_block("resnet_16ch", [32], 2, 20, 16),
@@ -150,7 +155,7 @@ def test_padding_of_the_intermediate_with_large_bias(ago):
 # ---- fused kernels -------------------------------------------------------------------
 
 FUSED_SMALL = ["mbv2_14", "mbv2_s1_odd", "mbv2_s2", "mbv2_s2_odd", "attn_small", "attn_ragged", "attn_runs2", "attn_runs4", "ffn_small", "ffn_rows_ragged", "ffn_g2", "ffn_g3",
-               "ffn_c2", "ffn_c3", "ffn_c4", "resnet_small", "resnet_odd", "resnet_16ch"]
+               "ffn_c2", "ffn_c3", "ffn_c4", "ffn_p1", "ffn_p2", "ffn_p3", "resnet_small", "resnet_odd", "resnet_16ch"]
 
 
 @pytest.mark.parametrize("name", FUSED_SMALL)
@@ -526,3 +531,11 @@ def test_fused_ffn_workspace_lent_to_another_handle(ago):
         assert_close(f.float().cpu().numpy().astype(np.float64), ref, what=f"ffn_512 fused after lending, round {rnd}")
         assert_close(m.float().cpu().numpy().astype(np.float64), ref, what=f"ffn_512 unfused, round {rnd}")
     fused.close(); mini.close()
+
+
+@pytest.mark.parametrize("name", ["ffn_small", "ffn_c3", "mbv2_14", "attn_small", "resnet_small"])
+def test_auto_mode_matches_oracle(ago, name):
+    # AGO_MODE_AUTO resolves to the fused kernel or to the per-mini-subgraph chain; either way the result is the chain's
+    wl = small_workloads()[name]
+    data = WL.generate(wl)
+    assert_close(run_gpu(ago, wl, data, "auto"), reference(name, wl, data), what=f"{name}/auto")
