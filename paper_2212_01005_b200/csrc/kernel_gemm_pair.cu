@@ -51,7 +51,10 @@ struct GemmPairParams {
   int b_kmajor;
   int c_fp32;              // output element: fp32 (else bf16)
   int kblocks, tiles_m, tiles_n, pairs;
+  // the simple operators in canonical order: + bias, activation 1, * scale, + tensor, activation 2
   const float* bias;       // or null
+  const void* add;         // or null: bf16 tensor [M][N] with the output's leading dimension
+  int64_t ldc;
   int act1, act2;          // EPI_RELU | EPI_RELU6 | EPI_GELU | -1
   float scale;
   unsigned int* status;
@@ -220,6 +223,17 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
 #pragma unroll
             for (int j = 0; j < 32; ++j) y[j] = pair_activate(y[j], p.act1) * p.scale;
           }
+          if (p.add && row0 + row < p.M) {   // + tensor: this thread's row, 16-byte pieces (N is a multiple of 8)
+            const __nv_bfloat16* arow = reinterpret_cast<const __nv_bfloat16*>(p.add) + (int64_t)(row0 + row) * p.ldc + col + j0;
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+              if (col + j0 + 8 * k < p.N) {
+                const uint4 t = __ldg(reinterpret_cast<const uint4*>(arow + 8 * k));
+                y[8 * k] += bf16_lo(t.x); y[8 * k + 1] += bf16_hi(t.x); y[8 * k + 2] += bf16_lo(t.y); y[8 * k + 3] += bf16_hi(t.y);
+                y[8 * k + 4] += bf16_lo(t.z); y[8 * k + 5] += bf16_hi(t.z); y[8 * k + 6] += bf16_lo(t.w); y[8 * k + 7] += bf16_hi(t.w);
+              }
+            }
+          }
           if (p.act2 >= 0) {
 #pragma unroll
             for (int j = 0; j < 32; ++j) y[j] = pair_activate(y[j], p.act2);
@@ -288,9 +302,9 @@ bool pair_map(const void* base, int d0, int d1, int64_t ld, int b0, int b1, CUte
   return true;
 }
 
-// (+ bias) (activation) (* scale) (activation): the simple operators this kernel applies; no tensor operand
+// (+ bias) (activation) (* scale) (+ tensor) (activation): the simple operators this kernel applies, in this order
 bool pair_epilogue(const EpiProgram& e, GemmPairParams* p) {
-  p->bias = nullptr; p->act1 = -1; p->act2 = -1; p->scale = 1.0f;
+  p->bias = nullptr; p->add = nullptr; p->act1 = -1; p->act2 = -1; p->scale = 1.0f;
   int stage = 0;
   for (int i = 0; i < e.n; ++i) {
     const int c = e.code[i];
@@ -298,7 +312,8 @@ bool pair_epilogue(const EpiProgram& e, GemmPairParams* p) {
     if (c == EPI_BIAS && stage < 1) { p->bias = static_cast<const float*>(e.ptr[i]); stage = 1; }
     else if (act && stage < 2) { p->act1 = c; stage = 2; }
     else if (c == EPI_SCALE && stage < 3) { p->scale = e.f[i]; stage = 3; }
-    else if (act && stage == 3) { p->act2 = c; stage = 4; }
+    else if (c == EPI_ADD && stage < 4) { p->add = e.ptr[i]; stage = 4; }
+    else if (act && stage == 4) { p->act2 = c; stage = 5; }
     else return false;
   }
   return true;
@@ -306,7 +321,9 @@ bool pair_epilogue(const EpiProgram& e, GemmPairParams* p) {
 
 }  // namespace
 
-// Large unbatched products with wide outputs: everything else stays on the small-tile kernel.
+// Unbatched products with enough rows to fill the SM pairs (wide or narrow, long or short reductions: the narrow,
+// short ones -- 1x1 convolutions of a few tens of channels -- are bound by the output stream, which the persistent
+// pairs overlap with the next tile's loads and products); everything else stays on the small-tile kernel.
 bool gemm_pair_supported(const GemmArgs& a) {
   GemmPairParams probe{};
   if (!pair_epilogue(a.epi, &probe)) return false;
@@ -314,7 +331,8 @@ bool gemm_pair_supported(const GemmArgs& a) {
   if (a.a_im2col && !(a.R == 1 && a.S == 1 && a.stride == 1 && a.pad == 0)) return false;
   if (a.K % 8 != 0 || a.N % 8 != 0 || a.ldb % 8 != 0 || a.ldc % 8 != 0) return false;
   if (!a.a_im2col && a.lda % 8 != 0) return false;
-  if (a.N < 128 || a.M < 512 || a.K < 64) return false;
+  if (probe.add && a.c_dtype != AGO_BF16) return false;   // the added tensor has the I/O dtype of a bf16 subgraph
+  if (a.M < 512) return false;
   // worth it once the 256-row tiles fill most of the SM pairs
   const long tiles = (long)((a.M + 255) / 256) * ((a.N + 255) / 256);
   return tiles * 2 >= device_sm_count() / 2;
@@ -331,6 +349,7 @@ cudaError_t launch_gemm_pair(const GemmArgs& a, cudaStream_t stream) {
   p.tiles_m = (a.M + 2 * kPM - 1) / (2 * kPM);
   p.tiles_n = (a.N + p.BN - 1) / p.BN;
   p.status = a.status;
+  p.ldc = a.ldc;
   const int64_t lda = a.a_im2col ? a.K : a.lda;
   CUtensorMap ma, mb, mc;
   if (!pair_map(a.A, a.K, a.M, lda, kPK, kPM, &ma)) return cudaErrorInvalidValue;
