@@ -46,8 +46,9 @@ using namespace dw;
 
 constexpr int kWarps = 32;                         // every warp computes; MMAs are issued inline by some of them
 constexpr int kThreads = kWarps * 32;
-constexpr int kGroupWarps = kWarps / 2;            // two groups of warps on alternating chunks
-constexpr int kGroupThreads = kGroupWarps * 32;
+// The warps form NG groups (2 or 4) that own the chunks c = g, g + NG, ...: two groups of 16 warps for strips whose
+// chunk is real work (their phases overlap), four groups of 8 warps for small strips, where a chunk is a chain of
+// latencies (MMA hand-off, tensor-memory round trip, two barriers) and more chains in flight is all that helps.
 constexpr int kTilesPerWarp = 2;                   // expand-epilogue tiles per warp: at most 8 tiles over the 4 warps of a lane quarter
 constexpr int kExpandIssuers = 2;                  // the last two warps of a group issue its expand GEMMs
 constexpr int kChunk = 16;      // expanded channels per chunk = one MMA K step of the project GEMM
@@ -64,6 +65,7 @@ struct Mbv2Params {
   __nv_bfloat16* out;
   unsigned int* status;
   int N, H, W, Cin, Cexp, Cout, stride, Ho, Wo, residual;
+  int groups;                   // warp groups: 2 or 4 (the kernel template's NG)
   int fold_b1;                  // the expand bias rides in two spare reduction channels of the expand GEMM (Cin < Kp)
   int R, strips, IH, IW, P_x, P_in, M1, M2;   // P_x = IH * W pixels in the input tile, P_in = IH * IW in an E chunk
   int Kp, row_bytes, swizzle;   // input / W1 tiles: padded K, bytes per row, tc::SwizzleMode
@@ -92,9 +94,11 @@ __device__ __forceinline__ void sts128(uint32_t saddr, uint32_t a, uint32_t b, u
 // block: <true, true> the whole block, <true, false> pointwise -> depthwise
 // (the depthwise result of every chunk goes to device memory), <false, true> depthwise -> pointwise (every chunk of
 // the input is copied into the E buffers instead of being computed).
-template <bool EXPAND, bool PROJECT, bool FOLD>
+template <bool EXPAND, bool PROJECT, bool FOLD, int NG>
 __global__ void __launch_bounds__(kThreads, 1)
 mbv2_fused_kernel(const Mbv2Params p) {
+  constexpr int kGroupWarps = kWarps / NG;
+  constexpr int kGroupThreads = kGroupWarps * 32;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t* sX = smem + p.off_x;
@@ -107,12 +111,12 @@ mbv2_fused_kernel(const Mbv2Params p) {
   float* sBd = reinterpret_cast<float*>(smem + p.off_bd);
   float* sB3 = reinterpret_cast<float*>(smem + p.off_b3);
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + p.off_bar);
-  uint64_t* bar_e = bars + 2;       // [2] expand accumulators of buffer b complete (MMA commit)
-  uint64_t* bar_d = bars + 4;       // [2] project MMA has consumed D[b] (MMA commit)
-  uint64_t* bar_first = bars + 6;   // project GEMM of chunk 0 complete (it overwrites the output accumulators: group 1 issues after it)
-  uint64_t* bar_done = bars + 10;   // every project MMA complete (the groups do not follow each other's bar_d phases)
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 12);
-  volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(bars + 13);
+  uint64_t* bar_e = bars;           // [NG] expand accumulators of group g complete (MMA commit)
+  uint64_t* bar_d = bars + 4;       // [NG] project MMA has consumed D[g] (MMA commit)
+  uint64_t* bar_first = bars + 8;   // project GEMM of chunk 0 complete (it overwrites the output accumulators: the other groups issue after it)
+  uint64_t* bar_done = bars + 9;    // every project MMA complete (the groups do not follow each other's bar_d phases)
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 10);
+  volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(bars + 11);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int n = (int)fast_div(blockIdx.x, (uint32_t)p.strips, p.strips_recip), strip = (int)blockIdx.x - n * p.strips;
@@ -123,12 +127,12 @@ mbv2_fused_kernel(const Mbv2Params p) {
 
   if (tid == kThreads - 1) {
     *abort_flag = 0u;
-    for (int i = 0; i < 2; ++i) {
+    for (int i = 0; i < NG; ++i) {
       mbar_init(bar_e + i, kExpandIssuers);
       mbar_init(bar_d + i, (uint32_t)p.M2);
     }
     mbar_init(bar_first, (uint32_t)p.M2);
-    mbar_init(bar_done, (uint32_t)(p.M2 * min(p.NC, 2)));
+    mbar_init(bar_done, (uint32_t)(p.M2 * min(p.NC, NG)));
     fence_mbar_init();
     fence_proxy_async_smem();
   }
@@ -264,7 +268,7 @@ mbv2_fused_kernel(const Mbv2Params p) {
     }
     auto load_chunk = [&](int c, int b) {   // chunk c -> E buffer (g, b); always one commit group
       if (c < p.NC) {
-        const uint32_t e0 = smem_u32(sE) + (uint32_t)((g * 2 + b) * e_bytes);
+        const uint32_t e0 = smem_u32(sE) + (uint32_t)((g * 2 + b) * e_bytes);   // two buffers per group
 #pragma unroll
         for (int k = 0; k < kPieces; ++k) {
           if ((ld_ok >> k) & 1u) {
@@ -277,7 +281,7 @@ mbv2_fused_kernel(const Mbv2Params p) {
     };
     grid_dependency_wait();      // first access to device memory below
     grid_launch_dependents();
-    if (!EXPAND) { load_chunk(g, 0); load_chunk(g + 2, 1); }   // the first two chunks travel while the weights are staged
+    if (!EXPAND) { load_chunk(g, 0); load_chunk(g + NG, 1); }   // the first two chunks travel while the weights are staged
 #pragma unroll
     for (int k = 0; k < kBX; ++k) {
       const uint32_t i = (uint32_t)(tid + k * kThreads);
@@ -316,9 +320,9 @@ mbv2_fused_kernel(const Mbv2Params p) {
       *reinterpret_cast<uint4*>(smem + d) = load_or_zero(src);
     }
     // the zero padding columns of the two E chunk buffers (written once: every chunk reuses them)
-    constexpr int kEShift = EXPAND ? 2 : 3;   // 2 E buffers x 2 planes, or 4 x 2 when the chunks are copied in (two per group)
-    for (int i = tid; i < p.IH << (kEShift + 1); i += kThreads) {
-      const int ih = i >> (kEShift + 1), side = (i >> kEShift) & 1, plane = i & ((1 << kEShift) - 1);
+    constexpr int kEPlanes = (EXPAND ? NG : 2 * NG) * 2;   // one E buffer per group (two when the chunks are copied in), two planes each
+    for (int i = tid; i < p.IH * 2 * kEPlanes; i += kThreads) {
+      const int ih = i / (2 * kEPlanes), side = (i / kEPlanes) & 1, plane = i % kEPlanes;
       *reinterpret_cast<uint4*>(sE + plane * p.e_plane + (ih * p.IW + side * (p.IW - 1)) * 16) = make_uint4(0, 0, 0, 0);
     }
     fence_proxy_async_smem();
@@ -355,7 +359,7 @@ mbv2_fused_kernel(const Mbv2Params p) {
     const uint32_t exp_a_step = (uint32_t)(kExpandIssuers * 128 * p.row_bytes) >> 4;
     const uint32_t exp_a_lo0 = (uint32_t)xdesc0 + ((uint32_t)(max(xi, 0) * 128 * p.row_bytes) >> 4);
     const uint32_t exp_d_tmem0 = tmem_base + p.ecol0 + (g * p.M1 + max(xi, 0)) * kChunk;
-    const uint32_t exp_b_step = (uint32_t)(2 * kChunk * p.row_bytes) >> 4;   // the group's next chunk is c + 2
+    const uint32_t exp_b_step = (uint32_t)(NG * kChunk * p.row_bytes) >> 4;   // the group's next chunk is c + NG
     uint32_t exp_b_lo = (uint32_t)w1desc0 + ((uint32_t)(g * kChunk * p.row_bytes) >> 4);
     const int ksteps = p.Kp / 16;
     auto issue_expand = [&]() {   // one lane; advances to the group's next chunk
@@ -377,12 +381,12 @@ mbv2_fused_kernel(const Mbv2Params p) {
     const uint32_t idesc_p = make_idesc_bf16(128, (uint32_t)p.Coutp);
     const uint32_t proj_a_lo = (uint32_t)ddesc0 + ((uint32_t)(g * d_bytes + gw * 128 * 16) >> 4);
     const uint32_t proj_d_tmem = tmem_base + p.pcol0 + gw * p.Coutp;
-    const uint32_t proj_b_step = (uint32_t)(2 * p.Coutp * kChunkRowBytes) >> 4;     // the group's next chunk is c + 2
+    const uint32_t proj_b_step = (uint32_t)(NG * p.Coutp * kChunkRowBytes) >> 4;     // the group's next chunk is c + NG
     uint32_t proj_b_lo = (uint32_t)w3desc0 + ((uint32_t)(g * p.Coutp * kChunkRowBytes) >> 4);
     if (EXPAND && xi >= 0 && lane == 0 && g < p.NC) {
       // group 1 issues its first expand GEMM once group 0's is through the tensor pipe: group 0 has the longer chain
       // of chunks, and its first epilogue would otherwise wait for both groups' MMAs
-      if (g == 1) mbar_wait(bar_e, 0, abort_flag, p.status, 0x107);
+      if (g >= 1) mbar_wait(bar_e + g - 1, 0, abort_flag, p.status, 0x107);
       issue_expand();
     }
     __syncwarp();
@@ -411,7 +415,7 @@ mbv2_fused_kernel(const Mbv2Params p) {
     uint32_t wd_addr = smem_u32(sWd) + (uint32_t)(g * 9 * kChunkRowBytes + cp * 4);
     uint32_t bd_addr = smem_u32(sBd) + (uint32_t)((g * kChunk + cp * 2) * 4);
     uint32_t b1_addr = smem_u32(sB1) + (uint32_t)(g * kChunk * 4);
-    for (int c = g, it = 0; c < p.NC; c += 2, ++it) {
+    for (int c = g, it = 0; c < p.NC; c += NG, ++it) {
       // ---- P3: expand epilogue of chunk c -> E[g]: + b1, ReLU6, zero outside the image, bf16 ----
       if (!EXPAND) cp_async_wait_but_one();   // this thread's pieces of chunk c have landed
       if (EXPAND) {
@@ -445,13 +449,13 @@ mbv2_fused_kernel(const Mbv2Params p) {
           sts128(e_off[k] + (uint32_t)p.e_plane, w[4], w[5], w[6], w[7]);
         }
       }
-      b1_addr += 2u * kChunk * 4u;
+      b1_addr += (uint32_t)NG * kChunk * 4u;
       tcgen05_fence_before_sync();
       }
       // D[g] was read by the project GEMM of chunk c - 2
       if (PROJECT && waiter && it >= 1) mbar_wait(bar_d + g, (uint32_t)(it - 1) & 1u, abort_flag, p.status, 0x103);
       named_barrier_sync(gbar, kGroupThreads);
-      if (EXPAND && xi >= 0 && c + 2 < p.NC) {   // expand buffer g is drained: the expand GEMM of the group's next chunk
+      if (EXPAND && xi >= 0 && c + NG < p.NC) {   // expand buffer g is drained: the expand GEMM of the group's next chunk
         if (lane == 0) {
           tcgen05_fence_after_sync();
           issue_expand();
@@ -466,7 +470,7 @@ mbv2_fused_kernel(const Mbv2Params p) {
         wgt[3] = lds32<96>(wd_addr); wgt[4] = lds32<128>(wd_addr); wgt[5] = lds32<160>(wd_addr);
         wgt[6] = lds32<192>(wd_addr); wgt[7] = lds32<224>(wd_addr); wgt[8] = lds32<256>(wd_addr);
         const float2 bias = make_float2(__uint_as_float(lds32<0>(bd_addr)), __uint_as_float(lds32<4>(bd_addr)));
-        wd_addr += 2u * 9u * kChunkRowBytes; bd_addr += 2u * kChunk * 4u;   // the group's next chunk is c + 2
+        wd_addr += (uint32_t)NG * 9u * kChunkRowBytes; bd_addr += (uint32_t)NG * kChunk * 4u;   // the group's next chunk is c + NG
         const uint32_t e_plane = e_plane0 + (EXPAND ? 0u : (uint32_t)((it & 1) * e_bytes));
         if (has_item) {   // the thread's first item: geometry fixed before the chunk loop
           if (p.stride == 1) depthwise_block(e_plane + it_e, d_plane + it_d, e_pitch, d_pitch, it_a, it_b, wgt, bias);
@@ -491,9 +495,9 @@ mbv2_fused_kernel(const Mbv2Params p) {
       }
       fence_proxy_async_smem();
       // the expand GEMM of the group's next chunk (issued after the previous barrier) is complete
-      if (EXPAND && waiter && c + 2 < p.NC) mbar_wait(bar_e + g, (uint32_t)(it + 1) & 1u, abort_flag, p.status, 0x102);
+      if (EXPAND && waiter && c + NG < p.NC) mbar_wait(bar_e + g, (uint32_t)(it + 1) & 1u, abort_flag, p.status, 0x102);
       named_barrier_sync(gbar, kGroupThreads);
-      if (!EXPAND) load_chunk(c + 4, it & 1);   // the E buffer of chunk c is free
+      if (!EXPAND) load_chunk(c + 2 * NG, it & 1);   // the E buffer of chunk c is free
       if (!PROJECT) {
         // the depthwise result of the chunk is the output: 16-byte pieces (pixel, plane) of D[g] to device memory
         const int pieces = rows_valid * p.Wo * 2;
@@ -507,12 +511,12 @@ mbv2_fused_kernel(const Mbv2Params p) {
       if (PROJECT && gw < p.M2) {   // D[g] is complete: the project GEMM of chunk c, one tile per warp
         if (lane == 0) {
           // chunk 0 overwrites the accumulators: everything else is issued after it
-          if (c == 1) mbar_wait(bar_first, 0, abort_flag, p.status, 0x106);
+          if (c >= 1 && c < NG) mbar_wait(bar_first, 0, abort_flag, p.status, 0x106);
           tcgen05_fence_after_sync();
           umma_bf16_lohi(proj_d_tmem, proj_a_lo, d_hi, proj_b_lo, w3_hi, idesc_p, c > 0);
           umma_commit(bar_d + g);
           if (c == 0) umma_commit(bar_first);
-          if (c + 2 >= p.NC && !skip_signal_for_test(p.status, 0x104)) umma_commit(bar_done);
+          if (c + NG >= p.NC && !skip_signal_for_test(p.status, 0x104)) umma_commit(bar_done);
         }
         __syncwarp();
       }
@@ -569,6 +573,7 @@ struct Mbv2Host {
 };
 
 bool layout(Mbv2Params& q, int R, bool expand, bool project, int* smem_bytes) {
+  const int NG = q.groups, group_threads = kThreads / NG;
   q.R = R;
   q.strips = (q.Ho + R - 1) / R;
   q.strips_recip = fast_div_recip(q.strips);
@@ -579,12 +584,15 @@ bool layout(Mbv2Params& q, int R, bool expand, bool project, int* smem_bytes) {
   q.M1 = (q.P_x + 127) / 128;
   q.M2 = (R * q.Wo + 127) / 128;
   if (q.IH > 256 || q.IW > 256 || q.M1 > 8) return false;
-  const int cols = (expand ? 2 * q.M1 * kChunk : 0) + (project ? q.M2 * q.Coutp : 0);
+  // per group: at most kTilesPerWarp expand tiles per warp of a lane quarter, one project tile per warp, and (when the
+  // chunks are copied in) four 16-byte pieces per thread
+  if (q.M1 > kTilesPerWarp * (kWarps / NG / 4) || q.M2 > kWarps / NG || (!expand && q.P_x * 2 > 4 * group_threads)) return false;
+  const int cols = (expand ? NG * q.M1 * kChunk : 0) + (project ? q.M2 * q.Coutp : 0);
   if (cols > 512) return false;
   q.tmem_cols = 32;
   while (q.tmem_cols < cols) q.tmem_cols *= 2;
   q.ecol0 = 0;
-  q.pcol0 = expand ? 2 * q.M1 * kChunk : 0;
+  q.pcol0 = expand ? NG * q.M1 * kChunk : 0;
   int off = 0;
   auto take = [&](int bytes) { int o = off; off = round_up(off + bytes, 1024); return o; };
   q.off_x = take(expand ? q.M1 * 128 * q.row_bytes : 0);
@@ -593,8 +601,8 @@ bool layout(Mbv2Params& q, int R, bool expand, bool project, int* smem_bytes) {
   // 2 x 64-byte accesses (4 pixels x 4 channel pairs per plane) never share a bank
   q.e_plane = round_up(q.P_in * 16, 128) + 64;
   q.d_plane = q.M2 * 128 * 16 + 64;
-  q.off_e = take((expand ? 2 : 4) * 2 * q.e_plane);   // one chunk buffer per group, two when the chunks are copied in
-  q.off_d = take(2 * 2 * q.d_plane);
+  q.off_e = take((expand ? NG : 2 * NG) * 2 * q.e_plane);   // one chunk buffer per group, two when the chunks are copied in
+  q.off_d = take(NG * 2 * q.d_plane);
   q.off_w3 = take(project ? q.NC * q.Coutp * kChunkRowBytes : 0);
   q.off_wd = take(9 * q.Cexp * 2);
   q.off_b1 = take(expand ? q.Cexp * 4 : 0);
@@ -639,26 +647,36 @@ ago_status_t mbv2_plan(Plan* plan, FusedState* st, std::string* err) {
   q.coutp_recip = recip(q.Coutp);
   q.w_recip = recip(q.W);
   q.cexp8_recip = recip(q.Cexp / 8);
-  {
-    constexpr int kSlots = kGroupThreads / 8;
-    q.nseg = (q.Wo + kSegCols - 1) / kSegCols;
-    q.per_row = q.stride == 1 ? q.nseg : q.Wo;
-    q.per_row_recip = recip(q.per_row);
-    q.step_r = kSlots / q.per_row; q.step_c = kSlots - q.step_r * q.per_row;
-    q.col_slots = kSlots / std::max(1, std::min(q.Wo, kSlots));
-  }
-  // Rows per CTA: fewest waves over the SMs, then least halo + tail work.
-  int best_R = 0; double best_cost = 0; int best_smem = 0;
+  q.nseg = (q.Wo + kSegCols - 1) / kSegCols;
+  q.per_row = q.stride == 1 ? q.nseg : q.Wo;
+  q.per_row_recip = recip(q.per_row);
+  auto set_groups = [&](Mbv2Params& t, int ng) {   // depthwise item geometry of a group of 32 / ng warps
+    const int slots = kThreads / ng / 8;
+    t.groups = ng;
+    t.step_r = slots / t.per_row; t.step_c = slots - t.step_r * t.per_row;
+    t.col_slots = slots / std::max(1, std::min(t.Wo, slots));
+  };
+  // Warp groups and rows per CTA: the least estimated time = waves x (fixed part + chunk loop), where the chunk loop
+  // is the larger of the strip's arithmetic (issue-bound: about 0.8 cycles per pixel-tile unit and chunk, measured
+  // on 56 x 56 strips) and the chain of latencies of the chunks one group owns (about 2.9k cycles per chunk,
+  // measured on 28 x 28 strips). Small strips therefore run with four groups, large ones with two.
+  int best_R = 0, best_ng = 2; double best_cost = 0; int best_smem = 0;
   const int sms = device_sm_count();
-  for (int R = 1; R <= q.Ho; ++R) {
-    Mbv2Params t = q; int smem = 0;
-    if (!layout(t, R, expand, project, &smem)) continue;
-    const long ctas = (long)q.N * t.strips;
-    const long waves = (ctas + sms - 1) / sms;
-    const double cost = (double)waves * (t.M1 * 128.0 + 3.0 * t.M2 * 128.0 + 200.0);
-    if (best_R == 0 || cost < best_cost) { best_R = R; best_cost = cost; best_smem = smem; }
+  for (int ng = 2; ng <= 4; ng += 2) {
+    for (int R = 1; R <= q.Ho; ++R) {
+      Mbv2Params t = q; int smem = 0;
+      set_groups(t, ng);
+      if (!layout(t, R, expand, project, &smem)) continue;
+      const long ctas = (long)q.N * t.strips;
+      const long waves = (ctas + sms - 1) / sms;
+      const double work = 0.8 * q.NC * (t.M1 * 128.0 + 3.0 * t.M2 * 128.0);
+      const double chain = 2900.0 * ((q.NC + ng - 1) / ng);
+      const double cost = (double)waves * (6000.0 + std::max(work, chain) + 0.01 * work);
+      if (best_R == 0 || cost < best_cost) { best_R = R; best_ng = ng; best_cost = cost; best_smem = smem; }
+    }
   }
   if (best_R == 0) return bad("no row-strip tiling fits shared memory / tensor memory");
+  set_groups(q, best_ng);
   layout(q, best_R, expand, project, &best_smem);
   if ((long)q.N * q.strips > 65535) return bad("more than 65535 row strips in the batch");
   host->smem_bytes = best_smem;
@@ -671,15 +689,20 @@ ago_status_t mbv2_plan(Plan* plan, FusedState* st, std::string* err) {
 
 namespace {
 
-template <bool EXPAND, bool PROJECT, bool FOLD>
-ago_status_t launch_variant(const Mbv2Params& q, int smem_bytes, cudaStream_t stream, std::string* err) {
+template <bool EXPAND, bool PROJECT, bool FOLD, int NG>
+ago_status_t launch_groups(const Mbv2Params& q, int smem_bytes, cudaStream_t stream, std::string* err) {
   static int smem_opt_in[64] = {};
-  cudaError_t e = ensure_max_dynamic_smem(reinterpret_cast<const void*>(mbv2_fused_kernel<EXPAND, PROJECT, FOLD>), smem_opt_in);
+  cudaError_t e = ensure_max_dynamic_smem(reinterpret_cast<const void*>(mbv2_fused_kernel<EXPAND, PROJECT, FOLD, NG>), smem_opt_in);
   if (e != cudaSuccess) { *err = std::string("cudaFuncSetAttribute: ") + cudaGetErrorString(e); return AGO_ERR_CUDA; }
   FusedLaunch launch(dim3((unsigned)(q.N * q.strips)), kThreads, (size_t)smem_bytes, stream);
-  e = cudaLaunchKernelEx(&launch.config, mbv2_fused_kernel<EXPAND, PROJECT, FOLD>, q);
+  e = cudaLaunchKernelEx(&launch.config, mbv2_fused_kernel<EXPAND, PROJECT, FOLD, NG>, q);
   if (e != cudaSuccess) { *err = std::string("fused inverted-residual launch: ") + cudaGetErrorString(e); return AGO_ERR_CUDA; }
   return AGO_OK;
+}
+template <bool EXPAND, bool PROJECT, bool FOLD>
+ago_status_t launch_variant(const Mbv2Params& q, int smem_bytes, cudaStream_t stream, std::string* err) {
+  return q.groups == 4 ? launch_groups<EXPAND, PROJECT, FOLD, 4>(q, smem_bytes, stream, err)
+                       : launch_groups<EXPAND, PROJECT, FOLD, 2>(q, smem_bytes, stream, err);
 }
 
 }  // namespace
