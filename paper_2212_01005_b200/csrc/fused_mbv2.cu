@@ -112,11 +112,11 @@ mbv2_fused_kernel(const Mbv2Params p) {
   float* sB3 = reinterpret_cast<float*>(smem + p.off_b3);
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + p.off_bar);
   uint64_t* bar_e = bars;           // [NG] expand accumulators of group g complete (MMA commit)
-  uint64_t* bar_d = bars + 4;       // [NG] project MMA has consumed D[g] (MMA commit)
-  uint64_t* bar_first = bars + 8;   // project GEMM of chunk 0 complete (it overwrites the output accumulators: the other groups issue after it)
-  uint64_t* bar_done = bars + 9;    // every project MMA complete (the groups do not follow each other's bar_d phases)
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 10);
-  volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(bars + 11);
+  uint64_t* bar_d = bars + 8;       // [NG] project MMA has consumed D[g] (MMA commit)
+  uint64_t* bar_first = bars + 16;  // project GEMM of chunk 0 complete (it overwrites the output accumulators: the other groups issue after it)
+  uint64_t* bar_done = bars + 17;   // every project MMA complete (the groups do not follow each other's bar_d phases)
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 18);
+  volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(bars + 19);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int n = (int)fast_div(blockIdx.x, (uint32_t)p.strips, p.strips_recip), strip = (int)blockIdx.x - n * p.strips;
@@ -386,7 +386,9 @@ mbv2_fused_kernel(const Mbv2Params p) {
     if (EXPAND && xi >= 0 && lane == 0 && g < p.NC) {
       // group 1 issues its first expand GEMM once group 0's is through the tensor pipe: group 0 has the longer chain
       // of chunks, and its first epilogue would otherwise wait for both groups' MMAs
-      if (g >= 1) mbar_wait(bar_e + g - 1, 0, abort_flag, p.status, 0x107);
+      // (with more than two groups the strips are small, the products short, and a chain of first products would cost
+      // more than it saves; a waiter that falls two phases behind a barrier would also read the wrong parity)
+      if (NG == 2 && g == 1) mbar_wait(bar_e, 0, abort_flag, p.status, 0x107);
       issue_expand();
     }
     __syncwarp();
@@ -608,7 +610,7 @@ bool layout(Mbv2Params& q, int R, bool expand, bool project, int* smem_bytes) {
   q.off_b1 = take(expand ? q.Cexp * 4 : 0);
   q.off_bd = take(q.Cexp * 4);
   q.off_b3 = take(project ? q.Coutp * 4 : 0);
-  q.off_bar = take(128);
+  q.off_bar = take(256);
   *smem_bytes = off + 1024;  // slack for the 1024-byte alignment of the base
   return *smem_bytes <= 227 * 1024;
 }
@@ -662,7 +664,7 @@ ago_status_t mbv2_plan(Plan* plan, FusedState* st, std::string* err) {
   // measured on 28 x 28 strips). Small strips therefore run with four groups, large ones with two.
   int best_R = 0, best_ng = 2; double best_cost = 0; int best_smem = 0;
   const int sms = device_sm_count();
-  for (int ng = 2; ng <= 4; ng += 2) {
+  for (int ng = 2; ng <= 8; ng *= 2) {
     for (int R = 1; R <= q.Ho; ++R) {
       Mbv2Params t = q; int smem = 0;
       set_groups(t, ng);
@@ -701,6 +703,7 @@ ago_status_t launch_groups(const Mbv2Params& q, int smem_bytes, cudaStream_t str
 }
 template <bool EXPAND, bool PROJECT, bool FOLD>
 ago_status_t launch_variant(const Mbv2Params& q, int smem_bytes, cudaStream_t stream, std::string* err) {
+  if (q.groups == 8) return launch_groups<EXPAND, PROJECT, FOLD, 8>(q, smem_bytes, stream, err);
   return q.groups == 4 ? launch_groups<EXPAND, PROJECT, FOLD, 4>(q, smem_bytes, stream, err)
                        : launch_groups<EXPAND, PROJECT, FOLD, 2>(q, smem_bytes, stream, err);
 }
