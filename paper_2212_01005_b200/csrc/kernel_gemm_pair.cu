@@ -16,7 +16,7 @@
 //   full[s]   leader only, count 1: the leader's TMA thread announces the bytes of both CTAs, both CTAs' loads complete there
 //   empty[s]  each CTA, count 1: the leader's MMA thread commits onto both after the stage's products
 //   accf[a]   each CTA, count 1: accumulator a complete (committed onto both CTAs by the leader)
-//   acce[a]   leader only, count 4: the two column halves of both CTAs have read accumulator a out of tensor memory
+//   acce[a]   leader only, count 3: its two epilogue groups and the peer (relayed by the peer's idle MMA warp) have read accumulator a
 #include <cuda.h>
 #include <cuda_bf16.h>
 
@@ -37,13 +37,13 @@ using namespace tc;
 
 constexpr int kPM = 128;                 // rows per CTA (256 per pair)
 constexpr int kPK = 64;                  // reduction elements per ring stage
-constexpr int kPStages = 6;
+constexpr int kPStages = 5;
 constexpr int kPStageBytes = 32 * 1024;  // A [128 x 64] + this CTA's half of B [<= 128 x 64]
-constexpr int kPStagingBytes = 16 * 1024;   // [128 rows x 128 bytes], one per column half
+constexpr int kPStagingBytes = 16 * 1024;   // [128 rows x 128 bytes]; two per group of epilogue warps (double-buffered)
 constexpr int kPEpiWarps = 8;            // (tensor-memory lane quarter) x (column half)
 constexpr int kPEpiThreads = kPEpiWarps * 32;
 constexpr int kPThreads = kPEpiThreads + 64;
-constexpr int kPSmemBytes = kPStages * kPStageBytes + 2 * kPStagingBytes + 256 + 1024;
+constexpr int kPSmemBytes = kPStages * kPStageBytes + 4 * kPStagingBytes + 256 + 1024;
 
 struct GemmPairParams {
   int M, N, K;
@@ -79,13 +79,14 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t* sRing = smem;
   uint8_t* sStage = smem + kPStages * kPStageBytes;
-  uint64_t* bars = reinterpret_cast<uint64_t*>(sStage + 2 * kPStagingBytes);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(sStage + 4 * kPStagingBytes);
   uint64_t* bar_full = bars;                   // [kPStages]
   uint64_t* bar_empty = bars + kPStages;       // [kPStages]
   uint64_t* bar_accf = bars + 2 * kPStages;    // [2]
   uint64_t* bar_acce = bar_accf + 2;           // [2]
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bar_acce + 2);
-  volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(bar_acce + 3);
+  uint64_t* bar_drain = bar_acce + 2;          // [2] peer only, count 2: both of its epilogue groups have read accumulator a
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bar_drain + 2);
+  volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(bar_drain + 3);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const uint32_t rank = cluster_ctarank();             // 0: leader
@@ -96,7 +97,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
   if (tid == kPEpiThreads) {
     *abort_flag = 0u;
     for (int i = 0; i < kPStages; ++i) { mbar_init(bar_full + i, 1); mbar_init(bar_empty + i, 1); }
-    for (int i = 0; i < 2; ++i) { mbar_init(bar_accf + i, 1); mbar_init(bar_acce + i, 4); }
+    for (int i = 0; i < 2; ++i) { mbar_init(bar_accf + i, 1); mbar_init(bar_acce + i, 3); mbar_init(bar_drain + i, 2); }
     fence_mbar_init();
     fence_proxy_async_smem();
   }
@@ -146,6 +147,17 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
     __syncwarp();
   } else if (warp == kPEpiWarps + 1) {
     // ================================ MMA issuer (leader CTA only) ================================
+    if (lane == 0 && rank != 0) {
+      // The peer's MMA warp has no products to issue: it relays "accumulator drained" to the leader. (An arrival on
+      // another CTA's barrier is a release at cluster scope, about a thousand cycles: kept off the epilogue warps.)
+      const uint32_t acce_leader = cluster_map(smem_u32(bar_acce), 0u);
+      int it = 0;
+      for (int t = pair; t < tiles; t += p.pairs, ++it) {
+        const int a = it & 1;
+        mbar_wait(bar_drain + a, (uint32_t)(it >> 1) & 1u, abort_flag, p.status, 0x605);
+        mbar_remote_arrive(acce_leader + (uint32_t)(a * 8));
+      }
+    }
     if (lane == 0 && rank == 0) {
       const uint32_t idesc = make_idesc_bf16(256, (uint32_t)p.BN, 0, p.b_kmajor ? 0 : 1);
       int s = 0, round = 0, it = 0;
@@ -184,24 +196,28 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
     const int row = q * 32 + lane;
     const uint32_t lane_base = (uint32_t)(q * 32) << 16;
     const int ht = tid & 127;                       // thread index within the column half
-    uint8_t* stage = sStage + h * kPStagingBytes;
+    uint8_t* stage0 = sStage + h * 2 * kPStagingBytes;
+    int sbuf = 0;                                   // staging buffer of the next block
     const int esz = p.c_fp32 ? 4 : 2;
     const int bc = 128 / esz;                       // columns per staged block (128 bytes per row)
-    const uint32_t acce_leader = cluster_map(smem_u32(bar_acce), 0u);
     int it = 0;
     for (int t = pair; t < tiles; t += p.pairs, ++it) {
       const int a = it & 1;
       const int tm = t % p.tiles_m, tn = t / p.tiles_m;
       const int row0 = tm * 2 * kPM + (int)rank * kPM;
-      const int col_t = tn * p.BN + h * half_n;     // first column of this half
+      const int col_t = tn * p.BN;                  // first column of the tile
       mbar_wait(bar_accf + a, (uint32_t)(it >> 1) & 1u, abort_flag, p.status, 0x604);
       tcgen05_fence_after_sync();
-      const uint32_t t_acc = tmem_base + lane_base + (uint32_t)(a * 256 + h * half_n);
-      for (int c0 = 0; c0 < half_n; c0 += bc) {
+      const uint32_t t_acc = tmem_base + lane_base + (uint32_t)(a * 256);
+      // the two groups of four warps take alternate blocks of 128 bytes of the tile's rows, so a narrow last tile
+      // (N = 144: blocks of 64, 64 and 16 columns) still splits between them
+      for (int c0 = h * bc; c0 < p.BN; c0 += 2 * bc) {
         const int col = col_t + c0;
-        if (col >= p.N) break;                      // uniform over the half: nothing of this block is stored
-        // the previous block's store has read the staging tile
-        if (ht == 0) bulk_wait_group_read_all();
+        if (col >= p.N) break;                      // uniform over the group: nothing of this block is stored
+        // the store that last used this staging buffer (two blocks ago) has read it; the previous block's may still be reading the other
+        uint8_t* stage = stage0 + sbuf * kPStagingBytes;
+        sbuf ^= 1;
+        if (ht == 0) bulk_wait_group_read_but_one();
         named_barrier_sync(1 + h, 128);
 #pragma unroll 1
         for (int j0 = 0; j0 < bc; j0 += 32) {
@@ -260,7 +276,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
       // this half's share of accumulator a is in registers / shared memory: hand it back to the MMA thread
       tcgen05_fence_before_sync();
       named_barrier_sync(1 + h, 128);
-      if (ht == 0) mbar_remote_arrive(acce_leader + (uint32_t)(a * 8));
+      if (ht == 0) mbar_arrive(rank == 0 ? bar_acce + a : bar_drain + a);   // the leader's MMA thread waits on bar_acce; the peer's goes through its relay
     }
     if (ht == 0) bulk_wait_group_all();             // the stores have left shared memory and are complete
   }
