@@ -12,27 +12,32 @@
 // is fetched as soon as the last score product of the old head has completed and the new V as soon as
 // its last P V has, both behind the softmax of the tiles in flight.
 //
-// The keys are processed in two halves by two independent groups of 384 threads (3 per query row and half).
+// The keys are processed in two halves by two independent groups of 128 threads (one thread per query row and half:
+// four warps per group, so every scheduler of the SM hosts one warp of each group and the MMA-issuing thread shares its
+// scheduler with two busy warps, not seven).
 // Each half is a softmax of its own -- its own row maximum, row sum and output accumulator P_h V_h in tensor
-// memory -- and the epilogue joins them: with m = max(m_0, m_1) and f_h = exp(m_h - m),
-// O = (f_0 O_0 + f_1 O_1) / (f_0 sum_0 + f_1 sum_1), the exact softmax over all keys. Nothing but the epilogue
-// orders the groups against each other, so they drift apart: while one group keeps the special-function
-// unit busy with its exponentials, the other waits for scores, reads tensor memory or exchanges maxima,
-// and the tensor core runs ahead on the next tile's scores.
+// memory -- and the epilogue joins them: with m_h the reference value of half h, m = max(m_0, m_1) and f_h = exp(m_h - m),
+// O = (f_0 O_0 + f_1 O_1) / (f_0 sum_0 + f_1 sum_1), the exact softmax over all keys. A thread owns its whole row of the
+// half, so neither pass exchanges anything with another thread; nothing but the epilogue orders the groups against
+// each other, so they drift apart: while one group keeps the special-function unit busy with its exponentials, the
+// other waits for scores or reads tensor memory, and the tensor core runs ahead on the next tile's scores.
 //
 //   P1  TMA: K, V [S x 64] once per head of the run, Q [128 x 64] per tile -> 128-byte-swizzled tiles
 //   P2  tcgen05.mma: S_h[128 x S/2] = Q K_h^T                            (TMEM, fp32, two buffers)
-//   P3/P4  per half 384 threads (3 per query row, <= 64 score columns each, read from tensor memory in chunks of 32:
-//       once for the row maximum, exchanged through shared memory, once more for
-//       p = exp2((s - m_h) * scale * log2 e) -> bf16 -> shared memory (K-major operand) and the row sum)
+//   P3/P4  per half 128 threads (a row each, read from tensor memory ONCE, in chunks of 32 columns through two register
+//       buffers -- the next chunk is in flight while the current one is consumed:
+//       p = exp2((s - m_h) * scale * log2 e) -> bf16 -> shared memory (K-major operand) and the row sum, with m_h the
+//       maximum of the row's first 32 scores. Softmax does not depend on the reference value; the true row maximum
+//       only keeps the exponentials in range, and a row sum that comes out too large (or not a number) sends the warp
+//       through the exact path: row maximum over all chunks first, then the probabilities again)
 //   P5  tcgen05.mma: O_h[128 x 64] = P_h V_h        (V is the N-major B operand, as it lies in HBM)
-//   P6  the group of half 1: TMEM -> registers, (f_0 O_0 + f_1 O_1) / sum, bf16 -> a swizzled tile in shared memory (the
-//       probability buffer of half 1, idle by then) -> one TMA store per tile (a row of one head is 128 bytes of a
-//       2 E-byte output row: stores from the row-per-lane accumulator layout would touch 32 lines per instruction)
+//   P6  four epilogue warps (a query row per thread): TMEM -> registers as soon as a half's product is complete (its
+//       accumulator is released at once), (f_0 O_0 + f_1 O_1) / sum, bf16 -> per warp, pieces of 16 columns x 32 rows
+//       staged in shared memory -> one TMA store per piece (stores from the row-per-lane register layout would touch
+//       32 lines per instruction and hold up the load/store unit that the probability stores need)
 //
-// Issue order of the MMA thread: when half 0's probabilities arrive, the next tile's half-0 scores go first (that
-// group has nothing else to do) and P_0 V second; when half 1's arrive, P_1 V goes first (the epilogue waits for
-// it) and the next half-1 scores second.
+// Issue order of the MMA thread: when a half's probabilities arrive, the next tile's scores of that half go first (its
+// group has nothing else to do) and P_h V second (only the epilogue warps wait for it).
 #include <cuda.h>
 #include <cuda_bf16.h>
 
@@ -52,11 +57,19 @@ using namespace tc;
 constexpr int kD = 64;                 // head dimension (one 128-byte swizzle row)
 constexpr int kBlockM = 128;           // query rows per tile
 constexpr int kKeyBlock = 128;         // keys per TMA box
-constexpr int kSubParts = 3;           // threads per query row and half (each owns <= 64 score columns: two chunks of 32)
-constexpr int kGroupThreads = kBlockM * kSubParts;
-constexpr int kComputeThreads = 2 * kGroupThreads;
-constexpr int kThreads = kComputeThreads + 64;   // + TMA warp + MMA warp
+constexpr int kGroupThreads = kBlockM;          // one thread per query row and half of the keys
+constexpr int kGroupWarps = kGroupThreads / 32;
+constexpr int kSoftmaxThreads = 2 * kGroupThreads;
+constexpr int kEpiWarp0 = kSoftmaxThreads / 32;  // four epilogue warps (a query row per thread) follow the softmax warps
+constexpr int kTmaWarp = kEpiWarp0 + 4;
+constexpr int kMmaWarp = kTmaWarp + 1;
+constexpr int kThreads = (kMmaWarp + 1) * 32;    // 448
 constexpr int kHalfCols = 192;         // tensor-memory columns reserved per score half
+constexpr int kMaxChunks = kHalfCols / 32;      // 32-column chunks of a row of one half
+// A row's exponentials are taken relative to the maximum of its first 32 scores, not of all of them (any reference gives
+// the same softmax; the true maximum only guarantees the range). A row sum at or above this limit, or not a number, sends
+// the warp through the exact two-pass path.
+constexpr float kSumLimit = 1099511627776.0f;   // 2^40
 constexpr uint32_t kOCol = 2 * kHalfCols;   // O_0 at kOCol, O_1 at kOCol + kD
 
 struct AttnParams {
@@ -68,9 +81,8 @@ struct AttnParams {
   int tiles;       // query tiles per head
   int total;       // items = B * heads * tiles
   int hw0, hw1;    // keys in half 0 / half 1 (multiples of 16, hw0 >= hw1 > 0)
-  int pw0, pw1;    // columns per thread in each half (multiples of 32, <= 64)
   float scale_log2e;
-  int off_q, off_k, off_v, off_p, off_red, off_bar;
+  int off_q, off_k, off_v, off_p, off_stage, off_red, off_bar;
   int p_half_bytes;
 };
 
@@ -80,6 +92,18 @@ __device__ __forceinline__ float ex2_approx(float x) {
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
+
+// Orders the compiler only: no use of these registers moves above this point, no later write to them above their last use.
+__device__ __forceinline__ void reg_order16(uint32_t (&v)[16]) {
+  asm volatile(""
+               : "+r"(v[0]), "+r"(v[1]), "+r"(v[2]), "+r"(v[3]), "+r"(v[4]), "+r"(v[5]), "+r"(v[6]), "+r"(v[7]), "+r"(v[8]),
+                 "+r"(v[9]), "+r"(v[10]), "+r"(v[11]), "+r"(v[12]), "+r"(v[13]), "+r"(v[14]), "+r"(v[15])
+               :
+               : "memory");
+}
+
+// Two probabilities -> a pair of bf16 (round to nearest even).
+__device__ __forceinline__ uint32_t pack_p(float e0, float e1) { return pack_bf16x2(e0, e1); }
 
 __global__ void __launch_bounds__(kThreads, 1)
 attention_fused_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
@@ -91,22 +115,19 @@ attention_fused_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
   uint8_t* sK = smem + p.off_k;
   uint8_t* sV = smem + p.off_v;
   uint8_t* sP = smem + p.off_p;                                // two halves of p_half_bytes
-  float* sMax = reinterpret_cast<float*>(smem + p.off_red);     // [half][tile parity][kSubParts][128]: partial row maxima
-  float* sSum = sMax + 2 * 2 * kSubParts * kBlockM;             // the same for the partial row sums
+  uint8_t* sStage = smem + p.off_stage;                        // per epilogue warp two [32 rows x 32 bytes] output pieces
+  float* sJoin = reinterpret_cast<float*>(smem + p.off_red);    // [tile parity][half][maximum, sum][128]: row statistics of the halves
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + p.off_bar);
   uint64_t* bar_k = bars + 0;
   uint64_t* bar_v = bars + 1;
   uint64_t* bar_q = bars + 2;       // Q tile landed
   uint64_t* bar_qfree = bars + 3;   // both score MMAs of the tile have read Q
   uint64_t* bar_s = bars + 4;       // [2] score half complete
-  uint64_t* bar_p = bars + 6;       // [2] probabilities of the half written, score half drained
+  uint64_t* bar_p = bars + 6;       // [2] probabilities of the half written, score half drained (one arrival per warp)
   uint64_t* bar_pfree = bars + 8;   // [2] P V of the half has read the probabilities
-  uint64_t* bar_o0 = bars + 10;     // P V of half 0 complete
-  uint64_t* bar_stage = bars + 11;  // output tile staged in shared memory
-  uint64_t* bar_o1 = bars + 12;     // P V of half 1 complete
-  uint64_t* bar_ofree = bars + 13;  // epilogue has read the output accumulators
+  uint64_t* bar_o = bars + 10;      // [2] P V of the half complete
+  uint64_t* bar_ofree = bars + 12;  // [2] the epilogue warps have read the half's output accumulator (one arrival per warp)
   uint64_t* bar_vfree = bars + 14;  // the last P V of a head has read V
-  uint64_t* bar_stfree = bars + 15; // the output store has read the staged tile
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 16);
   volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(bars + 17);
 
@@ -119,9 +140,9 @@ attention_fused_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
   grid_dependency_wait();      // the previous grid of the stream has completed; device memory may be touched
   grid_launch_dependents();
 
-  if (tid == kComputeThreads) {
+  if (tid == kTmaWarp * 32) {
     *abort_flag = 0u;
-    for (int i = 0; i < 16; ++i) mbar_init(bars + i, 1);
+    for (int i = 0; i < 16; ++i) mbar_init(bars + i, (i == 6 || i == 7 || i == 12 || i == 13) ? kGroupWarps : 1);
     fence_mbar_init();
     fence_proxy_async_smem();
     tma_prefetch_desc(&tmap_q);
@@ -144,7 +165,7 @@ attention_fused_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
   tcgen05_fence_after_sync();
   const uint32_t tmem_base = *tmem_slot;
 
-  if (warp == kComputeThreads / 32) {
+  if (warp == kTmaWarp) {
     // ============================ TMA producer: the remaining Q tiles, K and V of the following heads ============================
     if (lane == 0) {
       int t = t0, h = h0, b = b0;
@@ -168,7 +189,7 @@ attention_fused_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
       }
     }
     __syncwarp();
-  } else if (warp == kComputeThreads / 32 + 1) {
+  } else if (warp == kMmaWarp) {
     // ============================ MMA issue (one lane) ============================
     if (lane == 0) {
       const uint64_t qdesc = make_smem_desc(smem_u32(sQ), 0, 1024, SW_128B);
@@ -222,300 +243,241 @@ attention_fused_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
           issue_scores(0);                       // next tile's half 0 into the buffer just drained: its group is waiting for it
         }
         if (first_of_head) mbar_wait(bar_v, head_ph, abort_flag, p.status, 0x205);
-        if (i > 0) mbar_wait(bar_ofree, ph ^ 1u, abort_flag, p.status, 0x206);
+        if (i > 0) mbar_wait(bar_ofree + 0, ph ^ 1u, abort_flag, p.status, 0x206);
         tcgen05_fence_after_sync();
         issue_pv(0);
-        umma_commit(bar_o0);
+        umma_commit(bar_o + 0);
         umma_commit(bar_pfree + 0);
         // ---- half 1 ----
         mbar_wait(bar_p + 1, ph, abort_flag, p.status, 0x208);
         tcgen05_fence_after_sync();
-        issue_pv(1);                             // first: the epilogue of this tile waits for it
-        umma_commit(bar_o1);
-        umma_commit(bar_pfree + 1);
-        if (last_of_head) umma_commit(bar_vfree);
         if (i + 1 < n) {
           issue_scores(1);
           umma_commit(bar_qfree);
         }
+        if (i > 0) mbar_wait(bar_ofree + 1, ph ^ 1u, abort_flag, p.status, 0x209);
+        tcgen05_fence_after_sync();
+        issue_pv(1);
+        umma_commit(bar_o + 1);
+        umma_commit(bar_pfree + 1);
+        if (last_of_head) umma_commit(bar_vfree);
         first_of_head = last_of_head;
         if (last_of_head) { t = 0; head_ph ^= 1u; } else ++t;
       }
     }
     __syncwarp();
-  } else {
-    // ============================ softmax / epilogue warps ============================
+  } else if (warp < kEpiWarp0) {
+    // ============================ softmax warps ============================
+    const int grp = warp >> 2;                  // the half of the keys this thread's group owns (warps 0-3 / 4-7)
     const int row = (warp & 3) * 32 + lane;     // TMEM lane = query row of the tile
-    const int part = warp >> 2;
-    const int grp = part >= kSubParts ? 1 : 0;  // the half of the keys this thread's group owns
-    const int sub = part - grp * kSubParts;     // which slice of the half
     const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
     const float c = p.scale_log2e;
     const int hw = grp ? p.hw1 : p.hw0;
-    const int pw = grp ? p.pw1 : p.pw0;
-    const int nch = pw >> 5;                    // chunks of 32 columns per thread
     const int key_base = grp * p.hw0;
+    const int kv = min(hw, p.S - key_base);     // real keys of the half (> hw - 16; the other columns are padding)
+    const int nch = (hw + 31) >> 5;             // 32-column chunks that hold columns of the half
     const uint32_t s_addr = tmem_base + lane_base + grp * kHalfCols;
     uint8_t* pbase = sP + grp * p.p_half_bytes;
-    const uint32_t bar_id = 1u + (uint32_t)grp;
-    const bool leader = sub == 0 && row == 0;
-    float* gMax = sMax + grp * (2 * kSubParts * kBlockM);
-    float* gSum = sSum + grp * (2 * kSubParts * kBlockM);
+    uint8_t* prow = pbase + row * 128;          // this row in the first 64-key block of the probability operand
+    const uint32_t sw = (uint32_t)row & 7u;
 
-    uint32_t sv[32];
-    // One chunk of (at most) 32 score columns of this thread's row: col0 within the half, ncols in {0, 16, 32};
-    // fast = all 32 present and none of them padding: straight-line code, no predicates.
-    auto load_chunk = [&](int col0, int ncols) {
-      if (ncols > 16) tmem_ld_x32(s_addr + col0, sv); else tmem_ld_x16(s_addr + col0, sv);
-      tmem_ld_wait();
+    uint32_t va[32], vb[32];
+    // The outstanding load of a 32-register buffer has landed (one wait; the second statement only orders the compiler).
+    auto wait32 = [](uint32_t (&v)[32]) {
+      tmem_ld_wait_on(reinterpret_cast<uint32_t (&)[16]>(v[0]));
+      reg_order16(reinterpret_cast<uint32_t (&)[16]>(v[16]));
     };
-    auto chunk_max = [&](int col0, int ncols, bool fast) -> float {
-      float m = -INFINITY;
-      if (fast) {
-        float m4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
-#pragma unroll
-        for (int j = 0; j < 32; j += 4) {
-          m4[0] = fmaxf(m4[0], __uint_as_float(sv[j]));
-          m4[1] = fmaxf(m4[1], __uint_as_float(sv[j + 1]));
-          m4[2] = fmaxf(m4[2], __uint_as_float(sv[j + 2]));
-          m4[3] = fmaxf(m4[3], __uint_as_float(sv[j + 3]));
-        }
-        m = fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3]));
-      } else {
-        const int key0 = key_base + col0;
-#pragma unroll
-        for (int j = 0; j < 32; ++j) if (j < ncols && key0 + j < p.S) m = fmaxf(m, __uint_as_float(sv[j]));
-      }
-      return m;
+    auto wait_order32 = [](uint32_t (&v)[32]) {   // after a wait32 that covered this buffer's load as well
+      reg_order16(reinterpret_cast<uint32_t (&)[16]>(v[0]));
+      reg_order16(reinterpret_cast<uint32_t (&)[16]>(v[16]));
     };
-    auto chunk_exp = [&](int col0, int ncols, bool fast, float mc) -> float {
-      float sum = 0.0f;
-      if (fast) {
-        // 32 columns = four 16-byte chunks of this row inside one 64-key block (col0 is a multiple of 32)
-        uint8_t* rowp = pbase + (col0 >> 6) * (kBlockM * 128) + row * 128;
-        const uint32_t ch0 = (uint32_t)(col0 & 63) >> 3, sw = (uint32_t)row & 7u;
-        float s4[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-        for (int g = 0; g < 4; ++g) {
-          uint32_t w[4];
-#pragma unroll
-          for (int j = 0; j < 4; ++j) {
-            const float e0 = ex2_approx(fmaf(__uint_as_float(sv[g * 8 + 2 * j]), c, -mc));
-            const float e1 = ex2_approx(fmaf(__uint_as_float(sv[g * 8 + 2 * j + 1]), c, -mc));
-            s4[j] += e0 + e1;
-            w[j] = pack_bf16x2(e0, e1);
-          }
-          *reinterpret_cast<uint4*>(rowp + (((ch0 + g) ^ sw) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
-        }
-        sum = (s4[0] + s4[1]) + (s4[2] + s4[3]);
-      } else {
-        const int key0 = key_base + col0;
-#pragma unroll
-        for (int g = 0; g < 4; ++g) {            // 8 columns = one 16-byte chunk of a probability row
-          if (g * 8 < ncols) {
-            uint32_t w[4];
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-              const int e = g * 8 + 2 * j;
-              float e0 = ex2_approx(fmaf(__uint_as_float(sv[e]), c, -mc));
-              float e1 = ex2_approx(fmaf(__uint_as_float(sv[e + 1]), c, -mc));
-              if (key0 + e >= p.S) e0 = 0.0f;
-              if (key0 + e + 1 >= p.S) e1 = 0.0f;
-              sum += e0 + e1;
-              w[j] = pack_bf16x2(e0, e1);
-            }
-            const int cc = col0 + g * 8;
-            *reinterpret_cast<uint4*>(pbase + (cc >> 6) * (kBlockM * 128) + swz_offset(row, (uint32_t)(cc & 63) >> 3, 128)) =
-                make_uint4(w[0], w[1], w[2], w[3]);
-          }
-        }
-      }
-      return sum;
-    };
-    auto reduce3 = [&](const float* a, bool is_max) -> float {
-      const float x = a[row], y = a[kBlockM + row], z = a[2 * kBlockM + row];
-      return is_max ? fmaxf(x, fmaxf(y, z)) : x + y + z;
-    };
-
-    // Threads whose 64 columns are all present and real keys read them in four pieces of 16 through two register
-    // buffers: the load of the next piece is in flight while the current one is consumed.
-    const bool piped = pw == 64 && sub * pw + 64 <= hw && key_base + sub * pw + 64 <= p.S;
-    const uint32_t c_addr = s_addr + (uint32_t)(sub * pw);
-    auto max16 = [&](const uint32_t (&v)[16]) -> float {
+    auto max32 = [](const uint32_t (&v)[32]) -> float {
       float m4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
-      for (int j = 0; j < 16; j += 4) {
-        m4[0] = fmaxf(m4[0], __uint_as_float(v[j]));
-        m4[1] = fmaxf(m4[1], __uint_as_float(v[j + 1]));
-        m4[2] = fmaxf(m4[2], __uint_as_float(v[j + 2]));
-        m4[3] = fmaxf(m4[3], __uint_as_float(v[j + 3]));
+      for (int j = 0; j < 32; j += 8) {
+        m4[0] = fmaxf(m4[0], fmaxf(__uint_as_float(v[j]), __uint_as_float(v[j + 1])));
+        m4[1] = fmaxf(m4[1], fmaxf(__uint_as_float(v[j + 2]), __uint_as_float(v[j + 3])));
+        m4[2] = fmaxf(m4[2], fmaxf(__uint_as_float(v[j + 4]), __uint_as_float(v[j + 5])));
+        m4[3] = fmaxf(m4[3], fmaxf(__uint_as_float(v[j + 6]), __uint_as_float(v[j + 7])));
       }
       return fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3]));
     };
-    // 16 columns (piece q of the thread's 64) -> two 16-byte chunks of the probability row; returns their sum
-    auto exp16 = [&](const uint32_t (&v)[16], int q, float mc) -> float {
-      const int col = sub * 64 + q * 16;
-      uint8_t* rowp = pbase + (col >> 6) * (kBlockM * 128) + row * 128;
-      const uint32_t ch0 = (uint32_t)(col & 63) >> 3, sw = (uint32_t)row & 7u;
-      float s2[2] = {0.f, 0.f};
+    auto max_tail = [](const uint32_t (&v)[32], int nreal) -> float {
+      float m = -INFINITY;
 #pragma unroll
-      for (int g = 0; g < 2; ++g) {
+      for (int j = 0; j < 32; ++j) if (j < nreal) m = fmaxf(m, __uint_as_float(v[j]));
+      return m;
+    };
+    // 32 columns of real keys -> four 16-byte chunks of the probability row; s4 collects the row sum. All 32 exponentials
+    // are issued back to back, in place, before anything consumes one: the special-function unit takes a warp's
+    // instruction every eight cycles, and only independent ones in flight keep it busy from a single warp.
+    auto exp32 = [&](uint32_t (&v)[32], uint8_t* blk, uint32_t ch0, float mc, float (&s4)[4]) {
+#pragma unroll
+      for (int j = 0; j < 32; ++j) v[j] = __float_as_uint(ex2_approx(fmaf(__uint_as_float(v[j]), c, -mc)));
+#pragma unroll
+      for (int g = 0; g < 4; ++g) {
         uint32_t w[4];
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
-          const float e0 = ex2_approx(fmaf(__uint_as_float(v[g * 8 + 2 * j]), c, -mc));
-          const float e1 = ex2_approx(fmaf(__uint_as_float(v[g * 8 + 2 * j + 1]), c, -mc));
-          s2[j & 1] += e0 + e1;
-          w[j] = pack_bf16x2(e0, e1);
+          const float e0 = __uint_as_float(v[g * 8 + 2 * j]), e1 = __uint_as_float(v[g * 8 + 2 * j + 1]);
+          s4[j] += e0 + e1;
+          w[j] = pack_p(e0, e1);
         }
-        *reinterpret_cast<uint4*>(rowp + (((ch0 + g) ^ sw) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
+        *reinterpret_cast<uint4*>(blk + (((ch0 + g) ^ sw) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
       }
-      return s2[0] + s2[1];
+    };
+    // The last chunk of a half: ncols (16 or 32) columns belong to the half, the first nreal of them are keys; the
+    // probabilities of the padding columns are zeros (their V rows are zeros too, but must not meet a NaN).
+    auto exp_tail = [&](uint32_t (&v)[32], uint8_t* blk, uint32_t ch0, int ncols, int nreal, float mc, float (&s4)[4]) {
+#pragma unroll
+      for (int g = 0; g < 4; ++g) {
+        if (g * 8 < ncols) {
+          uint32_t w[4];
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            const int e = g * 8 + 2 * j;
+            float e0 = ex2_approx(fmaf(__uint_as_float(v[e]), c, -mc));
+            float e1 = ex2_approx(fmaf(__uint_as_float(v[e + 1]), c, -mc));
+            if (e >= nreal) e0 = 0.0f;
+            if (e + 1 >= nreal) e1 = 0.0f;
+            s4[j] += e0 + e1;
+            w[j] = pack_p(e0, e1);
+          }
+          *reinterpret_cast<uint4*>(blk + (((ch0 + g) ^ sw) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
+        }
+      }
     };
 
     for (int t = 0; t < n; ++t) {               // t: position of the item in this CTA's run
       const uint32_t ph = (uint32_t)t & 1u;
-      float* myMax = gMax + ph * (kSubParts * kBlockM);
-      float* mySum = gSum + ph * (kSubParts * kBlockM);
-      // ---------------- pass 1: row maximum of this half ----------------
+      float* xm = sJoin + (ph * 2 + grp) * (2 * kBlockM);   // this half's row maxima and sums of the tile, for the epilogue
+      // ---------------- reference value: maximum of the first chunk ----------------
       mbar_wait(bar_s + grp, ph, abort_flag, p.status, 0x210);
       tcgen05_fence_after_sync();
-      float m = -INFINITY;
-      if (piped) {
-        uint32_t (&va)[16] = reinterpret_cast<uint32_t (&)[16]>(sv[0]);
-        uint32_t (&vb)[16] = reinterpret_cast<uint32_t (&)[16]>(sv[16]);
-        tmem_ld_x16(c_addr, va);
-        tmem_ld_wait_on(va);
-        tmem_ld_x16(c_addr + 16, vb);
-        m = max16(va);
-        tmem_ld_wait_on(vb);
-        tmem_ld_x16(c_addr + 32, va);
-        m = fmaxf(m, max16(vb));
-        tmem_ld_wait_on(va);
-        tmem_ld_x16(c_addr + 48, vb);
-        m = fmaxf(m, max16(va));
-        tmem_ld_wait_on(vb);
-        m = fmaxf(m, max16(vb));
-      } else {
-        for (int ch = 0; ch < nch; ++ch) {
-          const int col0 = sub * pw + ch * 32;
-          const int ncols = max(0, min(hw, col0 + 32) - col0);
-          if (ncols > 0) {
-            load_chunk(col0, ncols);
-            m = fmaxf(m, chunk_max(col0, ncols, ncols == 32 && key_base + col0 + 32 <= p.S));
+      tmem_ld_x32(s_addr, va);
+      if (t > 0) {                               // P V of the previous tile has read this half's probability buffer
+        if (lane == 0) mbar_wait(bar_pfree + grp, ph ^ 1u, abort_flag, p.status, 0x211);
+        __syncwarp();
+      }
+      wait32(va);
+      if (nch > 1) tmem_ld_x32(s_addr + 32u, vb);
+      float m = kv >= 32 ? max32(va) : max_tail(va, kv);
+      float sum;
+      // The loops below are rolled on purpose: every softmax warp runs the same few hundred instructions per pair of
+      // chunks, which stay in the instruction cache, instead of a private stretch of straight-line code per chunk.
+#pragma unroll 1
+      for (int attempt = 0;; ++attempt) {
+        // ---------------- probabilities and row sum (chunk 0 is in va, chunk 1 on its way to vb) ----------------
+        const float mc = m * c;
+        float s4[4] = {0.f, 0.f, 0.f, 0.f};
+        uint8_t* blk = prow;
+#pragma unroll 1
+        for (int ch = 0; ch < nch; ch += 2, blk += kBlockM * 128) {
+          if (kv - ch * 32 >= 32) exp32(va, blk, 0u, mc, s4); else exp_tail(va, blk, 0u, hw - ch * 32, kv - ch * 32, mc, s4);
+          if (ch + 1 < nch) {
+            wait32(vb);
+            if (ch + 2 < nch) tmem_ld_x32(s_addr + (uint32_t)((ch + 2) * 32), va);
+            if (kv - ch * 32 >= 64) exp32(vb, blk, 4u, mc, s4); else exp_tail(vb, blk, 4u, hw - ch * 32 - 32, kv - ch * 32 - 32, mc, s4);
+            if (ch + 2 < nch) {
+              wait32(va);
+              if (ch + 3 < nch) tmem_ld_x32(s_addr + (uint32_t)((ch + 3) * 32), vb);
+            }
           }
         }
-      }
-      myMax[sub * kBlockM + row] = m;
-      if (leader && t > 0) {
-        mbar_wait(bar_pfree + grp, ph ^ 1u, abort_flag, p.status, 0x211);       // P V of the previous tile has read this half's probabilities
-        if (grp == 1) bulk_wait_group_read_all();       // and this thread's output store has read its staged tile (same buffer)
-      }
-      named_barrier_sync(bar_id, kGroupThreads);
-      const float mh = reduce3(myMax, true);
-      // ---------------- pass 2: probabilities and row sum ----------------
-      float sum = 0.0f;
-      if (piped) {
-        const float mc = mh * c;
-        uint32_t (&va)[16] = reinterpret_cast<uint32_t (&)[16]>(sv[0]);
-        uint32_t (&vb)[16] = reinterpret_cast<uint32_t (&)[16]>(sv[16]);
-        tmem_ld_x16(c_addr, va);
-        tmem_ld_wait_on(va);
-        tmem_ld_x16(c_addr + 16, vb);
-        sum = exp16(va, 0, mc);
-        tmem_ld_wait_on(vb);
-        tmem_ld_x16(c_addr + 32, va);
-        sum += exp16(vb, 1, mc);
-        tmem_ld_wait_on(va);
-        tmem_ld_x16(c_addr + 48, vb);
-        sum += exp16(va, 2, mc);
-        tmem_ld_wait_on(vb);
-        sum += exp16(vb, 3, mc);
-      } else {
+        sum = (s4[0] + s4[1]) + (s4[2] + s4[3]);
+        if (attempt == 1 || !__any_sync(0xffffffffu, !(sum < kSumLimit))) break;
+        // ---------------- exact path: the row maximum over all chunks first ----------------
+        m = -INFINITY;
+#pragma unroll 1
         for (int ch = 0; ch < nch; ++ch) {
-          const int col0 = sub * pw + ch * 32;
-          const int ncols = max(0, min(hw, col0 + 32) - col0);
-          if (ncols > 0) {
-            load_chunk(col0, ncols);
-            sum += chunk_exp(col0, ncols, ncols == 32 && key_base + col0 + 32 <= p.S, mh * c);
-          }
+          tmem_ld_x32(s_addr + (uint32_t)(ch * 32), va);
+          wait32(va);
+          m = fmaxf(m, kv - ch * 32 >= 32 ? max32(va) : max_tail(va, kv - ch * 32));
         }
+        tmem_ld_x32(s_addr, va);
+        wait32(va);
+        if (nch > 1) tmem_ld_x32(s_addr + 32u, vb);
       }
-      mySum[sub * kBlockM + row] = sum;
+      xm[row] = m;
+      xm[kBlockM + row] = sum;
       fence_proxy_async_smem();
       tcgen05_fence_before_sync();
-      named_barrier_sync(bar_id, kGroupThreads);
-      if (leader) mbar_arrive(bar_p + grp);      // probabilities written, score half drained
-
-      if (grp == 1) {
-        // ---------------- epilogue of the tile: join the halves, normalise, stage, store ----------------
-        // Half 0's product, maxima and sums are long complete (bar_o0 follows that group's barriers and its arrival on
-        // bar_p[0]): the weights and the f_0 O_0 terms are computed while the tensor core still works on P_1 V.
-        mbar_wait(bar_o0, ph, abort_flag, p.status, 0x214);
-        tcgen05_fence_after_sync();
-        uint32_t (&oa)[16] = reinterpret_cast<uint32_t (&)[16]>(sv[0]);
-        uint32_t (&ob)[16] = reinterpret_cast<uint32_t (&)[16]>(sv[16]);
-        const uint32_t o_addr = tmem_base + lane_base + kOCol + sub * 32;
-        float f1 = 0.0f;
-        if (sub < 2) {                           // 32 of the 64 output columns each
-          tmem_ld_x16(o_addr, oa);
-          tmem_ld_x16(o_addr + 16, ob);
-          const float m0 = reduce3(sMax + ph * (kSubParts * kBlockM), true);
-          const float s0 = reduce3(sSum + ph * (kSubParts * kBlockM), false);
-          const float s1 = reduce3(mySum, false);
-          const float mm = fmaxf(m0, mh);
-          float f0 = ex2_approx((m0 - mm) * c);
-          f1 = ex2_approx((mh - mm) * c);
-          const float inv = 1.0f / (f0 * s0 + f1 * s1);
-          f0 *= inv; f1 *= inv;
-          tmem_ld_wait_on(oa);
-          tmem_ld_wait_on(ob);
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar_p + grp);   // this warp's 32 rows of probabilities written, its score rows drained
+    }
+  } else {
+    // ============================ epilogue warps: join the halves, normalise, store ============================
+    // A thread owns a query row of the tile: 64 output values.
+    const int row = (warp & 3) * 32 + lane;     // TMEM lane = query row of the tile
+    const uint32_t o_addr = tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + kOCol;
+    const float c = p.scale_log2e;
+    uint32_t oa[32], ob[32], oc[16];
+    uint8_t* stage = sStage + (warp & 3) * 2048;
+    auto wait32 = [](uint32_t (&v)[32]) {
+      tmem_ld_wait_on(reinterpret_cast<uint32_t (&)[16]>(v[0]));
+      reg_order16(reinterpret_cast<uint32_t (&)[16]>(v[16]));
+    };
+    int u = g0 / p.tiles, tq = g0 - u * p.tiles;
+    for (int t = 0; t < n; ++t) {
+      const uint32_t ph = (uint32_t)t & 1u;
+      // Half 0's product is complete long before half 1's: it is read, and its accumulator released, at once.
+      mbar_wait(bar_o + 0, ph, abort_flag, p.status, 0x214);
+      tcgen05_fence_after_sync();
+      tmem_ld_x32(o_addr, oa);
+      tmem_ld_x32(o_addr + 32, ob);
+      wait32(oa);
+      reg_order16(reinterpret_cast<uint32_t (&)[16]>(ob[0]));
+      reg_order16(reinterpret_cast<uint32_t (&)[16]>(ob[16]));
+      tcgen05_fence_before_sync();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar_ofree + 0);            // O_0 is in registers: the next tile's P_0 V may overwrite it
+      const int b = u / p.heads;
+      mbar_wait(bar_o + 1, ph, abort_flag, p.status, 0x215);
+      tcgen05_fence_after_sync();
+      // Both groups' row statistics of this tile were written before their arrivals on bar_p, which the products follow.
+      const float* xm = sJoin + ph * (4 * kBlockM);
+      const float m0 = xm[row], s0 = xm[kBlockM + row], m1 = xm[2 * kBlockM + row], s1 = xm[3 * kBlockM + row];
+      const float mm = fmaxf(m0, m1);
+      float f0 = ex2_approx((m0 - mm) * c);
+      float f1 = ex2_approx((m1 - mm) * c);
+      const float inv = 1.0f / (f0 * s0 + f1 * s1);
+      f0 *= inv; f1 *= inv;
+      // Four pieces of 16 output columns: 32 bytes of each of the warp's 32 rows, staged (32-byte swizzle: rows four apart
+      // take the other 16-byte slot) and written by one TMA store per piece, which clips the rows past S. Stores from the
+      // row-per-lane register layout would touch 32 lines per instruction and hold up the load/store unit for everyone.
 #pragma unroll
-          for (int j = 0; j < 16; ++j) {
-            oa[j] = __float_as_uint(__uint_as_float(oa[j]) * f0);
-            ob[j] = __float_as_uint(__uint_as_float(ob[j]) * f0);
-          }
+      for (int q = 0; q < 4; ++q) {
+        tmem_ld_x16(o_addr + kD + (uint32_t)(q * 16), oc);
+        if (lane == 0) bulk_wait_group_read_but_one();       // the store issued two pieces ago has read this buffer
+        tmem_ld_wait_on(oc);
+        if (q == 3) {
+          tcgen05_fence_before_sync();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(bar_ofree + 1);        // O_1 is in registers
+        } else {
+          __syncwarp();
         }
-        mbar_wait(bar_o1, ph, abort_flag, p.status, 0x215);
-        tcgen05_fence_after_sync();
-        if (sub < 2) {
-          uint8_t* stage = pbase;                // P V of half 1 has completed: its probabilities are dead
-          uint32_t oc[16];
-          tmem_ld_x16(o_addr + kD, oc);
-          tmem_ld_wait_on(oc);
+        const uint32_t* o0 = q < 2 ? oa + q * 16 : ob + (q - 2) * 16;
 #pragma unroll
-          for (int j = 0; j < 16; ++j) oa[j] = __float_as_uint(fmaf(__uint_as_float(oc[j]), f1, __uint_as_float(oa[j])));
-          tmem_ld_x16(o_addr + kD + 16, oc);     // in flight while the first 16 columns are packed and staged
+        for (int j = 0; j < 16; ++j) oc[j] = __float_as_uint(fmaf(__uint_as_float(oc[j]), f1, __uint_as_float(o0[j]) * f0));
+        uint8_t* piece = stage + (q & 1) * 1024;
 #pragma unroll
-          for (int j = 0; j < 2; ++j)
-            *reinterpret_cast<uint4*>(stage + swz_offset(row, (uint32_t)(sub * 4 + j), 128)) =
-                make_uint4(pack_bf16x2(__uint_as_float(oa[8 * j]), __uint_as_float(oa[8 * j + 1])),
-                           pack_bf16x2(__uint_as_float(oa[8 * j + 2]), __uint_as_float(oa[8 * j + 3])),
-                           pack_bf16x2(__uint_as_float(oa[8 * j + 4]), __uint_as_float(oa[8 * j + 5])),
-                           pack_bf16x2(__uint_as_float(oa[8 * j + 6]), __uint_as_float(oa[8 * j + 7])));
-          tmem_ld_wait_on(oc);
-#pragma unroll
-          for (int j = 0; j < 16; ++j) ob[j] = __float_as_uint(fmaf(__uint_as_float(oc[j]), f1, __uint_as_float(ob[j])));
-#pragma unroll
-          for (int j = 0; j < 2; ++j)
-            *reinterpret_cast<uint4*>(stage + swz_offset(row, (uint32_t)(sub * 4 + 2 + j), 128)) =
-                make_uint4(pack_bf16x2(__uint_as_float(ob[8 * j]), __uint_as_float(ob[8 * j + 1])),
-                           pack_bf16x2(__uint_as_float(ob[8 * j + 2]), __uint_as_float(ob[8 * j + 3])),
-                           pack_bf16x2(__uint_as_float(ob[8 * j + 4]), __uint_as_float(ob[8 * j + 5])),
-                           pack_bf16x2(__uint_as_float(ob[8 * j + 6]), __uint_as_float(ob[8 * j + 7])));
-        }
+        for (int j = 0; j < 2; ++j)
+          *reinterpret_cast<uint4*>(piece + lane * 32 + ((((uint32_t)j) ^ (((uint32_t)lane >> 2) & 1u)) << 4)) =
+              make_uint4(pack_bf16x2(__uint_as_float(oc[8 * j]), __uint_as_float(oc[8 * j + 1])),
+                         pack_bf16x2(__uint_as_float(oc[8 * j + 2]), __uint_as_float(oc[8 * j + 3])),
+                         pack_bf16x2(__uint_as_float(oc[8 * j + 4]), __uint_as_float(oc[8 * j + 5])),
+                         pack_bf16x2(__uint_as_float(oc[8 * j + 6]), __uint_as_float(oc[8 * j + 7])));
         fence_proxy_async_smem();
-        tcgen05_fence_before_sync();
-        named_barrier_sync(bar_id, kGroupThreads);
-        if (leader) {
-          mbar_arrive(bar_ofree);
-          const int u = (g0 + t) / p.tiles, tq = g0 + t - u * p.tiles, b = u / p.heads;
-          tma_store_3d(&tmap_o, pbase, (u - b * p.heads) * kD, tq * kBlockM, b);   // rows past S are clipped
+        __syncwarp();
+        if (lane == 0) {
+          tma_store_3d(&tmap_o, piece, (u - b * p.heads) * kD + q * 16, tq * kBlockM + (warp & 3) * 32, b);
           bulk_commit_group();
         }
       }
+      if (++tq == p.tiles) { tq = 0; ++u; }
     }
-    if (leader && grp == 1) bulk_wait_group_all();
+    if (lane == 0) bulk_wait_group_all();
   }
   tcgen05_fence_before_sync();
   __syncthreads();
@@ -525,7 +487,7 @@ attention_fused_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
 struct AttnHost {
   AttnParams prm;
   int smem_bytes = 0;
-  std::unordered_map<const void*, CUtensorMap> maps;   // keyed by base pointer (box shape is the same for Q, K, V)
+  std::unordered_map<const void*, CUtensorMap> maps;   // keyed by base pointer (+1 for the output map)
 };
 
 int round16(int v) { return (v + 15) / 16 * 16; }
@@ -551,8 +513,6 @@ ago_status_t attention_plan(Plan* plan, FusedState* st, std::string* err) {
   q.total = q.B * q.heads * q.tiles;
   q.hw0 = round16((q.Spad + 1) / 2);
   q.hw1 = q.Spad - q.hw0;
-  q.pw0 = ((q.hw0 + kSubParts - 1) / kSubParts + 31) / 32 * 32;
-  q.pw1 = ((q.hw1 + kSubParts - 1) / kSubParts + 31) / 32 * 32;
   q.scale_log2e = plan->ops[1].op.f * 1.4426950408889634f;
   int off = 0;
   auto take = [&](int bytes) { int o = off; off = (off + bytes + 1023) / 1024 * 1024; return o; };
@@ -561,7 +521,8 @@ ago_status_t attention_plan(Plan* plan, FusedState* st, std::string* err) {
   q.off_v = take(q.nkb * kKeyBlock * kD * 2);
   q.p_half_bytes = ((q.hw0 + 63) / 64) * kBlockM * 128;
   q.off_p = take(2 * q.p_half_bytes);
-  q.off_red = take(2 * 2 * 2 * kSubParts * kBlockM * 4);
+  q.off_stage = take(4 * 2 * 1024);
+  q.off_red = take(2 * 2 * 2 * kBlockM * 4);
   q.off_bar = take(256);
   host->smem_bytes = off + 1024;
   if (host->smem_bytes > 227 * 1024) return bad("shared memory budget exceeded");
@@ -581,19 +542,22 @@ ago_status_t attention_run(const Plan& plan, FusedState* st, const void* const* 
   const CUtensorMap* maps[4];
   for (int i = 0; i < 4; ++i) {
     const void* base = i < 3 ? inputs[i] : output;
-    auto it = host->maps.find(base);
+    // keyed by pointer and role: the output map has another box and swizzle than the input maps
+    const void* key = reinterpret_cast<const void*>(reinterpret_cast<uintptr_t>(base) | (i == 3 ? 1u : 0u));
+    auto it = host->maps.find(key);
     if (it == host->maps.end()) {
       CUtensorMap m;
       const uint64_t dims[3] = {(uint64_t)q.E, (uint64_t)q.S, (uint64_t)q.B};
       const uint64_t strides[2] = {(uint64_t)q.E * 2, (uint64_t)q.S * q.E * 2};
       const uint32_t box[3] = {(uint32_t)kD, (uint32_t)kKeyBlock, 1};
-      if (!encode_tmap_bf16(&m, base, 3, dims, strides, box, 128, err)) return AGO_ERR_CUDA;
+      const uint32_t obox[3] = {16, 32, 1};        // an epilogue warp's piece: 16 columns of its 32 rows
+      if (!encode_tmap_bf16(&m, base, 3, dims, strides, i < 3 ? box : obox, i < 3 ? 128 : 32, err)) return AGO_ERR_CUDA;
       if (host->maps.size() > 4096) {     // pointers already fetched stay valid: unordered_map keeps its nodes until erased
         host->maps.clear();
         i = -1;
         continue;
       }
-      it = host->maps.emplace(base, m).first;
+      it = host->maps.emplace(key, m).first;
     }
     maps[i] = &it->second;
   }
