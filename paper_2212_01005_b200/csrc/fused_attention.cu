@@ -29,7 +29,8 @@
 //       p = exp2((s - m_h) * scale * log2 e) -> bf16 -> shared memory (K-major operand) and the row sum, with m_h the
 //       maximum of the row's first 32 scores. Softmax does not depend on the reference value; the true row maximum
 //       only keeps the exponentials in range, and a row sum that comes out too large (or not a number) sends the warp
-//       through the exact path: row maximum over all chunks first, then the probabilities again)
+//       through the exact path: row maximum over all chunks first, then the probabilities again. Three exponentials
+//       in four run on the special-function unit, the fourth as a cubic on the FMA pipe)
 //   P5  tcgen05.mma: O_h[128 x 64] = P_h V_h        (V is the N-major B operand, as it lies in HBM)
 //   P6  four epilogue warps (a query row per thread): TMEM -> registers as soon as a half's product is complete (its
 //       accumulator is released at once), (f_0 O_0 + f_1 O_1) / sum, bf16 -> per warp, pieces of 16 columns x 32 rows
@@ -91,6 +92,20 @@ __device__ __forceinline__ float ex2_approx(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
+}
+
+// 2^x on the FMA pipe, for a share of the exponentials (the special-function unit delivers 16 results per cycle and SM,
+// which bounds the probability pass): x is split with the magic-number addition into an integer n, which goes straight
+// into the exponent field, and a fraction f in [-0.5, 0.5], on which a cubic (fitted to 2^f, relative error < 8e-5, well
+// below the bf16 rounding of the result) is evaluated. Results below 2^-125 are clamped there instead of flushed to 0.
+__device__ __forceinline__ float ex2_poly(float x) {
+  x = fmaxf(x, -125.0f);
+  const float t = x + 12582912.0f;              // 1.5 * 2^23: round(x) appears in the low mantissa bits
+  const float f = x - (t - 12582912.0f);
+  float q = fmaf(f, 0.05517092f, 0.24260956f);
+  q = fmaf(q, f, 0.69326097f);
+  q = fmaf(q, f, 0.9999282f);
+  return __uint_as_float(__float_as_uint(q) + (__float_as_uint(t) << 23));
 }
 
 // Orders the compiler only: no use of these registers moves above this point, no later write to them above their last use.
@@ -313,7 +328,10 @@ attention_fused_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
     // instruction every eight cycles, and only independent ones in flight keep it busy from a single warp.
     auto exp32 = [&](uint32_t (&v)[32], uint8_t* blk, uint32_t ch0, float mc, float (&s4)[4]) {
 #pragma unroll
-      for (int j = 0; j < 32; ++j) v[j] = __float_as_uint(ex2_approx(fmaf(__uint_as_float(v[j]), c, -mc)));
+      for (int j = 0; j < 32; ++j) {
+        const float x = fmaf(__uint_as_float(v[j]), c, -mc);
+        v[j] = __float_as_uint((j & 3) == 3 ? ex2_poly(x) : ex2_approx(x));   // one in four on the FMA pipe
+      }
 #pragma unroll
       for (int g = 0; g < 4; ++g) {
         uint32_t w[4];

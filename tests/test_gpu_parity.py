@@ -299,6 +299,28 @@ def test_fused_attention_dominant_key_and_uniform_rows(ago):
     np.testing.assert_allclose(gpu[0, :, :64], np.broadcast_to(v[0, 77, :64].astype(np.float64), (144, 64)), atol=2e-2)
 
 
+@pytest.mark.parametrize("S", [200, 384])
+def test_fused_attention_scores_far_above_the_first_keys(ago, S):
+    # The kernel takes a row's exponentials relative to the maximum of its first 32 scores of each half and repeats the
+    # pass with the true row maximum when that reference turns out too low. Here the scores grow along the keys: row r
+    # scores g_r * 8 * (k // 8) on key k, with g_r = 1 for rows that need the exact pass (at S = 200 the last keys of the
+    # second half lie 80 powers of two above its first 32) and g_r = 1/4 for rows that, at S = 200, do not; both kinds
+    # sit in every warp.
+    wl = WL.attention("attn_growing", [53], 1, S, 2, 64)
+    data = WL.generate(wl)
+    q, k, v = (a.copy() for a in data["inputs"])
+    q[:] = 0; k[:] = 0
+    for head in range(2):
+        q[0, 0::2, head * 64] = 1.0
+        q[0, 1::2, head * 64] = 0.25
+        k[0, :, head * 64] = 64.0 * (np.arange(S) // 8)
+    data["inputs"] = [q, k, v]
+    gpu = run_gpu(ago, wl, data, "fused")
+    ref = O.run_chain(wl.ops, data["inputs"], data["weights"])
+    assert np.isfinite(gpu).all()
+    assert_close(gpu, ref, what=f"attn growing scores S={S}")
+
+
 @pytest.mark.parametrize("S", [128, 200, 256, 384])
 def test_fused_attention_each_query_selects_its_keys(ago, S):
     # Query row r scores 32 on the keys j with j = r + 5 (mod 64) and 0 elsewhere, so its probabilities are (almost) one-hot
