@@ -390,6 +390,11 @@ def main():
             rf = roofline(wl, peaks, sec, traffic.get(key, {}).get("bytes"), clocks, extra_bytes=inter)
             if key in traffic:
                 rf["traffic_source"] = traffic[key]["source"]
+            ws_traffic = int(b.sgs[c].query(B.AGO_Q_WORKSPACE_TRAFFIC))
+            if ws_traffic:
+                # partial sums a split-reduction kernel adds into and reads back from device memory (through L2): real
+                # traffic that the roofline's algorithmic bytes (inputs + weights + output) do not contain
+                rf["workspace_traffic_bytes"] = ws_traffic
             chains.append({"chain": wl.name, "mode": eff, "us_per_launch_set": round(sec * 1e6, 3), "kernels_per_launch_set": b.launches[c],
                            "tile_rows": int(b.sgs[c].query(B.AGO_Q_TILE_ROWS)), "smem_bytes": int(b.sgs[c].query(B.AGO_Q_SMEM_BYTES)),
                            "roofline": rf})

@@ -29,7 +29,8 @@ MODES = {"fused": AGO_MODE_FUSED, "per_mini_subgraph": AGO_MODE_PER_MINI_SUBGRAP
 
 (AGO_Q_NUM_WEIGHTS, AGO_Q_WEIGHT_BYTES, AGO_Q_OUTPUT_RANK, AGO_Q_OUTPUT_DIM, AGO_Q_OUTPUT_BYTES,
  AGO_Q_FLOPS_TENSOR, AGO_Q_FLOPS_CUDA, AGO_Q_SFU_OPS, AGO_Q_IO_BYTES, AGO_Q_NUM_LINKS, AGO_Q_LINK_CATEGORY,
- AGO_Q_NUM_LAUNCHES, AGO_Q_FUSED_KERNEL, AGO_Q_INTERMEDIATE_BYTES, AGO_Q_TILE_ROWS, AGO_Q_SMEM_BYTES, AGO_Q_MODE) = range(17)
+ AGO_Q_NUM_LAUNCHES, AGO_Q_FUSED_KERNEL, AGO_Q_INTERMEDIATE_BYTES, AGO_Q_TILE_ROWS, AGO_Q_SMEM_BYTES, AGO_Q_MODE,
+ AGO_Q_WORKSPACE_TRAFFIC) = range(18)
 
 AGO_LINK_DOWNSTREAM_DEPTHWISE, AGO_LINK_DOWNSTREAM_POINTWISE, AGO_LINK_GENERAL = 1, 2, 3
 (AGO_KERNEL_NONE, AGO_KERNEL_DEPTHWISE, AGO_KERNEL_MBV2_BLOCK, AGO_KERNEL_FFN, AGO_KERNEL_CONV3X3_PAIR,

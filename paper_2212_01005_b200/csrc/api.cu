@@ -434,6 +434,7 @@ ago_status_t ago_subgraph_query(ago_subgraph_t h, int32_t what, int64_t* out) {
     case AGO_Q_TILE_ROWS: *out = p.tile_rows; break;
     case AGO_Q_SMEM_BYTES: *out = p.smem_bytes; break;
     case AGO_Q_MODE: *out = p.mode; break;
+    case AGO_Q_WORKSPACE_TRAFFIC: *out = p.mode == AGO_MODE_FUSED ? p.workspace_traffic_bytes : 0; break;
     default: return fail(AGO_ERR_INVALID_ARG, "unknown query");
   }
   return AGO_OK;

@@ -354,6 +354,8 @@ ago_status_t ffn_plan(Plan* plan, FusedState* st, std::string* err) {
   host->smem_bytes = (q.stages + q.G) * kStageBytes + 256 + 1024;
   host->acc_bytes = ((size_t)q.M * q.N2 * 4 + 255) & ~size_t(255);
   host->ws_bytes = ffn_workspace_bytes(*plan);
+  // every CTA of a row block adds its partial output rows into the fp32 buffer; the last one reads it back and zeroes it
+  plan->workspace_traffic_bytes = (int64_t)(q.hctas + 2) * q.M * q.N2 * 4;
   st->impl = host;
   st->impl_free = [](void* p) { delete static_cast<FfnHost*>(p); };
   st->tile_rows = kBM; st->grid = q.hctas * ((q.M + kBM - 1) / kBM); st->smem_bytes = host->smem_bytes;

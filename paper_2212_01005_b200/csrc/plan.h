@@ -74,6 +74,7 @@ struct Plan {
   int64_t max_intermediate_bytes = 0;  // largest tensor passed between launches
   int tile_rows = 0;
   int smem_bytes = 0;
+  int64_t workspace_traffic_bytes = 0;   // fused kernel: bytes it moves through its device-memory workspace per run
   int num_launches = 1;
 };
 

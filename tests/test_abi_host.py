@@ -13,6 +13,22 @@ from paper_2212_01005_b200 import workloads as WL
 ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 
 
+def test_workspace_traffic_query_names_the_split_reduction_only():
+    # The feed-forward kernel for few rows splits the hidden dimension over CTAs that add partial output rows into an fp32
+    # buffer in device memory: hidden / 128 additions of the whole output, one read-back and one zeroing sweep. Kernels
+    # whose intermediates stay on chip, and every unfused mode, report 0.
+    wl = WL.get("ffn_512")
+    sg = B.Subgraph(wl.ops, wl.input_shapes, mode="fused")
+    m, n2, hid = 512, 768, 3072
+    assert sg.query(B.AGO_Q_WORKSPACE_TRAFFIC) == (hid // 128 + 2) * m * n2 * 4
+    sg.close()
+    for name, mode in (("ffn_512", "per_mini_subgraph"), ("ffn_12288", "fused"), ("mbv2_56", "fused"), ("attn_384", "fused")):
+        wl = WL.get(name)
+        sg = B.Subgraph(wl.ops, wl.input_shapes, mode=mode)
+        assert sg.query(B.AGO_Q_WORKSPACE_TRAFFIC) == 0, (name, mode)
+        sg.close()
+
+
 def test_library_exports_every_declared_symbol():
     lib = B.load()
     hdr = open(os.path.join(ROOT, "include", "ago.h")).read()
