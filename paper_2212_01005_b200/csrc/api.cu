@@ -308,6 +308,10 @@ namespace {
 // costs less than about a third of the contractions' tensor-core time: both modes are then bound by the contractions
 // (Section VI-B reports the same for pointwise -> pointwise chains). Data-sheet-class constants; only the ratio matters.
 bool fusion_pays(const Plan& p) {
+  // Exception: a feed-forward chain on so few rows that the fused kernel splits each row block's hidden tiles over
+  // several clusters. The two GEMM launches of the unfused mode have a handful of row tiles each and leave most SMs
+  // idle; the fused kernel fills them through the hidden dimension (config 1: 24 against 45 us).
+  if (p.fused_kernel == AGO_KERNEL_FFN && p.fused_variant == 2) return true;
   const double t_intermediates = (double)p.intermediate_bytes / 6.5e12;
   const double t_tensor = (double)p.flops_tensor / 1.6e15;
   return !(t_tensor > 0.0 && t_intermediates < 0.35 * t_tensor);

@@ -67,7 +67,8 @@ ago_status_t fused_plan(Plan* plan, FusedState* st, std::string* err) {
 }
 
 size_t fused_workspace_bytes(const Plan& plan) {
-  return plan.fused_kernel == AGO_KERNEL_FFN && plan.fused_variant == 0 ? ffn_workspace_bytes(plan) : 0;
+  if (plan.fused_kernel != AGO_KERNEL_FFN) return 0;
+  return plan.fused_variant == 0 ? ffn_workspace_bytes(plan) : ffn_cluster_workspace_bytes(plan);
 }
 
 ago_status_t fused_run(const Plan& plan, FusedState* st, const void* const* inputs, const void* const* weights,
@@ -86,7 +87,7 @@ ago_status_t fused_run(const Plan& plan, FusedState* st, const void* const* inpu
     case AGO_KERNEL_ATTENTION:
       return attention_run(plan, st, inputs, weights, output, status_word, stream, err);
     case AGO_KERNEL_FFN:
-      if (st->variant == 1) return ffn_cluster_run(plan, st, inputs, weights, output, status_word, stream, err);
+      if (st->variant == 1) return ffn_cluster_run(plan, st, inputs, weights, output, workspace, status_word, stream, err);
       return ffn_run(plan, st, inputs, weights, output, workspace, status_word, stream, err);
     case AGO_KERNEL_CONV3X3_PAIR:
       return conv3x3_run(plan, st, inputs, weights, output, status_word, stream, err);

@@ -1,5 +1,7 @@
-// Fused feed-forward chain on a thread-block cluster: Y = GELU(X W1 + b1) W2 + b2, one kernel, the hidden
-// activations H never leave the SMs and nothing is reduced through device memory.
+// Fused feed-forward chain on a thread-block cluster: Y = GELU(X W1 + b1) W2 + b2; the hidden activations H never leave
+// the SMs. With enough row blocks to fill the device nothing is reduced through device memory and the run is one kernel;
+// with few row blocks (config 1: 512 rows) each row block's hidden tiles are split over J clusters, whose output shares
+// meet in an fp32 buffer (J additions per element), and a second, small launch turns the buffer into the output.
 //
 // Tile choice (Section III-B, "downstream pointwise / matmul"): the second GEMM reuses H only along its output
 // columns, so the downstream tile keeps ALL output columns of a block of 128 rows. Those (768 fp32 columns for
@@ -55,7 +57,9 @@ struct FfnClusterParams {
   unsigned int* status;
   int M, K, Hid, N2;
   int CS, NC;              // CTAs per cluster, output columns per CTA (N2 / CS, a multiple of 64, <= 256)
-  int T;                   // steps = Hid / 128 / CS
+  int T;                   // steps per row block = Hid / 128 / CS
+  int J, Tp;               // a row block is split over J clusters, each with Tp = T / J of its steps (J = 1: no split)
+  float* acc;              // J > 1: fp32 [M x N2] partial sums, zero between launches
   int kblocks;             // K / 64
   int stages;              // ring stages = 7 - CS (at most 5)
 };
@@ -65,6 +69,10 @@ __device__ __forceinline__ float gelu_tanh_fast(float v) {
   float t;
   asm("tanh.approx.f32 %0, %1;" : "=f"(t) : "f"(u));
   return 0.5f * v * (1.0f + t);
+}
+
+__device__ __forceinline__ void red_add_v4(float* addr, float a, float b, float c, float d) {
+  asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(addr), "f"(a), "f"(b), "f"(c), "f"(d) : "memory");
 }
 
 __global__ void __launch_bounds__(kThreads, 1)
@@ -90,13 +98,18 @@ ffn_cluster_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int r = (int)cluster_ctarank();
-  const int T = p.T;
-  // A cluster walks over the row blocks blockIdx.y, + gridDim.y, ...: its steps (row block, hidden tile of this CTA)
-  // form one sequence, so the first GEMM of the next row block overlaps the tail of the current one.
+  const int T = p.Tp, J = p.J;
+  // A unit of work is (row block, one of the J parts of its hidden tiles): T steps. A cluster walks over the units
+  // blockIdx.y, + gridDim.y, ...: its steps form one sequence, so the first GEMM of the next unit overlaps the tail of
+  // the current one. With J = 1 a unit is a whole row block and its output is final; with J > 1 (few row blocks: the
+  // hidden dimension is what fills the SMs) the J clusters of a row block add their outputs in device memory.
   const int row_blocks = (p.M + kBM - 1) / kBM;
-  const int my_blocks = ((int)blockIdx.y < row_blocks) ? (row_blocks - 1 - (int)blockIdx.y) / (int)gridDim.y + 1 : 0;
-  const int steps = my_blocks * T;
-  auto row0_of = [&](int step) { return ((int)blockIdx.y + (step / T) * (int)gridDim.y) * kBM; };
+  const int units = row_blocks * J;
+  const int my_units = ((int)blockIdx.y < units) ? (units - 1 - (int)blockIdx.y) / (int)gridDim.y + 1 : 0;
+  const int steps = my_units * T;
+  auto unit_of = [&](int step) { return (int)blockIdx.y + (step / T) * (int)gridDim.y; };
+  auto row0_of = [&](int step) { return (unit_of(step) / J) * kBM; };
+  auto tile0_of = [&](int step) { return ((unit_of(step) % J) * T + step % T) * CS; };   // first of the step's CS hidden tiles
   grid_dependency_wait();      // the previous grid of the stream has completed; device memory may be touched
   grid_launch_dependents();
 
@@ -136,7 +149,7 @@ ffn_cluster_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
       };
       auto advance = [&]() { if (++s == stages) { s = 0; ++round; } };
       auto load_g1 = [&](int step) {       // first GEMM of this CTA's hidden tile of that step
-        const int hid0 = ((step % T) * CS + r) * kBH, row0 = row0_of(step);
+        const int hid0 = (tile0_of(step) + r) * kBH, row0 = row0_of(step);
         for (int kb = 0; kb < p.kblocks; ++kb) {
           uint8_t* st = next_stage();
           tma_load_2d(st, &tmap_x, bar_full + s, kb * kBK, row0);                          // X [128 rows x 64 k]
@@ -149,7 +162,7 @@ ffn_cluster_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
       for (int step = 0; step < steps; ++step) {
         if (step + 1 < steps) load_g1(step + 1);
         for (int k = 0; k < CS; ++k) {      // second GEMM over hidden tile t CS + k: two stages of 64 hidden units
-          const int hid0 = ((step % T) * CS + k) * kBH;
+          const int hid0 = (tile0_of(step) + k) * kBH;
           for (int h = 0; h < 2; ++h) {
             uint8_t* st = next_stage();
             for (int nb = 0; nb < 4; ++nb)   // W2 [64 k x 64 n] per block; blocks past NC read as zero and are not multiplied
@@ -229,7 +242,7 @@ ffn_cluster_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
       // every CTA has multiplied the previous content of slot r (and the copies that delivered it are complete)
       if (step >= 1) mbar_wait(bar_hdone, (uint32_t)(step - 1) & 1u, abort_flag, p.status, 0x707);
       uint8_t* tile = slot + half * (kBM * 128);
-      const float* bb = p.b1 + (size_t)(t * CS + r) * kBH + half * 64;
+      const float* bb = p.b1 + (size_t)(tile0_of(step) + r) * kBH + half * 64;
 #pragma unroll
       for (int c0 = 0; c0 < 64; c0 += 32) {
         uint32_t v[32];
@@ -271,6 +284,27 @@ ffn_cluster_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
         mbar_wait(bar_out, (uint32_t)bi & 1u, abort_flag, p.status, 0x708);
         tcgen05_fence_after_sync();
         const int hc = p.NC >> 1;                                          // columns per half: 32, 64, 96 or 128
+        if (J > 1) {
+          // ---- split row block: add this cluster's share into the fp32 buffer; a second, small kernel turns the buffer
+          // into the output (+ b2, bf16) with every SM of the device and leaves it zeroed. (A last-arriver sweep inside
+          // this kernel -- one CTA per column slice reading 96 KB back -- took 8 us on the critical path.) ----
+          float* arow = p.acc + (size_t)(row0 + row) * p.N2 + n0 + half * hc;
+          for (int c0 = 0; c0 < hc; c0 += 32) {
+            uint32_t v[32];
+            tmem_ld_x32(tmem_base + lane_base + kOutCol + half * hc + c0, v);
+            tmem_ld_wait();
+            if (row_ok) {
+#pragma unroll
+              for (int q = 0; q < 8; ++q)
+                red_add_v4(arow + c0 + q * 4, __uint_as_float(v[4 * q]), __uint_as_float(v[4 * q + 1]),
+                           __uint_as_float(v[4 * q + 2]), __uint_as_float(v[4 * q + 3]));
+            }
+          }
+          tcgen05_fence_before_sync();
+          named_barrier_sync(1, kEpiThreads);
+          if (tid == 0) mbar_arrive(bar_outfree);
+          continue;
+        }
         __nv_bfloat16* orow = p.out + (size_t)(row0 + row) * p.N2 + n0 + half * hc;
         const float* b2 = p.b2 + n0 + half * hc;
         for (int c0 = 0; c0 < hc; c0 += 32) {
@@ -302,10 +336,26 @@ ffn_cluster_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
   if (warp == 0) tmem_dealloc(tmem_base, 512);
 }
 
+// Second launch of a split run: out = bf16(acc + b2), acc = 0. One float4 per thread and iteration, coalesced.
+__global__ void __launch_bounds__(256) ffn_cluster_finalize_kernel(float* acc, const float* b2, __nv_bfloat16* out, long long total4, int n2) {
+  grid_dependency_wait();      // the additions of the first launch are complete and visible
+  grid_launch_dependents();
+  const long long stride = (long long)gridDim.x * blockDim.x;
+  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total4; i += stride) {
+    const float4 a = __ldcg(reinterpret_cast<const float4*>(acc) + i);
+    const float4 bb = __ldg(reinterpret_cast<const float4*>(b2 + (int)((i * 4) % n2)));
+    reinterpret_cast<float4*>(acc)[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+    reinterpret_cast<uint2*>(out)[i] = make_uint2(pack_bf16x2(a.x + bb.x, a.y + bb.y), pack_bf16x2(a.z + bb.z, a.w + bb.w));
+  }
+}
+
 struct FfnClusterHost {
   FfnClusterParams prm;
   int smem_bytes = 0;
-  int clusters = 0;   // clusters launched = min(row blocks, clusters the device keeps resident); 0: not asked yet
+  int clusters = 0;   // clusters launched = min(units of work, clusters the device keeps resident); 0: not asked yet
+  size_t acc_bytes = 0, ws_bytes = 0;   // split row blocks: fp32 partial sums
+  const void* clean_ws = nullptr;   // workspace known to be zeroed (kept so by the kernel itself) ...
+  unsigned clean_epoch = 0;         // ... as of this attach (FusedState::workspace_epoch)
   struct Key { const void* p; int which; bool operator==(const Key& o) const { return p == o.p && which == o.which; } };
   struct KeyHash { size_t operator()(const Key& k) const { return std::hash<const void*>()(k.p) ^ (size_t)k.which * 0x9e3779b97f4a7c15ull; } };
   std::unordered_map<Key, CUtensorMap, KeyHash> maps;
@@ -356,10 +406,18 @@ ago_status_t ffn_cluster_plan(Plan* plan, FusedState* st, std::string* err) {
     if (q.CS == 0 || cost < best) { q.CS = cs; q.NC = nc; best = cost; }
   }
   if (q.CS == 0) return AGO_ERR_UNSUPPORTED;
-  // one cluster per block of 128 rows: worth it only when the clusters fill the SMs; few rows are better served by the
-  // kernel that spreads the hidden tiles of a row block over independent CTAs
-  if ((long)((q.M + kBM - 1) / kBM) * q.CS < 120) return AGO_ERR_UNSUPPORTED;
   q.T = htiles / q.CS;
+  q.J = 1;
+  if ((long)row_blocks_plan * q.CS < 120) {
+    // Few row blocks: one cluster per block of 128 rows leaves most SMs idle, and the hidden dimension is what can fill
+    // them. A row block is split over J clusters (J divides its T steps); their outputs meet in an fp32 buffer in device
+    // memory, J additions per element instead of one per hidden tile. J = as many parts as still fit one round of
+    // resident clusters, each with at least one step.
+    for (int j = q.T; j >= 1; --j)
+      if (q.T % j == 0 && (long)row_blocks_plan * j <= resident[q.CS]) { q.J = j; break; }
+    if (q.J == 1 || q.N2 % 4 != 0 || (q.NC / 2) % 32 != 0) return AGO_ERR_UNSUPPORTED;   // nothing to split: the other kernel
+  }
+  q.Tp = q.T / q.J;
   q.kblocks = q.K / kBK;
   q.stages = std::min(kMaxStages, kBlocks - q.CS);
   auto* host = new FfnClusterHost();
@@ -368,14 +426,28 @@ ago_status_t ffn_cluster_plan(Plan* plan, FusedState* st, std::string* err) {
   st->impl = host;
   st->impl_free = [](void* p) { delete static_cast<FfnClusterHost*>(p); };
   st->variant = 1;
-  st->tile_rows = kBM; st->grid = q.CS * ((q.M + kBM - 1) / kBM); st->smem_bytes = host->smem_bytes;
+  st->tile_rows = kBM; st->grid = q.CS * q.J * ((q.M + kBM - 1) / kBM); st->smem_bytes = host->smem_bytes;
   plan->tile_rows = kBM; plan->smem_bytes = host->smem_bytes;
-  plan->fused_variant = 1;
+  plan->fused_variant = q.J > 1 ? 2 : 1;
+  if (q.J > 1) {
+    host->acc_bytes = ((size_t)q.M * q.N2 * 4 + 255) & ~size_t(255);
+    host->ws_bytes = host->acc_bytes;
+    // every cluster of a row block adds its share into the buffer; the second launch reads it back and zeroes it
+    plan->workspace_traffic_bytes = (int64_t)(q.J + 2) * q.M * q.N2 * 4;
+    plan->num_launches = 2;
+  }
   return AGO_OK;
 }
 
+size_t ffn_cluster_workspace_bytes(const Plan& plan) {
+  if (plan.fused_variant != 2) return 0;
+  const int64_t M = plan.inputs[0].numel() / plan.inputs[0].last();
+  const int64_t N2 = plan.output.last();
+  return ((size_t)M * N2 * 4 + 255) & ~size_t(255);
+}
+
 ago_status_t ffn_cluster_run(const Plan& plan, FusedState* st, const void* const* inputs, const void* const* weights,
-                             void* output, unsigned int* status_word, cudaStream_t stream, std::string* err) {
+                             void* output, void* workspace, unsigned int* status_word, cudaStream_t stream, std::string* err) {
   (void)plan;
   FfnClusterHost* host = static_cast<FfnClusterHost*>(st->impl);
   FfnClusterParams q = host->prm;
@@ -383,6 +455,18 @@ ago_status_t ffn_cluster_run(const Plan& plan, FusedState* st, const void* const
   q.b2 = static_cast<const float*>(weights[3]);
   q.out = static_cast<__nv_bfloat16*>(output);
   q.status = status_word;
+  if (q.J > 1) {
+    if (!workspace) { *err = "fused feed-forward (cluster, split row blocks): no workspace attached"; return AGO_ERR_INVALID_ARG; }
+    q.acc = static_cast<float*>(workspace);
+    if (host->clean_ws != workspace || host->clean_epoch != st->workspace_epoch) {
+      // a workspace is zeroed at the first run after each attach; after that every launch leaves it zeroed (the caller
+      // must not touch it in between)
+      cudaError_t e = cudaMemsetAsync(workspace, 0, host->ws_bytes, stream);
+      if (e != cudaSuccess) { *err = std::string("cudaMemsetAsync(workspace): ") + cudaGetErrorString(e); return AGO_ERR_CUDA; }
+      host->clean_ws = workspace;
+      host->clean_epoch = st->workspace_epoch;
+    }
+  }
   auto get_map = [&](const void* base, int which, CUtensorMap* out) -> bool {
     FfnClusterHost::Key key{base, which};
     auto it = host->maps.find(key);
@@ -410,18 +494,25 @@ ago_status_t ffn_cluster_run(const Plan& plan, FusedState* st, const void* const
   const int row_blocks = (q.M + kBM - 1) / kBM;
   if (host->clusters == 0) {
     // persistent clusters: as many as the device keeps resident at once (one CTA per SM, CS SMs of one GPC each)
-    fill_launch(&cfg, attr, q, row_blocks, host->smem_bytes, stream);
+    fill_launch(&cfg, attr, q, row_blocks * q.J, host->smem_bytes, stream);
     int resident = 0;
     cudaError_t e = cudaOccupancyMaxActiveClusters(&resident, ffn_cluster_kernel, &cfg);
     if (e != cudaSuccess || resident < 1) {
       *err = std::string("fused feed-forward (cluster): no cluster of this size is schedulable: ") + cudaGetErrorString(e);
       return AGO_ERR_CUDA;
     }
-    host->clusters = std::min(row_blocks, resident);
+    host->clusters = std::min(row_blocks * q.J, resident);
   }
   fill_launch(&cfg, attr, q, host->clusters, host->smem_bytes, stream);
   cudaError_t e = cudaLaunchKernelEx(&cfg, ffn_cluster_kernel, mx, mw1, mw2, q);
   if (e != cudaSuccess) { *err = std::string("fused feed-forward (cluster) launch: ") + cudaGetErrorString(e); return AGO_ERR_CUDA; }
+  if (q.J > 1) {
+    const long long total4 = (long long)q.M * q.N2 / 4;
+    const int blocks = (int)std::min<long long>((total4 + 255) / 256, 4LL * device_sm_count());
+    FusedLaunch fin(dim3((unsigned)blocks), 256, 0, stream);
+    e = cudaLaunchKernelEx(&fin.config, ffn_cluster_finalize_kernel, q.acc, q.b2, q.out, total4, q.N2);
+    if (e != cudaSuccess) { *err = std::string("fused feed-forward (cluster) finalisation launch: ") + cudaGetErrorString(e); return AGO_ERR_CUDA; }
+  }
   return AGO_OK;
 }
 

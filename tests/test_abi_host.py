@@ -14,13 +14,14 @@ ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 
 
 def test_workspace_traffic_query_names_the_split_reduction_only():
-    # The feed-forward kernel for few rows splits the hidden dimension over CTAs that add partial output rows into an fp32
-    # buffer in device memory: hidden / 128 additions of the whole output, one read-back and one zeroing sweep. Kernels
-    # whose intermediates stay on chip, and every unfused mode, report 0.
+    # The feed-forward kernel for few rows splits the hidden tiles of a row block over J clusters that add their output
+    # shares into an fp32 buffer in device memory: J additions of the whole output, one read-back and one zeroing sweep
+    # (config 1: 24 hidden tiles, clusters of 4, J = 6). Kernels whose intermediates stay on chip, and every unfused mode,
+    # report 0.
     wl = WL.get("ffn_512")
     sg = B.Subgraph(wl.ops, wl.input_shapes, mode="fused")
     m, n2, hid = 512, 768, 3072
-    assert sg.query(B.AGO_Q_WORKSPACE_TRAFFIC) == (hid // 128 + 2) * m * n2 * 4
+    assert sg.query(B.AGO_Q_WORKSPACE_TRAFFIC) == (6 + 2) * m * n2 * 4
     sg.close()
     for name, mode in (("ffn_512", "per_mini_subgraph"), ("ffn_12288", "fused"), ("mbv2_56", "fused"), ("attn_384", "fused")):
         wl = WL.get(name)
@@ -109,7 +110,9 @@ def test_fused_planner_matches_every_chain_family_and_its_limits():
         wl = WL.get(name)
         sg = B.Subgraph(wl.ops, wl.input_shapes, mode="fused")
         assert sg.query(B.AGO_Q_FUSED_KERNEL) == kernel, name
-        assert sg.query(B.AGO_Q_NUM_LAUNCHES) == 1
+        # one kernel, except where a row block's hidden tiles are split over clusters (config 1: few rows): a second,
+        # small launch turns the fp32 sums into the output
+        assert sg.query(B.AGO_Q_NUM_LAUNCHES) == (2 if name == "ffn_512" else 1), name
         assert 0 < sg.query(B.AGO_Q_SMEM_BYTES) <= 227 * 1024 and sg.query(B.AGO_Q_TILE_ROWS) >= 1
         sg.close()
     # the two depthwise convolutions of the pair kernel are stride 1; a strided pair has no kernel
@@ -131,7 +134,8 @@ def test_fused_planner_matches_every_chain_family_and_its_limits():
 
 
 def test_feed_forward_planner_picks_the_cluster_kernel_where_the_shape_splits():
-    # cluster kernel: no workspace (nothing is reduced through device memory); split-reduction kernel: an fp32 buffer
+    # cluster kernel on many row blocks: no workspace (nothing is reduced through device memory); few row blocks (their
+    # hidden tiles split over several clusters) and the kernel without clusters: an fp32 buffer
     def ws(M, K, hid, out):
         wl = WL.ffn("x", [1], M, K, hid, 1, d_out=out)
         sg = B.Subgraph(wl.ops, wl.input_shapes, mode="fused")
@@ -140,7 +144,7 @@ def test_feed_forward_planner_picks_the_cluster_kernel_where_the_shape_splits():
         return w
     assert ws(12288, 768, 3072, 768) == 0          # 96 row blocks, clusters of 3 or 4
     assert ws(9637, 64, 256, 384) == 0             # clusters of 2, ragged last row block
-    assert ws(512, 768, 3072, 768) >= 512 * 768 * 4    # four row blocks do not fill the SMs with clusters
+    assert ws(512, 768, 3072, 768) >= 512 * 768 * 4    # four row blocks: six clusters each
     assert ws(12800, 256, 384, 256) >= 12800 * 256 * 4  # three hidden tiles, 256 columns: no cluster size divides both
 
 
@@ -227,17 +231,20 @@ def test_bf16_helpers_round_to_nearest_even():
 
 def test_auto_mode_fuses_unless_the_contractions_bound_both_modes():
     # AGO_MODE_AUTO resolves at create time (host only): chains whose intermediates dominate the traffic are fused;
-    # the feed-forward chain (two large GEMMs, Section VI-B's pointwise -> pointwise observation) and chains without
-    # a fused kernel run per mini-subgraph
+    # the feed-forward chain on many rows (two large GEMMs, Section VI-B's pointwise -> pointwise observation) and chains
+    # without a fused kernel run per mini-subgraph; the feed-forward chain on few rows is fused (its unfused GEMMs
+    # cannot fill the SMs, the fused kernel splits the hidden dimension over clusters)
     from paper_2212_01005_b200 import workloads as WL
     want = {"attn_384": B.AGO_MODE_FUSED, "mbv2_56": B.AGO_MODE_FUSED, "mbv2_28s2": B.AGO_MODE_FUSED, "resnet_56": B.AGO_MODE_FUSED,
             "pw_pw_56": B.AGO_MODE_FUSED, "dw_dw_56": B.AGO_MODE_FUSED, "unfold_96": B.AGO_MODE_FUSED,
-            "ffn_12288": B.AGO_MODE_PER_MINI_SUBGRAPH, "ffn_512": B.AGO_MODE_PER_MINI_SUBGRAPH}
+            "ffn_12288": B.AGO_MODE_PER_MINI_SUBGRAPH, "ffn_512": B.AGO_MODE_FUSED}
     for name, mode in want.items():
         wl = WL.get(name)
         sg = B.Subgraph(wl.ops, wl.input_shapes, mode="auto")
         assert sg.query(B.AGO_Q_MODE) == mode, name
-        assert sg.query(B.AGO_Q_NUM_LAUNCHES) == (1 if mode == B.AGO_MODE_FUSED else B.Subgraph(wl.ops, wl.input_shapes, mode="per_mini_subgraph").query(B.AGO_Q_NUM_LAUNCHES))
+        same = B.Subgraph(wl.ops, wl.input_shapes, mode="fused" if mode == B.AGO_MODE_FUSED else "per_mini_subgraph")
+        assert sg.query(B.AGO_Q_NUM_LAUNCHES) == same.query(B.AGO_Q_NUM_LAUNCHES)
+        same.close()
         sg.close()
     lone = B.Subgraph([("gemm", {"N": 64}), ("relu", {})], [(256, 64)], mode="auto")     # no fused family: not an error in AUTO
     assert lone.query(B.AGO_Q_MODE) == B.AGO_MODE_PER_MINI_SUBGRAPH
