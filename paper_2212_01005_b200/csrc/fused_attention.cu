@@ -66,7 +66,6 @@ constexpr int kTmaWarp = kEpiWarp0 + 4;
 constexpr int kMmaWarp = kTmaWarp + 1;
 constexpr int kThreads = (kMmaWarp + 1) * 32;    // 448
 constexpr int kHalfCols = 192;         // tensor-memory columns reserved per score half
-constexpr int kMaxChunks = kHalfCols / 32;      // 32-column chunks of a row of one half
 // A row's exponentials are taken relative to the maximum of its first 32 scores, not of all of them (any reference gives
 // the same softmax; the true maximum only guarantees the range). A row sum at or above this limit, or not a number, sends
 // the warp through the exact two-pass path.
@@ -300,10 +299,6 @@ attention_fused_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
     // The outstanding load of a 32-register buffer has landed (one wait; the second statement only orders the compiler).
     auto wait32 = [](uint32_t (&v)[32]) {
       tmem_ld_wait_on(reinterpret_cast<uint32_t (&)[16]>(v[0]));
-      reg_order16(reinterpret_cast<uint32_t (&)[16]>(v[16]));
-    };
-    auto wait_order32 = [](uint32_t (&v)[32]) {   // after a wait32 that covered this buffer's load as well
-      reg_order16(reinterpret_cast<uint32_t (&)[16]>(v[0]));
       reg_order16(reinterpret_cast<uint32_t (&)[16]>(v[16]));
     };
     auto max32 = [](const uint32_t (&v)[32]) -> float {
