@@ -90,6 +90,21 @@ __device__ __forceinline__ void sts128(uint32_t saddr, uint32_t a, uint32_t b, u
   asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(saddr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
 }
 
+// One MMA with the accumulate flag known at compile time (no predicate to set at run time): descriptors as (low, high)
+// words. Next to thirty busy warps the issuing thread gets an issue slot every few tens of cycles, so every instruction
+// in front of an MMA counts.
+template <bool ACC>
+__device__ __forceinline__ void umma_lohi_c(uint32_t d_tmem, uint32_t a_lo, uint32_t a_hi, uint32_t b_lo, uint32_t b_hi, uint32_t idesc) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t.reg .b64 ad, bd;\n\t"
+      "mov.b64 ad, {%1, %2};\n\t"
+      "mov.b64 bd, {%3, %4};\n\t"
+      "setp.ne.b32 p, %6, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], ad, bd, %5, p;\n\t}"
+      ::"r"(d_tmem), "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "n"(ACC ? 1 : 0)
+      : "memory");
+}
+
 // FOLD: the expand bias rides in the expand GEMM (see the prologue). EXPAND / PROJECT select the pairs of the
 // block: <true, true> the whole block, <true, false> pointwise -> depthwise
 // (the depthwise result of every chunk goes to device memory), <false, true> depthwise -> pointwise (every chunk of
@@ -362,12 +377,28 @@ mbv2_fused_kernel(const Mbv2Params p) {
     const uint32_t exp_b_step = (uint32_t)(NG * kChunk * p.row_bytes) >> 4;   // the group's next chunk is c + NG
     uint32_t exp_b_lo = (uint32_t)w1desc0 + ((uint32_t)(g * kChunk * p.row_bytes) >> 4);
     const int ksteps = p.Kp / 16;
-    auto issue_expand = [&]() {   // one lane; advances to the group's next chunk
+    const int exp_tiles = xi >= 0 ? (p.M1 - xi + kExpandIssuers - 1) / kExpandIssuers : 0;   // tiles this warp issues per chunk
+    auto issue_expand = [&]() {   // one lane; advances to the group's next chunk. Straight-line per reduction length.
       uint32_t a_lo = exp_a_lo0, d_tmem = exp_d_tmem0;
-      for (int t = xi; t < p.M1; t += kExpandIssuers, a_lo += exp_a_step, d_tmem += kExpandIssuers * kChunk) {
-#pragma unroll
-        for (int ks = 0; ks < 4; ++ks)
-          if (ks < ksteps) umma_bf16_lohi(d_tmem, a_lo + 2u * ks, x_hi, exp_b_lo + 2u * ks, w1_hi, idesc_e, ks > 0);
+      const uint32_t b_lo = exp_b_lo;
+      if (ksteps == 2) {
+#pragma unroll 1
+        for (int t = 0; t < exp_tiles; ++t, a_lo += exp_a_step, d_tmem += kExpandIssuers * kChunk) {
+          umma_lohi_c<false>(d_tmem, a_lo, x_hi, b_lo, w1_hi, idesc_e);
+          umma_lohi_c<true>(d_tmem, a_lo + 2u, x_hi, b_lo + 2u, w1_hi, idesc_e);
+        }
+      } else if (ksteps == 4) {
+#pragma unroll 1
+        for (int t = 0; t < exp_tiles; ++t, a_lo += exp_a_step, d_tmem += kExpandIssuers * kChunk) {
+          umma_lohi_c<false>(d_tmem, a_lo, x_hi, b_lo, w1_hi, idesc_e);
+          umma_lohi_c<true>(d_tmem, a_lo + 2u, x_hi, b_lo + 2u, w1_hi, idesc_e);
+          umma_lohi_c<true>(d_tmem, a_lo + 4u, x_hi, b_lo + 4u, w1_hi, idesc_e);
+          umma_lohi_c<true>(d_tmem, a_lo + 6u, x_hi, b_lo + 6u, w1_hi, idesc_e);
+        }
+      } else {
+#pragma unroll 1
+        for (int t = 0; t < exp_tiles; ++t, a_lo += exp_a_step, d_tmem += kExpandIssuers * kChunk)
+          umma_lohi_c<false>(d_tmem, a_lo, x_hi, b_lo, w1_hi, idesc_e);
       }
       umma_commit(bar_e + g);
       exp_b_lo += exp_b_step;
