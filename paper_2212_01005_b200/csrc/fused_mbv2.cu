@@ -90,21 +90,6 @@ __device__ __forceinline__ void sts128(uint32_t saddr, uint32_t a, uint32_t b, u
   asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(saddr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
 }
 
-// One MMA with the accumulate flag known at compile time (no predicate to set at run time): descriptors as (low, high)
-// words. Next to thirty busy warps the issuing thread gets an issue slot every few tens of cycles, so every instruction
-// in front of an MMA counts.
-template <bool ACC>
-__device__ __forceinline__ void umma_lohi_c(uint32_t d_tmem, uint32_t a_lo, uint32_t a_hi, uint32_t b_lo, uint32_t b_hi, uint32_t idesc) {
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t.reg .b64 ad, bd;\n\t"
-      "mov.b64 ad, {%1, %2};\n\t"
-      "mov.b64 bd, {%3, %4};\n\t"
-      "setp.ne.b32 p, %6, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], ad, bd, %5, p;\n\t}"
-      ::"r"(d_tmem), "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "n"(ACC ? 1 : 0)
-      : "memory");
-}
-
 // FOLD: the expand bias rides in the expand GEMM (see the prologue). EXPAND / PROJECT select the pairs of the
 // block: <true, true> the whole block, <true, false> pointwise -> depthwise
 // (the depthwise result of every chunk goes to device memory), <false, true> depthwise -> pointwise (every chunk of
@@ -368,58 +353,61 @@ mbv2_fused_kernel(const Mbv2Params p) {
     // D: un-swizzled K-major; the two 8-channel planes are the two K core-matrix columns
     const uint64_t ddesc0 = make_smem_desc(smem_u32(sD), (uint32_t)p.d_plane, 128, SW_NONE);
     const uint64_t w3desc0 = make_smem_desc(smem_u32(sW3), 0, 256, SW_32B);
+    // MMAs are issued by whole, converged warps: the MMA itself is predicated on one elected lane, its descriptors are
+    // ready 64-bit values (see tc_common.cuh: several times the issue rate of a lane-0 branch next to busy warps).
+    const uint32_t elected = elect_one();
     // Expand issue state of the group's last two warps: tiles xi, xi + 2, ... of the group's chunks -> buffer g.
     const uint32_t idesc_e = make_idesc_bf16(128, kChunk);
-    const uint32_t x_hi = (uint32_t)(xdesc0 >> 32), w1_hi = (uint32_t)(w1desc0 >> 32);
-    const uint32_t exp_a_step = (uint32_t)(kExpandIssuers * 128 * p.row_bytes) >> 4;
-    const uint32_t exp_a_lo0 = (uint32_t)xdesc0 + ((uint32_t)(max(xi, 0) * 128 * p.row_bytes) >> 4);
+    const uint64_t exp_a_step = (uint64_t)((uint32_t)(kExpandIssuers * 128 * p.row_bytes) >> 4);
+    const uint64_t exp_a0 = xdesc0 + (uint64_t)((uint32_t)(max(xi, 0) * 128 * p.row_bytes) >> 4);
     const uint32_t exp_d_tmem0 = tmem_base + p.ecol0 + (g * p.M1 + max(xi, 0)) * kChunk;
-    const uint32_t exp_b_step = (uint32_t)(NG * kChunk * p.row_bytes) >> 4;   // the group's next chunk is c + NG
-    uint32_t exp_b_lo = (uint32_t)w1desc0 + ((uint32_t)(g * kChunk * p.row_bytes) >> 4);
+    const uint64_t exp_b_step = (uint64_t)((uint32_t)(NG * kChunk * p.row_bytes) >> 4);   // the group's next chunk is c + NG
+    uint64_t exp_b = w1desc0 + (uint64_t)((uint32_t)(g * kChunk * p.row_bytes) >> 4);
     const int ksteps = p.Kp / 16;
     const int exp_tiles = xi >= 0 ? (p.M1 - xi + kExpandIssuers - 1) / kExpandIssuers : 0;   // tiles this warp issues per chunk
-    auto issue_expand = [&]() {   // one lane; advances to the group's next chunk. Straight-line per reduction length.
-      uint32_t a_lo = exp_a_lo0, d_tmem = exp_d_tmem0;
-      const uint32_t b_lo = exp_b_lo;
+    auto issue_expand = [&]() {   // whole warp; advances to the group's next chunk. Straight-line per reduction length.
+      uint64_t a = exp_a0;
+      uint32_t d_tmem = exp_d_tmem0;
+      const uint64_t b = exp_b;
       if (ksteps == 2) {
 #pragma unroll 1
-        for (int t = 0; t < exp_tiles; ++t, a_lo += exp_a_step, d_tmem += kExpandIssuers * kChunk) {
-          umma_lohi_c<false>(d_tmem, a_lo, x_hi, b_lo, w1_hi, idesc_e);
-          umma_lohi_c<true>(d_tmem, a_lo + 2u, x_hi, b_lo + 2u, w1_hi, idesc_e);
+        for (int t = 0; t < exp_tiles; ++t, a += exp_a_step, d_tmem += kExpandIssuers * kChunk) {
+          umma_bf16_elected<false>(d_tmem, a, b, idesc_e, elected);
+          umma_bf16_elected<true>(d_tmem, a + 2u, b + 2u, idesc_e, elected);
         }
       } else if (ksteps == 4) {
 #pragma unroll 1
-        for (int t = 0; t < exp_tiles; ++t, a_lo += exp_a_step, d_tmem += kExpandIssuers * kChunk) {
-          umma_lohi_c<false>(d_tmem, a_lo, x_hi, b_lo, w1_hi, idesc_e);
-          umma_lohi_c<true>(d_tmem, a_lo + 2u, x_hi, b_lo + 2u, w1_hi, idesc_e);
-          umma_lohi_c<true>(d_tmem, a_lo + 4u, x_hi, b_lo + 4u, w1_hi, idesc_e);
-          umma_lohi_c<true>(d_tmem, a_lo + 6u, x_hi, b_lo + 6u, w1_hi, idesc_e);
+        for (int t = 0; t < exp_tiles; ++t, a += exp_a_step, d_tmem += kExpandIssuers * kChunk) {
+          umma_bf16_elected<false>(d_tmem, a, b, idesc_e, elected);
+          umma_bf16_elected<true>(d_tmem, a + 2u, b + 2u, idesc_e, elected);
+          umma_bf16_elected<true>(d_tmem, a + 4u, b + 4u, idesc_e, elected);
+          umma_bf16_elected<true>(d_tmem, a + 6u, b + 6u, idesc_e, elected);
         }
       } else {
 #pragma unroll 1
-        for (int t = 0; t < exp_tiles; ++t, a_lo += exp_a_step, d_tmem += kExpandIssuers * kChunk)
-          umma_lohi_c<false>(d_tmem, a_lo, x_hi, b_lo, w1_hi, idesc_e);
+        for (int t = 0; t < exp_tiles; ++t, a += exp_a_step, d_tmem += kExpandIssuers * kChunk)
+          umma_bf16_elected<false>(d_tmem, a, b, idesc_e, elected);
       }
-      umma_commit(bar_e + g);
-      exp_b_lo += exp_b_step;
+      umma_commit_elected(bar_e + g, elected);
+      exp_b += exp_b_step;
     };
     // Project issue state of warp gw < M2 (tile gw), kept in three registers: a warp that runs a serial instruction
     // chain next to warps with dense arithmetic gets an issue slot only every few tens of cycles, so the path from
     // the barrier to the MMA is one add, the MMA and the commit.
-    constexpr uint32_t kDescVersion = 1u << 14;   // high descriptor word: SBO >> 4, version 1 at bit 46, layout at bits 61..63
-    constexpr uint32_t d_hi = (128u >> 4) | kDescVersion | ((uint32_t)SW_NONE << 29);
-    constexpr uint32_t w3_hi = (256u >> 4) | kDescVersion | ((uint32_t)SW_32B << 29);
     const uint32_t idesc_p = make_idesc_bf16(128, (uint32_t)p.Coutp);
-    const uint32_t proj_a_lo = (uint32_t)ddesc0 + ((uint32_t)(g * d_bytes + gw * 128 * 16) >> 4);
+    const uint64_t proj_a = ddesc0 + (uint64_t)((uint32_t)(g * d_bytes + gw * 128 * 16) >> 4);
     const uint32_t proj_d_tmem = tmem_base + p.pcol0 + gw * p.Coutp;
-    const uint32_t proj_b_step = (uint32_t)(NG * p.Coutp * kChunkRowBytes) >> 4;     // the group's next chunk is c + NG
-    uint32_t proj_b_lo = (uint32_t)w3desc0 + ((uint32_t)(g * p.Coutp * kChunkRowBytes) >> 4);
-    if (EXPAND && xi >= 0 && lane == 0 && g < p.NC) {
+    const uint64_t proj_b_step = (uint64_t)((uint32_t)(NG * p.Coutp * kChunkRowBytes) >> 4);     // the group's next chunk is c + NG
+    uint64_t proj_b = w3desc0 + (uint64_t)((uint32_t)(g * p.Coutp * kChunkRowBytes) >> 4);
+    if (EXPAND && xi >= 0 && g < p.NC) {
       // group 1 issues its first expand GEMM once group 0's is through the tensor pipe: group 0 has the longer chain
       // of chunks, and its first epilogue would otherwise wait for both groups' MMAs
       // (with more than two groups the strips are small, the products short, and a chain of first products would cost
       // more than it saves; a waiter that falls two phases behind a barrier would also read the wrong parity)
-      if (NG == 2 && g == 1) mbar_wait(bar_e, 0, abort_flag, p.status, 0x107);
+      if (NG == 2 && g == 1) {
+        if (lane == 0) mbar_wait(bar_e, 0, abort_flag, p.status, 0x107);
+        __syncwarp();
+      }
       issue_expand();
     }
     __syncwarp();
@@ -489,11 +477,8 @@ mbv2_fused_kernel(const Mbv2Params p) {
       if (PROJECT && waiter && it >= 1) mbar_wait(bar_d + g, (uint32_t)(it - 1) & 1u, abort_flag, p.status, 0x103);
       named_barrier_sync(gbar, kGroupThreads);
       if (EXPAND && xi >= 0 && c + NG < p.NC) {   // expand buffer g is drained: the expand GEMM of the group's next chunk
-        if (lane == 0) {
-          tcgen05_fence_after_sync();
-          issue_expand();
-        }
-        __syncwarp();
+        tcgen05_fence_after_sync();
+        issue_expand();
       }
 
       // ---- P4: depthwise 3x3 + bias + ReLU6 on CUDA cores: E[g] -> D[g] (A operand of the project GEMM) ----
@@ -542,18 +527,18 @@ mbv2_fused_kernel(const Mbv2Params p) {
         }
       }
       if (PROJECT && gw < p.M2) {   // D[g] is complete: the project GEMM of chunk c, one tile per warp
-        if (lane == 0) {
-          // chunk 0 overwrites the accumulators: everything else is issued after it
-          if (c >= 1 && c < NG) mbar_wait(bar_first, 0, abort_flag, p.status, 0x106);
-          tcgen05_fence_after_sync();
-          umma_bf16_lohi(proj_d_tmem, proj_a_lo, d_hi, proj_b_lo, w3_hi, idesc_p, c > 0);
-          umma_commit(bar_d + g);
-          if (c == 0) umma_commit(bar_first);
-          if (c + NG >= p.NC && !skip_signal_for_test(p.status, 0x104)) umma_commit(bar_done);
+        // chunk 0 overwrites the accumulators: everything else is issued after it
+        if (c >= 1 && c < NG) {
+          if (lane == 0) mbar_wait(bar_first, 0, abort_flag, p.status, 0x106);
+          __syncwarp();
         }
-        __syncwarp();
+        tcgen05_fence_after_sync();
+        umma_bf16_elected_acc(proj_d_tmem, proj_a, proj_b, idesc_p, elected, c > 0 ? 1u : 0u);
+        umma_commit_elected(bar_d + g, elected);
+        if (c == 0) umma_commit_elected(bar_first, elected);
+        if (c + NG >= p.NC && !skip_signal_for_test(p.status, 0x104)) umma_commit_elected(bar_done, elected);
       }
-      proj_b_lo += proj_b_step;
+      proj_b += proj_b_step;
     }
 
     // ---- P6: project epilogue: + b3 (+ residual), bf16, 16-byte stores ----

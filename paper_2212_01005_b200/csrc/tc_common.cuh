@@ -314,6 +314,47 @@ __device__ __forceinline__ void umma_bf16_lohi(uint32_t d_tmem, uint32_t a_lo, u
       : "memory");
 }
 
+// ---- MMA issue from a converged warp --------------------------------------------------------------
+// Writing the issue as `if (lane == 0) { ... tcgen05.mma ... }` makes the operands lane-dependent values behind a divergent
+// branch; next to warps with dense arithmetic such an issuing thread got one MMA out every 170-550 cycles (measured, 28
+// FMA-bound neighbours). The same loop run by the whole warp, converged, with the MMA predicated on a lane elected once
+// and the descriptors ready as 64-bit values, issues one every 50-60 cycles. All lanes execute these helpers; `elected`
+// is elect_one() of the calling warp, taken while it is converged (the same lane then issues the MMAs and the commit).
+__device__ __forceinline__ uint32_t elect_one() {
+  uint32_t r;
+  asm volatile("{\n\t.reg .pred q;\n\telect.sync _|q, 0xffffffff;\n\tselp.u32 %0, 1, 0, q;\n\t}" : "=r"(r));
+  return r;
+}
+template <bool ACC>
+__device__ __forceinline__ void umma_bf16_elected(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t elected) {
+  asm volatile(
+      "{\n\t.reg .pred p, q;\n\t"
+      "setp.ne.b32 q, %4, 0;\n\t"
+      "setp.ne.b32 p, %5, 0;\n\t"
+      "@q tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(elected), "n"(ACC ? 1 : 0)
+      : "memory");
+}
+// accumulate flag known only at run time
+__device__ __forceinline__ void umma_bf16_elected_acc(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t elected,
+                                                      uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p, q;\n\t"
+      "setp.ne.b32 q, %4, 0;\n\t"
+      "setp.ne.b32 p, %5, 0;\n\t"
+      "@q tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(elected), "r"(accumulate)
+      : "memory");
+}
+__device__ __forceinline__ void umma_commit_elected(uint64_t* bar, uint32_t elected) {
+  asm volatile(
+      "{\n\t.reg .pred q;\n\t"
+      "setp.ne.b32 q, %1, 0;\n\t"
+      "@q tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n\t}"
+      ::"r"(smem_u32(bar)), "r"(elected)
+      : "memory");
+}
+
 // Arrive on `bar` once all MMAs issued so far by this thread have completed
 // (implies tcgen05.fence::before_thread_sync).
 __device__ __forceinline__ void umma_commit(uint64_t* bar) {
