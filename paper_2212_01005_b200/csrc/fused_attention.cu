@@ -204,8 +204,11 @@ attention_fused_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
     }
     __syncwarp();
   } else if (warp == kMmaWarp) {
-    // ============================ MMA issue (one lane) ============================
-    if (lane == 0) {
+    // ============================ MMA issue ============================
+    // The whole warp runs this role, converged: the MMAs and commits are predicated on one elected lane and take ready
+    // 64-bit descriptors (next to busy warps that issues several times faster than a lane-0 branch, see tc_common.cuh).
+    {
+      const uint32_t elected = elect_one();
       const uint64_t qdesc = make_smem_desc(smem_u32(sQ), 0, 1024, SW_128B);
       const uint64_t kdesc = make_smem_desc(smem_u32(sK), 0, 1024, SW_128B);
       const uint64_t pdesc = make_smem_desc(smem_u32(sP), 0, 1024, SW_128B);
@@ -213,27 +216,25 @@ attention_fused_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
       const uint32_t idesc_o = make_idesc_bf16(128, kD, 0, 1);    // V is N-major
       const uint32_t idesc_s[2] = {make_idesc_bf16(128, (uint32_t)p.hw0), make_idesc_bf16(128, (uint32_t)p.hw1)};
       const int hw[2] = {p.hw0, p.hw1};
-
-      // Descriptors as (low, high) words: the start address lives in the low word, so every operand of the unrolled
-      // issue loops is one 32-bit add away from its base.
-      const uint32_t q_lo = (uint32_t)qdesc, q_hi = (uint32_t)(qdesc >> 32), k_lo = (uint32_t)kdesc, k_hi = (uint32_t)(kdesc >> 32);
-      const uint32_t p_lo = (uint32_t)pdesc, p_hi = (uint32_t)(pdesc >> 32), v_lo = (uint32_t)vdesc, v_hi = (uint32_t)(vdesc >> 32);
       auto issue_scores = [&](int half) {
-        const uint32_t b0 = k_lo + ((uint32_t)(half * p.hw0 * kD * 2) >> 4);
+        const uint64_t b0 = kdesc + (uint64_t)((uint32_t)(half * p.hw0 * kD * 2) >> 4);
+        const uint32_t d = tmem_base + half * kHalfCols;
+        umma_bf16_elected<false>(d, qdesc, b0, idesc_s[half], elected);
 #pragma unroll
-        for (int ks = 0; ks < kD / 16; ++ks)
-          umma_bf16_lohi(tmem_base + half * kHalfCols, q_lo + 2u * ks, q_hi, b0 + 2u * ks, k_hi, idesc_s[half], ks > 0);
-        umma_commit(bar_s + half);
+        for (int ks = 1; ks < kD / 16; ++ks) umma_bf16_elected<true>(d, qdesc + 2u * ks, b0 + 2u * ks, idesc_s[half], elected);
+        umma_commit_elected(bar_s + half, elected);
       };
       auto issue_pv = [&](int half) {
-        const uint32_t a0 = p_lo + ((uint32_t)(half * p.p_half_bytes) >> 4);
-        const uint32_t b0 = v_lo + ((uint32_t)(half * p.hw0 * kD * 2) >> 4);
+        const uint64_t a0 = pdesc + (uint64_t)((uint32_t)(half * p.p_half_bytes) >> 4);
+        const uint64_t b0 = vdesc + (uint64_t)((uint32_t)(half * p.hw0 * kD * 2) >> 4);
+        const uint32_t d = tmem_base + kOCol + half * kD;
         const int ksteps = hw[half] / 16;
+        umma_bf16_elected<false>(d, a0, b0, idesc_o, elected);
 #pragma unroll
-        for (int ks = 0; ks < kHalfCols / 16; ++ks)
+        for (int ks = 1; ks < kHalfCols / 16; ++ks)
           if (ks < ksteps)
-            umma_bf16_lohi(tmem_base + kOCol + half * kD, a0 + (uint32_t)(((ks >> 2) * kBlockM * 128 + (ks & 3) * 32) >> 4), p_hi,
-                           b0 + (uint32_t)((ks * 16 * kD * 2) >> 4), v_hi, idesc_o, ks != 0);
+            umma_bf16_elected<true>(d, a0 + (uint64_t)(((ks >> 2) * kBlockM * 128 + (ks & 3) * 32) >> 4),
+                                    b0 + (uint64_t)((ks * 16 * kD * 2) >> 4), idesc_o, elected);
       };
 
       mbar_wait(bar_k, 0, abort_flag, p.status, 0x202);
@@ -241,7 +242,7 @@ attention_fused_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
       tcgen05_fence_after_sync();
       issue_scores(0);
       issue_scores(1);
-      umma_commit(bar_qfree);
+      umma_commit_elected(bar_qfree, elected);
       int t = t0;
       uint32_t head_ph = 0;      // parity of the K / V loads of the current head
       bool first_of_head = true;
@@ -260,21 +261,21 @@ attention_fused_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
         if (i > 0) mbar_wait(bar_ofree + 0, ph ^ 1u, abort_flag, p.status, 0x206);
         tcgen05_fence_after_sync();
         issue_pv(0);
-        umma_commit(bar_o + 0);
-        umma_commit(bar_pfree + 0);
+        umma_commit_elected(bar_o + 0, elected);
+        umma_commit_elected(bar_pfree + 0, elected);
         // ---- half 1 ----
         mbar_wait(bar_p + 1, ph, abort_flag, p.status, 0x208);
         tcgen05_fence_after_sync();
         if (i + 1 < n) {
           issue_scores(1);
-          umma_commit(bar_qfree);
+          umma_commit_elected(bar_qfree, elected);
         }
         if (i > 0) mbar_wait(bar_ofree + 1, ph ^ 1u, abort_flag, p.status, 0x209);
         tcgen05_fence_after_sync();
         issue_pv(1);
-        umma_commit(bar_o + 1);
-        umma_commit(bar_pfree + 1);
-        if (last_of_head) umma_commit(bar_vfree);
+        umma_commit_elected(bar_o + 1, elected);
+        umma_commit_elected(bar_pfree + 1, elected);
+        if (last_of_head) umma_commit_elected(bar_vfree, elected);
         first_of_head = last_of_head;
         if (last_of_head) { t = 0; head_ph ^= 1u; } else ++t;
       }
