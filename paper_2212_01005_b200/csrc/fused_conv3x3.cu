@@ -140,7 +140,10 @@ conv3x3_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
   } else if (warp > kEpiWarps) {
     // ================================ MMA issuers ================================
     const int iw = warp - kEpiWarps - 1;   // issuer iw takes tiles lo + iw, lo + iw + kMmaWarps, ...
-    if (lane == 0) {
+    // Each issuing warp runs its loop converged; MMAs and commits are predicated on one elected lane and take ready
+    // 64-bit descriptors (several times the issue rate of a lane-0 branch next to busy warps, see tc_common.cuh).
+    {
+      const uint32_t elected = elect_one();
       const uint32_t idesc = make_idesc_bf16(128, (uint32_t)p.C);
       const uint64_t wdesc0 = make_smem_desc(smem_u32(sW), 0, 8u * p.w_row_bytes, p.w_swizzle);
       mbar_wait(bar_x, 0, abort_flag, p.status, 0x402);
@@ -149,13 +152,13 @@ conv3x3_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
         const int conv = ps >> 1, grp = ps & 1;
         uint64_t* done = (conv == 0 ? bar_acc1 : bar_acc2) + grp;
         if (conv == 1 && !SINGLE) mbar_wait(bar_y + grp, 0, abort_flag, p.status, 0x403);   // the intermediate rows this group reads are written
-        if (pass_lo[ps] >= pass_hi[ps]) { umma_commit(done); continue; }
+        if (pass_lo[ps] >= pass_hi[ps]) { umma_commit_elected(done, elected); continue; }
         // A: swizzled [pixel][channel] rows; K step = 32 bytes inside a row, 8-row groups are 8 rows apart (SBO).
         // Descriptor arithmetic is hoisted: one add per tile, constant strides per K step.
         const uint32_t rowu = (uint32_t)p.w_row_bytes >> 4;   // one pixel row in 16-byte units
         const uint64_t adesc0 = make_smem_desc(smem_u32(conv == 0 ? sX : sY), 0, 8u * p.w_row_bytes, p.w_swizzle);
-        const uint32_t a_kstep = 2u;
         const int lo = pass_lo[ps], hi = pass_hi[ps];
+        const uint64_t a_tile_step = (uint64_t)(kMmaWarps * 128 * rowu);
         tcgen05_fence_after_sync();
         for (int tap = 0; tap < 9; ++tap) {
           const int s = i % p.wstages;
@@ -165,26 +168,26 @@ conv3x3_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
           }
           const int shift = (tap / 3) * p.Wp + (tap % 3) - 1;     // pixels = 16-byte units
           const uint64_t bdesc = wdesc0 + (uint64_t)((uint32_t)((s * 3 + tap % 3) * p.w_stage_bytes) >> 4);
-          // all per-MMA arithmetic is 32-bit adds on the descriptors' low words
-          const uint32_t a_hi = (uint32_t)(adesc0 >> 32), b_hi = (uint32_t)(bdesc >> 32), b_lo = (uint32_t)bdesc;
-          uint32_t a_lo = (uint32_t)adesc0 + (uint32_t)((lo + iw) * 128 + shift) * rowu;
+          // (lo + iw) * 128 + shift may be negative for the first tile's first taps: the add wraps in the address field
+          // exactly as the 32-bit add on the descriptor's low word did
+          uint64_t a = (adesc0 & 0xffffffff00000000ull) |
+                       (uint64_t)((uint32_t)adesc0 + (uint32_t)((lo + iw) * 128 + shift) * rowu);
           uint32_t d_tmem = tmem_base + (lo + iw) * p.C;
-          const uint32_t acc0 = tap != 0;
           if (ksteps == 4) {
-            for (int mt = lo + iw; mt < hi; mt += kMmaWarps, a_lo += kMmaWarps * 128 * rowu, d_tmem += kMmaWarps * p.C) {
-              umma_bf16_lohi(d_tmem, a_lo, a_hi, b_lo, b_hi, idesc, acc0);
-              umma_bf16_lohi(d_tmem, a_lo + a_kstep, a_hi, b_lo + 2, b_hi, idesc, 1);
-              umma_bf16_lohi(d_tmem, a_lo + 2 * a_kstep, a_hi, b_lo + 4, b_hi, idesc, 1);
-              umma_bf16_lohi(d_tmem, a_lo + 3 * a_kstep, a_hi, b_lo + 6, b_hi, idesc, 1);
+            for (int mt = lo + iw; mt < hi; mt += kMmaWarps, a += a_tile_step, d_tmem += kMmaWarps * p.C) {
+              umma_bf16_elected_acc(d_tmem, a, bdesc, idesc, elected, tap != 0);
+              umma_bf16_elected<true>(d_tmem, a + 2u, bdesc + 2u, idesc, elected);
+              umma_bf16_elected<true>(d_tmem, a + 4u, bdesc + 4u, idesc, elected);
+              umma_bf16_elected<true>(d_tmem, a + 6u, bdesc + 6u, idesc, elected);
             }
           } else {
-            for (int mt = lo + iw; mt < hi; mt += kMmaWarps, a_lo += kMmaWarps * 128 * rowu, d_tmem += kMmaWarps * p.C)
+            for (int mt = lo + iw; mt < hi; mt += kMmaWarps, a += a_tile_step, d_tmem += kMmaWarps * p.C)
               for (int ks = 0; ks < ksteps; ++ks)
-                umma_bf16_lohi(d_tmem, a_lo + ks * a_kstep, a_hi, b_lo + 2 * ks, b_hi, idesc, ks ? 1u : acc0);
+                umma_bf16_elected_acc(d_tmem, a + 2u * ks, bdesc + 2u * ks, idesc, elected, (ks | tap) != 0);
           }
-          if (tap % 3 == 2) { umma_commit(bar_empty + s); ++i; }
+          if (tap % 3 == 2) { umma_commit_elected(bar_empty + s, elected); ++i; }
         }
-        umma_commit(done);
+        umma_commit_elected(done, elected);
       }
     }
     __syncwarp();
