@@ -151,7 +151,9 @@ ffn_fused_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
     __syncwarp();
   } else if (warp == kEpiWarps + 1) {
     // ================================ MMA issuer ================================
-    if (lane == 0) {
+    // the whole warp, converged; MMAs and commits predicated on one elected lane (see tc_common.cuh)
+    {
+      const uint32_t elected = elect_one();
       const uint32_t idesc = make_idesc_bf16(128, 128, 0, 1);   // A K-major, B N-major (weights as they lie in HBM)
       int s = 0, round = 0;
       // first GEMM: Hacc[g & 1][128 x 128] = X * W1[:, tile g]
@@ -169,11 +171,11 @@ ffn_fused_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
           const uint64_t bd = make_smem_desc(st + 16384, 8192, 1024, SW_128B);
 #pragma unroll
           for (int ks = 0; ks < kBK / 16; ++ks)
-            umma_bf16(tmem_base + b * kBH, ad + 2u * ks, bd + (uint64_t)((ks * 2048) >> 4), idesc, (kb | ks) != 0);
-          umma_commit(bar_empty + s);
+            umma_bf16_elected_acc(tmem_base + b * kBH, ad + 2u * ks, bd + (uint64_t)((ks * 2048) >> 4), idesc, elected, (kb | ks) != 0);
+          umma_commit_elected(bar_empty + s, elected);
           if (++s == stages) { s = 0; ++round; }
         }
-        umma_commit(bar_hacc + b);
+        umma_commit_elected(bar_hacc + b, elected);
       }
       // second GEMM: acc[u & 1][128 x 128] = sum over the G tiles of H_g * W2[tile g, slice u]
       for (int u = 0; u < p.nslices; ++u) {
@@ -190,12 +192,12 @@ ffn_fused_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
           const uint64_t bd = make_smem_desc(smem_u32(sRing + s * kStageBytes), 16384, 1024, SW_128B);
 #pragma unroll
           for (int ks = 0; ks < kBH / 16; ++ks)
-            umma_bf16(tmem_base + kOutCol + ab * kBN, hdesc + (uint64_t)(((ks >> 2) * kBM * 128 + (ks & 3) * 32) >> 4),
-                      bd + (uint64_t)((ks * 2048) >> 4), idesc, (g | ks) != 0);
-          umma_commit(bar_empty + s);
+            umma_bf16_elected_acc(tmem_base + kOutCol + ab * kBN, hdesc + (uint64_t)(((ks >> 2) * kBM * 128 + (ks & 3) * 32) >> 4),
+                      bd + (uint64_t)((ks * 2048) >> 4), idesc, elected, (g | ks) != 0);
+          umma_commit_elected(bar_empty + s, elected);
           if (++s == stages) { s = 0; ++round; }
         }
-        umma_commit(bar_out + ab);
+        umma_commit_elected(bar_out + ab, elected);
       }
     }
     __syncwarp();

@@ -175,7 +175,9 @@ ffn_cluster_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
     __syncwarp();
   } else if (warp == kEpiWarps + 1) {
     // ================================ MMA issuer ================================
-    if (lane == 0) {
+    // the whole warp, converged; MMAs and commits predicated on one elected lane (see tc_common.cuh)
+    {
+      const uint32_t elected = elect_one();
       const uint32_t idesc1 = make_idesc_bf16(128, kBH, 0, 1);              // A K-major, B N-major (weights as they lie in memory)
       const uint32_t idesc2 = make_idesc_bf16(128, (uint32_t)p.NC, 0, 1);
       int s = 0, round = 0;
@@ -194,11 +196,11 @@ ffn_cluster_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
           const uint64_t bd = make_smem_desc(st + 16384, 8192, 1024, SW_128B);
 #pragma unroll
           for (int ks = 0; ks < kBK / 16; ++ks)
-            umma_bf16(tmem_base + b * kBH, ad + 2u * ks, bd + (uint64_t)((ks * 2048) >> 4), idesc1, (kb | ks) != 0);
-          umma_commit(bar_empty + s);
+            umma_bf16_elected_acc(tmem_base + b * kBH, ad + 2u * ks, bd + (uint64_t)((ks * 2048) >> 4), idesc1, elected, (kb | ks) != 0);
+          umma_commit_elected(bar_empty + s, elected);
           advance();
         }
-        umma_commit(bar_hacc + b);
+        umma_commit_elected(bar_hacc + b, elected);
       };
       if (steps > 0) g1(0);
       for (int step = 0; step < steps; ++step) {
@@ -217,14 +219,14 @@ ffn_cluster_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
             const uint64_t bd = make_smem_desc(smem_u32(sRing + s * kStageBytes), 8192, 1024, SW_128B);
 #pragma unroll
             for (int ks = 0; ks < 4; ++ks)
-              umma_bf16(tmem_base + kOutCol, hd + 2u * ks, bd + (uint64_t)((ks * 2048) >> 4), idesc2, (t | k | h | ks) != 0);
-            umma_commit(bar_empty + s);
+              umma_bf16_elected_acc(tmem_base + kOutCol, hd + 2u * ks, bd + (uint64_t)((ks * 2048) >> 4), idesc2, elected, (t | k | h | ks) != 0);
+            umma_commit_elected(bar_empty + s, elected);
             advance();
           }
           // slot k of this CTA has been read: tell its producer (CTA k)
-          umma_commit_cluster(cluster_map(smem_u32(bar_hdone), (uint32_t)k));
+          umma_commit_cluster_elected(cluster_map(smem_u32(bar_hdone), (uint32_t)k), elected);
         }
-        if (t == T - 1) umma_commit(bar_out);
+        if (t == T - 1) umma_commit_elected(bar_out, elected);
       }
     }
     __syncwarp();

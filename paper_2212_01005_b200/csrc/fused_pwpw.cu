@@ -171,8 +171,9 @@ pwpw_fused_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
       const int g = m / ab, rem = m - g * ab, i = rem / p.perm_b, j = rem - i * p.perm_b;
       sRows[tid] = (g * p.perm_b + j) * p.perm_a + i;
     }
-    // ---- P2: first product ----
-    if (tid == 0) {
+    // ---- P2: first product (warp 0, converged; MMAs predicated on one elected lane, see tc_common.cuh) ----
+    if (warp == 0) {
+      const uint32_t elected = elect_one();
       mbar_wait(bar_x, par, abort_flag, p.status, 0x600);
       tcgen05_fence_after_sync();
       for (int kb = 0; kb < p.nkb0; ++kb) {
@@ -183,9 +184,9 @@ pwpw_fused_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
                                        : make_smem_desc(smem_u32(sW1 + kb * p.w1_block), 0, 1024, SW_128B);
         const uint32_t bstep = p.w_nmajor ? 2048u >> 4 : 2u;
         const int ksteps = min(4, (p.C0p - kb * kBK) / 16);
-        for (int ks = 0; ks < ksteps; ++ks) umma_bf16(tmem_base, ad + 2u * ks, bd + bstep * ks, idesc1, (kb | ks) != 0);
+        for (int ks = 0; ks < ksteps; ++ks) umma_bf16_elected_acc(tmem_base, ad + 2u * ks, bd + bstep * ks, idesc1, elected, (kb | ks) != 0);
       }
-      umma_commit(bar_m1);
+      umma_commit_elected(bar_m1, elected);
     }
     __syncwarp();
     mbar_wait(bar_m1, par, abort_flag, p.status, 0x601);
@@ -227,16 +228,17 @@ pwpw_fused_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
     __syncthreads();
     tcgen05_fence_after_sync();
     // ---- P4: second product, over the drained columns of the first ----
-    if (tid == 0) {
+    if (warp == 0) {
+      const uint32_t elected = elect_one();
       for (int kb = 0; kb < p.nkb1; ++kb) {
         const uint64_t ad = make_smem_desc(smem_u32(sA + kb * kXBlock), 0, 1024, SW_128B);
         const uint64_t bd = p.w_nmajor ? make_smem_desc(smem_u32(sW2 + kb * 4 * 2048), (uint32_t)p.w2_block, 1024, SW_128B)
                                        : make_smem_desc(smem_u32(sW2 + kb * p.w2_block), 0, 1024, SW_128B);
         const uint32_t bstep = p.w_nmajor ? 2048u >> 4 : 2u;
         const int ksteps = min(4, (p.C1p - kb * kBK) / 16);
-        for (int ks = 0; ks < ksteps; ++ks) umma_bf16(tmem_base, ad + 2u * ks, bd + bstep * ks, idesc2, (kb | ks) != 0);
+        for (int ks = 0; ks < ksteps; ++ks) umma_bf16_elected_acc(tmem_base, ad + 2u * ks, bd + bstep * ks, idesc2, elected, (kb | ks) != 0);
       }
-      umma_commit(bar_m2);
+      umma_commit_elected(bar_m2, elected);
     }
     __syncwarp();
     mbar_wait(bar_m2, par, abort_flag, p.status, 0x602);

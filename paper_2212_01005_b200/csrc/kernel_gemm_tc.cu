@@ -118,7 +118,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
     __syncwarp();
   } else if (warp == kEpiThreads / 32 + 1) {
     // ================================ MMA issuer ================================
-    if (lane == 0) {
+    // the whole warp, converged; MMAs and commits predicated on one elected lane (see tc_common.cuh)
+    {
+      const uint32_t elected = elect_one();
       const uint32_t idesc = make_idesc_bf16(128, (uint32_t)ncols, 0, p.b_kmajor ? 0 : 1);
       for (int i = 0; i < p.kblocks; ++i) {
         const int s = i % kStages;
@@ -129,10 +131,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
         const uint64_t bd = p.b_kmajor ? make_smem_desc(st + 16384, 0, 1024, SW_128B) : make_smem_desc(st + 16384, 8192, 1024, SW_128B);
 #pragma unroll
         for (int ks = 0; ks < kBK / 16; ++ks)
-          umma_bf16(tmem_base, ad + 2u * ks, bd + (p.b_kmajor ? (uint64_t)(2u * ks) : (uint64_t)((ks * 2048) >> 4)), idesc, (i | ks) != 0);
-        umma_commit(bar_empty + s);
+          umma_bf16_elected_acc(tmem_base, ad + 2u * ks, bd + (p.b_kmajor ? (uint64_t)(2u * ks) : (uint64_t)((ks * 2048) >> 4)), idesc, elected, (i | ks) != 0);
+        umma_commit_elected(bar_empty + s, elected);
       }
-      if (!skip_signal_for_test(p.status, 0x503)) umma_commit(bar_acc);
+      if (!skip_signal_for_test(p.status, 0x503)) umma_commit_elected(bar_acc, elected);
     }
     __syncwarp();
   } else {

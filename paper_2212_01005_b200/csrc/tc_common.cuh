@@ -346,6 +346,14 @@ __device__ __forceinline__ void umma_bf16_elected_acc(uint32_t d_tmem, uint64_t 
       ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(elected), "r"(accumulate)
       : "memory");
 }
+__device__ __forceinline__ void umma_commit_cluster_elected(uint32_t bar_cluster_addr, uint32_t elected) {
+  asm volatile(
+      "{\n\t.reg .pred q;\n\t"
+      "setp.ne.b32 q, %1, 0;\n\t"
+      "@q tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n\t}"
+      ::"r"(bar_cluster_addr), "r"(elected)
+      : "memory");
+}
 __device__ __forceinline__ void umma_commit_elected(uint64_t* bar, uint32_t elected) {
   asm volatile(
       "{\n\t.reg .pred q;\n\t"
