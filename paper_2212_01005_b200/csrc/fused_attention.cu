@@ -28,17 +28,20 @@
 //       buffers -- the next chunk is in flight while the current one is consumed:
 //       p = exp2((s - m_h) * scale * log2 e) -> bf16 -> shared memory (K-major operand) and the row sum, with m_h the
 //       maximum of the row's first 32 scores. Softmax does not depend on the reference value; the true row maximum
-//       only keeps the exponentials in range, and a row sum that comes out too large (or not a number) sends the warp
-//       through the exact path: row maximum over all chunks first, then the probabilities again. Three exponentials
-//       in four run on the special-function unit, the fourth as a cubic on the FMA pipe)
+//       only keeps the exponentials in range: when the last chunk is in registers, the partial row sum (it bounds every
+//       exponential so far) and the last chunk's maximum tell whether it did; if not, the warp keeps the score half,
+//       takes the true row maximum from it and repeats the pass. Three exponentials in four run on the
+//       special-function unit, the fourth as a cubic on the FMA pipe)
 //   P5  tcgen05.mma: O_h[128 x 64] = P_h V_h        (V is the N-major B operand, as it lies in HBM)
 //   P6  four epilogue warps (a query row per thread): TMEM -> registers as soon as a half's product is complete (its
 //       accumulator is released at once), (f_0 O_0 + f_1 O_1) / sum, bf16 -> per warp, pieces of 16 columns x 32 rows
 //       staged in shared memory -> one TMA store per piece (stores from the row-per-lane register layout would touch
 //       32 lines per instruction and hold up the load/store unit that the probability stores need)
 //
-// Issue order of the MMA thread: when a half's probabilities arrive, the next tile's scores of that half go first (its
-// group has nothing else to do) and P_h V second (only the epilogue warps wait for it).
+// Issue order of the MMA warp, per half: as soon as the group has the last chunk of its score half in registers (and the
+// reference has proved good enough), the next tile's scores of that half, so that the group finds them ready when it has
+// written its last probabilities; when the probabilities have arrived, P_h V in blocks of 64 keys, each block's
+// completion releasing that block of the probability buffer for the next tile.
 #include <cuda.h>
 #include <cuda_bf16.h>
 
@@ -69,7 +72,8 @@ constexpr int kHalfCols = 192;         // tensor-memory columns reserved per sco
 // A row's exponentials are taken relative to the maximum of its first 32 scores, not of all of them (any reference gives
 // the same softmax; the true maximum only guarantees the range). A row sum at or above this limit, or not a number, sends
 // the warp through the exact two-pass path.
-constexpr float kSumLimit = 1099511627776.0f;   // 2^40
+constexpr float kSumLimit = 1099511627776.0f;   // 2^40: a partial row sum below it bounds every exponential so far
+constexpr float kRefSlack = 40.0f;              // the reference may lie this many powers of two below the last chunk's maximum
 constexpr uint32_t kOCol = 2 * kHalfCols;   // O_0 at kOCol, O_1 at kOCol + kD
 
 struct AttnParams {
@@ -137,13 +141,14 @@ attention_fused_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
   uint64_t* bar_q = bars + 2;       // Q tile landed
   uint64_t* bar_qfree = bars + 3;   // both score MMAs of the tile have read Q
   uint64_t* bar_s = bars + 4;       // [2] score half complete
-  uint64_t* bar_p = bars + 6;       // [2] probabilities of the half written, score half drained (one arrival per warp)
-  uint64_t* bar_pfree = bars + 8;   // [2] P V of the half has read the probabilities
+  uint64_t* bar_p = bars + 6;       // [2] probabilities of the half written (one arrival per warp)
+  uint64_t* bar_d = bars + 8;       // [2] score half drained: every row of it is in registers (one arrival per warp)
+  uint64_t* bar_pfree = bars + 16;  // [2][3] P V of the half has read 64-key block j of the probabilities
   uint64_t* bar_o = bars + 10;      // [2] P V of the half complete
   uint64_t* bar_ofree = bars + 12;  // [2] the epilogue warps have read the half's output accumulator (one arrival per warp)
   uint64_t* bar_vfree = bars + 14;  // the last P V of a head has read V
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 16);
-  volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(bars + 17);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 22);
+  volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(bars + 23);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   // This CTA's run of items [g0, g0 + n); item g = ((b * heads + h) * tiles + t).
@@ -156,7 +161,7 @@ attention_fused_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
 
   if (tid == kTmaWarp * 32) {
     *abort_flag = 0u;
-    for (int i = 0; i < 16; ++i) mbar_init(bars + i, (i == 6 || i == 7 || i == 12 || i == 13) ? kGroupWarps : 1);
+    for (int i = 0; i < 22; ++i) mbar_init(bars + i, ((i >= 6 && i <= 9) || i == 12 || i == 13) ? kGroupWarps : 1);
     fence_mbar_init();
     fence_proxy_async_smem();
     tma_prefetch_desc(&tmap_q);
@@ -224,17 +229,18 @@ attention_fused_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
         for (int ks = 1; ks < kD / 16; ++ks) umma_bf16_elected<true>(d, qdesc + 2u * ks, b0 + 2u * ks, idesc_s[half], elected);
         umma_commit_elected(bar_s + half, elected);
       };
-      auto issue_pv = [&](int half) {
-        const uint64_t a0 = pdesc + (uint64_t)((uint32_t)(half * p.p_half_bytes) >> 4);
-        const uint64_t b0 = vdesc + (uint64_t)((uint32_t)(half * p.hw0 * kD * 2) >> 4);
+      // P_h V in blocks of 64 keys (four K steps): each block's completion releases that block of the probability buffer
+      auto issue_pv_block = [&](int half, int blk) {
+        const uint64_t a0 = pdesc + (uint64_t)((uint32_t)(half * p.p_half_bytes + blk * kBlockM * 128) >> 4);
+        const uint64_t b0 = vdesc + (uint64_t)((uint32_t)((half * p.hw0 + blk * 64) * kD * 2) >> 4);
         const uint32_t d = tmem_base + kOCol + half * kD;
-        const int ksteps = hw[half] / 16;
-        umma_bf16_elected<false>(d, a0, b0, idesc_o, elected);
+        const int ksteps = hw[half] / 16 - blk * 4;      // K steps left from this block on
+        if (ksteps <= 0) return;
+        umma_bf16_elected_acc(d, a0, b0, idesc_o, elected, blk != 0);
 #pragma unroll
-        for (int ks = 1; ks < kHalfCols / 16; ++ks)
-          if (ks < ksteps)
-            umma_bf16_elected<true>(d, a0 + (uint64_t)(((ks >> 2) * kBlockM * 128 + (ks & 3) * 32) >> 4),
-                                    b0 + (uint64_t)((ks * 16 * kD * 2) >> 4), idesc_o, elected);
+        for (int ks = 1; ks < 4; ++ks)
+          if (ks < ksteps) umma_bf16_elected<true>(d, a0 + (uint64_t)((ks * 32) >> 4), b0 + (uint64_t)((ks * 16 * kD * 2) >> 4), idesc_o, elected);
+        umma_commit_elected(bar_pfree + half * 3 + blk, elected);
       };
 
       mbar_wait(bar_k, 0, abort_flag, p.status, 0x202);
@@ -249,32 +255,39 @@ attention_fused_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
       for (int i = 0; i < n; ++i) {
         const uint32_t ph = (uint32_t)i & 1u;
         const bool last_of_head = t + 1 == p.tiles;   // the next item of the run, if any, belongs to the next head
+        // Per half: score half drained (its last chunk is in the group's registers) -> the next tile's scores of the
+        // half, so that the group finds them ready when it has written its last probabilities; probabilities written ->
+        // P_h V, block by block (each block's completion releases that block of the probability buffer).
         // ---- half 0 ----
-        mbar_wait(bar_p + 0, ph, abort_flag, p.status, 0x204);
         if (i + 1 < n) {
+          mbar_wait(bar_d + 0, ph, abort_flag, p.status, 0x20a);
           mbar_wait(bar_q, ph ^ 1u, abort_flag, p.status, 0x207);
           if (last_of_head) mbar_wait(bar_k, head_ph ^ 1u, abort_flag, p.status, 0x202);
           tcgen05_fence_after_sync();
-          issue_scores(0);                       // next tile's half 0 into the buffer just drained: its group is waiting for it
+          issue_scores(0);
         }
+        mbar_wait(bar_p + 0, ph, abort_flag, p.status, 0x204);
         if (first_of_head) mbar_wait(bar_v, head_ph, abort_flag, p.status, 0x205);
         if (i > 0) mbar_wait(bar_ofree + 0, ph ^ 1u, abort_flag, p.status, 0x206);
         tcgen05_fence_after_sync();
-        issue_pv(0);
+        issue_pv_block(0, 0);
+        issue_pv_block(0, 1);
+        issue_pv_block(0, 2);
         umma_commit_elected(bar_o + 0, elected);
-        umma_commit_elected(bar_pfree + 0, elected);
         // ---- half 1 ----
-        mbar_wait(bar_p + 1, ph, abort_flag, p.status, 0x208);
-        tcgen05_fence_after_sync();
         if (i + 1 < n) {
+          mbar_wait(bar_d + 1, ph, abort_flag, p.status, 0x20b);
+          tcgen05_fence_after_sync();
           issue_scores(1);
           umma_commit_elected(bar_qfree, elected);
         }
+        mbar_wait(bar_p + 1, ph, abort_flag, p.status, 0x208);
         if (i > 0) mbar_wait(bar_ofree + 1, ph ^ 1u, abort_flag, p.status, 0x209);
         tcgen05_fence_after_sync();
-        issue_pv(1);
+        issue_pv_block(1, 0);
+        issue_pv_block(1, 1);
+        issue_pv_block(1, 2);
         umma_commit_elected(bar_o + 1, elected);
-        umma_commit_elected(bar_pfree + 1, elected);
         if (last_of_head) umma_commit_elected(bar_vfree, elected);
         first_of_head = last_of_head;
         if (last_of_head) { t = 0; head_ph ^= 1u; } else ++t;
@@ -369,37 +382,56 @@ attention_fused_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
       mbar_wait(bar_s + grp, ph, abort_flag, p.status, 0x210);
       tcgen05_fence_after_sync();
       tmem_ld_x32(s_addr, va);
-      if (t > 0) {                               // P V of the previous tile has read this half's probability buffer
-        if (lane == 0) mbar_wait(bar_pfree + grp, ph ^ 1u, abort_flag, p.status, 0x211);
-        __syncwarp();
-      }
       wait32(va);
       if (nch > 1) tmem_ld_x32(s_addr + 32u, vb);
       float m = kv >= 32 ? max32(va) : max_tail(va, kv);
       float sum;
+      // Once the last chunk of the row is in registers it is known whether the reference was good enough: the sum of the
+      // exponentials so far bounds every one of them, and the last chunk's maximum is taken directly. If so for every
+      // row of the warp, the score half is released to the next tile's score product at once; otherwise it is kept,
+      // the true row maximum is taken from it, and the pass is repeated before the half is released.
+      auto last_chunk_landed = [&](int attempt, float partial_sum, float last_max) -> bool {
+        const bool exact = attempt == 0 && __any_sync(0xffffffffu, !(partial_sum < kSumLimit) || !((last_max - m) * c < kRefSlack));
+        if (!exact) {
+          tcgen05_fence_before_sync();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(bar_d + grp);
+        }
+        return exact;
+      };
       // The loops below are rolled on purpose: every softmax warp runs the same few hundred instructions per pair of
       // chunks, which stay in the instruction cache, instead of a private stretch of straight-line code per chunk.
 #pragma unroll 1
       for (int attempt = 0;; ++attempt) {
         // ---------------- probabilities and row sum (chunk 0 is in va, chunk 1 on its way to vb) ----------------
+        bool exact = false;
+        if (nch == 1) exact = last_chunk_landed(attempt, 0.0f, m);
         const float mc = m * c;
         float s4[4] = {0.f, 0.f, 0.f, 0.f};
         uint8_t* blk = prow;
 #pragma unroll 1
         for (int ch = 0; ch < nch; ch += 2, blk += kBlockM * 128) {
+          if (t > 0 && attempt == 0) {           // P V of the previous tile has read this 64-key block of the buffer
+            if (lane == 0) mbar_wait(bar_pfree + grp * 3 + (ch >> 1), ph ^ 1u, abort_flag, p.status, 0x211);
+            __syncwarp();
+          }
           if (kv - ch * 32 >= 32) exp32(va, blk, 0u, mc, s4); else exp_tail(va, blk, 0u, hw - ch * 32, kv - ch * 32, mc, s4);
           if (ch + 1 < nch) {
             wait32(vb);
             if (ch + 2 < nch) tmem_ld_x32(s_addr + (uint32_t)((ch + 2) * 32), va);
+            else exact = last_chunk_landed(attempt, (s4[0] + s4[1]) + (s4[2] + s4[3]),
+                                           kv - ch * 32 >= 64 ? max32(vb) : max_tail(vb, kv - ch * 32 - 32));
             if (kv - ch * 32 >= 64) exp32(vb, blk, 4u, mc, s4); else exp_tail(vb, blk, 4u, hw - ch * 32 - 32, kv - ch * 32 - 32, mc, s4);
             if (ch + 2 < nch) {
               wait32(va);
               if (ch + 3 < nch) tmem_ld_x32(s_addr + (uint32_t)((ch + 3) * 32), vb);
+              else exact = last_chunk_landed(attempt, (s4[0] + s4[1]) + (s4[2] + s4[3]),
+                                             kv - ch * 32 >= 96 ? max32(va) : max_tail(va, kv - ch * 32 - 64));
             }
           }
         }
         sum = (s4[0] + s4[1]) + (s4[2] + s4[3]);
-        if (attempt == 1 || !__any_sync(0xffffffffu, !(sum < kSumLimit))) break;
+        if (!exact) break;
         // ---------------- exact path: the row maximum over all chunks first ----------------
         m = -INFINITY;
 #pragma unroll 1
