@@ -8,21 +8,40 @@
 // computes R + 2 rows of the first convolution (2 of them recomputed by the
 // neighbouring strips) from R + 4 input rows.
 //
-// Both convolutions are implicit GEMMs on tcgen05: the activation tile sits in
-// shared memory as [pixel][channels] rows in the swizzled K-major operand layout
-// (exactly what one TMA box load produces), with pixels linearised over the
-// PADDED width, so the operand of filter tap (dr, dc) is the same matrix at a
-// start address shifted by (dr * Wp + dc - 1) rows. The swizzle is a function of
-// the absolute shared-memory address, so such row-shifted start addresses are
-// valid operands (verified on the device against a known matrix). Weights stream
-// through a TMA ring, one filter row (3 taps) per stage.
+// Both convolutions are implicit GEMMs on tcgen05. The three taps of a filter row
+// share their A operand: one MMA with N = 3 C multiplies a 128-pixel tile by
+// [W(dr,0) | W(dr,1) | W(dr,2)] and accumulates three partial sums
+// D_dc[q] = sum_dr x[q + dr rows] W(dr,dc) side by side in tensor memory (12 MMAs
+// of N = 192 per tile for 64 channels instead of 36 of N = 64: with N = 64 the
+// tensor pipe waits for its shared-memory operands, 6 KB per 32 cycles of
+// arithmetic; with N = 192 it is 10 KB per 96). The output is
+// out[q + 1] = D_0[q] + D_1[q + 1] + D_2[q + 2]; tcgen05.shift moves D_1 one row
+// and D_2 two rows towards row 0 so that the three terms of an output sit in the
+// same TMEM lane and the epilogue only adds them. The shift works inside each
+// block of 32 lanes (a block's last row keeps its value), which fixes the layout:
+//
+//   * the image width is cut into segments of 28 output columns; a segment's
+//     activations are [row][32 pixels][channels] in shared memory (swizzled
+//     K-major rows, one TMA box per segment, zero outside the image): 32 input
+//     columns -> 30 columns of the intermediate -> 28 output columns, the two
+//     columns lost per convolution being the ones a 32-lane block cannot shift in;
+//   * a 128-row MMA tile is four image rows of one segment, one row per 32-lane
+//     block; the operand of filter row dr is the same matrix 32 pixels further;
+//   * the intermediate value of (row, pixel j) is produced in the TMEM lane of
+//     pixel j and written over the input at the same place (every later tile
+//     reads rows further down), so the second convolution runs on the same
+//     addresses.
+//
+// All nine taps of one convolution stay resident (three slots of one filter row
+// each); the second convolution's rows replace the first's slot by slot as the
+// last tile of the first convolution releases them.
 //
 //   P1  TMA: input strip with halo -> swizzled [pixel][channel] rows, zero outside the image
-//   P2  tcgen05.mma: 9 taps x (I / 16) K-steps per 128-pixel tile            (TMEM)
-//   P3  TMEM -> registers: + b1, ReLU, zero outside the image (the second
+//   P2  tcgen05.mma: 3 filter rows x (I / 16) K-steps per tile, N = 3 C; tcgen05.shift   (TMEM, two tiles in flight)
+//   P3  TMEM -> registers: sum of the three aligned terms, + b1, ReLU, zero outside the image (the second
 //       convolution pads the post-activation tensor), bf16 -> swizzled rows in shared memory
-//   P5  tcgen05.mma: second convolution over the resident rows               (TMEM)
-//   P6  TMEM -> registers: + b2 + x, ReLU, bf16, 16-byte stores
+//   P5  tcgen05.mma: second convolution over the resident rows                           (TMEM)
+//   P6  TMEM -> registers: sum, + b2 + x, ReLU, bf16, 16-byte stores
 #include <cuda.h>
 #include <cuda_bf16.h>
 
@@ -40,11 +59,12 @@ namespace {
 
 using namespace tc;
 
-constexpr int kEpiWarps = 16;                // four per TMEM lane quarter: each takes a quarter of the channels (at least 16)
+constexpr int kEpiWarps = 16;                // four per TMEM lane quarter: each takes 16 channels
 constexpr int kEpiThreads = kEpiWarps * 32;
-constexpr int kMmaWarps = 4;                 // one issuing lane each, alternating M tiles: a single thread issues an MMA every ~70 cycles, the tensor pipe takes one every ~50
-constexpr int kThreads = kEpiThreads + 32 + 32 * kMmaWarps;   // + TMA warp + MMA warps
-constexpr int kMaxWStages = 4;     // ring stages; each holds one filter row = 3 taps
+constexpr int kShiftWarps = 2;
+constexpr int kThreads = kEpiThreads + 64 + 32 * kShiftWarps;   // + TMA warp + MMA warp + shift warps
+constexpr int kSegCols = 28;                 // output columns per segment (32 input columns, 30 of the intermediate)
+constexpr int kMaxTiles1 = 32;               // tiles of the first convolution (one "rows written" barrier each)
 
 struct ConvParams {
   const __nv_bfloat16* x;
@@ -53,58 +73,64 @@ struct ConvParams {
   __nv_bfloat16* out;
   unsigned int* status;
   int N, H, W, C;          // C = input = middle = output channels
-  int R, strips, IH, Wp, P1, M1, P2, M2;
-  int a1, a2;              // tiles [0,a1) of conv1 / [0,a2) of conv2 form the first pipeline group
-  int stage_ok;            // the first 16 KB of the input rows are free for output staging whenever an output epilogue runs
+  int R, strips, IH;       // output rows per strip, strips per image, input rows per strip (R + 4; R + 2 for one convolution)
+  int NS, T1, T2, M1, M2;  // segments; tile rows (4 image rows each) and tiles (NS per tile row) of either convolution
+  int nact;                // epilogue warps that own channels: 4 * min(4, C / 16)
+  int stage_mode;          // output staging: 0 none (direct stores), 1 in the input rows that no valid output reads, 2 own area
   // single-convolution variant (a stage of the unfused mode): out = [relu](conv(x) + b2 [+ res])
   const __nv_bfloat16* res; // residual tensor (the pair kernel adds its own input)
   int residual, relu;
-  int w_row_bytes, w_swizzle, w_stage_bytes;
-  int wstages;             // ring stages in use (2..kMaxWStages)
-  int off_x, off_y, off_w, off_bias, off_bar;
-  uint32_t wp_recip;        // 2^32 / Wp + 1: pixel index -> (row, column) of the padded strip without a division
+  int w_row_bytes, w_swizzle, w_tap_bytes;
+  int off_x, off_w, off_bias, off_stage, off_bar;
 };
 
 // SINGLE = false: the fused pair. SINGLE = true: one convolution with its simple operators (second-convolution
-// passes only, reading the input rows directly), the tensor-core stage kernel of the unfused mode.
+// tiles only, reading the input rows directly), the tensor-core stage kernel of the unfused mode.
 template <bool SINGLE>
 __global__ void __launch_bounds__(kThreads, 1)
 conv3x3_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w1,
                     const __grid_constant__ CUtensorMap tmap_w2, const ConvParams p) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  uint8_t* sX = smem + p.off_x;   // first pixel row (1024-aligned; slack lies before it)
-  uint8_t* sY = smem + p.off_y;   // the intermediate rows reuse the input rows' memory, two pixels lower
-  uint8_t* sW = smem + p.off_w;
+  uint8_t* sX = smem + p.off_x;   // [segment][row][32 pixels][C]; the intermediate overwrites it in place
+  uint8_t* sW = smem + p.off_w;   // [3 filter rows][3 taps][C rows]
   float* sBias = reinterpret_cast<float*>(smem + p.off_bias);   // b1[C], b2[C]
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + p.off_bar);
-  uint64_t* bar_x = bars;                      // input strip landed
-  uint64_t* bar_full = bars + 1;                  // [kMaxWStages] filter row landed
-  uint64_t* bar_empty = bars + 1 + kMaxWStages;   // [kMaxWStages] filter row consumed
-  uint64_t* bar_acc1 = bars + 1 + 2 * kMaxWStages;   // [2] first convolution, tile group g complete
-  uint64_t* bar_y = bar_acc1 + 2;                 // [2] intermediate rows of group g written
-  uint64_t* bar_acc2 = bar_acc1 + 4;              // [2] second convolution, tile group g complete
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bar_acc1 + 6);
-  volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(bar_acc1 + 7);
+  uint64_t* bar_x = bars;                 // input strip landed
+  uint64_t* bar_wfull = bars + 1;         // [3] filter row landed (phase 0: first convolution, phase 1: second)
+  uint64_t* bar_wfree = bars + 4;         // [3] filter row of the first convolution no longer read
+  uint64_t* bar_acc = bars + 7;           // [2] accumulator of a tile complete (products and shifts)
+  uint64_t* bar_mma = bars + 13 + kMaxTiles1;   // [2] products of a tile complete
+  uint64_t* bar_shq = bars + 15 + kMaxTiles1;   // [2] shifts of a tile issued
+  uint64_t* bar_accfree = bars + 9;       // [2] accumulator read out by every epilogue warp
+  uint64_t* bar_y = bars + 11;            // [kMaxTiles1] intermediate rows of a tile written
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 11 + kMaxTiles1);
+  volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(bars + 12 + kMaxTiles1);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int n = blockIdx.x / p.strips, strip = blockIdx.x % p.strips;
   const int h0 = strip * p.R;
   const int rows_valid = min(p.R, p.H - h0);
   const int ksteps = p.C / 16;
+  const int ntiles = p.M1 + p.M2;          // tile sequence: first convolution's tiles, then the second's
+  const uint32_t nacc = 3u * (uint32_t)p.C;   // accumulator columns of a tile
+  const uint32_t seg_bytes = (uint32_t)(p.IH * 32 * p.w_row_bytes);
 
   grid_dependency_wait();      // the previous grid of the stream has completed; device memory may be touched
   grid_launch_dependents();
   if (tid == kEpiThreads) {
     *abort_flag = 0u;
     mbar_init(bar_x, 1);
-    for (int i = 0; i < kMaxWStages; ++i) { mbar_init(bar_full + i, 1); mbar_init(bar_empty + i, kMmaWarps); }
-    for (int i = 0; i < 6; ++i) mbar_init(bar_acc1 + i, (i == 2 || i == 3) ? 1 : kMmaWarps);   // bar_y is arrived by one epilogue thread
+    for (int i = 0; i < 3; ++i) { mbar_init(bar_wfull + i, 1); mbar_init(bar_wfree + i, 1); }
+    for (int i = 0; i < 2; ++i) { mbar_init(bar_acc + i, kShiftWarps); mbar_init(bar_mma + i, 1); mbar_init(bar_shq + i, kShiftWarps); mbar_init(bar_accfree + i, (uint32_t)p.nact); }
+    for (int i = 0; i < kMaxTiles1; ++i) mbar_init(bar_y + i, (uint32_t)p.nact);
     fence_mbar_init();
     fence_proxy_async_smem();
     tma_prefetch_desc(&tmap_x);
-    mbar_arrive_expect_tx(bar_x, (uint32_t)(p.IH * p.Wp * p.w_row_bytes));
-    tma_load_4d(sX, &tmap_x, bar_x, 0, -1, SINGLE ? h0 - 1 : h0 - 2, n);
+    mbar_arrive_expect_tx(bar_x, (uint32_t)p.NS * seg_bytes);
+    // segment s: 32 columns from 28 s - 2 (one convolution: 28 s - 1), rows from h0 - 2 (h0 - 1); zero outside the image
+    for (int s = 0; s < p.NS; ++s)
+      tma_load_4d(sX + (size_t)s * seg_bytes, &tmap_x, bar_x, 0, s * kSegCols - (SINGLE ? 1 : 2), SINGLE ? h0 - 1 : h0 - 2, n);
   }
   if (warp == 0) {
     tmem_alloc(tmem_slot, 512);
@@ -116,216 +142,216 @@ conv3x3_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
   tcgen05_fence_after_sync();
   const uint32_t tmem_base = *tmem_slot;
 
-  // The four MMA passes: (convolution, tile group) = (1,A) (1,B) (2,A) (2,B); each streams the 9 taps.
-  const int pass_lo[4] = {0, SINGLE ? 0 : p.a1, 0, p.a2};
-  const int pass_hi[4] = {SINGLE ? 0 : p.a1, SINGLE ? 0 : p.M1, p.a2, p.M2};
-
   if (warp == kEpiWarps) {
-    // ================================ TMA producer: weight taps ================================
+    // ================================ TMA producer: filter rows ================================
     if (lane == 0) {
       tma_prefetch_desc(&tmap_w1); tma_prefetch_desc(&tmap_w2);
-      int i = 0;
-      for (int ps = 0; ps < 4; ++ps) {
-        if (pass_lo[ps] >= pass_hi[ps]) continue;      // empty group: the MMA warp skips it too
-        for (int frow = 0; frow < 3; ++frow, ++i) {
-          const int s = i % p.wstages;
-          if (i >= p.wstages) mbar_wait(bar_empty + s, (uint32_t)((i / p.wstages) - 1) & 1u, abort_flag, p.status, 0x401);
-          mbar_arrive_expect_tx(bar_full + s, (uint32_t)(3 * p.C * p.w_row_bytes));
+      for (int conv = SINGLE ? 1 : 0; conv < 2; ++conv) {
+        for (int frow = 0; frow < 3; ++frow) {
+          if (!SINGLE && conv == 1) mbar_wait(bar_wfree + frow, 0, abort_flag, p.status, 0x401);
+          mbar_arrive_expect_tx(bar_wfull + frow, (uint32_t)(3 * p.w_tap_bytes));
           for (int t3 = 0; t3 < 3; ++t3)
-            tma_load_3d(sW + (s * 3 + t3) * p.w_stage_bytes, ps < 2 ? &tmap_w1 : &tmap_w2, bar_full + s, 0, frow * 3 + t3, 0);
+            tma_load_3d(sW + (frow * 3 + t3) * p.w_tap_bytes, conv == 0 ? &tmap_w1 : &tmap_w2, bar_wfull + frow, 0, frow * 3 + t3, 0);
         }
       }
     }
     __syncwarp();
-  } else if (warp > kEpiWarps) {
-    // ================================ MMA issuers ================================
-    const int iw = warp - kEpiWarps - 1;   // issuer iw takes tiles lo + iw, lo + iw + kMmaWarps, ...
-    // Each issuing warp runs its loop converged; MMAs and commits are predicated on one elected lane and take ready
-    // 64-bit descriptors (several times the issue rate of a lane-0 branch next to busy warps, see tc_common.cuh).
-    {
-      const uint32_t elected = elect_one();
-      const uint32_t idesc = make_idesc_bf16(128, (uint32_t)p.C);
-      const uint64_t wdesc0 = make_smem_desc(smem_u32(sW), 0, 8u * p.w_row_bytes, p.w_swizzle);
-      mbar_wait(bar_x, 0, abort_flag, p.status, 0x402);
-      int i = 0;
-      for (int ps = 0; ps < 4; ++ps) {
-        const int conv = ps >> 1, grp = ps & 1;
-        uint64_t* done = (conv == 0 ? bar_acc1 : bar_acc2) + grp;
-        if (conv == 1 && !SINGLE) mbar_wait(bar_y + grp, 0, abort_flag, p.status, 0x403);   // the intermediate rows this group reads are written
-        if (pass_lo[ps] >= pass_hi[ps]) { umma_commit_elected(done, elected); continue; }
-        // A: swizzled [pixel][channel] rows; K step = 32 bytes inside a row, 8-row groups are 8 rows apart (SBO).
-        // Descriptor arithmetic is hoisted: one add per tile, constant strides per K step.
-        const uint32_t rowu = (uint32_t)p.w_row_bytes >> 4;   // one pixel row in 16-byte units
-        const uint64_t adesc0 = make_smem_desc(smem_u32(conv == 0 ? sX : sY), 0, 8u * p.w_row_bytes, p.w_swizzle);
-        const int lo = pass_lo[ps], hi = pass_hi[ps];
-        const uint64_t a_tile_step = (uint64_t)(kMmaWarps * 128 * rowu);
-        tcgen05_fence_after_sync();
-        for (int tap = 0; tap < 9; ++tap) {
-          const int s = i % p.wstages;
-          if (tap % 3 == 0) {
-            mbar_wait(bar_full + s, (uint32_t)(i / p.wstages) & 1u, abort_flag, p.status, 0x404);
-            tcgen05_fence_after_sync();
-          }
-          const int shift = (tap / 3) * p.Wp + (tap % 3) - 1;     // pixels = 16-byte units
-          const uint64_t bdesc = wdesc0 + (uint64_t)((uint32_t)((s * 3 + tap % 3) * p.w_stage_bytes) >> 4);
-          // (lo + iw) * 128 + shift may be negative for the first tile's first taps: the add wraps in the address field
-          // exactly as the 32-bit add on the descriptor's low word did
-          uint64_t a = (adesc0 & 0xffffffff00000000ull) |
-                       (uint64_t)((uint32_t)adesc0 + (uint32_t)((lo + iw) * 128 + shift) * rowu);
-          uint32_t d_tmem = tmem_base + (lo + iw) * p.C;
-          if (ksteps == 4) {
-            for (int mt = lo + iw; mt < hi; mt += kMmaWarps, a += a_tile_step, d_tmem += kMmaWarps * p.C) {
-              umma_bf16_elected_acc(d_tmem, a, bdesc, idesc, elected, tap != 0);
-              umma_bf16_elected<true>(d_tmem, a + 2u, bdesc + 2u, idesc, elected);
-              umma_bf16_elected<true>(d_tmem, a + 4u, bdesc + 4u, idesc, elected);
-              umma_bf16_elected<true>(d_tmem, a + 6u, bdesc + 6u, idesc, elected);
-            }
-          } else {
-            for (int mt = lo + iw; mt < hi; mt += kMmaWarps, a += a_tile_step, d_tmem += kMmaWarps * p.C)
-              for (int ks = 0; ks < ksteps; ++ks)
-                umma_bf16_elected_acc(d_tmem, a + 2u * ks, bdesc + 2u * ks, idesc, elected, (ks | tap) != 0);
-          }
-          if (tap % 3 == 2) { umma_commit_elected(bar_empty + s, elected); ++i; }
-        }
-        umma_commit_elected(done, elected);
+  } else if (warp == kEpiWarps + 1) {
+    // ================================ MMA issuer ================================
+    // The warp runs its loop converged; MMAs and commits are predicated on one elected lane and take ready 64-bit
+    // descriptors (several times the issue rate of a lane-0 branch next to busy warps, see tc_common.cuh).
+    // One issuer, tiles in sequence into alternating accumulators; the shift warps align a tile once its products are complete.
+    const uint32_t elected = elect_one();
+    const uint32_t idesc = make_idesc_bf16(128, nacc);
+    const uint32_t rowu = (uint32_t)(32 * p.w_row_bytes) >> 4;   // one image row of a segment in 16-byte units
+    const uint64_t wdesc0 = make_smem_desc(smem_u32(sW), 0, 8u * p.w_row_bytes, p.w_swizzle);
+    const uint64_t xdesc0 = make_smem_desc(smem_u32(sX), 0, 8u * p.w_row_bytes, p.w_swizzle);
+    const uint32_t frow_step = (uint32_t)(3 * p.w_tap_bytes) >> 4;
+    mbar_wait(bar_x, 0, abort_flag, p.status, 0x402);
+    int w_conv = -1;                       // convolution whose filter rows have been waited for
+    int t = 0, s = 0;                      // tile row and segment of the tile
+    for (int seq = 0; seq < ntiles; ++seq) {
+      if (seq == p.M1) { t = 0; s = 0; }
+      const int conv = seq >= p.M1 ? 1 : 0, buf = seq & 1;
+      if (seq >= 2) mbar_wait(bar_accfree + buf, (uint32_t)((seq >> 1) - 1) & 1u, abort_flag, p.status, 0x403);
+      if (!SINGLE && conv == 1) {
+        // rows 4 t .. 4 t + 5 of the segment's intermediate: its tiles of tile rows t and t + 1
+        mbar_wait(bar_y + t * p.NS + s, 0, abort_flag, p.status, 0x404);
+        if (t + 1 < p.T1) mbar_wait(bar_y + (t + 1) * p.NS + s, 0, abort_flag, p.status, 0x404);
       }
-    }
-    __syncwarp();
-  } else {
-    // ================ epilogue warps: thread = (pixel row of a tile, half of the channels) ================
-    const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
-    const int row = (warp & 3) * 32 + lane;
-    const int ncol = max(16, p.C / (kEpiWarps / 4));
-    const int col0 = (warp >> 2) * ncol;
-    const bool has_cols = col0 < p.C;
-
-    // P3: intermediate = ReLU(acc + b1) inside the image, 0 outside -> swizzled rows; group A, then group B
-    const uint32_t y_addr = smem_u32(sY);
-    const uint32_t swz_mask = ((uint32_t)p.w_row_bytes >> 4) - 1u;
-    // a thread's columns are fixed (ncol == 16 for 16, 32 and 64 channels): its biases stay in registers
-    float bias1[16], bias2[16];
-#pragma unroll
-    for (int j = 0; j < 16; j += 4) {
-      const float4 u = has_cols ? *reinterpret_cast<const float4*>(sBias + col0 + j) : make_float4(0.f, 0.f, 0.f, 0.f);
-      const float4 w = has_cols ? *reinterpret_cast<const float4*>(sBias + p.C + col0 + j) : make_float4(0.f, 0.f, 0.f, 0.f);
-      bias1[j] = u.x; bias1[j + 1] = u.y; bias1[j + 2] = u.z; bias1[j + 3] = u.w;
-      bias2[j] = w.x; bias2[j + 1] = w.y; bias2[j + 2] = w.z; bias2[j + 3] = w.w;
-    }
-    for (int grp = 0; grp < (SINGLE ? 0 : 2); ++grp) {
-      mbar_wait(bar_acc1 + grp, 0, abort_flag, p.status, 0x405);
       tcgen05_fence_after_sync();
-      const int lo1 = grp ? p.a1 : 0, hi1 = grp ? p.M1 : p.a1;   // the group's tiles of the first convolution
-      for (int mt = lo1; mt < hi1 && has_cols; ++mt) {
-        const int m = mt * 128 + row;
-        const int a = (int)fast_div((uint32_t)m, (uint32_t)p.Wp, p.wp_recip), b = m - a * p.Wp;
-        const int gh = h0 - 1 + a;
-        const bool inside = m < p.P1 && gh >= 0 && gh < p.H && b >= 1 && b <= p.W;
-        for (int c0 = col0; c0 < col0 + ncol; c0 += 16) {
-          uint32_t v[16];
-          tmem_ld_x16(tmem_base + lane_base + mt * p.C + c0, v);
-          tmem_ld_wait();
-          uint32_t w[8];
-#pragma unroll
-          for (int j = 0; j < 8; ++j) {
-            const float y0 = fmaxf(__uint_as_float(v[2 * j]) + bias1[2 * j], 0.0f);
-            const float y1 = fmaxf(__uint_as_float(v[2 * j + 1]) + bias1[2 * j + 1], 0.0f);
-            w[j] = inside ? pack_bf16x2(y0, y1) : 0u;
-          }
-          if (m < p.P1 + p.Wp) {   // a little past the tile so that shifted reads of valid rows never see stale data
-            // 16-byte chunk index XOR address bits [7, ..): the swizzle the MMA and TMA apply to absolute addresses
-            uint32_t a0 = y_addr + (uint32_t)m * p.w_row_bytes + (uint32_t)c0 * 2u;
-            uint32_t a1 = a0 + 16u;
-            a0 ^= ((a0 >> 7) & swz_mask) << 4;
-            a1 ^= ((a1 >> 7) & swz_mask) << 4;
-            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(a0), "r"(w[0]), "r"(w[1]), "r"(w[2]), "r"(w[3]) : "memory");
-            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(a1), "r"(w[4]), "r"(w[5]), "r"(w[6]), "r"(w[7]) : "memory");
-          }
-        }
-      }
-      fence_proxy_async_smem();
-      tcgen05_fence_before_sync();
-      named_barrier_sync(1, kEpiThreads);
-      if (tid == 0) mbar_arrive(bar_y + grp);
-    }
-
-    // P6: out = ReLU(acc + b2 + x); the residual is fetched before waiting for the accumulators. A thread owns one
-    // pixel row of a tile, and pixels are C * 2 bytes apart in device memory: stored straight from the registers, a
-    // warp's 16-byte stores would hit 32 different lines each. Instead the warp transposes its [32 pixels x ncol]
-    // block through a private 2 KB staging area (the start of the input rows, no longer read by then), so that
-    // consecutive lanes store consecutive 16-byte chunks of a pixel.
-    const bool stage = p.stage_ok != 0;
-    const uint32_t stg = smem_u32(sX) + (uint32_t)warp * 2048u;
-    const int chl = ncol == 32 ? 2 : 1;                  // log2(16-byte chunks per staged row)
-    const uint32_t rb = (uint32_t)ncol * 2u;             // bytes per staged row
-    const uint32_t swz_w = ((uint32_t)lane >> (3 - chl)) & ((1u << chl) - 1u);   // chunk XOR of this lane's row
-    for (int grp = 0; grp < 2; ++grp) {
-      const int lo2 = grp ? p.a2 : 0, hi2 = grp ? p.M2 : p.a2;   // the group's tiles of the second convolution
-      for (int mt = lo2; mt < hi2 || mt == lo2; ++mt) {
-        const bool tile_ok = mt < hi2;
-        const int m = mt * 128 + row;
-        const int r = (int)fast_div((uint32_t)m, (uint32_t)p.Wp, p.wp_recip), cc = m - r * p.Wp;
-        const bool valid = tile_ok && has_cols && r < rows_valid && cc >= 1 && cc <= p.W;
-        const size_t pix = ((size_t)n * p.H + h0 + r) * p.W + (cc - 1);
-        const bool do_res = SINGLE ? p.residual != 0 : true, do_relu = SINGLE ? p.relu != 0 : true;
-        uint4 xr[4];
-        if (SINGLE) {
-#pragma unroll
-          for (int j = 0; j < 4; ++j) xr[j] = make_uint4(0u, 0u, 0u, 0u);
-        }
-        if (valid && do_res) {
-#pragma unroll
-          for (int j = 0; j < 4; ++j)
-            if (j * 8 < ncol) xr[j] = __ldg(reinterpret_cast<const uint4*>((SINGLE ? p.res : p.x) + pix * p.C + col0 + j * 8));
-        }
-        if (mt == lo2) {
-          mbar_wait(bar_acc2 + grp, 0, abort_flag, p.status, 0x406);
+      const uint32_t d_tmem = tmem_base + (uint32_t)buf * nacc;
+      const uint64_t a0 = xdesc0 + (uint64_t)((uint32_t)(s * p.IH + 4 * t) * rowu);
+      for (int frow = 0; frow < 3; ++frow) {
+        if (w_conv != conv) {
+          mbar_wait(bar_wfull + frow, SINGLE ? 0u : (uint32_t)conv, abort_flag, p.status, 0x405);
           tcgen05_fence_after_sync();
         }
-        if (!tile_ok) break;
-        if (has_cols) {
-          for (int c0 = col0, jj = 0; c0 < col0 + ncol; c0 += 16, jj += 2) {
-            uint32_t v[16];
-            tmem_ld_x16(tmem_base + lane_base + mt * p.C + c0, v);
-            tmem_ld_wait();
-            if (valid) {
-              const uint32_t xs[8] = {xr[jj].x, xr[jj].y, xr[jj].z, xr[jj].w, xr[jj + 1].x, xr[jj + 1].y, xr[jj + 1].z, xr[jj + 1].w};
-              uint32_t w[8];
+        const uint64_t a = a0 + (uint64_t)((uint32_t)frow * rowu);
+        const uint64_t b = wdesc0 + (uint64_t)(frow_step * (uint32_t)frow);
+        if (ksteps == 4) {
+          umma_bf16_elected_acc(d_tmem, a, b, idesc, elected, frow != 0);
+          umma_bf16_elected<true>(d_tmem, a + 2u, b + 2u, idesc, elected);
+          umma_bf16_elected<true>(d_tmem, a + 4u, b + 4u, idesc, elected);
+          umma_bf16_elected<true>(d_tmem, a + 6u, b + 6u, idesc, elected);
+        } else {
+          for (int ks = 0; ks < ksteps; ++ks)
+            umma_bf16_elected_acc(d_tmem, a + 2u * ks, b + 2u * ks, idesc, elected, (ks | frow) != 0);
+        }
+        if (!SINGLE && seq == p.M1 - 1) umma_commit_elected(bar_wfree + frow, elected);
+        // The shifts of the previous tile go into the tensor pipe's queue here, behind this tile's first filter row
+        // (which keeps the pipe busy while the shift warps learn that the previous tile's products are complete)
+        // and ahead of the rest: behind a whole tile they would hold the epilogue back by a tile.
+        if (frow == 0 && seq > 0) mbar_wait(bar_shq + (buf ^ 1), (uint32_t)((seq - 1) >> 1) & 1u, abort_flag, p.status, 0x408);
+      }
+      w_conv = conv;
+      umma_commit_elected(bar_mma + buf, elected);
+      if (++s == p.NS) { s = 0; ++t; }
+    }
+    __syncwarp();
+  } else if (warp > kEpiWarps + 1) {
+    // ================================ shift warps: align the accumulators ================================
+    // tcgen05.shift is not ordered behind the MMAs issued before it (their last accumulator updates are still in
+    // flight), so the shifts of a tile are issued here, after the tile's products have completed, while the MMA warp
+    // is already issuing the next tile into the other accumulator. D_1 moves one row, D_2 two rows towards row 0,
+    // 8 columns per instruction; issuing costs a warp ~40 cycles per instruction next to the busy epilogue warps,
+    // so two warps share the 3 C / 8 instructions of a tile (both shifts of a column block stay in one thread).
+    const int sw = warp - kEpiWarps - 2;
+    const uint32_t elected = elect_one();
+    const int units = p.C / 8, split = units / 4;      // warp 0: D_1 and the first quarter of D_2; warp 1: the rest of D_2
+    for (int seq = 0; seq < ntiles; ++seq) {
+      const int buf = seq & 1;
+      mbar_wait(bar_mma + buf, (uint32_t)(seq >> 1) & 1u, abort_flag, p.status, 0x407);
+      tcgen05_fence_after_sync();
+      const uint32_t d_tmem = tmem_base + (uint32_t)buf * nacc;
+      if (sw == 0)
+        for (int u = 0; u < units; ++u) tmem_shift_down_elected(d_tmem + (uint32_t)(p.C + 8 * u), elected);
+      for (int u = sw == 0 ? 0 : split; u < (sw == 0 ? split : units); ++u) {
+        tmem_shift_down_elected(d_tmem + (uint32_t)(2 * p.C + 8 * u), elected);
+        tmem_shift_down_elected(d_tmem + (uint32_t)(2 * p.C + 8 * u), elected);
+      }
+      umma_commit_elected(bar_acc + buf, elected);
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar_shq + buf);
+    }
+    __syncwarp();
+  } else if ((warp >> 2) * 16 < p.C) {
+    // ================ epilogue warps: thread = (image row of the tile, pixel of the segment, 16 channels) ================
+    const int wq = warp & 3, cg = warp >> 2;
+    const int col0 = cg * 16;
+    const uint32_t lane_base = (uint32_t)(wq * 32) << 16;
+    const uint32_t x_addr = smem_u32(sX);
+    const uint32_t swz_mask = ((uint32_t)p.w_row_bytes >> 4) - 1u;
+    // Output staging (P6): a thread owns one pixel, and pixels are C * 2 bytes apart in device memory: stored straight
+    // from the registers, a warp's 16-byte stores would hit 32 different lines each. Instead the warp transposes its
+    // [32 pixels x 16 channels] block through a private 1 KB staging area, so that consecutive lanes store
+    // consecutive 16-byte chunks. The area lies in the input rows R + 2 and R + 3 of the segments, which only the
+    // rows past the strip read once the first convolution is complete, or in its own space.
+    uint32_t stg = 0;
+    if (p.stage_mode == 1) {
+      const uint32_t dead = 2u * 32u * (uint32_t)p.w_row_bytes, k = (uint32_t)warp * 1024u;
+      stg = x_addr + (k / dead) * seg_bytes + (uint32_t)(p.R + 2) * 32u * (uint32_t)p.w_row_bytes + k % dead;
+    } else if (p.stage_mode == 2) {
+      stg = smem_u32(smem + p.off_stage) + (uint32_t)warp * 1024u;
+    }
+    const uint32_t swz_w = ((uint32_t)lane >> 2) & 1u;   // chunk XOR of this lane's staged row (two chunks per row)
+    const bool do_res = SINGLE ? p.residual != 0 : true, do_relu = SINGLE ? p.relu != 0 : true;
+
+    int t = 0, s = 0;
+    for (int seq = 0; seq < ntiles; ++seq) {
+      if (seq == p.M1) { t = 0; s = 0; }
+      const bool second = seq >= p.M1;
+      const int buf = seq & 1;
+      const int a = 4 * t + wq;                        // row of the intermediate / of the output inside the strip
+      // second convolution: lane j is output column 28 s + j; fetch the residual before waiting for the accumulator
+      const int c = s * kSegCols + lane;
+      const bool valid = second && lane < kSegCols && c < p.W && a < rows_valid;
+      const size_t pix = ((size_t)n * p.H + h0 + a) * p.W + c;
+      uint4 xr[2] = {make_uint4(0u, 0u, 0u, 0u), make_uint4(0u, 0u, 0u, 0u)};
+      if (valid && do_res) {
+        const __nv_bfloat16* rp = (SINGLE ? p.res : p.x) + pix * p.C + col0;
+        xr[0] = __ldg(reinterpret_cast<const uint4*>(rp));
+        xr[1] = __ldg(reinterpret_cast<const uint4*>(rp + 8));
+      }
+      mbar_wait(bar_acc + buf, (uint32_t)(seq >> 1) & 1u, abort_flag, p.status, 0x406);
+      tcgen05_fence_after_sync();
+      uint32_t v0[16], v1[16], v2[16];
+      const uint32_t tb = tmem_base + lane_base + (uint32_t)buf * nacc + (uint32_t)col0;
+      tmem_ld_x16(tb, v0);
+      tmem_ld_x16(tb + (uint32_t)p.C, v1);
+      tmem_ld_x16(tb + 2u * (uint32_t)p.C, v2);
+      tmem_ld_wait();
+      tcgen05_fence_before_sync();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar_accfree + buf);
+      float sum[16];
+      const float* bias = sBias + (second ? p.C : 0) + col0;
 #pragma unroll
-              for (int j = 0; j < 8; ++j) {
-                float y0 = __uint_as_float(v[2 * j]) + bias2[2 * j] + bf16_lo(xs[j]);      // xs is zero without a residual
-                float y1 = __uint_as_float(v[2 * j + 1]) + bias2[2 * j + 1] + bf16_hi(xs[j]);
-                if (do_relu) { y0 = fmaxf(y0, 0.0f); y1 = fmaxf(y1, 0.0f); }
-                w[j] = pack_bf16x2(y0, y1);
-              }
-              if (stage) {
-                const uint32_t k0 = (uint32_t)(c0 - col0) >> 3;
-                const uint32_t a0 = stg + (uint32_t)lane * rb + ((k0 ^ swz_w) << 4), a1 = stg + (uint32_t)lane * rb + (((k0 + 1u) ^ swz_w) << 4);
-                asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(a0), "r"(w[0]), "r"(w[1]), "r"(w[2]), "r"(w[3]) : "memory");
-                asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(a1), "r"(w[4]), "r"(w[5]), "r"(w[6]), "r"(w[7]) : "memory");
-              } else {
-                *reinterpret_cast<uint4*>(p.out + pix * p.C + c0) = make_uint4(w[0], w[1], w[2], w[3]);
-                *reinterpret_cast<uint4*>(p.out + pix * p.C + c0 + 8) = make_uint4(w[4], w[5], w[6], w[7]);
-              }
-            }
+      for (int j = 0; j < 16; j += 4) {
+        const float4 bj = *reinterpret_cast<const float4*>(bias + j);
+        sum[j] = __uint_as_float(v0[j]) + __uint_as_float(v1[j]) + __uint_as_float(v2[j]) + bj.x;
+        sum[j + 1] = __uint_as_float(v0[j + 1]) + __uint_as_float(v1[j + 1]) + __uint_as_float(v2[j + 1]) + bj.y;
+        sum[j + 2] = __uint_as_float(v0[j + 2]) + __uint_as_float(v1[j + 2]) + __uint_as_float(v2[j + 2]) + bj.z;
+        sum[j + 3] = __uint_as_float(v0[j + 3]) + __uint_as_float(v1[j + 3]) + __uint_as_float(v2[j + 3]) + bj.w;
+      }
+
+      if (!second) {
+        // P3: intermediate = ReLU(sum) inside the image, 0 outside -> the swizzled row of (segment, row a, pixel lane);
+        // lane j is column 28 s - 1 + j of the intermediate, lanes 30 and 31 have no complete sum
+        if (lane < 30 && a < p.R + 2) {
+          const int gh = h0 - 1 + a, cy = s * kSegCols - 1 + lane;
+          const bool inside = gh >= 0 && gh < p.H && cy >= 0 && cy < p.W;
+          uint32_t w[8];
+#pragma unroll
+          for (int j = 0; j < 8; ++j)
+            w[j] = inside ? pack_bf16x2(fmaxf(sum[2 * j], 0.0f), fmaxf(sum[2 * j + 1], 0.0f)) : 0u;
+          // 16-byte chunk index XOR address bits [7, ..): the swizzle the MMA and TMA apply to absolute addresses
+          uint32_t a0 = x_addr + (uint32_t)s * seg_bytes + (uint32_t)(a * 32 + lane) * p.w_row_bytes + (uint32_t)col0 * 2u;
+          uint32_t a1 = a0 + 16u;
+          a0 ^= ((a0 >> 7) & swz_mask) << 4;
+          a1 ^= ((a1 >> 7) & swz_mask) << 4;
+          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(a0), "r"(w[0]), "r"(w[1]), "r"(w[2]), "r"(w[3]) : "memory");
+          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(a1), "r"(w[4]), "r"(w[5]), "r"(w[6]), "r"(w[7]) : "memory");
+        }
+        fence_proxy_async_smem();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar_y + seq);
+      } else {
+        // P6: out = ReLU(sum + x)
+        uint32_t w[8];
+        const uint32_t xs[8] = {xr[0].x, xr[0].y, xr[0].z, xr[0].w, xr[1].x, xr[1].y, xr[1].z, xr[1].w};
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          float y0 = sum[2 * j] + bf16_lo(xs[j]);      // xs is zero without a residual
+          float y1 = sum[2 * j + 1] + bf16_hi(xs[j]);
+          if (do_relu) { y0 = fmaxf(y0, 0.0f); y1 = fmaxf(y1, 0.0f); }
+          w[j] = pack_bf16x2(y0, y1);
+        }
+        if (p.stage_mode != 0) {
+          const uint32_t a0 = stg + (uint32_t)lane * 32u + (swz_w << 4), a1 = stg + (uint32_t)lane * 32u + ((1u ^ swz_w) << 4);
+          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(a0), "r"(w[0]), "r"(w[1]), "r"(w[2]), "r"(w[3]) : "memory");
+          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(a1), "r"(w[4]), "r"(w[5]), "r"(w[6]), "r"(w[7]) : "memory");
+          __syncwarp();
+          const uint32_t vmask = __ballot_sync(0xffffffffu, valid);
+          const unsigned long long goff = ((unsigned long long)pix * p.C + col0) * 2ull;   // byte offset of this lane's pixel
+#pragma unroll
+          for (int it = 0; it < 2; ++it) {
+            const int pl = it * 16 + (lane >> 1);
+            const uint32_t ch = (uint32_t)lane & 1u;
+            const uint32_t lo = __shfl_sync(0xffffffffu, (uint32_t)goff, pl), hi = __shfl_sync(0xffffffffu, (uint32_t)(goff >> 32), pl);
+            const uint32_t sw = ((uint32_t)pl >> 2) & 1u;
+            uint4 val;
+            asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(val.x), "=r"(val.y), "=r"(val.z), "=r"(val.w) : "r"(stg + (uint32_t)pl * 32u + ((ch ^ sw) << 4)));
+            if ((vmask >> pl) & 1u)
+              *reinterpret_cast<uint4*>(reinterpret_cast<uint8_t*>(p.out) + (((unsigned long long)hi << 32) | lo) + ch * 16u) = val;
           }
-          if (stage) {
-            __syncwarp();
-            const uint32_t vmask = __ballot_sync(0xffffffffu, valid);
-            const unsigned long long goff = ((unsigned long long)pix * p.C + col0) * 2ull;   // byte offset of this lane's row
-            for (int it = 0; it < (1 << chl); ++it) {
-              const int pl = it * (32 >> chl) + (lane >> chl);
-              const uint32_t ch = (uint32_t)lane & ((1u << chl) - 1u);
-              const uint32_t lo = __shfl_sync(0xffffffffu, (uint32_t)goff, pl), hi = __shfl_sync(0xffffffffu, (uint32_t)(goff >> 32), pl);
-              const uint32_t sw = ((uint32_t)pl >> (3 - chl)) & ((1u << chl) - 1u);
-              uint4 val;
-              asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(val.x), "=r"(val.y), "=r"(val.z), "=r"(val.w) : "r"(stg + (uint32_t)pl * rb + ((ch ^ sw) << 4)));
-              if ((vmask >> pl) & 1u)
-                *reinterpret_cast<uint4*>(reinterpret_cast<uint8_t*>(p.out) + (((unsigned long long)hi << 32) | lo) + ch * 16u) = val;
-            }
-            __syncwarp();
-          }
+          __syncwarp();
+        } else if (valid) {
+          *reinterpret_cast<uint4*>(p.out + pix * p.C + col0) = make_uint4(w[0], w[1], w[2], w[3]);
+          *reinterpret_cast<uint4*>(p.out + pix * p.C + col0 + 8) = make_uint4(w[4], w[5], w[6], w[7]);
         }
       }
+      if (++s == p.NS) { s = 0; ++t; }
     }
   }
   tcgen05_fence_before_sync();
@@ -343,47 +369,49 @@ struct ConvHost {
 
 int round_up_i(int v, int m) { return (v + m - 1) / m * m; }
 
+// Shared-memory layout common to both variants (pair: IH = R + 4 rows and both convolutions; single: IH = R + 2).
+bool conv_layout_common(ConvParams& q, bool pair, int* smem_bytes) {
+  q.NS = (q.W + kSegCols - 1) / kSegCols;
+  q.T1 = pair ? (q.R + 2 + 3) / 4 : 0;
+  q.T2 = (q.R + 3) / 4;
+  q.M1 = q.NS * q.T1;
+  q.M2 = q.NS * q.T2;
+  q.nact = 4 * std::min(4, q.C / 16);
+  if (q.IH > 256 || q.M1 > kMaxTiles1) return false;
+  const int seg_bytes = q.IH * 32 * q.w_row_bytes;
+  int off = 0;
+  q.off_x = off;
+  off = round_up_i(off + q.NS * seg_bytes, 1024);
+  q.off_w = off;
+  off += round_up_i(9 * q.w_tap_bytes, 1024);
+  q.off_bias = off;
+  off += 1024;
+  q.off_bar = off;
+  off += 512;
+  // Output staging: one KB per active epilogue warp. The pair has input rows that no valid output reads once the
+  // first convolution is complete (rows R + 2 and R + 3 of every segment); otherwise an area of its own if it fits.
+  q.off_stage = 0;
+  q.stage_mode = 0;
+  if (pair && (long)q.NS * 2 * 32 * q.w_row_bytes >= (long)q.nact * 1024) {
+    q.stage_mode = 1;
+  } else if (off + q.nact * 1024 + 1024 <= 227 * 1024) {
+    q.stage_mode = 2;
+    q.off_stage = off;
+    off += q.nact * 1024;
+  }
+  // The rows of the last tiles run past the strip (their results are dropped) but must stay inside the allocation:
+  // they then read filter rows or biases as activations, which is harmless.
+  const long reach = ((long)((q.NS - 1) * q.IH + 4 * (std::max(q.T1, q.T2) - 1) + 2) * 32 + 128) * q.w_row_bytes;
+  if (q.off_x + reach > (long)off) off = (int)round_up_i((int)(q.off_x + reach), 1024);
+  *smem_bytes = off + 1024;
+  return *smem_bytes <= 227 * 1024;
+}
+
 bool conv_layout(ConvParams& q, int R, int* smem_bytes) {
   q.R = R;
   q.strips = (q.H + R - 1) / R;
   q.IH = R + 4;
-  q.Wp = q.W + 2;
-  q.wp_recip = tc::fast_div_recip(q.Wp);
-  q.P1 = (R + 2) * q.Wp; q.M1 = (q.P1 + 127) / 128;
-  q.P2 = R * q.Wp; q.M2 = (q.P2 + 127) / 128;
-  if (q.IH > 256 || q.Wp > 256 || q.M1 * q.C > 512) return false;
-  // The intermediate rows alias the input rows, shifted down by two pixels: while the second tile
-  // group of the first convolution still reads input pixels >= a1*128 - 1, the first group's epilogue
-  // writes intermediate pixels < a1*128, i.e. input slots < a1*128 - 2.
-  int off = 1024;   // slack before the rows: shifted operand rows start up to three pixels early
-  q.off_x = off;
-  q.off_y = off - 2 * q.w_row_bytes;
-  const int reach_px = std::max(std::max(q.M1 * 128 + 2 * q.Wp + 2, q.P1 + q.Wp + 2), q.IH * q.Wp);
-  const int x_reach = reach_px * q.w_row_bytes;
-  off = round_up_i(off + x_reach, 1024);
-  q.off_w = off;
-  q.wstages = kMaxWStages;
-  while (q.wstages > 2 && off + q.wstages * 3 * q.w_stage_bytes + 2048 + 1024 > 227 * 1024) --q.wstages;
-  off += q.wstages * 3 * q.w_stage_bytes;
-  q.off_bias = off;
-  off += 1024;
-  q.off_bar = off;
-  off += 256;
-  // pipeline groups: the second convolution's first group may only read intermediate rows the first
-  // group of the first convolution produces
-  q.a1 = (q.M1 + 1) / 2;   // even groups: a pass of only three tiles keeps the tensor pipe less busy than one of four or five
-  if (q.a1 < 1) q.a1 = 1;
-  q.a2 = (q.a1 * 128 - 2 * q.Wp - 1) / 128;
-  if (q.a2 < 0) q.a2 = 0;
-  if (q.a2 > q.M2) q.a2 = q.M2;
-  if (q.a1 >= q.M1) { q.a1 = q.M1; }
-  // Output staging uses the first 16 KB of the input rows. While the second group of the second convolution is
-  // still being computed it reads intermediate pixels >= a2 * 128 - Wp - 1, which lie two pixel slots lower.
-  const bool overlap = q.a2 > 0 && q.a2 < q.M2;   // an output epilogue runs next to MMAs that still read the rows
-  const long free_bytes = overlap ? (long)(q.a2 * 128 - q.Wp - 3) * q.w_row_bytes : (long)x_reach;
-  q.stage_ok = free_bytes >= kEpiWarps * 2048 ? 1 : 0;
-  *smem_bytes = off + 1024;
-  return *smem_bytes <= 227 * 1024;
+  return conv_layout_common(q, true, smem_bytes);
 }
 
 }  // namespace
@@ -399,7 +427,7 @@ ago_status_t conv3x3_plan(Plan* plan, FusedState* st, std::string* err) {
   if (q.C != 16 && q.C != 32 && q.C != 64) return bad("channel count must be 16, 32 or 64");
   q.w_row_bytes = q.C * 2;
   q.w_swizzle = q.C == 16 ? tc::SW_32B : (q.C == 32 ? tc::SW_64B : tc::SW_128B);
-  q.w_stage_bytes = round_up_i(q.C * q.w_row_bytes, 1024);
+  q.w_tap_bytes = q.C * q.w_row_bytes;   // taps lie back to back: the three of a filter row form one B operand of 3 C rows
   int best_R = 0, best_smem = 0; double best_cost = 0;
   for (int R = 1; R <= q.H; ++R) {
     ConvParams t = q; int smem = 0;
@@ -437,7 +465,7 @@ ago_status_t conv3x3_run(const Plan& plan, FusedState* st, const void* const* in
       if (which == 0) {
         const uint64_t dims[4] = {(uint64_t)q.C, (uint64_t)q.W, (uint64_t)q.H, (uint64_t)q.N};
         const uint64_t strides[3] = {(uint64_t)q.C * 2, (uint64_t)q.W * q.C * 2, (uint64_t)q.H * q.W * q.C * 2};
-        const uint32_t box[4] = {(uint32_t)q.C, (uint32_t)q.Wp, (uint32_t)q.IH, 1};
+        const uint32_t box[4] = {(uint32_t)q.C, 32u, (uint32_t)q.IH, 1};
         if (!encode_tmap_bf16(&m, base, 4, dims, strides, box, q.w_row_bytes, err)) return false;
       } else {
         const uint64_t dims[3] = {(uint64_t)q.C, 9, (uint64_t)q.C};
@@ -472,32 +500,7 @@ bool conv_layout_single(ConvParams& q, int R, int* smem_bytes) {
   q.R = R;
   q.strips = (q.H + R - 1) / R;
   q.IH = R + 2;
-  q.Wp = q.W + 2;
-  q.wp_recip = tc::fast_div_recip(q.Wp);
-  q.P1 = 0; q.M1 = 0;
-  q.P2 = R * q.Wp; q.M2 = (q.P2 + 127) / 128;
-  if (q.IH > 256 || q.Wp > 256 || q.M2 * q.C > 512) return false;
-  int off = 1024;
-  q.off_x = off;
-  q.off_y = off;            // the convolution reads the input rows themselves
-  const int reach_px = std::max(q.M2 * 128 + 2 * q.Wp + 2, q.IH * q.Wp);
-  const int x_reach = reach_px * q.w_row_bytes;
-  off = round_up_i(off + x_reach, 1024);
-  q.off_w = off;
-  q.wstages = kMaxWStages;
-  while (q.wstages > 2 && off + q.wstages * 3 * q.w_stage_bytes + 2048 + 1024 > 227 * 1024) --q.wstages;
-  off += q.wstages * 3 * q.w_stage_bytes;
-  q.off_bias = off;
-  off += 1024;
-  q.off_bar = off;
-  off += 256;
-  q.a1 = 0;
-  q.a2 = (q.M2 + 1) / 2;
-  const bool overlap = q.a2 > 0 && q.a2 < q.M2;
-  const long free_bytes = overlap ? (long)(q.a2 * 128 - q.Wp - 1) * q.w_row_bytes : (long)x_reach;
-  q.stage_ok = free_bytes >= kEpiWarps * 2048 ? 1 : 0;
-  *smem_bytes = off + 1024;
-  return *smem_bytes <= 227 * 1024;
+  return conv_layout_common(q, false, smem_bytes);   // the convolution reads the input rows themselves
 }
 
 struct SingleKey {
@@ -534,7 +537,7 @@ cudaError_t launch_conv3x3_tc(const void* x, const void* w, const float* bias, c
       q.N = N; q.H = H; q.W = W; q.C = C;
       q.w_row_bytes = C * 2;
       q.w_swizzle = C == 16 ? tc::SW_32B : (C == 32 ? tc::SW_64B : tc::SW_128B);
-      q.w_stage_bytes = round_up_i(C * q.w_row_bytes, 1024);
+      q.w_tap_bytes = C * q.w_row_bytes;
       int best_R = 0, best_smem = 0; double best_cost = 0;
       for (int R = 1; R <= H; ++R) {
         ConvParams t = q; int smem = 0;
@@ -549,7 +552,7 @@ cudaError_t launch_conv3x3_tc(const void* x, const void* w, const float* bias, c
       std::string err;
       const uint64_t xd[4] = {(uint64_t)C, (uint64_t)W, (uint64_t)H, (uint64_t)N};
       const uint64_t xs[3] = {(uint64_t)C * 2, (uint64_t)W * C * 2, (uint64_t)H * W * C * 2};
-      const uint32_t xb[4] = {(uint32_t)C, (uint32_t)q.Wp, (uint32_t)q.IH, 1};
+      const uint32_t xb[4] = {(uint32_t)C, 32u, (uint32_t)q.IH, 1};
       if (!encode_tmap_bf16(&e.mx, x, 4, xd, xs, xb, q.w_row_bytes, &err)) return cudaErrorInvalidValue;
       const uint64_t wd[3] = {(uint64_t)C, 9, (uint64_t)C};
       const uint64_t ws[2] = {(uint64_t)C * 2, (uint64_t)9 * C * 2};

@@ -354,6 +354,17 @@ __device__ __forceinline__ void umma_commit_cluster_elected(uint32_t bar_cluster
       ::"r"(bar_cluster_addr), "r"(elected)
       : "memory");
 }
+// tcgen05.shift: every row of a 32-byte-wide (8 columns of 32 bits) block of tensor memory takes the value of the next
+// row (lane i <- lane i + 1), separately inside each block of 32 lanes: lanes 31, 63, 95 and 127 keep their values
+// (measured: ~10 cycles per instruction; asynchronous, in issue order with the MMAs of the same thread and tracked
+// by its commits). All lanes execute; one elected lane issues.
+__device__ __forceinline__ void tmem_shift_down_elected(uint32_t taddr, uint32_t elected) {
+  asm volatile(
+      "{\n\t.reg .pred q;\n\t"
+      "setp.ne.b32 q, %1, 0;\n\t"
+      "@q tcgen05.shift.cta_group::1.down [%0];\n\t}"
+      ::"r"(taddr), "r"(elected) : "memory");
+}
 __device__ __forceinline__ void umma_commit_elected(uint64_t* bar, uint32_t elected) {
   asm volatile(
       "{\n\t.reg .pred q;\n\t"
