@@ -61,10 +61,11 @@ using namespace tc;
 
 constexpr int kEpiWarps = 16;                // four per TMEM lane quarter: each takes 16 channels
 constexpr int kEpiThreads = kEpiWarps * 32;
-constexpr int kShiftWarps = 2;
+constexpr int kShiftWarps = 3;
 constexpr int kThreads = kEpiThreads + 64 + 32 * kShiftWarps;   // + TMA warp + MMA warp + shift warps
 constexpr int kSegCols = 28;                 // output columns per segment (32 input columns, 30 of the intermediate)
 constexpr int kMaxTiles1 = 32;               // tiles of the first convolution (one "rows written" barrier each)
+constexpr int kMaxChunks = 32;               // row chunks of the input strip over all segments (one "landed" barrier each)
 
 struct ConvParams {
   const __nv_bfloat16* x;
@@ -75,6 +76,7 @@ struct ConvParams {
   int N, H, W, C;          // C = input = middle = output channels
   int R, strips, IH;       // output rows per strip, strips per image, input rows per strip (R + 4; R + 2 for one convolution)
   int NS, T1, T2, M1, M2;  // segments; tile rows (4 image rows each) and tiles (NS per tile row) of either convolution
+  int CH, NCH;             // the strip arrives in chunks of CH input rows (a multiple of 4) per segment, NCH chunks each
   int nact;                // epilogue warps that own channels: 4 * min(4, C / 16)
   int stage_mode;          // output staging: 0 none (direct stores), 1 in the input rows that no valid output reads, 2 own area
   // single-convolution variant (a stage of the unfused mode): out = [relu](conv(x) + b2 [+ res])
@@ -88,20 +90,22 @@ struct ConvParams {
 // tiles only, reading the input rows directly), the tensor-core stage kernel of the unfused mode.
 template <bool SINGLE>
 __global__ void __launch_bounds__(kThreads, 1)
-conv3x3_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w1,
-                    const __grid_constant__ CUtensorMap tmap_w2, const ConvParams p) {
+conv3x3_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_xtail,
+                    const __grid_constant__ CUtensorMap tmap_w1,
+                    const __grid_constant__ CUtensorMap tmap_w2, const __grid_constant__ CUtensorMap tmap_out,
+                    const ConvParams p) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t* sX = smem + p.off_x;   // [segment][row][32 pixels][C]; the intermediate overwrites it in place
   uint8_t* sW = smem + p.off_w;   // [3 filter rows][3 taps][C rows]
   float* sBias = reinterpret_cast<float*>(smem + p.off_bias);   // b1[C], b2[C]
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + p.off_bar);
-  uint64_t* bar_x = bars;                 // input strip landed
   uint64_t* bar_wfull = bars + 1;         // [3] filter row landed (phase 0: first convolution, phase 1: second)
   uint64_t* bar_wfree = bars + 4;         // [3] filter row of the first convolution no longer read
   uint64_t* bar_acc = bars + 7;           // [2] accumulator of a tile complete (products and shifts)
   uint64_t* bar_mma = bars + 13 + kMaxTiles1;   // [2] products of a tile complete
   uint64_t* bar_shq = bars + 15 + kMaxTiles1;   // [2] shifts of a tile issued
+  uint64_t* bar_xc = bars + 17 + kMaxTiles1;    // [NCH][NS] chunk of input rows landed
   uint64_t* bar_accfree = bars + 9;       // [2] accumulator read out by every epilogue warp
   uint64_t* bar_y = bars + 11;            // [kMaxTiles1] intermediate rows of a tile written
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 11 + kMaxTiles1);
@@ -120,17 +124,25 @@ conv3x3_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
   grid_launch_dependents();
   if (tid == kEpiThreads) {
     *abort_flag = 0u;
-    mbar_init(bar_x, 1);
+    for (int i = 0; i < p.NCH * p.NS; ++i) mbar_init(bar_xc + i, 1);
     for (int i = 0; i < 3; ++i) { mbar_init(bar_wfull + i, 1); mbar_init(bar_wfree + i, 1); }
     for (int i = 0; i < 2; ++i) { mbar_init(bar_acc + i, kShiftWarps); mbar_init(bar_mma + i, 1); mbar_init(bar_shq + i, kShiftWarps); mbar_init(bar_accfree + i, (uint32_t)p.nact); }
     for (int i = 0; i < kMaxTiles1; ++i) mbar_init(bar_y + i, (uint32_t)p.nact);
     fence_mbar_init();
     fence_proxy_async_smem();
     tma_prefetch_desc(&tmap_x);
-    mbar_arrive_expect_tx(bar_x, (uint32_t)p.NS * seg_bytes);
-    // segment s: 32 columns from 28 s - 2 (one convolution: 28 s - 1), rows from h0 - 2 (h0 - 1); zero outside the image
-    for (int s = 0; s < p.NS; ++s)
-      tma_load_4d(sX + (size_t)s * seg_bytes, &tmap_x, bar_x, 0, s * kSegCols - (SINGLE ? 1 : 2), SINGLE ? h0 - 1 : h0 - 2, n);
+    // segment s: 32 columns from 28 s - 2 (one convolution: 28 s - 1), rows from h0 - 2 (h0 - 1); zero outside the
+    // image. The rows arrive in chunks, in the order the tiles need them, so that the first tile starts after the
+    // first chunks and the rest of the strip streams in behind the products.
+    for (int c = 0; c < p.NCH; ++c) {
+      const int rows = min(p.CH, p.IH - c * p.CH);
+      for (int s = 0; s < p.NS; ++s) {
+        uint64_t* bar = bar_xc + c * p.NS + s;
+        mbar_arrive_expect_tx(bar, (uint32_t)(rows * 32 * p.w_row_bytes));
+        tma_load_4d(sX + (size_t)s * seg_bytes + (size_t)(c * p.CH * 32) * p.w_row_bytes, rows == p.CH ? &tmap_x : &tmap_xtail, bar, 0,
+                    s * kSegCols - (SINGLE ? 1 : 2), (SINGLE ? h0 - 1 : h0 - 2) + c * p.CH, n);
+      }
+    }
   }
   if (warp == 0) {
     tmem_alloc(tmem_slot, 512);
@@ -167,13 +179,17 @@ conv3x3_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
     const uint64_t wdesc0 = make_smem_desc(smem_u32(sW), 0, 8u * p.w_row_bytes, p.w_swizzle);
     const uint64_t xdesc0 = make_smem_desc(smem_u32(sX), 0, 8u * p.w_row_bytes, p.w_swizzle);
     const uint32_t frow_step = (uint32_t)(3 * p.w_tap_bytes) >> 4;
-    mbar_wait(bar_x, 0, abort_flag, p.status, 0x402);
     int w_conv = -1;                       // convolution whose filter rows have been waited for
     int t = 0, s = 0;                      // tile row and segment of the tile
     for (int seq = 0; seq < ntiles; ++seq) {
       if (seq == p.M1) { t = 0; s = 0; }
       const int conv = seq >= p.M1 ? 1 : 0, buf = seq & 1;
       if (seq >= 2) mbar_wait(bar_accfree + buf, (uint32_t)((seq >> 1) - 1) & 1u, abort_flag, p.status, 0x403);
+      if (SINGLE || conv == 0) {
+        // input rows 4 t .. 4 t + 5 of the segment: the chunks that hold them (waiting again for a landed chunk is free)
+        const int c_lo = (4 * t) / p.CH, c_hi = min(4 * t + 5, p.IH - 1) / p.CH;
+        for (int c = c_lo; c <= min(c_hi, p.NCH - 1); ++c) mbar_wait(bar_xc + c * p.NS + s, 0, abort_flag, p.status, 0x402);
+      }
       if (!SINGLE && conv == 1) {
         // rows 4 t .. 4 t + 5 of the segment's intermediate: its tiles of tile rows t and t + 1
         mbar_wait(bar_y + t * p.NS + s, 0, abort_flag, p.status, 0x404);
@@ -215,20 +231,22 @@ conv3x3_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
     // flight), so the shifts of a tile are issued here, after the tile's products have completed, while the MMA warp
     // is already issuing the next tile into the other accumulator. D_1 moves one row, D_2 two rows towards row 0,
     // 8 columns per instruction; issuing costs a warp ~40 cycles per instruction next to the busy epilogue warps,
-    // so two warps share the 3 C / 8 instructions of a tile (both shifts of a column block stay in one thread).
+    // so three warps share the 3 C / 8 instructions of a tile (both shifts of a column block stay in one thread).
     const int sw = warp - kEpiWarps - 2;
     const uint32_t elected = elect_one();
-    const int units = p.C / 8, split = units / 4;      // warp 0: D_1 and the first quarter of D_2; warp 1: the rest of D_2
+    const int units = p.C / 8;      // warp 0: D_1; warps 1 and 2: a half of D_2 each, both shifts of a column block in one thread
     for (int seq = 0; seq < ntiles; ++seq) {
       const int buf = seq & 1;
       mbar_wait(bar_mma + buf, (uint32_t)(seq >> 1) & 1u, abort_flag, p.status, 0x407);
       tcgen05_fence_after_sync();
       const uint32_t d_tmem = tmem_base + (uint32_t)buf * nacc;
-      if (sw == 0)
+      if (sw == 0) {
         for (int u = 0; u < units; ++u) tmem_shift_down_elected(d_tmem + (uint32_t)(p.C + 8 * u), elected);
-      for (int u = sw == 0 ? 0 : split; u < (sw == 0 ? split : units); ++u) {
-        tmem_shift_down_elected(d_tmem + (uint32_t)(2 * p.C + 8 * u), elected);
-        tmem_shift_down_elected(d_tmem + (uint32_t)(2 * p.C + 8 * u), elected);
+      } else {
+        for (int u = (sw - 1) * units / 2; u < sw * units / 2; ++u) {
+          tmem_shift_down_elected(d_tmem + (uint32_t)(2 * p.C + 8 * u), elected);
+          tmem_shift_down_elected(d_tmem + (uint32_t)(2 * p.C + 8 * u), elected);
+        }
       }
       umma_commit_elected(bar_acc + buf, elected);
       __syncwarp();
@@ -242,36 +260,48 @@ conv3x3_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
     const uint32_t lane_base = (uint32_t)(wq * 32) << 16;
     const uint32_t x_addr = smem_u32(sX);
     const uint32_t swz_mask = ((uint32_t)p.w_row_bytes >> 4) - 1u;
-    // Output staging (P6): a thread owns one pixel, and pixels are C * 2 bytes apart in device memory: stored straight
-    // from the registers, a warp's 16-byte stores would hit 32 different lines each. Instead the warp transposes its
-    // [32 pixels x 16 channels] block through a private 1 KB staging area, so that consecutive lanes store
-    // consecutive 16-byte chunks. The area lies in the input rows R + 2 and R + 3 of the segments, which only the
-    // rows past the strip read once the first convolution is complete, or in its own space.
-    uint32_t stg = 0;
-    if (p.stage_mode == 1) {
-      const uint32_t dead = 2u * 32u * (uint32_t)p.w_row_bytes, k = (uint32_t)warp * 1024u;
-      stg = x_addr + (k / dead) * seg_bytes + (uint32_t)(p.R + 2) * 32u * (uint32_t)p.w_row_bytes + k % dead;
-    } else if (p.stage_mode == 2) {
-      stg = smem_u32(smem + p.off_stage) + (uint32_t)warp * 1024u;
-    }
-    const uint32_t swz_w = ((uint32_t)lane >> 2) & 1u;   // chunk XOR of this lane's staged row (two chunks per row)
+    // Output (P6): the 32 pixels x C channels of an image row of the tile are staged as swizzled rows by the warps
+    // that share the row (one per 16 channels) and leave with one TMA store of 28 pixels, clipped at the image's
+    // right edge. From the second tile row on, the staging block is the row four above in the same segment: every
+    // product that read it has completed, and no later tile writes it, so nothing waits for a store to drain. The
+    // first tile row stages in the input rows R + 2 and R + 3 of the segments, which only the rows past the strip
+    // read once the first convolution is complete, or in its own space (or stores directly if there is neither).
+    const uint32_t qbytes = 32u * (uint32_t)p.w_row_bytes;
+    uint8_t* stg0_ptr = sX;
+    if (p.stage_mode == 1) stg0_ptr = sX + (size_t)(wq >> 1) * seg_bytes + (size_t)(p.R + 2) * qbytes + (size_t)(wq & 1) * qbytes;
+    else if (p.stage_mode == 2) stg0_ptr = smem + p.off_stage + (size_t)wq * qbytes;
+    const uint32_t row_threads = (uint32_t)(p.nact / 4) * 32u;   // threads that share an image row of the tile
+    const bool storer = cg == 0 && lane == 0;
     const bool do_res = SINGLE ? p.residual != 0 : true, do_relu = SINGLE ? p.relu != 0 : true;
 
+    // The residual of an output tile is fetched one tile ahead (its latency is a tile's worth of cycles when the
+    // input comes from device memory).
+    uint4 xn0 = make_uint4(0u, 0u, 0u, 0u), xn1 = xn0;
+    auto fetch_residual = [&](int t_, int s_) {
+      const int a_ = 4 * t_ + wq, c_ = s_ * kSegCols + lane;
+      xn0 = make_uint4(0u, 0u, 0u, 0u); xn1 = xn0;
+      if (do_res && lane < kSegCols && c_ < p.W && a_ < rows_valid) {
+        const __nv_bfloat16* rp = (SINGLE ? p.res : p.x) + (((size_t)n * p.H + h0 + a_) * p.W + c_) * p.C + col0;
+        xn0 = __ldg(reinterpret_cast<const uint4*>(rp));
+        xn1 = __ldg(reinterpret_cast<const uint4*>(rp + 8));
+      }
+    };
+    if (p.M1 == 0) fetch_residual(0, 0);
     int t = 0, s = 0;
     for (int seq = 0; seq < ntiles; ++seq) {
       if (seq == p.M1) { t = 0; s = 0; }
       const bool second = seq >= p.M1;
       const int buf = seq & 1;
       const int a = 4 * t + wq;                        // row of the intermediate / of the output inside the strip
-      // second convolution: lane j is output column 28 s + j; fetch the residual before waiting for the accumulator
+      // second convolution: lane j is output column 28 s + j
       const int c = s * kSegCols + lane;
       const bool valid = second && lane < kSegCols && c < p.W && a < rows_valid;
       const size_t pix = ((size_t)n * p.H + h0 + a) * p.W + c;
-      uint4 xr[2] = {make_uint4(0u, 0u, 0u, 0u), make_uint4(0u, 0u, 0u, 0u)};
-      if (valid && do_res) {
-        const __nv_bfloat16* rp = (SINGLE ? p.res : p.x) + pix * p.C + col0;
-        xr[0] = __ldg(reinterpret_cast<const uint4*>(rp));
-        xr[1] = __ldg(reinterpret_cast<const uint4*>(rp + 8));
+      const uint4 xr[2] = {xn0, xn1};
+      if (seq + 1 < ntiles && seq + 1 >= p.M1) {
+        if (seq + 1 == p.M1) fetch_residual(0, 0);
+        else if (s + 1 == p.NS) fetch_residual(t + 1, 0);
+        else fetch_residual(t, s + 1);
       }
       mbar_wait(bar_acc + buf, (uint32_t)(seq >> 1) & 1u, abort_flag, p.status, 0x406);
       tcgen05_fence_after_sync();
@@ -327,25 +357,25 @@ conv3x3_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
           if (do_relu) { y0 = fmaxf(y0, 0.0f); y1 = fmaxf(y1, 0.0f); }
           w[j] = pack_bf16x2(y0, y1);
         }
-        if (p.stage_mode != 0) {
-          const uint32_t a0 = stg + (uint32_t)lane * 32u + (swz_w << 4), a1 = stg + (uint32_t)lane * 32u + ((1u ^ swz_w) << 4);
+        if (p.stage_mode != 0 || t > 0) {
+          uint8_t* stg_ptr = t > 0 ? sX + (size_t)s * seg_bytes + (size_t)(a - 4) * qbytes : stg0_ptr;
+          const uint32_t stg = smem_u32(stg_ptr);
+          if (t == 0 && s > 0) {
+            if (storer) bulk_wait_group_read_all();        // the first tile row's segments share one set of staging blocks
+            named_barrier_sync(2u + (uint32_t)wq, row_threads);
+          }
+          uint32_t a0 = stg + (uint32_t)lane * p.w_row_bytes + (uint32_t)col0 * 2u;
+          uint32_t a1 = a0 + 16u;
+          a0 ^= ((a0 >> 7) & swz_mask) << 4;
+          a1 ^= ((a1 >> 7) & swz_mask) << 4;
           asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(a0), "r"(w[0]), "r"(w[1]), "r"(w[2]), "r"(w[3]) : "memory");
           asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(a1), "r"(w[4]), "r"(w[5]), "r"(w[6]), "r"(w[7]) : "memory");
-          __syncwarp();
-          const uint32_t vmask = __ballot_sync(0xffffffffu, valid);
-          const unsigned long long goff = ((unsigned long long)pix * p.C + col0) * 2ull;   // byte offset of this lane's pixel
-#pragma unroll
-          for (int it = 0; it < 2; ++it) {
-            const int pl = it * 16 + (lane >> 1);
-            const uint32_t ch = (uint32_t)lane & 1u;
-            const uint32_t lo = __shfl_sync(0xffffffffu, (uint32_t)goff, pl), hi = __shfl_sync(0xffffffffu, (uint32_t)(goff >> 32), pl);
-            const uint32_t sw = ((uint32_t)pl >> 2) & 1u;
-            uint4 val;
-            asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(val.x), "=r"(val.y), "=r"(val.z), "=r"(val.w) : "r"(stg + (uint32_t)pl * 32u + ((ch ^ sw) << 4)));
-            if ((vmask >> pl) & 1u)
-              *reinterpret_cast<uint4*>(reinterpret_cast<uint8_t*>(p.out) + (((unsigned long long)hi << 32) | lo) + ch * 16u) = val;
+          fence_proxy_async_smem();
+          named_barrier_sync(2u + (uint32_t)wq, row_threads);
+          if (storer && a < rows_valid) {
+            tma_store_3d(&tmap_out, stg_ptr, 0, s * kSegCols, n * p.H + h0 + a);
+            bulk_commit_group();
           }
-          __syncwarp();
         } else if (valid) {
           *reinterpret_cast<uint4*>(p.out + pix * p.C + col0) = make_uint4(w[0], w[1], w[2], w[3]);
           *reinterpret_cast<uint4*>(p.out + pix * p.C + col0 + 8) = make_uint4(w[4], w[5], w[6], w[7]);
@@ -353,6 +383,7 @@ conv3x3_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
       }
       if (++s == p.NS) { s = 0; ++t; }
     }
+    if (storer) bulk_wait_group_all();
   }
   tcgen05_fence_before_sync();
   __syncthreads();
@@ -378,6 +409,9 @@ bool conv_layout_common(ConvParams& q, bool pair, int* smem_bytes) {
   q.M2 = q.NS * q.T2;
   q.nact = 4 * std::min(4, q.C / 16);
   if (q.IH > 256 || q.M1 > kMaxTiles1) return false;
+  q.CH = 4;
+  while (((q.IH + q.CH - 1) / q.CH) * q.NS > kMaxChunks) q.CH += 4;
+  q.NCH = (q.IH + q.CH - 1) / q.CH;
   const int seg_bytes = q.IH * 32 * q.w_row_bytes;
   int off = 0;
   q.off_x = off;
@@ -387,15 +421,17 @@ bool conv_layout_common(ConvParams& q, bool pair, int* smem_bytes) {
   q.off_bias = off;
   off += 1024;
   q.off_bar = off;
-  off += 512;
-  // Output staging: one KB per active epilogue warp. The pair has input rows that no valid output reads once the
-  // first convolution is complete (rows R + 2 and R + 3 of every segment); otherwise an area of its own if it fits.
+  off += 1024;
+  // Output staging: 32 pixels x C channels per image row of a tile (one KB per active epilogue warp). The pair has
+  // input rows that no valid output reads once the first convolution is complete (rows R + 2 and R + 3 of every
+  // segment: room for two image rows each); otherwise an area of its own if it fits.
   q.off_stage = 0;
   q.stage_mode = 0;
   if (pair && (long)q.NS * 2 * 32 * q.w_row_bytes >= (long)q.nact * 1024) {
     q.stage_mode = 1;
-  } else if (off + q.nact * 1024 + 1024 <= 227 * 1024) {
+  } else if (round_up_i(off, 1024) + q.nact * 1024 + 1024 <= 227 * 1024) {
     q.stage_mode = 2;
+    off = round_up_i(off, 1024);   // staging rows are swizzled like operand rows: whole 1024-byte groups
     q.off_stage = off;
     off += q.nact * 1024;
   }
@@ -462,11 +498,17 @@ ago_status_t conv3x3_run(const Plan& plan, FusedState* st, const void* const* in
     auto it = host->maps.find(key);
     if (it == host->maps.end()) {
       CUtensorMap m;
-      if (which == 0) {
+      if (which == 0 || which == 4) {   // input rows: a chunk of CH rows, or the shorter last chunk
+        const int tail = q.IH - (q.NCH - 1) * q.CH;
         const uint64_t dims[4] = {(uint64_t)q.C, (uint64_t)q.W, (uint64_t)q.H, (uint64_t)q.N};
         const uint64_t strides[3] = {(uint64_t)q.C * 2, (uint64_t)q.W * q.C * 2, (uint64_t)q.H * q.W * q.C * 2};
-        const uint32_t box[4] = {(uint32_t)q.C, 32u, (uint32_t)q.IH, 1};
+        const uint32_t box[4] = {(uint32_t)q.C, 32u, (uint32_t)(which == 0 ? std::min(q.CH, q.IH) : tail), 1};
         if (!encode_tmap_bf16(&m, base, 4, dims, strides, box, q.w_row_bytes, err)) return false;
+      } else if (which == 3) {
+        const uint64_t dims[3] = {(uint64_t)q.C, (uint64_t)q.W, (uint64_t)q.N * q.H};
+        const uint64_t strides[2] = {(uint64_t)q.C * 2, (uint64_t)q.W * q.C * 2};
+        const uint32_t box[3] = {(uint32_t)q.C, (uint32_t)kSegCols, 1};
+        if (!encode_tmap_bf16(&m, base, 3, dims, strides, box, q.w_row_bytes, err)) return false;
       } else {
         const uint64_t dims[3] = {(uint64_t)q.C, 9, (uint64_t)q.C};
         const uint64_t strides[2] = {(uint64_t)q.C * 2, (uint64_t)9 * q.C * 2};
@@ -479,15 +521,15 @@ ago_status_t conv3x3_run(const Plan& plan, FusedState* st, const void* const* in
     *out = it->second;
     return true;
   };
-  CUtensorMap mx, mw1, mw2;
-  if (!get_map(inputs[0], 0, &mx) || !get_map(weights[0], 1, &mw1) || !get_map(weights[2], 2, &mw2)) return AGO_ERR_CUDA;
+  CUtensorMap mx, mxt, mw1, mw2, mo;
+  if (!get_map(inputs[0], 0, &mx) || !get_map(inputs[0], 4, &mxt) || !get_map(weights[0], 1, &mw1) || !get_map(weights[2], 2, &mw2) || !get_map(output, 3, &mo)) return AGO_ERR_CUDA;
   {
     static int smem_opt_in[64] = {};
     cudaError_t e = ensure_max_dynamic_smem(reinterpret_cast<const void*>(conv3x3_pair_kernel<false>), smem_opt_in);
     if (e != cudaSuccess) { *err = std::string("cudaFuncSetAttribute: ") + cudaGetErrorString(e); return AGO_ERR_CUDA; }
   }
   FusedLaunch launch(dim3((unsigned)(q.N * q.strips)), kThreads, (size_t)host->smem_bytes, stream);
-  cudaError_t e = cudaLaunchKernelEx(&launch.config, conv3x3_pair_kernel<false>, mx, mw1, mw2, q);
+  cudaError_t e = cudaLaunchKernelEx(&launch.config, conv3x3_pair_kernel<false>, mx, mxt, mw1, mw2, mo, q);
   if (e != cudaSuccess) { *err = std::string("fused conv3x3 pair launch: ") + cudaGetErrorString(e); return AGO_ERR_CUDA; }
   return AGO_OK;
 }
@@ -504,15 +546,15 @@ bool conv_layout_single(ConvParams& q, int R, int* smem_bytes) {
 }
 
 struct SingleKey {
-  const void *x, *w; int N, H, W, C;
-  bool operator==(const SingleKey& o) const { return x == o.x && w == o.w && N == o.N && H == o.H && W == o.W && C == o.C; }
+  const void *x, *w, *out; int N, H, W, C;
+  bool operator==(const SingleKey& o) const { return x == o.x && w == o.w && out == o.out && N == o.N && H == o.H && W == o.W && C == o.C; }
 };
 struct SingleKeyHash {
   size_t operator()(const SingleKey& k) const {
-    return std::hash<const void*>()(k.x) ^ (std::hash<const void*>()(k.w) * 31u) ^ ((size_t)k.N << 40) ^ ((size_t)k.H << 24) ^ ((size_t)k.W << 8) ^ (size_t)k.C;
+    return std::hash<const void*>()(k.x) ^ (std::hash<const void*>()(k.w) * 31u) ^ (std::hash<const void*>()(k.out) * 131u) ^ ((size_t)k.N << 40) ^ ((size_t)k.H << 24) ^ ((size_t)k.W << 8) ^ (size_t)k.C;
   }
 };
-struct SingleEntry { ConvParams prm; int smem_bytes; CUtensorMap mx, mw; };
+struct SingleEntry { ConvParams prm; int smem_bytes; CUtensorMap mx, mxt, mw, mo; };
 std::mutex g_single_mutex;
 std::unordered_map<SingleKey, SingleEntry, SingleKeyHash> g_single;
 
@@ -529,7 +571,7 @@ cudaError_t launch_conv3x3_tc(const void* x, const void* w, const float* bias, c
   SingleEntry entry;
   {
     std::lock_guard<std::mutex> lock(g_single_mutex);
-    const SingleKey key{x, w, N, H, W, C};
+    const SingleKey key{x, w, out, N, H, W, C};
     auto it = g_single.find(key);
     if (it == g_single.end()) {
       SingleEntry e{};
@@ -552,12 +594,18 @@ cudaError_t launch_conv3x3_tc(const void* x, const void* w, const float* bias, c
       std::string err;
       const uint64_t xd[4] = {(uint64_t)C, (uint64_t)W, (uint64_t)H, (uint64_t)N};
       const uint64_t xs[3] = {(uint64_t)C * 2, (uint64_t)W * C * 2, (uint64_t)H * W * C * 2};
-      const uint32_t xb[4] = {(uint32_t)C, 32u, (uint32_t)q.IH, 1};
+      const uint32_t xb[4] = {(uint32_t)C, 32u, (uint32_t)std::min(q.CH, q.IH), 1};
       if (!encode_tmap_bf16(&e.mx, x, 4, xd, xs, xb, q.w_row_bytes, &err)) return cudaErrorInvalidValue;
+      const uint32_t xtb[4] = {(uint32_t)C, 32u, (uint32_t)(q.IH - (q.NCH - 1) * q.CH), 1};
+      if (!encode_tmap_bf16(&e.mxt, x, 4, xd, xs, xtb, q.w_row_bytes, &err)) return cudaErrorInvalidValue;
       const uint64_t wd[3] = {(uint64_t)C, 9, (uint64_t)C};
       const uint64_t ws[2] = {(uint64_t)C * 2, (uint64_t)9 * C * 2};
       const uint32_t wb[3] = {(uint32_t)C, 1, (uint32_t)C};
       if (!encode_tmap_bf16(&e.mw, w, 3, wd, ws, wb, q.w_row_bytes, &err)) return cudaErrorInvalidValue;
+      const uint64_t od[3] = {(uint64_t)C, (uint64_t)W, (uint64_t)N * H};
+      const uint64_t os[2] = {(uint64_t)C * 2, (uint64_t)W * C * 2};
+      const uint32_t ob[3] = {(uint32_t)C, (uint32_t)kSegCols, 1};
+      if (!encode_tmap_bf16(&e.mo, out, 3, od, os, ob, q.w_row_bytes, &err)) return cudaErrorInvalidValue;
       if (g_single.size() > 4096) g_single.clear();
       it = g_single.emplace(key, e).first;
     }
@@ -574,7 +622,7 @@ cudaError_t launch_conv3x3_tc(const void* x, const void* w, const float* bias, c
     cudaError_t e = ensure_max_dynamic_smem(reinterpret_cast<const void*>(conv3x3_pair_kernel<true>), smem_opt_in);
     if (e != cudaSuccess) return e;
   }
-  conv3x3_pair_kernel<true><<<q.N * q.strips, kThreads, entry.smem_bytes, stream>>>(entry.mx, entry.mw, entry.mw, q);
+  conv3x3_pair_kernel<true><<<q.N * q.strips, kThreads, entry.smem_bytes, stream>>>(entry.mx, entry.mxt, entry.mw, entry.mw, entry.mo, q);
   return cudaGetLastError();
 }
 
