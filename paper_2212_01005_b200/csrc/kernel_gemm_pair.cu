@@ -158,7 +158,9 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
         mbar_remote_arrive(acce_leader + (uint32_t)(a * 8));
       }
     }
-    if (lane == 0 && rank == 0) {
+    if (rank == 0) {
+      // the whole warp runs the loop converged; MMAs and commits are predicated on one elected lane (tc_common.cuh)
+      const uint32_t elected = elect_one();
       const uint32_t idesc = make_idesc_bf16(256, (uint32_t)p.BN, 0, p.b_kmajor ? 0 : 1);
       int s = 0, round = 0, it = 0;
       for (int t = pair; t < tiles; t += p.pairs, ++it) {
@@ -176,16 +178,16 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
           const uint64_t bd = p.b_kmajor ? make_smem_desc(st + 16384, 0, 1024, SW_128B) : make_smem_desc(st + 16384, 8192, 1024, SW_128B);
 #pragma unroll
           for (int ks = 0; ks < kPK / 16; ++ks)
-            umma_bf16_pair(d_tmem, ad + 2u * ks, bd + (p.b_kmajor ? (uint64_t)(2u * ks) : (uint64_t)((ks * 2048) >> 4)), idesc, (kb | ks) != 0);
+            umma_bf16_pair_elected(d_tmem, ad + 2u * ks, bd + (p.b_kmajor ? (uint64_t)(2u * ks) : (uint64_t)((ks * 2048) >> 4)), idesc, elected, (kb | ks) != 0);
           const uint32_t e = smem_u32(bar_empty + s);
-          umma_commit_pair(cluster_map(e, 0u));
-          umma_commit_pair(cluster_map(e, 1u));
+          umma_commit_pair_elected(cluster_map(e, 0u), elected);
+          umma_commit_pair_elected(cluster_map(e, 1u), elected);
           if (++s == kPStages) { s = 0; ++round; }
         }
         if (!skip_signal_for_test(p.status, 0x604)) {
           const uint32_t f = smem_u32(bar_accf + a);
-          umma_commit_pair(cluster_map(f, 0u));
-          umma_commit_pair(cluster_map(f, 1u));
+          umma_commit_pair_elected(cluster_map(f, 0u), elected);
+          umma_commit_pair_elected(cluster_map(f, 1u), elected);
         }
       }
     }
