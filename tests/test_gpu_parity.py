@@ -43,6 +43,11 @@ def small_workloads():
         "resnet_small": WL.resnet_block("resnet_small", [26], 2, 12, 64),
         "resnet_odd": WL.resnet_block("resnet_odd", [27], 1, 9, 32),
         "resnet_16ch": WL.resnet_block("resnet_16ch", [32], 2, 20, 16),
+        # widths around the 28-column segments of the conv3x3 kernels: exactly one segment, a second segment of one
+        # column, two full segments and one column of a third; heights that leave ragged last strips and tile rows
+        "resnet_w28": WL.resnet_block("resnet_w28", [43], 1, 28, 64),
+        "resnet_w29": WL.resnet_block("resnet_w29", [44], 2, 29, 32),
+        "resnet_w57": WL.resnet_block("resnet_w57", [45], 1, 57, 16),
         "attn_small": WL.attention("attn_small", [28], 2, 128, 2, 64),
         "attn_ragged": WL.attention("attn_ragged", [29], 1, 200, 3, 64),
         # more query tiles than SMs: the persistent CTAs' runs of 1-2 and of 3-4 items cross from one head (and batch) into the next
@@ -158,7 +163,7 @@ def test_padding_of_the_intermediate_with_large_bias(ago):
 # ---- fused kernels -------------------------------------------------------------------
 
 FUSED_SMALL = ["mbv2_14", "mbv2_s1_odd", "mbv2_s2", "mbv2_s2_odd", "attn_small", "attn_ragged", "attn_runs2", "attn_runs4", "ffn_small", "ffn_rows_ragged", "ffn_g2", "ffn_g3",
-               "ffn_c2", "ffn_c3", "ffn_c4", "ffn_p1", "ffn_p2", "ffn_p3", "ffn_s3", "ffn_s4", "resnet_small", "resnet_odd", "resnet_16ch"]
+               "ffn_c2", "ffn_c3", "ffn_c4", "ffn_p1", "ffn_p2", "ffn_p3", "ffn_s3", "ffn_s4", "resnet_small", "resnet_odd", "resnet_16ch", "resnet_w28", "resnet_w29", "resnet_w57"]
 
 
 @pytest.mark.parametrize("name", FUSED_SMALL)
