@@ -161,7 +161,8 @@ ffn_cluster_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
       if (steps > 0) load_g1(0);
       for (int step = 0; step < steps; ++step) {
         if (step + 1 < steps) load_g1(step + 1);
-        for (int k = 0; k < CS; ++k) {      // second GEMM over hidden tile t CS + k: two stages of 64 hidden units
+        for (int i = 0; i < CS; ++i) {      // second GEMM over hidden tile t CS + k: two stages of 64 hidden units
+          const int k = (int)((r + CS - i) % CS);   // in the order the MMA warp consumes the slots: own tile first
           const int hid0 = (tile0_of(step) + k) * kBH;
           for (int h = 0; h < 2; ++h) {
             uint8_t* st = next_stage();
@@ -210,7 +211,10 @@ ffn_cluster_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
           mbar_wait(bar_outfree, (uint32_t)(bi - 1) & 1u, abort_flag, p.status, 0x709);
           tcgen05_fence_after_sync();
         }
-        for (int k = 0; k < CS; ++k) {
+        // Slots in the order their tiles arrive: this CTA's own tile first (no copy), then the tiles of ranks r - 1,
+        // r - 2, ... -- every producer sends to rank + 1 first, so rank r - q's tile is the q-th to land here.
+        for (int i = 0; i < CS; ++i) {
+          const int k = (int)((r + CS - i) % CS);
           mbar_wait(bar_hfull + k, (uint32_t)step & 1u, abort_flag, p.status, 0x704);   // H tile t CS + k is in slot k
           for (int h = 0; h < 2; ++h) {
             mbar_wait(bar_full + s, (uint32_t)round & 1u, abort_flag, p.status, 0x705);
@@ -219,7 +223,7 @@ ffn_cluster_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
             const uint64_t bd = make_smem_desc(smem_u32(sRing + s * kStageBytes), 8192, 1024, SW_128B);
 #pragma unroll
             for (int ks = 0; ks < 4; ++ks)
-              umma_bf16_elected_acc(tmem_base + kOutCol, hd + 2u * ks, bd + (uint64_t)((ks * 2048) >> 4), idesc2, elected, (t | k | h | ks) != 0);
+              umma_bf16_elected_acc(tmem_base + kOutCol, hd + 2u * ks, bd + (uint64_t)((ks * 2048) >> 4), idesc2, elected, (t | i | h | ks) != 0);
             umma_commit_elected(bar_empty + s, elected);
             advance();
           }
