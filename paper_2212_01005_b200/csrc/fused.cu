@@ -54,8 +54,10 @@ ago_status_t fused_plan(Plan* plan, FusedState* st, std::string* err) {
     case AGO_KERNEL_ATTENTION:
       return attention_plan(plan, st, err);
     case AGO_KERNEL_FFN: {
-      // the cluster kernel where the shape splits over 2..4 CTAs, else the kernel that tiles the reduction
-      const ago_status_t s = ffn_cluster_plan(plan, st, err);
+      // many rows: the cluster of two CTA pairs (256 rows per weight tile); else the cluster kernel where the shape
+      // splits over 2..4 CTAs; else the kernel that tiles the reduction
+      ago_status_t s = ffn_pair_plan(plan, st, err);
+      if (s == AGO_ERR_UNSUPPORTED) s = ffn_cluster_plan(plan, st, err);
       return s == AGO_ERR_UNSUPPORTED ? ffn_plan(plan, st, err) : s;
     }
     case AGO_KERNEL_CONV3X3_PAIR:
@@ -87,6 +89,7 @@ ago_status_t fused_run(const Plan& plan, FusedState* st, const void* const* inpu
     case AGO_KERNEL_ATTENTION:
       return attention_run(plan, st, inputs, weights, output, status_word, stream, err);
     case AGO_KERNEL_FFN:
+      if (st->variant == 3) return ffn_pair_run(plan, st, inputs, weights, output, status_word, stream, err);
       if (st->variant == 1) return ffn_cluster_run(plan, st, inputs, weights, output, workspace, status_word, stream, err);
       return ffn_run(plan, st, inputs, weights, output, workspace, status_word, stream, err);
     case AGO_KERNEL_CONV3X3_PAIR:

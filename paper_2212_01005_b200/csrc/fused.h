@@ -13,7 +13,7 @@ struct FusedState {
   int tile_rows = 0;       // downstream tile extent along the tiled dimension
   int grid = 0;            // CTAs
   int smem_bytes = 0;      // dynamic shared memory per CTA
-  int variant = 0;         // kernel variant within the family (feed-forward chain: 1 = thread-block cluster)
+  int variant = 0;         // kernel variant within the family (feed-forward chain: 1 = thread-block cluster, 3 = cluster of two CTA pairs)
   unsigned workspace_epoch = 0;   // bumped by every ago_subgraph_set_workspace: whatever a kernel family remembers about
                                   // the workspace contents (e.g. "already zeroed") is void after a new attach
   void* impl = nullptr;                  // kernel-family host state (parameters, tensor-map cache)
@@ -35,6 +35,9 @@ ago_status_t attention_plan(Plan* plan, FusedState* st, std::string* err);
 ago_status_t attention_run(const Plan& plan, FusedState* st, const void* const* inputs, const void* const* weights,
                            void* output, unsigned int* status_word, cudaStream_t stream, std::string* err);
 ago_status_t ffn_plan(Plan* plan, FusedState* st, std::string* err);
+ago_status_t ffn_pair_plan(Plan* plan, FusedState* st, std::string* err);
+ago_status_t ffn_pair_run(const Plan& plan, FusedState* st, const void* const* inputs, const void* const* weights,
+                          void* output, unsigned int* status_word, cudaStream_t stream, std::string* err);
 ago_status_t ffn_cluster_plan(Plan* plan, FusedState* st, std::string* err);   // AGO_ERR_UNSUPPORTED: no cluster split for this shape
 ago_status_t ffn_cluster_run(const Plan& plan, FusedState* st, const void* const* inputs, const void* const* weights,
                              void* output, void* workspace, unsigned int* status_word, cudaStream_t stream, std::string* err);
