@@ -70,6 +70,7 @@ ago_status_t fused_plan(Plan* plan, FusedState* st, std::string* err) {
 
 size_t fused_workspace_bytes(const Plan& plan) {
   if (plan.fused_kernel != AGO_KERNEL_FFN) return 0;
+  if (plan.fused_variant == 3) return ffn_pair_workspace_bytes(plan);
   return plan.fused_variant == 0 ? ffn_workspace_bytes(plan) : ffn_cluster_workspace_bytes(plan);
 }
 
@@ -89,7 +90,7 @@ ago_status_t fused_run(const Plan& plan, FusedState* st, const void* const* inpu
     case AGO_KERNEL_ATTENTION:
       return attention_run(plan, st, inputs, weights, output, status_word, stream, err);
     case AGO_KERNEL_FFN:
-      if (st->variant == 3) return ffn_pair_run(plan, st, inputs, weights, output, status_word, stream, err);
+      if (st->variant == 3) return ffn_pair_run(plan, st, inputs, weights, output, workspace, status_word, stream, err);
       if (st->variant == 1) return ffn_cluster_run(plan, st, inputs, weights, output, workspace, status_word, stream, err);
       return ffn_run(plan, st, inputs, weights, output, workspace, status_word, stream, err);
     case AGO_KERNEL_CONV3X3_PAIR:

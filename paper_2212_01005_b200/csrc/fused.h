@@ -37,7 +37,8 @@ ago_status_t attention_run(const Plan& plan, FusedState* st, const void* const* 
 ago_status_t ffn_plan(Plan* plan, FusedState* st, std::string* err);
 ago_status_t ffn_pair_plan(Plan* plan, FusedState* st, std::string* err);
 ago_status_t ffn_pair_run(const Plan& plan, FusedState* st, const void* const* inputs, const void* const* weights,
-                          void* output, unsigned int* status_word, cudaStream_t stream, std::string* err);
+                          void* output, void* workspace, unsigned int* status_word, cudaStream_t stream, std::string* err);
+size_t ffn_pair_workspace_bytes(const Plan& plan);
 ago_status_t ffn_cluster_plan(Plan* plan, FusedState* st, std::string* err);   // AGO_ERR_UNSUPPORTED: no cluster split for this shape
 ago_status_t ffn_cluster_run(const Plan& plan, FusedState* st, const void* const* inputs, const void* const* weights,
                              void* output, void* workspace, unsigned int* status_word, cudaStream_t stream, std::string* err);

@@ -65,6 +65,10 @@ struct FfnPairParams {
   int S;                   // steps per row block = Hid / 256
   int kblocks;             // K / 64
   int units;               // blocks of 256 rows
+  // The blocks of the last, partial round of resident clusters are split: each of the blocks [units_whole, units) is
+  // shared by J clusters, S / J steps each, whose output shares meet in an fp32 buffer in device memory.
+  int units_whole, J;
+  float* acc;              // [(units - units_whole) * 256][N2] fp32, zero before and after a run
 };
 
 __device__ __forceinline__ float gelu_tanh_pair(float v) {
@@ -103,10 +107,26 @@ ffn_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
   const bool leader = h == 0;
   const uint32_t lead_rank = rank & ~1u, mate_rank = rank ^ 1u, twin_rank = rank ^ 2u;   // pair leader, other CTA of the pair, same rows in the other pair
   const int S = p.S;
-  // a cluster walks over the row blocks blockIdx.y, + gridDim.y, ...; its steps form one sequence
-  const int my_units = ((int)blockIdx.y < p.units) ? (p.units - 1 - (int)blockIdx.y) / (int)gridDim.y + 1 : 0;
-  const int steps = my_units * S;
-  auto row0_of = [&](int g) { return ((int)blockIdx.y + (g / S) * (int)gridDim.y) * 2 * kFM + h * kFM; };
+  // Work items: the whole blocks [0, units_whole), then J parts of S / J steps for each of the other blocks. A cluster
+  // walks over the items blockIdx.y, + gridDim.y, ... (whole blocks first); its steps form one sequence.
+  const int G = (int)gridDim.y, cidx = (int)blockIdx.y, Sp = S / p.J;
+  const int n_all = p.units_whole + (p.units - p.units_whole) * p.J;
+  const int n_items = cidx < n_all ? (n_all - 1 - cidx) / G + 1 : 0;
+  const int n_w = cidx < p.units_whole ? (p.units_whole - 1 - cidx) / G + 1 : 0;
+  const int steps = n_w * S + (n_items - n_w) * Sp;
+  struct Step { int item, unit, sb; bool first, last, split; };   // sb: index of the pair of hidden tiles inside the block
+  auto step_of = [&](int g) {
+    Step r;
+    if (g < n_w * S) {
+      r.item = g / S; r.sb = g - r.item * S; r.unit = cidx + r.item * G;
+      r.first = r.sb == 0; r.last = r.sb == S - 1; r.split = false;
+    } else {
+      const int g2 = g - n_w * S, k = g2 / Sp, sp = g2 - k * Sp, q = cidx + (n_w + k) * G - p.units_whole;
+      r.item = n_w + k; r.unit = p.units_whole + q / p.J; r.sb = (q % p.J) * Sp + sp;
+      r.first = sp == 0; r.last = sp == Sp - 1; r.split = true;
+    }
+    return r;
+  };
   // output chunks of the pair's NC columns: one MMA each (N <= 256): 128 | 256 | 256 + 128
   const int cn0 = min(p.NC, 256), cn1 = p.NC - cn0;
   const uint32_t g2_tx = (uint32_t)(p.NC / 2) * kFK * 2u;            // W2 bytes per stage and CTA
@@ -149,7 +169,8 @@ ffn_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
       };
       auto advance = [&]() { if (++s == kFStages) { s = 0; ++round; } };
       auto load_g1 = [&](int g) {       // first GEMM of the pair's hidden tile of step g: this CTA's rows, its half of the tile
-        const int hid0 = (2 * (g % S) + P) * kFH + h * 64, row0 = row0_of(g);
+        const Step st_ = step_of(g);
+        const int hid0 = (2 * st_.sb + P) * kFH + h * 64, row0 = st_.unit * 2 * kFM + h * kFM;
         for (int kb = 0; kb < p.kblocks; ++kb) {
           uint32_t full;
           uint8_t* st = next_stage(g1_tx, &full);
@@ -162,7 +183,7 @@ ffn_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
       for (int g = 0; g < steps; ++g) {
         if (g + 1 < steps) load_g1(g + 1);
         for (int k = 0; k < 2; ++k) {   // second GEMM over the H tile of pair k: two stages of 64 hidden units
-          const int hid0 = (2 * (g % S) + k) * kFH;
+          const int hid0 = (2 * step_of(g).sb + k) * kFH;
           for (int kk = 0; kk < 2; ++kk) {
             uint32_t full;
             uint8_t* st = next_stage(g2_tx, &full);
@@ -215,8 +236,9 @@ ffn_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
       if (steps > 0) g1(0);
       for (int g = 0; g < steps; ++g) {
         if (g + 1 < steps) g1(g + 1);
-        const int sb = g % S, bi = g / S;
-        if (sb == 0 && bi >= 1) {   // the output accumulators of the previous row block have been read in both CTAs
+        const Step cur = step_of(g);
+        const int bi = cur.item;
+        if (cur.first && bi >= 1) {   // the output accumulators of the previous row block have been read in both CTAs
           mbar_wait_poll(bar_outfree, (uint32_t)(bi - 1) & 1u, abort_flag, p.status, 0x805);
           mbar_wait_poll(bar_poutfree, (uint32_t)(bi - 1) & 1u, abort_flag, p.status, 0x806);
           tcgen05_fence_after_sync();
@@ -234,7 +256,7 @@ ffn_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
             const uint64_t bd1 = make_smem_desc(st + (uint32_t)(cn0 / 128) * 8192u, 8192, 1024, SW_128B);
 #pragma unroll
             for (int ks = 0; ks < 4; ++ks) {
-              const uint32_t acc = (uint32_t)((sb | k | kk | ks) != 0);
+              const uint32_t acc = (uint32_t)(!cur.first || (k | kk | ks) != 0);
               umma_bf16_pair_elected(tmem_base + kFOutCol, hd + 2u * ks, bd0 + (uint64_t)((ks * 2048) >> 4), idesc2a, elected, acc);
               if (cn1 > 0) umma_bf16_pair_elected(tmem_base + kFOutCol + (uint32_t)cn0, hd + 2u * ks, bd1 + (uint64_t)((ks * 2048) >> 4), idesc2b, elected, acc);
             }
@@ -246,7 +268,7 @@ ffn_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
           umma_commit_pair_elected(cluster_map(e, (uint32_t)(2 * k)), elected);
           umma_commit_pair_elected(cluster_map(e, (uint32_t)(2 * k + 1)), elected);
         }
-        if (sb == S - 1) commit_pair_bar(bar_out);
+        if (cur.last) commit_pair_bar(bar_out);
       }
     } else if (lane == 0) {
       // ============ relay (the CTA that does not lead): "both slots full", "output drained" -> leader ============
@@ -256,8 +278,9 @@ ffn_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
         mbar_wait(bar_slot, (uint32_t)g & 1u, abort_flag, p.status, 0x80a);
         mbar_wait(bar_slot + 1, (uint32_t)g & 1u, abort_flag, p.status, 0x80b);
         mbar_remote_arrive(lead_pslots);
-        if (g % S == 0 && g >= S) {
-          mbar_wait(bar_outfree, (uint32_t)(g / S - 1) & 1u, abort_flag, p.status, 0x80c);
+        const Step cur = step_of(g);
+        if (cur.first && cur.item >= 1) {
+          mbar_wait(bar_outfree, (uint32_t)(cur.item - 1) & 1u, abort_flag, p.status, 0x80c);
           mbar_remote_arrive(lead_poutfree);
         }
       }
@@ -288,13 +311,32 @@ ffn_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
     const uint32_t twin_bar = cluster_map(smem_u32(bar_slot + P), twin_rank);
     const int hc = p.NC >> 1;                      // output columns per thread: 64, 128 or 192
 
-    auto drain_output = [&](int bi) {
-      // ---- output of row block bi: out (TMEM) -> + b2 -> bf16 -> device memory ----
-      const int row0 = ((int)blockIdx.y + bi * (int)gridDim.y) * 2 * kFM + h * kFM;
+    auto drain_output = [&](int bi, int unit, bool split) {
+      // ---- output of work item bi: out (TMEM) -> + b2 -> bf16 -> device memory; the share of a split block is added
+      // into the fp32 buffer instead (a second, small kernel turns the buffer into the output) ----
+      const int row0 = unit * 2 * kFM + h * kFM;
       const bool row_ok = row0 + row < p.M;
       mbar_wait(bar_out, (uint32_t)bi & 1u, abort_flag, p.status, 0x80f);
       tcgen05_fence_after_sync();
       const int n0 = P * p.NC + half * hc;
+      if (split) {
+        float* arow = p.acc + (size_t)(row0 + row - p.units_whole * 2 * kFM) * p.N2 + n0;
+        for (int c0 = 0; c0 < hc; c0 += 32) {
+          uint32_t v[32];
+          tmem_ld_x32(tmem_base + lane_base + kFOutCol + (uint32_t)(half * hc + c0), v);
+          tmem_ld_wait();
+          if (row_ok) {
+#pragma unroll
+            for (int q = 0; q < 8; ++q)
+              asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(arow + c0 + q * 4), "f"(__uint_as_float(v[4 * q])),
+                           "f"(__uint_as_float(v[4 * q + 1])), "f"(__uint_as_float(v[4 * q + 2])), "f"(__uint_as_float(v[4 * q + 3])) : "memory");
+          }
+        }
+        tcgen05_fence_before_sync();
+        named_barrier_sync(1, kFEpiThreads);
+        if (tid == 0) mbar_arrive(bar_outfree);
+        return;
+      }
       __nv_bfloat16* orow = p.out + (size_t)(row0 + row) * p.N2 + n0;
       const float* b2 = p.b2 + n0;
       for (int c0 = 0; c0 < hc; c0 += 32) {
@@ -319,8 +361,10 @@ ffn_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
       if (tid == 0) mbar_arrive(bar_outfree);
     };
 
+    int prev_item = 0, prev_unit = 0; bool prev_split = false;     // the item whose last step has been seen
     for (int g = 0; g < steps; ++g) {
-      const int sb = g % S;
+      const Step cur = step_of(g);
+      const int sb = cur.sb;
       mbar_wait(bar_hacc, (uint32_t)g & 1u, abort_flag, p.status, 0x810);
       tcgen05_fence_after_sync();
       // the whole share of this thread goes to registers first, so that the accumulator is free for the next first GEMM
@@ -355,9 +399,10 @@ ffn_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
         bulk_copy_to_cluster(twin_slot, smem_u32(slot), kFSlotBytes, twin_bar);   // ... and on its way to the other pair
       }
       // the output of the previous row block is complete once the first GEMM of this block's first step is
-      if (sb == 0 && g >= S) drain_output(g / S - 1);
+      if (cur.first && cur.item >= 1) drain_output(prev_item, prev_unit, prev_split);
+      if (cur.last) { prev_item = cur.item; prev_unit = cur.unit; prev_split = cur.split; }
     }
-    if (steps > 0) drain_output(steps / S - 1);
+    if (steps > 0) drain_output(prev_item, prev_unit, prev_split);
   }
   tcgen05_fence_before_sync();
   __syncthreads();
@@ -365,8 +410,35 @@ ffn_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
   if (warp == kFEpiWarps + 1) tmem_dealloc_pair(tmem_base, 512);
 }
 
+// Second launch of a run with split blocks: out = bf16(acc + b2), acc = 0 over the rows of the split blocks.
+__global__ void __launch_bounds__(256) ffn_pair_finalize_kernel(float* acc, const float* b2, __nv_bfloat16* out, long long total4, int n2) {
+  grid_dependency_wait();      // the additions of the first launch are complete and visible
+  grid_launch_dependents();
+  const long long stride = (long long)gridDim.x * blockDim.x;
+  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total4; i += stride) {
+    const float4 a = __ldcg(reinterpret_cast<const float4*>(acc) + i);
+    const float4 bb = __ldg(reinterpret_cast<const float4*>(b2 + (int)((i * 4) % n2)));
+    reinterpret_cast<float4*>(acc)[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+    reinterpret_cast<uint2*>(out)[i] = make_uint2(pack_bf16x2(a.x + bb.x, a.y + bb.y), pack_bf16x2(a.z + bb.z, a.w + bb.w));
+  }
+}
+
+// How the blocks of 256 rows are dealt to the resident clusters: the whole rounds as they are; the blocks of a last,
+// partial round are split into the largest J (a divisor of the S steps) whose parts still fit one round.
+void pair_split(int units, int S, int* units_whole, int* J) {
+  const int resident = device_sm_count() >= 148 ? 33 : std::max(1, device_sm_count() / 4 - 4);   // clusters of 4 (1 CTA per SM): 33 on a B200
+  *units_whole = units; *J = 1;
+  const int full = units / resident, rest = units % resident;
+  if (full < 1 || rest == 0) return;
+  for (int j = S; j >= 2; --j)
+    if (S % j == 0 && rest * j <= resident) { *units_whole = full * resident; *J = j; return; }
+}
+
 struct FfnPairHost {
   FfnPairParams prm;
+  size_t ws_bytes = 0;
+  const void* clean_ws = nullptr;   // workspace known to be zeroed (kept so by the finalisation kernel) ...
+  unsigned clean_epoch = 0;         // ... as of this attach (FusedState::workspace_epoch)
   int clusters = 0;   // clusters launched = min(row blocks, clusters the device keeps resident); 0: not asked yet
   struct Key { const void* p; int which; bool operator==(const Key& o) const { return p == o.p && which == o.which; } };
   struct KeyHash { size_t operator()(const Key& k) const { return std::hash<const void*>()(k.p) ^ (size_t)k.which * 0x9e3779b97f4a7c15ull; } };
@@ -391,6 +463,16 @@ void fill_pair_launch(cudaLaunchConfig_t* cfg, cudaLaunchAttribute* attr, int cl
 
 // AGO_ERR_UNSUPPORTED (without touching *err) when the shape does not split over two pairs: the caller falls back
 // to the unpaired cluster kernel or to the kernel that tiles the second GEMM's reduction.
+size_t ffn_pair_workspace_bytes(const Plan& plan) {
+  const int64_t K = plan.inputs[0].last(), M = plan.inputs[0].numel() / K;
+  const int64_t N2 = plan.output.last();
+  const int units = (int)((M + 2 * kFM - 1) / (2 * kFM)), S = plan.ops[0].op.p[0] / (2 * kFH);
+  int whole = units, J = 1;
+  pair_split(units, S, &whole, &J);
+  if (J == 1) return 0;
+  return ((size_t)(units - whole) * 2 * kFM * N2 * 4 + 255) & ~size_t(255);   // whole blocks of 256 rows: the last may be ragged
+}
+
 ago_status_t ffn_pair_plan(Plan* plan, FusedState* st, std::string* err) {
   (void)err;
   FfnPairParams q{};
@@ -409,15 +491,24 @@ ago_status_t ffn_pair_plan(Plan* plan, FusedState* st, std::string* err) {
   host->prm = q;
   st->impl = host;
   st->impl_free = [](void* p) { delete static_cast<FfnPairHost*>(p); };
+  pair_split(q.units, q.S, &q.units_whole, &q.J);
+  host->prm = q;
   st->variant = 3;
   plan->fused_variant = 3;
+  if (q.J > 1) {
+    const int64_t rows = std::min<int64_t>((int64_t)(q.units - q.units_whole) * 2 * kFM, (int64_t)q.M - (int64_t)q.units_whole * 2 * kFM);
+    host->ws_bytes = ffn_pair_workspace_bytes(*plan);
+    // every part adds its share into the buffer; the second launch reads it back and zeroes it
+    plan->workspace_traffic_bytes = (int64_t)(q.J + 2) * rows * q.N2 * 4;
+    plan->num_launches = 2;
+  }
   st->tile_rows = 2 * kFM; st->grid = 4 * q.units; st->smem_bytes = kFSmemBytes;
   plan->tile_rows = 2 * kFM; plan->smem_bytes = kFSmemBytes;
   return AGO_OK;
 }
 
 ago_status_t ffn_pair_run(const Plan& plan, FusedState* st, const void* const* inputs, const void* const* weights,
-                          void* output, unsigned int* status_word, cudaStream_t stream, std::string* err) {
+                          void* output, void* workspace, unsigned int* status_word, cudaStream_t stream, std::string* err) {
   (void)plan;
   FfnPairHost* host = static_cast<FfnPairHost*>(st->impl);
   FfnPairParams q = host->prm;
@@ -425,6 +516,19 @@ ago_status_t ffn_pair_run(const Plan& plan, FusedState* st, const void* const* i
   q.b2 = static_cast<const float*>(weights[3]);
   q.out = static_cast<__nv_bfloat16*>(output);
   q.status = status_word;
+  q.acc = nullptr;
+  if (q.J > 1) {
+    if (!workspace) { *err = "fused feed-forward (paired cluster, split last round): no workspace attached"; return AGO_ERR_INVALID_ARG; }
+    q.acc = static_cast<float*>(workspace);
+    if (host->clean_ws != workspace || host->clean_epoch != st->workspace_epoch) {
+      // a workspace is zeroed at the first run after each attach; after that every run leaves it zeroed (the caller
+      // must not touch it in between)
+      cudaError_t e = cudaMemsetAsync(workspace, 0, host->ws_bytes, stream);
+      if (e != cudaSuccess) { *err = std::string("cudaMemsetAsync(workspace): ") + cudaGetErrorString(e); return AGO_ERR_CUDA; }
+      host->clean_ws = workspace;
+      host->clean_epoch = st->workspace_epoch;
+    }
+  }
   auto get_map = [&](const void* base, int which, CUtensorMap* out) -> bool {
     FfnPairHost::Key key{base, which};
     auto it = host->maps.find(key);
@@ -462,6 +566,14 @@ ago_status_t ffn_pair_run(const Plan& plan, FusedState* st, const void* const* i
   fill_pair_launch(&cfg, attr, host->clusters, stream);
   cudaError_t e = cudaLaunchKernelEx(&cfg, ffn_pair_kernel, mx, mw1, mw2, q);
   if (e != cudaSuccess) { *err = std::string("fused feed-forward (paired cluster) launch: ") + cudaGetErrorString(e); return AGO_ERR_CUDA; }
+  if (q.J > 1) {
+    const long long row_first = (long long)q.units_whole * 2 * kFM;
+    const long long total4 = ((long long)q.M - row_first) * q.N2 / 4;
+    const int blocks = (int)std::min<long long>((total4 + 255) / 256, 4LL * device_sm_count());
+    FusedLaunch fin(dim3((unsigned)blocks), 256, 0, stream);
+    e = cudaLaunchKernelEx(&fin.config, ffn_pair_finalize_kernel, q.acc, q.b2, q.out + row_first * q.N2, total4, q.N2);
+    if (e != cudaSuccess) { *err = std::string("fused feed-forward (paired cluster) finalisation launch: ") + cudaGetErrorString(e); return AGO_ERR_CUDA; }
+  }
   return AGO_OK;
 }
 
