@@ -66,9 +66,11 @@ struct FfnPairParams {
   int kblocks;             // K / 64
   int units;               // blocks of 256 rows
   // The blocks of the last, partial round of resident clusters are split: each of the blocks [units_whole, units) is
-  // shared by J clusters, S / J steps each, whose output shares meet in an fp32 buffer in device memory.
+  // shared by J clusters, S / J steps each; part j stores its output share as fp32 in plane j of a buffer in device
+  // memory (plain stores: no atomics, nothing to zero, the same bits on every run) and a second launch adds the planes.
   int units_whole, J;
-  float* acc;              // [(units - units_whole) * 256][N2] fp32, zero before and after a run
+  float* acc;              // [J][split_rows][N2] fp32
+  int split_rows;          // rows of the split blocks that exist: M - units_whole * 256
 };
 
 __device__ __forceinline__ float gelu_tanh_pair(float v) {
@@ -114,15 +116,15 @@ ffn_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
   const int n_items = cidx < n_all ? (n_all - 1 - cidx) / G + 1 : 0;
   const int n_w = cidx < p.units_whole ? (p.units_whole - 1 - cidx) / G + 1 : 0;
   const int steps = n_w * S + (n_items - n_w) * Sp;
-  struct Step { int item, unit, sb; bool first, last, split; };   // sb: index of the pair of hidden tiles inside the block
+  struct Step { int item, unit, sb, part; bool first, last, split; };   // sb: index of the pair of hidden tiles inside the block
   auto step_of = [&](int g) {
     Step r;
     if (g < n_w * S) {
       r.item = g / S; r.sb = g - r.item * S; r.unit = cidx + r.item * G;
-      r.first = r.sb == 0; r.last = r.sb == S - 1; r.split = false;
+      r.first = r.sb == 0; r.last = r.sb == S - 1; r.split = false; r.part = 0;
     } else {
       const int g2 = g - n_w * S, k = g2 / Sp, sp = g2 - k * Sp, q = cidx + (n_w + k) * G - p.units_whole;
-      r.item = n_w + k; r.unit = p.units_whole + q / p.J; r.sb = (q % p.J) * Sp + sp;
+      r.item = n_w + k; r.unit = p.units_whole + q / p.J; r.part = q % p.J; r.sb = r.part * Sp + sp;
       r.first = sp == 0; r.last = sp == Sp - 1; r.split = true;
     }
     return r;
@@ -311,16 +313,16 @@ ffn_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
     const uint32_t twin_bar = cluster_map(smem_u32(bar_slot + P), twin_rank);
     const int hc = p.NC >> 1;                      // output columns per thread: 64, 128 or 192
 
-    auto drain_output = [&](int bi, int unit, bool split) {
-      // ---- output of work item bi: out (TMEM) -> + b2 -> bf16 -> device memory; the share of a split block is added
-      // into the fp32 buffer instead (a second, small kernel turns the buffer into the output) ----
+    auto drain_output = [&](int bi, int unit, bool split, int part) {
+      // ---- output of work item bi: out (TMEM) -> + b2 -> bf16 -> device memory; the share of a part of a split block goes
+      // to its plane of the fp32 buffer instead (a second, small kernel adds the planes and writes the output) ----
       const int row0 = unit * 2 * kFM + h * kFM;
       const bool row_ok = row0 + row < p.M;
       mbar_wait(bar_out, (uint32_t)bi & 1u, abort_flag, p.status, 0x80f);
       tcgen05_fence_after_sync();
       const int n0 = P * p.NC + half * hc;
       if (split) {
-        float* arow = p.acc + (size_t)(row0 + row - p.units_whole * 2 * kFM) * p.N2 + n0;
+        float* arow = p.acc + ((size_t)part * p.split_rows + (size_t)(row0 + row - p.units_whole * 2 * kFM)) * p.N2 + n0;
         for (int c0 = 0; c0 < hc; c0 += 32) {
           uint32_t v[32];
           tmem_ld_x32(tmem_base + lane_base + kFOutCol + (uint32_t)(half * hc + c0), v);
@@ -328,8 +330,7 @@ ffn_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
           if (row_ok) {
 #pragma unroll
             for (int q = 0; q < 8; ++q)
-              asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(arow + c0 + q * 4), "f"(__uint_as_float(v[4 * q])),
-                           "f"(__uint_as_float(v[4 * q + 1])), "f"(__uint_as_float(v[4 * q + 2])), "f"(__uint_as_float(v[4 * q + 3])) : "memory");
+              *reinterpret_cast<uint4*>(arow + c0 + q * 4) = make_uint4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
           }
         }
         tcgen05_fence_before_sync();
@@ -361,7 +362,7 @@ ffn_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
       if (tid == 0) mbar_arrive(bar_outfree);
     };
 
-    int prev_item = 0, prev_unit = 0; bool prev_split = false;     // the item whose last step has been seen
+    int prev_item = 0, prev_unit = 0, prev_part = 0; bool prev_split = false;     // the item whose last step has been seen
     for (int g = 0; g < steps; ++g) {
       const Step cur = step_of(g);
       const int sb = cur.sb;
@@ -399,10 +400,10 @@ ffn_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
         bulk_copy_to_cluster(twin_slot, smem_u32(slot), kFSlotBytes, twin_bar);   // ... and on its way to the other pair
       }
       // the output of the previous row block is complete once the first GEMM of this block's first step is
-      if (cur.first && cur.item >= 1) drain_output(prev_item, prev_unit, prev_split);
-      if (cur.last) { prev_item = cur.item; prev_unit = cur.unit; prev_split = cur.split; }
+      if (cur.first && cur.item >= 1) drain_output(prev_item, prev_unit, prev_split, prev_part);
+      if (cur.last) { prev_item = cur.item; prev_unit = cur.unit; prev_split = cur.split; prev_part = cur.part; }
     }
-    if (steps > 0) drain_output(prev_item, prev_unit, prev_split);
+    if (steps > 0) drain_output(prev_item, prev_unit, prev_split, prev_part);
   }
   tcgen05_fence_before_sync();
   __syncthreads();
@@ -410,16 +411,18 @@ ffn_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
   if (warp == kFEpiWarps + 1) tmem_dealloc_pair(tmem_base, 512);
 }
 
-// Second launch of a run with split blocks: out = bf16(acc + b2), acc = 0 over the rows of the split blocks.
-__global__ void __launch_bounds__(256) ffn_pair_finalize_kernel(float* acc, const float* b2, __nv_bfloat16* out, long long total4, int n2) {
-  grid_dependency_wait();      // the additions of the first launch are complete and visible
+// Second launch of a run with split blocks: out = bf16(sum of the J planes + b2) over the rows of the split blocks.
+__global__ void __launch_bounds__(256) ffn_pair_finalize_kernel(const float* acc, const float* b2, __nv_bfloat16* out, long long total4, int n2, int J) {
+  grid_dependency_wait();      // the stores of the first launch are complete and visible
   grid_launch_dependents();
   const long long stride = (long long)gridDim.x * blockDim.x;
   for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total4; i += stride) {
-    const float4 a = __ldcg(reinterpret_cast<const float4*>(acc) + i);
-    const float4 bb = __ldg(reinterpret_cast<const float4*>(b2 + (int)((i * 4) % n2)));
-    reinterpret_cast<float4*>(acc)[i] = make_float4(0.f, 0.f, 0.f, 0.f);
-    reinterpret_cast<uint2*>(out)[i] = make_uint2(pack_bf16x2(a.x + bb.x, a.y + bb.y), pack_bf16x2(a.z + bb.z, a.w + bb.w));
+    float4 a = __ldg(reinterpret_cast<const float4*>(b2 + (int)((i * 4) % n2)));
+    for (int j = 0; j < J; ++j) {
+      const float4 v = __ldcg(reinterpret_cast<const float4*>(acc) + (long long)j * total4 + i);
+      a.x += v.x; a.y += v.y; a.z += v.z; a.w += v.w;
+    }
+    reinterpret_cast<uint2*>(out)[i] = make_uint2(pack_bf16x2(a.x, a.y), pack_bf16x2(a.z, a.w));
   }
 }
 
@@ -437,8 +440,6 @@ void pair_split(int units, int S, int* units_whole, int* J) {
 struct FfnPairHost {
   FfnPairParams prm;
   size_t ws_bytes = 0;
-  const void* clean_ws = nullptr;   // workspace known to be zeroed (kept so by the finalisation kernel) ...
-  unsigned clean_epoch = 0;         // ... as of this attach (FusedState::workspace_epoch)
   int clusters = 0;   // clusters launched = min(row blocks, clusters the device keeps resident); 0: not asked yet
   struct Key { const void* p; int which; bool operator==(const Key& o) const { return p == o.p && which == o.which; } };
   struct KeyHash { size_t operator()(const Key& k) const { return std::hash<const void*>()(k.p) ^ (size_t)k.which * 0x9e3779b97f4a7c15ull; } };
@@ -470,7 +471,7 @@ size_t ffn_pair_workspace_bytes(const Plan& plan) {
   int whole = units, J = 1;
   pair_split(units, S, &whole, &J);
   if (J == 1) return 0;
-  return ((size_t)(units - whole) * 2 * kFM * N2 * 4 + 255) & ~size_t(255);   // whole blocks of 256 rows: the last may be ragged
+  return ((size_t)J * (size_t)(M - (int64_t)whole * 2 * kFM) * N2 * 4 + 255) & ~size_t(255);   // J planes over the rows of the split blocks
 }
 
 ago_status_t ffn_pair_plan(Plan* plan, FusedState* st, std::string* err) {
@@ -492,14 +493,15 @@ ago_status_t ffn_pair_plan(Plan* plan, FusedState* st, std::string* err) {
   st->impl = host;
   st->impl_free = [](void* p) { delete static_cast<FfnPairHost*>(p); };
   pair_split(q.units, q.S, &q.units_whole, &q.J);
+  q.split_rows = q.M - q.units_whole * 2 * kFM;
   host->prm = q;
   st->variant = 3;
   plan->fused_variant = 3;
   if (q.J > 1) {
     const int64_t rows = std::min<int64_t>((int64_t)(q.units - q.units_whole) * 2 * kFM, (int64_t)q.M - (int64_t)q.units_whole * 2 * kFM);
     host->ws_bytes = ffn_pair_workspace_bytes(*plan);
-    // every part adds its share into the buffer; the second launch reads it back and zeroes it
-    plan->workspace_traffic_bytes = (int64_t)(q.J + 2) * rows * q.N2 * 4;
+    // every part writes its plane, the second launch reads the planes back
+    plan->workspace_traffic_bytes = (int64_t)(2 * q.J) * rows * q.N2 * 4;
     plan->num_launches = 2;
   }
   st->tile_rows = 2 * kFM; st->grid = 4 * q.units; st->smem_bytes = kFSmemBytes;
@@ -519,15 +521,7 @@ ago_status_t ffn_pair_run(const Plan& plan, FusedState* st, const void* const* i
   q.acc = nullptr;
   if (q.J > 1) {
     if (!workspace) { *err = "fused feed-forward (paired cluster, split last round): no workspace attached"; return AGO_ERR_INVALID_ARG; }
-    q.acc = static_cast<float*>(workspace);
-    if (host->clean_ws != workspace || host->clean_epoch != st->workspace_epoch) {
-      // a workspace is zeroed at the first run after each attach; after that every run leaves it zeroed (the caller
-      // must not touch it in between)
-      cudaError_t e = cudaMemsetAsync(workspace, 0, host->ws_bytes, stream);
-      if (e != cudaSuccess) { *err = std::string("cudaMemsetAsync(workspace): ") + cudaGetErrorString(e); return AGO_ERR_CUDA; }
-      host->clean_ws = workspace;
-      host->clean_epoch = st->workspace_epoch;
-    }
+    q.acc = static_cast<float*>(workspace);   // every element of it is written before it is read: nothing to zero
   }
   auto get_map = [&](const void* base, int which, CUtensorMap* out) -> bool {
     FfnPairHost::Key key{base, which};
@@ -571,7 +565,7 @@ ago_status_t ffn_pair_run(const Plan& plan, FusedState* st, const void* const* i
     const long long total4 = ((long long)q.M - row_first) * q.N2 / 4;
     const int blocks = (int)std::min<long long>((total4 + 255) / 256, 4LL * device_sm_count());
     FusedLaunch fin(dim3((unsigned)blocks), 256, 0, stream);
-    e = cudaLaunchKernelEx(&fin.config, ffn_pair_finalize_kernel, q.acc, q.b2, q.out + row_first * q.N2, total4, q.N2);
+    e = cudaLaunchKernelEx(&fin.config, ffn_pair_finalize_kernel, (const float*)q.acc, q.b2, q.out + row_first * q.N2, total4, q.N2, q.J);
     if (e != cudaSuccess) { *err = std::string("fused feed-forward (paired cluster) finalisation launch: ") + cudaGetErrorString(e); return AGO_ERR_CUDA; }
   }
   return AGO_OK;

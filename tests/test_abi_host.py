@@ -26,7 +26,7 @@ def test_workspace_traffic_query_names_the_split_reduction_only():
     # config 4b: 48 blocks of 256 rows on 33 resident clusters; the 15 blocks of the second round are split in two
     wl = WL.get("ffn_12288")
     sg = B.Subgraph(wl.ops, wl.input_shapes, mode="fused")
-    assert sg.query(B.AGO_Q_WORKSPACE_TRAFFIC) == (2 + 2) * (15 * 256) * n2 * 4
+    assert sg.query(B.AGO_Q_WORKSPACE_TRAFFIC) == (2 + 2) * (15 * 256) * n2 * 4    # two planes written, two read back
     assert sg.query(B.AGO_Q_NUM_LAUNCHES) == 2
     sg.close()
     for name, mode in (("ffn_512", "per_mini_subgraph"), ("ffn_12288", "per_mini_subgraph"), ("mbv2_56", "fused"), ("attn_384", "fused")):
@@ -142,7 +142,7 @@ def test_fused_planner_matches_every_chain_family_and_its_limits():
 def test_feed_forward_planner_picks_the_cluster_kernel_where_the_shape_splits():
     # cluster kernels on many row blocks: no workspace (nothing is reduced through device memory) as long as the blocks
     # fill whole rounds of resident clusters; the blocks of a last, partial round are split over two or more clusters that
-    # meet in an fp32 buffer; few row blocks (their hidden tiles split over several clusters) and the kernel without
+    # write an fp32 plane each; few row blocks (their hidden tiles split over several clusters) and the kernel without
     # clusters: an fp32 buffer over all rows
     def ws(M, K, hid, out):
         wl = WL.ffn("x", [1], M, K, hid, 1, d_out=out)
@@ -151,7 +151,7 @@ def test_feed_forward_planner_picks_the_cluster_kernel_where_the_shape_splits():
         sg.close()
         return w
     assert ws(33 * 256, 768, 3072, 768) == 0       # paired clusters: 33 blocks of 256 rows = one whole round of 33 resident clusters
-    assert ws(12288, 768, 3072, 768) == 15 * 256 * 768 * 4   # 48 blocks: one whole round, the other 15 blocks split in two
+    assert ws(12288, 768, 3072, 768) == 2 * 15 * 256 * 768 * 4   # 48 blocks: one whole round, the other 15 split in two parts, an fp32 plane each
     assert ws(9637, 64, 256, 384) == 0             # clusters of 2, ragged last row block
     assert ws(512, 768, 3072, 768) >= 512 * 768 * 4    # four row blocks: six clusters each
     assert ws(12800, 256, 384, 256) >= 12800 * 256 * 4  # three hidden tiles, 256 columns: no cluster size divides both
