@@ -152,6 +152,8 @@ def test_feed_forward_planner_picks_the_cluster_kernel_where_the_shape_splits():
         return w
     assert ws(33 * 256, 768, 3072, 768) == 0       # paired clusters: 33 blocks of 256 rows = one whole round of 33 resident clusters
     assert ws(12288, 768, 3072, 768) == 2 * 15 * 256 * 768 * 4   # 48 blocks: one whole round, the other 15 split in two parts, an fp32 plane each
+    assert ws(40 * 256 - 100, 64, 512, 256) == 2 * (40 * 256 - 100 - 33 * 256) * 256 * 4   # 7 blocks (the last ragged) in two parts
+    assert ws(36 * 256, 128, 768, 512) == 3 * (3 * 256) * 512 * 4     # 3 blocks in three parts of one step
     assert ws(9637, 64, 256, 384) == 0             # clusters of 2, ragged last row block
     assert ws(512, 768, 3072, 768) >= 512 * 768 * 4    # four row blocks: six clusters each
     assert ws(12800, 256, 384, 256) >= 12800 * 256 * 4  # three hidden tiles, 256 columns: no cluster size divides both

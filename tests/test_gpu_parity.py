@@ -40,6 +40,10 @@ def small_workloads():
         # few row blocks: the hidden tiles of a row block are split over several clusters (ragged rows; clusters of 2 / 4)
         "ffn_s3": WL.ffn("ffn_s3", [41], 700, 128, 1536, 1, d_out=384),
         "ffn_s4": WL.ffn("ffn_s4", [42], 1024, 256, 1024, 1, d_out=512),
+        # many rows on the paired-cluster kernel with a last, partial round of resident clusters (33 on a B200): 40 blocks of 256
+        # rows, the last ragged, 7 of them split in two parts of one step; 36 blocks, 3 of them split in three parts
+        "ffn_r2": WL.ffn("ffn_r2", [46], 40 * 256 - 100, 64, 512, 1, d_out=256),
+        "ffn_r3": WL.ffn("ffn_r3", [47], 36 * 256, 128, 768, 1, d_out=512),
         "resnet_small": WL.resnet_block("resnet_small", [26], 2, 12, 64),
         "resnet_odd": WL.resnet_block("resnet_odd", [27], 1, 9, 32),
         "resnet_16ch": WL.resnet_block("resnet_16ch", [32], 2, 20, 16),
@@ -163,7 +167,7 @@ def test_padding_of_the_intermediate_with_large_bias(ago):
 # ---- fused kernels -------------------------------------------------------------------
 
 FUSED_SMALL = ["mbv2_14", "mbv2_s1_odd", "mbv2_s2", "mbv2_s2_odd", "attn_small", "attn_ragged", "attn_runs2", "attn_runs4", "ffn_small", "ffn_rows_ragged", "ffn_g2", "ffn_g3",
-               "ffn_c2", "ffn_c3", "ffn_c4", "ffn_p1", "ffn_p2", "ffn_p3", "ffn_s3", "ffn_s4", "resnet_small", "resnet_odd", "resnet_16ch", "resnet_w28", "resnet_w29", "resnet_w57"]
+               "ffn_c2", "ffn_c3", "ffn_c4", "ffn_p1", "ffn_p2", "ffn_p3", "ffn_s3", "ffn_s4", "ffn_r2", "ffn_r3", "resnet_small", "resnet_odd", "resnet_16ch", "resnet_w28", "resnet_w29", "resnet_w57"]
 
 
 @pytest.mark.parametrize("name", FUSED_SMALL)
