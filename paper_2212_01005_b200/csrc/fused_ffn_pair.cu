@@ -18,13 +18,17 @@
 // Per CTA (pair P, half h; h == 0 leads its pair), steps g = (row block, own hidden tile):
 //   TMA     one thread: 24 KB stages -- X [128 x 64] + W1 [64 x 64] (this CTA's half of the tile) for the first
 //           GEMM, W2 [64 x N2 / 4] for the second. Both CTAs' loads complete on the leader's barrier.
-//   MMA     one thread of the leader: G1(g + 1) into the H accumulator, then G2 over the two H tiles of step g
+//   MMA     one warp of the leader, converged, an elected lane issuing: G1(g + 1) into the H accumulator, then G2 over
+//           the two H tiles of step g
 //   epi     8 warps: H accumulator -> registers (accumulator handed back at once) -> + b1, GELU, bf16 -> own slot
 //           -> local "slot full" + bulk copy to the other pair; at the end of a row block: out -> + b2 -> bf16 -> Y
 //   helper  one thread: arms the barrier the other pair's copy completes on; in the non-leading CTA it also relays
 //           "accumulator drained" to the leader, and a thread of the idle MMA warp relays "slots full" and
 //           "output drained". (An arrival on another CTA's barrier is a release at cluster scope and costs about a
 //           thousand cycles: it is kept off the threads that feed the tensor pipe.)
+// Rounds: the clusters the device keeps resident (33 of four CTAs on a B200) walk over the blocks of 256 rows. The blocks of
+// a last, partial round are split into J parts of S / J steps on J clusters; part j stores its fp32 output share in plane j
+// of the workspace (plain stores) and a second, elementwise launch adds the planes, + b2, -> bf16.
 // Every wait is bounded; a CTA leaves only after a cluster barrier.
 #include <cuda.h>
 #include <cuda_bf16.h>
