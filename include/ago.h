@@ -135,8 +135,8 @@ typedef enum {
   AGO_Q_TILE_ROWS = 14,        /* fused kernel: downstream tile extent along the tiled dimension   */
   AGO_Q_SMEM_BYTES = 15,       /* fused kernel: dynamic shared memory per CTA                      */
   AGO_Q_MODE = 16,             /* the mode the handle runs in (what AGO_MODE_AUTO resolved to)     */
-  AGO_Q_WORKSPACE_TRAFFIC = 17 /* fused kernel: bytes per run added into / read back from its       */
-                               /* device-memory workspace (partial sums of a split reduction); not  */
+  AGO_Q_WORKSPACE_TRAFFIC = 17 /* fused kernel: bytes per run stored or added into / read back from */
+                               /* its device-memory workspace (partial sums of a split reduction); not */
                                /* part of AGO_Q_IO_BYTES; 0 when all intermediates stay on chip     */
 } ago_query_t;
 #define AGO_Q_INDEXED(what, i) ((int32_t)(what) | ((int32_t)(i) << 16))
