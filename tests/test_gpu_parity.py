@@ -154,6 +154,20 @@ def test_single_conv3x3_stage_epilogues(ago, shape, tail):
         assert_close(run_gpu(ago, wl, data, mode), ref, what=f"conv1 {shape} {tail}/{mode}")
 
 
+@pytest.mark.parametrize("shape", [(1, 1, 1, 16), (1, 2, 3, 32), (2, 5, 31, 64), (1, 33, 30, 16), (3, 17, 59, 32), (1, 40, 85, 16), (2, 3, 113, 16)])
+def test_conv3x3_pair_odd_shapes_every_mode(ago, shape):
+    # the residual block on non-square images from a single pixel to four and five 28-column segments, heights that are
+    # not multiples of the four-row tiles, every channel count the tensor-core kernels take; fused and both unfused modes
+    n, h, w, ch = shape
+    ops = [("conv2d", dict(O=ch, R=3, S=3, stride=1, pad=1, groups=1)), ("bias_add", {}), ("relu", {}),
+           ("conv2d", dict(O=ch, R=3, S=3, stride=1, pad=1, groups=1)), ("bias_add", {}), ("add_input", dict(input=0)), ("relu", {})]
+    wl = WL.Workload("conv_pair_odd", [72, h, w, ch], [shape], ops, samples=n, input_dist=["relu_normal"])
+    data = WL.generate(wl)
+    ref = O.run_chain(wl.ops, data["inputs"], data["weights"])
+    for mode in ("fused",) + tuple(UNFUSED):
+        assert_close(run_gpu(ago, wl, data, mode), ref, what=f"conv pair {shape}/{mode}")
+
+
 def test_padding_of_the_intermediate_with_large_bias(ago):
     # the halo of the depthwise / second conv input is zero, not act(bias)
     wl = WL.mbv2_block("pad", [33], 1, 6, 8, 16, 8, 1, True)
