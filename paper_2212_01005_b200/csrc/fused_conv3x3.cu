@@ -485,6 +485,7 @@ ago_status_t conv3x3_plan(Plan* plan, FusedState* st, std::string* err) {
 
 ago_status_t conv3x3_run(const Plan& plan, FusedState* st, const void* const* inputs, const void* const* weights,
                          void* output, unsigned int* status_word, cudaStream_t stream, std::string* err) {
+  (void)plan;
   ConvHost* host = static_cast<ConvHost*>(st->impl);
   ConvParams q = host->prm;
   q.x = static_cast<const __nv_bfloat16*>(inputs[0]);
